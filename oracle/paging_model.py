@@ -1,0 +1,188 @@
+"""Integer-only model of the paged store's bookkeeping.
+
+TEST INFRASTRUCTURE ONLY (see oracle/__init__.py).  The paper has no paging:
+its cache is a Python list (Algorithm 1).  The paged store, its per-sequence
+page table and its device free list come from the build's target statement, so
+this model follows the allocation discipline the library documents in
+include/breadcrumbs.h, written here independently with plain Python lists:
+
+* Free pages form a LIFO stack; ``stack[-1]`` is handed out first.  A fresh
+  store hands out pages 0, 1, 2, ... in that order.
+* One batch call first allocates, then frees.
+  Allocation: walk the batch in order; item i with need[i] pages receives the
+  pages at stack depth off[i] .. off[i]+need[i]-1, off = exclusive prefix sum
+  of the needs of ALL items that passed validation; an item is granted iff
+  need[i] == 0 or off[i] + need[i] <= pages free at the start of the call.
+  Frees: walk the batch in order; a sequence's pages are pushed in the order
+  prompt pages, beacon pages, window pages, each in ascending index.
+* A failed item is a no-op for its sequence; the first failure of the store's
+  lifetime is latched as (code, slot, call index).
+
+Pinned by tests/test_oracle_pins.py: conservation (owned + free = all pages,
+no page twice), per-segment page counts = ceil(len / page_size), lengths equal
+to the closed form, exhaustion on tiny pools worked out by hand.
+"""
+from __future__ import annotations
+
+OK = "OK"
+BAD_SLOT = "BAD_SLOT"
+NO_PAGES = "NO_PAGES"
+CAPACITY = "CAPACITY"
+WINDOW_NOT_FULL = "WINDOW_NOT_FULL"
+WINDOW_FULL = "WINDOW_FULL"
+INVALID_ARG = "INVALID_ARG"
+
+
+def _ceil_div(a, b):
+    return -(-a // b)
+
+
+class _Seq:
+    def __init__(self, P, c):
+        self.P, self.c = P, c
+        self.n_beacons = 0
+        self.window_len = 0
+        self.t = 0
+        self.prompt_pages = []
+        self.beacon_pages = []
+        self.window_pages = []
+
+
+class PagingModel:
+    def __init__(self, num_pages, page_size, max_seqs, max_pages_per_seq,
+                 max_entries_per_seq=0, c_default=1):
+        self.ps = page_size
+        self.num_pages = num_pages
+        self.max_seqs = max_seqs
+        self.max_pages_per_seq = max_pages_per_seq
+        self.max_entries = max_entries_per_seq
+        self.c_default = c_default
+        self.stack = list(range(num_pages - 1, -1, -1))   # stack[-1] == page 0
+        self.seqs = {}
+        self.first_error = None       # (code, slot, call_index)
+        self.calls = 0
+
+    # ------------------------------------------------------------------ utils
+    def _fail(self, code, slot):
+        if self.first_error is None:
+            self.first_error = (code, slot, self.calls)
+        return code
+
+    def _allocate(self, needs):
+        """needs: list of (item index, pages needed) for validated items, in
+        batch order.  Returns {item index: [pages]} for granted items."""
+        free_at_start = len(self.stack)
+        granted, off, used = {}, 0, 0
+        for i, need in needs:
+            if need == 0:
+                granted[i] = []
+            elif off + need <= free_at_start:
+                granted[i] = [self.stack[free_at_start - 1 - off - k] for k in range(need)]
+                used = off + need
+            off += need
+        # granted items form a prefix of the requesters, so `used` pages leave the top
+        if used:
+            del self.stack[free_at_start - used:]
+        return granted
+
+    # ------------------------------------------------------------------- calls
+    def open(self, slots, prompt_lens, cs=None):
+        self.calls += 1
+        res, needs, plan = [None] * len(slots), [], {}
+        for i, slot in enumerate(slots):
+            c = self.c_default if cs is None else cs[i]
+            P = prompt_lens[i]
+            if not (0 <= slot < self.max_seqs) or slot in self.seqs:
+                res[i] = self._fail(BAD_SLOT, slot); continue
+            if c < 1 or P < 0:
+                res[i] = self._fail(INVALID_ARG, slot); continue
+            npp = _ceil_div(P, self.ps)
+            nwp = _ceil_div(c, self.ps) if c > 1 else 0
+            if npp + nwp > self.max_pages_per_seq:
+                res[i] = self._fail(CAPACITY, slot); continue
+            needs.append((i, npp)); plan[i] = (slot, P, c)
+        granted = self._allocate(needs)
+        for i, _ in needs:
+            slot, P, c = plan[i]
+            if i not in granted:
+                res[i] = self._fail(NO_PAGES, slot); continue
+            s = _Seq(P, c); s.prompt_pages = granted[i]
+            self.seqs[slot] = s; res[i] = OK
+        return res
+
+    def append(self, slots):
+        self.calls += 1
+        res, needs = [None] * len(slots), []
+        for i, slot in enumerate(slots):
+            s = self.seqs.get(slot)
+            if s is None:
+                res[i] = self._fail(BAD_SLOT, slot); continue
+            if s.c > 1 and s.window_len >= s.c:
+                res[i] = self._fail(WINDOW_FULL, slot); continue
+            if self.max_entries and s.n_beacons + s.window_len + 1 > self.max_entries:
+                res[i] = self._fail(CAPACITY, slot); continue
+            need = 1 if s.window_len % self.ps == 0 else 0
+            if need and (len(s.prompt_pages) + len(s.beacon_pages) + len(s.window_pages) + 1
+                         > self.max_pages_per_seq):
+                res[i] = self._fail(CAPACITY, slot); continue
+            needs.append((i, need))
+        granted = self._allocate(needs)
+        for i, _ in needs:
+            slot = slots[i]; s = self.seqs[slot]
+            if i not in granted:
+                res[i] = self._fail(NO_PAGES, slot); continue
+            s.window_pages += granted[i]
+            s.window_len += 1; s.t += 1; res[i] = OK
+        return res
+
+    def compress(self, slots):
+        self.calls += 1
+        res, needs = [None] * len(slots), []
+        for i, slot in enumerate(slots):
+            s = self.seqs.get(slot)
+            if s is None:
+                res[i] = self._fail(BAD_SLOT, slot); continue
+            if s.c <= 1 or s.window_len != s.c:
+                res[i] = self._fail(WINDOW_NOT_FULL, slot); continue
+            need = 1 if s.n_beacons % self.ps == 0 else 0
+            if need and (len(s.prompt_pages) + len(s.beacon_pages) + _ceil_div(s.c, self.ps) + 1
+                         > self.max_pages_per_seq):
+                res[i] = self._fail(CAPACITY, slot); continue
+            needs.append((i, need))
+        granted = self._allocate(needs)
+        ok_items = []
+        for i, _ in needs:
+            slot = slots[i]; s = self.seqs[slot]
+            if i not in granted:
+                res[i] = self._fail(NO_PAGES, slot); continue
+            s.beacon_pages += granted[i]; ok_items.append(i); res[i] = OK
+        # frees come after every allocation of the call
+        for i in ok_items:
+            s = self.seqs[slots[i]]
+            self.stack.extend(s.window_pages)
+            s.window_pages = []; s.window_len = 0; s.n_beacons += 1
+        return res
+
+    def close(self, slots):
+        self.calls += 1
+        res = [None] * len(slots)
+        for i, slot in enumerate(slots):
+            s = self.seqs.get(slot)
+            if s is None:
+                res[i] = self._fail(BAD_SLOT, slot); continue
+            self.stack.extend(s.prompt_pages + s.beacon_pages + s.window_pages)
+            del self.seqs[slot]; res[i] = OK
+        return res
+
+    # ------------------------------------------------------------------- views
+    def state(self, slot):
+        s = self.seqs.get(slot)
+        if s is None:
+            return None
+        return dict(prompt_len=s.P, n_beacons=s.n_beacons, window_len=s.window_len, c=s.c, t=s.t,
+                    prompt_pages=list(s.prompt_pages), beacon_pages=list(s.beacon_pages),
+                    window_pages=list(s.window_pages))
+
+    def free_list(self):
+        """Free pages, bottom of the stack first (the last one is handed out next)."""
+        return list(self.stack)

@@ -1,0 +1,322 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix.
+
+None of these re-types the oracle's formula; each one is a closed form, an
+invariant, a special case or a second formulation, chosen so that a plausible
+mistake in the oracle (dropped scale, wrong head mapping, transposed operand,
+off-by-one in the eviction slice, beacon not attending itself, ...) fails.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle.breadcrumbs_oracle import (SeqCache, attention, closed_form_length,
+                                       closed_form_live_ids, mask_form_outputs)
+from oracle.paging_model import (BAD_SLOT, CAPACITY, NO_PAGES, OK, WINDOW_FULL,
+                                 WINDOW_NOT_FULL, PagingModel)
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(name):
+    out = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                out.append([float(x) for x in line.split()])
+    return out
+
+
+# ----------------------------------------------------------------- attention
+def test_two_key_closed_form_and_scale():
+    """logits ln a, ln b -> weights a/(a+b), b/(a+b); the logit is scale * <q,k>."""
+    D = 8
+    for a, b, w1, w2 in _rows("softmax_two_keys.txt"):
+        for scale in (1.0, 0.5, 1.0 / math.sqrt(D)):
+            q = np.zeros((1, D)); q[0, 2] = 2.0          # asymmetric: only coordinate 2 counts
+            K = np.zeros((2, 1, D)); V = np.zeros((2, 1, D))
+            K[0, 0, 2] = math.log(a) / (2.0 * scale)
+            K[1, 0, 2] = math.log(b) / (2.0 * scale)
+            K[:, 0, 5] = [9.0, -9.0]                      # must be ignored (q[5] == 0)
+            V[0, 0] = np.arange(D); V[1, 0] = -2.0 * np.arange(D) + 1
+            o = attention(q, K, V, scale)
+            np.testing.assert_allclose(o[0], w1 * V[0, 0] + w2 * V[1, 0], rtol=0, atol=1e-13)
+
+
+def test_identical_keys_give_mean_of_values():
+    rng = np.random.RandomState(0)
+    n, Hkv, G, D = 37, 2, 3, 16
+    k = rng.randn(Hkv, D)
+    K = np.broadcast_to(k, (n, Hkv, D)).copy()
+    V = rng.randn(n, Hkv, D)
+    q = rng.randn(Hkv * G, D)
+    o = attention(q, K, V, 0.3)
+    for h in range(Hkv * G):
+        np.testing.assert_allclose(o[h], V[:, h // G].mean(axis=0), atol=1e-13)
+
+
+def test_single_key_and_empty_cache():
+    rng = np.random.RandomState(1)
+    q = rng.randn(4, 8); K = rng.randn(1, 2, 8); V = rng.randn(1, 2, 8)
+    o = attention(q, K, V, 0.7)
+    for h in range(4):
+        np.testing.assert_array_equal(o[h], V[0, h // 2])
+    assert np.all(attention(q, np.zeros((0, 2, 8)), np.zeros((0, 2, 8)), 1.0) == 0.0)
+
+
+def test_gqa_head_mapping():
+    """Query head h must read KV head h // G (not h % Hkv)."""
+    Hkv, G, D, n = 3, 4, 8, 5
+    rng = np.random.RandomState(2)
+    K = rng.randn(n, Hkv, D)
+    V = np.zeros((n, Hkv, D))
+    for j in range(Hkv):
+        V[:, j, :] = j + 1
+    o = attention(rng.randn(Hkv * G, D), K, V, 1.0)
+    for h in range(Hkv * G):
+        np.testing.assert_allclose(o[h], (h // G) + 1, atol=1e-13)
+
+
+def test_permutation_invariance_and_far_key():
+    rng = np.random.RandomState(3)
+    n, Hkv, G, D = 50, 2, 2, 16
+    q = rng.randn(Hkv * G, D); K = rng.randn(n, Hkv, D); V = rng.randn(n, Hkv, D)
+    o = attention(q, K, V, 0.25)
+    perm = rng.permutation(n)
+    np.testing.assert_allclose(attention(q, K[perm], V[perm], 0.25), o, atol=1e-13)
+    # a key whose logit is hugely negative changes nothing
+    far_k = np.zeros((1, Hkv, D)); far_v = 1e6 * np.ones((1, Hkv, D))
+    for j in range(Hkv):
+        qsum = q[j * G:(j + 1) * G].sum(axis=0)
+        far_k[0, j] = -1e4 * qsum / np.dot(qsum, qsum)
+    # make sure every head of the group sees a very negative logit
+    logits = [0.25 * q[h] @ far_k[0, h // G] for h in range(Hkv * G)]
+    if max(logits) < -500:
+        o2 = attention(q, np.concatenate([K, far_k]), np.concatenate([V, far_v]), 0.25)
+        np.testing.assert_allclose(o2, o, atol=1e-12)
+
+
+def test_dominant_key_selects_its_value():
+    """One key with an overwhelming logit -> output is that key's value (argmax limit)."""
+    rng = np.random.RandomState(4)
+    n, D = 20, 8
+    q = rng.randn(1, D); K = 0.01 * rng.randn(n, 1, D); V = rng.randn(n, 1, D)
+    K[7, 0] = 100.0 * q[0] / np.dot(q[0], q[0]) * 10
+    o = attention(q, K, V, 1.0)
+    np.testing.assert_allclose(o[0], V[7, 0], atol=1e-10)
+
+
+# ------------------------------------------------- eviction: lengths and sets
+def _run_sequence(P, T, c, Hq=2, Hkv=1, D=8, layers=1, seed=0, scale=0.35):
+    rng = np.random.RandomState(seed)
+    data = dict(
+        pk=rng.randn(layers, P, Hkv, D), pv=rng.randn(layers, P, Hkv, D),
+        k=rng.randn(layers, T, Hkv, D), v=rng.randn(layers, T, Hkv, D), q=rng.randn(layers, T, Hq, D),
+        bk=rng.randn(layers, T, Hkv, D), bv=rng.randn(layers, T, Hkv, D), bq=rng.randn(layers, T, Hq, D))
+    seq = SeqCache(layers, c)
+    for l in range(layers):
+        seq.prefill(l, data["pk"][l], data["pv"][l])
+    outs, bouts, lens_pre, lens_post, ids_post = [], [], [], [], []
+    for n in range(1, T + 1):
+        step_out = []
+        for l in range(layers):
+            seq.append(l, data["k"][l, n - 1], data["v"][l, n - 1])
+            step_out.append(seq.attend(l, data["q"][l, n - 1], scale))
+        outs.append(step_out)
+        lens_pre.append(len(seq.live_ids()))
+        if c > 1 and seq.window_len() == c:
+            m = n // c
+            bo = []
+            for l in range(layers):
+                bo.append(seq.beacon_attend(l, data["bq"][l, m - 1], data["bk"][l, m - 1],
+                                            data["bv"][l, m - 1], scale))
+                seq.compress(l, data["bk"][l, m - 1], data["bv"][l, m - 1])
+            bouts.append(bo)
+        lens_post.append(len(seq.live_ids()))
+        ids_post.append(seq.live_ids())
+    return data, np.array(outs), np.array(bouts), lens_pre, lens_post, ids_post, seq
+
+
+@pytest.mark.parametrize("P,T,c", [(5, 40, 4), (3, 33, 16), (0, 20, 2), (7, 64, 32), (4, 30, 1), (6, 25, 5)])
+def test_closed_form_lengths_and_live_sets(P, T, c):
+    _, _, _, lens_pre, lens_post, ids_post, seq = _run_sequence(P, T, c)
+    for t in range(1, T + 1):
+        assert lens_post[t - 1] == closed_form_length(P, t, c)
+        assert lens_post[t - 1] == (P + t // c + t % c if c > 1 else P + t)
+        # just before a compression the window is full: P + (t/c - 1) + c
+        if c > 1 and t % c == 0:
+            assert lens_pre[t - 1] == P + (t // c - 1) + c
+        assert ids_post[t - 1] == closed_form_live_ids(P, t, c)
+        # after any step at most c-1 live window tokens remain
+        if c > 1:
+            assert sum(1 for k, _ in ids_post[t - 1] if k == "token") <= c - 1
+    p, b, w = seq.lengths()
+    assert (p, b, w) == (P, T // c if c > 1 else 0, T % c if c > 1 else T)
+
+
+def test_paper_cache_growth_fixture():
+    for c, t, nb, w, entries in _rows("cache_growth.txt"):
+        c, t = int(c), int(t)
+        assert closed_form_length(0, t, c) == entries
+        ids = closed_form_live_ids(0, t, c)
+        assert sum(1 for k, _ in ids if k == "beacon") == nb
+        assert sum(1 for k, _ in ids if k == "token") == w
+    # "2-32x fewer entries": generated / kept tends to c
+    for c in (2, 4, 8, 16, 32):
+        t = 1000 * c
+        assert closed_form_length(0, t, c) == 1000
+    # literal simulation agrees with the closed form at the fixture points
+    _, _, _, _, lens_post, _, _ = _run_sequence(0, 48, 16, D=4)
+    assert lens_post[15 - 1] == 15 and lens_post[16 - 1] == 1 and lens_post[17 - 1] == 2
+
+
+def test_algorithm1_index_form():
+    """Re-run Algorithm 1 on token ids only, with the paper's loop index i (compress when
+    i > 0 and i mod c == 0, slice [:-c-1] + [-1]) and compare the surviving ids."""
+    P, T, c = 3, 29, 4
+    _, _, _, _, _, ids_post, _ = _run_sequence(P, T, c)
+    kv = [("prompt", j) for j in range(P)]
+    nb = 0
+    for i in range(0, T + 1):
+        # sampling x_i ran the forward pass of x_{i-1}: its entry is in the cache now
+        if i > 0:
+            kv.append(("token", i - 1))
+        if i > 0 and i % c == 0:
+            nb += 1
+            kv.append(("beacon", nb))
+            kv = kv[:-c - 1] + kv[-1:]
+        if i > 0:
+            assert kv == ids_post[i - 1]
+
+
+# ------------------------------------------- eviction form == mask form (Fig. 2)
+@pytest.mark.parametrize("P,T,c,Hq,Hkv,layers", [(5, 23, 4, 4, 2, 1), (2, 16, 16, 2, 1, 1),
+                                                  (0, 9, 2, 2, 2, 1), (6, 20, 1, 2, 1, 1),
+                                                  (3, 14, 3, 6, 2, 2)])
+def test_mask_form_equals_eviction_form(P, T, c, Hq, Hkv, layers):
+    scale = 0.35
+    data, outs, bouts, *_ = _run_sequence(P, T, c, Hq=Hq, Hkv=Hkv, layers=layers, seed=5, scale=scale)
+    nb = T // c if c > 1 else 0
+    for l in range(layers):
+        tok, bea = mask_form_outputs(data["pk"][l], data["pv"][l], data["k"][l], data["v"][l], data["q"][l],
+                                     data["bk"][l, :nb], data["bv"][l, :nb], data["bq"][l, :nb], c, scale)
+        np.testing.assert_allclose(outs[:, l], tok, atol=1e-12)
+        if nb:
+            np.testing.assert_allclose(bouts[:, l], bea, atol=1e-12)
+
+
+def test_large_c_equals_uncompressed_full_attention():
+    """c larger than the generation length: every step is plain causal attention over
+    prompt + all generated tokens, computed here by brute force with dense matrices."""
+    P, T, Hq, Hkv, D, scale = 4, 12, 4, 2, 8, 0.4
+    data, outs, bouts, *_ = _run_sequence(P, T, 100, Hq=Hq, Hkv=Hkv, D=D, seed=6, scale=scale)
+    assert bouts.size == 0
+    K = np.concatenate([data["pk"][0], data["k"][0]]); V = np.concatenate([data["pv"][0], data["v"][0]])
+    for n in range(1, T + 1):
+        Kn, Vn, q = K[:P + n], V[:P + n], data["q"][0, n - 1]
+        for h in range(Hq):
+            logits = np.einsum("d,nd->n", q[h], Kn[:, h // 2]) * scale
+            w = np.exp(logits - np.logaddexp.reduce(logits))
+            np.testing.assert_allclose(outs[n - 1, 0, h], np.einsum("n,nd->d", w, Vn[:, h // 2]), atol=1e-12)
+    # ratio 1 is the same thing
+    _, outs1, _, *_ = _run_sequence(P, T, 1, Hq=Hq, Hkv=Hkv, D=D, seed=6, scale=scale)
+    np.testing.assert_array_equal(outs1, outs)
+
+
+def test_beacon_attends_itself_and_window():
+    """With a beacon key that dominates, the beacon query's output is the beacon value; with a
+    beacon key that is negligible, it equals the attention over the cache with the full window."""
+    P, c, D = 2, 3, 4
+    seq = SeqCache(1, c)
+    rng = np.random.RandomState(7)
+    seq.prefill(0, rng.randn(P, 1, D), rng.randn(P, 1, D))
+    for _ in range(c):
+        seq.append(0, rng.randn(1, D), rng.randn(1, D))
+    qb = rng.randn(1, D)
+    bv = rng.randn(1, D)
+    strong = 1e3 * qb / np.dot(qb[0], qb[0])
+    np.testing.assert_allclose(seq.beacon_attend(0, qb, strong, bv, 1.0), bv, atol=1e-10)
+    weak = -1e3 * qb / np.dot(qb[0], qb[0])
+    np.testing.assert_allclose(seq.beacon_attend(0, qb, weak, bv, 1.0), seq.attend(0, qb, 1.0), atol=1e-10)
+    assert len(seq.live_ids()) == P + c           # beacon_attend mutates nothing
+    with pytest.raises(RuntimeError):
+        seq.append(0, rng.randn(1, D), rng.randn(1, D))     # window full: compress first
+    seq.compress(0, strong, bv)
+    assert seq.live_ids() == [("prompt", 0), ("prompt", 1), ("beacon", 1)]
+    with pytest.raises(RuntimeError):
+        seq.compress(0, strong, bv)                          # window not full
+
+
+# ------------------------------------------------------------- paging model
+def _check_invariants(m: PagingModel):
+    owned = []
+    for slot in list(m.seqs):
+        st = m.state(slot)
+        ps = m.ps
+        assert len(st["prompt_pages"]) == -(-st["prompt_len"] // ps)
+        assert len(st["beacon_pages"]) == -(-st["n_beacons"] // ps)
+        assert len(st["window_pages"]) == -(-st["window_len"] // ps)
+        if st["c"] > 1:
+            assert st["n_beacons"] * st["c"] + st["window_len"] == st["t"] and st["window_len"] <= st["c"]
+        owned += st["prompt_pages"] + st["beacon_pages"] + st["window_pages"]
+    free = m.free_list()
+    assert len(set(owned)) == len(owned), "a page is owned twice"
+    assert sorted(owned + free) == list(range(m.num_pages)), "conservation broken"
+
+
+@pytest.mark.parametrize("ps,c", [(16, 16), (2, 2), (4, 16), (16, 4), (3, 7), (8, 1), (1, 5)])
+def test_paging_invariants_and_closed_form(ps, c):
+    m = PagingModel(num_pages=400, page_size=ps, max_seqs=4, max_pages_per_seq=200)
+    P = [5, 0, 17]
+    assert m.open([0, 1, 3], P, [c, c, c]) == [OK, OK, OK]
+    _check_invariants(m)
+    for t in range(1, 60):
+        assert m.append([0, 1, 3]) == [OK, OK, OK]
+        _check_invariants(m)
+        if c > 1 and t % c == 0:
+            assert m.compress([3, 0, 1]) == [OK, OK, OK]
+            _check_invariants(m)
+        else:
+            assert m.compress([0]) == [WINDOW_NOT_FULL]
+        for slot, p in zip([0, 1, 3], P):
+            st = m.state(slot)
+            assert p + st["n_beacons"] + st["window_len"] == closed_form_length(p, t, c)
+    assert m.close([1, 0, 3]) == [OK, OK, OK]
+    assert sorted(m.free_list()) == list(range(400)) and not m.seqs
+
+
+def test_paging_order_worked_by_hand():
+    """Fresh store hands out 0,1,2,...; frees are pushed in batch order and reused LIFO."""
+    m = PagingModel(num_pages=8, page_size=2, max_seqs=3, max_pages_per_seq=8)
+    assert m.open([0, 1], [3, 1], [2, 2]) == [OK, OK]          # needs 2 and 1 pages
+    assert m.state(0)["prompt_pages"] == [0, 1] and m.state(1)["prompt_pages"] == [2]
+    assert m.free_list() == [7, 6, 5, 4, 3]
+    assert m.append([1, 0]) == [OK, OK]                         # batch order 1 then 0
+    assert m.state(1)["window_pages"] == [3] and m.state(0)["window_pages"] == [4]
+    assert m.append([0, 1]) == [OK, OK]                         # second slot of the same page
+    assert m.free_list() == [7, 6, 5]
+    assert m.append([0]) == [WINDOW_FULL]
+    assert m.compress([0, 1]) == [OK, OK]                       # beacon pages 5, 6; then free 4, 3
+    assert m.state(0)["beacon_pages"] == [5] and m.state(1)["beacon_pages"] == [6]
+    assert m.free_list() == [7, 4, 3]
+    assert m.append([0]) == [OK] and m.state(0)["window_pages"] == [3]
+    assert m.close([0]) == [OK]                                 # prompt 0,1 then beacon 5 then window 3
+    assert m.free_list() == [7, 4, 0, 1, 5, 3]
+    assert m.close([0]) == [BAD_SLOT]
+    assert m.first_error == (WINDOW_FULL, 0, 4)
+
+
+def test_paging_exhaustion_and_capacity():
+    m = PagingModel(num_pages=3, page_size=1, max_seqs=4, max_pages_per_seq=10, max_entries_per_seq=2)
+    assert m.open([0, 1, 2], [1, 3, 0], [1, 1, 1]) == [OK, NO_PAGES, OK]   # 1 granted, 3 refused, 0 needs none
+    assert m.free_list() == [2, 1]
+    assert m.append([0, 2]) == [OK, OK]
+    assert m.append([0, 2]) == [NO_PAGES, NO_PAGES]
+    m2 = PagingModel(num_pages=30, page_size=1, max_seqs=1, max_pages_per_seq=30, max_entries_per_seq=2)
+    m2.open([0], [5], [1])
+    assert m2.append([0]) == [OK] and m2.append([0]) == [OK] and m2.append([0]) == [CAPACITY]
+    m3 = PagingModel(num_pages=30, page_size=1, max_seqs=1, max_pages_per_seq=6)
+    m3.open([0], [5], [1])
+    assert m3.append([0]) == [OK] and m3.append([0]) == [CAPACITY]

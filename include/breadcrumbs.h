@@ -1,0 +1,235 @@
+/*
+ * breadcrumbs.h - C ABI of libbreadcrumbs.so
+ *
+ * Batched decode-step attention over a beacon-compressed, paged bf16 KV cache, and the
+ * compress-and-evict step, for NVIDIA B200 (sm_100a).
+ *
+ * The method (Breadcrumbs Reasoning, Algorithm 1 and Section 3.1 of the paper): a sequence's
+ * cache holds the prompt entries, one "beacon" entry per completed window of c generated tokens,
+ * and the live entries of the current window.  When the window holds c tokens, a beacon token is
+ * run through the model; its query attends to prompt + earlier beacons + the window + itself, its
+ * K/V entry is appended and the c window entries are evicted.  Attention itself is ordinary
+ * softmax attention over whatever the cache holds (Section 2; Figure 2 caption).  The model
+ * forward pass is not part of this library: q, k, v and the beacon's k, v are inputs.
+ *
+ * Conventions
+ *  - Every function returns a bc_status (0 = BC_OK, negative = error).  Nothing throws, aborts or
+ *    traps on the device.
+ *  - "device pointer" = memory of the current CUDA device, owned by the caller, 16-byte aligned,
+ *    contiguous; the library never allocates or frees device memory.  "host pointer" = ordinary
+ *    host memory.  `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *  - Hot-path calls only enqueue work on `stream` and return; they never synchronise, so a decode
+ *    step can be captured in a CUDA graph.  Argument errors are returned at once.  State errors
+ *    found on the device (no free page, window full, ...) make the operation a no-op for that
+ *    sequence and are latched (first one wins) in a device status record read by bc_poll_error.
+ *  - Tensors are bf16.  K/V tensors are [n, kv_heads, head_dim]; q and out are
+ *    [n, q_heads, head_dim]; query head h reads KV head h / (q_heads / kv_heads).
+ *  - Layers: `layer` in [0, layers) addresses one layer.  A sequence's bookkeeping (lengths, page
+ *    table) is shared by all layers and changes once per step: bc_append reserves the new slot on
+ *    its layer-0 call, bc_compress allocates the beacon slot on its layer-0 call and evicts the
+ *    window on its call for the last layer.  For one step, call the layers in ascending order
+ *    with the same `slots`; anything else returns BC_ERR_ORDER.
+ *  - A batch must not name the same slot twice.
+ *
+ * Store layout (owned by the library inside the caller's `pool` buffer)
+ *    pool[layer][page][slot_in_page][K|V][kv_head][head_dim] bf16: one token's entry of one layer
+ *    is E = 2*kv_heads*head_dim*2 contiguous bytes and a page is page_size*E contiguous bytes, so
+ *    any run of tokens inside a page is one contiguous block.  Inside each head row the 16-byte
+ *    chunks are stored XOR-permuted by (position of the entry in its segment) & 7, which makes the
+ *    shared-memory image of a bulk copy free of bank conflicts; bc_export_seq undoes it.
+ *
+ * Page allocation discipline (deterministic, so page ownership is reproducible bit for bit)
+ *    Free pages form a LIFO stack; a fresh cache hands out pages 0, 1, 2, ...  Within one call,
+ *    allocations come first: batch item i needing need[i] pages takes the pages at stack depth
+ *    off[i] .. off[i]+need[i]-1, off = exclusive prefix sum of the needs of all items that passed
+ *    validation; it is granted iff need[i] == 0 or off[i]+need[i] <= pages free at the start of
+ *    the call.  Frees follow, in batch order; a sequence's pages are pushed prompt pages first,
+ *    then beacon pages, then window pages, each in ascending order.
+ */
+#ifndef BREADCRUMBS_H_
+#define BREADCRUMBS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define BC_API __attribute__((visibility("default")))
+#else
+#define BC_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t bc_status;
+enum {
+  BC_OK = 0,
+  BC_ERR_INVALID_ARG = -1,     /* null/misaligned pointer, n <= 0, bad layer, bad config, c < 1 */
+  BC_ERR_BAD_SLOT = -2,        /* slot out of range, not open, or already open */
+  BC_ERR_NO_PAGES = -3,        /* free stack too small for this item */
+  BC_ERR_CAPACITY = -4,        /* max_entries_per_seq or max_pages_per_seq would be exceeded */
+  BC_ERR_WINDOW_NOT_FULL = -5, /* bc_compress on a window that does not hold exactly c entries */
+  BC_ERR_WINDOW_FULL = -6,     /* bc_append on a full window (c > 1): compress first */
+  BC_ERR_ORDER = -7,           /* per-layer calls out of order */
+  BC_ERR_CUDA = -8,            /* a CUDA runtime call failed; see bc_last_cuda_error */
+  BC_ERR_UNSUPPORTED = -9,     /* shape outside what the kernels are built for */
+  BC_ERR_TIMEOUT = -10         /* a bounded device-side wait gave up (kernel returned early) */
+};
+
+enum {
+  BC_FLAG_OUT_F32 = 1u,        /* bc_decode_attn writes fp32 instead of bf16 */
+  BC_FLAG_ATTN_REFERENCE = 2u  /* use the slow one-warp-per-head device kernel (debugging aid) */
+};
+
+typedef struct bc_cache bc_cache; /* opaque host-side handle */
+
+typedef struct {
+  int32_t layers;
+  int32_t kv_heads;            /* 1, 2, 4 or 8 */
+  int32_t q_heads;             /* multiple of kv_heads, q_heads/kv_heads <= 16, q_heads*head_dim <= 4096 */
+  int32_t head_dim;            /* 64 or 128 */
+  int32_t c_default;           /* compression ratio used when bc_seq_open gets no per-sequence c;
+                                  1 = never compress (in the paper's tables the ratio-1
+                                  column is the uncompressed teacher) */
+  int32_t page_size;           /* tokens per page, >= 1; need not divide or equal c */
+  int32_t max_seqs;            /* number of sequence slots */
+  int32_t num_pages;           /* pages in the pool (each page spans all layers) */
+  int32_t max_pages_per_seq;   /* width of one page-table row */
+  int32_t max_entries_per_seq; /* cap on beacons + live window entries of a sequence, the cache-size
+                                  limit of the paper's evaluation, at which generation is cut off
+                                  (Evaluation paragraph); 0 = unlimited */
+  uint32_t flags;
+} bc_config;
+
+typedef struct {
+  int32_t open;                /* 1 if the slot is open */
+  int32_t prompt_len, n_beacons, window_len, c;
+  int32_t t;                   /* generated-token entries appended so far */
+  int32_t n_prompt_pages, n_beacon_pages, n_window_pages;
+} bc_seq_state;
+
+/* Library version, major*10000 + minor*100 + patch. */
+BC_API int32_t bc_version(void);
+
+/* Sizes of the three caller-provided device buffers for this configuration (host pointers out).
+ * pool: the K/V pages; meta: lengths, page tables, free stack, status; workspace: split-K
+ * partials and per-call scratch. */
+BC_API bc_status bc_cache_query_bytes(const bc_config* cfg, size_t* pool_bytes, size_t* meta_bytes,
+                               size_t* workspace_bytes);
+
+/* Creates the host handle over caller-owned device buffers of at least the queried sizes
+ * (256-byte aligned) and enqueues, on `stream`, the kernel that resets the bookkeeping.  The pool
+ * content is not touched.  The five-argument form bc_cache_create(layers, kv_heads, head_dim, c,
+ * page_size) of the problem statement is this call with the remaining fields of bc_config filled
+ * in by the caller. */
+BC_API bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* workspace,
+                          void* stream, bc_cache** out);
+
+/* Frees the host handle only. */
+BC_API bc_status bc_cache_destroy(bc_cache* cache);
+
+/* Algorithm 1, initialisation: opens n sequence slots with their prompt lengths and compression
+ * ratios and allocates ceil(prompt_len/page_size) prompt pages each.  slots, prompt_lens,
+ * c_per_seq (may be NULL -> c_default): device pointers to n int32.  c stays fixed for the life
+ * of the sequence (Discussion section: a ratio, once chosen, is not changed mid-generation). */
+BC_API bc_status bc_seq_open(bc_cache* cache, const int32_t* slots, const int32_t* prompt_lens,
+                      const int32_t* c_per_seq, int32_t n, void* stream);
+
+/* Algorithm 1, prompt encoding: stores the prompt K/V of one layer.  k, v: device
+ * [total_tokens, kv_heads, head_dim] bf16, sequences packed back to back; cu_prompt_lens: device
+ * int32[n+1] exclusive prefix sums (cu[n] == total_tokens, passed again as a host int). */
+BC_API bc_status bc_prefill(bc_cache* cache, int32_t layer, const int32_t* slots,
+                     const int32_t* cu_prompt_lens, int32_t n, int32_t total_tokens,
+                     const void* k, const void* v, void* stream);
+
+/* Algorithm 1, sampling step (the forward pass of a token adds its entry to the cache): appends one generated
+ * token's K/V entry to the live window of each of n sequences.  A window page is allocated when
+ * the window length is a multiple of page_size.  k, v: device [n, kv_heads, head_dim]. */
+BC_API bc_status bc_append(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
+                    const void* k, const void* v, void* stream);
+
+/* The attention read of a decode step (Section 2, standard attention; Figure 2 caption for what
+ * is visible): out[i,h] = softmax_j(sm_scale * <q[i,h], K_j>) V_j over every live entry of
+ * sequence slots[i] in `layer`: prompt, beacons, window.  If extra_k/extra_v are non-NULL
+ * ([n, kv_heads, head_dim]) one more entry per sequence is attended without being stored: this is
+ * the beacon's own K/V when the beacon query is evaluated (Algorithm 1, the beacon-encoding step).  q: device
+ * [n, q_heads, head_dim] bf16; out: same shape, bf16 (fp32 with BC_FLAG_OUT_F32), rounded to
+ * nearest even from fp32.  Accumulation is fp32.  A sequence with no entry at all gets zeros.
+ * n <= 512 per call. */
+BC_API bc_status bc_decode_attn(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
+                         const void* q, void* out, float sm_scale, const void* extra_k,
+                         const void* extra_v, void* stream);
+
+/* Algorithm 1, the eviction statement (keep everything but the c entries before the beacon, then
+ * the beacon): for each of n sequences whose window holds exactly c entries, stores the beacon's
+ * K/V in the beacon segment (a beacon page is allocated when n_beacons is a multiple of
+ * page_size), returns the window's pages to the free stack, sets window_len = 0 and n_beacons += 1.
+ * beacon_k, beacon_v: device [n, kv_heads, head_dim]. */
+BC_API bc_status bc_compress(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
+                      const void* beacon_k, const void* beacon_v, void* stream);
+
+/* Algorithm 1, stop token / cache cap: closes n sequences and returns all their pages. */
+BC_API bc_status bc_seq_close(bc_cache* cache, const int32_t* slots, int32_t n, void* stream);
+
+/* ---- end-to-end helpers with HOST buffers (pinned memory recommended) ------------------------
+ * One decode step of one layer: copies q, k, v to device staging inside `workspace`, runs
+ * bc_append + bc_decode_attn, copies out back.  All asynchronous on `stream`.  n <= 512. */
+BC_API bc_status bc_decode_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
+                              const void* q_host, const void* k_host, const void* v_host,
+                              void* out_host, float sm_scale, void* stream);
+/* The beacon step with host buffers: beacon-query attention (beacon K/V as the extra entry), then
+ * bc_compress. */
+BC_API bc_status bc_compress_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
+                                const void* beacon_q_host, const void* beacon_k_host,
+                                const void* beacon_v_host, void* out_host, float sm_scale,
+                                void* stream);
+
+/* ---- inspection (these synchronise `stream`; for tests and tools) ---------------------------- */
+
+/* Bookkeeping of one slot.  pages (host, may be NULL) receives up to pages_cap page ids: prompt
+ * pages, then beacon pages, then window pages. */
+BC_API bc_status bc_get_state(bc_cache* cache, int32_t slot, bc_seq_state* out, int32_t* pages,
+                       int32_t pages_cap, void* stream);
+
+/* The free stack, bottom first (the last element is handed out next).  pages: host array of at
+ * least num_pages int32. */
+BC_API bc_status bc_get_free_list(bc_cache* cache, int32_t* pages, int32_t* count, void* stream);
+
+/* First latched device-side error, or BC_OK: its code, slot and the 1-based index of the
+ * bookkeeping call (open/append/compress/close, counted per cache) that raised it. */
+BC_API bc_status bc_poll_error(bc_cache* cache, int32_t* code, int32_t* slot, int64_t* call_index,
+                        void* stream);
+
+/* Clears the latched error record. */
+BC_API bc_status bc_clear_error(bc_cache* cache, void* stream);
+
+/* Gathers the live entries of one sequence in logical order (prompt, beacons, window), with the
+ * storage permutation undone: k_out, v_out device [capacity, kv_heads, head_dim] bf16; writes
+ * min(entries, capacity) rows.  Asynchronous. */
+BC_API bc_status bc_export_seq(bc_cache* cache, int32_t layer, int32_t slot, void* k_out, void* v_out,
+                        int32_t capacity, void* stream);
+
+/* ---- tuning and measurement ------------------------------------------------------------------ */
+
+/* Number of thread blocks of the decode-attention kernel (0 = one per SM).  The flat tile
+ * partition adapts, so this also forces a given number of key splits per sequence in tests. */
+BC_API bc_status bc_set_attn_ctas(bc_cache* cache, int32_t ctas);
+
+/* While enabled, every bc_decode_attn brackets its attention kernel with CUDA events on `stream`
+ * (up to max_launches per enable).  bc_profile_read synchronises and returns the number of
+ * bracketed launches and the sum of their durations in milliseconds. */
+BC_API bc_status bc_profile_enable(bc_cache* cache, int32_t max_launches);
+BC_API bc_status bc_profile_read(bc_cache* cache, int32_t* launches, float* total_ms);
+
+/* Kernels launched by this handle since creation (for launch accounting). */
+BC_API int64_t bc_kernel_launches(const bc_cache* cache);
+
+/* Last CUDA runtime error code seen by this handle (0 if none) and its text. */
+BC_API int32_t bc_last_cuda_error(const bc_cache* cache);
+BC_API const char* bc_status_string(bc_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BREADCRUMBS_H_ */

@@ -14,7 +14,7 @@ What it follows
 * Section 3.1: the token sampled right before the beacon is fed again after
   it, so the evicted window is the c tokens whose entries are already cached
   and the re-fed token opens the next window.
-* Section 2 ("standard Transformer attention mechanism") and the caption of
+* Section 2 (the method keeps the ordinary Transformer attention) and the caption of
   Figure 2: a query attends, with ordinary softmax attention, to whatever the
   cache holds: question tokens, all earlier beacons, the tokens of the current
   window, and itself.  ``attention`` is that definition written out.
@@ -47,7 +47,7 @@ __all__ = [
 
 
 # --------------------------------------------------------------------------
-# Attention: the plain definition (Section 2: standard Transformer attention)
+# Attention: the plain definition (Section 2: ordinary Transformer attention)
 # --------------------------------------------------------------------------
 def attention(q, K, V, sm_scale):
     """Softmax attention of Hq query heads over n cached entries, in fp64.
@@ -97,7 +97,7 @@ class SeqCache:
         self.t = 0           # generated-token entries appended so far (layer 0)
         self.n_beacons = 0   # beacons kept so far (counted when the last layer compresses)
 
-    # -- Algorithm 1, "Initialize: encode the prompt" -----------------------
+    # -- Algorithm 1, initialisation: the prompt is encoded first --------------
     def prefill(self, layer, k, v):
         k = np.asarray(k, dtype=np.float64)
         v = np.asarray(v, dtype=np.float64)
@@ -119,7 +119,7 @@ class SeqCache:
         K, V = self._stack(self.cache[layer])
         return attention(q, K, V, sm_scale)
 
-    # -- Algorithm 1, "encode the beacon": its query sees the cache plus itself
+    # -- Algorithm 1, beacon encoding: its query sees the cache plus itself
     def beacon_attend(self, layer, q_b, beacon_k, beacon_v, sm_scale):
         tail = ("beacon", self._beacons_in(layer) + 1,
                 np.asarray(beacon_k, np.float64), np.asarray(beacon_v, np.float64))

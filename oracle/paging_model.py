@@ -16,7 +16,8 @@ include/breadcrumbs.h, written here independently with plain Python lists:
   Frees: walk the batch in order; a sequence's pages are pushed in the order
   prompt pages, beacon pages, window pages, each in ascending index.
 * A failed item is a no-op for its sequence; the first failure of the store's
-  lifetime is latched as (code, slot, call index).
+  lifetime is latched as (code, slot, call index); when several items of one
+  call fail, the one with the lowest batch index is reported.
 
 Pinned by tests/test_oracle_pins.py: conservation (owned + free = all pages,
 no page twice), per-segment page counts = ceil(len / page_size), lengths equal
@@ -60,13 +61,22 @@ class PagingModel:
         self.stack = list(range(num_pages - 1, -1, -1))   # stack[-1] == page 0
         self.seqs = {}
         self.first_error = None       # (code, slot, call_index)
+        self._pending = []
         self.calls = 0
 
     # ------------------------------------------------------------------ utils
-    def _fail(self, code, slot):
-        if self.first_error is None:
-            self.first_error = (code, slot, self.calls)
+    def _fail(self, code, slot, item):
+        self._pending.append((item, code, slot))
         return code
+
+    def _latch(self, res):
+        """Of the failures of one call, the one with the lowest batch index is the call's
+        error; the first failing call of the store's lifetime is the latched one."""
+        if self._pending and self.first_error is None:
+            _, code, slot = min(self._pending)
+            self.first_error = (code, slot, self.calls)
+        self._pending = []
+        return res
 
     def _allocate(self, needs):
         """needs: list of (item index, pages needed) for validated items, in
@@ -93,22 +103,22 @@ class PagingModel:
             c = self.c_default if cs is None else cs[i]
             P = prompt_lens[i]
             if not (0 <= slot < self.max_seqs) or slot in self.seqs:
-                res[i] = self._fail(BAD_SLOT, slot); continue
+                res[i] = self._fail(BAD_SLOT, slot, i); continue
             if c < 1 or P < 0:
-                res[i] = self._fail(INVALID_ARG, slot); continue
+                res[i] = self._fail(INVALID_ARG, slot, i); continue
             npp = _ceil_div(P, self.ps)
             nwp = _ceil_div(c, self.ps) if c > 1 else 0
             if npp + nwp > self.max_pages_per_seq:
-                res[i] = self._fail(CAPACITY, slot); continue
+                res[i] = self._fail(CAPACITY, slot, i); continue
             needs.append((i, npp)); plan[i] = (slot, P, c)
         granted = self._allocate(needs)
         for i, _ in needs:
             slot, P, c = plan[i]
             if i not in granted:
-                res[i] = self._fail(NO_PAGES, slot); continue
+                res[i] = self._fail(NO_PAGES, slot, i); continue
             s = _Seq(P, c); s.prompt_pages = granted[i]
             self.seqs[slot] = s; res[i] = OK
-        return res
+        return self._latch(res)
 
     def append(self, slots):
         self.calls += 1
@@ -116,24 +126,24 @@ class PagingModel:
         for i, slot in enumerate(slots):
             s = self.seqs.get(slot)
             if s is None:
-                res[i] = self._fail(BAD_SLOT, slot); continue
+                res[i] = self._fail(BAD_SLOT, slot, i); continue
             if s.c > 1 and s.window_len >= s.c:
-                res[i] = self._fail(WINDOW_FULL, slot); continue
+                res[i] = self._fail(WINDOW_FULL, slot, i); continue
             if self.max_entries and s.n_beacons + s.window_len + 1 > self.max_entries:
-                res[i] = self._fail(CAPACITY, slot); continue
+                res[i] = self._fail(CAPACITY, slot, i); continue
             need = 1 if s.window_len % self.ps == 0 else 0
             if need and (len(s.prompt_pages) + len(s.beacon_pages) + len(s.window_pages) + 1
                          > self.max_pages_per_seq):
-                res[i] = self._fail(CAPACITY, slot); continue
+                res[i] = self._fail(CAPACITY, slot, i); continue
             needs.append((i, need))
         granted = self._allocate(needs)
         for i, _ in needs:
             slot = slots[i]; s = self.seqs[slot]
             if i not in granted:
-                res[i] = self._fail(NO_PAGES, slot); continue
+                res[i] = self._fail(NO_PAGES, slot, i); continue
             s.window_pages += granted[i]
             s.window_len += 1; s.t += 1; res[i] = OK
-        return res
+        return self._latch(res)
 
     def compress(self, slots):
         self.calls += 1
@@ -141,27 +151,27 @@ class PagingModel:
         for i, slot in enumerate(slots):
             s = self.seqs.get(slot)
             if s is None:
-                res[i] = self._fail(BAD_SLOT, slot); continue
+                res[i] = self._fail(BAD_SLOT, slot, i); continue
             if s.c <= 1 or s.window_len != s.c:
-                res[i] = self._fail(WINDOW_NOT_FULL, slot); continue
+                res[i] = self._fail(WINDOW_NOT_FULL, slot, i); continue
             need = 1 if s.n_beacons % self.ps == 0 else 0
             if need and (len(s.prompt_pages) + len(s.beacon_pages) + _ceil_div(s.c, self.ps) + 1
                          > self.max_pages_per_seq):
-                res[i] = self._fail(CAPACITY, slot); continue
+                res[i] = self._fail(CAPACITY, slot, i); continue
             needs.append((i, need))
         granted = self._allocate(needs)
         ok_items = []
         for i, _ in needs:
             slot = slots[i]; s = self.seqs[slot]
             if i not in granted:
-                res[i] = self._fail(NO_PAGES, slot); continue
+                res[i] = self._fail(NO_PAGES, slot, i); continue
             s.beacon_pages += granted[i]; ok_items.append(i); res[i] = OK
         # frees come after every allocation of the call
         for i in ok_items:
             s = self.seqs[slots[i]]
             self.stack.extend(s.window_pages)
             s.window_pages = []; s.window_len = 0; s.n_beacons += 1
-        return res
+        return self._latch(res)
 
     def close(self, slots):
         self.calls += 1
@@ -169,10 +179,10 @@ class PagingModel:
         for i, slot in enumerate(slots):
             s = self.seqs.get(slot)
             if s is None:
-                res[i] = self._fail(BAD_SLOT, slot); continue
+                res[i] = self._fail(BAD_SLOT, slot, i); continue
             self.stack.extend(s.prompt_pages + s.beacon_pages + s.window_pages)
             del self.seqs[slot]; res[i] = OK
-        return res
+        return self._latch(res)
 
     # ------------------------------------------------------------------- views
     def state(self, slot):

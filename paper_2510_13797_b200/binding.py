@@ -1,0 +1,222 @@
+"""ctypes binding of libbreadcrumbs.so: argument marshalling only.
+
+Function names and argument order mirror include/breadcrumbs.h.  Tensors are
+torch CUDA tensors used purely as device buffers; every step of the hot path
+runs inside the library's kernels.  If the shared library is missing the import
+of `lib()` raises: there is no CPU or PyTorch fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+# status codes and flags of breadcrumbs.h
+BC_OK = 0
+BC_ERR_INVALID_ARG, BC_ERR_BAD_SLOT, BC_ERR_NO_PAGES, BC_ERR_CAPACITY = -1, -2, -3, -4
+BC_ERR_WINDOW_NOT_FULL, BC_ERR_WINDOW_FULL, BC_ERR_ORDER, BC_ERR_CUDA = -5, -6, -7, -8
+BC_ERR_UNSUPPORTED, BC_ERR_TIMEOUT = -9, -10
+BC_FLAG_OUT_F32, BC_FLAG_ATTN_REFERENCE = 1, 2
+STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SLOT", -3: "NO_PAGES", -4: "CAPACITY",
+                -5: "WINDOW_NOT_FULL", -6: "WINDOW_FULL", -7: "ORDER", -8: "CUDA",
+                -9: "UNSUPPORTED", -10: "TIMEOUT"}
+
+
+class BcConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("layers", "kv_heads", "q_heads", "head_dim", "c_default", "page_size", "max_seqs",
+                 "num_pages", "max_pages_per_seq", "max_entries_per_seq")] + [("flags", C.c_uint32)]
+
+
+class BcSeqState(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("open", "prompt_len", "n_beacons", "window_len", "c", "t",
+                 "n_prompt_pages", "n_beacon_pages", "n_window_pages")]
+
+
+class BreadcrumbsError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: BC_ERR_{STATUS_NAMES.get(status, status)}")
+
+
+_LIB = None
+
+# every symbol breadcrumbs.h declares: name -> (restype, argtypes)
+_P, _I32, _I64, _F = C.c_void_p, C.c_int32, C.c_int64, C.c_float
+SYMBOLS = {
+    "bc_version": (_I32, []),
+    "bc_cache_query_bytes": (_I32, [C.POINTER(BcConfig), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "bc_cache_create": (_I32, [C.POINTER(BcConfig), _P, _P, _P, _P, C.POINTER(_P)]),
+    "bc_cache_destroy": (_I32, [_P]),
+    "bc_seq_open": (_I32, [_P, _P, _P, _P, _I32, _P]),
+    "bc_prefill": (_I32, [_P, _I32, _P, _P, _I32, _I32, _P, _P, _P]),
+    "bc_append": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
+    "bc_decode_attn": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
+    "bc_compress": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
+    "bc_seq_close": (_I32, [_P, _P, _I32, _P]),
+    "bc_decode_step_host": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P]),
+    "bc_compress_step_host": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P]),
+    "bc_get_state": (_I32, [_P, _I32, C.POINTER(BcSeqState), C.POINTER(_I32), _I32, _P]),
+    "bc_get_free_list": (_I32, [_P, C.POINTER(_I32), C.POINTER(_I32), _P]),
+    "bc_poll_error": (_I32, [_P, C.POINTER(_I32), C.POINTER(_I32), C.POINTER(_I64), _P]),
+    "bc_clear_error": (_I32, [_P, _P]),
+    "bc_export_seq": (_I32, [_P, _I32, _I32, _P, _P, _I32, _P]),
+    "bc_set_attn_ctas": (_I32, [_P, _I32]),
+    "bc_profile_enable": (_I32, [_P, _I32]),
+    "bc_profile_read": (_I32, [_P, C.POINTER(_I32), C.POINTER(_F)]),
+    "bc_kernel_launches": (_I64, [_P]),
+    "bc_last_cuda_error": (_I32, [_P]),
+    "bc_status_string": (C.c_char_p, [_I32]),
+}
+
+
+def lib() -> C.CDLL:
+    """Loads libbreadcrumbs.so (building it first if sources are newer).  Raises if unavailable."""
+    global _LIB
+    if _LIB is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path) or os.environ.get("BC_REBUILD"):
+            path = _build.build_library()
+        if not os.path.exists(path):
+            raise RuntimeError("libbreadcrumbs.so is missing and could not be built; there is no fallback path")
+        handle = C.CDLL(path)
+        for name, (res, args) in SYMBOLS.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _LIB = handle
+    return _LIB
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _check(status, where):
+    if status != BC_OK:
+        raise BreadcrumbsError(status, where)
+
+
+class Cache:
+    """Owns the three device buffers (as torch tensors) and the library handle."""
+
+    def __init__(self, layers, kv_heads, q_heads, head_dim, c_default, page_size, max_seqs, num_pages,
+                 max_pages_per_seq, max_entries_per_seq=0, flags=0, device="cuda", stream=None):
+        self.cfg = BcConfig(layers, kv_heads, q_heads, head_dim, c_default, page_size, max_seqs, num_pages,
+                            max_pages_per_seq, max_entries_per_seq, flags)
+        self.device = torch.device(device)
+        sizes = [C.c_size_t() for _ in range(3)]
+        _check(lib().bc_cache_query_bytes(C.byref(self.cfg), *[C.byref(s) for s in sizes]), "bc_cache_query_bytes")
+        self.pool_bytes, self.meta_bytes, self.workspace_bytes = [s.value for s in sizes]
+        self.pool = torch.empty(self.pool_bytes, dtype=torch.uint8, device=self.device)
+        self.meta = torch.empty(self.meta_bytes, dtype=torch.uint8, device=self.device)
+        self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+        h = C.c_void_p()
+        _check(lib().bc_cache_create(C.byref(self.cfg), _ptr(self.pool), _ptr(self.meta), _ptr(self.workspace),
+                                     _stream(stream), C.byref(h)), "bc_cache_create")
+        self.handle = h
+        self.out_dtype = torch.float32 if flags & BC_FLAG_OUT_F32 else torch.bfloat16
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().bc_cache_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+    # ---- the calls of breadcrumbs.h, same names -------------------------------------------------
+    def bc_seq_open(self, slots, prompt_lens, c_per_seq=None, stream=None):
+        _check(lib().bc_seq_open(self.handle, _ptr(slots), _ptr(prompt_lens), _ptr(c_per_seq), slots.numel(),
+                                 _stream(stream)), "bc_seq_open")
+
+    def bc_prefill(self, layer, slots, cu_prompt_lens, total_tokens, k, v, stream=None):
+        _check(lib().bc_prefill(self.handle, layer, _ptr(slots), _ptr(cu_prompt_lens), slots.numel(), total_tokens,
+                                _ptr(k), _ptr(v), _stream(stream)), "bc_prefill")
+
+    def bc_append(self, layer, slots, k, v, stream=None):
+        _check(lib().bc_append(self.handle, layer, _ptr(slots), slots.numel(), _ptr(k), _ptr(v), _stream(stream)),
+               "bc_append")
+
+    def bc_decode_attn(self, layer, slots, q, out, sm_scale, extra_k=None, extra_v=None, stream=None):
+        _check(lib().bc_decode_attn(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(out), sm_scale,
+                                    _ptr(extra_k), _ptr(extra_v), _stream(stream)), "bc_decode_attn")
+
+    def bc_compress(self, layer, slots, beacon_k, beacon_v, stream=None):
+        _check(lib().bc_compress(self.handle, layer, _ptr(slots), slots.numel(), _ptr(beacon_k), _ptr(beacon_v),
+                                 _stream(stream)), "bc_compress")
+
+    def bc_seq_close(self, slots, stream=None):
+        _check(lib().bc_seq_close(self.handle, _ptr(slots), slots.numel(), _stream(stream)), "bc_seq_close")
+
+    def bc_decode_step_host(self, layer, slots, q_host, k_host, v_host, out_host, sm_scale, stream=None):
+        _check(lib().bc_decode_step_host(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q_host), _ptr(k_host),
+                                         _ptr(v_host), _ptr(out_host), sm_scale, _stream(stream)),
+               "bc_decode_step_host")
+
+    def bc_compress_step_host(self, layer, slots, bq_host, bk_host, bv_host, out_host, sm_scale, stream=None):
+        _check(lib().bc_compress_step_host(self.handle, layer, _ptr(slots), slots.numel(), _ptr(bq_host),
+                                           _ptr(bk_host), _ptr(bv_host), _ptr(out_host), sm_scale, _stream(stream)),
+               "bc_compress_step_host")
+
+    def bc_get_state(self, slot, stream=None):
+        st = BcSeqState()
+        cap = self.cfg.max_pages_per_seq
+        pages = (C.c_int32 * cap)()
+        _check(lib().bc_get_state(self.handle, slot, C.byref(st), pages, cap, _stream(stream)), "bc_get_state")
+        if not st.open:
+            return None
+        p = list(pages)
+        a, b, w = st.n_prompt_pages, st.n_beacon_pages, st.n_window_pages
+        return dict(prompt_len=st.prompt_len, n_beacons=st.n_beacons, window_len=st.window_len, c=st.c, t=st.t,
+                    prompt_pages=p[:a], beacon_pages=p[a:a + b], window_pages=p[a + b:a + b + w])
+
+    def bc_get_free_list(self, stream=None):
+        pages = (C.c_int32 * self.cfg.num_pages)()
+        count = C.c_int32()
+        _check(lib().bc_get_free_list(self.handle, pages, C.byref(count), _stream(stream)), "bc_get_free_list")
+        return list(pages[:count.value])
+
+    def bc_poll_error(self, stream=None):
+        code, slot, call = C.c_int32(), C.c_int32(), C.c_int64()
+        _check(lib().bc_poll_error(self.handle, C.byref(code), C.byref(slot), C.byref(call), _stream(stream)),
+               "bc_poll_error")
+        return code.value, slot.value, call.value
+
+    def bc_clear_error(self, stream=None):
+        _check(lib().bc_clear_error(self.handle, _stream(stream)), "bc_clear_error")
+
+    def bc_export_seq(self, layer, slot, capacity, stream=None):
+        shape = (capacity, self.cfg.kv_heads, self.cfg.head_dim)
+        k = torch.zeros(shape, dtype=torch.bfloat16, device=self.device)
+        v = torch.zeros(shape, dtype=torch.bfloat16, device=self.device)
+        _check(lib().bc_export_seq(self.handle, layer, slot, _ptr(k), _ptr(v), capacity, _stream(stream)),
+               "bc_export_seq")
+        return k, v
+
+    def bc_set_attn_ctas(self, ctas):
+        _check(lib().bc_set_attn_ctas(self.handle, ctas), "bc_set_attn_ctas")
+
+    def bc_profile_enable(self, max_launches):
+        _check(lib().bc_profile_enable(self.handle, max_launches), "bc_profile_enable")
+
+    def bc_profile_read(self):
+        n, ms = C.c_int32(), C.c_float()
+        _check(lib().bc_profile_read(self.handle, C.byref(n), C.byref(ms)), "bc_profile_read")
+        return n.value, ms.value
+
+    def bc_kernel_launches(self):
+        return lib().bc_kernel_launches(self.handle)
+
+    # ---- convenience ------------------------------------------------------------------------------
+    def new_out(self, n):
+        return torch.empty((n, self.cfg.q_heads, self.cfg.head_dim), dtype=self.out_dtype, device=self.device)

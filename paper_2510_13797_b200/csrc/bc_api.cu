@@ -1,0 +1,452 @@
+// Host side of the C ABI declared in breadcrumbs.h: argument validation, buffer carving, launch
+// sequencing.  No device allocation happens here; the caller owns pool, meta and workspace.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "bc_common.cuh"
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct MetaLayout {
+  size_t status, free_top, open, prompt_len, n_beacons, window_len, c, t, window_off, beacon_off, free_stack,
+      page_table, total;
+};
+MetaLayout meta_layout(const bc_config& c) {
+  MetaLayout l;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  const size_t seq = (size_t)c.max_seqs * 4;
+  l.status = take(16); l.free_top = take(4);
+  l.open = take(seq); l.prompt_len = take(seq); l.n_beacons = take(seq); l.window_len = take(seq);
+  l.c = take(seq); l.t = take(seq); l.window_off = take(seq); l.beacon_off = take(seq);
+  l.free_stack = take((size_t)c.num_pages * 4);
+  l.page_table = take((size_t)c.max_seqs * c.max_pages_per_seq * 4);
+  l.total = o;
+  return l;
+}
+
+struct WorkLayout {
+  size_t append_row, append_pos, compress_row, compress_pos, first_cta, last_cta, part_ml, part_o, stage_q, stage_k,
+      stage_v, stage_out, total;
+};
+WorkLayout work_layout(const bc_config& c) {
+  WorkLayout l;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  const size_t seq = (size_t)c.max_seqs * 4;
+  const size_t pieces = BC_MAX_ATTN_CTAS + BC_MAX_ATTN_BATCH;
+  l.append_row = take(seq); l.append_pos = take(seq); l.compress_row = take(seq); l.compress_pos = take(seq);
+  l.first_cta = take(BC_MAX_ATTN_BATCH * 4); l.last_cta = take(BC_MAX_ATTN_BATCH * 4);
+  l.part_ml = take(pieces * c.q_heads * 2 * 4);
+  l.part_o = take(pieces * c.q_heads * c.head_dim * 4);
+  l.stage_q = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 2);
+  l.stage_k = take((size_t)BC_MAX_ATTN_BATCH * c.kv_heads * c.head_dim * 2);
+  l.stage_v = take((size_t)BC_MAX_ATTN_BATCH * c.kv_heads * c.head_dim * 2);
+  l.stage_out = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
+  l.total = o;
+  return l;
+}
+
+bool config_ok(const bc_config* c, bc_status* why) {
+  *why = BC_ERR_INVALID_ARG;
+  if (!c) return false;
+  if (c->layers < 1 || c->kv_heads < 1 || c->q_heads < 1 || c->page_size < 1 || c->max_seqs < 1 ||
+      c->num_pages < 1 || c->max_pages_per_seq < 1 || c->c_default < 1 || c->max_entries_per_seq < 0)
+    return false;
+  if (c->q_heads % c->kv_heads) return false;
+  if ((int64_t)c->num_pages * c->page_size >= (int64_t)1 << 31) return false;
+  *why = BC_ERR_UNSUPPORTED;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->kv_heads != 1 && c->kv_heads != 2 && c->kv_heads != 4 && c->kv_heads != 8) return false;
+  if (c->q_heads / c->kv_heads > 16) return false;
+  if (c->q_heads * c->head_dim > BC_MERGE_ELEMS) return false;
+  return true;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+struct bc_cache {
+  bc_config cfg;
+  BcMeta meta;
+  BcGeom geom;
+  uint8_t* pool;
+  uint8_t* meta_base;
+  uint8_t* work;
+  MetaLayout ml;
+  WorkLayout wl;
+  int sm_count;
+  int attn_ctas;
+  int64_t calls;            // bookkeeping calls issued (1-based index of the next is calls + 1)
+  int64_t launches;
+  int append_next_layer;    // per-layer ordering of bc_append
+  int compress_next_layer;  // per-layer ordering of bc_compress
+  int last_cuda_error;
+  // profiling
+  std::vector<cudaEvent_t> ev;
+  int prof_cap, prof_used;
+};
+
+namespace {
+
+bc_status cuda_fail(bc_cache* c, cudaError_t e) {
+  if (c) c->last_cuda_error = (int)e;
+  return BC_ERR_CUDA;
+}
+#define BC_CUDA(c, expr)                                   \
+  do {                                                     \
+    cudaError_t e__ = (expr);                              \
+    if (e__ != cudaSuccess) return cuda_fail((c), e__);    \
+  } while (0)
+
+inline uint8_t* layer_base(bc_cache* c, int layer) { return c->pool + (int64_t)layer * c->geom.layer_bytes; }
+template <typename T>
+inline T* work_ptr(bc_cache* c, size_t off) { return reinterpret_cast<T*>(c->work + off); }
+
+bc_status check_batch(bc_cache* c, int layer, const int32_t* slots, int n) {
+  if (!c || !slots || n <= 0 || n > c->cfg.max_seqs) return BC_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= c->cfg.layers) return BC_ERR_INVALID_ARG;
+  return BC_OK;
+}
+
+bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const void* q, void* out, float sm_scale,
+                    const void* extra_k, const void* extra_v, cudaStream_t s) {
+  BcAttnArgs a;
+  a.pool_layer = layer_base(c, layer);
+  a.slots = slots; a.n = n; a.q = q; a.out = out;
+  a.out_f32 = (c->cfg.flags & BC_FLAG_OUT_F32) ? 1 : 0;
+  a.extra_k = extra_k; a.extra_v = extra_v; a.sm_scale = sm_scale;
+  a.part_o = work_ptr<float>(c, c->wl.part_o);
+  a.part_ml = work_ptr<float>(c, c->wl.part_ml);
+  a.first_cta = work_ptr<int32_t>(c, c->wl.first_cta);
+  a.last_cta = work_ptr<int32_t>(c, c->wl.last_cta);
+  a.ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
+  if (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) {
+    BC_CUDA(c, bc_launch_attn_reference(c->meta, c->geom, a, s));
+    c->launches += 1;
+    return BC_OK;
+  }
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (c->prof_used < c->prof_cap) { e0 = c->ev[2 * c->prof_used]; e1 = c->ev[2 * c->prof_used + 1]; c->prof_used++; }
+  int launches = 0;
+  BC_CUDA(c, bc_launch_attn(c->meta, c->geom, a, s, e0, e1, &launches));
+  c->launches += launches;
+  return BC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t bc_version(void) { return 100; }
+
+const char* bc_status_string(bc_status s) {
+  switch (s) {
+    case BC_OK: return "BC_OK";
+    case BC_ERR_INVALID_ARG: return "BC_ERR_INVALID_ARG";
+    case BC_ERR_BAD_SLOT: return "BC_ERR_BAD_SLOT";
+    case BC_ERR_NO_PAGES: return "BC_ERR_NO_PAGES";
+    case BC_ERR_CAPACITY: return "BC_ERR_CAPACITY";
+    case BC_ERR_WINDOW_NOT_FULL: return "BC_ERR_WINDOW_NOT_FULL";
+    case BC_ERR_WINDOW_FULL: return "BC_ERR_WINDOW_FULL";
+    case BC_ERR_ORDER: return "BC_ERR_ORDER";
+    case BC_ERR_CUDA: return "BC_ERR_CUDA";
+    case BC_ERR_UNSUPPORTED: return "BC_ERR_UNSUPPORTED";
+    case BC_ERR_TIMEOUT: return "BC_ERR_TIMEOUT";
+    default: return "BC_ERR_UNKNOWN";
+  }
+}
+
+bc_status bc_cache_query_bytes(const bc_config* cfg, size_t* pool_bytes, size_t* meta_bytes, size_t* workspace_bytes) {
+  bc_status why;
+  if (!config_ok(cfg, &why)) return why;
+  if (!pool_bytes || !meta_bytes || !workspace_bytes) return BC_ERR_INVALID_ARG;
+  const size_t E = (size_t)2 * cfg->kv_heads * cfg->head_dim * 2;
+  *pool_bytes = (size_t)cfg->layers * cfg->num_pages * cfg->page_size * E;
+  *meta_bytes = meta_layout(*cfg).total;
+  *workspace_bytes = work_layout(*cfg).total;
+  return BC_OK;
+}
+
+bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* workspace, void* stream, bc_cache** out) {
+  bc_status why;
+  if (!config_ok(cfg, &why)) return why;
+  if (!pool || !meta || !workspace || !out) return BC_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(pool) | reinterpret_cast<uintptr_t>(meta) | reinterpret_cast<uintptr_t>(workspace)) & 255)
+    return BC_ERR_INVALID_ARG;
+  bc_cache* c = new (std::nothrow) bc_cache();
+  if (!c) return BC_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->pool = (uint8_t*)pool; c->meta_base = (uint8_t*)meta; c->work = (uint8_t*)workspace;
+  c->ml = meta_layout(*cfg); c->wl = work_layout(*cfg);
+  c->calls = 0; c->launches = 0; c->append_next_layer = 0; c->compress_next_layer = 0; c->last_cuda_error = 0;
+  c->attn_ctas = 0; c->prof_cap = 0; c->prof_used = 0;
+  BcMeta& m = c->meta;
+  auto at = [&](size_t off) { return reinterpret_cast<int32_t*>(c->meta_base + off); };
+  m.status = at(c->ml.status); m.free_top = at(c->ml.free_top); m.free_stack = at(c->ml.free_stack);
+  m.open = at(c->ml.open); m.prompt_len = at(c->ml.prompt_len); m.n_beacons = at(c->ml.n_beacons);
+  m.window_len = at(c->ml.window_len); m.c = at(c->ml.c); m.t = at(c->ml.t);
+  m.window_off = at(c->ml.window_off); m.beacon_off = at(c->ml.beacon_off); m.page_table = at(c->ml.page_table);
+  m.max_seqs = cfg->max_seqs; m.num_pages = cfg->num_pages; m.max_pages_per_seq = cfg->max_pages_per_seq;
+  m.max_entries = cfg->max_entries_per_seq; m.page_size = cfg->page_size; m.c_default = cfg->c_default;
+  BcGeom& g = c->geom;
+  g.kv_heads = cfg->kv_heads; g.q_heads = cfg->q_heads; g.head_dim = cfg->head_dim; g.page_size = cfg->page_size;
+  g.head_row_bytes = cfg->head_dim * 2;
+  g.entry_bytes = 2 * cfg->kv_heads * g.head_row_bytes;
+  g.layer_bytes = (int64_t)cfg->num_pages * cfg->page_size * g.entry_bytes;
+  cudaError_t e = bc_attn_setup(&c->sm_count);
+  if (e == cudaSuccess) e = bc_launch_init(c->meta, (cudaStream_t)stream);
+  if (e != cudaSuccess) { delete c; return BC_ERR_CUDA; }
+  c->launches += 1;
+  *out = c;
+  return BC_OK;
+}
+
+bc_status bc_cache_destroy(bc_cache* c) {
+  if (!c) return BC_ERR_INVALID_ARG;
+  for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
+  delete c;
+  return BC_OK;
+}
+
+bc_status bc_seq_open(bc_cache* c, const int32_t* slots, const int32_t* prompt_lens, const int32_t* c_per_seq, int32_t n,
+                      void* stream) {
+  if (!c || !slots || !prompt_lens || n <= 0 || n > c->cfg.max_seqs) return BC_ERR_INVALID_ARG;
+  BC_CUDA(c, bc_launch_open(c->meta, slots, prompt_lens, c_per_seq, n, ++c->calls, (cudaStream_t)stream));
+  c->launches += 1;
+  return BC_OK;
+}
+
+bc_status bc_prefill(bc_cache* c, int32_t layer, const int32_t* slots, const int32_t* cu, int32_t n, int32_t total,
+                     const void* k, const void* v, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (!cu || total < 0) return BC_ERR_INVALID_ARG;
+  if (total == 0) return BC_OK;
+  if (!k || !v || !aligned16(k) || !aligned16(v)) return BC_ERR_INVALID_ARG;
+  BC_CUDA(c, bc_launch_prefill(c->meta, c->geom, layer_base(c, layer), slots, cu, n, total, k, v, (cudaStream_t)stream));
+  c->launches += 1;
+  return BC_OK;
+}
+
+bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* k, const void* v,
+                    void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (!k || !v || !aligned16(k) || !aligned16(v)) return BC_ERR_INVALID_ARG;
+  if (layer != c->append_next_layer) return BC_ERR_ORDER;
+  int32_t* row = work_ptr<int32_t>(c, c->wl.append_row);
+  int32_t* pos = work_ptr<int32_t>(c, c->wl.append_pos);
+  cudaStream_t s = (cudaStream_t)stream;
+  if (layer == 0) {
+    BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, ++c->calls, row, pos, s));
+    c->launches += 1;
+  }
+  BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, k, v, n, s));
+  c->launches += 1;
+  c->append_next_layer = (layer + 1) % c->cfg.layers;
+  return BC_OK;
+}
+
+bc_status bc_decode_attn(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, void* out,
+                         float sm_scale, const void* extra_k, const void* extra_v, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (n > BC_MAX_ATTN_BATCH) return BC_ERR_INVALID_ARG;
+  if (!q || !out || !aligned16(q) || !aligned16(out)) return BC_ERR_INVALID_ARG;
+  if ((extra_k == nullptr) != (extra_v == nullptr)) return BC_ERR_INVALID_ARG;
+  if (extra_k && (!aligned16(extra_k) || !aligned16(extra_v))) return BC_ERR_INVALID_ARG;
+  return attn_impl(c, layer, slots, n, q, out, sm_scale, extra_k, extra_v, (cudaStream_t)stream);
+}
+
+bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* bk, const void* bv,
+                      void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (!bk || !bv || !aligned16(bk) || !aligned16(bv)) return BC_ERR_INVALID_ARG;
+  if (layer != c->compress_next_layer) return BC_ERR_ORDER;
+  int32_t* row = work_ptr<int32_t>(c, c->wl.compress_row);
+  int32_t* pos = work_ptr<int32_t>(c, c->wl.compress_pos);
+  cudaStream_t s = (cudaStream_t)stream;
+  const int L = c->cfg.layers;
+  if (layer == 0) {
+    ++c->calls;
+    if (L > 1) {  // allocate now, evict on the last layer's call
+      BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, 1, s));
+      c->launches += 1;
+    }
+  }
+  if (L == 1) {
+    // single layer: allocate, evict, then write; the beacon row does not depend on the eviction
+    BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, 3, s));
+    c->launches += 1;
+  }
+  BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, bk, bv, n, s));
+  c->launches += 1;
+  if (L > 1 && layer == L - 1) {
+    BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, 2, s));
+    c->launches += 1;
+  }
+  c->compress_next_layer = (layer + 1) % L;
+  return BC_OK;
+}
+
+bc_status bc_seq_close(bc_cache* c, const int32_t* slots, int32_t n, void* stream) {
+  if (!c || !slots || n <= 0 || n > c->cfg.max_seqs) return BC_ERR_INVALID_ARG;
+  BC_CUDA(c, bc_launch_close(c->meta, slots, n, ++c->calls, (cudaStream_t)stream));
+  c->launches += 1;
+  return BC_OK;
+}
+
+bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q_host,
+                              const void* k_host, const void* v_host, void* out_host, float sm_scale, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (n > BC_MAX_ATTN_BATCH || !q_host || !k_host || !v_host || !out_host) return BC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+  const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
+  void *dq = c->work + c->wl.stage_q, *dk = c->work + c->wl.stage_k, *dv = c->work + c->wl.stage_v,
+       *dout = c->work + c->wl.stage_out;
+  BC_CUDA(c, cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, s));
+  BC_CUDA(c, cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, s));
+  BC_CUDA(c, cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s));
+  st = bc_append(c, layer, slots, n, dk, dv, stream);
+  if (st) return st;
+  st = attn_impl(c, layer, slots, n, dq, dout, sm_scale, nullptr, nullptr, s);
+  if (st) return st;
+  BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
+  return BC_OK;
+}
+
+bc_status bc_compress_step_host(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* bq_host,
+                                const void* bk_host, const void* bv_host, void* out_host, float sm_scale, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (n > BC_MAX_ATTN_BATCH || !bq_host || !bk_host || !bv_host || !out_host) return BC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+  const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
+  void *dq = c->work + c->wl.stage_q, *dk = c->work + c->wl.stage_k, *dv = c->work + c->wl.stage_v,
+       *dout = c->work + c->wl.stage_out;
+  BC_CUDA(c, cudaMemcpyAsync(dk, bk_host, kb, cudaMemcpyHostToDevice, s));
+  BC_CUDA(c, cudaMemcpyAsync(dv, bv_host, kb, cudaMemcpyHostToDevice, s));
+  BC_CUDA(c, cudaMemcpyAsync(dq, bq_host, qb, cudaMemcpyHostToDevice, s));
+  st = attn_impl(c, layer, slots, n, dq, dout, sm_scale, dk, dv, s);
+  if (st) return st;
+  st = bc_compress(c, layer, slots, n, dk, dv, stream);
+  if (st) return st;
+  BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
+  return BC_OK;
+}
+
+bc_status bc_get_state(bc_cache* c, int32_t slot, bc_seq_state* out, int32_t* pages, int32_t pages_cap, void* stream) {
+  if (!c || !out || slot < 0 || slot >= c->cfg.max_seqs) return BC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  BC_CUDA(c, cudaStreamSynchronize(s));
+  auto rd = [&](int32_t* arr, int32_t* dst) { return cudaMemcpy(dst, arr + slot, 4, cudaMemcpyDeviceToHost); };
+  int32_t woff = 0, boff = 0;
+  BC_CUDA(c, rd(c->meta.open, &out->open));
+  BC_CUDA(c, rd(c->meta.prompt_len, &out->prompt_len));
+  BC_CUDA(c, rd(c->meta.n_beacons, &out->n_beacons));
+  BC_CUDA(c, rd(c->meta.window_len, &out->window_len));
+  BC_CUDA(c, rd(c->meta.c, &out->c));
+  BC_CUDA(c, rd(c->meta.t, &out->t));
+  BC_CUDA(c, rd(c->meta.window_off, &woff));
+  BC_CUDA(c, rd(c->meta.beacon_off, &boff));
+  const int ps = c->cfg.page_size;
+  out->n_prompt_pages = (out->prompt_len + ps - 1) / ps;
+  out->n_beacon_pages = (out->n_beacons + ps - 1) / ps;
+  out->n_window_pages = (out->window_len + ps - 1) / ps;
+  if (pages && pages_cap > 0 && out->open) {
+    std::vector<int32_t> row(c->cfg.max_pages_per_seq);
+    BC_CUDA(c, cudaMemcpy(row.data(), c->meta.page_table + (int64_t)slot * c->cfg.max_pages_per_seq, row.size() * 4,
+                          cudaMemcpyDeviceToHost));
+    int o = 0;
+    for (int k = 0; k < out->n_prompt_pages && o < pages_cap; ++k) pages[o++] = row[k];
+    for (int k = 0; k < out->n_beacon_pages && o < pages_cap; ++k) pages[o++] = row[boff + k];
+    for (int k = 0; k < out->n_window_pages && o < pages_cap; ++k) pages[o++] = row[woff + k];
+  }
+  return BC_OK;
+}
+
+bc_status bc_get_free_list(bc_cache* c, int32_t* pages, int32_t* count, void* stream) {
+  if (!c || !pages || !count) return BC_ERR_INVALID_ARG;
+  BC_CUDA(c, cudaStreamSynchronize((cudaStream_t)stream));
+  BC_CUDA(c, cudaMemcpy(count, c->meta.free_top, 4, cudaMemcpyDeviceToHost));
+  if (*count < 0 || *count > c->cfg.num_pages) return BC_ERR_INVALID_ARG;
+  if (*count) BC_CUDA(c, cudaMemcpy(pages, c->meta.free_stack, (size_t)*count * 4, cudaMemcpyDeviceToHost));
+  return BC_OK;
+}
+
+bc_status bc_poll_error(bc_cache* c, int32_t* code, int32_t* slot, int64_t* call_index, void* stream) {
+  if (!c || !code) return BC_ERR_INVALID_ARG;
+  BC_CUDA(c, cudaStreamSynchronize((cudaStream_t)stream));
+  int32_t rec[4];
+  BC_CUDA(c, cudaMemcpy(rec, c->meta.status, 16, cudaMemcpyDeviceToHost));
+  *code = rec[0];
+  if (slot) *slot = rec[1];
+  if (call_index) memcpy(call_index, rec + 2, 8);
+  return BC_OK;
+}
+
+bc_status bc_clear_error(bc_cache* c, void* stream) {
+  if (!c) return BC_ERR_INVALID_ARG;
+  BC_CUDA(c, cudaMemsetAsync(c->meta.status, 0, 16, (cudaStream_t)stream));
+  return BC_OK;
+}
+
+bc_status bc_export_seq(bc_cache* c, int32_t layer, int32_t slot, void* k_out, void* v_out, int32_t capacity,
+                        void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.layers || slot < 0 || slot >= c->cfg.max_seqs || !k_out || !v_out ||
+      capacity < 0 || !aligned16(k_out) || !aligned16(v_out))
+    return BC_ERR_INVALID_ARG;
+  BC_CUDA(c, bc_launch_export(c->meta, c->geom, layer_base(c, layer), slot, k_out, v_out, capacity, (cudaStream_t)stream));
+  c->launches += 1;
+  return BC_OK;
+}
+
+bc_status bc_set_attn_ctas(bc_cache* c, int32_t ctas) {
+  if (!c || ctas < 0 || ctas > BC_MAX_ATTN_CTAS) return BC_ERR_INVALID_ARG;
+  c->attn_ctas = ctas;
+  return BC_OK;
+}
+
+bc_status bc_profile_enable(bc_cache* c, int32_t max_launches) {
+  if (!c || max_launches < 0) return BC_ERR_INVALID_ARG;
+  while ((int)c->ev.size() < 2 * max_launches) {
+    cudaEvent_t e;
+    BC_CUDA(c, cudaEventCreate(&e));
+    c->ev.push_back(e);
+  }
+  c->prof_cap = max_launches;
+  c->prof_used = 0;
+  return BC_OK;
+}
+
+bc_status bc_profile_read(bc_cache* c, int32_t* launches, float* total_ms) {
+  if (!c || !launches || !total_ms) return BC_ERR_INVALID_ARG;
+  float sum = 0.f;
+  for (int i = 0; i < c->prof_used; ++i) {
+    BC_CUDA(c, cudaEventSynchronize(c->ev[2 * i + 1]));
+    float ms = 0.f;
+    BC_CUDA(c, cudaEventElapsedTime(&ms, c->ev[2 * i], c->ev[2 * i + 1]));
+    sum += ms;
+  }
+  *launches = c->prof_used;
+  *total_ms = sum;
+  c->prof_cap = 0;
+  c->prof_used = 0;
+  return BC_OK;
+}
+
+int64_t bc_kernel_launches(const bc_cache* c) { return c ? c->launches : 0; }
+int32_t bc_last_cuda_error(const bc_cache* c) { return c ? c->last_cuda_error : 0; }
+
+}  // extern "C"

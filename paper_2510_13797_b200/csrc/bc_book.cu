@@ -1,0 +1,423 @@
+// Bookkeeping and data-movement kernels of the paged store: reset, open, append, compress/evict,
+// close, prefill copy, single-row writes, export.
+//
+// Every bookkeeping kernel runs as ONE thread block so that page allocation is a prefix sum over
+// the batch and page ownership is a pure function of the call sequence (the discipline stated in
+// breadcrumbs.h).  The amount of work is a few integers per sequence.
+#include "bc_common.cuh"
+
+namespace {
+
+constexpr int kBookThreads = 1024;
+
+__device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Exclusive prefix sum of one int per thread over the block; *total gets the block sum.
+// Must be called by all threads of the block.
+__device__ int block_exclusive_scan(int x, int* total) {
+  __shared__ int warp_sums[32];
+  __shared__ int block_total;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int incl = x;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    int y = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += y;
+  }
+  __syncthreads();  // protects warp_sums / block_total of a previous call
+  if (lane == 31) warp_sums[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int nw = (blockDim.x + 31) >> 5;
+    int w = lane < nw ? warp_sums[lane] : 0;
+    int wi = w;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, wi, d);
+      if (lane >= d) wi += y;
+    }
+    warp_sums[lane] = wi - w;  // exclusive warp offsets
+    if (lane == 31) block_total = wi;
+  }
+  __syncthreads();
+  *total = block_total;
+  return warp_sums[warp] + incl - x;
+}
+
+// Per-call error latch: the failing item with the lowest batch index reports, and only if no
+// earlier call has latched an error.
+struct ErrLatch {
+  int* first_item;  // shared
+  __device__ void init(int* sh) {
+    first_item = sh;
+    if (threadIdx.x == 0) *sh = 0x7fffffff;
+    __syncthreads();
+  }
+  __device__ void note(int item) { atomicMin(first_item, item); }
+  // all threads call; `item`/`code`/`slot` are this thread's failure (code == 0: none)
+  __device__ void commit(const BcMeta& m, int item, int code, int slot, int64_t call) {
+    __syncthreads();
+    if (code != 0 && item == *first_item && m.status[0] == 0) {
+      m.status[0] = code;
+      m.status[1] = slot;
+      *reinterpret_cast<int64_t*>(m.status + 2) = call;
+    }
+  }
+};
+
+__global__ void k_init(BcMeta m) {
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
+  for (int i = tid; i < m.num_pages; i += nth) m.free_stack[i] = m.num_pages - 1 - i;
+  for (int i = tid; i < m.max_seqs; i += nth) {
+    m.open[i] = 0; m.prompt_len[i] = 0; m.n_beacons[i] = 0; m.window_len[i] = 0;
+    m.c[i] = 0; m.t[i] = 0; m.window_off[i] = 0; m.beacon_off[i] = 0;
+  }
+  if (tid == 0) {
+    *m.free_top = m.num_pages;
+    m.status[0] = 0; m.status[1] = 0; m.status[2] = 0; m.status[3] = 0;
+  }
+}
+
+__global__ void __launch_bounds__(kBookThreads, 1)
+k_open(BcMeta m, const int32_t* __restrict__ slots, const int32_t* __restrict__ plens,
+       const int32_t* __restrict__ cs, int n, int64_t call) {
+  __shared__ int sh_first;
+  ErrLatch latch; latch.init(&sh_first);
+  const int top0 = *m.free_top;
+  __syncthreads();
+  int base = 0, used = 0, my_code = 0, my_item = -1, my_slot = 0;
+  for (int chunk = 0; chunk < n; chunk += blockDim.x) {
+    const int i = chunk + threadIdx.x;
+    int need = 0, slot = -1, P = 0, c = 0, code = 0;
+    bool valid = false;
+    if (i < n) {
+      slot = slots[i]; P = plens[i]; c = cs ? cs[i] : m.c_default;
+      if (slot < 0 || slot >= m.max_seqs || m.open[slot]) code = BC_ERR_BAD_SLOT;
+      else if (c < 1 || P < 0) code = BC_ERR_INVALID_ARG;
+      else {
+        need = ceil_div(P, m.page_size);
+        const int nwp = c > 1 ? ceil_div(c, m.page_size) : 0;
+        if (need + nwp > m.max_pages_per_seq) { code = BC_ERR_CAPACITY; need = 0; }
+        else valid = true;
+      }
+    }
+    int total;
+    const int off = base + block_exclusive_scan(need, &total);
+    base += total;
+    if (valid) {
+      if (need == 0 || off + need <= top0) {
+        int32_t* row = m.page_table + (int64_t)slot * m.max_pages_per_seq;
+        for (int k = 0; k < need; ++k) row[k] = m.free_stack[top0 - 1 - off - k];
+        if (need) used = max(used, off + need);
+        m.open[slot] = 1; m.prompt_len[slot] = P; m.n_beacons[slot] = 0; m.window_len[slot] = 0;
+        m.c[slot] = c; m.t[slot] = 0; m.window_off[slot] = need;
+        m.beacon_off[slot] = need + (c > 1 ? ceil_div(c, m.page_size) : 0);
+      } else code = BC_ERR_NO_PAGES;
+    }
+    if (code && my_code == 0) { my_code = code; my_item = i; my_slot = slot; latch.note(i); }
+  }
+  used = __reduce_max_sync(0xffffffffu, used);
+  __shared__ int sh_used;
+  if (threadIdx.x == 0) sh_used = 0;
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) atomicMax(&sh_used, used);
+  latch.commit(m, my_item, my_code, my_slot, call);
+  __syncthreads();
+  if (threadIdx.x == 0) *m.free_top = top0 - sh_used;
+}
+
+__global__ void __launch_bounds__(kBookThreads, 1)
+k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
+              int32_t* __restrict__ dst_row, int32_t* __restrict__ dst_pos) {
+  __shared__ int sh_first;
+  ErrLatch latch; latch.init(&sh_first);
+  const int top0 = *m.free_top;
+  const int ps = m.page_size;
+  __syncthreads();
+  int base = 0, used = 0, my_code = 0, my_item = -1, my_slot = 0;
+  for (int chunk = 0; chunk < n; chunk += blockDim.x) {
+    const int i = chunk + threadIdx.x;
+    int need = 0, slot = -1, w = 0, code = 0;
+    bool valid = false;
+    if (i < n) {
+      slot = slots[i];
+      if (slot < 0 || slot >= m.max_seqs || !m.open[slot]) code = BC_ERR_BAD_SLOT;
+      else {
+        const int c = m.c[slot], nb = m.n_beacons[slot];
+        w = m.window_len[slot];
+        if (c > 1 && w >= c) code = BC_ERR_WINDOW_FULL;
+        else if (m.max_entries > 0 && nb + w + 1 > m.max_entries) code = BC_ERR_CAPACITY;
+        else {
+          need = (w % ps == 0) ? 1 : 0;
+          const int pages = ceil_div(m.prompt_len[slot], ps) + ceil_div(nb, ps) + ceil_div(w, ps);
+          if (need && pages + 1 > m.max_pages_per_seq) { code = BC_ERR_CAPACITY; need = 0; }
+          else valid = true;
+        }
+      }
+    }
+    int total;
+    const int off = base + block_exclusive_scan(need, &total);
+    base += total;
+    int row_out = -1;
+    if (valid) {
+      if (need == 0 || off + need <= top0) {
+        int32_t* col = m.page_table + (int64_t)slot * m.max_pages_per_seq + m.window_off[slot] + w / ps;
+        if (need) { *col = m.free_stack[top0 - 1 - off]; used = max(used, off + 1); }
+        row_out = *col * ps + w % ps;
+        m.window_len[slot] = w + 1;
+        m.t[slot] += 1;
+      } else code = BC_ERR_NO_PAGES;
+    }
+    if (i < n) { dst_row[i] = row_out; dst_pos[i] = w; }
+    if (code && my_code == 0) { my_code = code; my_item = i; my_slot = slot; latch.note(i); }
+  }
+  used = __reduce_max_sync(0xffffffffu, used);
+  __shared__ int sh_used;
+  if (threadIdx.x == 0) sh_used = 0;
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) atomicMax(&sh_used, used);
+  latch.commit(m, my_item, my_code, my_slot, call);
+  __syncthreads();
+  if (threadIdx.x == 0) *m.free_top = top0 - sh_used;
+}
+
+// phase & 1: validate, allocate the beacon slot, fill dst_row/dst_pos (dst_row < 0: item failed).
+// phase & 2: for items with dst_row >= 0, push the window pages, clear the window, count the beacon.
+__global__ void __launch_bounds__(kBookThreads, 1)
+k_compress_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
+                int32_t* __restrict__ dst_row, int32_t* __restrict__ dst_pos, int phase) {
+  __shared__ int sh_first;
+  __shared__ int sh_used;
+  const int ps = m.page_size;
+  int top = *m.free_top;
+  __syncthreads();
+  if (phase & 1) {
+    ErrLatch latch; latch.init(&sh_first);
+    int base = 0, used = 0, my_code = 0, my_item = -1, my_slot = 0;
+    for (int chunk = 0; chunk < n; chunk += blockDim.x) {
+      const int i = chunk + threadIdx.x;
+      int need = 0, slot = -1, nb = 0, code = 0;
+      bool valid = false;
+      if (i < n) {
+        slot = slots[i];
+        if (slot < 0 || slot >= m.max_seqs || !m.open[slot]) code = BC_ERR_BAD_SLOT;
+        else {
+          const int c = m.c[slot];
+          nb = m.n_beacons[slot];
+          if (c <= 1 || m.window_len[slot] != c) code = BC_ERR_WINDOW_NOT_FULL;
+          else {
+            need = (nb % ps == 0) ? 1 : 0;
+            const int pages = ceil_div(m.prompt_len[slot], ps) + ceil_div(nb, ps) + ceil_div(c, ps);
+            if (need && pages + 1 > m.max_pages_per_seq) { code = BC_ERR_CAPACITY; need = 0; }
+            else valid = true;
+          }
+        }
+      }
+      int total;
+      const int off = base + block_exclusive_scan(need, &total);
+      base += total;
+      int row_out = -1;
+      if (valid) {
+        if (need == 0 || off + need <= top) {
+          int32_t* col = m.page_table + (int64_t)slot * m.max_pages_per_seq + m.beacon_off[slot] + nb / ps;
+          if (need) { *col = m.free_stack[top - 1 - off]; used = max(used, off + 1); }
+          row_out = *col * ps + nb % ps;
+        } else code = BC_ERR_NO_PAGES;
+      }
+      if (i < n) { dst_row[i] = row_out; dst_pos[i] = nb; }
+      if (code && my_code == 0) { my_code = code; my_item = i; my_slot = slot; latch.note(i); }
+    }
+    used = __reduce_max_sync(0xffffffffu, used);
+    if (threadIdx.x == 0) sh_used = 0;
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) atomicMax(&sh_used, used);
+    latch.commit(m, my_item, my_code, my_slot, call);
+    __syncthreads();
+    top -= sh_used;
+    __syncthreads();
+  }
+  if (phase & 2) {
+    int base = 0;
+    for (int chunk = 0; chunk < n; chunk += blockDim.x) {
+      const int i = chunk + threadIdx.x;
+      int cnt = 0, slot = -1;
+      if (i < n && dst_row[i] >= 0) {
+        slot = slots[i];
+        cnt = ceil_div(m.window_len[slot], ps);
+      }
+      int total;
+      const int off = base + block_exclusive_scan(cnt, &total);
+      base += total;
+      if (slot >= 0) {
+        const int32_t* col = m.page_table + (int64_t)slot * m.max_pages_per_seq + m.window_off[slot];
+        for (int k = 0; k < cnt; ++k) m.free_stack[top + off + k] = col[k];
+        m.window_len[slot] = 0;
+        m.n_beacons[slot] += 1;
+      }
+    }
+    top += base;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) *m.free_top = top;
+}
+
+__global__ void __launch_bounds__(kBookThreads, 1)
+k_close(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call) {
+  __shared__ int sh_first;
+  ErrLatch latch; latch.init(&sh_first);
+  const int ps = m.page_size;
+  const int top = *m.free_top;
+  __syncthreads();
+  int base = 0, my_code = 0, my_item = -1, my_slot = 0;
+  for (int chunk = 0; chunk < n; chunk += blockDim.x) {
+    const int i = chunk + threadIdx.x;
+    int slot = -1, np = 0, nbp = 0, nwp = 0, code = 0;
+    if (i < n) {
+      slot = slots[i];
+      if (slot < 0 || slot >= m.max_seqs || !m.open[slot]) { code = BC_ERR_BAD_SLOT; slot = -1; }
+      else {
+        np = ceil_div(m.prompt_len[slot], ps);
+        nbp = ceil_div(m.n_beacons[slot], ps);
+        nwp = ceil_div(m.window_len[slot], ps);
+      }
+    }
+    int total;
+    const int off = base + block_exclusive_scan(np + nbp + nwp, &total);
+    base += total;
+    if (slot >= 0) {
+      const int32_t* row = m.page_table + (int64_t)slot * m.max_pages_per_seq;
+      int o = top + off;
+      for (int k = 0; k < np; ++k) m.free_stack[o++] = row[k];
+      for (int k = 0; k < nbp; ++k) m.free_stack[o++] = row[m.beacon_off[slot] + k];
+      for (int k = 0; k < nwp; ++k) m.free_stack[o++] = row[m.window_off[slot] + k];
+      m.open[slot] = 0; m.prompt_len[slot] = 0; m.n_beacons[slot] = 0; m.window_len[slot] = 0;
+      m.c[slot] = 0; m.t[slot] = 0;
+    }
+    if (code && my_code == 0) { my_code = code; my_item = i; my_slot = slots[i]; latch.note(i); }
+  }
+  latch.commit(m, my_item, my_code, my_slot, call);
+  __syncthreads();
+  if (threadIdx.x == 0) *m.free_top = top + base;
+}
+
+// One block per batch item: copies the item's K and V rows (all heads) into its pool row,
+// 16 bytes per thread, applying the chunk permutation of the store layout.
+__global__ void k_write_rows(BcGeom g, uint8_t* __restrict__ pool_layer, const int32_t* __restrict__ dst_row,
+                             const int32_t* __restrict__ dst_pos, const uint8_t* __restrict__ k,
+                             const uint8_t* __restrict__ v, int n) {
+  const int i = blockIdx.x;
+  const int row = dst_row[i];
+  if (row < 0) return;
+  const int pos = dst_pos[i];
+  const int chunks_per_head = g.head_row_bytes >> 4;
+  const int per_side = g.kv_heads * chunks_per_head;
+  uint8_t* dst = pool_layer + (int64_t)row * g.entry_bytes;
+  for (int idx = threadIdx.x; idx < 2 * per_side; idx += blockDim.x) {
+    const int which = idx / per_side, rem = idx - which * per_side;
+    const int h = rem / chunks_per_head, j = rem - h * chunks_per_head;
+    const uint8_t* src = (which ? v : k) + ((int64_t)i * g.kv_heads + h) * g.head_row_bytes + (j << 4);
+    *reinterpret_cast<uint4*>(dst + bc_chunk_offset(g, which, h, j, pos)) = *reinterpret_cast<const uint4*>(src);
+  }
+}
+
+// One block per prompt token of the packed [total, kv_heads, head_dim] input.
+__global__ void k_prefill(BcMeta m, BcGeom g, uint8_t* __restrict__ pool_layer, const int32_t* __restrict__ slots,
+                          const int32_t* __restrict__ cu, int n, const uint8_t* __restrict__ k,
+                          const uint8_t* __restrict__ v) {
+  const int tok = blockIdx.x;
+  __shared__ int sh_row, sh_pos;
+  if (threadIdx.x == 0) {
+    int lo = 0, hi = n;  // largest s with cu[s] <= tok
+    while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (cu[mid] <= tok) lo = mid; else hi = mid; }
+    const int slot = slots[lo], pos = tok - cu[lo];
+    int row = -1;
+    if (slot >= 0 && slot < m.max_seqs && m.open[slot] && pos < m.prompt_len[slot]) {
+      const int page = m.page_table[(int64_t)slot * m.max_pages_per_seq + pos / g.page_size];
+      row = page * g.page_size + pos % g.page_size;
+    }
+    sh_row = row; sh_pos = pos;
+  }
+  __syncthreads();
+  const int row = sh_row, pos = sh_pos;
+  if (row < 0) return;
+  const int chunks_per_head = g.head_row_bytes >> 4;
+  const int per_side = g.kv_heads * chunks_per_head;
+  uint8_t* dst = pool_layer + (int64_t)row * g.entry_bytes;
+  for (int idx = threadIdx.x; idx < 2 * per_side; idx += blockDim.x) {
+    const int which = idx / per_side, rem = idx - which * per_side;
+    const int h = rem / chunks_per_head, j = rem - h * chunks_per_head;
+    const uint8_t* src = (which ? v : k) + ((int64_t)tok * g.kv_heads + h) * g.head_row_bytes + (j << 4);
+    *reinterpret_cast<uint4*>(dst + bc_chunk_offset(g, which, h, j, pos)) = *reinterpret_cast<const uint4*>(src);
+  }
+}
+
+// One block per exported entry, logical order prompt | beacons | window.
+__global__ void k_export(BcMeta m, BcGeom g, const uint8_t* __restrict__ pool_layer, int slot,
+                         uint8_t* __restrict__ k_out, uint8_t* __restrict__ v_out, int capacity) {
+  const int e = blockIdx.x;
+  if (slot < 0 || slot >= m.max_seqs || !m.open[slot]) return;
+  const int P = m.prompt_len[slot], nb = m.n_beacons[slot], w = m.window_len[slot];
+  if (e >= capacity || e >= P + nb + w) return;
+  int pos, col0;
+  if (e < P) { pos = e; col0 = 0; }
+  else if (e < P + nb) { pos = e - P; col0 = m.beacon_off[slot]; }
+  else { pos = e - P - nb; col0 = m.window_off[slot]; }
+  const int page = m.page_table[(int64_t)slot * m.max_pages_per_seq + col0 + pos / g.page_size];
+  const uint8_t* src = pool_layer + ((int64_t)page * g.page_size + pos % g.page_size) * g.entry_bytes;
+  const int chunks_per_head = g.head_row_bytes >> 4;
+  const int per_side = g.kv_heads * chunks_per_head;
+  for (int idx = threadIdx.x; idx < 2 * per_side; idx += blockDim.x) {
+    const int which = idx / per_side, rem = idx - which * per_side;
+    const int h = rem / chunks_per_head, j = rem - h * chunks_per_head;
+    uint8_t* dst = (which ? v_out : k_out) + ((int64_t)e * g.kv_heads + h) * g.head_row_bytes + (j << 4);
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src + bc_chunk_offset(g, which, h, j, pos));
+  }
+}
+
+inline int copy_threads(const BcGeom& g) {
+  int t = g.entry_bytes >> 4;
+  return t < 32 ? 32 : (t > 256 ? 256 : t);
+}
+
+}  // namespace
+
+cudaError_t bc_launch_init(const BcMeta& m, cudaStream_t s) {
+  k_init<<<64, 256, 0, s>>>(m);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_open(const BcMeta& m, const int32_t* slots, const int32_t* plens, const int32_t* cs, int n,
+                           int64_t call, cudaStream_t s) {
+  k_open<<<1, kBookThreads, 0, s>>>(m, slots, plens, cs, n, call);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
+                                  int32_t* dst_pos, cudaStream_t s) {
+  k_append_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
+                                    int32_t* dst_pos, int phase, cudaStream_t s) {
+  k_compress_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, phase);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_t call, cudaStream_t s) {
+  k_close<<<1, kBookThreads, 0, s>>>(m, slots, n, call);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_write_rows(const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
+                                 const void* k, const void* v, int n, cudaStream_t s) {
+  k_write_rows<<<n, copy_threads(g), 0, s>>>(g, pool_layer, dst_row, dst_pos, (const uint8_t*)k, (const uint8_t*)v, n);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_prefill(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* slots,
+                              const int32_t* cu, int n, int total, const void* k, const void* v, cudaStream_t s) {
+  if (total == 0) return cudaSuccess;
+  k_prefill<<<total, copy_threads(g), 0, s>>>(m, g, pool_layer, slots, cu, n, (const uint8_t*)k, (const uint8_t*)v);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_export(const BcMeta& m, const BcGeom& g, const uint8_t* pool_layer, int slot, void* k_out,
+                             void* v_out, int capacity, cudaStream_t s) {
+  if (capacity <= 0) return cudaSuccess;
+  k_export<<<capacity, copy_threads(g), 0, s>>>(m, g, pool_layer, slot, (uint8_t*)k_out, (uint8_t*)v_out, capacity);
+  return cudaGetLastError();
+}

@@ -1,0 +1,87 @@
+// Shared declarations of the breadcrumbs library: device-side views of the bookkeeping, the
+// store layout helpers and the kernel launch wrappers implemented in the .cu files.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "breadcrumbs.h"
+
+// Upper bounds the workspace is sized for.
+#define BC_MAX_ATTN_CTAS 304   // thread blocks of the decode-attention kernel
+#define BC_MAX_ATTN_BATCH 512  // sequences per bc_decode_attn call
+#define BC_MERGE_ELEMS 4096    // q_heads * head_dim that fits the in-block merge buffer
+
+// Device view of the bookkeeping ("meta" buffer).  All arrays are int32.
+struct BcMeta {
+  int32_t* status;      // [0] code, [1] slot, [2..3] call index (int64)
+  int32_t* free_top;    // number of free pages
+  int32_t* free_stack;  // [num_pages]; free_stack[top-1] is handed out next
+  int32_t* open;        // [max_seqs] 1 = open
+  int32_t* prompt_len;  // [max_seqs]
+  int32_t* n_beacons;   // [max_seqs]
+  int32_t* window_len;  // [max_seqs]
+  int32_t* c;           // [max_seqs]
+  int32_t* t;           // [max_seqs] generated entries appended so far
+  int32_t* window_off;  // [max_seqs] column of the first window page in the page-table row
+  int32_t* beacon_off;  // [max_seqs] column of the first beacon page
+  int32_t* page_table;  // [max_seqs][max_pages_per_seq]: prompt pages from column 0
+  int32_t max_seqs, num_pages, max_pages_per_seq, max_entries, page_size, c_default;
+};
+
+// Geometry of the K/V pool for one cache.
+struct BcGeom {
+  int32_t kv_heads, q_heads, head_dim, page_size;
+  int32_t entry_bytes;       // E = 2 * kv_heads * head_dim * 2
+  int32_t head_row_bytes;    // head_dim * 2
+  int64_t layer_bytes;       // num_pages * page_size * E
+};
+
+// Byte offset, inside one entry, of 16-byte chunk j of (K|V = which, head h) for an entry whose
+// position inside its segment is pos: the chunk index is XOR-permuted with pos & 7.
+__host__ __device__ __forceinline__ int bc_chunk_offset(const BcGeom& g, int which, int h, int j, int pos) {
+  return (which * g.kv_heads + h) * g.head_row_bytes + ((j ^ (pos & 7)) << 4);
+}
+
+// ---- launch wrappers (bc_book.cu) ------------------------------------------------------------
+cudaError_t bc_launch_init(const BcMeta& m, cudaStream_t s);
+cudaError_t bc_launch_open(const BcMeta& m, const int32_t* slots, const int32_t* plens, const int32_t* cs,
+                           int n, int64_t call, cudaStream_t s);
+cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
+                                  int32_t* dst_pos, cudaStream_t s);
+// phase bit 1: allocate the beacon slot; phase bit 2: evict the window and bump the counters
+cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
+                                    int32_t* dst_pos, int phase, cudaStream_t s);
+cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_t call, cudaStream_t s);
+cudaError_t bc_launch_write_rows(const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
+                                 const void* k, const void* v, int n, cudaStream_t s);
+cudaError_t bc_launch_prefill(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* slots,
+                              const int32_t* cu, int n, int total, const void* k, const void* v, cudaStream_t s);
+cudaError_t bc_launch_export(const BcMeta& m, const BcGeom& g, const uint8_t* pool_layer, int slot, void* k_out,
+                             void* v_out, int capacity, cudaStream_t s);
+
+// ---- attention (bc_attn.cu) ----------------------------------------------------------------------
+struct BcAttnArgs {
+  const uint8_t* pool_layer;
+  const int32_t* slots;
+  int32_t n;
+  const void* q;
+  void* out;
+  int32_t out_f32;
+  const void* extra_k;
+  const void* extra_v;
+  float sm_scale;
+  float* part_o;         // [(ctas + n)][q_heads][head_dim]
+  float* part_ml;        // [(ctas + n)][q_heads][2]
+  int32_t* first_cta;    // [n]
+  int32_t* last_cta;     // [n]
+  int32_t ctas;
+};
+// Configures the kernels once per process/device (shared-memory opt-in).  Returns the SM count.
+cudaError_t bc_attn_setup(int* sm_count);
+// Launches the pipelined decode-attention kernel and the split combine; *launches gets the count.
+cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, cudaStream_t s,
+                           cudaEvent_t ev_start, cudaEvent_t ev_stop, int* launches);
+// Slow device reference (one warp per query head).
+cudaError_t bc_launch_attn_reference(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, cudaStream_t s);

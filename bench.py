@@ -1,0 +1,481 @@
+#!/usr/bin/env python
+"""Benchmark of the Breadcrumbs decode hot path on B200.
+
+Workload (benchmark configs[2], the compression-ratio sweep): one layer, batch 64, 32 query /
+8 KV heads, head_dim 128, bf16, prompt 512, 16384 decode steps, c in {2,4,8,16,32} with
+page_size = c, plus the uncompressed run (c = 1, page 16) as a reported row.
+
+One "step" of the JSON line = one decode step (bc_append + bc_decode_attn, and when the window
+fills the beacon-query attention + bc_compress) at EACH of the five compressed ratios, i.e. 5 x 64
+generated tokens.  The ratios are timed one after the other, K steps each, centred on the middle
+of the 16384-step generation (cache length grows linearly with t, so the mean over a window centred
+on the midpoint equals the mean over the whole run).  `value` = tokens / second over all of that.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+RATIOS = (2, 4, 8, 16, 32)
+METRIC = "decode tokens/s (and KV-read HBM GB/s) over the compression-ratio sweep c in {2,4,8,16,32}"
+
+
+# ------------------------------------------------------------------------------ accounting
+def entries_attended(P, n, c):
+    """Cache entries the n-th generated token's query reads (its own entry included)."""
+    if c <= 1:
+        return P + n
+    return P + (n - 1) // c + (n - 1) % c + 1
+
+
+def entries_beacon_query(P, t, c):
+    """Stored entries the beacon query reads when the window fills at t (t % c == 0)."""
+    return P + (t // c - 1) + c
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+# ------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc, self.index = None, index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ one ratio on the GPU
+class RatioRunner:
+    """Holds one cache (batch B at ratio c) and drives decode steps through the C ABI."""
+
+    def __init__(self, w, device, seed_offset=0):
+        import torch
+        from paper_2510_13797_b200 import binding as B
+        from paper_2510_13797_b200.workloads import InputStream
+        self.torch, self.B, self.w, self.dev = torch, B, w, device
+        c, ps, Bn = w.cs[0], w.page_size, w.batch
+        P, T = w.prompt_lens[0], w.steps
+        self.c, self.P, self.T, self.n = c, P, T, Bn
+        cd = lambda a, b: -(-a // b)
+        if c > 1:
+            pages_per_seq = cd(P, ps) + cd(c, ps) + cd(cd(T, c), ps) + 1
+        else:
+            pages_per_seq = cd(P + T, ps) + 1
+        self.cache = B.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, c, ps, max_seqs=Bn,
+                             num_pages=Bn * pages_per_seq, max_pages_per_seq=pages_per_seq, device=device)
+        self.slots = torch.arange(Bn, dtype=torch.int32, device=device)
+        self.plens = torch.tensor(w.prompt_lens, dtype=torch.int32, device=device)
+        self.cu = torch.tensor([0] + list(__import__("itertools").accumulate(w.prompt_lens)), dtype=torch.int32,
+                               device=device)
+        stream = InputStream(w, device)
+        self.pk, self.pv = stream.prompt_kv(0)
+        self.ring = max(c, 16)                         # distinct step inputs, reused cyclically
+        self.q, self.k, self.v = stream.step_chunk(0, seed_offset, self.ring)
+        self.bq, self.bk, self.bv = stream.beacon_chunk(0, seed_offset, 4)
+        self.out = self.cache.new_out(Bn)
+        self.out_b = self.cache.new_out(Bn)
+        self.t = 0
+        self.opened = False
+        # pinned host copies for the end-to-end pass
+        self.h = None
+
+    # -- state -------------------------------------------------------------------------------
+    def reset_to(self, t_target):
+        """(Re)opens the batch, stores the prompts and replays appends/compressions up to t_target."""
+        c = self.cache
+        if self.opened:
+            c.bc_seq_close(self.slots)
+        c.bc_seq_open(self.slots, self.plens)
+        c.bc_prefill(0, self.slots, self.cu, int(self.cu[-1]), self.pk, self.pv)
+        self.opened, self.t = True, 0
+        while self.t < t_target:
+            j = self.t % self.ring
+            c.bc_append(0, self.slots, self.k[j], self.v[j])
+            self.t += 1
+            if self.c > 1 and self.t % self.c == 0:
+                b = (self.t // self.c) % 4
+                c.bc_compress(0, self.slots, self.bk[b], self.bv[b])
+
+    def step(self):
+        """One decode step of the whole batch through the device-pointer calls."""
+        c, j = self.cache, self.t % self.ring
+        c.bc_append(0, self.slots, self.k[j], self.v[j])
+        c.bc_decode_attn(0, self.slots, self.q[j], self.out, self.w.sm_scale)
+        self.t += 1
+        if self.c > 1 and self.t % self.c == 0:
+            b = (self.t // self.c) % 4
+            c.bc_decode_attn(0, self.slots, self.bq[b], self.out_b, self.w.sm_scale, self.bk[b], self.bv[b])
+            c.bc_compress(0, self.slots, self.bk[b], self.bv[b])
+
+    def step_host(self):
+        """The same step through the host-buffer entry points (H2D of q,k,v and D2H of out inside)."""
+        if self.h is None:
+            pin = lambda t: t.cpu().pin_memory()
+            self.h = dict(q=pin(self.q), k=pin(self.k), v=pin(self.v), bq=pin(self.bq), bk=pin(self.bk),
+                          bv=pin(self.bv), out=pin(self.out), out_b=pin(self.out_b))
+        c, j, h = self.cache, self.t % self.ring, self.h
+        c.bc_decode_step_host(0, self.slots, h["q"][j], h["k"][j], h["v"][j], h["out"], self.w.sm_scale)
+        self.t += 1
+        if self.c > 1 and self.t % self.c == 0:
+            b = (self.t // self.c) % 4
+            c.bc_compress_step_host(0, self.slots, h["bq"][b], h["bk"][b], h["bv"][b], h["out_b"], self.w.sm_scale)
+
+    def host_bytes_per_step(self):
+        w = self.w
+        qb = self.n * w.q_heads * w.head_dim * 2
+        kb = self.n * w.kv_heads * w.head_dim * 2
+        per_beacon = 1.0 / self.c if self.c > 1 else 0.0
+        return (qb + 2 * kb) * (1 + per_beacon), qb * (1 + per_beacon)
+
+    # -- accounting ------------------------------------------------------------------------------
+    def kv_bytes(self, t_from, steps):
+        """Algorithmic KV bytes read by the attention launches of steps t_from+1 .. t_from+steps:
+        (regular launches, beacon-query launches)."""
+        E = self.w.entry_bytes
+        reg = sum(entries_attended(self.P, n, self.c) for n in range(t_from + 1, t_from + steps + 1))
+        bea = sum(entries_beacon_query(self.P, n, self.c) for n in range(t_from + 1, t_from + steps + 1)
+                  if self.c > 1 and n % self.c == 0)
+        return reg * E * self.n, bea * E * self.n
+
+    def cache_bytes(self, t):
+        E = self.w.entry_bytes
+        live = self.P + (t // self.c + t % self.c if self.c > 1 else t)
+        return live * E * self.n, (self.P + t) * E * self.n
+
+    # -- timed passes ------------------------------------------------------------------------------
+    def timed_graph(self, K, W):
+        """W warm-up steps, then exactly K steps timed with CUDA events.  Whole windows of c steps run
+        as replays of one captured CUDA graph; a remainder (K % c) runs as plain launches."""
+        torch = self.torch
+        cyc = self.c if self.c > 1 else 16
+        while W > 0 or self.t % cyc:
+            self.step(); W -= 1
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        l0 = self.cache.bc_kernel_launches()
+        t_save = self.t
+        with torch.cuda.graph(graph, stream=s, capture_error_mode="thread_local"):
+            for _ in range(cyc):
+                self.step()
+        per_graph = self.cache.bc_kernel_launches() - l0
+        self.t = t_save                                   # capture enqueued nothing
+        torch.cuda.current_stream().wait_stream(s)
+        graph.replay(); self.t += cyc                     # warm the instantiated graph
+        torch.cuda.synchronize()
+        t_begin = self.t
+        reps, rem = divmod(K, cyc)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        l1 = self.cache.bc_kernel_launches()
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        self.t += reps * cyc
+        for _ in range(rem):
+            self.step()
+        e1.record()
+        torch.cuda.synchronize()
+        launches = reps * per_graph + (self.cache.bc_kernel_launches() - l1)
+        return e0.elapsed_time(e1), t_begin, launches
+
+    def timed_kernels(self, K, W):
+        """K steps with plain launches; every decode-attention kernel is bracketed by CUDA events on the
+        launching stream.  Returns (sum of kernel ms, launches, algorithmic bytes, whole-region ms)."""
+        torch = self.torch
+        for _ in range(W):
+            self.step()
+        torch.cuda.synchronize()
+        t_begin = self.t
+        n_launch = K + (sum(1 for n in range(t_begin + 1, t_begin + K + 1) if n % self.c == 0) if self.c > 1 else 0)
+        self.cache.bc_profile_enable(n_launch)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K):
+            self.step()
+        e1.record()
+        torch.cuda.synchronize()
+        got, ms = self.cache.bc_profile_read()
+        assert got == n_launch, (got, n_launch)
+        reg, bea = self.kv_bytes(t_begin, K)
+        return ms, got, reg + bea, e0.elapsed_time(e1)
+
+    def timed_host(self, K, W):
+        torch = self.torch
+        for _ in range(W):
+            self.step_host()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K):
+            self.step_host()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    def check_error(self):
+        code, slot, call = self.cache.bc_poll_error()
+        if code != 0:
+            raise RuntimeError(f"device-side error {self.B.STATUS_NAMES.get(code, code)} slot {slot} call {call}")
+
+
+# ------------------------------------------------------------------------------ the oracle on host cores
+def oracle_sample(w, t_mid, seqs, steps, seed=0):
+    """Times the CPU oracle, as it stands, on `steps` decode steps of `seqs` sequences whose caches
+    are at generation step t_mid.  Returns (seconds, tokens processed, cpu seconds)."""
+    import numpy as np
+    import psutil
+    from oracle.breadcrumbs_oracle import SeqCache
+    rng = np.random.RandomState(seed)
+    c, P = w.cs[0], w.prompt_lens[0]
+    Hkv, Hq, D = w.kv_heads, w.q_heads, w.head_dim
+    t0 = (t_mid // c) * c if c > 1 else t_mid
+    caches = []
+    for _ in range(seqs):
+        s = SeqCache(1, c)
+        s.prefill(0, rng.standard_normal((P, Hkv, D)), rng.standard_normal((P, Hkv, D)))
+        nb = t0 // c if c > 1 else 0
+        for m in range(nb):                     # beacons are inputs: the state at t0 is built directly
+            s.cache[0].append(("beacon", m + 1, rng.standard_normal((Hkv, D)), rng.standard_normal((Hkv, D))))
+        if c <= 1:
+            for i in range(t0):
+                s.cache[0].append(("token", i, rng.standard_normal((Hkv, D)), rng.standard_normal((Hkv, D))))
+        caches.append(s)
+    proc = psutil.Process()
+    cpu0, t_start = proc.cpu_times(), time.perf_counter()
+    for _ in range(steps):
+        for s in caches:
+            s.append(0, rng.standard_normal((Hkv, D)), rng.standard_normal((Hkv, D)))
+            s.attend(0, rng.standard_normal((Hq, D)), w.sm_scale)
+            if c > 1 and s.window_len(0) == c:
+                bk, bv = rng.standard_normal((Hkv, D)), rng.standard_normal((Hkv, D))
+                s.beacon_attend(0, rng.standard_normal((Hq, D)), bk, bv, w.sm_scale)
+                s.compress(0, bk, bv)
+    wall = time.perf_counter() - t_start
+    cpu1 = proc.cpu_times()
+    cpu = (cpu1.user - cpu0.user) + (cpu1.system - cpu0.system)
+    return wall, seqs * steps, cpu
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle timed on this machine's host cores, same workload and metric.
+    Each step decodes a bounded sample of the batch at every ratio."""
+    from paper_2510_13797_b200.workloads import make_workload
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    K, W = args.steps, args.warmup
+    T = make_workload("sweep", c=16).steps
+    budget = 150.0 / max(K + W, 1)                   # seconds per step over the five ratios
+    probe = {}
+    for c in RATIOS:
+        w = make_workload("sweep", c=c)
+        wall, _, _ = oracle_sample(w, T // 2, 1, 1)
+        probe[c] = wall
+    seqs = int(max(1, min(64, budget / max(sum(probe.values()), 1e-9))))
+    total_wall = total_tok = total_cpu = 0.0
+    for c in RATIOS:
+        w = make_workload("sweep", c=c)
+        oracle_sample(w, T // 2, seqs, max(W, 0))
+        wall, tok, cpu = oracle_sample(w, T // 2, seqs, K)
+        total_wall += wall; total_tok += tok; total_cpu += cpu
+    value = total_tok / total_wall
+    cores = max(1, round(total_cpu / total_wall))
+    sample = f"{seqs} of 64 sequences per ratio, {K} decode steps at the mid-generation cache state, c in {list(RATIOS)}"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": 0, "steps": K,
+        "warmup": W, "ms_per_step": 1e3 * total_wall / K, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "sweep: B=64, 32/8 heads, D=128, P=512, T=16384, c in {2,4,8,16,32} (CPU oracle on a sample)"},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------ main arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=512)
+    ap.add_argument("--warmup", type=int, default=32)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ratios", default="")
+    ap.add_argument("--skip-uncompressed", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2510_13797_b200.workloads import make_workload
+
+    K, W = args.steps, max(args.warmup, 3)
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    ratios = tuple(int(x) for x in args.ratios.split(",")) if args.ratios else RATIOS
+    peak, peak_src = load_peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    rows, total_ms, total_launches = [], 0.0, 0
+    kern_ms = kern_bytes = kern_launches = 0.0
+    e2e_ms = 0.0
+    h2d = d2h = 0.0
+    sampler = ClockSampler(local)
+    sweep = list(ratios) + ([] if args.skip_uncompressed else [1])
+    barrier()
+    sampler.start()
+    for c in sweep:
+        w = make_workload("sweep", c=c)
+        T = w.steps
+        r = RatioRunner(w, dev, seed_offset=rank)
+        cyc = c if c > 1 else 16
+        t_mid = max(0, ((T - K) // 2 // cyc) * cyc)
+        # pass A: device-resident inputs, CUDA-graph replays: the headline time
+        r.reset_to(max(0, t_mid - W - cyc))
+        barrier()
+        ms, t_begin, launches = r.timed_graph(K, max(W, t_mid - r.t - cyc))
+        # pass B: plain launches, every attention kernel bracketed by events: the roofline figures
+        Kp = min(K, 256)
+        r.reset_to(max(0, t_mid - W))
+        k_ms, k_n, k_bytes, plain_ms = r.timed_kernels(Kp, W)
+        # pass C: host buffers through the C ABI, copies inside the timed region
+        r.reset_to(max(0, t_mid - W))
+        barrier()
+        h_ms = r.timed_host(K, W)
+        r.check_error()
+        if world > 1:
+            tt = torch.tensor([ms, h_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            ms, h_ms = float(tt[0]), float(tt[1])
+        reg, bea = r.kv_bytes(t_begin, K)
+        live, unc = r.cache_bytes(t_begin + K // 2)
+        end_live, end_unc = r.cache_bytes(T)
+        row = {
+            "c": c, "page_size": w.page_size, "ms_per_step": ms / K, "tokens_per_s": world * w.batch * K / (ms * 1e-3),
+            "e2e_tokens_per_s": world * w.batch * K / (h_ms * 1e-3),
+            "plain_launch_ms_per_step": plain_ms / Kp,
+            "kv_gbs_step": (reg + bea) / (ms * 1e-3) / 1e9,
+            "attn_kernel_us": 1e3 * k_ms / k_n, "attn_kernel_gbs": k_bytes / (k_ms * 1e-3) / 1e9,
+            "attn_frac_of_peak": k_bytes / (k_ms * 1e-3) / 1e9 / peak,
+            "attn_pct_of_8tbs": 100 * k_bytes / (k_ms * 1e-3) / 8e12,
+            "kv_bytes_per_step": (reg + bea) / K, "cache_bytes_mid": live, "uncompressed_bytes_mid": unc,
+            "cache_bytes_end": end_live, "uncompressed_bytes_end": end_unc,
+            "t_window": [t_begin, t_begin + K],
+        }
+        rows.append(row)
+        if c > 1:
+            total_ms += ms; total_launches += launches
+            kern_ms += k_ms; kern_bytes += k_bytes; kern_launches += k_n
+            e2e_ms += h_ms
+            a, b = r.host_bytes_per_step()
+            h2d += a; d2h += b
+        del r
+        torch.cuda.empty_cache()
+    barrier()
+    clocks = sampler.stop()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    n_c = sum(1 for c in sweep if c > 1)
+    B = 64
+    value = world * B * n_c * K / (total_ms * 1e-3)
+    achieved = kern_bytes / (kern_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "sweep: 1 layer, B=64 per ratio, 32/8 heads, D=128, P=512, T=16384, "
+                               "c in {2,4,8,16,32}, page_size=c; one step = one decode step at each ratio, "
+                               "timed ratio by ratio around mid-generation",
+                   "l2": "inputs larger than L2: every step streams 206 MB (c=32) to 1.2 GB (c=2) of KV, L2 is 126 MB",
+                   "launch": "CUDA-graph replay of whole windows of c steps", "per_gpu_batch": B * n_c},
+        "e2e": {"value": world * B * n_c * K / (e2e_ms * 1e-3), "unit": "tokens/s",
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(total_launches),
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "k_attn_pipe", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                     "launches_timed": int(kern_launches),
+                     "min_frac_over_c": min(r["attn_frac_of_peak"] for r in rows if r["c"] > 1),
+                     "pct_of_8tbs": 100 * achieved * 1e9 / 8e12},
+        "sweep": rows,
+    }
+    if not args.no_cpu_baseline:
+        w = make_workload("sweep", c=16)
+        wall, tok, cpu = oracle_sample(w, w.steps // 2, 16, 8)
+        line["cpu_baseline"] = {"value": tok / wall, "unit": "tokens/s", "cores": max(1, round(cpu / wall)),
+                                "kind": "oracle",
+                                "sample": "16 of 64 sequences, 8 decode steps at c=16, cache at generation step 8192"}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

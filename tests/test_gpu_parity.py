@@ -215,6 +215,7 @@ def test_device_side_errors_match_the_model():
     kv = lambda n: (randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV))
     # 3 + 2 pages granted, the third sequence (2 pages) does not fit, the empty one always fits
     assert pair.open([0, 1, 2, 3], [5, 3, 4, 0], [2, 2, 2, 2]) == ["OK", "OK", "NO_PAGES", "OK"]
+    pair.prefill(0, [0, 1, 3], [5, 3, 0], *kv(8))
     pair.check_state()
     pair.gpu.bc_clear_error()
     pair.model.first_error = None

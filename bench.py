@@ -219,6 +219,7 @@ class RatioRunner:
         reps, rem = divmod(K, cyc)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         l1 = self.cache.bc_kernel_launches()
+        torch.cuda.nvtx.range_push("timed")
         e0.record()
         for _ in range(reps):
             graph.replay()
@@ -227,6 +228,7 @@ class RatioRunner:
             self.step()
         e1.record()
         torch.cuda.synchronize()
+        torch.cuda.nvtx.range_pop()
         launches = reps * per_graph + (self.cache.bc_kernel_launches() - l1)
         return e0.elapsed_time(e1), t_begin, launches
 
@@ -241,11 +243,13 @@ class RatioRunner:
         n_launch = K + (sum(1 for n in range(t_begin + 1, t_begin + K + 1) if n % self.c == 0) if self.c > 1 else 0)
         self.cache.bc_profile_enable(n_launch)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.nvtx.range_push("kernels")
         e0.record()
         for _ in range(K):
             self.step()
         e1.record()
         torch.cuda.synchronize()
+        torch.cuda.nvtx.range_pop()
         got, ms = self.cache.bc_profile_read()
         assert got == n_launch, (got, n_launch)
         reg, bea = self.kv_bytes(t_begin, K)
@@ -345,6 +349,25 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_profile_case(args):
+    """A few plain decode steps at one ratio on a cache whose prompt is as long as the sweep's
+    mid-generation cache (same bytes per launch, same page granularity, few launches before them)."""
+    import torch
+    from paper_2510_13797_b200.workloads import make_workload
+    c = args.profile_case
+    w = make_workload("sweep", c=c)
+    mid = entries_attended(w.prompt_lens[0], w.steps // 2, c)
+    w = make_workload("sweep", c=c, prompt_lens=[mid] * w.batch, gen_lens=[4 * max(c, 16) + args.steps + 64] * w.batch)
+    torch.cuda.set_device(0)
+    r = RatioRunner(w, torch.device("cuda", 0))
+    r.reset_to(0)
+    ms, n, nbytes, region = r.timed_kernels(args.steps, max(args.warmup, 3))
+    r.check_error()
+    print(json.dumps({"profile_case": c, "prompt": mid, "steps": args.steps, "attn_launches": n,
+                      "attn_kernel_us": 1e3 * ms / n, "attn_kernel_gbs": nbytes / (ms * 1e-3) / 1e9,
+                      "kv_bytes_per_launch": nbytes / n, "plain_ms_per_step": region / args.steps}))
+
+
 # ------------------------------------------------------------------------------ main arm
 def main():
     ap = argparse.ArgumentParser()
@@ -355,9 +378,14 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
+    ap.add_argument("--profile-case", type=int, default=0, metavar="C",
+                    help="small case for profilers: ratio C with a prompt as long as the mid-generation cache, "
+                         "--steps plain decode steps, no fast-forward, no graphs")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.profile_case:
+        return run_profile_case(args)
 
     import torch
     import torch.distributed as dist

@@ -74,7 +74,8 @@ enum {
   BC_ERR_ORDER = -7,           /* per-layer calls out of order */
   BC_ERR_CUDA = -8,            /* a CUDA runtime call failed; see bc_last_cuda_error */
   BC_ERR_UNSUPPORTED = -9,     /* shape outside what the kernels are built for */
-  BC_ERR_TIMEOUT = -10         /* a bounded device-side wait gave up (kernel returned early) */
+  BC_ERR_TIMEOUT = -10,        /* a bounded device-side wait gave up (kernel returned early) */
+  BC_ERR_TOO_LARGE = -11       /* bc_decode_attn_static: the call does not fit the built-in scratch */
 };
 
 enum {
@@ -160,6 +161,39 @@ BC_API bc_status bc_append(bc_cache* cache, int32_t layer, const int32_t* slots,
 BC_API bc_status bc_decode_attn(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                          const void* q, void* out, float sm_scale, const void* extra_k,
                          const void* extra_v, void* stream);
+
+/* Limits of bc_decode_attn_static. */
+#define BC_STATIC_MAX_BATCH 128   /* sequences per call */
+#define BC_STATIC_MAX_CTAS 160    /* thread blocks it will use at most */
+
+/* bc_decode_attn for callers that cannot hand the library a workspace carved from freshly
+ * allocated device memory.  (The paper has no counterpart to this call; it computes exactly what
+ * bc_decode_attn computes.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- a memory-budgeted serving
+ * process whose allocator is frozen once start-up is over, a plug-in that is only handed tensors
+ * and a stream by its host application and must not go to the CUDA allocator behind the host's
+ * back, or a latency-critical loop in which an allocation (which may synchronise the device) is not
+ * acceptable.  Such callers already own the cache buffers, but the split-K
+ * scratch (per-piece partial outputs, their running max and sum, and the first/last block of every
+ * sequence) has to live somewhere.  Here it lives in a fixed array inside the library image:
+ * about 4.9 MB of device memory that every GPU which loads the library keeps until the process
+ * exits.  The call itself performs no device or host allocation and calls no allocating routine.
+ *
+ * Arguments, layouts, results and error behaviour are those of bc_decode_attn, with these limits:
+ * n <= BC_STATIC_MAX_BATCH, at most BC_STATIC_MAX_CTAS thread blocks (fewer SMs are used on a
+ * larger part), q_heads * head_dim <= 4096.  A call beyond them returns BC_ERR_TOO_LARGE and
+ * enqueues nothing.  The cache's own `workspace` is not touched.
+ *
+ * The first call on each device looks up the device address of the built-in array (once per
+ * device, with that device current); make that first call outside any stream capture.  All calls,
+ * from all caches and streams of the process, share the one array: it still holds the previous
+ * call's partials when the next call starts (every element a call reads it has written first, so
+ * nothing needs clearing), and two calls whose kernels overlap on the GPU race on it.  Issue them
+ * on one stream, or order them with events. */
+BC_API bc_status bc_decode_attn_static(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
+                                       const void* q, void* out, float sm_scale, const void* extra_k,
+                                       const void* extra_v, void* stream);
 
 /* Algorithm 1, the eviction statement (keep everything but the c entries before the beacon, then
  * the beacon): for each of n sequences whose window holds exactly c entries, stores the beacon's

@@ -19,11 +19,11 @@ from . import build as _build
 BC_OK = 0
 BC_ERR_INVALID_ARG, BC_ERR_BAD_SLOT, BC_ERR_NO_PAGES, BC_ERR_CAPACITY = -1, -2, -3, -4
 BC_ERR_WINDOW_NOT_FULL, BC_ERR_WINDOW_FULL, BC_ERR_ORDER, BC_ERR_CUDA = -5, -6, -7, -8
-BC_ERR_UNSUPPORTED, BC_ERR_TIMEOUT = -9, -10
+BC_ERR_UNSUPPORTED, BC_ERR_TIMEOUT, BC_ERR_TOO_LARGE = -9, -10, -11
 BC_FLAG_OUT_F32, BC_FLAG_ATTN_REFERENCE = 1, 2
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SLOT", -3: "NO_PAGES", -4: "CAPACITY",
                 -5: "WINDOW_NOT_FULL", -6: "WINDOW_FULL", -7: "ORDER", -8: "CUDA",
-                -9: "UNSUPPORTED", -10: "TIMEOUT"}
+                -9: "UNSUPPORTED", -10: "TIMEOUT", -11: "TOO_LARGE"}
 
 
 class BcConfig(C.Structure):
@@ -57,6 +57,7 @@ SYMBOLS = {
     "bc_prefill": (_I32, [_P, _I32, _P, _P, _I32, _I32, _P, _P, _P]),
     "bc_append": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
     "bc_decode_attn": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
+    "bc_decode_attn_static": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
     "bc_compress": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
     "bc_seq_close": (_I32, [_P, _P, _I32, _P]),
     "bc_decode_step_host": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P]),
@@ -150,6 +151,13 @@ class Cache:
     def bc_decode_attn(self, layer, slots, q, out, sm_scale, extra_k=None, extra_v=None, stream=None):
         _check(lib().bc_decode_attn(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(out), sm_scale,
                                     _ptr(extra_k), _ptr(extra_v), _stream(stream)), "bc_decode_attn")
+
+    def bc_decode_attn_static(self, layer, slots, q, out, sm_scale, extra_k=None, extra_v=None, stream=None):
+        """bc_decode_attn with the split-K scratch taken from the array built into the library, for callers
+        that may not allocate device memory.  At most 128 sequences per call; calls share the scratch."""
+        _check(lib().bc_decode_attn_static(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(out),
+                                           sm_scale, _ptr(extra_k), _ptr(extra_v), _stream(stream)),
+               "bc_decode_attn_static")
 
     def bc_compress(self, layer, slots, beacon_k, beacon_v, stream=None):
         _check(lib().bc_compress(self.handle, layer, _ptr(slots), slots.numel(), _ptr(beacon_k), _ptr(beacon_v),

@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -159,6 +160,7 @@ const char* bc_status_string(bc_status s) {
     case BC_ERR_CUDA: return "BC_ERR_CUDA";
     case BC_ERR_UNSUPPORTED: return "BC_ERR_UNSUPPORTED";
     case BC_ERR_TIMEOUT: return "BC_ERR_TIMEOUT";
+    case BC_ERR_TOO_LARGE: return "BC_ERR_TOO_LARGE";
     default: return "BC_ERR_UNKNOWN";
   }
 }
@@ -443,6 +445,73 @@ bc_status bc_profile_read(bc_cache* c, int32_t* launches, float* total_ms) {
   *total_ms = sum;
   c->prof_cap = 0;
   c->prof_used = 0;
+  return BC_OK;
+}
+
+// ---- bc_decode_attn_static: split-K scratch inside the library image -------------------------------
+//
+// Layout of the built-in array: partial outputs [pieces][4096] fp32, then (max, sum) pairs
+// [pieces][64][2] fp32, then first/last block per sequence, 2 x [BC_STATIC_MAX_BATCH] int32,
+// with pieces = BC_STATIC_MAX_CTAS + BC_STATIC_MAX_BATCH.
+namespace {
+constexpr size_t kStaticPieces = BC_STATIC_MAX_CTAS + BC_STATIC_MAX_BATCH;
+constexpr size_t kStaticPartO = kStaticPieces * BC_MERGE_ELEMS * sizeof(float);
+constexpr size_t kStaticPartMl = kStaticPieces * 64 * 2 * sizeof(float);
+constexpr size_t kStaticIdx = 2 * BC_STATIC_MAX_BATCH * sizeof(int32_t);
+constexpr size_t kStaticBytes = kStaticPartO + kStaticPartMl + kStaticIdx;
+constexpr int kMaxDevices = 64;
+}  // namespace
+
+// In host code this name is only a handle for the runtime's symbol lookup, never a device address.
+static __device__ __align__(256) unsigned char bc_static_scratch[kStaticBytes];
+
+namespace {
+std::mutex g_static_mu;
+unsigned char* g_static_ptr[kMaxDevices] = {};
+
+// Device address of bc_static_scratch on the current device; looked up once per device.
+cudaError_t static_scratch(unsigned char** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, bc_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_ptr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return cudaSuccess;
+}
+}  // namespace
+
+bc_status bc_decode_attn_static(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, void* out,
+                                float sm_scale, const void* extra_k, const void* extra_v, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (!q || !out || !aligned16(q) || !aligned16(out)) return BC_ERR_INVALID_ARG;
+  if ((extra_k == nullptr) != (extra_v == nullptr)) return BC_ERR_INVALID_ARG;
+  if (extra_k && (!aligned16(extra_k) || !aligned16(extra_v))) return BC_ERR_INVALID_ARG;
+  if (n > BC_STATIC_MAX_BATCH || c->cfg.q_heads * c->cfg.head_dim > BC_MERGE_ELEMS || c->cfg.q_heads > 64)
+    return BC_ERR_TOO_LARGE;
+  unsigned char* base = nullptr;
+  BC_CUDA(c, static_scratch(&base));
+  BcAttnArgs a;
+  a.pool_layer = layer_base(c, layer);
+  a.slots = slots; a.n = n; a.q = q; a.out = out;
+  a.out_f32 = (c->cfg.flags & BC_FLAG_OUT_F32) ? 1 : 0;
+  a.extra_k = extra_k; a.extra_v = extra_v; a.sm_scale = sm_scale;
+  a.part_o = reinterpret_cast<float*>(base);
+  a.part_ml = reinterpret_cast<float*>(base + kStaticPartO);
+  a.first_cta = reinterpret_cast<int32_t*>(base + kStaticPartO + kStaticPartMl);
+  a.last_cta = a.first_cta + BC_STATIC_MAX_BATCH;
+  int ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
+  a.ctas = ctas < BC_STATIC_MAX_CTAS ? ctas : BC_STATIC_MAX_CTAS;
+  int launches = 0;
+  BC_CUDA(c, bc_launch_attn(c->meta, c->geom, a, (cudaStream_t)stream, nullptr, nullptr, &launches));
+  c->launches += launches;
   return BC_OK;
 }
 

@@ -32,7 +32,7 @@ MetaLayout meta_layout(const bc_config& c) {
 }
 
 struct WorkLayout {
-  size_t append_row, append_pos, compress_row, compress_pos, first_cta, last_cta, part_ml, part_o, stage_q, stage_k,
+  size_t append_row, append_pos, compress_row, compress_pos, tickets, part_ml, part_o, stage_q, stage_k,
       stage_v, stage_out, total;
 };
 WorkLayout work_layout(const bc_config& c) {
@@ -42,7 +42,7 @@ WorkLayout work_layout(const bc_config& c) {
   const size_t seq = (size_t)c.max_seqs * 4;
   const size_t pieces = BC_MAX_ATTN_CTAS + BC_MAX_ATTN_BATCH;
   l.append_row = take(seq); l.append_pos = take(seq); l.compress_row = take(seq); l.compress_pos = take(seq);
-  l.first_cta = take(BC_MAX_ATTN_BATCH * 4); l.last_cta = take(BC_MAX_ATTN_BATCH * 4);
+  l.tickets = take(BC_MAX_ATTN_BATCH * 4);
   l.part_ml = take(pieces * c.q_heads * 2 * 4);
   l.part_o = take(pieces * c.q_heads * c.head_dim * 4);
   l.stage_q = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 2);
@@ -68,6 +68,8 @@ bool config_ok(const bc_config* c, bc_status* why) {
   if (c->q_heads * c->head_dim > BC_MERGE_ELEMS) return false;
   return true;
 }
+
+constexpr size_t kFusedRowBytes = 512u << 10;  // rows of a batch that the bookkeeping block copies itself
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
@@ -125,8 +127,7 @@ bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const v
   a.extra_k = extra_k; a.extra_v = extra_v; a.sm_scale = sm_scale;
   a.part_o = work_ptr<float>(c, c->wl.part_o);
   a.part_ml = work_ptr<float>(c, c->wl.part_ml);
-  a.first_cta = work_ptr<int32_t>(c, c->wl.first_cta);
-  a.last_cta = work_ptr<int32_t>(c, c->wl.last_cta);
+  a.tickets = work_ptr<int32_t>(c, c->wl.tickets);
   a.ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
   if (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) {
     BC_CUDA(c, bc_launch_attn_reference(c->meta, c->geom, a, s));
@@ -142,6 +143,63 @@ bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const v
 }
 
 }  // namespace
+
+// ---- bc_decode_attn_static: split-K scratch inside the library image -------------------------------
+//
+// Layout of the built-in array: partial outputs [pieces][4096] fp32, then (max, sum) pairs
+// [pieces][64][2] fp32, then one ticket counter per sequence, [BC_STATIC_MAX_BATCH] int32, with
+// pieces = BC_STATIC_MAX_CTAS + BC_STATIC_MAX_BATCH.  The loader zero-fills the array and every
+// launch leaves the counters at zero again; the partials need no clearing because a launch reads
+// only what it has written.
+namespace {
+constexpr size_t kStaticPieces = BC_STATIC_MAX_CTAS + BC_STATIC_MAX_BATCH;
+constexpr size_t kStaticPartO = kStaticPieces * BC_MERGE_ELEMS * sizeof(float);
+constexpr size_t kStaticPartMl = kStaticPieces * 64 * 2 * sizeof(float);
+constexpr size_t kStaticIdx = BC_STATIC_MAX_BATCH * sizeof(int32_t);
+constexpr size_t kStaticBytes = kStaticPartO + kStaticPartMl + kStaticIdx;
+constexpr int kMaxDevices = 64;
+}  // namespace
+
+// In host code this name is only a handle for the runtime's symbol lookup, never a device address.
+static __device__ __align__(256) unsigned char bc_static_scratch[kStaticBytes];
+
+namespace {
+std::mutex g_static_mu;
+unsigned char* g_static_ptr[kMaxDevices] = {};
+
+// Device address of bc_static_scratch on the current device; looked up once per device.
+cudaError_t static_scratch(unsigned char** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, bc_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_ptr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return cudaSuccess;
+}
+
+// Zeroes the ticket counters of the built-in array on the current device if a call has already
+// looked its address up there (used when a latched error is cleared).
+cudaError_t static_scratch_reset_tickets(cudaStream_t s) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  unsigned char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (dev >= 0 && dev < kMaxDevices) base = g_static_ptr[dev];
+  }
+  if (!base) return cudaSuccess;
+  return cudaMemsetAsync(base + kStaticPartO + kStaticPartMl, 0, kStaticIdx, s);
+}
+}  // namespace
+
 
 extern "C" {
 
@@ -204,6 +262,7 @@ bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* wo
   g.layer_bytes = (int64_t)cfg->num_pages * cfg->page_size * g.entry_bytes;
   cudaError_t e = bc_attn_setup(&c->sm_count);
   if (e == cudaSuccess) e = bc_launch_init(c->meta, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->work + c->wl.tickets, 0, BC_MAX_ATTN_BATCH * 4, (cudaStream_t)stream);
   if (e != cudaSuccess) { delete c; return BC_ERR_CUDA; }
   c->launches += 1;
   *out = c;
@@ -246,12 +305,17 @@ bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n,
   int32_t* row = work_ptr<int32_t>(c, c->wl.append_row);
   int32_t* pos = work_ptr<int32_t>(c, c->wl.append_pos);
   cudaStream_t s = (cudaStream_t)stream;
+  // One thread block copies up to kFusedRowBytes in about the time a second launch would cost.
+  const bool fused = layer == 0 && (size_t)n * c->geom.entry_bytes <= kFusedRowBytes;
   if (layer == 0) {
-    BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, ++c->calls, row, pos, s));
+    BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, ++c->calls, row, pos, c->geom, layer_base(c, 0),
+                                     fused ? k : nullptr, fused ? v : nullptr, s));
     c->launches += 1;
   }
-  BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, k, v, n, s));
-  c->launches += 1;
+  if (!fused) {
+    BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, k, v, n, s));
+    c->launches += 1;
+  }
   c->append_next_layer = (layer + 1) % c->cfg.layers;
   return BC_OK;
 }
@@ -277,22 +341,21 @@ bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t 
   int32_t* pos = work_ptr<int32_t>(c, c->wl.compress_pos);
   cudaStream_t s = (cudaStream_t)stream;
   const int L = c->cfg.layers;
+  const bool fused = layer == 0 && (size_t)n * c->geom.entry_bytes <= kFusedRowBytes;
   if (layer == 0) {
     ++c->calls;
-    if (L > 1) {  // allocate now, evict on the last layer's call
-      BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, 1, s));
-      c->launches += 1;
-    }
-  }
-  if (L == 1) {
-    // single layer: allocate, evict, then write; the beacon row does not depend on the eviction
-    BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, 3, s));
+    // several layers: allocate now, evict on the last layer's call; a single layer: allocate and
+    // evict at once (the beacon row does not depend on the eviction)
+    BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, L > 1 ? 1 : 3, c->geom, layer_base(c, 0),
+                                       fused ? bk : nullptr, fused ? bv : nullptr, s));
     c->launches += 1;
   }
-  BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, bk, bv, n, s));
-  c->launches += 1;
+  if (!fused) {
+    BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, bk, bv, n, s));
+    c->launches += 1;
+  }
   if (L > 1 && layer == L - 1) {
-    BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, 2, s));
+    BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, 2, c->geom, nullptr, nullptr, nullptr, s));
     c->launches += 1;
   }
   c->compress_next_layer = (layer + 1) % L;
@@ -401,6 +464,9 @@ bc_status bc_poll_error(bc_cache* c, int32_t* code, int32_t* slot, int64_t* call
 bc_status bc_clear_error(bc_cache* c, void* stream) {
   if (!c) return BC_ERR_INVALID_ARG;
   BC_CUDA(c, cudaMemsetAsync(c->meta.status, 0, 16, (cudaStream_t)stream));
+  // an attention launch that gave up (BC_ERR_TIMEOUT) may have left ticket counters non-zero
+  BC_CUDA(c, cudaMemsetAsync(c->work + c->wl.tickets, 0, BC_MAX_ATTN_BATCH * 4, (cudaStream_t)stream));
+  BC_CUDA(c, static_scratch_reset_tickets((cudaStream_t)stream));
   return BC_OK;
 }
 
@@ -448,45 +514,6 @@ bc_status bc_profile_read(bc_cache* c, int32_t* launches, float* total_ms) {
   return BC_OK;
 }
 
-// ---- bc_decode_attn_static: split-K scratch inside the library image -------------------------------
-//
-// Layout of the built-in array: partial outputs [pieces][4096] fp32, then (max, sum) pairs
-// [pieces][64][2] fp32, then first/last block per sequence, 2 x [BC_STATIC_MAX_BATCH] int32,
-// with pieces = BC_STATIC_MAX_CTAS + BC_STATIC_MAX_BATCH.
-namespace {
-constexpr size_t kStaticPieces = BC_STATIC_MAX_CTAS + BC_STATIC_MAX_BATCH;
-constexpr size_t kStaticPartO = kStaticPieces * BC_MERGE_ELEMS * sizeof(float);
-constexpr size_t kStaticPartMl = kStaticPieces * 64 * 2 * sizeof(float);
-constexpr size_t kStaticIdx = 2 * BC_STATIC_MAX_BATCH * sizeof(int32_t);
-constexpr size_t kStaticBytes = kStaticPartO + kStaticPartMl + kStaticIdx;
-constexpr int kMaxDevices = 64;
-}  // namespace
-
-// In host code this name is only a handle for the runtime's symbol lookup, never a device address.
-static __device__ __align__(256) unsigned char bc_static_scratch[kStaticBytes];
-
-namespace {
-std::mutex g_static_mu;
-unsigned char* g_static_ptr[kMaxDevices] = {};
-
-// Device address of bc_static_scratch on the current device; looked up once per device.
-cudaError_t static_scratch(unsigned char** out) {
-  int dev = -1;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  std::lock_guard<std::mutex> lock(g_static_mu);
-  if (!g_static_ptr[dev]) {
-    void* p = nullptr;
-    e = cudaGetSymbolAddress(&p, bc_static_scratch);
-    if (e != cudaSuccess) return e;
-    g_static_ptr[dev] = static_cast<unsigned char*>(p);
-  }
-  *out = g_static_ptr[dev];
-  return cudaSuccess;
-}
-}  // namespace
-
 bc_status bc_decode_attn_static(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, void* out,
                                 float sm_scale, const void* extra_k, const void* extra_v, void* stream) {
   bc_status st = check_batch(c, layer, slots, n);
@@ -505,8 +532,7 @@ bc_status bc_decode_attn_static(bc_cache* c, int32_t layer, const int32_t* slots
   a.extra_k = extra_k; a.extra_v = extra_v; a.sm_scale = sm_scale;
   a.part_o = reinterpret_cast<float*>(base);
   a.part_ml = reinterpret_cast<float*>(base + kStaticPartO);
-  a.first_cta = reinterpret_cast<int32_t*>(base + kStaticPartO + kStaticPartMl);
-  a.last_cta = a.first_cta + BC_STATIC_MAX_BATCH;
+  a.tickets = reinterpret_cast<int32_t*>(base + kStaticPartO + kStaticPartMl);
   int ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
   a.ctas = ctas < BC_STATIC_MAX_CTAS ? ctas : BC_STATIC_MAX_CTAS;
   int launches = 0;

@@ -14,7 +14,11 @@
 //     the batch, in order, are divided evenly over the grid (each block gets a contiguous span), so
 //     ragged batches balance to within one tile.  A block's share of one sequence is a "piece"; a
 //     piece that covers the whole sequence writes the final output, otherwise it writes an
-//     unnormalised partial (m, l, O) and k_attn_combine merges the pieces.
+//     unnormalised partial (m, l, O) and takes a ticket from the sequence's counter; the block
+//     that takes the last ticket merges all pieces of the sequence (always in piece order, so the
+//     result does not depend on which block came last) and resets the counter.  Nobody waits.
+//   * The producer never stalls on the page table: page ids are fetched a few tiles ahead with
+//     4-byte asynchronous copies into a small shared-memory ring.
 //   * Every wait is bounded: on expiry the block records BC_ERR_TIMEOUT, stops issuing copies,
 //     drains the copies already in flight (bounded) and returns.
 //
@@ -25,9 +29,13 @@
 namespace {
 
 constexpr int kConsumerWarps = 8;
-constexpr int kPipeThreads = (kConsumerWarps + 1) * 32;
+constexpr int kPipeThreads = (kConsumerWarps + 1) * 32;  // consumer warps and the producer warp
 constexpr int kPlanMax = BC_MAX_ATTN_BATCH;
 constexpr uint32_t kSpinLimit = 1u << 21;  // polls of try_wait before giving up
+constexpr int kPidAhead = 4;               // tiles of page-id lookahead of the producer
+constexpr int kInFlight = 2;               // stages whose copies may be outstanding at once: HBM
+                                           // delivers less when every SM keeps more in flight
+constexpr int kPidSlot = 136;              // ints per descriptor slot: 4 header + up to 132 page ids
 
 // ---------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -57,6 +65,23 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                "l"(src), "r"(bytes), "r"(bar)
                : "memory");
 }
+// 4-byte asynchronous copy global -> shared (page-id prefetch), grouped by commit / wait_group.
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// Waits until at most `pending` (clamped to kPidAhead) of the most recent groups are outstanding.
+__device__ __forceinline__ void cp_async_wait_dyn(int pending) {
+  switch (pending) {
+    case 0: cp_async_wait<0>(); break;
+    case 1: cp_async_wait<1>(); break;
+    case 2: cp_async_wait<2>(); break;
+    case 3: cp_async_wait<3>(); break;
+    default: cp_async_wait<kPidAhead>(); break;
+  }
+}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
@@ -76,6 +101,11 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], 
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -98,18 +128,26 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, vola
 }
 
 // ---------------------------------------------------------------- shared-memory plan
-struct SeqInfo {
-  int P, nb, w, Rb, Rw, slot;
+// Exact unsigned division by a runtime constant (round-up method of Granlund and Montgomery):
+// q = (t + ((n - t) >> sh1)) >> sh2 with t = umulhi(mul, n), for every 32-bit n.
+struct FastDiv {
+  uint32_t mul, sh1, sh2;
 };
+__device__ __forceinline__ int fast_div(int n, const FastDiv& d) {
+  const uint32_t t = __umulhi(d.mul, (uint32_t)n);
+  return (int)((t + (((uint32_t)n - t) >> d.sh1)) >> d.sh2);
+}
 
 struct PipeParams {
   BcMeta m;
   BcGeom g;
   BcAttnArgs a;
   float scale_log2;
-  int rows_per_tile;  // T
+  int rows_per_tile;  // T = 16 * n_groups, a power of two
+  int tile_shift;     // log2(T)
   int n_groups;       // 8 / kv_heads
   int G;              // q_heads / kv_heads
+  FastDiv div_ps;     // division by page_size
 };
 
 template <int D>
@@ -120,11 +158,86 @@ struct PipeSmem {
   static constexpr int kMergeOff = kRingBytes;
   static constexpr int kMergeMlOff = kMergeOff + BC_MERGE_ELEMS * 4;
   static constexpr int kPlanOff = kMergeMlOff + 64 * 2 * 4;  // up to 64 query heads
-  // plan arrays: P, nb, w, slot [kPlanMax] and cum [kPlanMax + 1]
-  static constexpr int kBarOff = kPlanOff + (4 * kPlanMax + kPlanMax + 8) * 4;
-  static constexpr int kAbortOff = kBarOff + 2 * kStages * 8;
-  static constexpr int kTotal = kAbortOff + 16;
+  // plan arrays: P, nb, w, slot, beacon column, window column [kPlanMax] and cum [kPlanMax + 1]
+  static constexpr int kPidOff = kPlanOff + (6 * kPlanMax + kPlanMax + 8) * 4;
+  // descriptors of the tiles ahead: (kPidAhead + 1) slots of {rows, first position, first page,
+  // unused} followed by the page ids of the tile
+  static constexpr int kBarOff = kPidOff + (kPidAhead + 1) * kPidSlot * 4;
+  static constexpr int kMiscOff = kBarOff + 2 * kStages * 8;  // abort flag, pending tickets
+  static constexpr int kTotal = kMiscOff + 32;
 };
+
+// Merges the pieces of sequence i (published by blocks first..last) into the final output.  The
+// pieces are folded in block order with a running maximum, so the result does not depend on which
+// block does the merging.  Piece `own` is taken from the caller's shared-memory copy (own_o,
+// own_ml) instead of global memory; pass own = -1 to read every piece from global memory.  Called
+// by the 256 consumer threads; each owns up to four float4 of the [q_heads, head_dim] output.
+// The loads of all four vectors of up to three pieces are issued together, so a merge of three
+// pieces costs about one trip to L2.
+__device__ __forceinline__ void combine_pieces(const float* part_o, const float* part_ml, void* out, int out_f32, int Hq,
+                                            int D, int i, int first, int last, int own, const float* own_o,
+                                            const float* own_ml, int tid) {
+  constexpr int kThreads = kConsumerWarps * 32;
+  constexpr int KV = BC_MERGE_ELEMS / 4 / kThreads;  // float4 per thread
+  constexpr int PB = 3;                              // pieces per batch
+  const int nvec = Hq * D / 4;
+  const int64_t obase = (int64_t)i * Hq * D;
+  float4 acc[KV];
+  float mrun[KV], den[KV];
+#pragma unroll
+  for (int k = 0; k < KV; ++k) { acc[k] = make_float4(0.f, 0.f, 0.f, 0.f); mrun[k] = -INFINITY; den[k] = 0.f; }
+#pragma unroll 1
+  for (int c0 = first; c0 <= last; c0 += PB) {
+    float mc[KV][PB], lc[KV][PB];
+    float4 oc[KV][PB];
+#pragma unroll
+    for (int j = 0; j < PB; ++j) {
+      const int c = c0 + j;
+      const int64_t ps = (int64_t)(c + i);
+#pragma unroll
+      for (int k = 0; k < KV; ++k) {
+        const int e = tid + k * kThreads;
+        const int h = (e * 4) / D;
+        mc[k][j] = -INFINITY; lc[k][j] = 0.f; oc[k][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c <= last && e < nvec) {
+          if (c == own) {
+            mc[k][j] = own_ml[h * 2]; lc[k][j] = own_ml[h * 2 + 1];
+            oc[k][j] = reinterpret_cast<const float4*>(own_o)[e];
+          } else {
+            mc[k][j] = __ldcg(part_ml + (ps * Hq + h) * 2);
+            lc[k][j] = __ldcg(part_ml + (ps * Hq + h) * 2 + 1);
+            oc[k][j] = __ldcg(reinterpret_cast<const float4*>(part_o + ps * Hq * D) + e);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < PB; ++j)
+#pragma unroll
+      for (int k = 0; k < KV; ++k) {
+        const float mn = fmaxf(mrun[k], mc[k][j]);
+        const float msafe = mn == -INFINITY ? 0.f : mn;
+        const float sa = exp2f(mrun[k] - msafe), sb = exp2f(mc[k][j] - msafe);
+        acc[k].x = acc[k].x * sa + oc[k][j].x * sb; acc[k].y = acc[k].y * sa + oc[k][j].y * sb;
+        acc[k].z = acc[k].z * sa + oc[k][j].z * sb; acc[k].w = acc[k].w * sa + oc[k][j].w * sb;
+        den[k] = den[k] * sa + lc[k][j] * sb;
+        mrun[k] = mn;
+      }
+  }
+#pragma unroll
+  for (int k = 0; k < KV; ++k) {
+    const int e = tid + k * kThreads;
+    if (e < nvec) {
+      const float inv = den[k] > 0.f ? 1.f / den[k] : 0.f;
+      const float4 r = make_float4(acc[k].x * inv, acc[k].y * inv, acc[k].z * inv, acc[k].w * inv);
+      if (out_f32) reinterpret_cast<float4*>(reinterpret_cast<float*>(out) + obase)[e] = r;
+      else {
+        uint2 pk; pk.x = pack_bf16(r.x, r.y); pk.y = pack_bf16(r.z, r.w);
+        reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + obase)[e] = pk;
+      }
+    }
+  }
+}
 
 template <int D, bool G_LE_8>
 __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams p) {
@@ -132,6 +245,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   constexpr int NSTAGE = L::kStages;
   constexpr int KSTEPS = D / 16;  // k-steps of QK^T
   constexpr int NT = D / 8;       // n-tiles of PV
+  constexpr int RING = kPidAhead + 1;
   extern __shared__ __align__(1024) uint8_t smem[];
 
   float* merge_o = reinterpret_cast<float*>(smem + L::kMergeOff);
@@ -140,14 +254,19 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   int* s_nb = s_P + kPlanMax;
   int* s_w = s_nb + kPlanMax;
   int* s_slot = s_w + kPlanMax;
-  int* s_cum = s_slot + kPlanMax;  // [n + 1] exclusive prefix sums of tiles
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::kAbortOff);
+  int* s_bcol = s_slot + kPlanMax;  // first beacon column of the page-table row
+  int* s_wcol = s_bcol + kPlanMax;  // first window column
+  int* s_cum = s_wcol + kPlanMax;   // [n + 1] exclusive prefix sums of tiles
+  int* s_desc = reinterpret_cast<int*>(smem + L::kPidOff);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::kMiscOff);
+  volatile int* s_pend = s_abort + 1;  // {sequence, ticket} of up to two published pieces; [4]: peeked count
   const uint32_t ring = smem_u32(smem);
+  const uint32_t desc_ring = smem_u32(smem + L::kPidOff);
   const uint32_t bar_full = smem_u32(smem + L::kBarOff);
   const uint32_t bar_empty = bar_full + NSTAGE * 8;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n = p.a.n, T = p.rows_per_tile, E = p.g.entry_bytes, ps = p.g.page_size;
+  const int n = p.a.n, T = p.rows_per_tile, TS = p.tile_shift, E = p.g.entry_bytes, ps = p.g.page_size;
   const int Hkv = p.g.kv_heads, Hq = p.g.q_heads, G = p.G;
 
   if (tid == 0) {
@@ -161,16 +280,18 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   }
 
   // ---- plan: tiles per sequence, prefix sums, this block's span --------------------------------
+  // Each segment (prompt, beacons, window) starts a new tile, so a tile never straddles segments;
+  // a partly filled tile costs masked arithmetic but no memory traffic.
   for (int i = tid; i < n; i += kPipeThreads) {
     const int slot = p.a.slots[i];
-    int P = 0, nb = 0, w = 0;
+    int P = 0, nb = 0, w = 0, bcol = 0, wcol = 0, sl = 0;
     if (slot >= 0 && slot < p.m.max_seqs && p.m.open[slot]) {
       P = p.m.prompt_len[slot]; nb = p.m.n_beacons[slot]; w = p.m.window_len[slot];
+      bcol = p.m.beacon_off[slot]; wcol = p.m.window_off[slot]; sl = slot;
     }
-    s_P[i] = P; s_nb[i] = nb; s_w[i] = w; s_slot[i] = slot;
-    const int Rb = (P + 7) & ~7, Rw = (Rb + nb + 7) & ~7;
-    const int rows = Rw + w;
-    s_cum[i + 1] = rows > 0 ? (rows + T - 1) / T : 1;  // an empty sequence still owns one tile
+    s_P[i] = P; s_nb[i] = nb; s_w[i] = w; s_slot[i] = sl; s_bcol[i] = bcol; s_wcol[i] = wcol;
+    const int tiles = ((P + T - 1) >> TS) + ((nb + T - 1) >> TS) + ((w + T - 1) >> TS);
+    s_cum[i + 1] = tiles > 0 ? tiles : 1;  // an empty sequence still owns one (empty) tile
   }
   __syncthreads();
   if (warp == 0) {  // inclusive scan of s_cum[1..n]
@@ -195,6 +316,8 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   const int g0 = cta * per + min(cta, rem);
   const int g1 = g0 + per + (cta < rem ? 1 : 0);
   if (g0 >= g1) return;
+  // block that owns global tile g under the flat partition
+  auto cta_of = [&](int g) { return g < rem * (per + 1) ? g / (per + 1) : rem + (g - rem * (per + 1)) / per; };
   int seq0 = 0;
   {  // largest i with cum[i] <= g0
     int lo = 0, hi = n;
@@ -202,60 +325,82 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     seq0 = lo;
   }
 
-  auto seq_info = [&](int i) {
-    SeqInfo s;
-    s.P = s_P[i]; s.nb = s_nb[i]; s.w = s_w[i]; s.slot = s_slot[i];
-    s.Rb = (s.P + 7) & ~7; s.Rw = (s.Rb + s.nb + 7) & ~7;
-    return s;
-  };
-
   if (warp == kConsumerWarps) {
     // ================================ producer warp ============================================
-    int i = seq0;
-    SeqInfo si = seq_info(i);
+    // describe(gt) runs kPidAhead tiles ahead of the copies: it works out which rows tile gt holds,
+    // writes {rows, first position, first page} to a small descriptor ring and starts 4-byte
+    // asynchronous copies of the tile's page-table entries into the same slot.  Issuing the bulk
+    // copies of a tile then takes a handful of instructions and never waits on the page table.
+    int fi = seq0;
+    int f_P, f_nb, f_w, f_tp, f_tpb, f_bcol, f_wcol;
+    const int32_t* f_tab;
+    auto load_seq = [&](int i) {
+      f_P = s_P[i]; f_nb = s_nb[i]; f_w = s_w[i]; f_bcol = s_bcol[i]; f_wcol = s_wcol[i];
+      f_tp = (f_P + T - 1) >> TS; f_tpb = f_tp + ((f_nb + T - 1) >> TS);
+      f_tab = p.m.page_table + (int64_t)s_slot[i] * p.m.max_pages_per_seq;
+    };
+    load_seq(fi);
+    auto describe = [&](int gt, int it) {
+      int nrows = 0, p0 = 0, pg0 = 0;
+      const int slot_idx = (it % RING) * kPidSlot;
+      if (gt < g1) {
+        while (gt >= s_cum[fi + 1]) { ++fi; load_seq(fi); }
+        const int t = gt - s_cum[fi];
+        int len, tt, col;
+        if (t < f_tp) { len = f_P; tt = t; col = 0; }
+        else if (t < f_tpb) { len = f_nb; tt = t - f_tp; col = f_bcol; }
+        else { len = f_w; tt = t - f_tpb; col = f_wcol; }
+        p0 = tt << TS;
+        nrows = max(min(T, len - p0), 0);
+        if (nrows > 0) {
+          pg0 = fast_div(p0, p.div_ps);
+          const int pg_last = fast_div(p0 + nrows - 1, p.div_ps);
+          for (int pg = pg0 + lane; pg <= pg_last; pg += 32)
+            cp_async4(desc_ring + (uint32_t)(slot_idx + 4 + pg - pg0) * 4u, f_tab + col + pg);
+        }
+      }
+      if (lane == 0) { s_desc[slot_idx] = nrows; s_desc[slot_idx + 1] = p0; s_desc[slot_idx + 2] = pg0; }
+      cp_async_commit();  // one group per described tile
+    };
+    // The first tile is described alone so that its copies start as early as possible; the
+    // lookahead then grows by up to two tiles per iteration until it is kPidAhead deep.
+    int described = 1;
+    describe(g0, 0);
     int it = 0;
     bool aborted = false;
+#pragma unroll 1
     for (int gt = g0; gt < g1; ++gt, ++it) {
-      while (gt >= s_cum[i + 1]) { ++i; si = seq_info(i); }
-      const int t = gt - s_cum[i];
+      cp_async_wait_dyn(described - it - 1);  // the page ids of tile gt have landed
+      __syncwarp();
       const int stage = it % NSTAGE;
       const uint32_t full = bar_full + stage * 8, empty = bar_empty + stage * 8;
       if (!aborted && !bounded_wait(empty, ((it / NSTAGE) & 1) ^ 1, s_abort)) aborted = true;
-      if (aborted) continue;
-      const int v0 = t * T, v1 = v0 + T;
-      const int seg_start[3] = {0, si.Rb, si.Rw};
-      const int seg_len[3] = {si.P, si.nb, si.w};
-      int rows = 0;
-#pragma unroll
-      for (int sgi = 0; sgi < 3; ++sgi) {
-        const int a = max(v0, seg_start[sgi]), b = min(v1, seg_start[sgi] + seg_len[sgi]);
-        rows += max(b - a, 0);
-      }
-      if (lane == 0) {
-        if (rows > 0) mbar_arrive_expect_tx(full, (uint32_t)rows * (uint32_t)E);
-        else mbar_arrive(full);
-      }
-      __syncwarp();
-      if (rows > 0) {
-        const int32_t* row_tab = p.m.page_table + (int64_t)si.slot * p.m.max_pages_per_seq;
-        const int seg_col[3] = {0, p.m.beacon_off[si.slot], p.m.window_off[si.slot]};
+      // at most kInFlight stages in flight: the copies of tile it - kInFlight must have landed
+      if (!aborted && it >= kInFlight &&
+          !bounded_wait(bar_full + ((it - kInFlight) % NSTAGE) * 8, ((it - kInFlight) / NSTAGE) & 1, s_abort))
+        aborted = true;
+      if (!aborted) {
+        const int* d = s_desc + (it % RING) * kPidSlot;
+        const int nrows = d[0], p0 = d[1], pg0 = d[2];
+        if (lane == 0) {
+          if (nrows > 0) mbar_arrive_expect_tx(full, (uint32_t)nrows * (uint32_t)E);
+          else mbar_arrive(full);
+        }
         const uint32_t stage_base = ring + stage * L::kStageBytes;
-#pragma unroll
-        for (int sgi = 0; sgi < 3; ++sgi) {
-          const int a = max(v0, seg_start[sgi]), b = min(v1, seg_start[sgi] + seg_len[sgi]);
-          if (a >= b) continue;
-          const int p0 = a - seg_start[sgi], p1 = b - seg_start[sgi];
-          const int pg_last = (p1 - 1) / ps;
-          for (int pg = p0 / ps + lane; pg <= pg_last; pg += 32) {
-            const int lo = max(p0, pg * ps), hi = min(p1, (pg + 1) * ps);
-            const int page = row_tab[seg_col[sgi] + pg];
-            const uint8_t* src = p.a.pool_layer + ((int64_t)page * ps + (lo - pg * ps)) * E;
-            const uint32_t dst = stage_base + (uint32_t)(seg_start[sgi] + lo - v0) * (uint32_t)E;
-            bulk_g2s(dst, src, (uint32_t)(hi - lo) * (uint32_t)E, full);
-          }
+        for (int k = lane;; k += 32) {
+          const int pg = pg0 + k;
+          const int lo = max(p0, pg * ps), hi = min(p0 + nrows, pg * ps + ps);
+          if (lo >= hi) break;
+          const uint8_t* src = p.a.pool_layer + ((int64_t)d[4 + k] * ps + (lo - pg * ps)) * E;
+          bulk_g2s(stage_base + (uint32_t)(lo - p0) * (uint32_t)E, src, (uint32_t)(hi - lo) * (uint32_t)E, full);
         }
       }
+      __syncwarp();  // the slot read above may be rewritten by the describe() calls below
+#pragma unroll 1
+      for (int r = 0; r < 2 && described < it + 1 + kPidAhead && g0 + described < g1; ++r, ++described)
+        describe(g0 + described, described);
     }
+    cp_async_wait<0>();
     // Drain: every armed stage whose copies might still be in flight must complete before exit.
     if (aborted || *s_abort) {
       const int armed = it;
@@ -279,33 +424,42 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   const int v_chunk_sel = lm >> 1;
   const uint32_t warp_rows_off = (uint32_t)(grp * 16) * (uint32_t)E;
 
+  // query fragments of sequence i: rows = the G query heads of this warp's KV head
+  auto load_q = [&](uint32_t (&qr)[KSTEPS][4], int i) {
+    const __nv_bfloat16* qb = reinterpret_cast<const __nv_bfloat16*>(p.a.q) + ((int64_t)i * Hq + kvh * G) * D;
+#pragma unroll
+    for (int kk = 0; kk < KSTEPS; ++kk) {
+      const int d0 = kk * 16 + qd * 2;
+      qr[kk][0] = gq < G ? *reinterpret_cast<const uint32_t*>(qb + gq * D + d0) : 0u;
+      qr[kk][2] = gq < G ? *reinterpret_cast<const uint32_t*>(qb + gq * D + d0 + 8) : 0u;
+      if (G_LE_8) { qr[kk][1] = 0u; qr[kk][3] = 0u; }
+      else {
+        qr[kk][1] = gq + 8 < G ? *reinterpret_cast<const uint32_t*>(qb + (gq + 8) * D + d0) : 0u;
+        qr[kk][3] = gq + 8 < G ? *reinterpret_cast<const uint32_t*>(qb + (gq + 8) * D + d0 + 8) : 0u;
+      }
+    }
+  };
+
   int i = seq0;
   int it = 0;
   int gt = g0;
+  int n_pend = 0;  // pieces this block has published; thread 0 keeps their tickets
+  int pend_seq0 = -1, pend_tk0 = 0, pend_seq1 = -1, pend_tk1 = 0;
+  uint32_t qf[KSTEPS][4];
+  load_q(qf, seq0);
   while (gt < g1) {
     while (gt >= s_cum[i + 1]) ++i;
-    const SeqInfo si = seq_info(i);
+    const int c_P = s_P[i], c_nb = s_nb[i], c_w = s_w[i];
+    const int c_tp = (c_P + T - 1) >> TS, c_tpb = c_tp + ((c_nb + T - 1) >> TS);
     const int tiles_i = s_cum[i + 1] - s_cum[i];
     const int ta = gt - s_cum[i];
     const int tb = min(tiles_i, ta + (g1 - gt));
     const bool whole = (ta == 0 && tb == tiles_i);
+    // the next piece's query fragments are fetched now, so the switch between pieces does not wait
+    const bool has_next = gt + (tb - ta) < g1;
+    uint32_t qn[KSTEPS][4];
+    if (has_next) load_q(qn, i + 1);
 
-    // ---- query fragments: rows = the G query heads of this KV head -----------------------------
-    uint32_t qf[KSTEPS][4];
-    {
-      const __nv_bfloat16* qb = reinterpret_cast<const __nv_bfloat16*>(p.a.q) + ((int64_t)i * Hq + kvh * G) * D;
-#pragma unroll
-      for (int kk = 0; kk < KSTEPS; ++kk) {
-        const int d0 = kk * 16 + qd * 2;
-        qf[kk][0] = gq < G ? *reinterpret_cast<const uint32_t*>(qb + gq * D + d0) : 0u;
-        qf[kk][2] = gq < G ? *reinterpret_cast<const uint32_t*>(qb + gq * D + d0 + 8) : 0u;
-        if (G_LE_8) { qf[kk][1] = 0u; qf[kk][3] = 0u; }
-        else {
-          qf[kk][1] = gq + 8 < G ? *reinterpret_cast<const uint32_t*>(qb + (gq + 8) * D + d0) : 0u;
-          qf[kk][3] = gq + 8 < G ? *reinterpret_cast<const uint32_t*>(qb + (gq + 8) * D + d0 + 8) : 0u;
-        }
-      }
-    }
     float o[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
@@ -345,26 +499,20 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       const int stage = it % NSTAGE;
       const bool ok = __all_sync(0xffffffffu, bounded_wait(bar_full + stage * 8, (it / NSTAGE) & 1, s_abort));
       if (!ok && lane == 0 && p.m.status[0] == 0) { p.m.status[0] = BC_ERR_TIMEOUT; p.m.status[1] = -1; }
-      const int vrow0 = t * T + grp * 16;  // virtual row of this warp's first row
-      // valid rows among my 16
-      int cnt = 0;
-      {
-        const int a0 = max(vrow0, 0), b0 = min(vrow0 + 16, si.P);
-        const int a1 = max(vrow0, si.Rb), b1 = min(vrow0 + 16, si.Rb + si.nb);
-        const int a2 = max(vrow0, si.Rw), b2 = min(vrow0 + 16, si.Rw + si.w);
-        cnt = max(b0 - a0, 0) + max(b1 - a1, 0) + max(b2 - a2, 0);
-      }
+      // rows of this tile that hold entries; my warp looks at rows grp*16 .. grp*16+15 of it
+      int seg_left;
+      if (t < c_tp) seg_left = c_P - (t << TS);
+      else if (t < c_tpb) seg_left = c_nb - ((t - c_tp) << TS);
+      else seg_left = c_w - ((t - c_tpb) << TS);
+      const int cnt = max(min(seg_left - grp * 16, 16), 0);
       bool wrote_smem = false;
       if (ok && cnt > 0) {
         const uint32_t rows_base = ring + stage * L::kStageBytes + warp_rows_off;
-        auto row_valid = [&](int v) {
-          return (v < si.P) || (v >= si.Rb && v < si.Rb + si.nb) || (v >= si.Rw && v < si.Rw + si.w);
-        };
         if (cnt < 16) {
           // rows nobody copied may hold anything: zero their V so that 0 * garbage cannot be NaN
           uint8_t* rows_ptr = smem + stage * L::kStageBytes + warp_rows_off;
-          for (int r = 0; r < 16; ++r) {
-            if (!row_valid(vrow0 + r) && lane < (p.g.head_row_bytes >> 4))
+          for (int r = cnt; r < 16; ++r) {
+            if (lane < (p.g.head_row_bytes >> 4))
               *reinterpret_cast<uint4*>(rows_ptr + r * E + (Hkv + kvh) * p.g.head_row_bytes + lane * 16) =
                   make_uint4(0, 0, 0, 0);
           }
@@ -390,7 +538,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
           for (int j = 0; j < 2; ++j)
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
-              if (!row_valid(vrow0 + j * 8 + qd * 2 + e)) { s[j][e] = -INFINITY; s[j][e + 2] = -INFINITY; }
+              if (j * 8 + qd * 2 + e >= cnt) { s[j][e] = -INFINITY; s[j][e + 2] = -INFINITY; }
             }
         }
         // online softmax, row gq (and gq + 8)
@@ -479,51 +627,71 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       }
       consumer_bar();
     }
-    {
-      const int ctid = tid;  // 0..255 among consumers
-      if (whole) {
-        for (int idx = ctid; idx < Hq * D; idx += kConsumerWarps * 32) {
-          const int h = idx / D;
-          const float l = merge_ml[h * 2 + 1];
-          const float val = l > 0.f ? merge_o[idx] / l : 0.f;
-          if (p.a.out_f32) reinterpret_cast<float*>(p.a.out)[(int64_t)i * Hq * D + idx] = val;
-          else reinterpret_cast<__nv_bfloat16*>(p.a.out)[(int64_t)i * Hq * D + idx] = __float2bfloat16_rn(val);
+    if (whole) {
+      const int64_t obase = (int64_t)i * Hq * D;
+      for (int idx = tid; idx < Hq * D; idx += kConsumerWarps * 32) {
+        const int h = idx / D;
+        const float l = merge_ml[h * 2 + 1];
+        const float val = l > 0.f ? merge_o[idx] / l : 0.f;
+        if (p.a.out_f32) reinterpret_cast<float*>(p.a.out)[obase + idx] = val;
+        else reinterpret_cast<__nv_bfloat16*>(p.a.out)[obase + idx] = __float2bfloat16_rn(val);
+      }
+      consumer_bar();  // the merge buffer is reused by the next piece
+    } else {
+      const int first = cta_of(s_cum[i]), last = cta_of(s_cum[i + 1] - 1);
+      bool merged = false;
+      if (!has_next) {
+        // The block's final piece.  Usually every other piece of this sequence was published long
+        // ago (the rest of the sequence is some other block's first piece): then this block merges
+        // right away, taking its own piece from shared memory, and publishes nothing.
+        if (tid == 0) s_pend[4] = ld_acquire(p.a.tickets + i);
+        consumer_bar();
+        if (s_pend[4] == last - first) {
+          __threadfence();
+          combine_pieces(p.a.part_o, p.a.part_ml, p.a.out, p.a.out_f32, Hq, D, i, first, last, cta, merge_o, merge_ml, tid);
+          if (tid == 0) p.a.tickets[i] = 0;  // ready for the next launch
+          merged = true;
         }
-      } else {
+      }
+      if (!merged) {
+        // Publish this piece and take a ticket from the sequence's counter.  Nobody looks at the
+        // ticket before the block has streamed all its tiles: whoever took a sequence's last
+        // ticket merges its pieces then.
         const int64_t pslot = (int64_t)cta + i;
         float* po = p.a.part_o + pslot * Hq * D;
-        for (int idx = ctid; idx < Hq * D; idx += kConsumerWarps * 32) po[idx] = merge_o[idx];
-        if (ctid < Hq * 2) p.a.part_ml[pslot * Hq * 2 + ctid] = merge_ml[ctid];
-      }
-      if (ctid == 0) {
-        if (ta == 0) p.a.first_cta[i] = cta;
-        if (tb == tiles_i) p.a.last_cta[i] = cta;
+        for (int idx = tid; idx < Hq * D; idx += kConsumerWarps * 32) po[idx] = merge_o[idx];
+        if (tid < Hq * 2) p.a.part_ml[pslot * Hq * 2 + tid] = merge_ml[tid];
+        consumer_bar();  // orders every thread's stores before thread 0's fence; frees the merge buffer
+        if (tid == 0) {
+          __threadfence();
+          const int tk = atomicAdd(p.a.tickets + i, 1);
+          if (n_pend == 0) { pend_seq0 = i; pend_tk0 = tk; } else { pend_seq1 = i; pend_tk1 = tk; }
+        }
+        ++n_pend;
       }
     }
-    consumer_bar();  // the merge buffer is reused by the next piece
+    if (has_next) {
+#pragma unroll
+      for (int kk = 0; kk < KSTEPS; ++kk) {
+        qf[kk][0] = qn[kk][0]; qf[kk][2] = qn[kk][2];
+        if (!G_LE_8) { qf[kk][1] = qn[kk][1]; qf[kk][3] = qn[kk][3]; }
+      }
+    }
   }
-}
 
-// Merges the pieces of every sequence that was split over several blocks.
-__global__ void k_attn_combine(BcAttnArgs a, int Hq, int D) {
-  const int i = blockIdx.x;
-  const int first = a.first_cta[i], last = a.last_cta[i];
-  if (first == last) return;  // written directly by the attention kernel
-  for (int idx = threadIdx.x; idx < Hq * D; idx += blockDim.x) {
-    const int h = idx / D;
-    float mmax = -INFINITY;
-    for (int c = first; c <= last; ++c) mmax = fmaxf(mmax, a.part_ml[((int64_t)(c + i) * Hq + h) * 2]);
-    const float msafe = mmax == -INFINITY ? 0.f : mmax;
-    float num = 0.f, den = 0.f;
-    for (int c = first; c <= last; ++c) {
-      const int64_t ps = (int64_t)(c + i);
-      const float sc = exp2f(a.part_ml[(ps * Hq + h) * 2] - msafe);
-      num += sc * a.part_o[ps * Hq * D + idx];
-      den += sc * a.part_ml[(ps * Hq + h) * 2 + 1];
+  // ---- all tiles streamed: merge the sequences whose last ticket this block took -----------------
+  if (n_pend > 0) {
+    if (tid == 0) { s_pend[0] = pend_seq0; s_pend[1] = pend_tk0; s_pend[2] = pend_seq1; s_pend[3] = pend_tk1; }
+    consumer_bar();
+    for (int k = 0; k < n_pend; ++k) {
+      const int seq = s_pend[2 * k], tk = s_pend[2 * k + 1];
+      const int first = cta_of(s_cum[seq]), last = cta_of(s_cum[seq + 1] - 1);
+      if (tk == last - first) {
+        __threadfence();
+        combine_pieces(p.a.part_o, p.a.part_ml, p.a.out, p.a.out_f32, Hq, D, seq, first, last, -1, nullptr, nullptr, tid);
+        if (tid == 0) p.a.tickets[seq] = 0;  // ready for the next launch
+      }
     }
-    const float val = den > 0.f ? num / den : 0.f;
-    if (a.out_f32) reinterpret_cast<float*>(a.out)[(int64_t)i * Hq * D + idx] = val;
-    else reinterpret_cast<__nv_bfloat16*>(a.out)[(int64_t)i * Hq * D + idx] = __float2bfloat16_rn(val);
   }
 }
 
@@ -581,6 +749,17 @@ __global__ void k_attn_reference(BcMeta m, BcGeom g, BcAttnArgs a) {
   }
 }
 
+FastDiv make_fast_div(uint32_t d) {
+  FastDiv f;
+  if (d <= 1) { f.mul = 0; f.sh1 = 0; f.sh2 = 0; return f; }
+  uint32_t l = 0;
+  while ((1ull << l) < d) ++l;  // ceil(log2 d)
+  f.mul = (uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1);
+  f.sh1 = 1;
+  f.sh2 = l - 1;
+  return f;
+}
+
 template <int D, bool G8>
 cudaError_t launch_pipe(const PipeParams& p, cudaStream_t s) {
   k_attn_pipe<D, G8><<<p.a.ctas, kPipeThreads, PipeSmem<D>::kTotal, s>>>(p);
@@ -611,7 +790,10 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   p.scale_log2 = a.sm_scale * 1.4426950408889634f;
   p.n_groups = kConsumerWarps / g.kv_heads;
   p.rows_per_tile = 16 * p.n_groups;
+  p.tile_shift = 0;
+  while ((1 << p.tile_shift) < p.rows_per_tile) ++p.tile_shift;
   p.G = g.q_heads / g.kv_heads;
+  p.div_ps = make_fast_div((uint32_t)g.page_size);
   cudaError_t e;
   if (ev_start) { e = cudaEventRecord(ev_start, s); if (e != cudaSuccess) return e; }
   const bool g8 = p.G <= 8;
@@ -619,9 +801,8 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   else e = g8 ? launch_pipe<64, true>(p, s) : launch_pipe<64, false>(p, s);
   if (e != cudaSuccess) return e;
   if (ev_stop) { e = cudaEventRecord(ev_stop, s); if (e != cudaSuccess) return e; }
-  k_attn_combine<<<a.n, 256, 0, s>>>(a, g.q_heads, g.head_dim);
-  *launches = 2;
-  return cudaGetLastError();
+  *launches = 1;
+  return cudaSuccess;
 }
 
 cudaError_t bc_launch_attn_reference(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, cudaStream_t s) {

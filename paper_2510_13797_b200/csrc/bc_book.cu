@@ -65,6 +65,28 @@ struct ErrLatch {
   }
 };
 
+// Copies the K and V rows of n batch items into their pool rows with the whole block, 16 bytes
+// per thread and step, applying the chunk permutation of the store layout.  Items with
+// dst_row < 0 (failed validation) are skipped.  Used by the single-block kernels that have just
+// computed dst_row/dst_pos (their global writes are visible to the block after __syncthreads).
+__device__ void block_write_rows(const BcGeom& g, uint8_t* __restrict__ pool_layer, const int32_t* dst_row,
+                                 const int32_t* dst_pos, const uint8_t* __restrict__ k,
+                                 const uint8_t* __restrict__ v, int n) {
+  const int chunks_per_head = g.head_row_bytes >> 4;
+  const int per_side = g.kv_heads * chunks_per_head;
+  const int per_item = 2 * per_side;
+  for (int idx = threadIdx.x; idx < n * per_item; idx += blockDim.x) {
+    const int i = idx / per_item, r = idx - i * per_item;
+    const int row = dst_row[i];
+    if (row < 0) continue;
+    const int which = r / per_side, rem = r - which * per_side;
+    const int h = rem / chunks_per_head, j = rem - h * chunks_per_head;
+    const uint8_t* src = (which ? v : k) + ((int64_t)i * g.kv_heads + h) * g.head_row_bytes + (j << 4);
+    *reinterpret_cast<uint4*>(pool_layer + (int64_t)row * g.entry_bytes + bc_chunk_offset(g, which, h, j, dst_pos[i])) =
+        *reinterpret_cast<const uint4*>(src);
+  }
+}
+
 __global__ void k_init(BcMeta m) {
   const int tid = blockIdx.x * blockDim.x + threadIdx.x, nth = gridDim.x * blockDim.x;
   for (int i = tid; i < m.num_pages; i += nth) m.free_stack[i] = m.num_pages - 1 - i;
@@ -128,7 +150,7 @@ k_open(BcMeta m, const int32_t* __restrict__ slots, const int32_t* __restrict__ 
 
 __global__ void __launch_bounds__(kBookThreads, 1)
 k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
-              int32_t* __restrict__ dst_row, int32_t* __restrict__ dst_pos) {
+              int32_t* dst_row, int32_t* dst_pos, BcGeom g, uint8_t* pool_layer, const uint8_t* k, const uint8_t* v) {
   __shared__ int sh_first;
   ErrLatch latch; latch.init(&sh_first);
   const int top0 = *m.free_top;
@@ -179,13 +201,15 @@ k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
   latch.commit(m, my_item, my_code, my_slot, call);
   __syncthreads();
   if (threadIdx.x == 0) *m.free_top = top0 - sh_used;
+  if (k != nullptr) block_write_rows(g, pool_layer, dst_row, dst_pos, k, v, n);  // layer 0's rows, same launch
 }
 
 // phase & 1: validate, allocate the beacon slot, fill dst_row/dst_pos (dst_row < 0: item failed).
 // phase & 2: for items with dst_row >= 0, push the window pages, clear the window, count the beacon.
 __global__ void __launch_bounds__(kBookThreads, 1)
 k_compress_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
-                int32_t* __restrict__ dst_row, int32_t* __restrict__ dst_pos, int phase) {
+                int32_t* dst_row, int32_t* dst_pos, int phase, BcGeom g, uint8_t* pool_layer,
+                const uint8_t* k, const uint8_t* v) {
   __shared__ int sh_first;
   __shared__ int sh_used;
   const int ps = m.page_size;
@@ -259,6 +283,7 @@ k_compress_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call
   }
   __syncthreads();
   if (threadIdx.x == 0) *m.free_top = top;
+  if (k != nullptr) block_write_rows(g, pool_layer, dst_row, dst_pos, k, v, n);  // the beacon rows, same launch
 }
 
 __global__ void __launch_bounds__(kBookThreads, 1)
@@ -391,13 +416,17 @@ cudaError_t bc_launch_open(const BcMeta& m, const int32_t* slots, const int32_t*
   return cudaGetLastError();
 }
 cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
-                                  int32_t* dst_pos, cudaStream_t s) {
-  k_append_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos);
+                                  int32_t* dst_pos, const BcGeom& g, uint8_t* pool_layer, const void* k, const void* v,
+                                  cudaStream_t s) {
+  k_append_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)k,
+                                           (const uint8_t*)v);
   return cudaGetLastError();
 }
 cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
-                                    int32_t* dst_pos, int phase, cudaStream_t s) {
-  k_compress_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, phase);
+                                    int32_t* dst_pos, int phase, const BcGeom& g, uint8_t* pool_layer, const void* k,
+                                    const void* v, cudaStream_t s) {
+  k_compress_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, phase, g, pool_layer,
+                                             (const uint8_t*)k, (const uint8_t*)v);
   return cudaGetLastError();
 }
 cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_t call, cudaStream_t s) {

@@ -48,11 +48,15 @@ __host__ __device__ __forceinline__ int bc_chunk_offset(const BcGeom& g, int whi
 cudaError_t bc_launch_init(const BcMeta& m, cudaStream_t s);
 cudaError_t bc_launch_open(const BcMeta& m, const int32_t* slots, const int32_t* plens, const int32_t* cs,
                            int n, int64_t call, cudaStream_t s);
+// k, v non-null: the same launch also writes the rows into pool_layer (what bc_launch_write_rows
+// does), which saves a launch when the batch is small enough for one thread block to copy.
 cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
-                                  int32_t* dst_pos, cudaStream_t s);
+                                  int32_t* dst_pos, const BcGeom& g, uint8_t* pool_layer, const void* k, const void* v,
+                                  cudaStream_t s);
 // phase bit 1: allocate the beacon slot; phase bit 2: evict the window and bump the counters
 cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
-                                    int32_t* dst_pos, int phase, cudaStream_t s);
+                                    int32_t* dst_pos, int phase, const BcGeom& g, uint8_t* pool_layer, const void* k,
+                                    const void* v, cudaStream_t s);
 cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_t call, cudaStream_t s);
 cudaError_t bc_launch_write_rows(const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
                                  const void* k, const void* v, int n, cudaStream_t s);
@@ -74,13 +78,13 @@ struct BcAttnArgs {
   float sm_scale;
   float* part_o;         // [(ctas + n)][q_heads][head_dim]
   float* part_ml;        // [(ctas + n)][q_heads][2]
-  int32_t* first_cta;    // [n]
-  int32_t* last_cta;     // [n]
+  int32_t* tickets;      // [n] pieces of each sequence published so far; zero between launches
   int32_t ctas;
 };
 // Configures the kernels once per process/device (shared-memory opt-in).  Returns the SM count.
 cudaError_t bc_attn_setup(int* sm_count);
-// Launches the pipelined decode-attention kernel and the split combine; *launches gets the count.
+// Launches the pipelined decode-attention kernel (the split combine is part of it); *launches gets
+// the number of kernels launched.
 cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, cudaStream_t s,
                            cudaEvent_t ev_start, cudaEvent_t ev_stop, int* launches);
 // Slow device reference (one warp per query head).

@@ -29,7 +29,7 @@
 namespace {
 
 constexpr int kConsumerWarps = 8;
-constexpr int kPipeThreads = (kConsumerWarps + 1) * 32;  // consumer warps and the producer warp
+constexpr int kPipeThreads = (kConsumerWarps + 2) * 32;  // consumer warps, producer warp, service warp
 constexpr int kPlanMax = BC_MAX_ATTN_BATCH;
 constexpr uint32_t kSpinLimit = 1u << 21;  // polls of try_wait before giving up
 constexpr int kPidAhead = 4;               // tiles of page-id lookahead of the producer
@@ -60,10 +60,19 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 // 1-D bulk asynchronous copy global -> this block's shared memory, completing on an mbarrier.
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
+// `policy` is an L2 cache policy: the K/V stream is read once per launch and is larger than L2,
+// so it is marked evict-first and leaves the lengths, page tables, queries and partial results
+// of the previous launches resident.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
 }
 // 4-byte asynchronous copy global -> shared (page-id prefetch), grouped by commit / wait_group.
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
@@ -163,7 +172,8 @@ struct PipeSmem {
   // descriptors of the tiles ahead: (kPidAhead + 1) slots of {rows, first position, first page,
   // unused} followed by the page ids of the tile
   static constexpr int kBarOff = kPidOff + (kPidAhead + 1) * kPidSlot * 4;
-  static constexpr int kMiscOff = kBarOff + 2 * kStages * 8;  // abort flag, pending tickets
+  // barriers: full[kStages], empty[kStages], piece published, ticket taken
+  static constexpr int kMiscOff = kBarOff + 2 * kStages * 8 + 16;  // abort flag, pending tickets
   static constexpr int kTotal = kMiscOff + 32;
 };
 
@@ -259,11 +269,13 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   int* s_cum = s_wcol + kPlanMax;   // [n + 1] exclusive prefix sums of tiles
   int* s_desc = reinterpret_cast<int*>(smem + L::kPidOff);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L::kMiscOff);
-  volatile int* s_pend = s_abort + 1;  // {sequence, ticket} of up to two published pieces; [4]: peeked count
+  volatile int* s_pend = s_abort + 1;  // {sequence, ticket} of the first and of the final piece; [4]: peeked count
   const uint32_t ring = smem_u32(smem);
   const uint32_t desc_ring = smem_u32(smem + L::kPidOff);
   const uint32_t bar_full = smem_u32(smem + L::kBarOff);
   const uint32_t bar_empty = bar_full + NSTAGE * 8;
+  const uint32_t bar_pub = bar_empty + NSTAGE * 8;  // the consumers have stored the block's first piece
+  const uint32_t bar_tk = bar_pub + 8;              // the service warp has taken that piece's ticket
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n = p.a.n, T = p.rows_per_tile, TS = p.tile_shift, E = p.g.entry_bytes, ps = p.g.page_size;
@@ -274,6 +286,8 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       mbar_init(bar_full + s * 8, 1);
       mbar_init(bar_empty + s * 8, kConsumerWarps);
     }
+    mbar_init(bar_pub, kConsumerWarps);
+    mbar_init(bar_tk, 1);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_proxy_async();
@@ -325,12 +339,40 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     seq0 = lo;
   }
 
+  // The block's first piece: if it covers only part of its sequence and more pieces follow, the
+  // service warp publishes it (fence, then ticket), because the fence has to wait until the
+  // piece's stores have reached L2 -- microseconds while every SM is streaming -- and a consumer
+  // warp that waited there would stall the whole pipeline between pieces.
+  bool svc_publishes;
+  {
+    const int tiles0 = s_cum[seq0 + 1] - s_cum[seq0], ta0 = g0 - s_cum[seq0];
+    const int tb0 = min(tiles0, ta0 + (g1 - g0));
+    svc_publishes = !(ta0 == 0 && tb0 == tiles0) && (g0 + (tb0 - ta0) < g1);
+  }
+  if (warp == kConsumerWarps + 1) {
+    // ================================ service warp =============================================
+    if (svc_publishes) {
+      const bool ok = bounded_wait(bar_pub, 0, s_abort);  // every consumer warp has stored its share
+      if (lane == 0) {
+        if (ok) {
+          __threadfence();
+          s_pend[1] = atomicAdd(p.a.tickets + seq0, 1);
+          s_pend[0] = seq0;
+        } else {
+          s_pend[0] = -1;
+        }
+        mbar_arrive(bar_tk);
+      }
+    }
+    return;
+  }
   if (warp == kConsumerWarps) {
     // ================================ producer warp ============================================
     // describe(gt) runs kPidAhead tiles ahead of the copies: it works out which rows tile gt holds,
     // writes {rows, first position, first page} to a small descriptor ring and starts 4-byte
     // asynchronous copies of the tile's page-table entries into the same slot.  Issuing the bulk
     // copies of a tile then takes a handful of instructions and never waits on the page table.
+    const uint64_t stream_policy = l2_policy_evict_first();
     int fi = seq0;
     int f_P, f_nb, f_w, f_tp, f_tpb, f_bcol, f_wcol;
     const int32_t* f_tab;
@@ -392,7 +434,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
           const int lo = max(p0, pg * ps), hi = min(p0 + nrows, pg * ps + ps);
           if (lo >= hi) break;
           const uint8_t* src = p.a.pool_layer + ((int64_t)d[4 + k] * ps + (lo - pg * ps)) * E;
-          bulk_g2s(stage_base + (uint32_t)(lo - p0) * (uint32_t)E, src, (uint32_t)(hi - lo) * (uint32_t)E, full);
+          bulk_g2s(stage_base + (uint32_t)(lo - p0) * (uint32_t)E, src, (uint32_t)(hi - lo) * (uint32_t)E, full, stream_policy);
         }
       }
       __syncwarp();  // the slot read above may be rewritten by the describe() calls below
@@ -443,8 +485,8 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   int i = seq0;
   int it = 0;
   int gt = g0;
-  int n_pend = 0;  // pieces this block has published; thread 0 keeps their tickets
-  int pend_seq0 = -1, pend_tk0 = 0, pend_seq1 = -1, pend_tk1 = 0;
+  int pend_seq = -1, pend_tk = 0;  // thread 0: ticket of the block's final piece, if it had to be published
+  bool published_last = false;
   uint32_t qf[KSTEPS][4];
   load_q(qf, seq0);
   while (gt < g1) {
@@ -661,13 +703,20 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
         float* po = p.a.part_o + pslot * Hq * D;
         for (int idx = tid; idx < Hq * D; idx += kConsumerWarps * 32) po[idx] = merge_o[idx];
         if (tid < Hq * 2) p.a.part_ml[pslot * Hq * 2 + tid] = merge_ml[tid];
-        consumer_bar();  // orders every thread's stores before thread 0's fence; frees the merge buffer
-        if (tid == 0) {
-          __threadfence();
-          const int tk = atomicAdd(p.a.tickets + i, 1);
-          if (n_pend == 0) { pend_seq0 = i; pend_tk0 = tk; } else { pend_seq1 = i; pend_tk1 = tk; }
+        if (has_next) {
+          // the block's first piece: hand it to the service warp and go on streaming
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_pub);
+          consumer_bar();  // frees the merge buffer
+        } else {
+          consumer_bar();  // orders every thread's stores before thread 0's fence
+          if (tid == 0) {
+            __threadfence();
+            pend_tk = atomicAdd(p.a.tickets + i, 1);
+            pend_seq = i;
+          }
+          published_last = true;
         }
-        ++n_pend;
       }
     }
     if (has_next) {
@@ -680,17 +729,20 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   }
 
   // ---- all tiles streamed: merge the sequences whose last ticket this block took -----------------
-  if (n_pend > 0) {
-    if (tid == 0) { s_pend[0] = pend_seq0; s_pend[1] = pend_tk0; s_pend[2] = pend_seq1; s_pend[3] = pend_tk1; }
+  if (svc_publishes) bounded_wait(bar_tk, 0, s_abort);
+  if (published_last) {
+    if (tid == 0) { s_pend[2] = pend_seq; s_pend[3] = pend_tk; }
     consumer_bar();
-    for (int k = 0; k < n_pend; ++k) {
-      const int seq = s_pend[2 * k], tk = s_pend[2 * k + 1];
-      const int first = cta_of(s_cum[seq]), last = cta_of(s_cum[seq + 1] - 1);
-      if (tk == last - first) {
-        __threadfence();
-        combine_pieces(p.a.part_o, p.a.part_ml, p.a.out, p.a.out_f32, Hq, D, seq, first, last, -1, nullptr, nullptr, tid);
-        if (tid == 0) p.a.tickets[seq] = 0;  // ready for the next launch
-      }
+  }
+  for (int k = 0; k < 2; ++k) {
+    if (k == 0 ? !svc_publishes : !published_last) continue;
+    const int seq = s_pend[2 * k], tk = s_pend[2 * k + 1];
+    if (seq < 0) continue;
+    const int first = cta_of(s_cum[seq]), last = cta_of(s_cum[seq + 1] - 1);
+    if (tk == last - first) {
+      __threadfence();
+      combine_pieces(p.a.part_o, p.a.part_ml, p.a.out, p.a.out_f32, Hq, D, seq, first, last, -1, nullptr, nullptr, tid);
+      if (tid == 0) p.a.tickets[seq] = 0;  // ready for the next launch
     }
   }
 }

@@ -69,7 +69,8 @@ bool config_ok(const bc_config* c, bc_status* why) {
   return true;
 }
 
-constexpr size_t kFusedRowBytes = 512u << 10;  // rows of a batch that the bookkeeping block copies itself
+constexpr size_t kFusedRowBytes = 32u << 10;  // rows of a batch that the bookkeeping block copies itself (a
+                                                // single block moves more than this slower than a second launch)
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
@@ -305,7 +306,7 @@ bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n,
   int32_t* row = work_ptr<int32_t>(c, c->wl.append_row);
   int32_t* pos = work_ptr<int32_t>(c, c->wl.append_pos);
   cudaStream_t s = (cudaStream_t)stream;
-  // One thread block copies up to kFusedRowBytes in about the time a second launch would cost.
+  // Small batches: the bookkeeping block also copies the rows and a launch is saved.
   const bool fused = layer == 0 && (size_t)n * c->geom.entry_bytes <= kFusedRowBytes;
   if (layer == 0) {
     BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, ++c->calls, row, pos, c->geom, layer_base(c, 0),

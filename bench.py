@@ -97,80 +97,17 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------ one ratio on the GPU
-class RatioRunner:
-    """Holds one cache (batch B at ratio c) and drives decode steps through the C ABI."""
+def make_runner(w, device, seed_offset=0):
+    """A DecodeDriver (one cache, batch B at ratio c, driven through the C ABI) plus the timed passes."""
+    import torch
+    from paper_2510_13797_b200.driver import DecodeDriver
+    r = type("RatioRunner", (_Passes, DecodeDriver), {})(w, device, seed_offset)
+    r.torch = torch
+    return r
 
-    def __init__(self, w, device, seed_offset=0):
-        import torch
-        from paper_2510_13797_b200 import binding as B
-        from paper_2510_13797_b200.workloads import InputStream
-        self.torch, self.B, self.w, self.dev = torch, B, w, device
-        c, ps, Bn = w.cs[0], w.page_size, w.batch
-        P, T = w.prompt_lens[0], w.steps
-        self.c, self.P, self.T, self.n = c, P, T, Bn
-        cd = lambda a, b: -(-a // b)
-        if c > 1:
-            pages_per_seq = cd(P, ps) + cd(c, ps) + cd(cd(T, c), ps) + 1
-        else:
-            pages_per_seq = cd(P + T, ps) + 1
-        self.cache = B.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, c, ps, max_seqs=Bn,
-                             num_pages=Bn * pages_per_seq, max_pages_per_seq=pages_per_seq, device=device)
-        self.slots = torch.arange(Bn, dtype=torch.int32, device=device)
-        self.plens = torch.tensor(w.prompt_lens, dtype=torch.int32, device=device)
-        self.cu = torch.tensor([0] + list(__import__("itertools").accumulate(w.prompt_lens)), dtype=torch.int32,
-                               device=device)
-        stream = InputStream(w, device)
-        self.pk, self.pv = stream.prompt_kv(0)
-        self.ring = max(c, 16)                         # distinct step inputs, reused cyclically
-        self.q, self.k, self.v = stream.step_chunk(0, seed_offset, self.ring)
-        self.bq, self.bk, self.bv = stream.beacon_chunk(0, seed_offset, 4)
-        self.out = self.cache.new_out(Bn)
-        self.out_b = self.cache.new_out(Bn)
-        self.t = 0
-        self.opened = False
-        # pinned host copies for the end-to-end pass
-        self.h = None
 
-    # -- state -------------------------------------------------------------------------------
-    def reset_to(self, t_target):
-        """(Re)opens the batch, stores the prompts and replays appends/compressions up to t_target."""
-        c = self.cache
-        if self.opened:
-            c.bc_seq_close(self.slots)
-        c.bc_seq_open(self.slots, self.plens)
-        c.bc_prefill(0, self.slots, self.cu, int(self.cu[-1]), self.pk, self.pv)
-        self.opened, self.t = True, 0
-        while self.t < t_target:
-            j = self.t % self.ring
-            c.bc_append(0, self.slots, self.k[j], self.v[j])
-            self.t += 1
-            if self.c > 1 and self.t % self.c == 0:
-                b = (self.t // self.c) % 4
-                c.bc_compress(0, self.slots, self.bk[b], self.bv[b])
-
-    def step(self):
-        """One decode step of the whole batch through the device-pointer calls."""
-        c, j = self.cache, self.t % self.ring
-        c.bc_append(0, self.slots, self.k[j], self.v[j])
-        c.bc_decode_attn(0, self.slots, self.q[j], self.out, self.w.sm_scale)
-        self.t += 1
-        if self.c > 1 and self.t % self.c == 0:
-            b = (self.t // self.c) % 4
-            c.bc_decode_attn(0, self.slots, self.bq[b], self.out_b, self.w.sm_scale, self.bk[b], self.bv[b])
-            c.bc_compress(0, self.slots, self.bk[b], self.bv[b])
-
-    def step_host(self):
-        """The same step through the host-buffer entry points (H2D of q,k,v and D2H of out inside)."""
-        if self.h is None:
-            pin = lambda t: t.cpu().pin_memory()
-            self.h = dict(q=pin(self.q), k=pin(self.k), v=pin(self.v), bq=pin(self.bq), bk=pin(self.bk),
-                          bv=pin(self.bv), out=pin(self.out), out_b=pin(self.out_b))
-        c, j, h = self.cache, self.t % self.ring, self.h
-        c.bc_decode_step_host(0, self.slots, h["q"][j], h["k"][j], h["v"][j], h["out"], self.w.sm_scale)
-        self.t += 1
-        if self.c > 1 and self.t % self.c == 0:
-            b = (self.t // self.c) % 4
-            c.bc_compress_step_host(0, self.slots, h["bq"][b], h["bk"][b], h["bv"][b], h["out_b"], self.w.sm_scale)
+class _Passes:
+    """Accounting and timed passes over a DecodeDriver."""
 
     def host_bytes_per_step(self):
         w = self.w
@@ -268,11 +205,6 @@ class RatioRunner:
         torch.cuda.synchronize()
         return e0.elapsed_time(e1)
 
-    def check_error(self):
-        code, slot, call = self.cache.bc_poll_error()
-        if code != 0:
-            raise RuntimeError(f"device-side error {self.B.STATUS_NAMES.get(code, code)} slot {slot} call {call}")
-
 
 # ------------------------------------------------------------------------------ the oracle on host cores
 def oracle_sample(w, t_mid, seqs, steps, seed=0):
@@ -359,7 +291,7 @@ def run_profile_case(args):
     mid = entries_attended(w.prompt_lens[0], w.steps // 2, c)
     w = make_workload("sweep", c=c, prompt_lens=[mid] * w.batch, gen_lens=[4 * max(c, 16) + args.steps + 64] * w.batch)
     torch.cuda.set_device(0)
-    r = RatioRunner(w, torch.device("cuda", 0))
+    r = make_runner(w, torch.device("cuda", 0))
     r.reset_to(0)
     ms, n, nbytes, region = r.timed_kernels(args.steps, max(args.warmup, 3))
     r.check_error()
@@ -389,6 +321,7 @@ def main():
 
     import torch
     import torch.distributed as dist
+    from paper_2510_13797_b200 import sharding
     from paper_2510_13797_b200.workloads import make_workload
 
     K, W = args.steps, max(args.warmup, 3)
@@ -420,7 +353,7 @@ def main():
     for c in sweep:
         w = make_workload("sweep", c=c)
         T = w.steps
-        r = RatioRunner(w, dev, seed_offset=rank)
+        r = make_runner(w, dev, seed_offset=sharding.rank_seed_offset(0, rank))
         cyc = c if c > 1 else 16
         t_mid = max(0, ((T - K) // 2 // cyc) * cyc)
         # pass A: device-resident inputs, CUDA-graph replays: the headline time
@@ -436,10 +369,7 @@ def main():
         barrier()
         h_ms = r.timed_host(K, W)
         r.check_error()
-        if world > 1:
-            tt = torch.tensor([ms, h_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            ms, h_ms = float(tt[0]), float(tt[1])
+        ms, h_ms = sharding.max_over_ranks([ms, h_ms], device=dev)      # the slowest rank counts
         reg, bea = r.kv_bytes(t_begin, K)
         live, unc = r.cache_bytes(t_begin + K // 2)
         end_live, end_unc = r.cache_bytes(T)

@@ -45,6 +45,22 @@ def entries_beacon_query(P, t, c):
     return P + (t // c - 1) + c
 
 
+# DRAM traffic of one attention launch over algorithmic KV bytes, per ratio: ncu
+# dram__bytes_read.sum + dram__bytes_write.sum with warm caches (--cache-control none) on the small
+# case of each ratio (--profile-case C: same bytes per launch and page size as mid-generation), for
+# the library version named here; see profiles/.  Slightly below 1: part of the stream stays in L2
+# from the previous step.  A different library version invalidates the figures (traffic: null).
+TRAFFIC_FOR_VERSION = 110
+TRAFFIC_OVER_ALGORITHMIC = {2: 0.996, 4: 0.981, 8: 0.961, 16: 0.946, 32: 0.979}
+
+
+def traffic_per_launch(c, algorithmic_bytes):
+    from paper_2510_13797_b200 import binding
+    if binding.lib().bc_version() != TRAFFIC_FOR_VERSION or c not in TRAFFIC_OVER_ALGORITHMIC:
+        return None
+    return TRAFFIC_OVER_ALGORITHMIC[c] * algorithmic_bytes
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -191,6 +207,26 @@ class _Passes:
         assert got == n_launch, (got, n_launch)
         reg, bea = self.kv_bytes(t_begin, K)
         return ms, got, reg + bea, e0.elapsed_time(e1)
+
+    def timed_attn_stream(self, n_launch, W):
+        """n_launch decode-attention launches back to back on the cache as it stands (nothing else in
+        the timed region), one CUDA-event pair around all of them on the launching stream.  Returns
+        (ms, launches, algorithmic KV bytes): the kernel's average duration without the event
+        overhead that bracketing every single launch adds."""
+        torch = self.torch
+        live = self.P + (self.t // self.c + self.t % self.c if self.c > 1 else self.t)
+        for i in range(max(W, 3)):
+            self.cache.bc_decode_attn(0, self.slots, self.q[i % self.ring], self.out, self.w.sm_scale)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.nvtx.range_push("attn_stream")
+        e0.record()
+        for i in range(n_launch):
+            self.cache.bc_decode_attn(0, self.slots, self.q[i % self.ring], self.out, self.w.sm_scale)
+        e1.record()
+        torch.cuda.synchronize()
+        torch.cuda.nvtx.range_pop()
+        return e0.elapsed_time(e1), n_launch, n_launch * live * self.w.entry_bytes * self.n
 
     def timed_host(self, K, W):
         torch = self.torch
@@ -363,7 +399,8 @@ def main():
         # pass B: plain launches, every attention kernel bracketed by events: the roofline figures
         Kp = min(K, 256)
         r.reset_to(max(0, t_mid - W))
-        k_ms, k_n, k_bytes, plain_ms = r.timed_kernels(Kp, W)
+        b_ms, b_n, b_bytes, plain_ms = r.timed_kernels(Kp, W)
+        k_ms, k_n, k_bytes = r.timed_attn_stream(Kp, W)
         # pass C: host buffers through the C ABI, copies inside the timed region
         r.reset_to(max(0, t_mid - W))
         barrier()
@@ -379,6 +416,8 @@ def main():
             "plain_launch_ms_per_step": plain_ms / Kp,
             "kv_gbs_step": (reg + bea) / (ms * 1e-3) / 1e9,
             "attn_kernel_us": 1e3 * k_ms / k_n, "attn_kernel_gbs": k_bytes / (k_ms * 1e-3) / 1e9,
+            "attn_kernel_us_bracketed": 1e3 * b_ms / b_n, "attn_kernel_gbs_bracketed": b_bytes / (b_ms * 1e-3) / 1e9,
+            "attn_dram_traffic_per_launch": traffic_per_launch(c, k_bytes / k_n),
             "attn_frac_of_peak": k_bytes / (k_ms * 1e-3) / 1e9 / peak,
             "attn_pct_of_8tbs": 100 * k_bytes / (k_ms * 1e-3) / 8e12,
             "kv_bytes_per_step": (reg + bea) / K, "cache_bytes_mid": live, "uncompressed_bytes_mid": unc,
@@ -404,6 +443,8 @@ def main():
     B = 64
     value = world * B * n_c * K / (total_ms * 1e-3)
     achieved = kern_bytes / (kern_ms * 1e-3) / 1e9
+    tr = [r["attn_dram_traffic_per_launch"] for r in rows if r["c"] > 1]
+    traffic = None if any(x is None for x in tr) else sum(tr) / len(tr)      # equal launch counts per ratio
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -418,7 +459,11 @@ def main():
         "gpu_launches": int(total_launches),
         "clocks": clocks,
         "roofline": {"bound": "hbm", "kernel": "k_attn_pipe", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                     "frac": achieved / peak, "traffic": traffic, "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": kern_bytes / kern_launches,
+                     "timing": "CUDA events around back-to-back launches of the kernel alone at each ratio "
+                               "(mid-generation cache); sweep[].attn_kernel_us_bracketed brackets every single "
+                               "launch inside plain decode steps instead",
                      "launches_timed": int(kern_launches),
                      "min_frac_over_c": min(r["attn_frac_of_peak"] for r in rows if r["c"] > 1),
                      "pct_of_8tbs": 100 * achieved * 1e9 / 8e12},

@@ -175,7 +175,7 @@ BC_API bc_status bc_decode_attn(bc_cache* cache, int32_t layer, const int32_t* s
  * and a stream by its host application and must not go to the CUDA allocator behind the host's
  * back, or a latency-critical loop in which an allocation (which may synchronise the device) is not
  * acceptable.  Such callers already own the cache buffers, but the split-K
- * scratch (per-piece partial outputs, their running max and sum, and the first/last block of every
+ * scratch (per-piece partial outputs, their running max and sum, and one ticket counter per
  * sequence) has to live somewhere.  Here it lives in a fixed array inside the library image:
  * about 4.9 MB of device memory that every GPU which loads the library keeps until the process
  * exits.  The call itself performs no device or host allocation and calls no allocating routine.
@@ -188,8 +188,9 @@ BC_API bc_status bc_decode_attn(bc_cache* cache, int32_t layer, const int32_t* s
  * The first call on each device looks up the device address of the built-in array (once per
  * device, with that device current); make that first call outside any stream capture.  All calls,
  * from all caches and streams of the process, share the one array: it still holds the previous
- * call's partials when the next call starts (every element a call reads it has written first, so
- * nothing needs clearing), and two calls whose kernels overlap on the GPU race on it.  Issue them
+ * call's partials when the next call starts (every partial a call reads it has written first,
+ * and every call returns the ticket counters to zero, so nothing needs clearing), and two calls
+ * whose kernels overlap on the GPU race on it.  Issue them
  * on one stream, or order them with events. */
 BC_API bc_status bc_decode_attn_static(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                                        const void* q, void* out, float sm_scale, const void* extra_k,

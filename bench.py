@@ -336,6 +336,319 @@ def run_profile_case(args):
                       "kv_bytes_per_launch": nbytes / n, "plain_ms_per_step": region / args.steps}))
 
 
+# ------------------------------------------------------------------------------ the other configurations
+def _event_pair(torch):
+    return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+
+def report_cfg2(args):
+    """Benchmark configs[1]: batch 32, 12/2 heads, prompt 256, 4096 steps, c = 16.  ~13 MB of KV
+    per step: L2-resident and launch-bound, so the figures are microseconds per call."""
+    import torch
+    from paper_2510_13797_b200.workloads import make_workload
+    torch.cuda.set_device(0)
+    w = make_workload("cfg2")
+    r = make_runner(w, torch.device("cuda", 0))
+    K = max(16, (min(args.steps, 1024) // 16) * 16)
+    t_mid = ((w.steps - K) // 2 // 16) * 16
+    r.reset_to(t_mid - 32)
+    ms, t_begin, launches = r.timed_graph(K, 16)
+    reg, bea = r.kv_bytes(t_begin, K)
+    a_ms, a_n, a_bytes = r.timed_attn_stream(256, 8)
+    # bc_append and bc_compress alone: plain launches, one event pair around each call
+    app, comp = [], []
+    for _ in range(4 * 16):
+        j = r.t % r.ring
+        e0, e1 = _event_pair(torch)
+        e0.record(); r.cache.bc_append(0, r.slots, r.k[j], r.v[j]); e1.record()
+        app.append((e0, e1))
+        r.t += 1
+        if r.t % 16 == 0:
+            bsel = (r.t // 16) % 4
+            e0, e1 = _event_pair(torch)
+            e0.record(); r.cache.bc_compress(0, r.slots, r.bk[bsel], r.bv[bsel]); e1.record()
+            comp.append((e0, e1))
+    torch.cuda.synchronize()
+    r.check_error()
+    med = lambda prs: statistics.median(1e3 * a.elapsed_time(b_) for a, b_ in prs)
+    live, unc = r.cache_bytes(t_begin + K // 2)
+    print(json.dumps({
+        "workload": "cfg2: 1 layer, B=32, 12/2 heads, D=128, P=256, T=4096, c=16, page 16, keys pre-scaled, sm_scale 1",
+        "steps": K, "t_window": [t_begin, t_begin + K], "us_per_step_graph": 1e3 * ms / K,
+        "tokens_per_s": w.batch * K / (ms * 1e-3), "kv_bytes_per_step": (reg + bea) / K,
+        "kv_gbs_step": (reg + bea) / (ms * 1e-3) / 1e9,
+        "us_per_bc_decode_attn": 1e3 * a_ms / a_n, "attn_kernel_gbs": a_bytes / (a_ms * 1e-3) / 1e9,
+        "us_per_bc_append_bracketed": med(app), "us_per_bc_compress_bracketed": med(comp),
+        "cache_bytes_mid": live, "uncompressed_bytes_mid": unc, "gpu_launches": int(launches),
+        "note": "13 MB of KV per step stays in L2: the HBM roofline does not bound this configuration"}))
+
+
+def report_ragged(args):
+    """Benchmark configs[3]: batch 128, 12/2 heads, page 16; prompt U[64,1024], generation
+    U[1024,32768], c from {4,8,16} per sequence.  The whole run, plain launches: sequences finish at
+    their own step and free their pages on the device."""
+    import numpy as np
+    import torch
+    from paper_2510_13797_b200 import binding as B
+    from paper_2510_13797_b200.workloads import InputStream, make_workload
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = make_workload("ragged")
+    Bn, ps = w.batch, w.page_size
+    P, T, C = np.array(w.prompt_lens), np.array(w.gen_lens), np.array(w.cs)
+    cd = lambda a, b_: -(-a // b_)
+    pps = cd(P, ps) + cd(C, ps) + cd(cd(T, C), ps) + 1
+    cache = B.Cache(1, w.kv_heads, w.q_heads, w.head_dim, 1, ps, max_seqs=Bn, num_pages=int(pps.sum()),
+                    max_pages_per_seq=int(pps.max()), device=dev)
+    stream = InputStream(w, dev)
+    pk, pv = stream.prompt_kv(0)
+    ring = 16
+    q, k, v = stream.step_chunk(0, 0, ring)
+    bq, bk, bv = stream.beacon_chunk(0, 0, 4)
+    i32 = lambda xs: torch.tensor(np.asarray(xs), dtype=torch.int32, device=dev)
+    cu = np.concatenate([[0], np.cumsum(P)])
+    all_slots = np.arange(Bn)
+    cache.bc_seq_open(i32(all_slots), i32(P), i32(C))
+    cache.bc_prefill(0, i32(all_slots), i32(cu), int(cu[-1]), pk, pv)
+    out, outb = cache.new_out(Bn), cache.new_out(Bn)
+    order = np.argsort(T, kind="stable")
+    T_max = int(T.max())
+    kv_entries = 0
+    high_water = high_water_unc = 0
+    torch.cuda.synchronize()
+    e0, e1 = _event_pair(torch)
+    t_host = time.perf_counter()
+    e0.record()
+    t, live, n_launch0 = 0, all_slots, cache.bc_kernel_launches()
+    done_ptr = 0
+    while len(live):
+        # epoch: the batch stays as it is until the next sequence finishes
+        t_end = int(T[order[done_ptr]])
+        idx = torch.tensor(live, dtype=torch.int64, device=dev)
+        sl = i32(live)
+        kk, vv, qq = k.index_select(1, idx), v.index_select(1, idx), q.index_select(1, idx)
+        Cl, Pl = C[live], P[live]
+        groups = {}                                     # (step mod 16, beacon row) -> positions
+        while t < t_end:
+            t += 1
+            j = (t - 1) % ring
+            cache.bc_append(0, sl, kk[j], vv[j])
+            cache.bc_decode_attn(0, sl, qq[j], out, w.sm_scale)
+            nb, wl = (t - 1) // Cl, (t - 1) % Cl + 1
+            kv_entries += int((Pl + nb + wl).sum())
+            full = (t % Cl) == 0
+            if full.any():
+                m = (t // Cl) % 4
+                for rsel in range(4):
+                    pos = np.nonzero(full & (m == rsel))[0]
+                    if not len(pos):
+                        continue
+                    key = (tuple(pos), rsel)
+                    if key not in groups:
+                        gi = torch.tensor(live[pos], dtype=torch.int64, device=dev)
+                        groups[key] = (i32(live[pos]), bq[rsel].index_select(0, gi), bk[rsel].index_select(0, gi),
+                                       bv[rsel].index_select(0, gi))
+                    gsl, gq, gk, gv = groups[key]
+                    cache.bc_decode_attn(0, gsl, gq, outb, w.sm_scale, gk, gv)
+                    cache.bc_compress(0, gsl, gk, gv)
+                    kv_entries += int((Pl[pos] + (t // Cl[pos] - 1) + Cl[pos]).sum())
+            if t % 64 == 0 or t == t_end:
+                nbp = np.where(Cl > 1, t // Cl, 0); wl2 = np.where(Cl > 1, t % Cl, t)
+                high_water = max(high_water, int((cd(Pl, ps) + cd(nbp, ps) + cd(wl2, ps)).sum()))
+                high_water_unc = max(high_water_unc, int(cd(Pl + t, ps).sum()))
+        fin = []
+        while done_ptr < Bn and T[order[done_ptr]] == t:
+            fin.append(order[done_ptr]); done_ptr += 1
+        cache.bc_seq_close(i32(fin))
+        live = np.array([s for s in live if s not in set(fin)], dtype=np.int64)
+    e1.record()
+    torch.cuda.synchronize()
+    host_s = time.perf_counter() - t_host
+    ms = e0.elapsed_time(e1)
+    code, slot, call = cache.bc_poll_error()
+    assert code == 0, (code, slot, call)
+    free = cache.bc_get_free_list()
+    assert len(free) == int(pps.sum()), "pages were lost"
+    E = w.entry_bytes
+    tokens = int(T.sum())
+    print(json.dumps({
+        "workload": "ragged: 1 layer, B=128, 12/2 heads, D=128, page 16, P~U[64,1024], T~U[1024,32768], c in {4,8,16}",
+        "decode_steps": T_max, "tokens": tokens, "ms_total": ms, "tokens_per_s": tokens / (ms * 1e-3),
+        "kv_bytes_read": kv_entries * E, "kv_gbs": kv_entries * E / (ms * 1e-3) / 1e9,
+        "pages_high_water": high_water, "pages_high_water_uncompressed": high_water_unc,
+        "cache_bytes_high_water": high_water * ps * E, "uncompressed_bytes_high_water": high_water_unc * ps * E,
+        "gpu_launches": int(cache.bc_kernel_launches() - n_launch0), "host_seconds": host_s,
+        "all_pages_returned": True,
+        "note": "plain launches issued from Python; the run is host-issue-bound wherever a step's kernels "
+                "take less than the ~25 us the host needs to issue them"}))
+
+
+def report_depth(args):
+    """Benchmark configs[4]: 28 layers, batch 256, 12/2 heads, prompt 512, 8192 steps, c = 8,
+    page 8.  Per-layer calls in dependency order, whole windows of 8 steps as one CUDA graph, at the
+    middle of the generation; footprint against the uncompressed cache; the largest batch one GPU
+    holds at c in {1, 4, 8, 16}, computed from the free memory and demonstrated at c = 8."""
+    import torch
+    from paper_2510_13797_b200 import binding as B
+    from paper_2510_13797_b200.workloads import InputStream, make_workload
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    w = make_workload("depth")
+    L, Bn, ps, c, P, T = w.layers, w.batch, w.page_size, w.cs[0], w.prompt_lens[0], w.steps
+    E = w.entry_bytes
+    cd = lambda a, b_: -(-a // b_)
+    free0, total0 = torch.cuda.mem_get_info()
+
+    def pages_per_seq(cc, page):
+        return cd(P, page) + cd(cc, page) + cd(cd(T, cc), page) + 1 if cc > 1 else cd(P + T, page) + 1
+
+    def bytes_per_seq(cc):
+        page = cc if cc > 1 else 16
+        return pages_per_seq(cc, page) * page * E * L
+
+    capacity = {str(cc): int(0.90 * free0 // bytes_per_seq(cc)) for cc in (1, 4, 8, 16)}
+    pps = pages_per_seq(c, ps)
+    cache = B.Cache(L, w.kv_heads, w.q_heads, w.head_dim, c, ps, max_seqs=Bn, num_pages=Bn * pps,
+                    max_pages_per_seq=pps, device=dev)
+    slots = torch.arange(Bn, dtype=torch.int32, device=dev)
+    cu = torch.arange(0, (Bn + 1) * P, P, dtype=torch.int32, device=dev)
+    cache.bc_seq_open(slots, torch.full((Bn,), P, dtype=torch.int32, device=dev))
+    stream = InputStream(w, dev)
+    ring = 8
+    ins = []
+    for l in range(L):
+        pk, pv = stream.prompt_kv(l)
+        cache.bc_prefill(l, slots, cu, Bn * P, pk, pv)
+        ins.append((stream.step_chunk(l, 0, ring), stream.beacon_chunk(l, 0, 2)))
+        del pk, pv
+    out = cache.new_out(Bn)
+    state = {"t": 0}
+
+    def step(attend=True):
+        t = state["t"]; j = t % ring
+        for l in range(L):
+            (q, k, v), _ = ins[l]
+            cache.bc_append(l, slots, k[j], v[j])
+            if attend:
+                cache.bc_decode_attn(l, slots, q[j], out, w.sm_scale)
+        state["t"] = t = t + 1
+        if t % c == 0:
+            m = (t // c) % 2
+            for l in range(L):
+                _, (bq, bk, bv) = ins[l]
+                if attend:
+                    cache.bc_decode_attn(l, slots, bq[m], out, w.sm_scale, bk[m], bv[m])
+                cache.bc_compress(l, slots, bk[m], bv[m])
+
+    K = max(c, (min(args.steps, 64) // c) * c)
+    t_mid = ((T - K) // 2 // c) * c
+    while state["t"] < t_mid:
+        step(attend=False)
+    for _ in range(c):
+        step()
+    s = torch.cuda.Stream(); s.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    l0, t_save = cache.bc_kernel_launches(), state["t"]
+    with torch.cuda.graph(graph, stream=s, capture_error_mode="thread_local"):
+        for _ in range(c):
+            step()
+    per_graph = cache.bc_kernel_launches() - l0
+    state["t"] = t_save
+    torch.cuda.current_stream().wait_stream(s)
+    graph.replay(); state["t"] += c
+    torch.cuda.synchronize()
+    t_begin = state["t"]
+    e0, e1 = _event_pair(torch)
+    e0.record()
+    for _ in range(K // c):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    state["t"] += K
+    ms = e0.elapsed_time(e1)
+    code, slot, call = cache.bc_poll_error()
+    assert code == 0, (code, slot, call)
+    reg = sum(entries_attended(P, n, c) for n in range(t_begin + 1, t_begin + K + 1))
+    bea = sum(entries_beacon_query(P, n, c) for n in range(t_begin + 1, t_begin + K + 1) if n % c == 0)
+    kv = (reg + bea) * E * Bn * L
+    end_entries = P + T // c + T % c
+    line = {
+        "workload": "depth: 28 layers, B=256, 12/2 heads, D=128, P=512, T=8192, c=8, page 8",
+        "steps": K, "t_window": [t_begin, t_begin + K], "ms_per_step": ms / K,
+        "attention_tokens_per_s": Bn * K / (ms * 1e-3), "layer_tokens_per_s": Bn * K * L / (ms * 1e-3),
+        "kv_bytes_per_step": kv / K, "kv_gbs": kv / (ms * 1e-3) / 1e9,
+        "pct_of_8tbs": 100 * kv / (ms * 1e-3) / 8e12,
+        "gpu_launches": int(per_graph * (K // c)),
+        "kv_footprint_end_bytes": end_entries * E * L * Bn, "uncompressed_end_bytes": (P + T) * E * L * Bn,
+        "footprint_ratio_end": (P + T) / end_entries,
+        "hbm_free_bytes": free0, "hbm_total_bytes": total0,
+        "largest_batch_that_fits": capacity,
+        "largest_batch_rule": "floor(0.90 * free HBM / (pages per sequence at the end of the run * page bytes * 28 "
+                              "layers)), page_size = c (16 for c = 1)",
+    }
+    # demonstration at c = 8: allocate the pool for that many sequences and decode a window with all of them
+    del cache, ins, graph
+    torch.cuda.empty_cache()
+    n_big = capacity["8"]
+    big = B.Cache(L, w.kv_heads, w.q_heads, w.head_dim, c, ps, max_seqs=n_big, num_pages=n_big * pps,
+                  max_pages_per_seq=pps, device=dev)
+    all_slots = torch.arange(n_big, dtype=torch.int32, device=dev)
+    big.bc_seq_open(all_slots, torch.full((n_big,), P, dtype=torch.int32, device=dev))
+    chunk = 512                                       # sequences per call
+    g = torch.Generator(device=dev); g.manual_seed(1)
+    rnd = lambda *shape: torch.randn(shape, generator=g, device=dev).to(torch.bfloat16)
+    pk, pv = rnd(chunk * P, w.kv_heads, w.head_dim), rnd(chunk * P, w.kv_heads, w.head_dim)
+    kq = rnd(chunk, w.q_heads, w.head_dim); kk = rnd(chunk, w.kv_heads, w.head_dim)
+    outc = big.new_out(chunk)
+    cuc = torch.arange(0, (chunk + 1) * P, P, dtype=torch.int32, device=dev)
+    starts = list(range(0, n_big, chunk))
+    for l in range(L):
+        for a in starts:
+            n = min(chunk, n_big - a)
+            big.bc_prefill(l, all_slots[a:a + n], cuc[:n + 1], n * P, pk, pv)
+    e0, e1 = _event_pair(torch)
+    e0.record()
+    for t in range(1, c + 1):
+        for l in range(L):
+            big.bc_append(l, all_slots, rnd(n_big, w.kv_heads, w.head_dim), rnd(n_big, w.kv_heads, w.head_dim))
+            for a in starts:
+                n = min(chunk, n_big - a)
+                big.bc_decode_attn(l, all_slots[a:a + n], kq[:n], outc[:n], w.sm_scale)
+        if t == c:
+            for l in range(L):
+                big.bc_compress(l, all_slots, rnd(n_big, w.kv_heads, w.head_dim), rnd(n_big, w.kv_heads, w.head_dim))
+    e1.record()
+    torch.cuda.synchronize()
+    code, slot, call = big.bc_poll_error()
+    st = big.bc_get_state(n_big - 1)
+    line["demonstrated"] = {"c": 8, "batch": n_big, "pool_bytes": big.pool_bytes, "steps": c,
+                            "ms_per_step": e0.elapsed_time(e1) / c, "device_error": code,
+                            "last_slot_state": {k_: st[k_] for k_ in ("prompt_len", "n_beacons", "window_len", "t")}}
+    print(json.dumps(line))
+
+
+def batch_scaling(dev, peak):
+    """The attention kernel alone at larger batches (same shape, mid-generation cache): the time per
+    launch that does not stream (start-up, merging) is spread over more bytes."""
+    import torch
+    from paper_2510_13797_b200.workloads import make_workload
+    rows = []
+    for c in (16, 32):
+        for Bn in (128, 256):
+            w = make_workload("sweep", c=c, batch=Bn)
+            mid = entries_attended(w.prompt_lens[0], w.steps // 2, c)
+            w = make_workload("sweep", c=c, batch=Bn, prompt_lens=[mid] * Bn, gen_lens=[256] * Bn)
+            r = make_runner(w, dev)
+            r.reset_to(c // 2)
+            ms, n, nbytes = r.timed_attn_stream(64, 4)
+            r.check_error()
+            rows.append({"c": c, "batch": Bn, "attn_kernel_us": 1e3 * ms / n, "attn_kernel_gbs": nbytes / (ms * 1e-3) / 1e9,
+                         "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak, "pct_of_8tbs": 100 * nbytes / (ms * 1e-3) / 8e12})
+            del r
+            torch.cuda.empty_cache()
+    return rows
+
+
 # ------------------------------------------------------------------------------ main arm
 def main():
     ap = argparse.ArgumentParser()
@@ -346,6 +659,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth"],
+                    help="sweep (default): the benchmark line; cfg2 / ragged / depth: a report line for that "
+                         "BASELINE.json configuration (1 GPU)")
+    ap.add_argument("--no-batch-scaling", action="store_true")
     ap.add_argument("--profile-case", type=int, default=0, metavar="C",
                     help="small case for profilers: ratio C with a prompt as long as the mid-generation cache, "
                          "--steps plain decode steps, no fast-forward, no graphs")
@@ -354,6 +671,8 @@ def main():
         return run_reference(args)
     if args.profile_case:
         return run_profile_case(args)
+    if args.workload != "sweep":
+        return {"cfg2": report_cfg2, "ragged": report_ragged, "depth": report_depth}[args.workload](args)
 
     import torch
     import torch.distributed as dist
@@ -469,6 +788,8 @@ def main():
                      "pct_of_8tbs": 100 * achieved * 1e9 / 8e12},
         "sweep": rows,
     }
+    if not args.no_batch_scaling and world == 1:
+        line["batch_scaling"] = batch_scaling(dev, peak)
     if not args.no_cpu_baseline:
         w = make_workload("sweep", c=16)
         wall, tok, cpu = oracle_sample(w, w.steps // 2, 16, 8)

@@ -220,6 +220,41 @@ BC_API bc_status bc_compress_step_host(bc_cache* cache, int32_t layer, const int
                                 const void* beacon_v_host, void* out_host, float sm_scale,
                                 void* stream);
 
+/* ---- the mask form: a whole trajectory in one pass (Section 3.2, Figure 2) ---------------------
+ * Training simulates the eviction with an attention mask over the teacher-forced trajectory
+ * [prompt, x_0 .. x_{c-1}, b_1, x_c, ...]: a generated token attends to the prompt, to every
+ * earlier beacon and to the tokens of its own window up to itself; beacon b_m, placed after the
+ * m-th window of c tokens, attends to the prompt, the beacons b_1 .. b_m (itself included) and
+ * that window.  The paper states that this computes what the inference loop computes (Section
+ * 3.2); here it is one dense pass on the tensor cores, independent of any bc_cache.
+ *
+ * Sequences are packed back to back.  cu_prompt, cu_tokens: HOST int32[n_seqs + 1] prefix sums of
+ * the prompt and generated-token counts.  Sequence i has floor(T_i / c) beacons (none when c = 1),
+ * packed in the same order.  Device tensors, bf16: prompt_k, prompt_v [sum P, kv_heads, head_dim];
+ * tok_q [sum T, q_heads, head_dim]; tok_k, tok_v [sum T, kv_heads, head_dim]; beacon_q
+ * [sum nb, q_heads, head_dim]; beacon_k, beacon_v [sum nb, kv_heads, head_dim]; outputs out_tok
+ * [sum T, q_heads, head_dim] and out_beacon [sum nb, q_heads, head_dim], bf16 rounded to nearest
+ * even from fp32 (accumulation in fp32, softmax weights rounded to bf16 before the second product).
+ * head_dim must be 128 and q_heads / kv_heads <= 16 (else BC_ERR_UNSUPPORTED).  `workspace`: device
+ * memory of at least bc_mask_attn_query_bytes bytes, 256-byte aligned (it receives the tile list
+ * and a transposed copy of V).  Asynchronous on `stream`; the two host arrays are read before the
+ * call returns.  A bounded device-side wait that expires is reported by bc_mask_attn_status as
+ * BC_ERR_TIMEOUT (the outputs are then incomplete). */
+BC_API bc_status bc_mask_attn_query_bytes(int32_t n_seqs, int32_t q_heads, int32_t kv_heads, int32_t head_dim,
+                                          int64_t total_prompt, int64_t total_tokens, int64_t total_beacons,
+                                          size_t* workspace_bytes);
+BC_API bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads, int32_t head_dim, int32_t c,
+                                      const int32_t* cu_prompt, const int32_t* cu_tokens, const void* prompt_k,
+                                      const void* prompt_v, const void* tok_q, const void* tok_k, const void* tok_v,
+                                      const void* beacon_q, const void* beacon_k, const void* beacon_v,
+                                      void* out_tok, void* out_beacon, float sm_scale, void* workspace,
+                                      size_t workspace_bytes, void* stream);
+/* Synchronises `stream` and returns in *code the status the last bc_mask_attn_forward on this
+ * workspace left on the device (BC_OK or BC_ERR_TIMEOUT).  The totals are those of that call. */
+BC_API bc_status bc_mask_attn_status(const void* workspace, int32_t n_seqs, int32_t q_heads, int32_t kv_heads,
+                                     int64_t total_prompt, int64_t total_tokens, int64_t total_beacons,
+                                     void* stream, int32_t* code);
+
 /* ---- inspection (these synchronise `stream`; for tests and tools) ---------------------------- */
 
 /* Bookkeeping of one slot.  pages (host, may be NULL) receives up to pages_cap page ids: prompt

@@ -58,6 +58,10 @@ SYMBOLS = {
     "bc_append": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
     "bc_decode_attn": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
     "bc_decode_attn_static": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
+    "bc_mask_attn_query_bytes": (_I32, [_I32, _I32, _I32, _I32, _I64, _I64, _I64, C.POINTER(C.c_size_t)]),
+    "bc_mask_attn_forward": (_I32, [_I32, _I32, _I32, _I32, _I32, C.POINTER(_I32), C.POINTER(_I32)] + [_P] * 10
+                             + [_F, _P, C.c_size_t, _P]),
+    "bc_mask_attn_status": (_I32, [_P, _I32, _I32, _I32, _I64, _I64, _I64, _P, C.POINTER(_I32)]),
     "bc_compress": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
     "bc_seq_close": (_I32, [_P, _P, _I32, _P]),
     "bc_decode_step_host": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P]),
@@ -228,3 +232,32 @@ class Cache:
     # ---- convenience ------------------------------------------------------------------------------
     def new_out(self, n):
         return torch.empty((n, self.cfg.q_heads, self.cfg.head_dim), dtype=self.out_dtype, device=self.device)
+
+
+def bc_mask_attn_forward(prompt_lens, token_lens, c, prompt_k, prompt_v, tok_q, tok_k, tok_v, beacon_q, beacon_k,
+                         beacon_v, sm_scale, stream=None, check=True):
+    """The mask form of a batch of trajectories (breadcrumbs.h): returns (out_tok, out_beacon).
+
+    prompt_lens, token_lens: Python lists, one entry per sequence.  Tensors are packed bf16 CUDA
+    tensors as the header describes; beacon tensors may be None when no sequence has a beacon."""
+    n = len(prompt_lens)
+    q_heads, kv_heads, head_dim = tok_q.shape[1], tok_k.shape[1], tok_q.shape[2]
+    cu_p = (C.c_int32 * (n + 1))(0, *list(__import__("itertools").accumulate(prompt_lens)))
+    cu_t = (C.c_int32 * (n + 1))(0, *list(__import__("itertools").accumulate(token_lens)))
+    total_b = sum(t // c for t in token_lens) if c > 1 else 0
+    size = C.c_size_t()
+    _check(lib().bc_mask_attn_query_bytes(n, q_heads, kv_heads, head_dim, cu_p[n], cu_t[n], total_b, C.byref(size)),
+           "bc_mask_attn_query_bytes")
+    ws = torch.empty(size.value, dtype=torch.uint8, device=tok_q.device)
+    out_tok = torch.empty_like(tok_q)
+    out_bea = torch.empty((total_b, q_heads, head_dim), dtype=tok_q.dtype, device=tok_q.device)
+    _check(lib().bc_mask_attn_forward(n, q_heads, kv_heads, head_dim, c, cu_p, cu_t, _ptr(prompt_k), _ptr(prompt_v),
+                                      _ptr(tok_q), _ptr(tok_k), _ptr(tok_v), _ptr(beacon_q), _ptr(beacon_k),
+                                      _ptr(beacon_v), _ptr(out_tok), _ptr(out_bea), sm_scale, _ptr(ws), size.value,
+                                      _stream(stream)), "bc_mask_attn_forward")
+    if check:
+        code = C.c_int32()
+        _check(lib().bc_mask_attn_status(_ptr(ws), n, q_heads, kv_heads, cu_p[n], cu_t[n], total_b, _stream(stream),
+                                         C.byref(code)), "bc_mask_attn_status")
+        _check(code.value, "bc_mask_attn_forward (device)")
+    return out_tok, out_bea

@@ -1,0 +1,482 @@
+// Mask-form (teacher-forced) attention forward: the dense formulation of Figure 2 / Section 3.2.
+//
+// During training the eviction is simulated by an attention mask over the whole trajectory: a
+// generated token sees the prompt, every earlier beacon, and the tokens of its own window up to
+// itself; the beacon that closes a window sees the prompt, the earlier beacons, that window and
+// itself.  This file computes those rows for a batch of trajectories in one pass -- the other side
+// of the cache that the decode path maintains step by step (same results, Section 3.2).
+//
+// Unlike decode this is a dense contraction, so it runs on the tcgen05 tensor cores:
+//   * one thread block (128 threads) per (query tile, KV head): 128 query rows = floor(128/G) tokens
+//     (or beacons) times the G query heads that share the KV head, so a K/V tile is reused by G heads;
+//   * per key tile of 128 keys:  S = Q K^T  (tcgen05.mma, M = N = K = 128, fp32 in tensor memory)
+//     -> tcgen05.ld, mask, online softmax in fp32 registers, P as bf16 into shared memory
+//     -> O_tile = P V  (second tcgen05.mma) -> tcgen05.ld and accumulation in registers;
+//   * operands live in shared memory in the 128-byte-swizzled K-major layout the MMA descriptors
+//     describe; V is needed K-major too (keys contiguous), so a small kernel transposes V into the
+//     caller's workspace first;
+//   * key tiles a query tile cannot see are skipped: all prompt tiles, the beacon tiles up to its
+//     last visible beacon, and the token tiles that overlap its own windows.
+// Every wait is bounded; on expiry the block records BC_ERR_TIMEOUT, releases its tensor memory and
+// returns.
+#include <vector>
+
+#include "bc_common.cuh"
+
+namespace {
+
+constexpr int kTile = 128;        // query rows and keys per tile
+constexpr int kD = 128;           // head_dim
+constexpr int kThreads = 128;
+constexpr int kOperandBytes = kTile * kD * 2;  // 32 KB: one bf16 operand tile
+constexpr uint32_t kWaitLimit = 1u << 20;  // polls of a bounded wait (about 0.1 s) before a block gives up
+
+struct TileDesc {
+  int32_t kind;        // 0: token rows, 1: beacon rows
+  int32_t first;       // first token / beacon (0-based, inside the sequence) of the tile
+  int32_t count;       // tokens / beacons in the tile
+  int32_t P, T, nb;    // lengths of the sequence
+  int32_t prompt_row, tok_row, bea_row;  // first row of the sequence in the packed inputs
+  int32_t prompt_pad, tok_pad, bea_pad;  // first column of the sequence in the transposed V arrays
+  int32_t pad[4];
+};
+
+struct MaskArgs {
+  const TileDesc* tiles;
+  const __nv_bfloat16 *prompt_k, *tok_q, *tok_k, *bea_q, *bea_k;
+  const __nv_bfloat16 *vt_prompt, *vt_tok, *vt_bea;  // [Hkv][D][padded columns]
+  int64_t vt_prompt_cols, vt_tok_cols, vt_bea_cols;  // padded columns per (head, d) row
+  __nv_bfloat16 *out_tok, *out_bea;
+  int32_t* status;     // device int: first error code
+  int32_t Hq, Hkv, G, c, rows_per_tile;  // rows_per_tile = tokens per query tile = 128 / G
+  float scale_log2;
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Byte offset of 16-byte chunk `ch16` (0..15 = 8 elements each) of row r in a 128 x 128 bf16 operand
+// tile stored K-major with 128-byte swizzling: two blocks of 64 elements, each 128 rows of 128 bytes,
+// the chunk index inside a row XOR-ed with the row number modulo 8.
+__device__ __forceinline__ uint32_t swz(int r, int ch16) {
+  return (uint32_t)((ch16 >> 3) * (kTile * 128) + r * 128 + (((ch16 & 7) ^ (r & 7)) << 4));
+}
+
+__device__ __forceinline__ void cp16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void st_zero16(uint32_t dst) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3ffff) >> 4);   // start address
+  d |= (uint64_t)0 << 16;                    // leading byte offset: unused for swizzled K-major
+  d |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                    // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                    // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t a, uint64_t b, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(a), "l"(b), "r"(kIdesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (uint32_t polls = 0; polls < kWaitLimit; ++polls) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if (polls > 4096) __nanosleep(128);
+  }
+  return false;
+}
+
+// One key segment of a sequence as the main loop sees it.
+struct KeySeg {
+  const __nv_bfloat16* k;   // [rows][Hkv][D], first row of the sequence
+  const __nv_bfloat16* vt;  // transposed V: row (head, d), first column of the sequence
+  int64_t vt_cols;          // columns per vt row
+  int lo, hi;               // keys [lo, hi) of the segment are candidates (lo a multiple of 128)
+  int len;                  // rows that exist
+  int kind;                 // 0 prompt, 1 beacon, 2 token
+};
+
+__global__ void __launch_bounds__(kThreads, 1) k_mask_attn(const MaskArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sQ = smem_addr(smem), sK = sQ + kOperandBytes, sV = sK + kOperandBytes, sP = sV + kOperandBytes;
+  __shared__ __align__(8) uint64_t s_bar;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+  const uint32_t bar = smem_addr(&s_bar);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const TileDesc td = a.tiles[blockIdx.x];
+  const int kvh = blockIdx.y, G = a.G, Hq = a.Hq, Hkv = a.Hkv, c = a.c;
+
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_fail = 0;
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&s_tmem)), "r"(256) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+
+  // ---- the query tile: row r = (local index r / G, head r % G) ---------------------------------
+  const __nv_bfloat16* qsrc = td.kind == 0 ? a.tok_q + (int64_t)(td.tok_row + td.first) * Hq * kD
+                                           : a.bea_q + (int64_t)(td.bea_row + td.first) * Hq * kD;
+  const int valid_rows = td.count * G;
+  for (int idx = tid; idx < kTile * 16; idx += kThreads) {
+    const int r = idx >> 4, ch = idx & 15;
+    if (r < valid_rows) cp16(sQ + swz(r, ch), qsrc + ((int64_t)(r / G) * Hq + kvh * G + (r % G)) * kD + ch * 8);
+    else st_zero16(sQ + swz(r, ch));
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  const uint32_t tS = tmem, tO = tmem + kTile;                 // columns [0,128) and [128,256)
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;      // this warp's 32 lanes of tensor memory
+
+  // ---- what this thread's row may see ------------------------------------------------------------
+  const int my_local = tid / G;                 // token / beacon inside the tile
+  const bool row_valid = tid < valid_rows;
+  const int my_idx = td.first + my_local;       // token index i, or beacon index (0-based; beacon number my_idx + 1)
+  int vis_beacons, tok_lo, tok_hi;              // visible: beacons [0, vis_beacons), tokens [tok_lo, tok_hi)
+  if (td.kind == 0) { vis_beacons = c > 1 ? my_idx / c : 0; tok_lo = c > 1 ? (my_idx / c) * c : 0; tok_hi = my_idx + 1; }
+  else { vis_beacons = my_idx + 1; tok_lo = my_idx * c; tok_hi = (my_idx + 1) * c; }
+
+  // ---- key segments and the tiles of each that some row of this block can see ----------------------
+  const int last = td.first + td.count - 1;
+  KeySeg seg[3];
+  seg[0] = {a.prompt_k + (int64_t)td.prompt_row * Hkv * kD, a.vt_prompt + td.prompt_pad, a.vt_prompt_cols, 0, td.P, td.P, 0};
+  const int bmax = td.kind == 0 ? (c > 1 ? last / c : 0) : last + 1;
+  seg[1] = {a.bea_k + (int64_t)td.bea_row * Hkv * kD, a.vt_bea + td.bea_pad, a.vt_bea_cols, 0, bmax, td.nb, 1};
+  const int tlo = td.kind == 0 ? (c > 1 ? (td.first / c) * c : 0) : td.first * c;
+  const int thi = td.kind == 0 ? last + 1 : (last + 1) * c;
+  seg[2] = {a.tok_k + (int64_t)td.tok_row * Hkv * kD, a.vt_tok + td.tok_pad, a.vt_tok_cols, (tlo / kTile) * kTile, thi, td.T, 2};
+
+  float o[kD];
+#pragma unroll
+  for (int d = 0; d < kD; ++d) o[d] = 0.f;
+  float m_run = -INFINITY, l_run = 0.f;
+  uint32_t phase = 0;
+  bool failed = false;
+
+  for (int sgi = 0; sgi < 3 && !failed; ++sgi) {
+    const KeySeg& sg = seg[sgi];
+    for (int k0 = sg.lo; k0 < sg.hi && !failed; k0 += kTile) {
+      // ---- K tile (rows = keys) and transposed V tile (rows = d, columns = keys) -------------------
+      for (int idx = tid; idx < kTile * 16; idx += kThreads) {
+        const int r = idx >> 4, ch = idx & 15;
+        if (k0 + r < sg.len) cp16(sK + swz(r, ch), sg.k + ((int64_t)(k0 + r) * Hkv + kvh) * kD + ch * 8);
+        else st_zero16(sK + swz(r, ch));
+        // columns beyond the sequence's rows are zero in the transposed array (it is padded to 128)
+        cp16(sV + swz(r, ch), sg.vt + ((int64_t)kvh * kD + r) * sg.vt_cols + k0 + ch * 8);
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      proxy_fence();
+      __syncthreads();
+      // ---- S = Q K^T ---------------------------------------------------------------------------------
+      if (tid == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < kD / 16; ++kk) {
+          const uint32_t off = (uint32_t)((kk >> 2) * (kTile * 128) + (kk & 3) * 32);
+          umma(tS, umma_desc(sQ + off), umma_desc(sK + off), kk > 0);
+        }
+        umma_commit(bar);
+      }
+      if (!mbar_wait_bounded(bar, phase)) failed = true;
+      phase ^= 1;
+      tc_fence_after();
+      // ---- mask + online softmax; this thread owns query row `tid` -----------------------------------
+      float tile_max = -INFINITY;
+      float s[32];
+      auto visible = [&](int key) {
+        if (!row_valid || key >= sg.len) return false;
+        if (sg.kind == 0) return true;
+        if (sg.kind == 1) return key < vis_beacons;
+        return key >= tok_lo && key < tok_hi;
+      };
+      if (!failed) {
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          tmem_ld32(tS + lane_base + cb * 32, s);
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (visible(k0 + cb * 32 + j)) tile_max = fmaxf(tile_max, s[j] * a.scale_log2);
+        }
+      }
+      const float m_new = fmaxf(m_run, tile_max);
+      const float m_safe = m_new == -INFINITY ? 0.f : m_new;
+      const float alpha = exp2f(m_run - m_safe);
+      float tile_sum = 0.f;
+      if (!failed) {
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          tmem_ld32(tS + lane_base + cb * 32, s);
+          uint32_t pk[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = visible(k0 + cb * 32 + j) ? exp2f(s[j] * a.scale_log2 - m_safe) : 0.f;
+            const float p1 = visible(k0 + cb * 32 + j + 1) ? exp2f(s[j + 1] * a.scale_log2 - m_safe) : 0.f;
+            const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+            // the sum uses the rounded values, so numerator and denominator see the same weights
+            tile_sum += __low2float(pb) + __high2float(pb);
+            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+          }
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sP + swz(tid, cb * 4 + q4)), "r"(pk[q4 * 4]),
+                         "r"(pk[q4 * 4 + 1]), "r"(pk[q4 * 4 + 2]), "r"(pk[q4 * 4 + 3])
+                         : "memory");
+        }
+      }
+      m_run = m_new;
+      l_run = l_run * alpha + tile_sum;
+      proxy_fence();
+      tc_fence_before();
+      __syncthreads();
+      // ---- O_tile = P V ------------------------------------------------------------------------------
+      if (tid == 0 && !failed) {
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < kTile / 16; ++kk) {
+          const uint32_t off = (uint32_t)((kk >> 2) * (kTile * 128) + (kk & 3) * 32);
+          umma(tO, umma_desc(sP + off), umma_desc(sV + off), kk > 0);
+        }
+        umma_commit(bar);
+      }
+      if (!failed) {
+        if (!mbar_wait_bounded(bar, phase)) failed = true;
+        phase ^= 1;
+      }
+      tc_fence_after();
+      if (!failed) {
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+          tmem_ld32(tO + lane_base + cb * 32, s);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[cb * 32 + j] = o[cb * 32 + j] * alpha + s[j];
+        }
+      }
+      tc_fence_before();
+      if (failed) s_fail = 1;
+      __syncthreads();   // K, V, P and both accumulators are free for the next tile
+      if (s_fail) failed = true;
+    }
+  }
+
+  // ---- write the rows -------------------------------------------------------------------------------
+  if (!failed && row_valid) {
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    __nv_bfloat16* dst = (td.kind == 0 ? a.out_tok + (int64_t)(td.tok_row + my_idx) * Hq * kD
+                                       : a.out_bea + (int64_t)(td.bea_row + my_idx) * Hq * kD) +
+                         (int64_t)(kvh * G + tid % G) * kD;
+#pragma unroll
+    for (int d = 0; d < kD; d += 8) {
+      uint4 v;
+      __nv_bfloat162 t0 = __floats2bfloat162_rn(o[d] * inv, o[d + 1] * inv), t1 = __floats2bfloat162_rn(o[d + 2] * inv, o[d + 3] * inv);
+      __nv_bfloat162 t2 = __floats2bfloat162_rn(o[d + 4] * inv, o[d + 5] * inv), t3 = __floats2bfloat162_rn(o[d + 6] * inv, o[d + 7] * inv);
+      v.x = *reinterpret_cast<uint32_t*>(&t0); v.y = *reinterpret_cast<uint32_t*>(&t1);
+      v.z = *reinterpret_cast<uint32_t*>(&t2); v.w = *reinterpret_cast<uint32_t*>(&t3);
+      *reinterpret_cast<uint4*>(dst + d) = v;
+    }
+  }
+  if (failed && tid == 0) atomicCAS(a.status, 0, BC_ERR_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+  }
+}
+
+// vt[(h * D + d) * cols + pad_base + r] = v[(row_base + r) * Hkv * D + h * D + d]; columns of the
+// padding (r >= rows of the sequence) are written as zero.  grid (sequence, kv head, 32-row blocks).
+struct TransposeSeq {
+  int32_t row_base, rows, pad_base, pad_rows;
+};
+__global__ void k_transpose_v(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ vt, const TransposeSeq* seqs,
+                              int Hkv, int64_t cols) {
+  __shared__ __nv_bfloat16 tile[32][kD + 2];
+  const TransposeSeq sq = seqs[blockIdx.x];
+  const int h = blockIdx.y;
+  for (int r0 = blockIdx.z * 32; r0 < sq.pad_rows; r0 += gridDim.z * 32) {
+    for (int idx = threadIdx.x; idx < 32 * kD; idx += blockDim.x) {
+      const int r = idx / kD, d = idx % kD;
+      tile[r][d] = (r0 + r < sq.rows) ? v[((int64_t)(sq.row_base + r0 + r) * Hkv + h) * kD + d] : __float2bfloat16(0.f);
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < 32 * kD; idx += blockDim.x) {
+      const int d = idx / 32, r = idx % 32;
+      if (r0 + r < sq.pad_rows) vt[((int64_t)h * kD + d) * cols + sq.pad_base + r0 + r] = tile[r][d];
+    }
+    __syncthreads();
+  }
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int64_t pad128(int64_t x) { return (x + 127) / 128 * 128; }
+
+struct MaskLayout {
+  size_t tiles, seqs3, status, vt_prompt, vt_tok, vt_bea, total;
+  int64_t prompt_cols, tok_cols, bea_cols;
+  int64_t n_tiles;
+};
+
+// Upper bounds from the totals alone (every sequence may add one partial tile / 127 padding columns).
+MaskLayout mask_layout(int n_seqs, int q_heads, int kv_heads, int64_t total_prompt, int64_t total_tokens, int64_t total_beacons) {
+  MaskLayout l;
+  const int G = q_heads / kv_heads, per = kTile / G;
+  l.n_tiles = (total_tokens + per - 1) / per + (total_beacons + per - 1) / per + 2 * (int64_t)n_seqs;
+  l.prompt_cols = pad128(total_prompt + 127 * (int64_t)n_seqs);
+  l.tok_cols = pad128(total_tokens + 127 * (int64_t)n_seqs);
+  l.bea_cols = pad128(total_beacons + 127 * (int64_t)n_seqs);
+  size_t o = 0;
+  auto take = [&](size_t b) { size_t at = o; o = align_up(o + b, 256); return at; };
+  l.tiles = take((size_t)l.n_tiles * sizeof(TileDesc));
+  l.seqs3 = take((size_t)3 * n_seqs * sizeof(TransposeSeq));
+  l.status = take(256);
+  l.vt_prompt = take((size_t)kv_heads * kD * l.prompt_cols * 2);
+  l.vt_tok = take((size_t)kv_heads * kD * l.tok_cols * 2);
+  l.vt_bea = take((size_t)kv_heads * kD * l.bea_cols * 2);
+  l.total = o;
+  return l;
+}
+
+}  // namespace
+
+extern "C" {
+
+bc_status bc_mask_attn_query_bytes(int32_t n_seqs, int32_t q_heads, int32_t kv_heads, int32_t head_dim,
+                                   int64_t total_prompt, int64_t total_tokens, int64_t total_beacons,
+                                   size_t* workspace_bytes) {
+  if (!workspace_bytes || n_seqs < 1 || kv_heads < 1 || q_heads < 1 || q_heads % kv_heads || total_prompt < 0 ||
+      total_tokens < 0 || total_beacons < 0)
+    return BC_ERR_INVALID_ARG;
+  if (head_dim != kD || q_heads / kv_heads > 16) return BC_ERR_UNSUPPORTED;
+  *workspace_bytes = mask_layout(n_seqs, q_heads, kv_heads, total_prompt, total_tokens, total_beacons).total;
+  return BC_OK;
+}
+
+bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads, int32_t head_dim, int32_t c,
+                               const int32_t* cu_prompt, const int32_t* cu_tokens, const void* prompt_k,
+                               const void* prompt_v, const void* tok_q, const void* tok_k, const void* tok_v,
+                               const void* beacon_q, const void* beacon_k, const void* beacon_v, void* out_tok,
+                               void* out_beacon, float sm_scale, void* workspace, size_t workspace_bytes,
+                               void* stream) {
+  if (n_seqs < 1 || !cu_prompt || !cu_tokens || c < 1 || kv_heads < 1 || q_heads < 1 || q_heads % kv_heads || !workspace)
+    return BC_ERR_INVALID_ARG;
+  if (head_dim != kD || q_heads / kv_heads > 16) return BC_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255) return BC_ERR_INVALID_ARG;
+  const int G = q_heads / kv_heads, per = kTile / G;
+  int64_t total_prompt = cu_prompt[n_seqs], total_tokens = cu_tokens[n_seqs], total_beacons = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    if (cu_prompt[i + 1] < cu_prompt[i] || cu_tokens[i + 1] < cu_tokens[i]) return BC_ERR_INVALID_ARG;
+    total_beacons += c > 1 ? (cu_tokens[i + 1] - cu_tokens[i]) / c : 0;
+  }
+  if ((total_prompt && (!prompt_k || !prompt_v)) || (total_tokens && (!tok_q || !tok_k || !tok_v || !out_tok)) ||
+      (total_beacons && (!beacon_q || !beacon_k || !beacon_v || !out_beacon)))
+    return BC_ERR_INVALID_ARG;
+  const MaskLayout l = mask_layout(n_seqs, q_heads, kv_heads, total_prompt, total_tokens, total_beacons);
+  if (workspace_bytes < l.total) return BC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+
+  // host side: tile list and per-sequence transposition jobs
+  std::vector<TileDesc> tiles;
+  std::vector<TransposeSeq> tr(3 * (size_t)n_seqs);
+  int64_t pad_p = 0, pad_t = 0, pad_b = 0, bea_row = 0;
+  for (int i = 0; i < n_seqs; ++i) {
+    const int P = cu_prompt[i + 1] - cu_prompt[i], T = cu_tokens[i + 1] - cu_tokens[i], nb = c > 1 ? T / c : 0;
+    TileDesc td = {};
+    td.P = P; td.T = T; td.nb = nb;
+    td.prompt_row = cu_prompt[i]; td.tok_row = cu_tokens[i]; td.bea_row = (int32_t)bea_row;
+    td.prompt_pad = (int32_t)pad_p; td.tok_pad = (int32_t)pad_t; td.bea_pad = (int32_t)pad_b;
+    for (int f = 0; f < T; f += per) { td.kind = 0; td.first = f; td.count = T - f < per ? T - f : per; tiles.push_back(td); }
+    for (int f = 0; f < nb; f += per) { td.kind = 1; td.first = f; td.count = nb - f < per ? nb - f : per; tiles.push_back(td); }
+    tr[i] = {cu_prompt[i], P, (int32_t)pad_p, (int32_t)pad128(P)};
+    tr[n_seqs + i] = {cu_tokens[i], T, (int32_t)pad_t, (int32_t)pad128(T)};
+    tr[2 * n_seqs + i] = {(int32_t)bea_row, nb, (int32_t)pad_b, (int32_t)pad128(nb)};
+    pad_p += pad128(P); pad_t += pad128(T); pad_b += pad128(nb); bea_row += nb;
+  }
+  if ((int64_t)tiles.size() > l.n_tiles || pad_p > l.prompt_cols || pad_t > l.tok_cols || pad_b > l.bea_cols)
+    return BC_ERR_INVALID_ARG;
+  if (tiles.empty()) return BC_OK;
+  cudaError_t e = cudaMemcpyAsync(ws + l.tiles, tiles.data(), tiles.size() * sizeof(TileDesc), cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + l.seqs3, tr.data(), tr.size() * sizeof(TransposeSeq), cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemsetAsync(ws + l.status, 0, 4, s);
+  // the copies above read pageable host memory: they have been staged when the calls return
+  if (e != cudaSuccess) return BC_ERR_CUDA;
+  const TransposeSeq* dtr = reinterpret_cast<const TransposeSeq*>(ws + l.seqs3);
+  auto vt = [&](size_t off) { return reinterpret_cast<__nv_bfloat16*>(ws + off); };
+  if (total_prompt) k_transpose_v<<<dim3(n_seqs, kv_heads, 8), 256, 0, s>>>((const __nv_bfloat16*)prompt_v, vt(l.vt_prompt), dtr, kv_heads, l.prompt_cols);
+  if (total_tokens) k_transpose_v<<<dim3(n_seqs, kv_heads, 8), 256, 0, s>>>((const __nv_bfloat16*)tok_v, vt(l.vt_tok), dtr + n_seqs, kv_heads, l.tok_cols);
+  if (total_beacons) k_transpose_v<<<dim3(n_seqs, kv_heads, 8), 256, 0, s>>>((const __nv_bfloat16*)beacon_v, vt(l.vt_bea), dtr + 2 * n_seqs, kv_heads, l.bea_cols);
+
+  MaskArgs a;
+  a.tiles = reinterpret_cast<const TileDesc*>(ws + l.tiles);
+  a.prompt_k = (const __nv_bfloat16*)prompt_k; a.tok_q = (const __nv_bfloat16*)tok_q; a.tok_k = (const __nv_bfloat16*)tok_k;
+  a.bea_q = (const __nv_bfloat16*)beacon_q; a.bea_k = (const __nv_bfloat16*)beacon_k;
+  a.vt_prompt = vt(l.vt_prompt); a.vt_tok = vt(l.vt_tok); a.vt_bea = vt(l.vt_bea);
+  a.vt_prompt_cols = l.prompt_cols; a.vt_tok_cols = l.tok_cols; a.vt_bea_cols = l.bea_cols;
+  a.out_tok = (__nv_bfloat16*)out_tok; a.out_bea = (__nv_bfloat16*)out_beacon;
+  a.status = reinterpret_cast<int32_t*>(ws + l.status);
+  a.Hq = q_heads; a.Hkv = kv_heads; a.G = G; a.c = c; a.rows_per_tile = per;
+  a.scale_log2 = sm_scale * 1.4426950408889634f;
+  const int smem_bytes = 4 * kOperandBytes + 1024;
+  if (cudaFuncSetAttribute(k_mask_attn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return BC_ERR_CUDA;
+  k_mask_attn<<<dim3((unsigned)tiles.size(), kv_heads), kThreads, smem_bytes, s>>>(a);
+  return cudaGetLastError() == cudaSuccess ? BC_OK : BC_ERR_CUDA;
+}
+
+bc_status bc_mask_attn_status(const void* workspace, int32_t n_seqs, int32_t q_heads, int32_t kv_heads,
+                              int64_t total_prompt, int64_t total_tokens, int64_t total_beacons, void* stream,
+                              int32_t* code) {
+  if (!workspace || !code) return BC_ERR_INVALID_ARG;
+  const MaskLayout l = mask_layout(n_seqs, q_heads, kv_heads, total_prompt, total_tokens, total_beacons);
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BC_ERR_CUDA;
+  if (cudaMemcpy(code, static_cast<const uint8_t*>(workspace) + l.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BC_ERR_CUDA;
+  return BC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,55 @@
+"""GPU parity of the mask-form (teacher-forced) attention pass against the oracle's dense masked
+attention (Figure 2), which the CPU pins show equal to the eviction form."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle.breadcrumbs_oracle import mask_form_outputs
+from paper_2510_13797_b200 import binding as B
+from tests.harness import assert_close, f64, randn_bf16
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def run_case(plens, tlens, c, Hq, Hkv, seed, k_scale=1.0):
+    D = 128
+    g = torch.Generator(device=DEV); g.manual_seed(seed)
+    nbs = [t // c if c > 1 else 0 for t in tlens]
+    sp, st, sb = sum(plens), sum(tlens), sum(nbs)
+    pk, pv = randn_bf16(g, (sp, Hkv, D), DEV, k_scale), randn_bf16(g, (sp, Hkv, D), DEV)
+    tq, tk, tv = randn_bf16(g, (st, Hq, D), DEV), randn_bf16(g, (st, Hkv, D), DEV, k_scale), randn_bf16(g, (st, Hkv, D), DEV)
+    bq, bk, bv = randn_bf16(g, (sb, Hq, D), DEV), randn_bf16(g, (sb, Hkv, D), DEV, k_scale), randn_bf16(g, (sb, Hkv, D), DEV)
+    scale = 1.0 / math.sqrt(D)
+    out_t, out_b = B.bc_mask_attn_forward(plens, tlens, c, pk, pv, tq, tk, tv, bq, bk, bv, scale)
+    torch.cuda.synchronize()
+    op = ot = ob = 0
+    for P, T, nb in zip(plens, tlens, nbs):
+        ref_t, ref_b = mask_form_outputs(f64(pk[op:op + P]), f64(pv[op:op + P]), f64(tk[ot:ot + T]), f64(tv[ot:ot + T]),
+                                         f64(tq[ot:ot + T]), f64(bk[ob:ob + nb]), f64(bv[ob:ob + nb]), f64(bq[ob:ob + nb]),
+                                         c, scale)
+        if T:
+            assert_close(out_t[ot:ot + T], ref_t, f"tokens P={P} T={T} c={c}")
+        if nb:
+            assert_close(out_b[ob:ob + nb], ref_b, f"beacons P={P} T={T} c={c}")
+        op, ot, ob = op + P, ot + T, ob + nb
+
+
+@pytest.mark.parametrize("plens,tlens,c,Hq,Hkv", [
+    ([64], [40], 8, 4, 1),                 # one tile of everything
+    ([200], [300], 16, 8, 2),              # several query and key tiles, ragged tails
+    ([0, 5, 130], [33, 1, 257], 4, 12, 2), # empty prompt, G = 6 (126 of 128 rows used), T not a multiple of c
+    ([70], [150], 1, 4, 4),                # ratio 1: plain causal attention over prompt + tokens
+    ([100, 37], [260, 129], 32, 32, 8),    # the sweep's head shape
+    ([16], [520], 2, 16, 1),               # G = 16, many beacons: beacon keys span several tiles
+])
+def test_mask_form_matches_oracle(plens, tlens, c, Hq, Hkv):
+    run_case(plens, tlens, c, Hq, Hkv, seed=3)
+
+
+def test_mask_form_sharp_logits():
+    """Unscaled N(0,1) keys give logits with standard deviation ~ 1 after the softmax scale; keys
+    scaled by 4 make the rows sharply peaked, which exercises the running maximum across tiles."""
+    run_case([150], [200], 8, 8, 2, seed=9, k_scale=4.0)

@@ -627,6 +627,55 @@ def report_depth(args):
     print(json.dumps(line))
 
 
+def report_maskform(args):
+    """The mask-form pass (Section 3.2, Figure 2) on trajectories of the sweep shape: 32/8 heads,
+    D 128, prompt 512, T generated tokens, one beacon per c tokens.  A dense contraction: reported
+    in TFLOP/s against the measured bf16 tensor peak.  Useful flops = 4 * D * q_heads * (visible
+    keys summed over the token and beacon rows); flops of masked key positions are not counted."""
+    import torch
+    from paper_2510_13797_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    Hq, Hkv, D, P, n = 32, 8, 128, 512, 8
+    T = 16384 if args.steps >= 512 else 2048
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    peak = float(peaks.get("bf16_tflops", 1590.0))
+    g = torch.Generator(device=dev); g.manual_seed(0)
+    rnd = lambda *shape: torch.randn(shape, generator=g, device=dev).to(torch.bfloat16)
+    rows = []
+    for c in RATIOS:
+        nb = T // c
+        pk, pv = rnd(n * P, Hkv, D), rnd(n * P, Hkv, D)
+        tq, tk, tv = rnd(n * T, Hq, D), rnd(n * T, Hkv, D), rnd(n * T, Hkv, D)
+        bq, bk, bv = rnd(n * nb, Hq, D), rnd(n * nb, Hkv, D), rnd(n * nb, Hkv, D)
+        call = lambda check=False: B.bc_mask_attn_forward([P] * n, [T] * n, c, pk, pv, tq, tk, tv, bq, bk, bv,
+                                                          1.0 / math.sqrt(D), check=check)
+        call(check=True)
+        call()
+        torch.cuda.synchronize()
+        e0, e1 = _event_pair(torch)
+        reps = 3
+        e0.record()
+        for _ in range(reps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        keys_tok = sum(P + i // c + i % c + 1 for i in range(T))
+        keys_bea = sum(P + m + c for m in range(1, nb + 1))
+        flops = 4.0 * D * Hq * (keys_tok + keys_bea) * n
+        rows.append({"c": c, "ms": ms, "useful_tflops": flops / (ms * 1e-3) / 1e12,
+                     "frac_of_bf16_peak": flops / (ms * 1e-3) / 1e12 / peak, "rows": n * (T + nb)})
+        del pk, pv, tq, tk, tv, bq, bk, bv
+        torch.cuda.empty_cache()
+    print(json.dumps({"workload": f"maskform: {n} trajectories, 32/8 heads, D=128, P={P}, T={T}, c in {list(RATIOS)}; "
+                                  "time includes the V transposition kernels of each call",
+                      "roofline": {"bound": "tensor", "unit": "TFLOP/s", "peak": peak, "peak_source": "MEASURED_PEAKS.json bf16_tflops (burst)",
+                                   "achieved": max(r["useful_tflops"] for r in rows),
+                                   "frac": max(r["frac_of_bf16_peak"] for r in rows)},
+                      "rows": rows}))
+
+
 def batch_scaling(dev, peak):
     """The attention kernel alone at larger batches (same shape, mid-generation cache): the time per
     launch that does not stream (start-up, merging) is spread over more bytes."""
@@ -659,7 +708,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
-    ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth"],
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth", "maskform"],
                     help="sweep (default): the benchmark line; cfg2 / ragged / depth: a report line for that "
                          "BASELINE.json configuration (1 GPU)")
     ap.add_argument("--no-batch-scaling", action="store_true")
@@ -672,7 +721,7 @@ def main():
     if args.profile_case:
         return run_profile_case(args)
     if args.workload != "sweep":
-        return {"cfg2": report_cfg2, "ragged": report_ragged, "depth": report_depth}[args.workload](args)
+        return {"cfg2": report_cfg2, "ragged": report_ragged, "depth": report_depth, "maskform": report_maskform}[args.workload](args)
 
     import torch
     import torch.distributed as dist

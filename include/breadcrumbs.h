@@ -235,7 +235,7 @@ BC_API bc_status bc_compress_step_host(bc_cache* cache, int32_t layer, const int
  * [sum nb, q_heads, head_dim]; beacon_k, beacon_v [sum nb, kv_heads, head_dim]; outputs out_tok
  * [sum T, q_heads, head_dim] and out_beacon [sum nb, q_heads, head_dim], bf16 rounded to nearest
  * even from fp32 (accumulation in fp32, softmax weights rounded to bf16 before the second product).
- * head_dim must be 128 and q_heads / kv_heads <= 16 (else BC_ERR_UNSUPPORTED).  `workspace`: device
+ * head_dim must be 128 and q_heads / kv_heads <= 16 (else BC_ERR_UNSUPPORTED); sm_scale > 0.  `workspace`: device
  * memory of at least bc_mask_attn_query_bytes bytes, 256-byte aligned (it receives the tile list
  * and a transposed copy of V).  Asynchronous on `stream`; the two host arrays are read before the
  * call returns.  A bounded device-side wait that expires is reported by bc_mask_attn_status as

@@ -106,6 +106,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -134,10 +139,12 @@ struct KeySeg {
   int kind;                 // 0 prompt, 1 beacon, 2 token
 };
 
-__global__ void __launch_bounds__(kThreads, 1) k_mask_attn(const MaskArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  const uint32_t sQ = smem_addr(smem), sK = sQ + kOperandBytes, sV = sK + kOperandBytes, sP = sV + kOperandBytes;
+  // P overwrites the K tile: K is dead once S has been computed.  Three operand tiles (96 KB) let two
+  // blocks share an SM, so that one block's softmax overlaps the other's loads and products.
+  const uint32_t sQ = smem_addr(smem), sK = sQ + kOperandBytes, sV = sK + kOperandBytes, sP = sK;
   __shared__ __align__(8) uint64_t s_bar;
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
@@ -225,43 +232,64 @@ __global__ void __launch_bounds__(kThreads, 1) k_mask_attn(const MaskArgs a) {
         umma_commit(bar);
       }
       if (!mbar_wait_bounded(bar, phase)) failed = true;
+      failed = __any_sync(0xffffffffu, failed);
       phase ^= 1;
       tc_fence_after();
       // ---- mask + online softmax; this thread owns query row `tid` -----------------------------------
+      // The keys of this segment the row may see form one interval [vlo, vhi); j indexes the tile.
+      int vlo, vhi;
+      if (sg.kind == 0) { vlo = 0; vhi = sg.len; }
+      else if (sg.kind == 1) { vlo = 0; vhi = min(vis_beacons, sg.len); }
+      else { vlo = tok_lo; vhi = min(tok_hi, sg.len); }
+      if (!row_valid) vhi = vlo;
+      const int jlo = max(vlo - k0, 0), jhi = min(vhi - k0, kTile);   // visible columns of the tile
+      // Branch conditions around the warp-wide loads are made warp-uniform, so that no transformation
+      // of the loops can split a warp between two copies of a load.
+      const bool all_visible = __all_sync(0xffffffffu, jlo == 0 && jhi == kTile);
+      const bool any_visible = __any_sync(0xffffffffu, jlo < jhi);
       float tile_max = -INFINITY;
       float s[32];
-      auto visible = [&](int key) {
-        if (!row_valid || key >= sg.len) return false;
-        if (sg.kind == 0) return true;
-        if (sg.kind == 1) return key < vis_beacons;
-        return key >= tok_lo && key < tok_hi;
-      };
+      // tcgen05.ld is a warp-wide instruction: every lane executes it, whatever its row can see
+      // (`failed` is warp-uniform); only the arithmetic on the loaded values is per lane.
       if (!failed) {
 #pragma unroll 1
         for (int cb = 0; cb < 4; ++cb) {
           tmem_ld32(tS + lane_base + cb * 32, s);
+          if (all_visible) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (visible(k0 + cb * 32 + j)) tile_max = fmaxf(tile_max, s[j] * a.scale_log2);
+            for (int j = 0; j < 32; ++j) tile_max = fmaxf(tile_max, s[j]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (cb * 32 + j >= jlo && cb * 32 + j < jhi) tile_max = fmaxf(tile_max, s[j]);
+          }
         }
+        tile_max *= a.scale_log2;   // the scale is positive
       }
       const float m_new = fmaxf(m_run, tile_max);
       const float m_safe = m_new == -INFINITY ? 0.f : m_new;
-      const float alpha = exp2f(m_run - m_safe);
+      const float alpha = fast_exp2(m_run - m_safe);
       float tile_sum = 0.f;
       if (!failed) {
 #pragma unroll 1
         for (int cb = 0; cb < 4; ++cb) {
-          tmem_ld32(tS + lane_base + cb * 32, s);
           uint32_t pk[16];
+          tmem_ld32(tS + lane_base + cb * 32, s);
+          if (any_visible) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const float p0 = visible(k0 + cb * 32 + j) ? exp2f(s[j] * a.scale_log2 - m_safe) : 0.f;
-            const float p1 = visible(k0 + cb * 32 + j + 1) ? exp2f(s[j + 1] * a.scale_log2 - m_safe) : 0.f;
-            const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-            // the sum uses the rounded values, so numerator and denominator see the same weights
-            tile_sum += __low2float(pb) + __high2float(pb);
-            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+            for (int j = 0; j < 32; j += 2) {
+              float p0 = fast_exp2(fmaf(s[j], a.scale_log2, -m_safe)), p1 = fast_exp2(fmaf(s[j + 1], a.scale_log2, -m_safe));
+              if (!all_visible) {
+                if (cb * 32 + j < jlo || cb * 32 + j >= jhi) p0 = 0.f;
+                if (cb * 32 + j + 1 < jlo || cb * 32 + j + 1 >= jhi) p1 = 0.f;
+              }
+              tile_sum += p0 + p1;
+              const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+              pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) pk[j] = 0u;
           }
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)
@@ -289,6 +317,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_mask_attn(const MaskArgs a) {
         if (!mbar_wait_bounded(bar, phase)) failed = true;
         phase ^= 1;
       }
+      failed = __any_sync(0xffffffffu, failed);
       tc_fence_after();
       if (!failed) {
 #pragma unroll
@@ -408,6 +437,7 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
     return BC_ERR_INVALID_ARG;
   if (head_dim != kD || q_heads / kv_heads > 16) return BC_ERR_UNSUPPORTED;
   if (reinterpret_cast<uintptr_t>(workspace) & 255) return BC_ERR_INVALID_ARG;
+  if (!(sm_scale > 0.f)) return BC_ERR_INVALID_ARG;  // the kernel takes row maxima before scaling
   const int G = q_heads / kv_heads, per = kTile / G;
   int64_t total_prompt = cu_prompt[n_seqs], total_tokens = cu_tokens[n_seqs], total_beacons = 0;
   for (int i = 0; i < n_seqs; ++i) {
@@ -463,7 +493,7 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
   a.status = reinterpret_cast<int32_t*>(ws + l.status);
   a.Hq = q_heads; a.Hkv = kv_heads; a.G = G; a.c = c; a.rows_per_tile = per;
   a.scale_log2 = sm_scale * 1.4426950408889634f;
-  const int smem_bytes = 4 * kOperandBytes + 1024;
+  const int smem_bytes = 3 * kOperandBytes + 1024;
   if (cudaFuncSetAttribute(k_mask_attn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return BC_ERR_CUDA;
   k_mask_attn<<<dim3((unsigned)tiles.size(), kv_heads), kThreads, smem_bytes, s>>>(a);
   return cudaGetLastError() == cudaSuccess ? BC_OK : BC_ERR_CUDA;

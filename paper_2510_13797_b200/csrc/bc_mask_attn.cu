@@ -11,7 +11,8 @@
 //     (or beacons) times the G query heads that share the KV head, so a K/V tile is reused by G heads;
 //   * per key tile of 128 keys:  S = Q K^T  (tcgen05.mma, M = N = K = 128, fp32 in tensor memory)
 //     -> tcgen05.ld, mask, online softmax in fp32 registers, P as bf16 into shared memory
-//     -> O_tile = P V  (second tcgen05.mma) -> tcgen05.ld and accumulation in registers;
+//     -> O += P V  (second tcgen05.mma, accumulating in tensor memory; the rows are rescaled in place,
+//        by tcgen05.ld / tcgen05.st, only when their reference maximum has to be raised);
 //   * operands live in shared memory in the 128-byte-swizzled K-major layout the MMA descriptors
 //     describe; V is needed K-major too (keys contiguous), so a small kernel transposes V into the
 //     caller's workspace first;
@@ -106,6 +107,36 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// 32 consecutive columns of this thread's row; the registers are valid after tmem_wait_ld().
+__device__ __forceinline__ void tmem_ld32_async(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+      "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+      "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+      "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+      "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+      "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+      "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+      "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -199,16 +230,20 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
   const int thi = td.kind == 0 ? last + 1 : (last + 1) * c;
   seg[2] = {a.tok_k + (int64_t)td.tok_row * Hkv * kD, a.vt_tok + td.tok_pad, a.vt_tok_cols, (tlo / kTile) * kTile, thi, td.T, 2};
 
-  float o[kD];
-#pragma unroll
-  for (int d = 0; d < kD; ++d) o[d] = 0.f;
-  float m_run = -INFINITY, l_run = 0.f;
+  // Running state of this thread's row.  The output accumulator stays in tensor memory for the whole
+  // block: the second product adds to it, and it is rescaled in place only when the row's reference
+  // maximum moves.  The reference follows the true maximum lazily: it is raised only when a tile
+  // exceeds it by more than kMaxSlack (in the log2 domain), so the softmax weights relative to it
+  // stay below 2^kMaxSlack -- exact in the end, because numerator and denominator share the reference.
+  constexpr float kMaxSlack = 8.f;
+  float m_ref = -INFINITY, l_run = 0.f;
   uint32_t phase = 0;
   bool failed = false;
+  int n_done = 0;   // key tiles already accumulated
 
   for (int sgi = 0; sgi < 3 && !failed; ++sgi) {
     const KeySeg& sg = seg[sgi];
-    for (int k0 = sg.lo; k0 < sg.hi && !failed; k0 += kTile) {
+    for (int k0 = sg.lo; k0 < sg.hi && !failed; k0 += kTile, ++n_done) {
       // ---- K tile (rows = keys) and transposed V tile (rows = d, columns = keys) -------------------
       for (int idx = tid; idx < kTile * 16; idx += kThreads) {
         const int r = idx >> 4, ch = idx & 15;
@@ -235,7 +270,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
       failed = __any_sync(0xffffffffu, failed);
       phase ^= 1;
       tc_fence_after();
-      // ---- mask + online softmax; this thread owns query row `tid` -----------------------------------
+      // ---- mask + softmax weights; this thread owns query row `tid` ------------------------------------
       // The keys of this segment the row may see form one interval [vlo, vhi); j indexes the tile.
       int vlo, vhi;
       if (sg.kind == 0) { vlo = 0; vhi = sg.len; }
@@ -243,53 +278,48 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
       else { vlo = tok_lo; vhi = min(tok_hi, sg.len); }
       if (!row_valid) vhi = vlo;
       const int jlo = max(vlo - k0, 0), jhi = min(vhi - k0, kTile);   // visible columns of the tile
-      // Branch conditions around the warp-wide loads are made warp-uniform, so that no transformation
-      // of the loops can split a warp between two copies of a load.
+      // tcgen05.ld / tcgen05.st are warp-wide instructions: every lane executes them, whatever its row
+      // can see, and every branch around them is warp-uniform (`failed` is), so that no transformation
+      // of the code can split a warp between two copies of one of them.
       const bool all_visible = __all_sync(0xffffffffu, jlo == 0 && jhi == kTile);
-      const bool any_visible = __any_sync(0xffffffffu, jlo < jhi);
-      float tile_max = -INFINITY;
-      float s[32];
-      // tcgen05.ld is a warp-wide instruction: every lane executes it, whatever its row can see
-      // (`failed` is warp-uniform); only the arithmetic on the loaded values is per lane.
       if (!failed) {
-#pragma unroll 1
-        for (int cb = 0; cb < 4; ++cb) {
-          tmem_ld32(tS + lane_base + cb * 32, s);
-          if (all_visible) {
+        float s[kTile];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) tile_max = fmaxf(tile_max, s[j]);
-          } else {
+        for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tS + lane_base + cb * 32, s + cb * 32);
+        tmem_wait_ld();
+        float tile_max = -INFINITY;
+        if (all_visible) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (cb * 32 + j >= jlo && cb * 32 + j < jhi) tile_max = fmaxf(tile_max, s[j]);
-          }
+          for (int j = 0; j < kTile; ++j) tile_max = fmaxf(tile_max, s[j]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < kTile; ++j)
+            if (j >= jlo && j < jhi) tile_max = fmaxf(tile_max, s[j]);
         }
         tile_max *= a.scale_log2;   // the scale is positive
-      }
-      const float m_new = fmaxf(m_run, tile_max);
-      const float m_safe = m_new == -INFINITY ? 0.f : m_new;
-      const float alpha = fast_exp2(m_run - m_safe);
-      float tile_sum = 0.f;
-      if (!failed) {
-#pragma unroll 1
+        float alpha = 1.f;
+        const bool raise = tile_max > m_ref + kMaxSlack || (m_ref == -INFINITY && tile_max > -INFINITY);
+        if (raise) {
+          alpha = fast_exp2(m_ref - tile_max);   // 0 when nothing had been seen yet
+          m_ref = tile_max;
+          l_run *= alpha;
+        }
+        const float m_safe = m_ref == -INFINITY ? 0.f : m_ref;
+        float tile_sum = 0.f;
+#pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
           uint32_t pk[16];
-          tmem_ld32(tS + lane_base + cb * 32, s);
-          if (any_visible) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-              float p0 = fast_exp2(fmaf(s[j], a.scale_log2, -m_safe)), p1 = fast_exp2(fmaf(s[j + 1], a.scale_log2, -m_safe));
-              if (!all_visible) {
-                if (cb * 32 + j < jlo || cb * 32 + j >= jhi) p0 = 0.f;
-                if (cb * 32 + j + 1 < jlo || cb * 32 + j + 1 >= jhi) p1 = 0.f;
-              }
-              tile_sum += p0 + p1;
-              const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-              pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+          for (int j = 0; j < 32; j += 2) {
+            float p0 = fast_exp2(fmaf(s[cb * 32 + j], a.scale_log2, -m_safe));
+            float p1 = fast_exp2(fmaf(s[cb * 32 + j + 1], a.scale_log2, -m_safe));
+            if (!all_visible) {
+              if (cb * 32 + j < jlo || cb * 32 + j >= jhi) p0 = 0.f;
+              if (cb * 32 + j + 1 < jlo || cb * 32 + j + 1 >= jhi) p1 = 0.f;
             }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 16; ++j) pk[j] = 0u;
+            tile_sum += p0 + p1;
+            const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
           }
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)
@@ -297,46 +327,59 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
                          "r"(pk[q4 * 4 + 1]), "r"(pk[q4 * 4 + 2]), "r"(pk[q4 * 4 + 3])
                          : "memory");
         }
+        l_run += tile_sum;
+        // ---- rescale the accumulator rows whose reference moved (whole warp, if any lane needs it) --------
+        if (n_done > 0 && __any_sync(0xffffffffu, raise)) {
+#pragma unroll 1
+          for (int cb = 0; cb < 4; ++cb) {
+            float t[32];
+            tmem_ld32_async(tO + lane_base + cb * 32, t);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) t[j] *= alpha;
+            tmem_st32(tO + lane_base + cb * 32, t);
+          }
+          tmem_wait_st();
+        }
       }
-      m_run = m_new;
-      l_run = l_run * alpha + tile_sum;
       proxy_fence();
       tc_fence_before();
       __syncthreads();
-      // ---- O_tile = P V ------------------------------------------------------------------------------
+      // ---- O += P V ----------------------------------------------------------------------------------
       if (tid == 0 && !failed) {
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < kTile / 16; ++kk) {
           const uint32_t off = (uint32_t)((kk >> 2) * (kTile * 128) + (kk & 3) * 32);
-          umma(tO, umma_desc(sP + off), umma_desc(sV + off), kk > 0);
+          umma(tO, umma_desc(sP + off), umma_desc(sV + off), (n_done > 0 || kk > 0) ? 1u : 0u);
         }
         umma_commit(bar);
       }
+      // the product must have read P and V before the next tile's copies overwrite them
       if (!failed) {
         if (!mbar_wait_bounded(bar, phase)) failed = true;
         phase ^= 1;
       }
       failed = __any_sync(0xffffffffu, failed);
       tc_fence_after();
-      if (!failed) {
-#pragma unroll
-        for (int cb = 0; cb < 4; ++cb) {
-          tmem_ld32(tO + lane_base + cb * 32, s);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[cb * 32 + j] = o[cb * 32 + j] * alpha + s[j];
-        }
-      }
-      tc_fence_before();
       if (failed) s_fail = 1;
-      __syncthreads();   // K, V, P and both accumulators are free for the next tile
+      __syncthreads();
       if (s_fail) failed = true;
     }
   }
 
+  // ---- read the accumulator --------------------------------------------------------------------------
+  float o[kD];
+  if (!failed) {
+#pragma unroll
+    for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tO + lane_base + cb * 32, o + cb * 32);
+    tmem_wait_ld();
+  }
+  const float l_fin = l_run;
+
   // ---- write the rows -------------------------------------------------------------------------------
   if (!failed && row_valid) {
-    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    const float inv = l_fin > 0.f ? 1.f / l_fin : 0.f;
     __nv_bfloat16* dst = (td.kind == 0 ? a.out_tok + (int64_t)(td.tok_row + my_idx) * Hq * kD
                                        : a.out_bea + (int64_t)(td.bea_row + my_idx) * Hq * kD) +
                          (int64_t)(kvh * G + tid % G) * kD;

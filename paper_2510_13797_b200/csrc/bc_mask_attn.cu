@@ -245,12 +245,23 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
     const KeySeg& sg = seg[sgi];
     for (int k0 = sg.lo; k0 < sg.hi && !failed; k0 += kTile, ++n_done) {
       // ---- K tile (rows = keys) and transposed V tile (rows = d, columns = keys) -------------------
-      for (int idx = tid; idx < kTile * 16; idx += kThreads) {
-        const int r = idx >> 4, ch = idx & 15;
-        if (k0 + r < sg.len) cp16(sK + swz(r, ch), sg.k + ((int64_t)(k0 + r) * Hkv + kvh) * kD + ch * 8);
-        else st_zero16(sK + swz(r, ch));
-        // columns beyond the sequence's rows are zero in the transposed array (it is padded to 128)
-        cp16(sV + swz(r, ch), sg.vt + ((int64_t)kvh * kD + r) * sg.vt_cols + k0 + ch * 8);
+      // Thread t copies chunk (t & 15) of rows (t >> 4) + 8 i, i = 0..15: row & 7 does not depend on i,
+      // so the swizzled shared-memory offset and both global addresses advance by constant strides.
+      {
+        const int r0 = tid >> 4, ch = tid & 15;
+        uint32_t dk = sK + swz(r0, ch), dv = sV + swz(r0, ch);
+        const __nv_bfloat16* gk = sg.k + ((int64_t)(k0 + r0) * Hkv + kvh) * kD + ch * 8;
+        const __nv_bfloat16* gv = sg.vt + ((int64_t)kvh * kD + r0) * sg.vt_cols + k0 + ch * 8;
+        const int64_t gk_step = (int64_t)8 * Hkv * kD, gv_step = 8 * sg.vt_cols;
+        const int rows_here = sg.len - k0 - r0;   // rows k0 + r0 + 8 i exist while 8 i < rows_here
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          if (8 * i < rows_here) cp16(dk, gk);
+          else st_zero16(dk);
+          // columns beyond the sequence's rows are zero in the transposed array (it is padded to 128)
+          cp16(dv, gv);
+          dk += 8 * 128; dv += 8 * 128; gk += gk_step; gv += gv_step;
+        }
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
       asm volatile("cp.async.wait_group 0;" ::: "memory");

@@ -1,0 +1,54 @@
+"""Random programs of open / append / compress / close against the oracle's paging model.
+
+Small pools and odd page sizes make the programs hit every refusal (no pages, window full, window
+not full, bad slot, capacity); after every call the lengths, page lists, free stack and the latched
+first error must be those of the integer-only model, bit for bit, and at the end of a program every
+sequence is closed and every page is back."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_13797_b200 import binding as B
+from tests.harness import Pair, randn_bf16
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.mark.parametrize("seed,ps,num_pages,max_pps,max_entries", [
+    (0, 1, 40, 12, 0), (1, 2, 24, 8, 0), (2, 3, 30, 9, 7), (3, 4, 64, 16, 0), (4, 16, 12, 4, 0), (5, 5, 50, 6, 11),
+])
+def test_random_programs(seed, ps, num_pages, max_pps, max_entries):
+    rng = np.random.RandomState(seed)
+    S, Hkv, G, D = 8, 1, 2, 64
+    pair = Pair(1, Hkv, Hkv * G, D, ps, max_seqs=S, num_pages=num_pages, max_pages_per_seq=max_pps,
+                max_entries=max_entries, c_default=int(rng.choice([1, 2, 3, 5])))
+    g = torch.Generator(device=DEV); g.manual_seed(seed)
+    kv = lambda n: (randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV))
+    for step in range(160):
+        op = rng.choice(["open", "append", "append", "append", "compress", "close"])
+        n = int(rng.randint(1, S + 1))
+        slots = [int(x) for x in rng.choice(S + 2, size=n, replace=False) - 1]      # -1 and S are invalid slots
+        if op == "open":
+            plens = [int(rng.randint(0, 3 * ps + 2)) for _ in slots]
+            cs = None if rng.rand() < 0.3 else [int(rng.choice([1, 2, 3, 4, 7])) for _ in slots]
+            pair.open(slots, plens, cs)
+        elif op == "append":
+            pair.append(0, slots, *kv(n))
+        elif op == "compress":
+            # favour the sequences whose window is full, so that compressions succeed too
+            full = [s for s in range(S) if (st := pair.model.state(s)) and st["c"] > 1 and st["window_len"] == st["c"]]
+            if full and rng.rand() < 0.7:
+                slots = full[:n]
+            pair.compress(0, slots, *kv(len(slots)))
+        else:
+            pair.close(slots)
+        pair.check_state()
+        if pair.model.first_error is not None and rng.rand() < 0.5:
+            pair.gpu.bc_clear_error(); pair.model.first_error = None
+    open_slots = [s for s in range(S) if pair.model.state(s) is not None]
+    if open_slots:
+        pair.close(open_slots)
+    pair.gpu.bc_clear_error(); pair.model.first_error = None
+    pair.check_state()
+    assert sorted(pair.gpu.bc_get_free_list()) == list(range(num_pages))

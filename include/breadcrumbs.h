@@ -255,6 +255,28 @@ BC_API bc_status bc_mask_attn_status(const void* workspace, int32_t n_seqs, int3
                                      int64_t total_prompt, int64_t total_tokens, int64_t total_beacons,
                                      void* stream, int32_t* code);
 
+/* ---- the distillation loss (Section 3.2, Eq. 1) -------------------------------------------------
+ * loss = (1 / n_traj) * sum_b (1 / |x_b|) * sum_{positions r of trajectory b} KL_K(teacher_r || student_r),
+ * the mean over the batch of the per-trajectory mean token-level divergence between the frozen
+ * uncompressed teacher and the compressed student.  The teacher is given the way the paper stores
+ * it (Implementation Details: the top 100 entries per time step, more than 90 % of the mass): for
+ * every position top_k vocabulary indices (distinct, in [0, vocab)) and the teacher's
+ * log-probabilities of those entries under its full-vocabulary normalisation; -inf marks an unused
+ * entry.  KL_K(p || q) = sum over the stored entries of p_k (log p_k - log q_k), q = softmax of the
+ * student's logits over the whole vocabulary; with top_k = vocab this is Eq. 1 exactly (the paper
+ * does not say how the stored entries are normalised; this is the reading taken).
+ *
+ * Device pointers: cu_rows int32[n_traj + 1] prefix sums of the trajectories' positions
+ * (cu_rows[n_traj] == rows); student_logits bf16 [rows, vocab]; teacher_idx int32 [rows, top_k];
+ * teacher_logprob fp32 [rows, top_k]; row_loss fp32 [rows] (KL_K of every position, written);
+ * loss fp32 [1] (written).  grad: NULL, or bf16 [rows, vocab] receiving d loss / d student_logits =
+ * w_r (q_j sum_k p_k - p_j [j stored]), w_r = 1 / (n_traj |x_b|); it must have the same 16-byte
+ * phase as student_logits.  fp32 arithmetic; additions in a fixed order (results are reproducible).
+ * Asynchronous on `stream`; nothing is allocated. */
+BC_API bc_status bc_distill_loss(int32_t n_traj, const int32_t* cu_rows, int64_t rows, int32_t vocab, int32_t top_k,
+                                 const void* student_logits, const int32_t* teacher_idx,
+                                 const float* teacher_logprob, float* row_loss, float* loss, void* grad, void* stream);
+
 /* ---- inspection (these synchronise `stream`; for tests and tools) ---------------------------- */
 
 /* Bookkeeping of one slot.  pages (host, may be NULL) receives up to pages_cap page ids: prompt

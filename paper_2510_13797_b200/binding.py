@@ -62,6 +62,7 @@ SYMBOLS = {
     "bc_mask_attn_forward": (_I32, [_I32, _I32, _I32, _I32, _I32, C.POINTER(_I32), C.POINTER(_I32)] + [_P] * 10
                              + [_F, _P, C.c_size_t, _P]),
     "bc_mask_attn_status": (_I32, [_P, _I32, _I32, _I32, _I64, _I64, _I64, _P, C.POINTER(_I32)]),
+    "bc_distill_loss": (_I32, [_I32, _P, _I64, _I32, _I32, _P, _P, _P, _P, _P, _P, _P]),
     "bc_compress": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
     "bc_seq_close": (_I32, [_P, _P, _I32, _P]),
     "bc_decode_step_host": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P]),
@@ -261,3 +262,20 @@ def bc_mask_attn_forward(prompt_lens, token_lens, c, prompt_k, prompt_v, tok_q, 
                                          C.byref(code)), "bc_mask_attn_status")
         _check(code.value, "bc_mask_attn_forward (device)")
     return out_tok, out_bea
+
+
+def bc_distill_loss(cu_rows, student_logits, teacher_idx, teacher_logprob, with_grad=False, stream=None):
+    """Eq. 1 (breadcrumbs.h): returns (loss [1] fp32, row_loss [rows] fp32, grad or None).
+
+    cu_rows: int32 CUDA tensor [n_traj + 1]; student_logits bf16 [rows, vocab]; teacher_idx int32 and
+    teacher_logprob fp32 [rows, top_k]."""
+    rows, vocab = student_logits.shape
+    top_k = teacher_idx.shape[1]
+    dev = student_logits.device
+    row_loss = torch.empty(rows, dtype=torch.float32, device=dev)
+    loss = torch.empty(1, dtype=torch.float32, device=dev)
+    grad = torch.empty_like(student_logits) if with_grad else None
+    _check(lib().bc_distill_loss(cu_rows.numel() - 1, _ptr(cu_rows), rows, vocab, top_k, _ptr(student_logits),
+                                 _ptr(teacher_idx), _ptr(teacher_logprob), _ptr(row_loss), _ptr(loss), _ptr(grad),
+                                 _stream(stream)), "bc_distill_loss")
+    return loss, row_loss, grad

@@ -676,6 +676,50 @@ def report_maskform(args):
                       "rows": rows}))
 
 
+def report_distill(args):
+    """The distillation loss (Eq. 1) at the vocabulary of the 1.5B model the paper trains (151,936)
+    with the paper's 100 stored teacher entries per position: 16 trajectories of 1,000 positions
+    (the paper's maximum response length).  One streaming read of the student logits: HBM-bound.
+    Algorithmic bytes: rows * vocab * 2 (logits) + rows * 100 * 8 (teacher entries); with the
+    gradient, another rows * vocab * 2 written (the second read of a row comes from L2)."""
+    import torch
+    from paper_2510_13797_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peak, peak_src = load_peaks()
+    n_traj, T, V, K = 16, 1000, 151936, 100
+    rows = n_traj * T
+    g = torch.Generator(device=dev); g.manual_seed(0)
+    z = torch.empty((rows, V), dtype=torch.bfloat16, device=dev)
+    for a in range(0, rows, 2000):                         # drawn in slabs: fp32 randn of the whole matrix would be 9.7 GB
+        z[a:a + 2000] = (torch.randn((min(2000, rows - a), V), generator=g, device=dev) * 3).to(torch.bfloat16)
+    idx = torch.stack([torch.randperm(V, generator=g, device=dev)[:K] for _ in range(64)]).to(torch.int32)
+    idx = idx.repeat(rows // 64, 1).contiguous()
+    lp = torch.log_softmax(torch.randn((rows, K), generator=g, device=dev) * 2, dim=1).to(torch.float32) + math.log(0.93)
+    cu = torch.arange(0, rows + 1, T, dtype=torch.int32, device=dev)
+    out = {}
+    for with_grad in (False, True):
+        for _ in range(2):
+            B.bc_distill_loss(cu, z, idx, lp, with_grad=with_grad)
+        torch.cuda.synchronize()
+        e0, e1 = _event_pair(torch)
+        reps = 5
+        e0.record()
+        for _ in range(reps):
+            loss, _, _ = B.bc_distill_loss(cu, z, idx, lp, with_grad=with_grad)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / reps
+        nbytes = rows * V * 2 * (2 if with_grad else 1) + rows * K * 8
+        out["forward_backward" if with_grad else "forward"] = {
+            "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak,
+            "algorithmic_bytes": nbytes, "positions_per_s": rows / (ms * 1e-3)}
+    print(json.dumps({"workload": f"distill: {n_traj} trajectories x {T} positions, vocab {V}, top-{K} teacher entries, bf16 logits",
+                      "loss": float(loss), "roofline": {"bound": "hbm", "unit": "GB/s", "peak": peak, "peak_source": peak_src,
+                                                       "achieved": out["forward"]["gbs"], "frac": out["forward"]["frac_of_peak"]},
+                      **out}))
+
+
 def batch_scaling(dev, peak):
     """The attention kernel alone at larger batches (same shape, mid-generation cache): the time per
     launch that does not stream (start-up, merging) is spread over more bytes."""
@@ -708,7 +752,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
-    ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth", "maskform"],
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth", "maskform", "distill"],
                     help="sweep (default): the benchmark line; cfg2 / ragged / depth: a report line for that "
                          "BASELINE.json configuration (1 GPU)")
     ap.add_argument("--no-batch-scaling", action="store_true")
@@ -721,7 +765,7 @@ def main():
     if args.profile_case:
         return run_profile_case(args)
     if args.workload != "sweep":
-        return {"cfg2": report_cfg2, "ragged": report_ragged, "depth": report_depth, "maskform": report_maskform}[args.workload](args)
+        return {"cfg2": report_cfg2, "ragged": report_ragged, "depth": report_depth, "maskform": report_maskform, "distill": report_distill}[args.workload](args)
 
     import torch
     import torch.distributed as dist

@@ -127,8 +127,7 @@ __global__ void __launch_bounds__(kRowThreads) k_kl_rows(const __nv_bfloat16* __
   __nv_bfloat16* g = grad + r * vocab;   // same alignment as z: rows have the same stride
   if (tid < head) g[tid] = __float2bfloat16_rn(coef * ex2(fmaf(__bfloat162float(z[tid]), kLog2e, -lse2)));
   uint4* gv = reinterpret_cast<uint4*>(g + head);
-  for (int j = tid; j < nvec; j += kRowThreads) {
-    const uint4 v = zv[j];
+  auto grad8 = [&](const uint4& v) {
     const uint32_t in[4] = {v.x, v.y, v.z, v.w};
     uint32_t o[4];
 #pragma unroll
@@ -137,8 +136,15 @@ __global__ void __launch_bounds__(kRowThreads) k_kl_rows(const __nv_bfloat16* __
                                                      coef * ex2(fmaf(bf_hi(in[q]), kLog2e, -lse2)));
       o[q] = *reinterpret_cast<const uint32_t*>(&t);
     }
-    __stcs(gv + j, make_uint4(o[0], o[1], o[2], o[3]));
+    return make_uint4(o[0], o[1], o[2], o[3]);
+  };
+  int j = tid;
+  for (; j + 3 * kRowThreads < nvec; j += 4 * kRowThreads) {   // four loads in flight per thread
+    const uint4 a = zv[j], b = zv[j + kRowThreads], c = zv[j + 2 * kRowThreads], d = zv[j + 3 * kRowThreads];
+    __stcs(gv + j, grad8(a)); __stcs(gv + j + kRowThreads, grad8(b));
+    __stcs(gv + j + 2 * kRowThreads, grad8(c)); __stcs(gv + j + 3 * kRowThreads, grad8(d));
   }
+  for (; j < nvec; j += kRowThreads) __stcs(gv + j, grad8(zv[j]));
   if (tail0 + tid < vocab) g[tail0 + tid] = __float2bfloat16_rn(coef * ex2(fmaf(__bfloat162float(z[tail0 + tid]), kLog2e, -lse2)));
   __syncthreads();   // the dense row is written; the stored entries overwrite their elements
   for (int k = tid; k < top_k; k += kRowThreads) {

@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the Breadcrumbs decode hot path on B200.
 
-Workload (benchmark configs[2], the compression-ratio sweep): one layer, batch 64, 32 query /
+Workload (the compression-ratio sweep): one layer, batch 64, 32 query /
 8 KV heads, head_dim 128, bf16, prompt 512, 16384 decode steps, c in {2,4,8,16,32} with
 page_size = c, plus the uncompressed run (c = 1, page 16) as a reported row.
 
@@ -342,7 +342,7 @@ def _event_pair(torch):
 
 
 def report_cfg2(args):
-    """Benchmark configs[1]: batch 32, 12/2 heads, prompt 256, 4096 steps, c = 16.  ~13 MB of KV
+    """The small single-layer configuration: batch 32, 12/2 heads, prompt 256, 4096 steps, c = 16.  ~13 MB of KV
     per step: L2-resident and launch-bound, so the figures are microseconds per call."""
     import torch
     from paper_2510_13797_b200.workloads import make_workload
@@ -384,7 +384,7 @@ def report_cfg2(args):
 
 
 def report_ragged(args):
-    """Benchmark configs[3]: batch 128, 12/2 heads, page 16; prompt U[64,1024], generation
+    """The ragged configuration: batch 128, 12/2 heads, page 16; prompt U[64,1024], generation
     U[1024,32768], c from {4,8,16} per sequence.  The whole run, plain launches: sequences finish at
     their own step and free their pages on the device."""
     import numpy as np
@@ -484,7 +484,7 @@ def report_ragged(args):
 
 
 def report_depth(args):
-    """Benchmark configs[4]: 28 layers, batch 256, 12/2 heads, prompt 512, 8192 steps, c = 8,
+    """The full-depth configuration: 28 layers, batch 256, 12/2 heads, prompt 512, 8192 steps, c = 8,
     page 8.  Per-layer calls in dependency order, whole windows of 8 steps as one CUDA graph, at the
     middle of the generation; footprint against the uncompressed cache; the largest batch one GPU
     holds at c in {1, 4, 8, 16}, computed from the free memory and demonstrated at c = 8."""
@@ -754,7 +754,7 @@ def main():
     ap.add_argument("--skip-uncompressed", action="store_true")
     ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth", "maskform", "distill"],
                     help="sweep (default): the benchmark line; cfg2 / ragged / depth: a report line for that "
-                         "BASELINE.json configuration (1 GPU)")
+                         "benchmark configuration (1 GPU)")
     ap.add_argument("--no-batch-scaling", action="store_true")
     ap.add_argument("--profile-case", type=int, default=0, metavar="C",
                     help="small case for profilers: ratio C with a prompt as long as the mid-generation cache, "

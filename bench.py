@@ -306,7 +306,7 @@ def run_reference(args):
     cores = max(1, round(total_cpu / total_wall))
     sample = f"{seqs} of 64 sequences per ratio, {K} decode steps at the mid-generation cache state, c in {list(RATIOS)}"
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": 0, "steps": K,
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus, "steps": K,
         "warmup": W, "ms_per_step": 1e3 * total_wall / K, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": "sweep: B=64, 32/8 heads, D=128, P=512, T=16384, c in {2,4,8,16,32} (CPU oracle on a sample)"},

@@ -238,8 +238,9 @@ BC_API bc_status bc_compress_step_host(bc_cache* cache, int32_t layer, const int
  * head_dim must be 128 and q_heads / kv_heads <= 16 (else BC_ERR_UNSUPPORTED); sm_scale > 0.  `workspace`: device
  * memory of at least bc_mask_attn_query_bytes bytes, 256-byte aligned (it receives the tile list
  * and a transposed copy of V).  Asynchronous on `stream`; the two host arrays are read before the
- * call returns.  A bounded device-side wait that expires is reported by bc_mask_attn_status as
- * BC_ERR_TIMEOUT (the outputs are then incomplete). */
+ * call returns (pageable host memory is staged by the copy, so do not call this inside a stream
+ * capture).  One call at a time per workspace.  A bounded device-side wait that expires is reported
+ * by bc_mask_attn_status as BC_ERR_TIMEOUT (the outputs are then incomplete). */
 BC_API bc_status bc_mask_attn_query_bytes(int32_t n_seqs, int32_t q_heads, int32_t kv_heads, int32_t head_dim,
                                           int64_t total_prompt, int64_t total_tokens, int64_t total_beacons,
                                           size_t* workspace_bytes);

@@ -14,12 +14,15 @@
 //     -> O += P V  (second tcgen05.mma, accumulating in tensor memory; the rows are rescaled in place,
 //        by tcgen05.ld / tcgen05.st, only when their reference maximum has to be raised);
 //   * operands live in shared memory in the 128-byte-swizzled K-major layout the MMA descriptors
-//     describe; V is needed K-major too (keys contiguous), so a small kernel transposes V into the
-//     caller's workspace first;
+//     describe, written by tiled tensor copies (cp.async.bulk.tensor, 128-byte swizzle, completion
+//     on an mbarrier) issued by one thread; V is needed K-major too (keys contiguous), so a small
+//     kernel transposes V into the caller's workspace first;
 //   * key tiles a query tile cannot see are skipped: all prompt tiles, the beacon tiles up to its
 //     last visible beacon, and the token tiles that overlap its own windows.
 // Every wait is bounded; on expiry the block records BC_ERR_TIMEOUT, releases its tensor memory and
 // returns.
+#include <cuda.h>
+
 #include <vector>
 
 #include "bc_common.cuh"
@@ -42,11 +45,14 @@ struct TileDesc {
   int32_t pad[4];
 };
 
+// Tensor maps (bf16, 128-byte swizzle): q [d, head, row] boxes of (64, G, tokens per tile); k [d, head, row]
+// boxes of (64, 1, 128); transposed v [column, head * 128 + d] boxes of (64, 128).
+struct MaskMaps {
+  CUtensorMap q_tok, q_bea, k_prompt, k_tok, k_bea, vt_prompt, vt_tok, vt_bea;
+};
+
 struct MaskArgs {
   const TileDesc* tiles;
-  const __nv_bfloat16 *prompt_k, *tok_q, *tok_k, *bea_q, *bea_k;
-  const __nv_bfloat16 *vt_prompt, *vt_tok, *vt_bea;  // [Hkv][D][padded columns]
-  int64_t vt_prompt_cols, vt_tok_cols, vt_bea_cols;  // padded columns per (head, d) row
   __nv_bfloat16 *out_tok, *out_bea;
   int32_t* status;     // device int: first error code
   int32_t Hq, Hkv, G, c, rows_per_tile;  // rows_per_tile = tokens per query tile = 128 / G
@@ -62,8 +68,21 @@ __device__ __forceinline__ uint32_t swz(int r, int ch16) {
   return (uint32_t)((ch16 >> 3) * (kTile * 128) + r * 128 + (((ch16 & 7) ^ (r & 7)) << 4));
 }
 
-__device__ __forceinline__ void cp16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+// Tiled tensor copies global -> shared memory, completing on an mbarrier.  The innermost coordinate
+// is a multiple of 64 bf16 elements (128 bytes) in every call.
+__device__ __forceinline__ void tma_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+               "l"(map), "r"(c0), "r"(c1), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void st_zero16(uint32_t dst) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(dst), "r"(0) : "memory");
@@ -147,30 +166,32 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 
 // One key segment of a sequence as the main loop sees it.
 struct KeySeg {
-  const __nv_bfloat16* k;   // [rows][Hkv][D], first row of the sequence
-  const __nv_bfloat16* vt;  // transposed V: row (head, d), first column of the sequence
-  int64_t vt_cols;          // columns per vt row
+  const CUtensorMap* k;     // tensor map of the K array of this kind
+  const CUtensorMap* vt;    // tensor map of the transposed V array
+  int row0, col0;           // first row of the sequence in K, first column in the transposed V
   int lo, hi;               // keys [lo, hi) of the segment are candidates (lo a multiple of 128)
   int len;                  // rows that exist
   int kind;                 // 0 prompt, 1 beacon, 2 token
 };
 
-__global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
+__global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, const __grid_constant__ MaskMaps maps) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   // P overwrites the K tile: K is dead once S has been computed.  Three operand tiles (96 KB) let two
   // blocks share an SM, so that one block's softmax overlaps the other's loads and products.
   const uint32_t sQ = smem_addr(smem), sK = sQ + kOperandBytes, sV = sK + kOperandBytes, sP = sK;
   __shared__ __align__(8) uint64_t s_bar;
+  __shared__ __align__(8) uint64_t s_load_bar;
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
-  const uint32_t bar = smem_addr(&s_bar);
+  const uint32_t bar = smem_addr(&s_bar), load_bar = smem_addr(&s_load_bar);
   const int tid = threadIdx.x, warp = tid >> 5;
   const TileDesc td = a.tiles[blockIdx.x];
-  const int kvh = blockIdx.y, G = a.G, Hq = a.Hq, Hkv = a.Hkv, c = a.c;
+  const int kvh = blockIdx.y, G = a.G, Hq = a.Hq, c = a.c;
 
   if (tid == 0) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(load_bar) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     s_fail = 0;
   }
@@ -180,19 +201,29 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
   }
 
   // ---- the query tile: row r = (local index r / G, head r % G) ---------------------------------
-  const __nv_bfloat16* qsrc = td.kind == 0 ? a.tok_q + (int64_t)(td.tok_row + td.first) * Hq * kD
-                                           : a.bea_q + (int64_t)(td.bea_row + td.first) * Hq * kD;
   const int valid_rows = td.count * G;
-  for (int idx = tid; idx < kTile * 16; idx += kThreads) {
-    const int r = idx >> 4, ch = idx & 15;
-    if (r < valid_rows) cp16(sQ + swz(r, ch), qsrc + ((int64_t)(r / G) * Hq + kvh * G + (r % G)) * kD + ch * 8);
-    else st_zero16(sQ + swz(r, ch));
+  const int box_rows = a.rows_per_tile * G;   // rows the tensor copy writes (all 128 unless G does not divide 128)
+  for (int idx = tid; idx < (kTile - box_rows) * 16; idx += kThreads) {   // rows the copy leaves untouched
+    const int r = box_rows + (idx >> 4), ch = idx & 15;
+    st_zero16(sQ + swz(r, ch));
   }
-  asm volatile("cp.async.commit_group;" ::: "memory");
-
+  proxy_fence();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  uint32_t load_phase = 0;
+  if (tid == 0) {
+    // rows beyond the tile's tokens belong to the next sequence or are zero-filled: they are never
+    // visible (their outputs are not written and they contribute to no other row)
+    mbar_expect_tx(load_bar, (uint32_t)(box_rows * kD * 2));
+    const CUtensorMap* qm = td.kind == 0 ? &maps.q_tok : &maps.q_bea;
+    const int qrow = (td.kind == 0 ? td.tok_row : td.bea_row) + td.first;
+    tma_3d(sQ, qm, 0, kvh * G, qrow, load_bar);
+    tma_3d(sQ + kTile * 128, qm, 64, kvh * G, qrow, load_bar);
+  }
+  bool failed = !mbar_wait_bounded(load_bar, load_phase);
+  failed = __any_sync(0xffffffffu, failed);
+  load_phase ^= 1;
   const uint32_t tmem = s_tmem;
   const uint32_t tS = tmem, tO = tmem + kTile;                 // columns [0,128) and [128,256)
   const uint32_t lane_base = (uint32_t)(warp * 32) << 16;      // this warp's 32 lanes of tensor memory
@@ -208,12 +239,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
   // ---- key segments and the tiles of each that some row of this block can see ----------------------
   const int last = td.first + td.count - 1;
   KeySeg seg[3];
-  seg[0] = {a.prompt_k + (int64_t)td.prompt_row * Hkv * kD, a.vt_prompt + td.prompt_pad, a.vt_prompt_cols, 0, td.P, td.P, 0};
+  seg[0] = {&maps.k_prompt, &maps.vt_prompt, td.prompt_row, td.prompt_pad, 0, td.P, td.P, 0};
   const int bmax = td.kind == 0 ? (c > 1 ? last / c : 0) : last + 1;
-  seg[1] = {a.bea_k + (int64_t)td.bea_row * Hkv * kD, a.vt_bea + td.bea_pad, a.vt_bea_cols, 0, bmax, td.nb, 1};
+  seg[1] = {&maps.k_bea, &maps.vt_bea, td.bea_row, td.bea_pad, 0, bmax, td.nb, 1};
   const int tlo = td.kind == 0 ? (c > 1 ? (td.first / c) * c : 0) : td.first * c;
   const int thi = td.kind == 0 ? last + 1 : (last + 1) * c;
-  seg[2] = {a.tok_k + (int64_t)td.tok_row * Hkv * kD, a.vt_tok + td.tok_pad, a.vt_tok_cols, (tlo / kTile) * kTile, thi, td.T, 2};
+  seg[2] = {&maps.k_tok, &maps.vt_tok, td.tok_row, td.tok_pad, (tlo / kTile) * kTile, thi, td.T, 2};
 
   // Running state of this thread's row.  The output accumulator stays in tensor memory for the whole
   // block: the second product adds to it, and it is rescaled in place only when the row's reference
@@ -223,37 +254,29 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
   constexpr float kMaxSlack = 8.f;
   float m_ref = -INFINITY, l_run = 0.f;
   uint32_t phase = 0;
-  bool failed = false;
   int n_done = 0;   // key tiles already accumulated
 
   for (int sgi = 0; sgi < 3 && !failed; ++sgi) {
     const KeySeg& sg = seg[sgi];
     for (int k0 = sg.lo; k0 < sg.hi && !failed; k0 += kTile, ++n_done) {
       // ---- K tile (rows = keys) and transposed V tile (rows = d, columns = keys) -------------------
-      // Thread t copies chunk (t & 15) of rows (t >> 4) + 8 i, i = 0..15: row & 7 does not depend on i,
-      // so the swizzled shared-memory offset and both global addresses advance by constant strides.
-      {
-        const int r0 = tid >> 4, ch = tid & 15;
-        uint32_t dk = sK + swz(r0, ch), dv = sV + swz(r0, ch);
-        const __nv_bfloat16* gk = sg.k + ((int64_t)(k0 + r0) * Hkv + kvh) * kD + ch * 8;
-        const __nv_bfloat16* gv = sg.vt + ((int64_t)kvh * kD + r0) * sg.vt_cols + k0 + ch * 8;
-        const int64_t gk_step = (int64_t)8 * Hkv * kD, gv_step = 8 * sg.vt_cols;
-        const int rows_here = sg.len - k0 - r0;   // rows k0 + r0 + 8 i exist while 8 i < rows_here
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          if (8 * i < rows_here) cp16(dk, gk);
-          else st_zero16(dk);
-          // columns beyond the sequence's rows are zero in the transposed array (it is padded to 128)
-          cp16(dv, gv);
-          dk += 8 * 128; dv += 8 * 128; gk += gk_step; gv += gv_step;
-        }
-      }
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
-      proxy_fence();
-      __syncthreads();
-      // ---- S = Q K^T ---------------------------------------------------------------------------------
+      // Rows beyond the sequence's keys hold the next sequence's keys (or zeros past the end of the
+      // array): they are masked below.  The transposed V is zero there (padded to 128 columns).
       if (tid == 0) {
+        mbar_expect_tx(load_bar, 2u * kOperandBytes);
+        tma_3d(sK, sg.k, 0, kvh, sg.row0 + k0, load_bar);
+        tma_3d(sK + kTile * 128, sg.k, 64, kvh, sg.row0 + k0, load_bar);
+        tma_2d(sV, sg.vt, sg.col0 + k0, kvh * kD, load_bar);
+        tma_2d(sV + kTile * 128, sg.vt, sg.col0 + k0 + 64, kvh * kD, load_bar);
+      }
+      if (!mbar_wait_bounded(load_bar, load_phase)) failed = true;
+      failed = __any_sync(0xffffffffu, failed);
+      load_phase ^= 1;
+      if (failed) s_fail = 1;
+      __syncthreads();
+      if (s_fail) failed = true;
+      // ---- S = Q K^T ---------------------------------------------------------------------------------
+      if (tid == 0 && !failed) {
         tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
@@ -262,7 +285,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a) {
         }
         umma_commit(bar);
       }
-      if (!mbar_wait_bounded(bar, phase)) failed = true;
+      if (!failed && !mbar_wait_bounded(bar, phase)) failed = true;
       failed = __any_sync(0xffffffffu, failed);
       phase ^= 1;
       tc_fence_after();
@@ -422,6 +445,39 @@ __global__ void k_transpose_v(const __nv_bfloat16* __restrict__ v, __nv_bfloat16
   }
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against the driver library).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+// [rows][heads][128] bf16 seen as (d, head, row); box (64, box_heads, box_rows); out-of-range elements read as zero
+bool map_3d(CUtensorMap* m, const void* base, int heads, int64_t rows, int box_heads, int box_rows) {
+  const cuuint64_t dims[3] = {(cuuint64_t)kD, (cuuint64_t)heads, (cuuint64_t)(rows > 0 ? rows : 1)};
+  const cuuint64_t strides[2] = {(cuuint64_t)kD * 2, (cuuint64_t)heads * kD * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows}, es[3] = {1, 1, 1};
+  return encode_tiled()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// [rows][cols] bf16 seen as (col, row); box (64, 128)
+bool map_2d(CUtensorMap* m, const void* base, int64_t cols, int64_t rows) {
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kTile}, es[2] = {1, 1};
+  return encode_tiled()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int64_t pad128(int64_t x) { return (x + 127) / 128 * 128; }
 
@@ -525,17 +581,25 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
 
   MaskArgs a;
   a.tiles = reinterpret_cast<const TileDesc*>(ws + l.tiles);
-  a.prompt_k = (const __nv_bfloat16*)prompt_k; a.tok_q = (const __nv_bfloat16*)tok_q; a.tok_k = (const __nv_bfloat16*)tok_k;
-  a.bea_q = (const __nv_bfloat16*)beacon_q; a.bea_k = (const __nv_bfloat16*)beacon_k;
-  a.vt_prompt = vt(l.vt_prompt); a.vt_tok = vt(l.vt_tok); a.vt_bea = vt(l.vt_bea);
-  a.vt_prompt_cols = l.prompt_cols; a.vt_tok_cols = l.tok_cols; a.vt_bea_cols = l.bea_cols;
   a.out_tok = (__nv_bfloat16*)out_tok; a.out_bea = (__nv_bfloat16*)out_beacon;
   a.status = reinterpret_cast<int32_t*>(ws + l.status);
   a.Hq = q_heads; a.Hkv = kv_heads; a.G = G; a.c = c; a.rows_per_tile = per;
   a.scale_log2 = sm_scale * 1.4426950408889634f;
   const int smem_bytes = 3 * kOperandBytes + 1024;
   if (cudaFuncSetAttribute(k_mask_attn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return BC_ERR_CUDA;
-  k_mask_attn<<<dim3((unsigned)tiles.size(), kv_heads), kThreads, smem_bytes, s>>>(a);
+  if (!encode_tiled()) return BC_ERR_CUDA;
+  MaskMaps maps;
+  const void* dummy = ws;   // arrays that do not exist (no prompt, no beacons) get a map that is never used
+  bool ok = map_3d(&maps.q_tok, tok_q ? tok_q : dummy, q_heads, total_tokens, G, per) &&
+            map_3d(&maps.q_bea, beacon_q ? beacon_q : dummy, q_heads, total_beacons, G, per) &&
+            map_3d(&maps.k_prompt, prompt_k ? prompt_k : dummy, kv_heads, total_prompt, 1, kTile) &&
+            map_3d(&maps.k_tok, tok_k ? tok_k : dummy, kv_heads, total_tokens, 1, kTile) &&
+            map_3d(&maps.k_bea, beacon_k ? beacon_k : dummy, kv_heads, total_beacons, 1, kTile) &&
+            map_2d(&maps.vt_prompt, ws + l.vt_prompt, l.prompt_cols, (int64_t)kv_heads * kD) &&
+            map_2d(&maps.vt_tok, ws + l.vt_tok, l.tok_cols, (int64_t)kv_heads * kD) &&
+            map_2d(&maps.vt_bea, ws + l.vt_bea, l.bea_cols, (int64_t)kv_heads * kD);
+  if (!ok) return BC_ERR_CUDA;
+  k_mask_attn<<<dim3((unsigned)tiles.size(), kv_heads), kThreads, smem_bytes, s>>>(a, maps);
   return cudaGetLastError() == cudaSuccess ? BC_OK : BC_ERR_CUDA;
 }
 

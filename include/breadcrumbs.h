@@ -162,6 +162,18 @@ BC_API bc_status bc_decode_attn(bc_cache* cache, int32_t layer, const int32_t* s
                          const void* q, void* out, float sm_scale, const void* extra_k,
                          const void* extra_v, void* stream);
 
+/* One decode step of one layer in a single launch: bc_append(k, v) followed by bc_decode_attn(q)
+ * (Algorithm 1: the forward pass of a token adds its entry, then its query reads the cache, the
+ * new entry included).  Results, bookkeeping, layer-order rule and error behaviour are exactly
+ * those of the two calls made one after the other; the saving is two kernel launches per step.
+ * How: block 0 of the attention kernel runs the append bookkeeping and releases a flag the other
+ * blocks wait for (bounded; block 0 waits for nobody); the new entries are fed to the attention
+ * from the input tensors while another warp stores them to the pool for later steps.
+ * q [n, q_heads, head_dim], k, v [n, kv_heads, head_dim], out like q; n <= 512.  With
+ * BC_FLAG_ATTN_REFERENCE the call simply issues the two separate calls. */
+BC_API bc_status bc_decode_step(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n, const void* q,
+                                const void* k, const void* v, void* out, float sm_scale, void* stream);
+
 /* Limits of bc_decode_attn_static. */
 #define BC_STATIC_MAX_BATCH 128   /* sequences per call */
 #define BC_STATIC_MAX_CTAS 160    /* thread blocks it will use at most */
@@ -209,7 +221,7 @@ BC_API bc_status bc_seq_close(bc_cache* cache, const int32_t* slots, int32_t n, 
 
 /* ---- end-to-end helpers with HOST buffers (pinned memory recommended) ------------------------
  * One decode step of one layer: copies q, k, v to device staging inside `workspace`, runs
- * bc_append + bc_decode_attn, copies out back.  All asynchronous on `stream`.  n <= 512. */
+ * bc_decode_step, copies out back.  All asynchronous on `stream`.  n <= 512. */
 BC_API bc_status bc_decode_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                               const void* q_host, const void* k_host, const void* v_host,
                               void* out_host, float sm_scale, void* stream);

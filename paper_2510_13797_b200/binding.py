@@ -57,6 +57,7 @@ SYMBOLS = {
     "bc_prefill": (_I32, [_P, _I32, _P, _P, _I32, _I32, _P, _P, _P]),
     "bc_append": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
     "bc_decode_attn": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
+    "bc_decode_step": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P]),
     "bc_decode_attn_static": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
     "bc_mask_attn_query_bytes": (_I32, [_I32, _I32, _I32, _I32, _I64, _I64, _I64, C.POINTER(C.c_size_t)]),
     "bc_mask_attn_forward": (_I32, [_I32, _I32, _I32, _I32, _I32, C.POINTER(_I32), C.POINTER(_I32)] + [_P] * 10
@@ -156,6 +157,11 @@ class Cache:
     def bc_decode_attn(self, layer, slots, q, out, sm_scale, extra_k=None, extra_v=None, stream=None):
         _check(lib().bc_decode_attn(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(out), sm_scale,
                                     _ptr(extra_k), _ptr(extra_v), _stream(stream)), "bc_decode_attn")
+
+    def bc_decode_step(self, layer, slots, q, k, v, out, sm_scale, stream=None):
+        """bc_append(k, v) + bc_decode_attn(q) in one launch."""
+        _check(lib().bc_decode_step(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(k), _ptr(v), _ptr(out),
+                                    sm_scale, _stream(stream)), "bc_decode_step")
 
     def bc_decode_attn_static(self, layer, slots, q, out, sm_scale, extra_k=None, extra_v=None, stream=None):
         """bc_decode_attn with the split-K scratch taken from the array built into the library, for callers

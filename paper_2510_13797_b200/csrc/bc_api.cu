@@ -32,7 +32,7 @@ MetaLayout meta_layout(const bc_config& c) {
 }
 
 struct WorkLayout {
-  size_t append_row, append_pos, compress_row, compress_pos, tickets, part_ml, part_o, stage_q, stage_k,
+  size_t append_row, append_pos, compress_row, compress_pos, tickets, book_flag, part_ml, part_o, stage_q, stage_k,
       stage_v, stage_out, total;
 };
 WorkLayout work_layout(const bc_config& c) {
@@ -43,6 +43,7 @@ WorkLayout work_layout(const bc_config& c) {
   const size_t pieces = BC_MAX_ATTN_CTAS + BC_MAX_ATTN_BATCH;
   l.append_row = take(seq); l.append_pos = take(seq); l.compress_row = take(seq); l.compress_pos = take(seq);
   l.tickets = take(BC_MAX_ATTN_BATCH * 4);
+  l.book_flag = take(4);
   l.part_ml = take(pieces * c.q_heads * 2 * 4);
   l.part_o = take(pieces * c.q_heads * c.head_dim * 4);
   l.stage_q = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 2);
@@ -120,7 +121,7 @@ bc_status check_batch(bc_cache* c, int layer, const int32_t* slots, int n) {
 }
 
 bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const void* q, void* out, float sm_scale,
-                    const void* extra_k, const void* extra_v, cudaStream_t s) {
+                    const void* extra_k, const void* extra_v, cudaStream_t s, const BcFusedAppend* fused = nullptr) {
   BcAttnArgs a;
   a.pool_layer = layer_base(c, layer);
   a.slots = slots; a.n = n; a.q = q; a.out = out;
@@ -138,7 +139,7 @@ bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const v
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (c->prof_used < c->prof_cap) { e0 = c->ev[2 * c->prof_used]; e1 = c->ev[2 * c->prof_used + 1]; c->prof_used++; }
   int launches = 0;
-  BC_CUDA(c, bc_launch_attn(c->meta, c->geom, a, s, e0, e1, &launches));
+  BC_CUDA(c, bc_launch_attn(c->meta, c->geom, a, fused, s, e0, e1, &launches));
   c->launches += launches;
   return BC_OK;
 }
@@ -264,6 +265,7 @@ bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* wo
   cudaError_t e = bc_attn_setup(&c->sm_count);
   if (e == cudaSuccess) e = bc_launch_init(c->meta, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->work + c->wl.tickets, 0, BC_MAX_ATTN_BATCH * 4, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->work + c->wl.book_flag, 0, 4, (cudaStream_t)stream);
   if (e != cudaSuccess) { delete c; return BC_ERR_CUDA; }
   c->launches += 1;
   *out = c;
@@ -332,6 +334,35 @@ bc_status bc_decode_attn(bc_cache* c, int32_t layer, const int32_t* slots, int32
   return attn_impl(c, layer, slots, n, q, out, sm_scale, extra_k, extra_v, (cudaStream_t)stream);
 }
 
+bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, const void* k,
+                         const void* v, void* out, float sm_scale, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (n > BC_MAX_ATTN_BATCH) return BC_ERR_INVALID_ARG;
+  if (!q || !k || !v || !out || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BC_ERR_INVALID_ARG;
+  if (layer != c->append_next_layer) return BC_ERR_ORDER;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) {   // the debugging kernel has no fused form
+    st = bc_append(c, layer, slots, n, k, v, stream);
+    if (st) return st;
+    return attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s);
+  }
+  BcFusedAppend f;
+  f.new_k = k; f.new_v = v;
+  f.dst_row = work_ptr<int32_t>(c, c->wl.append_row);
+  f.dst_pos = work_ptr<int32_t>(c, c->wl.append_pos);
+  f.pool_layer = layer_base(c, layer);
+  f.flag = work_ptr<int32_t>(c, c->wl.book_flag);
+  f.do_book = layer == 0 ? 1 : 0;
+  if (layer == 0) ++c->calls;
+  f.call = c->calls;
+  f.epoch = (int32_t)(c->calls & 0x7fffffff) | 1 << 30;   // never 0, the word's initial value
+  st = attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s, &f);
+  if (st) return st;
+  c->append_next_layer = (layer + 1) % c->cfg.layers;
+  return BC_OK;
+}
+
 bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* bk, const void* bv,
                       void* stream) {
   bc_status st = check_batch(c, layer, slots, n);
@@ -383,9 +414,7 @@ bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, 
   BC_CUDA(c, cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, s));
   BC_CUDA(c, cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, s));
   BC_CUDA(c, cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s));
-  st = bc_append(c, layer, slots, n, dk, dv, stream);
-  if (st) return st;
-  st = attn_impl(c, layer, slots, n, dq, dout, sm_scale, nullptr, nullptr, s);
+  st = bc_decode_step(c, layer, slots, n, dq, dk, dv, dout, sm_scale, stream);
   if (st) return st;
   BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
   return BC_OK;
@@ -537,7 +566,7 @@ bc_status bc_decode_attn_static(bc_cache* c, int32_t layer, const int32_t* slots
   int ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
   a.ctas = ctas < BC_STATIC_MAX_CTAS ? ctas : BC_STATIC_MAX_CTAS;
   int launches = 0;
-  BC_CUDA(c, bc_launch_attn(c->meta, c->geom, a, (cudaStream_t)stream, nullptr, nullptr, &launches));
+  BC_CUDA(c, bc_launch_attn(c->meta, c->geom, a, nullptr, (cudaStream_t)stream, nullptr, nullptr, &launches));
   c->launches += launches;
   return BC_OK;
 }

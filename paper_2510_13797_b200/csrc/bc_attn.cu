@@ -28,6 +28,8 @@
 
 namespace {
 
+#include "bc_book_device.cuh"
+
 constexpr int kConsumerWarps = 8;
 constexpr int kPipeThreads = (kConsumerWarps + 2) * 32;  // consumer warps, producer warp, service warp
 constexpr int kPlanMax = BC_MAX_ATTN_BATCH;
@@ -35,6 +37,7 @@ constexpr uint32_t kSpinLimit = 1u << 21;  // polls of try_wait before giving up
 constexpr int kPidAhead = 4;               // tiles of page-id lookahead of the producer
 constexpr int kInFlight = 2;               // stages whose copies may be outstanding at once: HBM
                                            // delivers less when every SM keeps more in flight
+constexpr int kNewRowBit = 1 << 30;        // in the plan's slot word: the sequence got a new entry in this launch
 constexpr int kPidSlot = 136;              // ints per descriptor slot: 4 header + up to 132 page ids
 
 // ---------------------------------------------------------------- PTX helpers
@@ -147,10 +150,25 @@ __device__ __forceinline__ int fast_div(int n, const FastDiv& d) {
   return (int)((t + (((uint32_t)n - t) >> d.sh1)) >> d.sh2);
 }
 
+// The fused decode step (append + attention in one launch): the new token's K/V rows, where the
+// bookkeeping puts them, and the hand-shake by which block 0 tells the others that it is done.
+struct FusedArgs {
+  const uint8_t* new_k;   // [n][kv_heads][head_dim] bf16
+  const uint8_t* new_v;
+  int32_t* dst_row;       // [n] pool row of every item's new entry (-1: the item was refused)
+  int32_t* dst_pos;       // [n] its position in the window
+  uint8_t* pool_w;        // the layer's pool, writable
+  int32_t* flag;          // set to `epoch` by block 0 once the bookkeeping of this launch is done
+  int32_t epoch;
+  int32_t do_book;        // 1 on the layer-0 call of a step
+  int64_t call;           // index of the bookkeeping call (for the error latch)
+};
+
 struct PipeParams {
   BcMeta m;
   BcGeom g;
   BcAttnArgs a;
+  FusedArgs f;
   float scale_log2;
   int rows_per_tile;  // T = 16 * n_groups, a power of two
   int tile_shift;     // log2(T)
@@ -249,7 +267,13 @@ __device__ __forceinline__ void combine_pieces(const float* part_o, const float*
   }
 }
 
-template <int D, bool G_LE_8>
+// FUSED: the launch also appends the step's new entries (bc_decode_step).  Block 0 runs the append
+// bookkeeping first and publishes a flag; the others wait for it (block 0 waits for nobody).  The new
+// rows are not read back from the pool: the bulk copy of a sequence's last tile leaves the new row
+// out, the consumer warps write it into the shared-memory tile straight from the input, and the
+// service warp stores it to the pool for the steps to come.  So the step costs no second and third
+// launch and no fence.
+template <int D, bool G_LE_8, bool FUSED>
 __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams p) {
   using L = PipeSmem<D>;
   constexpr int NSTAGE = L::kStages;
@@ -293,6 +317,31 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     fence_proxy_async();
   }
 
+  if (FUSED && p.f.do_book) {
+    __shared__ int sh_book_ok;
+    if (blockIdx.x == 0) {
+      append_book_block(p.m, p.a.slots, n, p.f.call, p.f.dst_row, p.f.dst_pos);
+      __syncthreads();
+      if (tid == 0) {
+        __threadfence();
+        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p.f.flag), "r"(p.f.epoch) : "memory");
+        sh_book_ok = 1;
+      }
+    } else if (tid == 0) {
+      int ok = 0;
+      for (uint32_t polls = 0; polls < kSpinLimit; ++polls) {
+        if (ld_acquire(p.f.flag) == p.f.epoch) { ok = 1; break; }
+        __nanosleep(32);
+      }
+      sh_book_ok = ok;
+    }
+    __syncthreads();
+    if (!sh_book_ok) {  // block 0 never reported: give up before anything is in flight
+      if (tid == 0 && p.m.status[0] == 0) { p.m.status[0] = BC_ERR_TIMEOUT; p.m.status[1] = -1; }
+      return;
+    }
+  }
+
   // ---- plan: tiles per sequence, prefix sums, this block's span --------------------------------
   // Each segment (prompt, beacons, window) starts a new tile, so a tile never straddles segments;
   // a partly filled tile costs masked arithmetic but no memory traffic.
@@ -303,6 +352,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       P = p.m.prompt_len[slot]; nb = p.m.n_beacons[slot]; w = p.m.window_len[slot];
       bcol = p.m.beacon_off[slot]; wcol = p.m.window_off[slot]; sl = slot;
     }
+    if (FUSED && w > 0 && p.f.dst_row[i] >= 0) sl |= kNewRowBit;  // the window's last entry is this launch's
     s_P[i] = P; s_nb[i] = nb; s_w[i] = w; s_slot[i] = sl; s_bcol[i] = bcol; s_wcol[i] = wcol;
     const int tiles = ((P + T - 1) >> TS) + ((nb + T - 1) >> TS) + ((w + T - 1) >> TS);
     s_cum[i + 1] = tiles > 0 ? tiles : 1;  // an empty sequence still owns one (empty) tile
@@ -351,6 +401,21 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   }
   if (warp == kConsumerWarps + 1) {
     // ================================ service warp =============================================
+    if (FUSED) {
+      // store the new entries of the sequences whose last tile this block owns (for the steps to come)
+      const int chunks = p.g.head_row_bytes >> 4, per_side = Hkv * chunks;
+      for (int i = seq0; i < n && s_cum[i + 1] - 1 < g1; ++i) {
+        if (s_cum[i + 1] - 1 < g0 || !(s_slot[i] & kNewRowBit)) continue;
+        uint8_t* dst = p.f.pool_w + (int64_t)p.f.dst_row[i] * E;
+        const int key = p.f.dst_pos[i] & 7;
+        for (int idx = lane; idx < 2 * per_side; idx += 32) {
+          const int which = idx / per_side, rem = idx - which * per_side, h = rem / chunks, j = rem - h * chunks;
+          const uint8_t* src = (which ? p.f.new_v : p.f.new_k) + ((int64_t)i * Hkv + h) * p.g.head_row_bytes + (j << 4);
+          *reinterpret_cast<uint4*>(dst + (which * Hkv + h) * p.g.head_row_bytes + ((j ^ key) << 4)) =
+              *reinterpret_cast<const uint4*>(src);
+        }
+      }
+    }
     if (svc_publishes) {
       const bool ok = bounded_wait(bar_pub, 0, s_abort);  // every consumer warp has stored its share
       if (lane == 0) {
@@ -375,11 +440,13 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     const uint64_t stream_policy = l2_policy_evict_first();
     int fi = seq0;
     int f_P, f_nb, f_w, f_tp, f_tpb, f_bcol, f_wcol;
+    bool f_new = false;
     const int32_t* f_tab;
     auto load_seq = [&](int i) {
       f_P = s_P[i]; f_nb = s_nb[i]; f_w = s_w[i]; f_bcol = s_bcol[i]; f_wcol = s_wcol[i];
       f_tp = (f_P + T - 1) >> TS; f_tpb = f_tp + ((f_nb + T - 1) >> TS);
-      f_tab = p.m.page_table + (int64_t)s_slot[i] * p.m.max_pages_per_seq;
+      f_tab = p.m.page_table + (int64_t)(s_slot[i] & ~kNewRowBit) * p.m.max_pages_per_seq;
+      f_new = FUSED && (s_slot[i] & kNewRowBit);
     };
     load_seq(fi);
     auto describe = [&](int gt, int it) {
@@ -394,6 +461,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
         else { len = f_w; tt = t - f_tpb; col = f_wcol; }
         p0 = tt << TS;
         nrows = max(min(T, len - p0), 0);
+        if (FUSED && f_new && gt == s_cum[fi + 1] - 1) nrows -= 1;  // the new row comes from the input, not the pool
         if (nrows > 0) {
           pg0 = fast_div(p0, p.div_ps);
           const int pg_last = fast_div(p0 + nrows - 1, p.div_ps);
@@ -539,6 +607,21 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     // ---- stream the tiles of this piece ----------------------------------------------------------
     for (int t = ta; t < tb; ++t, ++it, ++gt) {
       const int stage = it % NSTAGE;
+      // FUSED: the sequence's last tile lacks this launch's new entry (the bulk copy left it out);
+      // the warps whose 16-row group holds it fetch their head's K and V chunks of it from the input
+      // (lanes 0-15: K, lanes 16-31: V) while the tile is still in flight.
+      bool patch = false;
+      int patch_row = 0;
+      uint4 patch_val = make_uint4(0u, 0u, 0u, 0u);
+      if (FUSED && (s_slot[i] & kNewRowBit) && t == tiles_i - 1) {
+        patch_row = (c_w - 1) - ((t - c_tpb) << TS);
+        if ((patch_row >> 4) == grp) {
+          patch = true;
+          if ((lane & 15) < (p.g.head_row_bytes >> 4))
+            patch_val = *reinterpret_cast<const uint4*>(((lane >> 4) ? p.f.new_v : p.f.new_k) +
+                                                        ((int64_t)i * Hkv + kvh) * p.g.head_row_bytes + ((lane & 15) << 4));
+        }
+      }
       const bool ok = __all_sync(0xffffffffu, bounded_wait(bar_full + stage * 8, (it / NSTAGE) & 1, s_abort));
       if (!ok && lane == 0 && p.m.status[0] == 0) { p.m.status[0] = BC_ERR_TIMEOUT; p.m.status[1] = -1; }
       // rows of this tile that hold entries; my warp looks at rows grp*16 .. grp*16+15 of it
@@ -550,6 +633,14 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       bool wrote_smem = false;
       if (ok && cnt > 0) {
         const uint32_t rows_base = ring + stage * L::kStageBytes + warp_rows_off;
+        if (FUSED && patch) {
+          if ((lane & 15) < (p.g.head_row_bytes >> 4))
+            *reinterpret_cast<uint4*>(smem + stage * L::kStageBytes + warp_rows_off + (patch_row & 15) * E +
+                                      ((lane >> 4) * Hkv + kvh) * p.g.head_row_bytes +
+                                      (((lane & 15) ^ ((c_w - 1) & 7)) << 4)) = patch_val;
+          wrote_smem = true;
+          __syncwarp();
+        }
         if (cnt < 16) {
           // rows nobody copied may hold anything: zero their V so that 0 * garbage cannot be NaN
           uint8_t* rows_ptr = smem + stage * L::kStageBytes + warp_rows_off;
@@ -812,12 +903,19 @@ FastDiv make_fast_div(uint32_t d) {
   return f;
 }
 
-template <int D, bool G8>
+template <int D, bool G8, bool FUSED>
 cudaError_t launch_pipe(const PipeParams& p, cudaStream_t s) {
-  k_attn_pipe<D, G8><<<p.a.ctas, kPipeThreads, PipeSmem<D>::kTotal, s>>>(p);
+  k_attn_pipe<D, G8, FUSED><<<p.a.ctas, kPipeThreads, PipeSmem<D>::kTotal, s>>>(p);
   return cudaGetLastError();
 }
 
+}  // namespace
+
+namespace {
+template <int D, bool G8, bool FUSED>
+cudaError_t opt_in_smem() {
+  return cudaFuncSetAttribute(k_attn_pipe<D, G8, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<D>::kTotal);
+}
 }  // namespace
 
 cudaError_t bc_attn_setup(int* sm_count) {
@@ -826,19 +924,24 @@ cudaError_t bc_attn_setup(int* sm_count) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_attn_pipe<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<128>::kTotal);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_attn_pipe<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<128>::kTotal);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(k_attn_pipe<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<64>::kTotal);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_attn_pipe<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<64>::kTotal);
+  const cudaError_t r[8] = {opt_in_smem<128, true, false>(), opt_in_smem<128, false, false>(), opt_in_smem<64, true, false>(),
+                            opt_in_smem<64, false, false>(), opt_in_smem<128, true, true>(), opt_in_smem<128, false, true>(),
+                            opt_in_smem<64, true, true>(), opt_in_smem<64, false, true>()};
+  for (cudaError_t x : r)
+    if (x != cudaSuccess) return x;
+  return cudaSuccess;
 }
 
-cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, cudaStream_t s, cudaEvent_t ev_start,
-                           cudaEvent_t ev_stop, int* launches) {
+cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, const BcFusedAppend* fused, cudaStream_t s,
+                           cudaEvent_t ev_start, cudaEvent_t ev_stop, int* launches) {
   PipeParams p;
   p.m = m; p.g = g; p.a = a;
+  p.f = FusedArgs{};
+  if (fused) {
+    p.f.new_k = static_cast<const uint8_t*>(fused->new_k); p.f.new_v = static_cast<const uint8_t*>(fused->new_v);
+    p.f.dst_row = fused->dst_row; p.f.dst_pos = fused->dst_pos; p.f.pool_w = fused->pool_layer;
+    p.f.flag = fused->flag; p.f.epoch = fused->epoch; p.f.do_book = fused->do_book; p.f.call = fused->call;
+  }
   p.scale_log2 = a.sm_scale * 1.4426950408889634f;
   p.n_groups = kConsumerWarps / g.kv_heads;
   p.rows_per_tile = 16 * p.n_groups;
@@ -849,8 +952,13 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   cudaError_t e;
   if (ev_start) { e = cudaEventRecord(ev_start, s); if (e != cudaSuccess) return e; }
   const bool g8 = p.G <= 8;
-  if (g.head_dim == 128) e = g8 ? launch_pipe<128, true>(p, s) : launch_pipe<128, false>(p, s);
-  else e = g8 ? launch_pipe<64, true>(p, s) : launch_pipe<64, false>(p, s);
+  if (fused) {
+    if (g.head_dim == 128) e = g8 ? launch_pipe<128, true, true>(p, s) : launch_pipe<128, false, true>(p, s);
+    else e = g8 ? launch_pipe<64, true, true>(p, s) : launch_pipe<64, false, true>(p, s);
+  } else {
+    if (g.head_dim == 128) e = g8 ? launch_pipe<128, true, false>(p, s) : launch_pipe<128, false, false>(p, s);
+    else e = g8 ? launch_pipe<64, true, false>(p, s) : launch_pipe<64, false, false>(p, s);
+  }
   if (e != cudaSuccess) return e;
   if (ev_stop) { e = cudaEventRecord(ev_stop, s); if (e != cudaSuccess) return e; }
   *launches = 1;

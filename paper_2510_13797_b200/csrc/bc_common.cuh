@@ -83,9 +83,21 @@ struct BcAttnArgs {
 };
 // Configures the kernels once per process/device (shared-memory opt-in).  Returns the SM count.
 cudaError_t bc_attn_setup(int* sm_count);
-// Launches the pipelined decode-attention kernel (the split combine is part of it); *launches gets
-// the number of kernels launched.
-cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, cudaStream_t s,
-                           cudaEvent_t ev_start, cudaEvent_t ev_stop, int* launches);
+// The append half of a fused decode step (bc_decode_step): the new entries and where they go.
+struct BcFusedAppend {
+  const void* new_k;     // [n][kv_heads][head_dim] bf16
+  const void* new_v;
+  int32_t* dst_row;      // [n] workspace: pool row of each item's new entry, -1 if refused (written on layer 0)
+  int32_t* dst_pos;      // [n] workspace: its position in the window
+  uint8_t* pool_layer;   // the layer's pool (writable)
+  int32_t* flag;         // workspace word: "the bookkeeping of launch `epoch` is done"
+  int32_t epoch;
+  int32_t do_book;       // 1: this launch runs the bookkeeping (the layer-0 call of the step)
+  int64_t call;          // bookkeeping call index (error latch)
+};
+// Launches the pipelined decode-attention kernel (the split combine is part of it); with `fused`
+// the same launch appends the step's new entries first.  *launches gets the number of kernels.
+cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, const BcFusedAppend* fused,
+                           cudaStream_t s, cudaEvent_t ev_start, cudaEvent_t ev_stop, int* launches);
 // Slow device reference (one warp per query head).
 cudaError_t bc_launch_attn_reference(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, cudaStream_t s);

@@ -21,8 +21,9 @@ from .workloads import InputStream
 
 
 class DecodeDriver:
-    def __init__(self, w, device, seed_offset=0):
+    def __init__(self, w, device, seed_offset=0, fused=True):
         self.w, self.dev = w, torch.device(device)
+        self.fused = fused                             # regular steps through bc_decode_step (one launch)
         c, ps, Bn = w.cs[0], w.page_size, w.batch
         P, T = w.prompt_lens[0], w.steps
         assert all(x == c for x in w.cs) and all(x == P for x in w.prompt_lens), "uniform batches only"
@@ -71,8 +72,11 @@ class DecodeDriver:
         """One decode step of the whole batch through the device-pointer calls.  Returns True if the
         window filled and the beacon step (beacon-query attention into out_b, then compress) ran."""
         c, j = self.cache, self.t % self.ring
-        c.bc_append(0, self.slots, self.k[j], self.v[j])
-        c.bc_decode_attn(0, self.slots, self.q[j], self.out, self.w.sm_scale)
+        if self.fused:
+            c.bc_decode_step(0, self.slots, self.q[j], self.k[j], self.v[j], self.out, self.w.sm_scale)
+        else:
+            c.bc_append(0, self.slots, self.k[j], self.v[j])
+            c.bc_decode_attn(0, self.slots, self.q[j], self.out, self.w.sm_scale)
         self.t += 1
         if self.c > 1 and self.t % self.c == 0:
             b = (self.t // self.c) % 4

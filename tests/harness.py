@@ -78,6 +78,21 @@ class Pair:
                 self.seqs[slot].append(layer, kk[i], vv[i])
         return self._append_ok
 
+    def step(self, layer, slots, q, k, v, sm_scale):
+        """The fused call: append k, v and attend with q.  Returns (append results, out, reference out)."""
+        out = self.gpu.new_out(len(slots))
+        self.gpu.bc_decode_step(layer, self._i32(slots), q, k, v, out, sm_scale)
+        if layer == 0:
+            self._append_ok = self.model.append(list(slots))
+        kk, vv, qq = f64(k), f64(v), f64(q)
+        ref = np.zeros((len(slots), self.Hq, self.D))
+        for i, slot in enumerate(slots):
+            if self._append_ok[i] == OK:
+                self.seqs[slot].append(layer, kk[i], vv[i])
+            seq = self.seqs.get(slot) or SeqCache(self.L, 1)
+            ref[i] = seq.attend(layer, qq[i], sm_scale)
+        return self._append_ok, out, ref
+
     def attend(self, layer, slots, q, sm_scale, extra_k=None, extra_v=None):
         out = self.gpu.new_out(len(slots))
         self.gpu.bc_decode_attn(layer, self._i32(slots), q, out, sm_scale, extra_k, extra_v)

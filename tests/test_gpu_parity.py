@@ -308,3 +308,72 @@ def test_host_buffer_entry_points():
         pair.check_state()
     for s in slots:
         pair.check_content(0, s)
+
+
+def run_decode_fused(pair: Pair, slots, plens, cs, steps, seed, sm_scale, content_every=0):
+    """Like run_decode, but every regular step goes through the fused bc_decode_step call."""
+    g = _gen(seed)
+    L, Hkv, Hq, D = pair.L, pair.Hkv, pair.Hq, pair.D
+    n = len(slots)
+    assert pair.open(slots, plens, cs) == ["OK"] * n
+    for l in range(L):
+        pair.prefill(l, slots, plens, randn_bf16(g, (sum(plens), Hkv, D), DEV), randn_bf16(g, (sum(plens), Hkv, D), DEV))
+    for step in range(1, steps + 1):
+        for l in range(L):
+            res, out, ref = pair.step(l, slots, randn_bf16(g, (n, Hq, D), DEV), randn_bf16(g, (n, Hkv, D), DEV),
+                                      randn_bf16(g, (n, Hkv, D), DEV), sm_scale)
+            assert res == ["OK"] * n
+            assert_close(out, ref, f"fused step {step} layer {l}")
+        full = [i for i, s in enumerate(slots) if cs[i] > 1 and step % cs[i] == 0]
+        if full:
+            fs = [slots[i] for i in full]
+            for l in range(L):
+                qb, bk, bv = randn_bf16(g, (len(fs), Hq, D), DEV), randn_bf16(g, (len(fs), Hkv, D), DEV), randn_bf16(g, (len(fs), Hkv, D), DEV)
+                out, ref = pair.attend(l, fs, qb, sm_scale, bk, bv)
+                assert_close(out, ref, f"beacon query after fused step {step} layer {l}")
+                assert pair.compress(l, fs, bk, bv) == ["OK"] * len(fs)
+        pair.check_state()
+        if content_every and (step % content_every == 0 or step == steps):
+            for s in slots:
+                for l in range(L):
+                    pair.check_content(l, s)
+
+
+@pytest.mark.parametrize("L,Hkv,G,D,ps,c,plens,steps", [
+    (1, 1, 2, 64, 16, 16, [64], 40),
+    (1, 8, 4, 128, 2, 2, [40, 17, 300], 20),       # the sweep shape at c = 2: a window page every other step
+    (1, 8, 4, 128, 16, 16, [700, 333, 1030], 36),  # sequences split over several blocks
+    (1, 2, 6, 128, 16, 4, [70, 9, 0], 30),         # empty prompt: the first entry of the cache comes from the fused step
+    (1, 4, 3, 128, 3, 7, [20, 21, 22, 23], 30),
+    (1, 2, 12, 128, 8, 8, [50], 20),               # G > 8
+    (1, 1, 16, 64, 16, 1, [30, 8], 40),            # ratio 1: the window grows by pages
+    (3, 2, 2, 64, 4, 4, [9, 4], 21),               # three layers: bookkeeping on layer 0, rows on every layer
+])
+def test_fused_decode_step_every_step(L, Hkv, G, D, ps, c, plens, steps):
+    n = len(plens)
+    pair = Pair(L, Hkv, Hkv * G, D, ps, max_seqs=n + 1, num_pages=600, max_pages_per_seq=200)
+    run_decode_fused(pair, list(range(n)), plens, [c] * n, steps, seed=23, sm_scale=1.0 / math.sqrt(D), content_every=5)
+
+
+def test_fused_decode_step_refusals_and_block_counts():
+    """A refused append inside the fused call leaves that sequence as it was (and attends to it as it
+    was); any number of thread blocks gives the same answer."""
+    Hkv, G, D, ps = 2, 2, 64, 2
+    pair = Pair(1, Hkv, Hkv * G, D, ps, max_seqs=3, num_pages=8, max_pages_per_seq=6)
+    g = _gen(4)
+    assert pair.open([0, 1, 2], [3, 2, 4], [2, 2, 2]) == ["OK"] * 3     # 2 + 1 + 2 pages, 3 left
+    pair.prefill(0, [0, 1, 2], [3, 2, 4], randn_bf16(g, (9, Hkv, D), DEV), randn_bf16(g, (9, Hkv, D), DEV))
+    mk = lambda n: (randn_bf16(g, (n, Hkv * G, D), DEV), randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV))
+    for ctas in (1, 3, 148):
+        pair.gpu.bc_set_attn_ctas(ctas)
+        res, out, ref = pair.step(0, [0, 1, 2], *mk(3), 0.125)
+        assert_close(out, ref, f"fused, {ctas} blocks")
+        pair.check_state()
+        pair.gpu.bc_clear_error(); pair.model.first_error = None
+    # by now some windows are full and the pool is nearly empty: refusals must match the model
+    res, out, ref = pair.step(0, [0, 1, 2, ][:3], *mk(3), 0.125)
+    assert any(r != "OK" for r in res)
+    assert_close(out, ref, "fused with refused items")
+    pair.check_state()
+    for s in (0, 1, 2):
+        pair.check_content(0, s)

@@ -165,7 +165,10 @@ BC_API bc_status bc_decode_attn(bc_cache* cache, int32_t layer, const int32_t* s
 /* One decode step of one layer in a single launch: bc_append(k, v) followed by bc_decode_attn(q)
  * (Algorithm 1: the forward pass of a token adds its entry, then its query reads the cache, the
  * new entry included).  Results, bookkeeping, layer-order rule and error behaviour are exactly
- * those of the two calls made one after the other; the saving is two kernel launches per step.
+ * those of the two calls made one after the other; the saving is two kernel launches per step
+ * (measured on the ratio sweep: within 2 % of the separate calls when the step is replayed from a
+ * CUDA graph, where launches are cheap; the other blocks wait about as long for block 0 as the two
+ * small kernels take).
  * How: block 0 of the attention kernel runs the append bookkeeping and releases a flag the other
  * blocks wait for (bounded; block 0 waits for nobody); the new entries are fed to the attention
  * from the input tensors while another warp stores them to the pool for later steps.
@@ -221,7 +224,7 @@ BC_API bc_status bc_seq_close(bc_cache* cache, const int32_t* slots, int32_t n, 
 
 /* ---- end-to-end helpers with HOST buffers (pinned memory recommended) ------------------------
  * One decode step of one layer: copies q, k, v to device staging inside `workspace`, runs
- * bc_decode_step, copies out back.  All asynchronous on `stream`.  n <= 512. */
+ * bc_append + bc_decode_attn, copies out back.  All asynchronous on `stream`.  n <= 512. */
 BC_API bc_status bc_decode_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                               const void* q_host, const void* k_host, const void* v_host,
                               void* out_host, float sm_scale, void* stream);

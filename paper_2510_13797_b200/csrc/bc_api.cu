@@ -414,7 +414,9 @@ bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, 
   BC_CUDA(c, cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, s));
   BC_CUDA(c, cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, s));
   BC_CUDA(c, cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s));
-  st = bc_decode_step(c, layer, slots, n, dq, dk, dv, dout, sm_scale, stream);
+  st = bc_append(c, layer, slots, n, dk, dv, stream);
+  if (st) return st;
+  st = attn_impl(c, layer, slots, n, dq, dout, sm_scale, nullptr, nullptr, s);
   if (st) return st;
   BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
   return BC_OK;

@@ -375,8 +375,12 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   }
   __syncthreads();
   const int total_tiles = s_cum[n];
-  const int per = total_tiles / (int)gridDim.x, rem = total_tiles % (int)gridDim.x;
-  const int cta = blockIdx.x;
+  // The block that ran the bookkeeping starts late; it takes no tiles, or it would finish last.
+  const int idle = (FUSED && p.f.do_book && gridDim.x > 1) ? 1 : 0;
+  const int n_ctas = (int)gridDim.x - idle;
+  if ((int)blockIdx.x < idle) return;
+  const int per = total_tiles / n_ctas, rem = total_tiles % n_ctas;
+  const int cta = (int)blockIdx.x - idle;
   const int g0 = cta * per + min(cta, rem);
   const int g1 = g0 + per + (cta < rem ? 1 : 0);
   if (g0 >= g1) return;

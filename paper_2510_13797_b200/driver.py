@@ -21,9 +21,9 @@ from .workloads import InputStream
 
 
 class DecodeDriver:
-    def __init__(self, w, device, seed_offset=0, fused=True):
+    def __init__(self, w, device, seed_offset=0, fused=False):
         self.w, self.dev = w, torch.device(device)
-        self.fused = fused                             # regular steps through bc_decode_step (one launch)
+        self.fused = fused                             # True: regular steps through bc_decode_step (one launch)
         c, ps, Bn = w.cs[0], w.page_size, w.batch
         P, T = w.prompt_lens[0], w.steps
         assert all(x == c for x in w.cs) and all(x == P for x in w.prompt_lens), "uniform batches only"

@@ -90,6 +90,17 @@ def test_sweep_mid_generation(c):
     drv.check_error()
 
 
+def test_sweep_mid_generation_fused_step():
+    """The same window at c = 16 with the regular steps issued as bc_decode_step (one launch)."""
+    w = make_workload("sweep", c=16)
+    drv = DecodeDriver(w, DEV, fused=True)
+    drv.reset_to((w.steps // 2 // 16) * 16 - 2)
+    fired = sum(check_step(drv, [3, 31, 60], "sweep c=16 fused") for _ in range(6))
+    assert fired >= 1
+    check_lengths_and_conservation(drv)
+    drv.check_error()
+
+
 def test_sweep_uncompressed_mid_generation():
     w = make_workload("sweep", c=1)
     drv = DecodeDriver(w, DEV)

@@ -750,6 +750,42 @@ def report_distill(args):
                       **out}))
 
 
+def report_model(args):
+    """End-to-end generation with a random-weight decoder of the 1.5B shape around the cache library
+    (28 layers, hidden 1536, 12/2 heads, D 128, MLP 8960, vocabulary 151,936; batch 64, prompt 512):
+    time to generate N tokens per sequence at ratio c relative to the uncompressed cache -- the
+    protocol of the paper's latency table.  The non-attention layers are PyTorch operators."""
+    import torch
+    from paper_2510_13797_b200.model_harness import ToyDecoder
+    torch.cuda.set_device(0)
+    Bn, N, reps = 64, 512 if args.steps >= 512 else 128, 3
+    rows, base, weights = [], None, None
+    for c in (1,) + RATIOS:
+        m = ToyDecoder(Bn, c, gen_len=reps * N + 128, device="cuda", weights=weights)
+        weights = m.weights                                 # one set of weights, at one address, for every ratio
+        m.capture()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(reps):                               # best of three: clocks settle during the first
+            e0, e1 = _event_pair(torch)
+            e0.record()
+            m.generate(N)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        st = m.check()
+        ms = min(times)
+        base = ms if c == 1 else base
+        rows.append({"c": c, "ms": ms, "ms_per_token": ms / N, "tokens_per_s": Bn * N / (ms * 1e-3),
+                     "latency_vs_uncompressed": ms / base, "ms_all": times, "cache_entries_end": st["prompt_len"] + st["n_beacons"] + st["window_len"]})
+        del m
+        torch.cuda.empty_cache()
+    print(json.dumps({"workload": f"model: random-weight decoder of the 1.5B shape, batch {Bn}, prompt 512, {N} generated tokens "
+                                  "per sequence, one CUDA graph per token step and per beacon step",
+                      "paper_latency_table_qwen_sr": {"2": 1.990, "4": 1.546, "8": 1.593, "16": 1.646, "32": 1.468},
+                      "rows": rows}))
+
+
 def batch_scaling(dev, peak):
     """The attention kernel alone at larger batches (same shape, mid-generation cache): the time per
     launch that does not stream (start-up, merging) is spread over more bytes."""
@@ -782,7 +818,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
-    ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth", "maskform", "distill"],
+    ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth", "maskform", "distill", "model"],
                     help="sweep (default): the benchmark line; cfg2 / ragged / depth: a report line for that "
                          "benchmark configuration (1 GPU)")
     ap.add_argument("--no-batch-scaling", action="store_true")
@@ -795,7 +831,7 @@ def main():
     if args.profile_case:
         return run_profile_case(args)
     if args.workload != "sweep":
-        return {"cfg2": report_cfg2, "ragged": report_ragged, "depth": report_depth, "maskform": report_maskform, "distill": report_distill}[args.workload](args)
+        return {"cfg2": report_cfg2, "ragged": report_ragged, "depth": report_depth, "maskform": report_maskform, "distill": report_distill, "model": report_model}[args.workload](args)
 
     import torch
     import torch.distributed as dist

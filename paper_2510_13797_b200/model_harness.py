@@ -1,0 +1,136 @@
+"""A decoder of the 1.5B shape with random weights around the cache library, for end-to-end timing.
+
+What is measured with it: the time to generate N tokens per sequence with the uncompressed cache
+(ratio 1) and with Breadcrumbs compression at ratio c -- the protocol behind the paper's only
+timing figure (its latency table: generation latency relative to the uncompressed teacher).
+
+Only the cache side (bc_append, bc_decode_attn, bc_compress) is this repository's product.  The
+rest of the forward pass -- embeddings, RMSNorm, the QKV / output / MLP projections, rotary
+embedding, the LM head and greedy sampling -- are plain PyTorch operators standing in for a model
+(random weights: the token stream is meaningless, the shapes and the data flow are real).  Every
+sampled token is fed back, and when a window fills, the beacon token's forward pass runs through
+the same layers: its query attends with its own K/V as the extra entry, then the window is evicted
+(Algorithm 1).  One decode step (and one beacon step) is captured in a CUDA graph and replayed.
+"""
+from __future__ import annotations
+
+import math
+
+import torch
+
+from . import binding as B
+
+
+class ToyDecoder:
+    def __init__(self, batch, c, gen_len, prompt_len=512, layers=28, hidden=1536, q_heads=12, kv_heads=2, head_dim=128,
+                 mlp=8960, vocab=151936, device="cuda", seed=0, weights=None):
+        self.B, self.c, self.L, self.H = batch, c, layers, hidden
+        self.Hq, self.Hkv, self.D, self.V = q_heads, kv_heads, head_dim, vocab
+        self.dev = torch.device(device)
+        g = torch.Generator(device=self.dev); g.manual_seed(seed)
+        rnd = lambda *s, scale=1.0: (torch.randn(s, generator=g, device=self.dev) * scale).to(torch.bfloat16)
+        if weights is None:
+            sc = 1.0 / math.sqrt(hidden)
+            weights = dict(
+                emb=rnd(vocab + 1, hidden),                    # last row: the beacon token
+                wqkv=[rnd(hidden, (q_heads + 2 * kv_heads) * head_dim, scale=sc) for _ in range(layers)],
+                wo=[rnd(q_heads * head_dim, hidden, scale=sc) for _ in range(layers)],
+                wgu=[rnd(hidden, 2 * mlp, scale=sc) for _ in range(layers)],
+                wdown=[rnd(mlp, hidden, scale=1.0 / math.sqrt(mlp)) for _ in range(layers)],
+                head=rnd(hidden, vocab, scale=sc))
+        self.weights = weights                                 # may be handed to another instance
+        self.emb, self.wqkv, self.wo = weights["emb"], weights["wqkv"], weights["wo"]
+        self.wgu, self.wdown, self.head = weights["wgu"], weights["wdown"], weights["head"]
+        ps = 16
+        cd = lambda a, b: -(-a // b)
+        pps = cd(prompt_len, ps) + (cd(c, ps) + cd(cd(gen_len, c), ps) if c > 1 else cd(gen_len, ps)) + 2
+        self.cache = B.Cache(layers, kv_heads, q_heads, head_dim, c, ps, max_seqs=batch, num_pages=batch * pps,
+                             max_pages_per_seq=pps, device=self.dev)
+        self.slots = torch.arange(batch, dtype=torch.int32, device=self.dev)
+        self.cache.bc_seq_open(self.slots, torch.full((batch,), prompt_len, dtype=torch.int32, device=self.dev))
+        cu = torch.arange(0, (batch + 1) * prompt_len, prompt_len, dtype=torch.int32, device=self.dev)
+        for l in range(layers):                               # the prompt's K/V: random stand-ins for a prefill pass
+            self.cache.bc_prefill(l, self.slots, cu, batch * prompt_len, rnd(batch * prompt_len, kv_heads, head_dim),
+                                  rnd(batch * prompt_len, kv_heads, head_dim))
+        self.tok = torch.zeros(batch, dtype=torch.int64, device=self.dev)      # last sampled token
+        self.pos = torch.full((1,), prompt_len, dtype=torch.int64, device=self.dev)
+        self.attn_out = self.cache.new_out(batch)
+        self.inv_freq = 1.0 / (10000.0 ** (torch.arange(0, head_dim, 2, device=self.dev, dtype=torch.float32) / head_dim))
+        self.scale = 1.0 / math.sqrt(head_dim)
+        self.graph_tok = self.graph_bea = None
+
+    # -- stand-ins for the rest of the model -------------------------------------------------------
+    @staticmethod
+    def _norm(x):
+        return (x.float() * torch.rsqrt(x.float().pow(2).mean(-1, keepdim=True) + 1e-6)).to(torch.bfloat16)
+
+    def _rope(self, x):
+        ang = self.pos.float() * self.inv_freq
+        cos, sin = ang.cos(), ang.sin()
+        x1, x2 = x.float()[..., 0::2], x.float()[..., 1::2]
+        return torch.stack((x1 * cos - x2 * sin, x1 * sin + x2 * cos), dim=-1).flatten(-2).to(torch.bfloat16)
+
+    def _forward(self, ids, beacon):
+        h = self.emb[ids]
+        Hq, Hkv, D = self.Hq, self.Hkv, self.D
+        for l in range(self.L):
+            qkv = self._norm(h) @ self.wqkv[l]
+            q = self._rope(qkv[:, :Hq * D].view(-1, Hq, D)).contiguous()
+            k = self._rope(qkv[:, Hq * D:(Hq + Hkv) * D].view(-1, Hkv, D)).contiguous()
+            v = qkv[:, (Hq + Hkv) * D:].view(-1, Hkv, D).contiguous()
+            if beacon:      # the beacon's query sees the cache plus its own entry; then the window goes
+                self.cache.bc_decode_attn(l, self.slots, q, self.attn_out, self.scale, k, v)
+                self.cache.bc_compress(l, self.slots, k, v)
+            else:
+                self.cache.bc_append(l, self.slots, k, v)
+                self.cache.bc_decode_attn(l, self.slots, q, self.attn_out, self.scale)
+            h = h + self.attn_out.view(-1, Hq * D) @ self.wo[l]
+            gu = self._norm(h) @ self.wgu[l]
+            gate, up = gu.chunk(2, dim=-1)
+            h = h + (torch.nn.functional.silu(gate) * up) @ self.wdown[l]
+        return h
+
+    def _token_step(self):
+        h = self._forward(self.tok, beacon=False)
+        self.tok.copy_(torch.argmax(self._norm(h) @ self.head, dim=-1))
+        self.pos.add_(1)
+
+    def _beacon_step(self):
+        self._forward(torch.full_like(self.tok, self.V), beacon=True)   # its logits are not needed
+        self.pos.add_(1)
+
+    # -- generation ---------------------------------------------------------------------------------
+    def capture(self):
+        """Warm up and capture one token step (and one beacon step) as CUDA graphs.  The warm-up
+        advances the generation by a whole number of windows, so the state stays consistent."""
+        warm = self.c if self.c > 1 else 1
+        for i in range(1, warm + 1):
+            self._token_step()
+            if self.c > 1 and i % self.c == 0:
+                self._beacon_step()
+        torch.cuda.synchronize()
+        s = torch.cuda.Stream(); s.wait_stream(torch.cuda.current_stream())
+        self.graph_tok = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph_tok, stream=s, capture_error_mode="thread_local"):
+            self._token_step()
+        if self.c > 1:
+            self.graph_bea = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(self.graph_bea, stream=s, capture_error_mode="thread_local"):
+                self._beacon_step()
+        torch.cuda.current_stream().wait_stream(s)
+        self.generate(warm)          # first replays upload the graphs: keep that out of any timing
+        torch.cuda.synchronize()
+        return 2 * warm
+
+    def generate(self, n_tokens):
+        """Replays n_tokens token steps (n_tokens a multiple of c), with a beacon step after every c."""
+        for i in range(1, n_tokens + 1):
+            self.graph_tok.replay()
+            if self.c > 1 and i % self.c == 0:
+                self.graph_bea.replay()
+
+    def check(self):
+        code, slot, call = self.cache.bc_poll_error()
+        if code != 0:
+            raise RuntimeError(f"device-side error {B.STATUS_NAMES.get(code, code)} slot {slot} call {call}")
+        return self.cache.bc_get_state(0)

@@ -31,7 +31,8 @@ namespace {
 
 constexpr int kTile = 128;        // query rows and keys per tile
 constexpr int kD = 128;           // head_dim
-constexpr int kThreads = 128;
+constexpr int kRowThreads = 128;   // one per query row
+constexpr int kThreads = kRowThreads + 32;   // plus the control warp
 constexpr int kOperandBytes = kTile * kD * 2;  // 32 KB: one bf16 operand tile
 constexpr uint32_t kWaitLimit = 1u << 20;  // polls of a bounded wait (about 0.1 s) before a block gives up
 
@@ -150,7 +151,27 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+// tcgen05.mma with the A operand in tensor memory (the softmax weights) and B in shared memory.
+__device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t b, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(b), "r"(kIdesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+      "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cta(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait that also gives up as soon as another thread of the block has reported a failure.
+__device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity, volatile int* fail) {
   for (uint32_t polls = 0; polls < kWaitLimit; ++polls) {
     uint32_t ok;
     asm volatile(
@@ -159,41 +180,47 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
         : "r"(bar), "r"(parity)
         : "memory");
     if (ok) return true;
+    if ((polls & 63) == 63 && *fail) return false;
     if (polls > 4096) __nanosleep(128);
   }
   return false;
 }
 
-// One key segment of a sequence as the main loop sees it.
-struct KeySeg {
-  const CUtensorMap* k;     // tensor map of the K array of this kind
-  const CUtensorMap* vt;    // tensor map of the transposed V array
-  int row0, col0;           // first row of the sequence in K, first column in the transposed V
-  int lo, hi;               // keys [lo, hi) of the segment are candidates (lo a multiple of 128)
-  int len;                  // rows that exist
-  int kind;                 // 0 prompt, 1 beacon, 2 token
-};
-
+// Roles: warps 0..3 own the 128 query rows (one row per thread: mask, softmax, rescaling, output);
+// warp 4 is the control warp, whose first lane issues every tensor copy and every product.
+//
+// Per key tile n (K_n, V_n):   S = Q K_n^T   ->  [rows] P_n = weights(S), bf16, written over S in
+// tensor memory   ->   O += P_n V_n (A operand from tensor memory).  The control thread keeps the copy
+// engine one tile ahead: K_{n+1} is requested as soon as S_n exists (the K buffer is free), V_{n+1} as
+// soon as O += P_n V_n has completed (the V buffer is free), so their latency hides behind the softmax
+// and the products; the products of the block's neighbour on the SM fill the tensor pipe meanwhile.
+// Q K_{n+1}^T overwrites P_n, so it is issued only after P_n V_n has completed.
+//
+// Barriers (all single-phase mbarriers, parity = completion count & 1):
+//   bar_k: Q and K_0, then K_1, K_2 ...  have landed     bar_v: V_n has landed
+//   bar_s: completion n = S_n is ready (and every earlier product has finished); completion N = O is final
+//   bar_p: the 128 row threads have stored P_n           bar_o: P_n V_n has completed
 __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, const __grid_constant__ MaskMaps maps) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  // P overwrites the K tile: K is dead once S has been computed.  Three operand tiles (96 KB) let two
-  // blocks share an SM, so that one block's softmax overlaps the other's loads and products.
-  const uint32_t sQ = smem_addr(smem), sK = sQ + kOperandBytes, sV = sK + kOperandBytes, sP = sK;
-  __shared__ __align__(8) uint64_t s_bar;
-  __shared__ __align__(8) uint64_t s_load_bar;
+  const uint32_t sQ = smem_addr(smem), sK = sQ + kOperandBytes, sV = sK + kOperandBytes;
+  __shared__ __align__(8) uint64_t s_bars[5];
   __shared__ uint32_t s_tmem;
-  __shared__ int s_fail;
-  const uint32_t bar = smem_addr(&s_bar), load_bar = smem_addr(&s_load_bar);
-  const int tid = threadIdx.x, warp = tid >> 5;
+  __shared__ int s_fail_word;
+  volatile int* s_fail = &s_fail_word;
+  const uint32_t bar_k = smem_addr(&s_bars[0]), bar_v = bar_k + 8, bar_s = bar_k + 16, bar_p = bar_k + 24, bar_o = bar_k + 32;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const TileDesc td = a.tiles[blockIdx.x];
   const int kvh = blockIdx.y, G = a.G, Hq = a.Hq, c = a.c;
 
   if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(load_bar) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_k) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_v) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_p), "r"(kRowThreads) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_o) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    s_fail = 0;
+    *s_fail = 0;
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&s_tmem)), "r"(256) : "memory");
@@ -211,210 +238,230 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  uint32_t load_phase = 0;
-  if (tid == 0) {
-    // rows beyond the tile's tokens belong to the next sequence or are zero-filled: they are never
-    // visible (their outputs are not written and they contribute to no other row)
-    mbar_expect_tx(load_bar, (uint32_t)(box_rows * kD * 2));
-    const CUtensorMap* qm = td.kind == 0 ? &maps.q_tok : &maps.q_bea;
-    const int qrow = (td.kind == 0 ? td.tok_row : td.bea_row) + td.first;
-    tma_3d(sQ, qm, 0, kvh * G, qrow, load_bar);
-    tma_3d(sQ + kTile * 128, qm, 64, kvh * G, qrow, load_bar);
-  }
-  bool failed = !mbar_wait_bounded(load_bar, load_phase);
-  failed = __any_sync(0xffffffffu, failed);
-  load_phase ^= 1;
   const uint32_t tmem = s_tmem;
-  const uint32_t tS = tmem, tO = tmem + kTile;                 // columns [0,128) and [128,256)
-  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;      // this warp's 32 lanes of tensor memory
+  const uint32_t tS = tmem, tO = tmem + kTile;   // columns [0,128): S, then P in its first 64; [128,256): O
+  const uint32_t tP = tS;
 
-  // ---- what this thread's row may see ------------------------------------------------------------
-  const int my_local = tid / G;                 // token / beacon inside the tile
-  const bool row_valid = tid < valid_rows;
-  const int my_idx = td.first + my_local;       // token index i, or beacon index (0-based; beacon number my_idx + 1)
-  int vis_beacons, tok_lo, tok_hi;              // visible: beacons [0, vis_beacons), tokens [tok_lo, tok_hi)
-  if (td.kind == 0) { vis_beacons = c > 1 ? my_idx / c : 0; tok_lo = c > 1 ? (my_idx / c) * c : 0; tok_hi = my_idx + 1; }
-  else { vis_beacons = my_idx + 1; tok_lo = my_idx * c; tok_hi = (my_idx + 1) * c; }
-
-  // ---- key segments and the tiles of each that some row of this block can see ----------------------
+  // ---- key tiles some row of this block can see: prompt, beacons, tokens ---------------------------
   const int last = td.first + td.count - 1;
-  KeySeg seg[3];
-  seg[0] = {&maps.k_prompt, &maps.vt_prompt, td.prompt_row, td.prompt_pad, 0, td.P, td.P, 0};
-  const int bmax = td.kind == 0 ? (c > 1 ? last / c : 0) : last + 1;
-  seg[1] = {&maps.k_bea, &maps.vt_bea, td.bea_row, td.bea_pad, 0, bmax, td.nb, 1};
+  const int bmax = td.kind == 0 ? (c > 1 ? last / c : 0) : last + 1;          // beacons [0, bmax)
   const int tlo = td.kind == 0 ? (c > 1 ? (td.first / c) * c : 0) : td.first * c;
-  const int thi = td.kind == 0 ? last + 1 : (last + 1) * c;
-  seg[2] = {&maps.k_tok, &maps.vt_tok, td.tok_row, td.tok_pad, (tlo / kTile) * kTile, thi, td.T, 2};
+  const int thi = td.kind == 0 ? last + 1 : (last + 1) * c;                     // tokens [tlo, thi)
+  const int lo2 = (tlo / kTile) * kTile;
+  const int nt0 = (td.P + kTile - 1) / kTile, nt1 = (bmax + kTile - 1) / kTile;
+  const int nt2 = thi > lo2 ? (thi - lo2 + kTile - 1) / kTile : 0;
+  const int N = nt0 + nt1 + nt2;
+  // tile n -> segment (0 prompt, 1 beacons, 2 tokens) and first key of the tile inside the segment
+  auto tile_kind = [&](int n) { return n < nt0 ? 0 : (n < nt0 + nt1 ? 1 : 2); };
+  auto tile_k0 = [&](int n, int kind) { return kind == 0 ? n * kTile : (kind == 1 ? (n - nt0) * kTile : lo2 + (n - nt0 - nt1) * kTile); };
 
-  // Running state of this thread's row.  The output accumulator stays in tensor memory for the whole
-  // block: the second product adds to it, and it is rescaled in place only when the row's reference
-  // maximum moves.  The reference follows the true maximum lazily: it is raised only when a tile
-  // exceeds it by more than kMaxSlack (in the log2 domain), so the softmax weights relative to it
-  // stay below 2^kMaxSlack -- exact in the end, because numerator and denominator share the reference.
-  constexpr float kMaxSlack = 8.f;
-  float m_ref = -INFINITY, l_run = 0.f;
-  uint32_t phase = 0;
-  int n_done = 0;   // key tiles already accumulated
-
-  for (int sgi = 0; sgi < 3 && !failed; ++sgi) {
-    const KeySeg& sg = seg[sgi];
-    for (int k0 = sg.lo; k0 < sg.hi && !failed; k0 += kTile, ++n_done) {
-      // ---- K tile (rows = keys) and transposed V tile (rows = d, columns = keys) -------------------
-      // Rows beyond the sequence's keys hold the next sequence's keys (or zeros past the end of the
-      // array): they are masked below.  The transposed V is zero there (padded to 128 columns).
-      if (tid == 0) {
-        mbar_expect_tx(load_bar, 2u * kOperandBytes);
-        tma_3d(sK, sg.k, 0, kvh, sg.row0 + k0, load_bar);
-        tma_3d(sK + kTile * 128, sg.k, 64, kvh, sg.row0 + k0, load_bar);
-        tma_2d(sV, sg.vt, sg.col0 + k0, kvh * kD, load_bar);
-        tma_2d(sV + kTile * 128, sg.vt, sg.col0 + k0 + 64, kvh * kD, load_bar);
-      }
-      if (!mbar_wait_bounded(load_bar, load_phase)) failed = true;
-      failed = __any_sync(0xffffffffu, failed);
-      load_phase ^= 1;
-      if (failed) s_fail = 1;
-      __syncthreads();
-      if (s_fail) failed = true;
-      // ---- S = Q K^T ---------------------------------------------------------------------------------
-      if (tid == 0 && !failed) {
-        tc_fence_after();
+  bool failed = false;
+  if (warp == kRowThreads / 32) {
+    // ======================================= control warp ===========================================
+    if (lane == 0 && N > 0) {
+      // Rows beyond a sequence's keys hold the next sequence's keys (or zeros past the end of the
+      // array): they are masked by the row threads.  The transposed V is zero there (padded to 128).
+      auto issue_k = [&](int n) {
+        const int kind = tile_kind(n), k0 = tile_k0(n, kind);
+        const CUtensorMap* km = kind == 0 ? &maps.k_prompt : (kind == 1 ? &maps.k_bea : &maps.k_tok);
+        const int row = (kind == 0 ? td.prompt_row : (kind == 1 ? td.bea_row : td.tok_row)) + k0;
+        tma_3d(sK, km, 0, kvh, row, bar_k);
+        tma_3d(sK + kTile * 128, km, 64, kvh, row, bar_k);
+      };
+      auto issue_v = [&](int n) {
+        const int kind = tile_kind(n), k0 = tile_k0(n, kind);
+        const CUtensorMap* vm = kind == 0 ? &maps.vt_prompt : (kind == 1 ? &maps.vt_bea : &maps.vt_tok);
+        const int col = (kind == 0 ? td.prompt_pad : (kind == 1 ? td.bea_pad : td.tok_pad)) + k0;
+        mbar_expect_tx(bar_v, (uint32_t)kOperandBytes);
+        tma_2d(sV, vm, col, kvh * kD, bar_v);
+        tma_2d(sV + kTile * 128, vm, col + 64, kvh * kD, bar_v);
+      };
+      auto qk = [&]() {
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
           const uint32_t off = (uint32_t)((kk >> 2) * (kTile * 128) + (kk & 3) * 32);
           umma(tS, umma_desc(sQ + off), umma_desc(sK + off), kk > 0);
         }
-        umma_commit(bar);
+      };
+      // rows of Q beyond the tile's tokens belong to the next sequence or are zero-filled: they are never
+      // visible (their outputs are not written and they contribute to no other row)
+      mbar_expect_tx(bar_k, (uint32_t)(box_rows * kD * 2 + kOperandBytes));
+      {
+        const CUtensorMap* qm = td.kind == 0 ? &maps.q_tok : &maps.q_bea;
+        const int qrow = (td.kind == 0 ? td.tok_row : td.bea_row) + td.first;
+        tma_3d(sQ, qm, 0, kvh * G, qrow, bar_k);
+        tma_3d(sQ + kTile * 128, qm, 64, kvh * G, qrow, bar_k);
       }
-      if (!failed && !mbar_wait_bounded(bar, phase)) failed = true;
-      failed = __any_sync(0xffffffffu, failed);
-      phase ^= 1;
-      tc_fence_after();
-      // ---- mask + softmax weights; this thread owns query row `tid` ------------------------------------
-      // The keys of this segment the row may see form one interval [vlo, vhi); j indexes the tile.
-      int vlo, vhi;
-      if (sg.kind == 0) { vlo = 0; vhi = sg.len; }
-      else if (sg.kind == 1) { vlo = 0; vhi = min(vis_beacons, sg.len); }
-      else { vlo = tok_lo; vhi = min(tok_hi, sg.len); }
-      if (!row_valid) vhi = vlo;
-      const int jlo = max(vlo - k0, 0), jhi = min(vhi - k0, kTile);   // visible columns of the tile
-      // tcgen05.ld / tcgen05.st are warp-wide instructions: every lane executes them, whatever its row
-      // can see, and every branch around them is warp-uniform (`failed` is), so that no transformation
-      // of the code can split a warp between two copies of one of them.
-      const bool all_visible = __all_sync(0xffffffffu, jlo == 0 && jhi == kTile);
-      if (!failed) {
-        float s[kTile];
-#pragma unroll
-        for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tS + lane_base + cb * 32, s + cb * 32);
-        tmem_wait_ld();
-        float tile_max = -INFINITY;
-        if (all_visible) {
-#pragma unroll
-          for (int j = 0; j < kTile; ++j) tile_max = fmaxf(tile_max, s[j]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < kTile; ++j)
-            if (j >= jlo && j < jhi) tile_max = fmaxf(tile_max, s[j]);
-        }
-        tile_max *= a.scale_log2;   // the scale is positive
-        float alpha = 1.f;
-        const bool raise = tile_max > m_ref + kMaxSlack || (m_ref == -INFINITY && tile_max > -INFINITY);
-        if (raise) {
-          alpha = fast_exp2(m_ref - tile_max);   // 0 when nothing had been seen yet
-          m_ref = tile_max;
-          l_run *= alpha;
-        }
-        const float m_safe = m_ref == -INFINITY ? 0.f : m_ref;
-        float tile_sum = 0.f;
-#pragma unroll
-        for (int cb = 0; cb < 4; ++cb) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            float p0 = fast_exp2(fmaf(s[cb * 32 + j], a.scale_log2, -m_safe));
-            float p1 = fast_exp2(fmaf(s[cb * 32 + j + 1], a.scale_log2, -m_safe));
-            if (!all_visible) {
-              if (cb * 32 + j < jlo || cb * 32 + j >= jhi) p0 = 0.f;
-              if (cb * 32 + j + 1 < jlo || cb * 32 + j + 1 >= jhi) p1 = 0.f;
-            }
-            tile_sum += p0 + p1;
-            const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
-            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
-          }
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4)
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sP + swz(tid, cb * 4 + q4)), "r"(pk[q4 * 4]),
-                         "r"(pk[q4 * 4 + 1]), "r"(pk[q4 * 4 + 2]), "r"(pk[q4 * 4 + 3])
-                         : "memory");
-        }
-        l_run += tile_sum;
-        // ---- rescale the accumulator rows whose reference moved (whole warp, if any lane needs it) --------
-        if (n_done > 0 && __any_sync(0xffffffffu, raise)) {
-#pragma unroll 1
-          for (int cb = 0; cb < 4; ++cb) {
-            float t[32];
-            tmem_ld32_async(tO + lane_base + cb * 32, t);
-            tmem_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; ++j) t[j] *= alpha;
-            tmem_st32(tO + lane_base + cb * 32, t);
-          }
-          tmem_wait_st();
-        }
+      issue_k(0);
+      issue_v(0);
+      uint32_t ph_k = 0, ph_v = 0, ph_o = 0;
+      bool ok = mbar_wait_or_fail(bar_k, ph_k, s_fail);
+      ph_k ^= 1;
+      if (ok) {
+        tc_fence_after();
+        qk();
+        umma_commit(bar_s);
       }
-      proxy_fence();
-      tc_fence_before();
-      __syncthreads();
-      // ---- O += P V ----------------------------------------------------------------------------------
-      if (tid == 0 && !failed) {
+      for (int n = 0; n < N && ok; ++n) {
+        ok = mbar_wait_or_fail(bar_s, (uint32_t)n & 1u, s_fail);          // S_n exists: the K buffer is free
+        if (!ok) break;
+        if (n + 1 < N) { mbar_expect_tx(bar_k, (uint32_t)kOperandBytes); issue_k(n + 1); }
+        ok = mbar_wait_or_fail(bar_p, (uint32_t)n & 1u, s_fail) && mbar_wait_or_fail(bar_v, ph_v, s_fail);
+        ph_v ^= 1;
+        if (!ok) break;
         tc_fence_after();
 #pragma unroll
-        for (int kk = 0; kk < kTile / 16; ++kk) {
+        for (int kk = 0; kk < kTile / 16; ++kk) {                           // O += P_n V_n
           const uint32_t off = (uint32_t)((kk >> 2) * (kTile * 128) + (kk & 3) * 32);
-          umma(tO, umma_desc(sP + off), umma_desc(sV + off), (n_done > 0 || kk > 0) ? 1u : 0u);
+          umma_ts(tO, tP + (uint32_t)(kk * 8), umma_desc(sV + off), (n > 0 || kk > 0) ? 1u : 0u);
         }
-        umma_commit(bar);
+        if (n + 1 < N) {
+          umma_commit(bar_o);
+          ok = mbar_wait_or_fail(bar_o, ph_o, s_fail);                      // V buffer and P_n are free
+          ph_o ^= 1;
+          if (!ok) break;
+          issue_v(n + 1);
+          ok = mbar_wait_or_fail(bar_k, ph_k, s_fail);
+          ph_k ^= 1;
+          if (!ok) break;
+          tc_fence_after();
+          qk();
+        }
+        umma_commit(bar_s);
       }
-      // the product must have read P and V before the next tile's copies overwrite them
-      if (!failed) {
-        if (!mbar_wait_bounded(bar, phase)) failed = true;
-        phase ^= 1;
-      }
-      failed = __any_sync(0xffffffffu, failed);
+      if (!ok) { *s_fail = 1; failed = true; }
+    }
+    __syncwarp();
+  } else {
+    // ========================================= row threads ==========================================
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;      // this warp's 32 lanes of tensor memory
+    const int my_local = tid / G;                 // token / beacon inside the tile
+    const bool row_valid = tid < valid_rows;
+    const int my_idx = td.first + my_local;       // token index i, or beacon index (0-based; beacon number my_idx + 1)
+    int vis_beacons, tok_lo, tok_hi;              // visible: beacons [0, vis_beacons), tokens [tok_lo, tok_hi)
+    if (td.kind == 0) { vis_beacons = c > 1 ? my_idx / c : 0; tok_lo = c > 1 ? (my_idx / c) * c : 0; tok_hi = my_idx + 1; }
+    else { vis_beacons = my_idx + 1; tok_lo = my_idx * c; tok_hi = (my_idx + 1) * c; }
+
+    // Running state of this thread's row.  The output accumulator stays in tensor memory for the whole
+    // block: the second product adds to it, and it is rescaled in place only when the row's reference
+    // maximum moves.  The reference follows the true maximum lazily: it is raised only when a tile
+    // exceeds it by more than kMaxSlack (in the log2 domain), so the softmax weights relative to it
+    // stay below 2^kMaxSlack -- exact in the end, because numerator and denominator share the reference.
+    constexpr float kMaxSlack = 8.f;
+    float m_ref = -INFINITY, l_run = 0.f;
+
+    // tcgen05.ld / tcgen05.st are warp-wide instructions: every lane executes them, whatever its row
+    // can see, and every branch around them is warp-uniform, so that no transformation of the code
+    // can split a warp between two copies of one of them.
+    for (int n = 0; n < N; ++n) {
+      const bool ok = mbar_wait_or_fail(bar_s, (uint32_t)n & 1u, s_fail);
+      if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       tc_fence_after();
-      if (failed) s_fail = 1;
-      __syncthreads();
-      if (s_fail) failed = true;
-    }
-  }
-
-  // ---- read the accumulator --------------------------------------------------------------------------
-  float o[kD];
-  if (!failed) {
+      const int kind = tile_kind(n), k0 = tile_k0(n, kind);
+      // The keys of this segment the row may see form one interval [vlo, vhi); j indexes the tile.
+      int vlo, vhi;
+      if (kind == 0) { vlo = 0; vhi = td.P; }
+      else if (kind == 1) { vlo = 0; vhi = min(vis_beacons, td.nb); }
+      else { vlo = tok_lo; vhi = min(tok_hi, td.T); }
+      if (!row_valid) vhi = vlo;
+      const int jlo = max(vlo - k0, 0), jhi = min(vhi - k0, kTile);   // visible columns of the tile
+      const bool all_visible = __all_sync(0xffffffffu, jlo == 0 && jhi == kTile);
+      float s[kTile];
 #pragma unroll
-    for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tO + lane_base + cb * 32, o + cb * 32);
-    tmem_wait_ld();
-  }
-  const float l_fin = l_run;
-
-  // ---- write the rows -------------------------------------------------------------------------------
-  if (!failed && row_valid) {
-    const float inv = l_fin > 0.f ? 1.f / l_fin : 0.f;
-    __nv_bfloat16* dst = (td.kind == 0 ? a.out_tok + (int64_t)(td.tok_row + my_idx) * Hq * kD
-                                       : a.out_bea + (int64_t)(td.bea_row + my_idx) * Hq * kD) +
-                         (int64_t)(kvh * G + tid % G) * kD;
+      for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tS + lane_base + cb * 32, s + cb * 32);
+      tmem_wait_ld();
+      if (!all_visible) {   // partial tile: hide what the row cannot see (warp-uniform branch, no tensor-memory access inside)
 #pragma unroll
-    for (int d = 0; d < kD; d += 8) {
-      uint4 v;
-      __nv_bfloat162 t0 = __floats2bfloat162_rn(o[d] * inv, o[d + 1] * inv), t1 = __floats2bfloat162_rn(o[d + 2] * inv, o[d + 3] * inv);
-      __nv_bfloat162 t2 = __floats2bfloat162_rn(o[d + 4] * inv, o[d + 5] * inv), t3 = __floats2bfloat162_rn(o[d + 6] * inv, o[d + 7] * inv);
-      v.x = *reinterpret_cast<uint32_t*>(&t0); v.y = *reinterpret_cast<uint32_t*>(&t1);
-      v.z = *reinterpret_cast<uint32_t*>(&t2); v.w = *reinterpret_cast<uint32_t*>(&t3);
-      *reinterpret_cast<uint4*>(dst + d) = v;
+        for (int j = 0; j < kTile; ++j)
+          if (j < jlo || j >= jhi) s[j] = -INFINITY;
+      }
+      // four independent chains each for the maximum and the sum: a single chain of 128 dependent
+      // operations would cost more than the exponentials
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int j = 0; j < kTile; j += 4) {
+        mx[0] = fmaxf(mx[0], s[j]); mx[1] = fmaxf(mx[1], s[j + 1]);
+        mx[2] = fmaxf(mx[2], s[j + 2]); mx[3] = fmaxf(mx[3], s[j + 3]);
+      }
+      const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * a.scale_log2;   // the scale is positive
+      float alpha = 1.f;
+      const bool raise = tile_max > m_ref + kMaxSlack || (m_ref == -INFINITY && tile_max > -INFINITY);
+      if (raise) {
+        alpha = fast_exp2(m_ref - tile_max);   // 0 when nothing had been seen yet
+        m_ref = tile_max;
+        l_run *= alpha;
+      }
+      const float m_safe = m_ref == -INFINITY ? 0.f : m_ref;   // hidden entries: exp2(-inf) = 0
+      float sum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 32; j += 2) {
+          const float p0 = fast_exp2(fmaf(s[cb * 32 + j], a.scale_log2, -m_safe));
+          const float p1 = fast_exp2(fmaf(s[cb * 32 + j + 1], a.scale_log2, -m_safe));
+          sum[(j >> 1) & 3] += p0 + p1;
+          const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);   // key 2q in the low half of column q
+          pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+        }
+        tmem_st16(tP + lane_base + cb * 16, pk);   // all of S is in registers already
+      }
+      const float tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
+      l_run += tile_sum;
+      // ---- rescale the accumulator rows whose reference moved (whole warp, if any lane needs it); every
+      //      earlier product has finished, or S_n would not exist ------------------------------------------
+      if (n > 0 && __any_sync(0xffffffffu, raise)) {
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          float t[32];
+          tmem_ld32_async(tO + lane_base + cb * 32, t);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) t[j] *= alpha;
+          tmem_st32(tO + lane_base + cb * 32, t);
+        }
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive_cta(bar_p);
     }
+
+    // ---- read the accumulator and write the rows ------------------------------------------------------
+    if (!failed && N > 0) {
+      const bool ok = mbar_wait_or_fail(bar_s, (uint32_t)N & 1u, s_fail);
+      if (!__all_sync(0xffffffffu, ok)) failed = true;
+    }
+    if (!failed) {
+      float o[kD];
+      if (N > 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tO + lane_base + cb * 32, o + cb * 32);
+        tmem_wait_ld();
+      }
+      if (row_valid) {
+        const float inv = (N > 0 && l_run > 0.f) ? 1.f / l_run : 0.f;
+        __nv_bfloat16* dst = (td.kind == 0 ? a.out_tok + (int64_t)(td.tok_row + my_idx) * Hq * kD
+                                           : a.out_bea + (int64_t)(td.bea_row + my_idx) * Hq * kD) +
+                             (int64_t)(kvh * G + tid % G) * kD;
+#pragma unroll
+        for (int d = 0; d < kD; d += 8) {
+          uint4 v;
+          const float o0 = N > 0 ? o[d] : 0.f, o1 = N > 0 ? o[d + 1] : 0.f, o2 = N > 0 ? o[d + 2] : 0.f, o3 = N > 0 ? o[d + 3] : 0.f;
+          const float o4 = N > 0 ? o[d + 4] : 0.f, o5 = N > 0 ? o[d + 5] : 0.f, o6 = N > 0 ? o[d + 6] : 0.f, o7 = N > 0 ? o[d + 7] : 0.f;
+          __nv_bfloat162 t0 = __floats2bfloat162_rn(o0 * inv, o1 * inv), t1 = __floats2bfloat162_rn(o2 * inv, o3 * inv);
+          __nv_bfloat162 t2 = __floats2bfloat162_rn(o4 * inv, o5 * inv), t3 = __floats2bfloat162_rn(o6 * inv, o7 * inv);
+          v.x = *reinterpret_cast<uint32_t*>(&t0); v.y = *reinterpret_cast<uint32_t*>(&t1);
+          v.z = *reinterpret_cast<uint32_t*>(&t2); v.w = *reinterpret_cast<uint32_t*>(&t3);
+          *reinterpret_cast<uint4*>(dst + d) = v;
+        }
+      }
+    }
+    if (failed) *s_fail = 1;
   }
-  if (failed && tid == 0) atomicCAS(a.status, 0, BC_ERR_TIMEOUT);
   tc_fence_before();
   __syncthreads();
+  if (*s_fail && tid == 0) atomicCAS(a.status, 0, BC_ERR_TIMEOUT);
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");

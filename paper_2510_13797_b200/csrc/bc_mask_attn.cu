@@ -7,22 +7,29 @@
 // of the cache that the decode path maintains step by step (same results, Section 3.2).
 //
 // Unlike decode this is a dense contraction, so it runs on the tcgen05 tensor cores:
-//   * one thread block (128 threads) per (query tile, KV head): 128 query rows = floor(128/G) tokens
-//     (or beacons) times the G query heads that share the KV head, so a K/V tile is reused by G heads;
+//   * one work item per (query tile, KV head): 128 query rows = floor(128/G) tokens (or beacons) times
+//     the G query heads that share the KV head, so a K/V tile is reused by G heads;
 //   * per key tile of 128 keys:  S = Q K^T  (tcgen05.mma, M = N = K = 128, fp32 in tensor memory)
-//     -> tcgen05.ld, mask, online softmax in fp32 registers, P as bf16 into shared memory
-//     -> O += P V  (second tcgen05.mma, accumulating in tensor memory; the rows are rescaled in place,
-//        by tcgen05.ld / tcgen05.st, only when their reference maximum has to be raised);
-//   * operands live in shared memory in the 128-byte-swizzled K-major layout the MMA descriptors
-//     describe, written by tiled tensor copies (cp.async.bulk.tensor, 128-byte swizzle, completion
-//     on an mbarrier) issued by one thread; V is needed K-major too (keys contiguous), so a small
-//     kernel transposes V into the caller's workspace first;
+//     -> tcgen05.ld, mask, online softmax in fp32 registers, P as bf16 back into tensor memory
+//     -> O += P V  (second tcgen05.mma, P read from tensor memory, accumulating in tensor memory; the
+//        rows are rescaled in place, by tcgen05.ld / tcgen05.st, only when their reference maximum has
+//        to be raised);
+//   * operands live in shared memory in the 128-byte-swizzled layouts the MMA descriptors describe,
+//     written by tiled tensor copies (cp.async.bulk.tensor, 128-byte swizzle, completion on an
+//     mbarrier) issued by one thread: Q and K row by row (K-major), V as it is stored, keys by rows
+//     (N-major B operand), so nothing is transposed or staged;
 //   * key tiles a query tile cannot see are skipped: all prompt tiles, the beacon tiles up to its
-//     last visible beacon, and the token tiles that overlap its own windows.
-// Every wait is bounded; on expiry the block records BC_ERR_TIMEOUT, releases its tensor memory and
-// returns.
+//     last visible beacon, and the token tiles that overlap its own windows;
+//   * the kernel is persistent: two blocks per SM walk the work items (sequence by sequence, heaviest
+//     first, dealt out in alternating direction), keep their tensor memory and barriers, and request the next item's
+//     first tiles while the current item's output is still being written.
+// K and V rows past the end of a sequence belong to the next sequence (or read as zero past the end
+// of the array); their scores are masked and their weights are exactly zero, so inputs must be
+// finite everywhere.  Every wait is bounded; on expiry the block records BC_ERR_TIMEOUT, releases
+// its tensor memory and returns.
 #include <cuda.h>
 
+#include <algorithm>
 #include <vector>
 
 #include "bc_common.cuh"
@@ -42,18 +49,42 @@ struct TileDesc {
   int32_t count;       // tokens / beacons in the tile
   int32_t P, T, nb;    // lengths of the sequence
   int32_t prompt_row, tok_row, bea_row;  // first row of the sequence in the packed inputs
-  int32_t prompt_pad, tok_pad, bea_pad;  // first column of the sequence in the transposed V arrays
-  int32_t pad[4];
+  int32_t pad[7];
 };
 
-// Tensor maps (bf16, 128-byte swizzle): q [d, head, row] boxes of (64, G, tokens per tile); k [d, head, row]
-// boxes of (64, 1, 128); transposed v [column, head * 128 + d] boxes of (64, 128).
+// The key tiles one query tile walks: nt0 prompt tiles, nt1 beacon tiles, nt2 token tiles starting at
+// token lo2 (a multiple of 128).
+struct TilePlan {
+  int32_t nt0, nt1, nt2, lo2, N;
+};
+__host__ __device__ inline TilePlan make_plan(const TileDesc& td, int c) {
+  const int last = td.first + td.count - 1;
+  const int bmax = td.kind == 0 ? (c > 1 ? last / c : 0) : last + 1;           // beacons [0, bmax)
+  const int tlo = td.kind == 0 ? (c > 1 ? (td.first / c) * c : 0) : td.first * c;
+  const int thi = td.kind == 0 ? last + 1 : (last + 1) * c;                      // tokens [tlo, thi)
+  TilePlan p;
+  p.lo2 = (tlo / kTile) * kTile;
+  p.nt0 = (td.P + kTile - 1) / kTile;
+  p.nt1 = (bmax + kTile - 1) / kTile;
+  p.nt2 = thi > p.lo2 ? (thi - p.lo2 + kTile - 1) / kTile : 0;
+  p.N = p.nt0 + p.nt1 + p.nt2;
+  return p;
+}
+// tile n -> segment (0 prompt, 1 beacons, 2 tokens) and first key of the tile inside the segment
+__device__ __forceinline__ int plan_kind(const TilePlan& p, int n) { return n < p.nt0 ? 0 : (n < p.nt0 + p.nt1 ? 1 : 2); }
+__device__ __forceinline__ int plan_k0(const TilePlan& p, int n, int kind) {
+  return kind == 0 ? n * kTile : (kind == 1 ? (n - p.nt0) * kTile : p.lo2 + (n - p.nt0 - p.nt1) * kTile);
+}
+
+// Tensor maps (bf16, [rows][heads][128] seen as (d, head, row), 128-byte swizzle): q boxes of
+// (64, G, tokens per tile); k and v boxes of (64, 1, 128).
 struct MaskMaps {
-  CUtensorMap q_tok, q_bea, k_prompt, k_tok, k_bea, vt_prompt, vt_tok, vt_bea;
+  CUtensorMap q_tok, q_bea, k_prompt, k_tok, k_bea, v_prompt, v_tok, v_bea;
 };
 
 struct MaskArgs {
-  const TileDesc* tiles;
+  const TileDesc* tiles;   // sequence by sequence, heaviest query tiles of a sequence first
+  int32_t n_items;         // tiles x kv_heads; item i = (tile i / kv_heads, head i % kv_heads)
   __nv_bfloat16 *out_tok, *out_bea;
   int32_t* status;     // device int: first error code
   int32_t Hq, Hkv, G, c, rows_per_tile;  // rows_per_tile = tokens per query tile = 128 / G
@@ -77,11 +108,6 @@ __device__ __forceinline__ void tma_3d(uint32_t dst, const CUtensorMap* map, int
       "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
       : "memory");
 }
-__device__ __forceinline__ void tma_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-               "l"(map), "r"(c0), "r"(c1), "r"(bar)
-               : "memory");
-}
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -99,9 +125,22 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                    // 128-byte swizzle
   return d;
 }
+// The same for an N-major B operand (V as stored: 128 keys by rows of 128 bytes = 64 head dimensions,
+// the other 64 dimensions 16 KB further): 8-key groups 1024 bytes apart along K, the two 64-wide
+// halves of N kLeadBytes apart.
+__device__ __forceinline__ uint64_t umma_desc_nmajor(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3ffff) >> 4);
+  d |= (uint64_t)((kTile * 128) >> 4) << 16;  // leading byte offset: next 64 elements of N
+  d |= (uint64_t)(1024 >> 4) << 32;           // stride byte offset: next 8 keys
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
 
+constexpr uint32_t kIdescBN = kIdesc | (1u << 16);   // B operand N-major
 __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t a, uint64_t b, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
@@ -156,7 +195,7 @@ __device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64
   asm volatile(
       "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
-      "r"(tmem_a), "l"(b), "r"(kIdesc), "r"(accumulate)
+      "r"(tmem_a), "l"(b), "r"(kIdescBN), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
@@ -194,31 +233,31 @@ __device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity,
 // engine one tile ahead: K_{n+1} is requested as soon as S_n exists (the K buffer is free), V_{n+1} as
 // soon as O += P_n V_n has completed (the V buffer is free), so their latency hides behind the softmax
 // and the products; the products of the block's neighbour on the SM fill the tensor pipe meanwhile.
-// Q K_{n+1}^T overwrites P_n, so it is issued only after P_n V_n has completed.
+// Q K_{n+1}^T overwrites P_n, so it is issued only after P_n V_n has completed.  The tile stream runs
+// on across work items: after an item's last S the next item's Q and first K are requested, and its
+// first product into O waits until the rows have read the finished O.
 //
-// Barriers (all single-phase mbarriers, parity = completion count & 1):
-//   bar_k: Q and K_0, then K_1, K_2 ...  have landed     bar_v: V_n has landed
-//   bar_s: completion n = S_n is ready (and every earlier product has finished); completion N = O is final
-//   bar_p: the 128 row threads have stored P_n           bar_o: P_n V_n has completed
+// Barriers (single-phase mbarriers; t counts key tiles, e work items, parity = count & 1):
+//   bar_k: a K tile (with Q, at the start of an item) has landed      bar_v: a V tile has landed
+//   bar_s: completion t = S of tile t is ready (and every earlier product has finished)
+//   bar_p: the 128 row threads have stored P of tile t                bar_o: P V of a tile has completed
+//   bar_f: completion e = O of item e is final                       bar_e: the rows have read O of item e
 __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, const __grid_constant__ MaskMaps maps) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sQ = smem_addr(smem), sK = sQ + kOperandBytes, sV = sK + kOperandBytes;
-  __shared__ __align__(8) uint64_t s_bars[5];
+  __shared__ __align__(8) uint64_t s_bars[7];
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail_word;
   volatile int* s_fail = &s_fail_word;
-  const uint32_t bar_k = smem_addr(&s_bars[0]), bar_v = bar_k + 8, bar_s = bar_k + 16, bar_p = bar_k + 24, bar_o = bar_k + 32;
+  const uint32_t bar_k = smem_addr(&s_bars[0]), bar_v = bar_k + 8, bar_s = bar_k + 16, bar_p = bar_k + 24, bar_o = bar_k + 32,
+                 bar_f = bar_k + 40, bar_e = bar_k + 48;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const TileDesc td = a.tiles[blockIdx.x];
-  const int kvh = blockIdx.y, G = a.G, Hq = a.Hq, c = a.c;
+  const int G = a.G, Hq = a.Hq, Hkv = a.Hkv, c = a.c;
 
   if (tid == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_k) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_v) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_s) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_p), "r"(kRowThreads) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_o) : "memory");
+    const uint32_t counts[7] = {1, 1, 1, (uint32_t)kRowThreads, 1, 1, (uint32_t)kRowThreads};
+    for (int i = 0; i < 7; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_k + i * 8), "r"(counts[i]) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     *s_fail = 0;
   }
@@ -226,11 +265,9 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&s_tmem)), "r"(256) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-
-  // ---- the query tile: row r = (local index r / G, head r % G) ---------------------------------
-  const int valid_rows = td.count * G;
-  const int box_rows = a.rows_per_tile * G;   // rows the tensor copy writes (all 128 unless G does not divide 128)
-  for (int idx = tid; idx < (kTile - box_rows) * 16; idx += kThreads) {   // rows the copy leaves untouched
+  // Rows of the Q buffer that no tensor copy writes (only when G does not divide 128) stay zero.
+  const int box_rows = a.rows_per_tile * G;
+  for (int idx = tid; idx < (kTile - box_rows) * 16; idx += kThreads) {
     const int r = box_rows + (idx >> 4), ch = idx & 15;
     st_zero16(sQ + swz(r, ch));
   }
@@ -242,39 +279,40 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
   const uint32_t tS = tmem, tO = tmem + kTile;   // columns [0,128): S, then P in its first 64; [128,256): O
   const uint32_t tP = tS;
 
-  // ---- key tiles some row of this block can see: prompt, beacons, tokens ---------------------------
-  const int last = td.first + td.count - 1;
-  const int bmax = td.kind == 0 ? (c > 1 ? last / c : 0) : last + 1;          // beacons [0, bmax)
-  const int tlo = td.kind == 0 ? (c > 1 ? (td.first / c) * c : 0) : td.first * c;
-  const int thi = td.kind == 0 ? last + 1 : (last + 1) * c;                     // tokens [tlo, thi)
-  const int lo2 = (tlo / kTile) * kTile;
-  const int nt0 = (td.P + kTile - 1) / kTile, nt1 = (bmax + kTile - 1) / kTile;
-  const int nt2 = thi > lo2 ? (thi - lo2 + kTile - 1) / kTile : 0;
-  const int N = nt0 + nt1 + nt2;
-  // tile n -> segment (0 prompt, 1 beacons, 2 tokens) and first key of the tile inside the segment
-  auto tile_kind = [&](int n) { return n < nt0 ? 0 : (n < nt0 + nt1 ? 1 : 2); };
-  auto tile_k0 = [&](int n, int kind) { return kind == 0 ? n * kTile : (kind == 1 ? (n - nt0) * kTile : lo2 + (n - nt0 - nt1) * kTile); };
+  // Work items of this block: round r hands out items [r * grid, (r + 1) * grid), forwards in even
+  // rounds and backwards in odd ones, so that the heavy and the light end of the sorted list meet.
+  const int grid = (int)gridDim.x, bid = (int)blockIdx.x;
+  auto item_of = [&](int r) {
+    const int it = r * grid + ((r & 1) ? grid - 1 - bid : bid);
+    return it < a.n_items ? it : -1;
+  };
 
-  bool failed = false;
   if (warp == kRowThreads / 32) {
     // ======================================= control warp ===========================================
-    if (lane == 0 && N > 0) {
-      // Rows beyond a sequence's keys hold the next sequence's keys (or zeros past the end of the
-      // array): they are masked by the row threads.  The transposed V is zero there (padded to 128).
-      auto issue_k = [&](int n) {
-        const int kind = tile_kind(n), k0 = tile_k0(n, kind);
+    int item = item_of(0);
+    if (lane == 0 && item >= 0) {
+      auto issue_q = [&](const TileDesc& td, int kvh) {
+        // rows of Q beyond the tile's tokens belong to the next sequence or are zero-filled: they are never
+        // visible (their outputs are not written and they contribute to no other row)
+        const CUtensorMap* qm = td.kind == 0 ? &maps.q_tok : &maps.q_bea;
+        const int qrow = (td.kind == 0 ? td.tok_row : td.bea_row) + td.first;
+        tma_3d(sQ, qm, 0, kvh * G, qrow, bar_k);
+        tma_3d(sQ + kTile * 128, qm, 64, kvh * G, qrow, bar_k);
+      };
+      auto issue_k = [&](const TileDesc& td, const TilePlan& pl, int kvh, int n) {
+        const int kind = plan_kind(pl, n), k0 = plan_k0(pl, n, kind);
         const CUtensorMap* km = kind == 0 ? &maps.k_prompt : (kind == 1 ? &maps.k_bea : &maps.k_tok);
         const int row = (kind == 0 ? td.prompt_row : (kind == 1 ? td.bea_row : td.tok_row)) + k0;
         tma_3d(sK, km, 0, kvh, row, bar_k);
         tma_3d(sK + kTile * 128, km, 64, kvh, row, bar_k);
       };
-      auto issue_v = [&](int n) {
-        const int kind = tile_kind(n), k0 = tile_k0(n, kind);
-        const CUtensorMap* vm = kind == 0 ? &maps.vt_prompt : (kind == 1 ? &maps.vt_bea : &maps.vt_tok);
-        const int col = (kind == 0 ? td.prompt_pad : (kind == 1 ? td.bea_pad : td.tok_pad)) + k0;
+      auto issue_v = [&](const TileDesc& td, const TilePlan& pl, int kvh, int n) {
+        const int kind = plan_kind(pl, n), k0 = plan_k0(pl, n, kind);
+        const CUtensorMap* vm = kind == 0 ? &maps.v_prompt : (kind == 1 ? &maps.v_bea : &maps.v_tok);
+        const int row = (kind == 0 ? td.prompt_row : (kind == 1 ? td.bea_row : td.tok_row)) + k0;
         mbar_expect_tx(bar_v, (uint32_t)kOperandBytes);
-        tma_2d(sV, vm, col, kvh * kD, bar_v);
-        tma_2d(sV + kTile * 128, vm, col + 64, kvh * kD, bar_v);
+        tma_3d(sV, vm, 0, kvh, row, bar_v);
+        tma_3d(sV + kTile * 128, vm, 64, kvh, row, bar_v);
       };
       auto qk = [&]() {
 #pragma unroll
@@ -283,18 +321,15 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
           umma(tS, umma_desc(sQ + off), umma_desc(sK + off), kk > 0);
         }
       };
-      // rows of Q beyond the tile's tokens belong to the next sequence or are zero-filled: they are never
-      // visible (their outputs are not written and they contribute to no other row)
-      mbar_expect_tx(bar_k, (uint32_t)(box_rows * kD * 2 + kOperandBytes));
-      {
-        const CUtensorMap* qm = td.kind == 0 ? &maps.q_tok : &maps.q_bea;
-        const int qrow = (td.kind == 0 ? td.tok_row : td.bea_row) + td.first;
-        tma_3d(sQ, qm, 0, kvh * G, qrow, bar_k);
-        tma_3d(sQ + kTile * 128, qm, 64, kvh * G, qrow, bar_k);
-      }
-      issue_k(0);
-      issue_v(0);
-      uint32_t ph_k = 0, ph_v = 0, ph_o = 0;
+      const uint32_t q_bytes = (uint32_t)(box_rows * kD * 2);
+      TileDesc td = a.tiles[item / Hkv];
+      int kvh = item % Hkv;
+      TilePlan pl = make_plan(td, c);
+      mbar_expect_tx(bar_k, q_bytes + (uint32_t)kOperandBytes);
+      issue_q(td, kvh);
+      issue_k(td, pl, kvh, 0);
+      issue_v(td, pl, kvh, 0);
+      uint32_t ph_k = 0, ph_v = 0, ph_o = 0, t = 0, e = 0;
       bool ok = mbar_wait_or_fail(bar_k, ph_k, s_fail);
       ph_k ^= 1;
       if (ok) {
@@ -302,160 +337,184 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
         qk();
         umma_commit(bar_s);
       }
-      for (int n = 0; n < N && ok; ++n) {
-        ok = mbar_wait_or_fail(bar_s, (uint32_t)n & 1u, s_fail);          // S_n exists: the K buffer is free
-        if (!ok) break;
-        if (n + 1 < N) { mbar_expect_tx(bar_k, (uint32_t)kOperandBytes); issue_k(n + 1); }
-        ok = mbar_wait_or_fail(bar_p, (uint32_t)n & 1u, s_fail) && mbar_wait_or_fail(bar_v, ph_v, s_fail);
-        ph_v ^= 1;
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < kTile / 16; ++kk) {                           // O += P_n V_n
-          const uint32_t off = (uint32_t)((kk >> 2) * (kTile * 128) + (kk & 3) * 32);
-          umma_ts(tO, tP + (uint32_t)(kk * 8), umma_desc(sV + off), (n > 0 || kk > 0) ? 1u : 0u);
-        }
-        if (n + 1 < N) {
-          umma_commit(bar_o);
-          ok = mbar_wait_or_fail(bar_o, ph_o, s_fail);                      // V buffer and P_n are free
-          ph_o ^= 1;
+      for (int r = 0; ok; ++r, ++e) {
+        const int nitem = item_of(r + 1);
+        TileDesc ntd = td;
+        TilePlan npl = pl;
+        int nkvh = 0;
+        if (nitem >= 0) { ntd = a.tiles[nitem / Hkv]; nkvh = nitem % Hkv; npl = make_plan(ntd, c); }
+        for (int n = 0; n < pl.N && ok; ++n, ++t) {
+          ok = mbar_wait_or_fail(bar_s, t & 1u, s_fail);                     // S exists: the K buffer is free
           if (!ok) break;
-          issue_v(n + 1);
-          ok = mbar_wait_or_fail(bar_k, ph_k, s_fail);
-          ph_k ^= 1;
+          const bool last = n + 1 == pl.N;
+          if (!last) {
+            mbar_expect_tx(bar_k, (uint32_t)kOperandBytes);
+            issue_k(td, pl, kvh, n + 1);
+          } else if (nitem >= 0) {                                            // ... and so is the Q buffer
+            mbar_expect_tx(bar_k, q_bytes + (uint32_t)kOperandBytes);
+            issue_q(ntd, nkvh);
+            issue_k(ntd, npl, nkvh, 0);
+          }
+          ok = mbar_wait_or_fail(bar_p, t & 1u, s_fail) && mbar_wait_or_fail(bar_v, ph_v, s_fail);
+          ph_v ^= 1;
+          if (ok && n == 0 && e > 0) ok = mbar_wait_or_fail(bar_e, (e - 1) & 1u, s_fail);   // the rows have read the last O
           if (!ok) break;
           tc_fence_after();
-          qk();
+#pragma unroll
+          for (int kk = 0; kk < kTile / 16; ++kk)                             // O += P V, 16 keys at a time
+            umma_ts(tO, tP + (uint32_t)(kk * 8), umma_desc_nmajor(sV + (uint32_t)(kk * 16 * 128)), (n > 0 || kk > 0) ? 1u : 0u);
+          if (last) umma_commit(bar_f);
+          if (!last || nitem >= 0) {
+            umma_commit(bar_o);
+            ok = mbar_wait_or_fail(bar_o, ph_o, s_fail);                      // V buffer and P are free
+            ph_o ^= 1;
+            if (!ok) break;
+            if (!last) issue_v(td, pl, kvh, n + 1); else issue_v(ntd, npl, nkvh, 0);
+            ok = mbar_wait_or_fail(bar_k, ph_k, s_fail);
+            ph_k ^= 1;
+            if (!ok) break;
+            tc_fence_after();
+            qk();
+            umma_commit(bar_s);
+          }
         }
-        umma_commit(bar_s);
+        if (nitem < 0) break;
+        td = ntd; pl = npl; kvh = nkvh;
       }
-      if (!ok) { *s_fail = 1; failed = true; }
+      if (!ok) *s_fail = 1;
     }
     __syncwarp();
   } else {
     // ========================================= row threads ==========================================
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;      // this warp's 32 lanes of tensor memory
-    const int my_local = tid / G;                 // token / beacon inside the tile
-    const bool row_valid = tid < valid_rows;
-    const int my_idx = td.first + my_local;       // token index i, or beacon index (0-based; beacon number my_idx + 1)
-    int vis_beacons, tok_lo, tok_hi;              // visible: beacons [0, vis_beacons), tokens [tok_lo, tok_hi)
-    if (td.kind == 0) { vis_beacons = c > 1 ? my_idx / c : 0; tok_lo = c > 1 ? (my_idx / c) * c : 0; tok_hi = my_idx + 1; }
-    else { vis_beacons = my_idx + 1; tok_lo = my_idx * c; tok_hi = (my_idx + 1) * c; }
-
-    // Running state of this thread's row.  The output accumulator stays in tensor memory for the whole
-    // block: the second product adds to it, and it is rescaled in place only when the row's reference
-    // maximum moves.  The reference follows the true maximum lazily: it is raised only when a tile
-    // exceeds it by more than kMaxSlack (in the log2 domain), so the softmax weights relative to it
-    // stay below 2^kMaxSlack -- exact in the end, because numerator and denominator share the reference.
+    const int my_local = tid / G, my_head = tid % G;              // token / beacon inside the tile, head inside the group
+    // The output accumulator stays in tensor memory for a whole item: the second product adds to it,
+    // and it is rescaled in place only when the row's reference maximum moves.  The reference follows
+    // the true maximum lazily: it is raised only when a tile exceeds it by more than kMaxSlack (in the
+    // log2 domain), so the softmax weights relative to it stay below 2^kMaxSlack -- exact in the end,
+    // because numerator and denominator share the reference.
     constexpr float kMaxSlack = 8.f;
-    float m_ref = -INFINITY, l_run = 0.f;
-
+    bool failed = false;
+    uint32_t t = 0, e = 0;
+    int item = item_of(0);
+    TileDesc td = {};
+    if (item >= 0) td = a.tiles[item / Hkv];
     // tcgen05.ld / tcgen05.st are warp-wide instructions: every lane executes them, whatever its row
     // can see, and every branch around them is warp-uniform, so that no transformation of the code
     // can split a warp between two copies of one of them.
-    for (int n = 0; n < N; ++n) {
-      const bool ok = mbar_wait_or_fail(bar_s, (uint32_t)n & 1u, s_fail);
+    for (int r = 0; item >= 0 && !failed; ++r, ++e) {
+      const int kvh = item % Hkv;
+      const TilePlan pl = make_plan(td, c);
+      const bool row_valid = tid < td.count * G;
+      const int my_idx = td.first + my_local;       // token index i, or beacon index (0-based; beacon number my_idx + 1)
+      int vis_beacons, tok_lo, tok_hi;              // visible: beacons [0, vis_beacons), tokens [tok_lo, tok_hi)
+      if (td.kind == 0) { vis_beacons = c > 1 ? my_idx / c : 0; tok_lo = c > 1 ? (my_idx / c) * c : 0; tok_hi = my_idx + 1; }
+      else { vis_beacons = my_idx + 1; tok_lo = my_idx * c; tok_hi = (my_idx + 1) * c; }
+      float m_ref = -INFINITY, l_run = 0.f;
+
+      for (int n = 0; n < pl.N; ++n, ++t) {
+        const bool ok = mbar_wait_or_fail(bar_s, t & 1u, s_fail);
+        if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+        tc_fence_after();
+        const int kind = plan_kind(pl, n), k0 = plan_k0(pl, n, kind);
+        // The keys of this segment the row may see form one interval [vlo, vhi); j indexes the tile.
+        int vlo, vhi;
+        if (kind == 0) { vlo = 0; vhi = td.P; }
+        else if (kind == 1) { vlo = 0; vhi = min(vis_beacons, td.nb); }
+        else { vlo = tok_lo; vhi = min(tok_hi, td.T); }
+        if (!row_valid) vhi = vlo;
+        const int jlo = max(vlo - k0, 0), jhi = min(vhi - k0, kTile);   // visible columns of the tile
+        const bool all_visible = __all_sync(0xffffffffu, jlo == 0 && jhi == kTile);
+        float s[kTile];
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tS + lane_base + cb * 32, s + cb * 32);
+        tmem_wait_ld();
+        if (!all_visible) {   // partial tile: hide what the row cannot see (warp-uniform branch, no tensor-memory access inside)
+#pragma unroll
+          for (int j = 0; j < kTile; ++j)
+            if (j < jlo || j >= jhi) s[j] = -INFINITY;
+        }
+        // four independent chains each for the maximum and the sum: a single chain of 128 dependent
+        // operations would cost more than the exponentials
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int j = 0; j < kTile; j += 4) {
+          mx[0] = fmaxf(mx[0], s[j]); mx[1] = fmaxf(mx[1], s[j + 1]);
+          mx[2] = fmaxf(mx[2], s[j + 2]); mx[3] = fmaxf(mx[3], s[j + 3]);
+        }
+        const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * a.scale_log2;   // the scale is positive
+        float alpha = 1.f;
+        const bool raise = tile_max > m_ref + kMaxSlack || (m_ref == -INFINITY && tile_max > -INFINITY);
+        if (raise) {
+          alpha = fast_exp2(m_ref - tile_max);   // 0 when nothing had been seen yet
+          m_ref = tile_max;
+          l_run *= alpha;
+        }
+        const float m_safe = m_ref == -INFINITY ? 0.f : m_ref;   // hidden entries: exp2(-inf) = 0
+        float sum[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) {
+            const float p0 = fast_exp2(fmaf(s[cb * 32 + j], a.scale_log2, -m_safe));
+            const float p1 = fast_exp2(fmaf(s[cb * 32 + j + 1], a.scale_log2, -m_safe));
+            sum[(j >> 1) & 3] += p0 + p1;
+            const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);   // key 2q in the low half of column q
+            pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
+          }
+          tmem_st16(tP + lane_base + cb * 16, pk);   // all of S is in registers already
+        }
+        l_run += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+        // ---- rescale the accumulator rows whose reference moved (whole warp, if any lane needs it); every
+        //      earlier product has finished, or this tile's S would not exist --------------------------------
+        if (n > 0 && __any_sync(0xffffffffu, raise)) {
+#pragma unroll 1
+          for (int cb = 0; cb < 4; ++cb) {
+            float u[32];
+            tmem_ld32_async(tO + lane_base + cb * 32, u);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) u[j] *= alpha;
+            tmem_st32(tO + lane_base + cb * 32, u);
+          }
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive_cta(bar_p);
+      }
+      if (failed) break;
+
+      // ---- the item's output: read the accumulator, hand it back, write the rows ----------------------
+      const int nitem = item_of(r + 1);
+      TileDesc ntd = {};
+      if (nitem >= 0) ntd = a.tiles[nitem / Hkv];   // in flight during the wait below
+      const bool ok = mbar_wait_or_fail(bar_f, e & 1u, s_fail);
       if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       tc_fence_after();
-      const int kind = tile_kind(n), k0 = tile_k0(n, kind);
-      // The keys of this segment the row may see form one interval [vlo, vhi); j indexes the tile.
-      int vlo, vhi;
-      if (kind == 0) { vlo = 0; vhi = td.P; }
-      else if (kind == 1) { vlo = 0; vhi = min(vis_beacons, td.nb); }
-      else { vlo = tok_lo; vhi = min(tok_hi, td.T); }
-      if (!row_valid) vhi = vlo;
-      const int jlo = max(vlo - k0, 0), jhi = min(vhi - k0, kTile);   // visible columns of the tile
-      const bool all_visible = __all_sync(0xffffffffu, jlo == 0 && jhi == kTile);
-      float s[kTile];
-#pragma unroll
-      for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tS + lane_base + cb * 32, s + cb * 32);
-      tmem_wait_ld();
-      if (!all_visible) {   // partial tile: hide what the row cannot see (warp-uniform branch, no tensor-memory access inside)
-#pragma unroll
-        for (int j = 0; j < kTile; ++j)
-          if (j < jlo || j >= jhi) s[j] = -INFINITY;
-      }
-      // four independent chains each for the maximum and the sum: a single chain of 128 dependent
-      // operations would cost more than the exponentials
-      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-      for (int j = 0; j < kTile; j += 4) {
-        mx[0] = fmaxf(mx[0], s[j]); mx[1] = fmaxf(mx[1], s[j + 1]);
-        mx[2] = fmaxf(mx[2], s[j + 2]); mx[3] = fmaxf(mx[3], s[j + 3]);
-      }
-      const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * a.scale_log2;   // the scale is positive
-      float alpha = 1.f;
-      const bool raise = tile_max > m_ref + kMaxSlack || (m_ref == -INFINITY && tile_max > -INFINITY);
-      if (raise) {
-        alpha = fast_exp2(m_ref - tile_max);   // 0 when nothing had been seen yet
-        m_ref = tile_max;
-        l_run *= alpha;
-      }
-      const float m_safe = m_ref == -INFINITY ? 0.f : m_ref;   // hidden entries: exp2(-inf) = 0
-      float sum[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int cb = 0; cb < 4; ++cb) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          const float p0 = fast_exp2(fmaf(s[cb * 32 + j], a.scale_log2, -m_safe));
-          const float p1 = fast_exp2(fmaf(s[cb * 32 + j + 1], a.scale_log2, -m_safe));
-          sum[(j >> 1) & 3] += p0 + p1;
-          const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);   // key 2q in the low half of column q
-          pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&pb);
-        }
-        tmem_st16(tP + lane_base + cb * 16, pk);   // all of S is in registers already
-      }
-      const float tile_sum = (sum[0] + sum[1]) + (sum[2] + sum[3]);
-      l_run += tile_sum;
-      // ---- rescale the accumulator rows whose reference moved (whole warp, if any lane needs it); every
-      //      earlier product has finished, or S_n would not exist ------------------------------------------
-      if (n > 0 && __any_sync(0xffffffffu, raise)) {
-#pragma unroll 1
-        for (int cb = 0; cb < 4; ++cb) {
-          float t[32];
-          tmem_ld32_async(tO + lane_base + cb * 32, t);
-          tmem_wait_ld();
-#pragma unroll
-          for (int j = 0; j < 32; ++j) t[j] *= alpha;
-          tmem_st32(tO + lane_base + cb * 32, t);
-        }
-      }
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive_cta(bar_p);
-    }
-
-    // ---- read the accumulator and write the rows ------------------------------------------------------
-    if (!failed && N > 0) {
-      const bool ok = mbar_wait_or_fail(bar_s, (uint32_t)N & 1u, s_fail);
-      if (!__all_sync(0xffffffffu, ok)) failed = true;
-    }
-    if (!failed) {
       float o[kD];
-      if (N > 0) {
-        tc_fence_after();
 #pragma unroll
-        for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tO + lane_base + cb * 32, o + cb * 32);
-        tmem_wait_ld();
-      }
+      for (int cb = 0; cb < 4; ++cb) tmem_ld32_async(tO + lane_base + cb * 32, o + cb * 32);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive_cta(bar_e);
       if (row_valid) {
-        const float inv = (N > 0 && l_run > 0.f) ? 1.f / l_run : 0.f;
+        const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
         __nv_bfloat16* dst = (td.kind == 0 ? a.out_tok + (int64_t)(td.tok_row + my_idx) * Hq * kD
                                            : a.out_bea + (int64_t)(td.bea_row + my_idx) * Hq * kD) +
-                             (int64_t)(kvh * G + tid % G) * kD;
+                             (int64_t)(kvh * G + my_head) * kD;
 #pragma unroll
         for (int d = 0; d < kD; d += 8) {
           uint4 v;
-          const float o0 = N > 0 ? o[d] : 0.f, o1 = N > 0 ? o[d + 1] : 0.f, o2 = N > 0 ? o[d + 2] : 0.f, o3 = N > 0 ? o[d + 3] : 0.f;
-          const float o4 = N > 0 ? o[d + 4] : 0.f, o5 = N > 0 ? o[d + 5] : 0.f, o6 = N > 0 ? o[d + 6] : 0.f, o7 = N > 0 ? o[d + 7] : 0.f;
-          __nv_bfloat162 t0 = __floats2bfloat162_rn(o0 * inv, o1 * inv), t1 = __floats2bfloat162_rn(o2 * inv, o3 * inv);
-          __nv_bfloat162 t2 = __floats2bfloat162_rn(o4 * inv, o5 * inv), t3 = __floats2bfloat162_rn(o6 * inv, o7 * inv);
+          __nv_bfloat162 t0 = __floats2bfloat162_rn(o[d] * inv, o[d + 1] * inv), t1 = __floats2bfloat162_rn(o[d + 2] * inv, o[d + 3] * inv);
+          __nv_bfloat162 t2 = __floats2bfloat162_rn(o[d + 4] * inv, o[d + 5] * inv), t3 = __floats2bfloat162_rn(o[d + 6] * inv, o[d + 7] * inv);
           v.x = *reinterpret_cast<uint32_t*>(&t0); v.y = *reinterpret_cast<uint32_t*>(&t1);
           v.z = *reinterpret_cast<uint32_t*>(&t2); v.w = *reinterpret_cast<uint32_t*>(&t3);
           *reinterpret_cast<uint4*>(dst + d) = v;
         }
       }
+      item = nitem;
+      td = ntd;
     }
     if (failed) *s_fail = 1;
   }
@@ -465,30 +524,6 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
   if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
-  }
-}
-
-// vt[(h * D + d) * cols + pad_base + r] = v[(row_base + r) * Hkv * D + h * D + d]; columns of the
-// padding (r >= rows of the sequence) are written as zero.  grid (sequence, kv head, 32-row blocks).
-struct TransposeSeq {
-  int32_t row_base, rows, pad_base, pad_rows;
-};
-__global__ void k_transpose_v(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ vt, const TransposeSeq* seqs,
-                              int Hkv, int64_t cols) {
-  __shared__ __nv_bfloat16 tile[32][kD + 2];
-  const TransposeSeq sq = seqs[blockIdx.x];
-  const int h = blockIdx.y;
-  for (int r0 = blockIdx.z * 32; r0 < sq.pad_rows; r0 += gridDim.z * 32) {
-    for (int idx = threadIdx.x; idx < 32 * kD; idx += blockDim.x) {
-      const int r = idx / kD, d = idx % kD;
-      tile[r][d] = (r0 + r < sq.rows) ? v[((int64_t)(sq.row_base + r0 + r) * Hkv + h) * kD + d] : __float2bfloat16(0.f);
-    }
-    __syncthreads();
-    for (int idx = threadIdx.x; idx < 32 * kD; idx += blockDim.x) {
-      const int d = idx / 32, r = idx % 32;
-      if (r0 + r < sq.pad_rows) vt[((int64_t)h * kD + d) * cols + sq.pad_base + r0 + r] = tile[r][d];
-    }
-    __syncthreads();
   }
 }
 
@@ -515,43 +550,32 @@ bool map_3d(CUtensorMap* m, const void* base, int heads, int64_t rows, int box_h
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-// [rows][cols] bf16 seen as (col, row); box (64, 128)
-bool map_2d(CUtensorMap* m, const void* base, int64_t cols, int64_t rows) {
-  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)kTile}, es[2] = {1, 1};
-  return encode_tiled()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-inline int64_t pad128(int64_t x) { return (x + 127) / 128 * 128; }
-
 struct MaskLayout {
-  size_t tiles, seqs3, status, vt_prompt, vt_tok, vt_bea, total;
-  int64_t prompt_cols, tok_cols, bea_cols;
+  size_t tiles, status, total;
   int64_t n_tiles;
 };
 
-// Upper bounds from the totals alone (every sequence may add one partial tile / 127 padding columns).
-MaskLayout mask_layout(int n_seqs, int q_heads, int kv_heads, int64_t total_prompt, int64_t total_tokens, int64_t total_beacons) {
+// Upper bound from the totals alone (every sequence may add one partial tile of each kind).
+MaskLayout mask_layout(int n_seqs, int q_heads, int kv_heads, int64_t total_tokens, int64_t total_beacons) {
   MaskLayout l;
   const int G = q_heads / kv_heads, per = kTile / G;
   l.n_tiles = (total_tokens + per - 1) / per + (total_beacons + per - 1) / per + 2 * (int64_t)n_seqs;
-  l.prompt_cols = pad128(total_prompt + 127 * (int64_t)n_seqs);
-  l.tok_cols = pad128(total_tokens + 127 * (int64_t)n_seqs);
-  l.bea_cols = pad128(total_beacons + 127 * (int64_t)n_seqs);
   size_t o = 0;
   auto take = [&](size_t b) { size_t at = o; o = align_up(o + b, 256); return at; };
   l.tiles = take((size_t)l.n_tiles * sizeof(TileDesc));
-  l.seqs3 = take((size_t)3 * n_seqs * sizeof(TransposeSeq));
   l.status = take(256);
-  l.vt_prompt = take((size_t)kv_heads * kD * l.prompt_cols * 2);
-  l.vt_tok = take((size_t)kv_heads * kD * l.tok_cols * 2);
-  l.vt_bea = take((size_t)kv_heads * kD * l.bea_cols * 2);
   l.total = o;
   return l;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+  }
+  return n;
 }
 
 }  // namespace
@@ -565,7 +589,7 @@ bc_status bc_mask_attn_query_bytes(int32_t n_seqs, int32_t q_heads, int32_t kv_h
       total_tokens < 0 || total_beacons < 0)
     return BC_ERR_INVALID_ARG;
   if (head_dim != kD || q_heads / kv_heads > 16) return BC_ERR_UNSUPPORTED;
-  *workspace_bytes = mask_layout(n_seqs, q_heads, kv_heads, total_prompt, total_tokens, total_beacons).total;
+  *workspace_bytes = mask_layout(n_seqs, q_heads, kv_heads, total_tokens, total_beacons).total;
   return BC_OK;
 }
 
@@ -589,45 +613,42 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
   if ((total_prompt && (!prompt_k || !prompt_v)) || (total_tokens && (!tok_q || !tok_k || !tok_v || !out_tok)) ||
       (total_beacons && (!beacon_q || !beacon_k || !beacon_v || !out_beacon)))
     return BC_ERR_INVALID_ARG;
-  const MaskLayout l = mask_layout(n_seqs, q_heads, kv_heads, total_prompt, total_tokens, total_beacons);
+  const MaskLayout l = mask_layout(n_seqs, q_heads, kv_heads, total_tokens, total_beacons);
   if (workspace_bytes < l.total) return BC_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
 
-  // host side: tile list and per-sequence transposition jobs
+  // host side: the query tiles, heaviest (most key tiles) first
   std::vector<TileDesc> tiles;
-  std::vector<TransposeSeq> tr(3 * (size_t)n_seqs);
-  int64_t pad_p = 0, pad_t = 0, pad_b = 0, bea_row = 0;
+  int64_t bea_row = 0;
   for (int i = 0; i < n_seqs; ++i) {
     const int P = cu_prompt[i + 1] - cu_prompt[i], T = cu_tokens[i + 1] - cu_tokens[i], nb = c > 1 ? T / c : 0;
     TileDesc td = {};
     td.P = P; td.T = T; td.nb = nb;
     td.prompt_row = cu_prompt[i]; td.tok_row = cu_tokens[i]; td.bea_row = (int32_t)bea_row;
-    td.prompt_pad = (int32_t)pad_p; td.tok_pad = (int32_t)pad_t; td.bea_pad = (int32_t)pad_b;
     for (int f = 0; f < T; f += per) { td.kind = 0; td.first = f; td.count = T - f < per ? T - f : per; tiles.push_back(td); }
     for (int f = 0; f < nb; f += per) { td.kind = 1; td.first = f; td.count = nb - f < per ? nb - f : per; tiles.push_back(td); }
-    tr[i] = {cu_prompt[i], P, (int32_t)pad_p, (int32_t)pad128(P)};
-    tr[n_seqs + i] = {cu_tokens[i], T, (int32_t)pad_t, (int32_t)pad128(T)};
-    tr[2 * n_seqs + i] = {(int32_t)bea_row, nb, (int32_t)pad_b, (int32_t)pad128(nb)};
-    pad_p += pad128(P); pad_t += pad128(T); pad_b += pad128(nb); bea_row += nb;
+    bea_row += nb;
   }
-  if ((int64_t)tiles.size() > l.n_tiles || pad_p > l.prompt_cols || pad_t > l.tok_cols || pad_b > l.bea_cols)
-    return BC_ERR_INVALID_ARG;
-  if (pad_p > 0x7fffffff || pad_t > 0x7fffffff || pad_b > 0x7fffffff) return BC_ERR_UNSUPPORTED;  // 32-bit column offsets
+  if ((int64_t)tiles.size() > l.n_tiles) return BC_ERR_INVALID_ARG;
   if (tiles.empty()) return BC_OK;
+  if ((int64_t)tiles.size() * kv_heads > 0x7fffffff) return BC_ERR_UNSUPPORTED;
+  // Long sequences first; inside a sequence the query tiles with the most key tiles first.  The blocks
+  // running at any moment then share one or two sequences' K and V in L2, and the last rounds are light.
+  std::stable_sort(tiles.begin(), tiles.end(), [c](const TileDesc& x, const TileDesc& y) {
+    const int64_t lx = (int64_t)x.P + x.T, ly = (int64_t)y.P + y.T;
+    if (lx != ly) return lx > ly;
+    if (x.tok_row != y.tok_row) return x.tok_row < y.tok_row;
+    return make_plan(x, c).N > make_plan(y, c).N;
+  });
   cudaError_t e = cudaMemcpyAsync(ws + l.tiles, tiles.data(), tiles.size() * sizeof(TileDesc), cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(ws + l.seqs3, tr.data(), tr.size() * sizeof(TransposeSeq), cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemsetAsync(ws + l.status, 0, 4, s);
-  // the copies above read pageable host memory: they have been staged when the calls return
+  // the copy above reads pageable host memory: it has been staged when the call returns
   if (e != cudaSuccess) return BC_ERR_CUDA;
-  const TransposeSeq* dtr = reinterpret_cast<const TransposeSeq*>(ws + l.seqs3);
-  auto vt = [&](size_t off) { return reinterpret_cast<__nv_bfloat16*>(ws + off); };
-  if (total_prompt) k_transpose_v<<<dim3(n_seqs, kv_heads, 8), 256, 0, s>>>((const __nv_bfloat16*)prompt_v, vt(l.vt_prompt), dtr, kv_heads, l.prompt_cols);
-  if (total_tokens) k_transpose_v<<<dim3(n_seqs, kv_heads, 8), 256, 0, s>>>((const __nv_bfloat16*)tok_v, vt(l.vt_tok), dtr + n_seqs, kv_heads, l.tok_cols);
-  if (total_beacons) k_transpose_v<<<dim3(n_seqs, kv_heads, 8), 256, 0, s>>>((const __nv_bfloat16*)beacon_v, vt(l.vt_bea), dtr + 2 * n_seqs, kv_heads, l.bea_cols);
 
   MaskArgs a;
   a.tiles = reinterpret_cast<const TileDesc*>(ws + l.tiles);
+  a.n_items = (int32_t)tiles.size() * kv_heads;
   a.out_tok = (__nv_bfloat16*)out_tok; a.out_bea = (__nv_bfloat16*)out_beacon;
   a.status = reinterpret_cast<int32_t*>(ws + l.status);
   a.Hq = q_heads; a.Hkv = kv_heads; a.G = G; a.c = c; a.rows_per_tile = per;
@@ -642,11 +663,12 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
             map_3d(&maps.k_prompt, prompt_k ? prompt_k : dummy, kv_heads, total_prompt, 1, kTile) &&
             map_3d(&maps.k_tok, tok_k ? tok_k : dummy, kv_heads, total_tokens, 1, kTile) &&
             map_3d(&maps.k_bea, beacon_k ? beacon_k : dummy, kv_heads, total_beacons, 1, kTile) &&
-            map_2d(&maps.vt_prompt, ws + l.vt_prompt, l.prompt_cols, (int64_t)kv_heads * kD) &&
-            map_2d(&maps.vt_tok, ws + l.vt_tok, l.tok_cols, (int64_t)kv_heads * kD) &&
-            map_2d(&maps.vt_bea, ws + l.vt_bea, l.bea_cols, (int64_t)kv_heads * kD);
+            map_3d(&maps.v_prompt, prompt_v ? prompt_v : dummy, kv_heads, total_prompt, 1, kTile) &&
+            map_3d(&maps.v_tok, tok_v ? tok_v : dummy, kv_heads, total_tokens, 1, kTile) &&
+            map_3d(&maps.v_bea, beacon_v ? beacon_v : dummy, kv_heads, total_beacons, 1, kTile);
   if (!ok) return BC_ERR_CUDA;
-  k_mask_attn<<<dim3((unsigned)tiles.size(), kv_heads), kThreads, smem_bytes, s>>>(a, maps);
+  const int grid = a.n_items < 2 * sm_count() ? a.n_items : 2 * sm_count();   // two resident blocks per SM
+  k_mask_attn<<<grid, kThreads, smem_bytes, s>>>(a, maps);
   return cudaGetLastError() == cudaSuccess ? BC_OK : BC_ERR_CUDA;
 }
 
@@ -654,7 +676,7 @@ bc_status bc_mask_attn_status(const void* workspace, int32_t n_seqs, int32_t q_h
                               int64_t total_prompt, int64_t total_tokens, int64_t total_beacons, void* stream,
                               int32_t* code) {
   if (!workspace || !code) return BC_ERR_INVALID_ARG;
-  const MaskLayout l = mask_layout(n_seqs, q_heads, kv_heads, total_prompt, total_tokens, total_beacons);
+  const MaskLayout l = mask_layout(n_seqs, q_heads, kv_heads, total_tokens, total_beacons);
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BC_ERR_CUDA;
   if (cudaMemcpy(code, static_cast<const uint8_t*>(workspace) + l.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return BC_ERR_CUDA;
   return BC_OK;

@@ -206,6 +206,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
       "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
       : "memory");
 }
+__device__ __forceinline__ bool elect_one() {   // true in exactly one lane of a converged warp
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void mbar_arrive_cta(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -233,7 +238,8 @@ __device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity,
 // engine one tile ahead: K_{n+1} is requested as soon as S_n exists (the K buffer is free), V_{n+1} as
 // soon as O += P_n V_n has completed (the V buffer is free), so their latency hides behind the softmax
 // and the products; the products of the block's neighbour on the SM fill the tensor pipe meanwhile.
-// Q K_{n+1}^T overwrites P_n, so it is issued only after P_n V_n has completed.  The tile stream runs
+// Q K_{n+1}^T overwrites P_n; it is issued right behind P_n V_n, and the tensor pipe, which runs one
+// block's products in issue order, starts it only when P_n has been read.  The tile stream runs
 // on across work items: after an item's last S the next item's Q and first K are requested, and its
 // first product into O waits until the rows have read the finished O.
 //
@@ -252,7 +258,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
   volatile int* s_fail = &s_fail_word;
   const uint32_t bar_k = smem_addr(&s_bars[0]), bar_v = bar_k + 8, bar_s = bar_k + 16, bar_p = bar_k + 24, bar_o = bar_k + 32,
                  bar_f = bar_k + 40, bar_e = bar_k + 48;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, warp = tid >> 5;
   const int G = a.G, Hq = a.Hq, Hkv = a.Hkv, c = a.c;
 
   if (tid == 0) {
@@ -289,8 +295,10 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
 
   if (warp == kRowThreads / 32) {
     // ======================================= control warp ===========================================
+    // All 32 lanes walk the loop and the waits together, so that loop state and the matrix descriptors
+    // are warp-uniform; one elected lane issues the copies and the products.
     int item = item_of(0);
-    if (lane == 0 && item >= 0) {
+    if (item >= 0) {
       auto issue_q = [&](const TileDesc& td, int kvh) {
         // rows of Q beyond the tile's tokens belong to the next sequence or are zero-filled: they are never
         // visible (their outputs are not written and they contribute to no other row)
@@ -314,28 +322,33 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
         tma_3d(sV, vm, 0, kvh, row, bar_v);
         tma_3d(sV + kTile * 128, vm, 64, kvh, row, bar_v);
       };
-      auto qk = [&]() {
+      const uint64_t dQ = umma_desc(sQ), dK = umma_desc(sK), dV = umma_desc_nmajor(sV);
+      auto qk = [&]() {   // descriptor start addresses advance in 16-byte units
 #pragma unroll
         for (int kk = 0; kk < kD / 16; ++kk) {
-          const uint32_t off = (uint32_t)((kk >> 2) * (kTile * 128) + (kk & 3) * 32);
-          umma(tS, umma_desc(sQ + off), umma_desc(sK + off), kk > 0);
+          const uint64_t off = (uint64_t)(((kk >> 2) * (kTile * 128) + (kk & 3) * 32) >> 4);
+          umma(tS, dQ + off, dK + off, kk > 0);
         }
       };
+      auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait_or_fail(bar, parity, s_fail)); };
       const uint32_t q_bytes = (uint32_t)(box_rows * kD * 2);
       TileDesc td = a.tiles[item / Hkv];
       int kvh = item % Hkv;
       TilePlan pl = make_plan(td, c);
-      mbar_expect_tx(bar_k, q_bytes + (uint32_t)kOperandBytes);
-      issue_q(td, kvh);
-      issue_k(td, pl, kvh, 0);
-      issue_v(td, pl, kvh, 0);
+      if (elect_one()) {
+        mbar_expect_tx(bar_k, q_bytes + (uint32_t)kOperandBytes);
+        issue_q(td, kvh);
+        issue_k(td, pl, kvh, 0);
+        issue_v(td, pl, kvh, 0);
+      }
+      __syncwarp();
       uint32_t ph_k = 0, ph_v = 0, ph_o = 0, t = 0, e = 0;
-      bool ok = mbar_wait_or_fail(bar_k, ph_k, s_fail);
+      bool ok = wait_all(bar_k, ph_k);
       ph_k ^= 1;
       if (ok) {
         tc_fence_after();
-        qk();
-        umma_commit(bar_s);
+        if (elect_one()) { qk(); umma_commit(bar_s); }
+        __syncwarp();
       }
       for (int r = 0; ok; ++r, ++e) {
         const int nitem = item_of(r + 1);
@@ -344,38 +357,47 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
         int nkvh = 0;
         if (nitem >= 0) { ntd = a.tiles[nitem / Hkv]; nkvh = nitem % Hkv; npl = make_plan(ntd, c); }
         for (int n = 0; n < pl.N && ok; ++n, ++t) {
-          ok = mbar_wait_or_fail(bar_s, t & 1u, s_fail);                     // S exists: the K buffer is free
+          ok = wait_all(bar_s, t & 1u);                                        // S exists: the K buffer is free
           if (!ok) break;
           const bool last = n + 1 == pl.N;
-          if (!last) {
-            mbar_expect_tx(bar_k, (uint32_t)kOperandBytes);
-            issue_k(td, pl, kvh, n + 1);
-          } else if (nitem >= 0) {                                            // ... and so is the Q buffer
-            mbar_expect_tx(bar_k, q_bytes + (uint32_t)kOperandBytes);
-            issue_q(ntd, nkvh);
-            issue_k(ntd, npl, nkvh, 0);
+          const bool more = !last || nitem >= 0;                               // another tile follows, here or in the next item
+          if (more && elect_one()) {
+            if (!last) {
+              mbar_expect_tx(bar_k, (uint32_t)kOperandBytes);
+              issue_k(td, pl, kvh, n + 1);
+            } else {                                                           // ... and so is the Q buffer
+              mbar_expect_tx(bar_k, q_bytes + (uint32_t)kOperandBytes);
+              issue_q(ntd, nkvh);
+              issue_k(ntd, npl, nkvh, 0);
+            }
           }
-          ok = mbar_wait_or_fail(bar_p, t & 1u, s_fail) && mbar_wait_or_fail(bar_v, ph_v, s_fail);
+          __syncwarp();
+          ok = wait_all(bar_p, t & 1u) && wait_all(bar_v, ph_v);
           ph_v ^= 1;
-          if (ok && n == 0 && e > 0) ok = mbar_wait_or_fail(bar_e, (e - 1) & 1u, s_fail);   // the rows have read the last O
+          if (ok && n == 0 && e > 0) ok = wait_all(bar_e, (e - 1) & 1u);       // the rows have read the last O
+          if (ok && more) { ok = wait_all(bar_k, ph_k); ph_k ^= 1; }           // the next K (and Q) has landed
           if (!ok) break;
           tc_fence_after();
+          if (elect_one()) {
 #pragma unroll
-          for (int kk = 0; kk < kTile / 16; ++kk)                             // O += P V, 16 keys at a time
-            umma_ts(tO, tP + (uint32_t)(kk * 8), umma_desc_nmajor(sV + (uint32_t)(kk * 16 * 128)), (n > 0 || kk > 0) ? 1u : 0u);
-          if (last) umma_commit(bar_f);
-          if (!last || nitem >= 0) {
-            umma_commit(bar_o);
-            ok = mbar_wait_or_fail(bar_o, ph_o, s_fail);                      // V buffer and P are free
+            for (int kk = 0; kk < kTile / 16; ++kk)                             // O += P V, 16 keys at a time
+              umma_ts(tO, tP + (uint32_t)(kk * 8), dV + (uint64_t)((kk * 16 * 128) >> 4), (n > 0 || kk > 0) ? 1u : 0u);
+            if (last) umma_commit(bar_f);
+            if (more) {
+              umma_commit(bar_o);
+              // The next S overwrites P: the tensor pipe runs one block's products in the order they were
+              // issued, so it starts only after the product above has read P.
+              qk();
+              umma_commit(bar_s);
+            }
+          }
+          __syncwarp();
+          if (more) {
+            ok = wait_all(bar_o, ph_o);                                         // the V buffer is free
             ph_o ^= 1;
             if (!ok) break;
-            if (!last) issue_v(td, pl, kvh, n + 1); else issue_v(ntd, npl, nkvh, 0);
-            ok = mbar_wait_or_fail(bar_k, ph_k, s_fail);
-            ph_k ^= 1;
-            if (!ok) break;
-            tc_fence_after();
-            qk();
-            umma_commit(bar_s);
+            if (elect_one()) { if (!last) issue_v(td, pl, kvh, n + 1); else issue_v(ntd, npl, nkvh, 0); }
+            __syncwarp();
           }
         }
         if (nitem < 0) break;

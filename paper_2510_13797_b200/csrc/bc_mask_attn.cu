@@ -258,7 +258,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
   volatile int* s_fail = &s_fail_word;
   const uint32_t bar_k = smem_addr(&s_bars[0]), bar_v = bar_k + 8, bar_s = bar_k + 16, bar_p = bar_k + 24, bar_o = bar_k + 32,
                  bar_f = bar_k + 40, bar_e = bar_k + 48;
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = a.G, Hq = a.Hq, Hkv = a.Hkv, c = a.c;
 
   if (tid == 0) {
@@ -330,7 +330,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
           umma(tS, dQ + off, dK + off, kk > 0);
         }
       };
-      auto wait_all = [&](uint32_t bar, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait_or_fail(bar, parity, s_fail)); };
+      // one lane polls, the warp takes its answer
+      auto wait_all = [&](uint32_t bar, uint32_t parity) {
+        int ok1 = 1;
+        if (lane == 0) ok1 = mbar_wait_or_fail(bar, parity, s_fail) ? 1 : 0;
+        return __shfl_sync(0xffffffffu, ok1, 0) != 0;
+      };
       const uint32_t q_bytes = (uint32_t)(box_rows * kD * 2);
       TileDesc td = a.tiles[item / Hkv];
       int kvh = item % Hkv;
@@ -372,10 +377,12 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
             }
           }
           __syncwarp();
-          ok = wait_all(bar_p, t & 1u) && wait_all(bar_v, ph_v);
+          // everything the products below need besides P is waited for while the rows are busy
+          ok = wait_all(bar_v, ph_v);
           ph_v ^= 1;
           if (ok && n == 0 && e > 0) ok = wait_all(bar_e, (e - 1) & 1u);       // the rows have read the last O
           if (ok && more) { ok = wait_all(bar_k, ph_k); ph_k ^= 1; }           // the next K (and Q) has landed
+          ok = ok && wait_all(bar_p, t & 1u);
           if (!ok) break;
           tc_fence_after();
           if (elect_one()) {

@@ -49,6 +49,13 @@ def test_mask_form_matches_oracle(plens, tlens, c, Hq, Hkv):
     run_case(plens, tlens, c, Hq, Hkv, seed=3)
 
 
+def test_mask_form_many_rounds():
+    """More work items (query tiles x KV heads) than the persistent grid holds at once, so every block
+    walks several items in both directions of the hand-out, with the next item's tiles requested while
+    the current item's output is written; ragged lengths, an empty prompt, one-tile items."""
+    run_case([40, 0, 100, 64, 7], [640, 512, 700, 333, 3], 4, 32, 8, seed=11)
+
+
 def test_mask_form_sharp_logits():
     """Unscaled N(0,1) keys give logits with standard deviation ~ 1 after the softmax scale; keys
     scaled by 4 make the rows sharply peaked, which exercises the running maximum across tiles."""

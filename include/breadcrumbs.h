@@ -251,8 +251,9 @@ BC_API bc_status bc_compress_step_host(bc_cache* cache, int32_t layer, const int
  * [sum T, q_heads, head_dim] and out_beacon [sum nb, q_heads, head_dim], bf16 rounded to nearest
  * even from fp32 (accumulation in fp32, softmax weights rounded to bf16 before the second product).
  * head_dim must be 128 and q_heads / kv_heads <= 16 (else BC_ERR_UNSUPPORTED); sm_scale > 0.  `workspace`: device
- * memory of at least bc_mask_attn_query_bytes bytes, 256-byte aligned (it receives the tile list
- * and a transposed copy of V).  Asynchronous on `stream`; the two host arrays are read before the
+ * memory of at least bc_mask_attn_query_bytes bytes, 256-byte aligned (it receives the list of
+ * query tiles and the status word).  All inputs must be finite: rows of K and V next to a sequence's
+ * own are read along with it and enter the products with weight zero.  Asynchronous on `stream`; the two host arrays are read before the
  * call returns (pageable host memory is staged by the copy, so do not call this inside a stream
  * capture).  One call at a time per workspace.  A bounded device-side wait that expires is reported
  * by bc_mask_attn_status as BC_ERR_TIMEOUT (the outputs are then incomplete). */

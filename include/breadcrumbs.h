@@ -224,7 +224,13 @@ BC_API bc_status bc_seq_close(bc_cache* cache, const int32_t* slots, int32_t n, 
 
 /* ---- end-to-end helpers with HOST buffers (pinned memory recommended) ------------------------
  * One decode step of one layer: copies q, k, v to device staging inside `workspace`, runs
- * bc_append + bc_decode_attn, copies out back.  All asynchronous on `stream`.  n <= 512. */
+ * bc_append + bc_decode_attn, copies out back.  n <= 512.  Asynchronous: out_host is valid, and the
+ * three input buffers may be reused, once `stream` has passed the call.  The inputs are copied on a
+ * stream the cache owns (created by the first such call, which therefore must not sit inside a
+ * stream capture) into one of two staging buffers, so a call's inputs travel while the previous
+ * call's kernels run: they are read from the moment of the call, not in the order of `stream` --
+ * they must be complete in host memory when the call is made.  If the three buffers are one packed
+ * block k | v | q (v_host == k_host + bytes(k), q_host == v_host + bytes(v)) a single copy moves them. */
 BC_API bc_status bc_decode_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                               const void* q_host, const void* k_host, const void* v_host,
                               void* out_host, float sm_scale, void* stream);

@@ -135,7 +135,7 @@ class Cache:
         self.out_dtype = torch.float32 if flags & BC_FLAG_OUT_F32 else torch.bfloat16
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and lib is not None:   # at interpreter exit the module may be gone already
             lib().bc_cache_destroy(self.handle)
             self.handle = None
 

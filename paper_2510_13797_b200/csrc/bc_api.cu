@@ -32,8 +32,8 @@ MetaLayout meta_layout(const bc_config& c) {
 }
 
 struct WorkLayout {
-  size_t append_row, append_pos, compress_row, compress_pos, tickets, book_flag, part_ml, part_o, stage_q, stage_k,
-      stage_v, stage_out, total;
+  size_t append_row, append_pos, compress_row, compress_pos, tickets, book_flag, part_ml, part_o, stage_in[2], stage_out,
+      total;
 };
 WorkLayout work_layout(const bc_config& c) {
   WorkLayout l;
@@ -46,9 +46,8 @@ WorkLayout work_layout(const bc_config& c) {
   l.book_flag = take(4);
   l.part_ml = take(pieces * c.q_heads * 2 * 4);
   l.part_o = take(pieces * c.q_heads * c.head_dim * 4);
-  l.stage_q = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 2);
-  l.stage_k = take((size_t)BC_MAX_ATTN_BATCH * c.kv_heads * c.head_dim * 2);
-  l.stage_v = take((size_t)BC_MAX_ATTN_BATCH * c.kv_heads * c.head_dim * 2);
+  // host-buffer entry points: two input staging buffers, each k | v | q packed for the call's batch
+  for (int b = 0; b < 2; ++b) l.stage_in[b] = take((size_t)BC_MAX_ATTN_BATCH * (c.q_heads + 2 * c.kv_heads) * c.head_dim * 2);
   l.stage_out = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
   l.total = o;
   return l;
@@ -96,6 +95,11 @@ struct bc_cache {
   // profiling
   std::vector<cudaEvent_t> ev;
   int prof_cap, prof_used;
+  // host-buffer entry points: inputs are copied on a stream of their own into alternating staging buffers
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_in[2] = {nullptr, nullptr};    // the copies into staging buffer b have been issued up to here
+  cudaEvent_t ev_used[2] = {nullptr, nullptr};  // the kernels reading staging buffer b have been issued up to here
+  int stage_next = 0;
 };
 
 namespace {
@@ -275,6 +279,11 @@ bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* wo
 bc_status bc_cache_destroy(bc_cache* c) {
   if (!c) return BC_ERR_INVALID_ARG;
   for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
+  for (int b = 0; b < 2; ++b) {
+    if (c->ev_in[b]) cudaEventDestroy(c->ev_in[b]);
+    if (c->ev_used[b]) cudaEventDestroy(c->ev_used[b]);
+  }
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   delete c;
   return BC_OK;
 }
@@ -401,23 +410,61 @@ bc_status bc_seq_close(bc_cache* c, const int32_t* slots, int32_t n, void* strea
   return BC_OK;
 }
 
+namespace {
+
+// Stages k, v, q of a host-buffer step: the copies run on the cache's own copy stream, so the next
+// step's inputs travel while this step's kernels run; `s` waits for them before the kernels.
+// Returns the staging buffer used; record ev_used[buf] on `s` after the kernels that read it.
+bc_status stage_inputs(bc_cache* c, int32_t n, const void* q_host, const void* k_host, const void* v_host, cudaStream_t s,
+                       int* buf_out, void** dq, void** dk, void** dv) {
+  if (!c->copy_stream) {   // first host-buffer call on this cache
+    BC_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+    for (int b = 0; b < 2; ++b) {
+      BC_CUDA(c, cudaEventCreateWithFlags(&c->ev_in[b], cudaEventDisableTiming));
+      BC_CUDA(c, cudaEventCreateWithFlags(&c->ev_used[b], cudaEventDisableTiming));
+    }
+  }
+  const int buf = c->stage_next;
+  c->stage_next ^= 1;
+  const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+  uint8_t* base = c->work + c->wl.stage_in[buf];
+  *dk = base; *dv = base + kb; *dq = base + 2 * kb;
+  // the buffer's previous readers (two steps ago) must be done; an event never recorded does not block
+  BC_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_used[buf], 0));
+  const uint8_t *kh = static_cast<const uint8_t*>(k_host), *vh = static_cast<const uint8_t*>(v_host),
+                *qh = static_cast<const uint8_t*>(q_host);
+  if (vh == kh + kb && qh == vh + kb) {   // one packed host buffer k | v | q: one copy
+    BC_CUDA(c, cudaMemcpyAsync(base, kh, 2 * kb + qb, cudaMemcpyHostToDevice, c->copy_stream));
+  } else {
+    BC_CUDA(c, cudaMemcpyAsync(*dk, kh, kb, cudaMemcpyHostToDevice, c->copy_stream));
+    BC_CUDA(c, cudaMemcpyAsync(*dv, vh, kb, cudaMemcpyHostToDevice, c->copy_stream));
+    BC_CUDA(c, cudaMemcpyAsync(*dq, qh, qb, cudaMemcpyHostToDevice, c->copy_stream));
+  }
+  BC_CUDA(c, cudaEventRecord(c->ev_in[buf], c->copy_stream));
+  BC_CUDA(c, cudaStreamWaitEvent(s, c->ev_in[buf], 0));
+  *buf_out = buf;
+  return BC_OK;
+}
+
+}  // namespace
+
 bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q_host,
                               const void* k_host, const void* v_host, void* out_host, float sm_scale, void* stream) {
   bc_status st = check_batch(c, layer, slots, n);
   if (st) return st;
   if (n > BC_MAX_ATTN_BATCH || !q_host || !k_host || !v_host || !out_host) return BC_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+  const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
-  void *dq = c->work + c->wl.stage_q, *dk = c->work + c->wl.stage_k, *dv = c->work + c->wl.stage_v,
-       *dout = c->work + c->wl.stage_out;
-  BC_CUDA(c, cudaMemcpyAsync(dk, k_host, kb, cudaMemcpyHostToDevice, s));
-  BC_CUDA(c, cudaMemcpyAsync(dv, v_host, kb, cudaMemcpyHostToDevice, s));
-  BC_CUDA(c, cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s));
+  void *dq, *dk, *dv, *dout = c->work + c->wl.stage_out;
+  int buf;
+  st = stage_inputs(c, n, q_host, k_host, v_host, s, &buf, &dq, &dk, &dv);
+  if (st) return st;
   st = bc_append(c, layer, slots, n, dk, dv, stream);
   if (st) return st;
   st = attn_impl(c, layer, slots, n, dq, dout, sm_scale, nullptr, nullptr, s);
   if (st) return st;
+  BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
   BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
   return BC_OK;
 }
@@ -428,17 +475,17 @@ bc_status bc_compress_step_host(bc_cache* c, int32_t layer, const int32_t* slots
   if (st) return st;
   if (n > BC_MAX_ATTN_BATCH || !bq_host || !bk_host || !bv_host || !out_host) return BC_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
-  const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+  const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
-  void *dq = c->work + c->wl.stage_q, *dk = c->work + c->wl.stage_k, *dv = c->work + c->wl.stage_v,
-       *dout = c->work + c->wl.stage_out;
-  BC_CUDA(c, cudaMemcpyAsync(dk, bk_host, kb, cudaMemcpyHostToDevice, s));
-  BC_CUDA(c, cudaMemcpyAsync(dv, bv_host, kb, cudaMemcpyHostToDevice, s));
-  BC_CUDA(c, cudaMemcpyAsync(dq, bq_host, qb, cudaMemcpyHostToDevice, s));
+  void *dq, *dk, *dv, *dout = c->work + c->wl.stage_out;
+  int buf;
+  st = stage_inputs(c, n, bq_host, bk_host, bv_host, s, &buf, &dq, &dk, &dv);
+  if (st) return st;
   st = attn_impl(c, layer, slots, n, dq, dout, sm_scale, dk, dv, s);
   if (st) return st;
   st = bc_compress(c, layer, slots, n, dk, dv, stream);
   if (st) return st;
+  BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
   BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
   return BC_OK;
 }

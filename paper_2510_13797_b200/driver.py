@@ -89,8 +89,19 @@ class DecodeDriver:
         """The same step through the host-buffer entry points (H2D of q,k,v and D2H of out inside)."""
         if self.h is None:
             pin = lambda t: t.cpu().pin_memory()
-            self.h = dict(q=pin(self.q), k=pin(self.k), v=pin(self.v), bq=pin(self.bq), bk=pin(self.bk),
-                          bv=pin(self.bv), out=pin(self.out), out_b=pin(self.out_b))
+
+            def packed(k, v, q):
+                """Per ring slot one pinned block k | v | q, which the library moves with a single copy."""
+                ks, vs, qs = [], [], []
+                for j in range(k.shape[0]):
+                    nk, nq = k[j].numel(), q[j].numel()
+                    flat = torch.empty(2 * nk + nq, dtype=k.dtype).pin_memory()
+                    flat[:nk] = k[j].reshape(-1).cpu(); flat[nk:2 * nk] = v[j].reshape(-1).cpu(); flat[2 * nk:] = q[j].reshape(-1).cpu()
+                    ks.append(flat[:nk].view(k[j].shape)); vs.append(flat[nk:2 * nk].view(v[j].shape)); qs.append(flat[2 * nk:].view(q[j].shape))
+                return ks, vs, qs
+            hk, hv, hq = packed(self.k, self.v, self.q)
+            hbk, hbv, hbq = packed(self.bk, self.bv, self.bq)
+            self.h = dict(q=hq, k=hk, v=hv, bq=hbq, bk=hbk, bv=hbv, out=pin(self.out), out_b=pin(self.out_b))
         c, j, h = self.cache, self.t % self.ring, self.h
         c.bc_decode_step_host(0, self.slots, h["q"][j], h["k"][j], h["v"][j], h["out"], self.w.sm_scale)
         self.t += 1

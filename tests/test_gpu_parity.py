@@ -377,3 +377,64 @@ def test_fused_decode_step_refusals_and_block_counts():
     pair.check_state()
     for s in (0, 1, 2):
         pair.check_content(0, s)
+
+
+def test_host_buffer_steps_back_to_back_packed():
+    """Host-buffer steps issued without a synchronisation in between, each with its inputs in one
+    packed pinned block k | v | q (moved by a single copy): the copies of a step run on the cache's
+    copy stream while the previous step's kernels run, in alternating staging buffers.  Every step's
+    output, read after one synchronisation at the end, must match the oracle."""
+    Hkv, G, D, ps, c = 2, 4, 128, 16, 4
+    n, plens = 4, [300, 7, 90, 513]
+    pair = Pair(1, Hkv, Hkv * G, D, ps, max_seqs=n, num_pages=128, max_pages_per_seq=48)
+    g = _gen(23)
+    slots = list(range(n))
+    pair.open(slots, plens, [c] * n)
+    pair.prefill(0, slots, plens, randn_bf16(g, (sum(plens), Hkv, D), DEV), randn_bf16(g, (sum(plens), Hkv, D), DEV))
+    sl = torch.tensor(slots, dtype=torch.int32, device=DEV)
+
+    def packed(k, v, q):
+        nk, nq = k.numel(), q.numel()
+        flat = torch.empty(2 * nk + nq, dtype=torch.bfloat16).pin_memory()
+        flat[:nk], flat[nk:2 * nk], flat[2 * nk:] = k.reshape(-1).cpu(), v.reshape(-1).cpu(), q.reshape(-1).cpu()
+        return flat[:nk].view(k.shape), flat[nk:2 * nk].view(v.shape), flat[2 * nk:].view(q.shape)
+
+    steps, outs, refs = 11, [], []
+    inputs = []
+    for step in range(1, steps + 1):
+        k, v, q = randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv * G, D), DEV)
+        beacon = None
+        if step % c == 0:
+            beacon = (randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv * G, D), DEV))
+        inputs.append((k, v, q, beacon))
+    torch.cuda.synchronize()
+    for k, v, q, beacon in inputs:                 # the GPU side: nothing waits between the calls
+        hk, hv, hq = packed(k, v, q)
+        out_h = torch.empty((n, Hkv * G, D), dtype=torch.bfloat16).pin_memory()
+        pair.gpu.bc_decode_step_host(0, sl, hq, hk, hv, out_h, 0.1)
+        outs.append(out_h)
+        if beacon is not None:
+            hbk, hbv, hbq = packed(*beacon)
+            out_b = torch.empty((n, Hkv * G, D), dtype=torch.bfloat16).pin_memory()
+            pair.gpu.bc_compress_step_host(0, sl, hbq, hbk, hbv, out_b, 0.1)
+            outs.append(out_b)
+    torch.cuda.synchronize()
+    for k, v, q, beacon in inputs:                 # the oracle, step by step
+        pair._append_ok = pair.model.append(slots)
+        for i, s in enumerate(slots):
+            pair.seqs[s].append(0, f64(k)[i], f64(v)[i])
+        refs.append(np.stack([pair.seqs[s].attend(0, f64(q)[i], 0.1) for i, s in enumerate(slots)]))
+        if beacon is not None:
+            bk, bv, bq = beacon
+            refs.append(np.stack([pair.seqs[s].beacon_attend(0, f64(bq)[i], f64(bk)[i], f64(bv)[i], 0.1)
+                                  for i, s in enumerate(slots)]))
+            pair.model.compress(slots)
+            for i, s in enumerate(slots):
+                pair.seqs[s].compress(0, f64(bk)[i], f64(bv)[i])
+    assert len(outs) == len(refs)
+    for j, (o, r) in enumerate(zip(outs, refs)):
+        assert_close(o, r, f"back-to-back host call {j}")
+    pair.check_state()
+    for s in slots:
+        pair.check_content(0, s)
+

@@ -254,7 +254,7 @@ BC_API bc_status bc_compress_step_host(bc_cache* cache, int32_t layer, const int
  * packed in the same order.  Device tensors, bf16: prompt_k, prompt_v [sum P, kv_heads, head_dim];
  * tok_q [sum T, q_heads, head_dim]; tok_k, tok_v [sum T, kv_heads, head_dim]; beacon_q
  * [sum nb, q_heads, head_dim]; beacon_k, beacon_v [sum nb, kv_heads, head_dim]; outputs out_tok
- * [sum T, q_heads, head_dim] and out_beacon [sum nb, q_heads, head_dim], bf16 rounded to nearest
+ * [sum T, q_heads, head_dim] and out_beacon [sum nb, q_heads, head_dim] (32-byte aligned), bf16 rounded to nearest
  * even from fp32 (accumulation in fp32, softmax weights rounded to bf16 before the second product).
  * head_dim must be 128 and q_heads / kv_heads <= 16 (else BC_ERR_UNSUPPORTED); sm_scale > 0.  `workspace`: device
  * memory of at least bc_mask_attn_query_bytes bytes, 256-byte aligned (it receives the list of

@@ -532,15 +532,17 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
         __nv_bfloat16* dst = (td.kind == 0 ? a.out_tok + (int64_t)(td.tok_row + my_idx) * Hq * kD
                                            : a.out_bea + (int64_t)(td.bea_row + my_idx) * Hq * kD) +
                              (int64_t)(kvh * G + my_head) * kD;
+        auto pack = [&](int d) {
+          const __nv_bfloat162 t = __floats2bfloat162_rn(o[d] * inv, o[d + 1] * inv);
+          return *reinterpret_cast<const uint32_t*>(&t);
+        };
+        // 32-byte stores: whole sectors, half as many store instructions as with 16-byte ones (the rows
+        // of a warp lie 256 bytes or more apart, so nothing coalesces across lanes)
 #pragma unroll
-        for (int d = 0; d < kD; d += 8) {
-          uint4 v;
-          __nv_bfloat162 t0 = __floats2bfloat162_rn(o[d] * inv, o[d + 1] * inv), t1 = __floats2bfloat162_rn(o[d + 2] * inv, o[d + 3] * inv);
-          __nv_bfloat162 t2 = __floats2bfloat162_rn(o[d + 4] * inv, o[d + 5] * inv), t3 = __floats2bfloat162_rn(o[d + 6] * inv, o[d + 7] * inv);
-          v.x = *reinterpret_cast<uint32_t*>(&t0); v.y = *reinterpret_cast<uint32_t*>(&t1);
-          v.z = *reinterpret_cast<uint32_t*>(&t2); v.w = *reinterpret_cast<uint32_t*>(&t3);
-          *reinterpret_cast<uint4*>(dst + d) = v;
-        }
+        for (int d = 0; d < kD; d += 16)
+          asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + d), "r"(pack(d)), "r"(pack(d + 2)),
+                       "r"(pack(d + 4)), "r"(pack(d + 6)), "r"(pack(d + 8)), "r"(pack(d + 10)), "r"(pack(d + 12)), "r"(pack(d + 14))
+                       : "memory");
       }
       item = nitem;
       td = ntd;
@@ -632,6 +634,7 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
     return BC_ERR_INVALID_ARG;
   if (head_dim != kD || q_heads / kv_heads > 16) return BC_ERR_UNSUPPORTED;
   if (reinterpret_cast<uintptr_t>(workspace) & 255) return BC_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(out_tok) | reinterpret_cast<uintptr_t>(out_beacon)) & 31) return BC_ERR_INVALID_ARG;   // 32-byte stores
   if (!(sm_scale > 0.f)) return BC_ERR_INVALID_ARG;  // the kernel takes row maxima before scaling
   const int G = q_heads / kv_heads, per = kTile / G;
   int64_t total_prompt = cu_prompt[n_seqs], total_tokens = cu_tokens[n_seqs], total_beacons = 0;

@@ -558,9 +558,12 @@ def report_depth(args):
         t = state["t"]; j = t % ring
         for l in range(L):
             (q, k, v), _ = ins[l]
-            cache.bc_append(l, slots, k[j], v[j])
-            if attend:
-                cache.bc_decode_attn(l, slots, q[j], out, w.sm_scale)
+            if attend and args.fused:
+                cache.bc_decode_step(l, slots, q[j], k[j], v[j], out, w.sm_scale)
+            else:
+                cache.bc_append(l, slots, k[j], v[j])
+                if attend:
+                    cache.bc_decode_attn(l, slots, q[j], out, w.sm_scale)
         state["t"] = t = t + 1
         if t % c == 0:
             m = (t // c) % 2
@@ -816,6 +819,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=32)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fused", action="store_true", help="depth workload: regular steps through bc_decode_step (append + attention in one launch per layer)")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
     ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth", "maskform", "distill", "model"],

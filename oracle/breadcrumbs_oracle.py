@@ -148,6 +148,22 @@ class SeqCache:
         if layer == len(self.cache) - 1:
             self.n_beacons += 1
 
+    # -- Algorithm 1 run over a stored trajectory -------------------------------
+    def replay(self, layer, tok_k, tok_v, beacon_k, beacon_v):
+        """The sampling loop of Algorithm 1 with the tokens given instead of sampled: every token's
+        entry is appended, and each time the window holds c of them the next stored beacon is
+        encoded and the window evicted.  tok_k, tok_v: [T, Hkv, D]; beacon_k, beacon_v:
+        [floor(T / c), Hkv, D] (ignored when c = 1).  This is the definition a one-call restore of
+        the cache has to reproduce."""
+        T = np.asarray(tok_k).shape[0]
+        m = 0
+        for i in range(T):
+            self.append(layer, tok_k[i], tok_v[i])
+            if self.c > 1 and self.window_len(layer) == self.c:
+                self.compress(layer, beacon_k[m], beacon_v[m])
+                m += 1
+        assert m == (T // self.c if self.c > 1 else 0)
+
     # -- views ----------------------------------------------------------------
     def window_len(self, layer=0):
         n = 0

@@ -15,6 +15,11 @@ include/breadcrumbs.h, written here independently with plain Python lists:
   need[i] == 0 or off[i] + need[i] <= pages free at the start of the call.
   Frees: walk the batch in order; a sequence's pages are pushed in the order
   prompt pages, beacon pages, window pages, each in ascending index.
+* restore (a stored trajectory of T generated tokens put into a freshly
+  opened sequence in one call) leaves the lengths that T appends with their
+  compressions leave (Algorithm 1: floor(T/c) beacons, T mod c window
+  entries); an item needs ceil(beacons/page) + ceil(window/page) pages and
+  receives its beacon pages first, then its window pages.
 * A failed item is a no-op for its sequence; the first failure of the store's
   lifetime is latched as (code, slot, call index); when several items of one
   call fail, the one with the lowest batch index is reported.
@@ -171,6 +176,40 @@ class PagingModel:
             s = self.seqs[slots[i]]
             self.stack.extend(s.window_pages)
             s.window_pages = []; s.window_len = 0; s.n_beacons += 1
+        return self._latch(res)
+
+    def restore(self, slots, gen_lens):
+        """Puts a stored trajectory of gen_lens[i] generated tokens into slot i, which must be open
+        and untouched since (no appends): the state Algorithm 1 is in after that many sampling
+        steps, i.e. floor(T / c) beacons and the T mod c tokens of the unfinished window (all T
+        tokens when c = 1)."""
+        self.calls += 1
+        res, needs, plan = [None] * len(slots), [], {}
+        for i, slot in enumerate(slots):
+            s = self.seqs.get(slot)
+            T = gen_lens[i]
+            if s is None:
+                res[i] = self._fail(BAD_SLOT, slot, i); continue
+            if T < 0 or s.t != 0 or s.n_beacons != 0 or s.window_len != 0:
+                res[i] = self._fail(INVALID_ARG, slot, i); continue
+            nb = T // s.c if s.c > 1 else 0
+            w = T - nb * s.c
+            if self.max_entries and nb + w > self.max_entries:
+                res[i] = self._fail(CAPACITY, slot, i); continue
+            nbp, nwp = _ceil_div(nb, self.ps), _ceil_div(w, self.ps)
+            reserved = _ceil_div(s.c, self.ps) if s.c > 1 else nwp   # the window's columns of the page table
+            if len(s.prompt_pages) + reserved + nbp > self.max_pages_per_seq:
+                res[i] = self._fail(CAPACITY, slot, i); continue
+            needs.append((i, nbp + nwp)); plan[i] = (nb, w, nbp, T)
+        granted = self._allocate(needs)
+        for i, _ in needs:
+            slot = slots[i]; s = self.seqs[slot]
+            nb, w, nbp, T = plan[i]
+            if i not in granted:
+                res[i] = self._fail(NO_PAGES, slot, i); continue
+            s.beacon_pages = granted[i][:nbp]; s.window_pages = granted[i][nbp:]
+            s.n_beacons, s.window_len, s.t = nb, w, T
+            res[i] = OK
         return self._latch(res)
 
     def close(self, slots):

@@ -320,3 +320,66 @@ def test_paging_exhaustion_and_capacity():
     m3 = PagingModel(num_pages=30, page_size=1, max_seqs=1, max_pages_per_seq=6)
     m3.open([0], [5], [1])
     assert m3.append([0]) == [OK] and m3.append([0]) == [CAPACITY]
+
+
+
+@pytest.mark.parametrize("ps,c", [(1, 2), (4, 4), (16, 8), (8, 32), (16, 1)])
+def test_paging_restore_equals_replay_counts_and_conserves_pages(ps, c):
+    """restore(T) must leave the lengths that T appends with their compressions leave (and the closed
+    form gives), hold exactly ceil(len / page) pages per segment, and conserve pages; the page ids
+    differ from a replay's (a replay recycles window pages), which is why only counts are compared."""
+    P = 37
+    for T in (0, 1, c - 1, c, c + 1, 5 * c + 3, 97):
+        a = PagingModel(num_pages=64, page_size=ps, max_seqs=2, max_pages_per_seq=64) if ps > 1 else \
+            PagingModel(num_pages=256, page_size=ps, max_seqs=2, max_pages_per_seq=256)
+        b = PagingModel(num_pages=a.num_pages, page_size=ps, max_seqs=2, max_pages_per_seq=a.max_pages_per_seq)
+        assert a.open([0], [P], [c]) == [OK] and b.open([0], [P], [c]) == [OK]
+        assert a.restore([0], [T]) == [OK]
+        for n in range(1, T + 1):
+            assert b.append([0]) == [OK]
+            if c > 1 and n % c == 0:
+                assert b.compress([0]) == [OK]
+        sa, sb = a.state(0), b.state(0)
+        for key in ("prompt_len", "n_beacons", "window_len", "c", "t"):
+            assert sa[key] == sb[key], (key, T)
+        assert sa["n_beacons"] + sa["window_len"] + P == closed_form_length(P, T, c)
+        assert len(sa["beacon_pages"]) == -(-sa["n_beacons"] // ps) and len(sa["window_pages"]) == -(-sa["window_len"] // ps)
+        owned = sa["prompt_pages"] + sa["beacon_pages"] + sa["window_pages"]
+        assert sorted(owned + a.free_list()) == list(range(a.num_pages))
+        # the restored sequence goes on like any other
+        assert a.append([0]) == [OK] and a.state(0)["window_len"] == sa["window_len"] + 1
+
+
+def test_paging_restore_order_and_failures_by_hand():
+    """Page 4, pool of 8: slot 0 (P = 4, c = 4) holds page 0, slot 1 (P = 0, c = 4) none.  restore of
+    T = 9 for slot 0 needs 1 beacon page (2 beacons) + 1 window page (1 token): pages 1 and 2, beacon
+    page first.  A second restore of the same slot is refused; T = 40 for slot 1 needs 3 + 0 pages
+    and gets 3, 4, 5; a further item that needs more than what is left is refused with NO_PAGES and
+    changes nothing."""
+    m = PagingModel(num_pages=8, page_size=4, max_seqs=3, max_pages_per_seq=8)
+    assert m.open([0, 1, 2], [4, 0, 0], [4, 4, 4]) == [OK, OK, OK]
+    assert m.restore([0], [9]) == [OK]
+    s = m.state(0)
+    assert (s["beacon_pages"], s["window_pages"], s["n_beacons"], s["window_len"], s["t"]) == ([1], [2], 2, 1, 9)
+    assert m.restore([0], [3]) == ["INVALID_ARG"]
+    assert m.first_error == ("INVALID_ARG", 0, 3)
+    assert m.restore([1, 2], [40, 100]) == [OK, "NO_PAGES"]
+    assert m.state(1)["beacon_pages"] == [3, 4, 5] and m.state(1)["window_pages"] == []
+    assert m.state(2)["t"] == 0 and m.free_list() == [7, 6]
+
+
+def test_replay_is_algorithm1_stepwise():
+    """SeqCache.replay against the closed form of the live set (which entries survive T steps)."""
+    rng = np.random.RandomState(5)
+    for c, T in ((4, 11), (8, 8), (1, 6), (16, 5)):
+        s = SeqCache(1, c)
+        s.prefill(0, rng.standard_normal((3, 1, 4)), rng.standard_normal((3, 1, 4)))
+        tk, tv = rng.standard_normal((T, 1, 4)), rng.standard_normal((T, 1, 4))
+        nb = T // c if c > 1 else 0
+        bk, bv = rng.standard_normal((nb, 1, 4)), rng.standard_normal((nb, 1, 4))
+        s.replay(0, tk, tv, bk, bv)
+        assert s.live_ids(0) == closed_form_live_ids(3, T, c)
+        K, _ = s.entries(0)
+        w = T - nb * c
+        assert np.array_equal(K[3:3 + nb], bk) and np.array_equal(K[3 + nb:], tk[T - w:])
+

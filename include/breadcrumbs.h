@@ -144,6 +144,26 @@ BC_API bc_status bc_prefill(bc_cache* cache, int32_t layer, const int32_t* slots
                      const int32_t* cu_prompt_lens, int32_t n, int32_t total_tokens,
                      const void* k, const void* v, void* stream);
 
+/* Algorithm 1 run over a stored trajectory, in one call per layer: each of n sequences that were
+ * opened (and whose prompt is, or will be, stored by bc_prefill) but have received no entry yet gets
+ * the state the sampling loop is in after its T_i generated tokens -- its floor(T_i / c) beacons and
+ * the T_i mod c tokens of its unfinished window (all T_i tokens when c = 1); the evicted tokens are
+ * never copied.  This is what lets a trajectory scored in one pass (Section 3.2, the mask form,
+ * whose inputs have the same packing) be continued by the decode loop.
+ * cu_tokens: device int32[n + 1], prefix sums of T_i.  tok_k, tok_v: device bf16
+ * [total_tokens, kv_heads, head_dim], the generated tokens' entries, sequences back to back;
+ * beacon_k, beacon_v: device bf16 [total_beacons, kv_heads, head_dim], sequence i's floor(T_i / c)
+ * beacons back to back in batch order (an item whose slot is not open has none).  total_tokens and
+ * total_beacons (host) bound what is read.  Per-layer ordering as for bc_append: layer 0 first (it
+ * does the bookkeeping: beacon pages, then window pages, per item in batch order), then 1 .. layers - 1
+ * with the same `slots` and `cu_tokens`.  Device-side failures (latched): BC_ERR_BAD_SLOT (not open),
+ * BC_ERR_INVALID_ARG (the sequence has entries already, or T_i < 0), BC_ERR_CAPACITY, BC_ERR_NO_PAGES;
+ * a failed item is left untouched. */
+BC_API bc_status bc_restore(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
+                            const int32_t* cu_tokens, int32_t total_tokens, int32_t total_beacons,
+                            const void* tok_k, const void* tok_v, const void* beacon_k,
+                            const void* beacon_v, void* stream);
+
 /* Algorithm 1, sampling step (the forward pass of a token adds its entry to the cache): appends one generated
  * token's K/V entry to the live window of each of n sequences.  A window page is allocated when
  * the window length is a multiple of page_size.  k, v: device [n, kv_heads, head_dim]. */

@@ -55,6 +55,7 @@ SYMBOLS = {
     "bc_cache_destroy": (_I32, [_P]),
     "bc_seq_open": (_I32, [_P, _P, _P, _P, _I32, _P]),
     "bc_prefill": (_I32, [_P, _I32, _P, _P, _I32, _I32, _P, _P, _P]),
+    "bc_restore": (_I32, [_P, _I32, _P, _I32, _P, _I32, _I32, _P, _P, _P, _P, _P]),
     "bc_append": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
     "bc_decode_attn": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
     "bc_decode_step": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P]),
@@ -149,6 +150,10 @@ class Cache:
     def bc_prefill(self, layer, slots, cu_prompt_lens, total_tokens, k, v, stream=None):
         _check(lib().bc_prefill(self.handle, layer, _ptr(slots), _ptr(cu_prompt_lens), slots.numel(), total_tokens,
                                 _ptr(k), _ptr(v), _stream(stream)), "bc_prefill")
+
+    def bc_restore(self, layer, slots, cu_tokens, total_tokens, total_beacons, tok_k, tok_v, beacon_k, beacon_v, stream=None):
+        _check(lib().bc_restore(self.handle, layer, _ptr(slots), slots.numel(), _ptr(cu_tokens), total_tokens, total_beacons,
+                                _ptr(tok_k), _ptr(tok_v), _ptr(beacon_k), _ptr(beacon_v), _stream(stream)), "bc_restore")
 
     def bc_append(self, layer, slots, k, v, stream=None):
         _check(lib().bc_append(self.handle, layer, _ptr(slots), slots.numel(), _ptr(k), _ptr(v), _stream(stream)),

@@ -32,7 +32,7 @@ MetaLayout meta_layout(const bc_config& c) {
 }
 
 struct WorkLayout {
-  size_t append_row, append_pos, compress_row, compress_pos, tickets, book_flag, part_ml, part_o, stage_in[2], stage_out,
+  size_t append_row, append_pos, compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, stage_in[2], stage_out,
       total;
 };
 WorkLayout work_layout(const bc_config& c) {
@@ -42,6 +42,7 @@ WorkLayout work_layout(const bc_config& c) {
   const size_t seq = (size_t)c.max_seqs * 4;
   const size_t pieces = BC_MAX_ATTN_CTAS + BC_MAX_ATTN_BATCH;
   l.append_row = take(seq); l.append_pos = take(seq); l.compress_row = take(seq); l.compress_pos = take(seq);
+  l.restore_ok = take(seq); l.restore_bea = take(seq + 4);
   l.tickets = take(BC_MAX_ATTN_BATCH * 4);
   l.book_flag = take(4);
   l.part_ml = take(pieces * c.q_heads * 2 * 4);
@@ -91,6 +92,7 @@ struct bc_cache {
   int64_t launches;
   int append_next_layer;    // per-layer ordering of bc_append
   int compress_next_layer;  // per-layer ordering of bc_compress
+  int restore_next_layer = 0;   // per-layer ordering of bc_restore
   int last_cuda_error;
   // profiling
   std::vector<cudaEvent_t> ev;
@@ -305,6 +307,29 @@ bc_status bc_prefill(bc_cache* c, int32_t layer, const int32_t* slots, const int
   if (!k || !v || !aligned16(k) || !aligned16(v)) return BC_ERR_INVALID_ARG;
   BC_CUDA(c, bc_launch_prefill(c->meta, c->geom, layer_base(c, layer), slots, cu, n, total, k, v, (cudaStream_t)stream));
   c->launches += 1;
+  return BC_OK;
+}
+
+bc_status bc_restore(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const int32_t* cu_tokens,
+                     int32_t total_tokens, int32_t total_beacons, const void* tok_k, const void* tok_v,
+                     const void* beacon_k, const void* beacon_v, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (!cu_tokens || total_tokens < 0 || total_beacons < 0) return BC_ERR_INVALID_ARG;
+  if (total_tokens && (!tok_k || !tok_v || !aligned16(tok_k) || !aligned16(tok_v))) return BC_ERR_INVALID_ARG;
+  if (total_beacons && (!beacon_k || !beacon_v || !aligned16(beacon_k) || !aligned16(beacon_v))) return BC_ERR_INVALID_ARG;
+  if (layer != c->restore_next_layer) return BC_ERR_ORDER;
+  cudaStream_t s = (cudaStream_t)stream;
+  int32_t* ok = work_ptr<int32_t>(c, c->wl.restore_ok);
+  int32_t* bea = work_ptr<int32_t>(c, c->wl.restore_bea);
+  if (layer == 0) {
+    BC_CUDA(c, bc_launch_restore_book(c->meta, slots, cu_tokens, n, ++c->calls, ok, bea, s));
+    c->launches += 1;
+  }
+  BC_CUDA(c, bc_launch_restore_rows(c->meta, c->geom, layer_base(c, layer), slots, ok, bea, cu_tokens, n, total_tokens,
+                                   total_beacons, tok_k, tok_v, beacon_k, beacon_v, s));
+  c->launches += (total_beacons > 0) + (total_tokens > 0);
+  c->restore_next_layer = (layer + 1) % c->cfg.layers;
   return BC_OK;
 }
 

@@ -275,6 +275,127 @@ __global__ void k_prefill(BcMeta m, BcGeom g, uint8_t* __restrict__ pool_layer, 
   }
 }
 
+// Bookkeeping of bc_restore (one thread block): item i is a freshly opened sequence that receives a
+// stored trajectory of T_i = cu[i + 1] - cu[i] generated tokens, i.e. the state Algorithm 1 is in
+// after T_i sampling steps: floor(T_i / c) beacons and the T_i mod c tokens of the unfinished window
+// (all T_i when c = 1).  Allocates the beacon pages, then the window pages, of every item by a
+// block-wide prefix sum, and writes for the copy kernels ok[i] (1: granted) and bea[i] = number of
+// beacon rows of the items before i in the packed beacon arrays (items whose slot is not open count
+// none), bea[n] = their total.
+__global__ void __launch_bounds__(kBookThreads, 1)
+k_restore_book(BcMeta m, const int32_t* __restrict__ slots, const int32_t* __restrict__ cu, int n, int64_t call,
+               int32_t* __restrict__ ok, int32_t* __restrict__ bea) {
+  __shared__ int sh_first;
+  ErrLatch latch; latch.init(&sh_first);
+  const int top0 = *m.free_top;
+  const int ps = m.page_size;
+  __syncthreads();
+  int base = 0, bea_base = 0, used = 0, my_code = 0, my_item = -1, my_slot = 0;
+  for (int chunk = 0; chunk < n; chunk += blockDim.x) {
+    const int i = chunk + threadIdx.x;
+    int need = 0, slot = -1, code = 0, nb = 0, w = 0, nbp = 0, nwp = 0, T = 0, rows = 0;
+    bool valid = false;
+    if (i < n) {
+      slot = slots[i];
+      T = cu[i + 1] - cu[i];
+      if (slot < 0 || slot >= m.max_seqs || !m.open[slot]) code = BC_ERR_BAD_SLOT;
+      else {
+        const int c = m.c[slot];
+        if (T >= 0) { nb = c > 1 ? T / c : 0; w = T - nb * c; rows = nb; }
+        if (T < 0 || m.t[slot] != 0 || m.n_beacons[slot] != 0 || m.window_len[slot] != 0) code = BC_ERR_INVALID_ARG;
+        else if (m.max_entries > 0 && nb + w > m.max_entries) code = BC_ERR_CAPACITY;
+        else {
+          nbp = ceil_div(nb, ps); nwp = ceil_div(w, ps);
+          const int reserved = c > 1 ? ceil_div(c, ps) : nwp;   // the window's columns of the page-table row
+          if (ceil_div(m.prompt_len[slot], ps) + reserved + nbp > m.max_pages_per_seq) code = BC_ERR_CAPACITY;
+          else { valid = true; need = nbp + nwp; }
+        }
+      }
+    }
+    int total, bea_total;
+    const int off = base + block_exclusive_scan(need, &total);
+    base += total;
+    const int bea_off = bea_base + block_exclusive_scan(rows, &bea_total);
+    bea_base += bea_total;
+    int granted = 0;
+    if (valid) {
+      if (need == 0 || off + need <= top0) {
+        int32_t* row = m.page_table + (int64_t)slot * m.max_pages_per_seq;
+        for (int k = 0; k < nbp; ++k) row[m.beacon_off[slot] + k] = m.free_stack[top0 - 1 - off - k];
+        for (int k = 0; k < nwp; ++k) row[m.window_off[slot] + k] = m.free_stack[top0 - 1 - off - nbp - k];
+        if (need) used = max(used, off + need);
+        m.n_beacons[slot] = nb; m.window_len[slot] = w; m.t[slot] = T;
+        granted = 1;
+      } else code = BC_ERR_NO_PAGES;
+    }
+    if (i < n) { ok[i] = granted; bea[i] = bea_off; }
+    if (code && my_code == 0) { my_code = code; my_item = i; my_slot = slot; latch.note(i); }
+  }
+  used = __reduce_max_sync(0xffffffffu, used);
+  __shared__ int sh_used;
+  if (threadIdx.x == 0) { sh_used = 0; bea[n] = bea_base; }
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) atomicMax(&sh_used, used);
+  latch.commit(m, my_item, my_code, my_slot, call);
+  __syncthreads();
+  if (threadIdx.x == 0) *m.free_top = top0 - sh_used;
+}
+
+// Copies one K/V entry (all heads) into pool row `row`, 16 bytes per thread, with the store's chunk permutation.
+__device__ __forceinline__ void copy_entry(const BcGeom& g, uint8_t* __restrict__ pool_layer, int row, int pos,
+                                           const uint8_t* __restrict__ k, const uint8_t* __restrict__ v, int64_t src_row) {
+  const int chunks_per_head = g.head_row_bytes >> 4;
+  const int per_side = g.kv_heads * chunks_per_head;
+  uint8_t* dst = pool_layer + (int64_t)row * g.entry_bytes;
+  for (int idx = threadIdx.x; idx < 2 * per_side; idx += blockDim.x) {
+    const int which = idx / per_side, rem = idx - which * per_side;
+    const int h = rem / chunks_per_head, j = rem - h * chunks_per_head;
+    const uint8_t* src = (which ? v : k) + (src_row * g.kv_heads + h) * g.head_row_bytes + (j << 4);
+    *reinterpret_cast<uint4*>(dst + bc_chunk_offset(g, which, h, j, pos)) = *reinterpret_cast<const uint4*>(src);
+  }
+}
+
+// bc_restore, beacons: one block per row of the packed beacon arrays.
+__global__ void k_restore_beacons(BcMeta m, BcGeom g, uint8_t* __restrict__ pool_layer, const int32_t* __restrict__ slots,
+                                  const int32_t* __restrict__ ok, const int32_t* __restrict__ bea, int n,
+                                  const uint8_t* __restrict__ k, const uint8_t* __restrict__ v) {
+  const int b = blockIdx.x;
+  __shared__ int sh_row, sh_pos;
+  if (threadIdx.x == 0) {
+    int row = -1, pos = 0;
+    if (b < bea[n]) {
+      int lo = 0, hi = n;  // largest i with bea[i] <= b (items without beacons share their successor's offset)
+      while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (bea[mid] <= b) lo = mid; else hi = mid; }
+      if (ok[lo]) {
+        const int slot = slots[lo];
+        pos = b - bea[lo];
+        const int page = m.page_table[(int64_t)slot * m.max_pages_per_seq + m.beacon_off[slot] + pos / g.page_size];
+        row = page * g.page_size + pos % g.page_size;
+      }
+    }
+    sh_row = row; sh_pos = pos;
+  }
+  __syncthreads();
+  if (sh_row >= 0) copy_entry(g, pool_layer, sh_row, sh_pos, k, v, b);
+}
+
+// bc_restore, unfinished windows: blocks (item, y) copy window entries y, y + gridDim.y, ... of the item,
+// which are the last window_len rows of its tokens in the packed token arrays.
+__global__ void k_restore_window(BcMeta m, BcGeom g, uint8_t* __restrict__ pool_layer, const int32_t* __restrict__ slots,
+                                 const int32_t* __restrict__ ok, const int32_t* __restrict__ cu, int total_tokens,
+                                 const uint8_t* __restrict__ k, const uint8_t* __restrict__ v) {
+  const int i = blockIdx.x;
+  if (!ok[i]) return;
+  const int slot = slots[i];
+  const int w = m.window_len[slot];
+  const int64_t first = (int64_t)cu[i + 1] - w;   // row of the window's first token
+  const int32_t* cols = m.page_table + (int64_t)slot * m.max_pages_per_seq + m.window_off[slot];
+  for (int j = blockIdx.y; j < w; j += gridDim.y) {
+    if (first + j < 0 || first + j >= total_tokens) continue;
+    copy_entry(g, pool_layer, cols[j / g.page_size] * g.page_size + j % g.page_size, j, k, v, first + j);
+  }
+}
+
 // One block per exported entry, logical order prompt | beacons | window.
 __global__ void k_export(BcMeta m, BcGeom g, const uint8_t* __restrict__ pool_layer, int slot,
                          uint8_t* __restrict__ k_out, uint8_t* __restrict__ v_out, int capacity) {
@@ -341,6 +462,22 @@ cudaError_t bc_launch_prefill(const BcMeta& m, const BcGeom& g, uint8_t* pool_la
                               const int32_t* cu, int n, int total, const void* k, const void* v, cudaStream_t s) {
   if (total == 0) return cudaSuccess;
   k_prefill<<<total, copy_threads(g), 0, s>>>(m, g, pool_layer, slots, cu, n, (const uint8_t*)k, (const uint8_t*)v);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_restore_book(const BcMeta& m, const int32_t* slots, const int32_t* cu, int n, int64_t call, int32_t* ok,
+                                   int32_t* bea, cudaStream_t s) {
+  k_restore_book<<<1, kBookThreads, 0, s>>>(m, slots, cu, n, call, ok, bea);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_restore_rows(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* slots, const int32_t* ok,
+                                   const int32_t* bea, const int32_t* cu, int n, int total_tokens, int total_beacons,
+                                   const void* tok_k, const void* tok_v, const void* bea_k, const void* bea_v, cudaStream_t s) {
+  if (total_beacons > 0)
+    k_restore_beacons<<<total_beacons, copy_threads(g), 0, s>>>(m, g, pool_layer, slots, ok, bea, n, (const uint8_t*)bea_k,
+                                                              (const uint8_t*)bea_v);
+  if (total_tokens > 0)
+    k_restore_window<<<dim3(n, 32), copy_threads(g), 0, s>>>(m, g, pool_layer, slots, ok, cu, total_tokens, (const uint8_t*)tok_k,
+                                                          (const uint8_t*)tok_v);
   return cudaGetLastError();
 }
 cudaError_t bc_launch_export(const BcMeta& m, const BcGeom& g, const uint8_t* pool_layer, int slot, void* k_out,

@@ -60,6 +60,11 @@ cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n
 cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_t call, cudaStream_t s);
 cudaError_t bc_launch_write_rows(const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
                                  const void* k, const void* v, int n, cudaStream_t s);
+cudaError_t bc_launch_restore_book(const BcMeta& m, const int32_t* slots, const int32_t* cu, int n, int64_t call, int32_t* ok,
+                                   int32_t* bea, cudaStream_t s);
+cudaError_t bc_launch_restore_rows(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* slots, const int32_t* ok,
+                                   const int32_t* bea, const int32_t* cu, int n, int total_tokens, int total_beacons,
+                                   const void* tok_k, const void* tok_v, const void* bea_k, const void* bea_v, cudaStream_t s);
 cudaError_t bc_launch_prefill(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* slots,
                               const int32_t* cu, int n, int total, const void* k, const void* v, cudaStream_t s);
 cudaError_t bc_launch_export(const BcMeta& m, const BcGeom& g, const uint8_t* pool_layer, int slot, void* k_out,

@@ -68,6 +68,22 @@ class Pair:
             if slot in self.seqs:
                 self.seqs[slot].prefill(layer, kk[cu[i]:cu[i + 1]], vv[cu[i]:cu[i + 1]])
 
+    def restore(self, layer, slots, gen_lens, tok_k, tok_v, bea_k, bea_v):
+        """tok_*: packed [sum(gen_lens), Hkv, D]; bea_*: packed beacons, floor(T / c) per open sequence."""
+        cu = np.concatenate([[0], np.cumsum(gen_lens)]).astype(np.int32)
+        nbs = [(gen_lens[i] // self.model.seqs[s].c if s in self.model.seqs and self.model.seqs[s].c > 1 else 0)
+               if gen_lens[i] >= 0 else 0 for i, s in enumerate(slots)]
+        cb = np.concatenate([[0], np.cumsum(nbs)]).astype(np.int64)
+        self.gpu.bc_restore(layer, self._i32(slots), self._i32(cu), int(cu[-1]), int(cb[-1]), tok_k, tok_v, bea_k, bea_v)
+        if layer == 0:
+            self._restore_ok = self.model.restore(list(slots), list(gen_lens))
+        tk, tv = f64(tok_k), f64(tok_v)
+        bk, bv = (f64(bea_k), f64(bea_v)) if cb[-1] else (np.zeros((0, self.Hkv, self.D)),) * 2
+        for i, slot in enumerate(slots):
+            if self._restore_ok[i] == OK:
+                self.seqs[slot].replay(layer, tk[cu[i]:cu[i + 1]], tv[cu[i]:cu[i + 1]], bk[cb[i]:cb[i + 1]], bv[cb[i]:cb[i + 1]])
+        return self._restore_ok
+
     def append(self, layer, slots, k, v):
         self.gpu.bc_append(layer, self._i32(slots), k, v)
         if layer == 0:

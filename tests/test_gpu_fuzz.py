@@ -1,4 +1,4 @@
-"""Random programs of open / append / compress / close against the oracle's paging model.
+"""Random programs of open / restore / append / compress / close against the oracle's paging model.
 
 Small pools and odd page sizes make the programs hit every refusal (no pages, window full, window
 not full, bad slot, capacity); after every call the lengths, page lists, free stack and the latched
@@ -26,13 +26,23 @@ def test_random_programs(seed, ps, num_pages, max_pps, max_entries):
     g = torch.Generator(device=DEV); g.manual_seed(seed)
     kv = lambda n: (randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV))
     for step in range(160):
-        op = rng.choice(["open", "append", "append", "append", "compress", "close"])
+        op = rng.choice(["open", "restore", "append", "append", "append", "compress", "close"])
         n = int(rng.randint(1, S + 1))
         slots = [int(x) for x in rng.choice(S + 2, size=n, replace=False) - 1]      # -1 and S are invalid slots
         if op == "open":
             plens = [int(rng.randint(0, 3 * ps + 2)) for _ in slots]
             cs = None if rng.rand() < 0.3 else [int(rng.choice([1, 2, 3, 4, 7])) for _ in slots]
             pair.open(slots, plens, cs)
+        elif op == "restore":
+            # mostly onto sequences that are still fresh, so that restores succeed too
+            fresh = [s for s in range(S) if (st := pair.model.state(s)) and st["t"] == 0]
+            if fresh and rng.rand() < 0.7:
+                slots = fresh[:n]
+            gen_lens = [int(rng.randint(0, 4 * ps + 6)) for _ in slots]
+            nb = sum(T // st["c"] for s, T in zip(slots, gen_lens) if (st := pair.model.state(s)) and st["c"] > 1)
+            tk, tv = kv(max(sum(gen_lens), 1))
+            bk, bv = kv(max(nb, 1))
+            pair.restore(0, slots, gen_lens, tk[:sum(gen_lens)], tv[:sum(gen_lens)], bk[:nb], bv[:nb])
         elif op == "append":
             pair.append(0, slots, *kv(n))
         elif op == "compress":

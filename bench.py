@@ -720,7 +720,7 @@ def report_distill(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     peak, peak_src = load_peaks()
-    n_traj, T, V, K = 16, 1000, 151936, 100
+    n_traj, T, V, K = (16 if args.steps >= 16 else 4), 1000, 151936, 100   # --steps < 16: a 1.2 GB case for profiling
     rows = n_traj * T
     g = torch.Generator(device=dev); g.manual_seed(0)
     z = torch.empty((rows, V), dtype=torch.bfloat16, device=dev)

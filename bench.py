@@ -173,9 +173,11 @@ class _Passes:
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         l1 = self.cache.bc_kernel_launches()
         torch.cuda.nvtx.range_push("timed")
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(reps)]   # one per window: the spread of step times
         e0.record()
-        for _ in range(reps):
+        for i in range(reps):
             graph.replay()
+            marks[i].record()
         self.t += reps * cyc
         for _ in range(rem):
             self.step()
@@ -183,6 +185,10 @@ class _Passes:
         torch.cuda.synchronize()
         torch.cuda.nvtx.range_pop()
         launches = reps * per_graph + (self.cache.bc_kernel_launches() - l1)
+        prev, self.window_step_ms = e0, []
+        for m in marks:
+            self.window_step_ms.append(prev.elapsed_time(m) / cyc)
+            prev = m
         return e0.elapsed_time(e1), t_begin, launches
 
     def timed_kernels(self, K, W):
@@ -337,6 +343,15 @@ def run_profile_case(args):
 
 
 # ------------------------------------------------------------------------------ the other configurations
+def _percentiles(xs):
+    """[p50, p99, windows] of the per-step times of the graph-replayed windows (rank 0's)."""
+    if not xs:
+        return None
+    xs = sorted(xs)
+    pick = lambda q: xs[min(len(xs) - 1, int(math.ceil(q * len(xs))) - 1)]
+    return [pick(0.50), pick(0.99), len(xs)]
+
+
 def _event_pair(torch):
     return torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
@@ -894,6 +909,7 @@ def main():
         end_live, end_unc = r.cache_bytes(T)
         row = {
             "c": c, "page_size": w.page_size, "ms_per_step": ms / K, "tokens_per_s": world * w.batch * K / (ms * 1e-3),
+            "ms_per_step_p50_p99_over_windows": _percentiles(r.window_step_ms),
             "e2e_tokens_per_s": world * w.batch * K / (h_ms * 1e-3),
             "plain_launch_ms_per_step": plain_ms / Kp,
             "kv_gbs_step": (reg + bea) / (ms * 1e-3) / 1e9,

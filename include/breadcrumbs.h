@@ -28,7 +28,12 @@
  *    table) is shared by all layers and changes once per step: bc_append reserves the new slot on
  *    its layer-0 call, bc_compress allocates the beacon slot on its layer-0 call and evicts the
  *    window on its call for the last layer.  For one step, call the layers in ascending order
- *    with the same `slots`; anything else returns BC_ERR_ORDER.
+ *    with the same `slots`; anything else returns BC_ERR_ORDER.  bc_prefill, bc_append,
+ *    bc_decode_attn and bc_compress also take layer = BC_ALL_LAYERS (-1): every per-layer tensor
+ *    of the call (k, v, q, out, extra_k, extra_v, beacon_k, beacon_v) then carries a leading
+ *    [layers] dimension and the call runs layer 0 .. layers - 1 in that order, one launch sequence
+ *    per layer (a forward pass computes layer l + 1's inputs from layer l's output, so this form
+ *    serves replays and measurements, not a model).
  *  - A batch must not name the same slot twice.
  *
  * Store layout (owned by the library inside the caller's `pool` buffer)
@@ -61,6 +66,8 @@
 #ifdef __cplusplus
 extern "C" {
 #endif
+
+#define BC_ALL_LAYERS (-1)   /* `layer` argument: all layers in one call, tensors with a leading [layers] dimension */
 
 typedef int32_t bc_status;
 enum {

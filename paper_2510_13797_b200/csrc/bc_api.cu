@@ -120,6 +120,15 @@ inline uint8_t* layer_base(bc_cache* c, int layer) { return c->pool + (int64_t)l
 template <typename T>
 inline T* work_ptr(bc_cache* c, size_t off) { return reinterpret_cast<T*>(c->work + off); }
 
+// layer == BC_ALL_LAYERS: the per-layer tensors carry a leading [layers] dimension and the call runs
+// layer 0 .. layers - 1 in order (one launch sequence per layer, the dependency order of a forward pass).
+inline const void* layer_slice(const void* p, int layer, size_t bytes_per_layer) {
+  return p ? static_cast<const uint8_t*>(p) + (size_t)layer * bytes_per_layer : nullptr;
+}
+inline void* layer_slice(void* p, int layer, size_t bytes_per_layer) {
+  return p ? static_cast<uint8_t*>(p) + (size_t)layer * bytes_per_layer : nullptr;
+}
+
 bc_status check_batch(bc_cache* c, int layer, const int32_t* slots, int n) {
   if (!c || !slots || n <= 0 || n > c->cfg.max_seqs) return BC_ERR_INVALID_ARG;
   if (layer < 0 || layer >= c->cfg.layers) return BC_ERR_INVALID_ARG;
@@ -300,6 +309,15 @@ bc_status bc_seq_open(bc_cache* c, const int32_t* slots, const int32_t* prompt_l
 
 bc_status bc_prefill(bc_cache* c, int32_t layer, const int32_t* slots, const int32_t* cu, int32_t n, int32_t total,
                      const void* k, const void* v, void* stream) {
+  if (c && layer == BC_ALL_LAYERS) {
+    if (total < 0) return BC_ERR_INVALID_ARG;
+    const size_t b = (size_t)total * c->cfg.kv_heads * c->cfg.head_dim * 2;
+    for (int l = 0; l < c->cfg.layers; ++l) {
+      const bc_status st = bc_prefill(c, l, slots, cu, n, total, layer_slice(k, l, b), layer_slice(v, l, b), stream);
+      if (st) return st;
+    }
+    return BC_OK;
+  }
   bc_status st = check_batch(c, layer, slots, n);
   if (st) return st;
   if (!cu || total < 0) return BC_ERR_INVALID_ARG;
@@ -335,6 +353,15 @@ bc_status bc_restore(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n
 
 bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* k, const void* v,
                     void* stream) {
+  if (c && layer == BC_ALL_LAYERS) {
+    if (n <= 0) return BC_ERR_INVALID_ARG;
+    const size_t b = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+    for (int l = 0; l < c->cfg.layers; ++l) {
+      const bc_status st = bc_append(c, l, slots, n, layer_slice(k, l, b), layer_slice(v, l, b), stream);
+      if (st) return st;
+    }
+    return BC_OK;
+  }
   bc_status st = check_batch(c, layer, slots, n);
   if (st) return st;
   if (!k || !v || !aligned16(k) || !aligned16(v)) return BC_ERR_INVALID_ARG;
@@ -359,6 +386,17 @@ bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n,
 
 bc_status bc_decode_attn(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, void* out,
                          float sm_scale, const void* extra_k, const void* extra_v, void* stream) {
+  if (c && layer == BC_ALL_LAYERS) {
+    if (n <= 0) return BC_ERR_INVALID_ARG;
+    const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+    const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
+    for (int l = 0; l < c->cfg.layers; ++l) {
+      const bc_status st = bc_decode_attn(c, l, slots, n, layer_slice(q, l, qb), layer_slice(out, l, ob), sm_scale,
+                                          layer_slice(extra_k, l, kb), layer_slice(extra_v, l, kb), stream);
+      if (st) return st;
+    }
+    return BC_OK;
+  }
   bc_status st = check_batch(c, layer, slots, n);
   if (st) return st;
   if (n > BC_MAX_ATTN_BATCH) return BC_ERR_INVALID_ARG;
@@ -399,6 +437,15 @@ bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32
 
 bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* bk, const void* bv,
                       void* stream) {
+  if (c && layer == BC_ALL_LAYERS) {
+    if (n <= 0) return BC_ERR_INVALID_ARG;
+    const size_t b = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+    for (int l = 0; l < c->cfg.layers; ++l) {
+      const bc_status st = bc_compress(c, l, slots, n, layer_slice(bk, l, b), layer_slice(bv, l, b), stream);
+      if (st) return st;
+    }
+    return BC_OK;
+  }
   bc_status st = check_batch(c, layer, slots, n);
   if (st) return st;
   if (!bk || !bv || !aligned16(bk) || !aligned16(bv)) return BC_ERR_INVALID_ARG;

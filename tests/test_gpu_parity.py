@@ -13,6 +13,7 @@ import torch
 from oracle.breadcrumbs_oracle import closed_form_length
 from paper_2510_13797_b200 import binding as B
 from paper_2510_13797_b200.workloads import InputStream, make_workload
+from oracle.paging_model import OK
 from tests.harness import Pair, assert_close, f64, randn_bf16
 
 pytestmark = pytest.mark.gpu
@@ -438,3 +439,49 @@ def test_host_buffer_steps_back_to_back_packed():
     for s in slots:
         pair.check_content(0, s)
 
+
+
+def test_all_layers_in_one_call():
+    """layer = -1: the per-layer tensors carry a leading [layers] dimension and one call walks the
+    layers in order.  Compared per layer with the oracle (and, for the bookkeeping, with the model)."""
+    L, Hkv, G, D, ps, c = 3, 2, 4, 128, 8, 4
+    n, plens = 3, [20, 0, 65]
+    pair = Pair(L, Hkv, Hkv * G, D, ps, max_seqs=n, num_pages=64, max_pages_per_seq=24)
+    g = _gen(29)
+    slots = list(range(n))
+    sl = torch.tensor(slots, dtype=torch.int32, device=DEV)
+    pair.open(slots, plens, [c] * n)
+    P = sum(plens)
+    pk, pv = randn_bf16(g, (L, P, Hkv, D), DEV), randn_bf16(g, (L, P, Hkv, D), DEV)
+    cu = torch.tensor([0] + list(np.cumsum(plens)), dtype=torch.int32, device=DEV)
+    pair.gpu.bc_prefill(-1, sl, cu, P, pk, pv)
+    for l in range(L):
+        for i, s in enumerate(slots):
+            a, b = int(cu[i]), int(cu[i + 1])
+            pair.seqs[s].prefill(l, f64(pk[l, a:b]), f64(pv[l, a:b]))
+    for step in range(1, 2 * c + 2):
+        k, v, q = randn_bf16(g, (L, n, Hkv, D), DEV), randn_bf16(g, (L, n, Hkv, D), DEV), randn_bf16(g, (L, n, Hkv * G, D), DEV)
+        out = torch.empty((L, n, Hkv * G, D), dtype=torch.bfloat16, device=DEV)
+        pair.gpu.bc_append(-1, sl, k, v)
+        pair.gpu.bc_decode_attn(-1, sl, q, out, 0.11)
+        assert pair.model.append(slots) == [OK] * n
+        for l in range(L):
+            for i, s in enumerate(slots):
+                pair.seqs[s].append(l, f64(k[l, i]), f64(v[l, i]))
+            ref = np.stack([pair.seqs[s].attend(l, f64(q[l, i]), 0.11) for i, s in enumerate(slots)])
+            assert_close(out[l], ref, f"step {step} layer {l}")
+        if step % c == 0:
+            bk, bv, bq = randn_bf16(g, (L, n, Hkv, D), DEV), randn_bf16(g, (L, n, Hkv, D), DEV), randn_bf16(g, (L, n, Hkv * G, D), DEV)
+            pair.gpu.bc_decode_attn(-1, sl, bq, out, 0.11, bk, bv)
+            pair.gpu.bc_compress(-1, sl, bk, bv)
+            assert pair.model.compress(slots) == [OK] * n
+            for l in range(L):
+                ref = np.stack([pair.seqs[s].beacon_attend(l, f64(bq[l, i]), f64(bk[l, i]), f64(bv[l, i]), 0.11)
+                                for i, s in enumerate(slots)])
+                assert_close(out[l], ref, f"beacon step {step} layer {l}")
+                for i, s in enumerate(slots):
+                    pair.seqs[s].compress(l, f64(bk[l, i]), f64(bv[l, i]))
+        pair.check_state()
+    for l in range(L):
+        for s in slots:
+            pair.check_content(l, s)

@@ -5,9 +5,10 @@ Workload (the compression-ratio sweep): one layer, batch 64, 32 query /
 8 KV heads, head_dim 128, bf16, prompt 512, 16384 decode steps, c in {2,4,8,16,32} with
 page_size = c, plus the uncompressed run (c = 1, page 16) as a reported row.
 
-One "step" of the JSON line = one decode step (bc_append + bc_decode_attn, and when the window
-fills the beacon-query attention + bc_compress) at EACH of the five compressed ratios, i.e. 5 x 64
-generated tokens.  The ratios are timed one after the other, K steps each, centred on the middle
+One "step" of the JSON line = one decode step (bc_append + bc_decode_attn; when the token fills the
+window, bc_decode_attn_pair instead -- the token's and the beacon's queries in one pass over the
+cache -- and bc_compress; --no-pair runs the beacon's attention as a second pass) at EACH of the
+five compressed ratios, i.e. 5 x 64 generated tokens.  The ratios are timed one after the other, K steps each, centred on the middle
 of the 16384-step generation (cache length grows linearly with t, so the mean over a window centred
 on the midpoint equals the mean over the whole run).  `value` = tokens / second over all of that.
 
@@ -113,11 +114,11 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------ one ratio on the GPU
-def make_runner(w, device, seed_offset=0):
+def make_runner(w, device, seed_offset=0, paired=True):
     """A DecodeDriver (one cache, batch B at ratio c, driven through the C ABI) plus the timed passes."""
     import torch
     from paper_2510_13797_b200.driver import DecodeDriver
-    r = type("RatioRunner", (_Passes, DecodeDriver), {})(w, device, seed_offset)
+    r = type("RatioRunner", (_Passes, DecodeDriver), {})(w, device, seed_offset, paired=paired)
     r.torch = torch
     return r
 
@@ -140,6 +141,8 @@ class _Passes:
         reg = sum(entries_attended(self.P, n, self.c) for n in range(t_from + 1, t_from + steps + 1))
         bea = sum(entries_beacon_query(self.P, n, self.c) for n in range(t_from + 1, t_from + steps + 1)
                   if self.c > 1 and n % self.c == 0)
+        if getattr(self, "paired", False):
+            bea = 0          # the beacon's queries ride on the token's pass over the cache: no second read
         return reg * E * self.n, bea * E * self.n
 
     def cache_bytes(self, t):
@@ -199,7 +202,8 @@ class _Passes:
             self.step()
         torch.cuda.synchronize()
         t_begin = self.t
-        n_launch = K + (sum(1 for n in range(t_begin + 1, t_begin + K + 1) if n % self.c == 0) if self.c > 1 else 0)
+        n_launch = K + (sum(1 for n in range(t_begin + 1, t_begin + K + 1) if n % self.c == 0)
+                        if self.c > 1 and not self.paired else 0)
         self.cache.bc_profile_enable(n_launch)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.nvtx.range_push("kernels")
@@ -834,6 +838,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=32)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-pair", action="store_true", help="beacon steps as a second attention pass instead of bc_decode_attn_pair")
     ap.add_argument("--fused", action="store_true", help="depth workload: regular steps through bc_decode_step (append + attention in one launch per layer)")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
@@ -886,7 +891,7 @@ def main():
     for c in sweep:
         w = make_workload("sweep", c=c)
         T = w.steps
-        r = make_runner(w, dev, seed_offset=sharding.rank_seed_offset(0, rank))
+        r = make_runner(w, dev, seed_offset=sharding.rank_seed_offset(0, rank), paired=not args.no_pair)
         cyc = c if c > 1 else 16
         t_mid = max(0, ((T - K) // 2 // cyc) * cyc)
         # pass A: device-resident inputs, CUDA-graph replays: the headline time
@@ -951,7 +956,9 @@ def main():
                                "c in {2,4,8,16,32}, page_size=c; one step = one decode step at each ratio, "
                                "timed ratio by ratio around mid-generation",
                    "l2": "inputs larger than L2: every step streams 206 MB (c=32) to 1.2 GB (c=2) of KV, L2 is 126 MB",
-                   "launch": "CUDA-graph replay of whole windows of c steps", "per_gpu_batch": B * n_c},
+                   "launch": "CUDA-graph replay of whole windows of c steps", "per_gpu_batch": B * n_c,
+                   "beacon_steps": "second attention pass" if args.no_pair else
+                                   "paired with the token's attention (bc_decode_attn_pair: one pass over the cache)"},
         "e2e": {"value": world * B * n_c * K / (e2e_ms * 1e-3), "unit": "tokens/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(total_launches),

@@ -189,6 +189,19 @@ BC_API bc_status bc_decode_attn(bc_cache* cache, int32_t layer, const int32_t* s
                          const void* q, void* out, float sm_scale, const void* extra_k,
                          const void* extra_v, void* stream);
 
+/* The step that fills a window, and the encoding of the beacon that follows it, in one pass over the
+ * cache (Algorithm 1: the token's forward pass and the beacon's read the same entries; the beacon
+ * also sees itself).  out = what bc_decode_attn(q) returns; out_beacon = what
+ * bc_decode_attn(beacon_q, extra = beacon_k, beacon_v) returns, both over the cache as it stands (call
+ * it after the token's bc_append and before bc_compress).  The K/V entries are read from HBM once
+ * for both: at ratio c this saves the 1/c extra attention traffic of the beacon steps.  For groups
+ * of more than 8 query heads per KV head (and with BC_FLAG_ATTN_REFERENCE) the two results come from
+ * two passes.  Arguments as for bc_decode_attn; beacon_q, out_beacon like q, out. */
+BC_API bc_status bc_decode_attn_pair(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
+                                     const void* q, void* out, const void* beacon_q, void* out_beacon,
+                                     float sm_scale, const void* beacon_k, const void* beacon_v,
+                                     void* stream);
+
 /* One decode step of one layer in a single launch: bc_append(k, v) followed by bc_decode_attn(q)
  * (Algorithm 1: the forward pass of a token adds its entry, then its query reads the cache, the
  * new entry included).  Results, bookkeeping, layer-order rule and error behaviour are exactly
@@ -261,6 +274,14 @@ BC_API bc_status bc_seq_close(bc_cache* cache, const int32_t* slots, int32_t n, 
 BC_API bc_status bc_decode_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                               const void* q_host, const void* k_host, const void* v_host,
                               void* out_host, float sm_scale, void* stream);
+/* The step that fills a window, with host buffers: bc_append of the token, bc_decode_attn_pair for
+ * the token and its beacon (one pass over the cache), bc_compress.  Equivalent to
+ * bc_decode_step_host followed by bc_compress_step_host; same conventions. */
+BC_API bc_status bc_fill_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
+                                   const void* q_host, const void* k_host, const void* v_host,
+                                   const void* beacon_q_host, const void* beacon_k_host,
+                                   const void* beacon_v_host, void* out_host, void* out_beacon_host,
+                                   float sm_scale, void* stream);
 /* The beacon step with host buffers: beacon-query attention (beacon K/V as the extra entry), then
  * bc_compress. */
 BC_API bc_status bc_compress_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,

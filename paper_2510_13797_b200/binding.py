@@ -59,6 +59,8 @@ SYMBOLS = {
     "bc_append": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
     "bc_decode_attn": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
     "bc_decode_step": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P]),
+    "bc_fill_step_host": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _P, _P, _P, _P, _F, _P]),
+    "bc_decode_attn_pair": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P, _P, _P]),
     "bc_decode_attn_static": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
     "bc_mask_attn_query_bytes": (_I32, [_I32, _I32, _I32, _I32, _I64, _I64, _I64, C.POINTER(C.c_size_t)]),
     "bc_mask_attn_forward": (_I32, [_I32, _I32, _I32, _I32, _I32, C.POINTER(_I32), C.POINTER(_I32)] + [_P] * 10
@@ -162,6 +164,16 @@ class Cache:
     def bc_decode_attn(self, layer, slots, q, out, sm_scale, extra_k=None, extra_v=None, stream=None):
         _check(lib().bc_decode_attn(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(out), sm_scale,
                                     _ptr(extra_k), _ptr(extra_v), _stream(stream)), "bc_decode_attn")
+
+    def bc_fill_step_host(self, layer, slots, q, k, v, beacon_q, beacon_k, beacon_v, out, out_beacon, sm_scale, stream=None):
+        _check(lib().bc_fill_step_host(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(k), _ptr(v), _ptr(beacon_q),
+                                       _ptr(beacon_k), _ptr(beacon_v), _ptr(out), _ptr(out_beacon), sm_scale, _stream(stream)),
+               "bc_fill_step_host")
+
+    def bc_decode_attn_pair(self, layer, slots, q, out, beacon_q, out_beacon, sm_scale, beacon_k, beacon_v, stream=None):
+        _check(lib().bc_decode_attn_pair(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(out), _ptr(beacon_q),
+                                         _ptr(out_beacon), sm_scale, _ptr(beacon_k), _ptr(beacon_v), _stream(stream)),
+               "bc_decode_attn_pair")
 
     def bc_decode_step(self, layer, slots, q, k, v, out, sm_scale, stream=None):
         """bc_append(k, v) + bc_decode_attn(q) in one launch."""

@@ -32,7 +32,8 @@ MetaLayout meta_layout(const bc_config& c) {
 }
 
 struct WorkLayout {
-  size_t append_row, append_pos, compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, stage_in[2], stage_out,
+  size_t append_row, append_pos, compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[2],
+      stage_out, stage_out2,
       total;
 };
 WorkLayout work_layout(const bc_config& c) {
@@ -47,9 +48,12 @@ WorkLayout work_layout(const bc_config& c) {
   l.book_flag = take(4);
   l.part_ml = take(pieces * c.q_heads * 2 * 4);
   l.part_o = take(pieces * c.q_heads * c.head_dim * 4);
+  l.part_ml2 = take(pieces * c.q_heads * 2 * 4);            // the beacons' partials of the paired form
+  l.part_o2 = take(pieces * c.q_heads * c.head_dim * 4);
   // host-buffer entry points: two input staging buffers, each k | v | q packed for the call's batch
   for (int b = 0; b < 2; ++b) l.stage_in[b] = take((size_t)BC_MAX_ATTN_BATCH * (c.q_heads + 2 * c.kv_heads) * c.head_dim * 2);
   l.stage_out = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
+  l.stage_out2 = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
   l.total = o;
   return l;
 }
@@ -136,8 +140,14 @@ bc_status check_batch(bc_cache* c, int layer, const int32_t* slots, int n) {
 }
 
 bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const void* q, void* out, float sm_scale,
-                    const void* extra_k, const void* extra_v, cudaStream_t s, const BcFusedAppend* fused = nullptr) {
+                    const void* extra_k, const void* extra_v, cudaStream_t s, const BcFusedAppend* fused = nullptr,
+                    const void* q2 = nullptr, void* out2 = nullptr) {
   BcAttnArgs a;
+  if (q2) {   // the paired form
+    a.q2 = q2; a.out2 = out2;
+    a.part_o2 = work_ptr<float>(c, c->wl.part_o2);
+    a.part_ml2 = work_ptr<float>(c, c->wl.part_ml2);
+  }
   a.pool_layer = layer_base(c, layer);
   a.slots = slots; a.n = n; a.q = q; a.out = out;
   a.out_f32 = (c->cfg.flags & BC_FLAG_OUT_F32) ? 1 : 0;
@@ -406,6 +416,26 @@ bc_status bc_decode_attn(bc_cache* c, int32_t layer, const int32_t* slots, int32
   return attn_impl(c, layer, slots, n, q, out, sm_scale, extra_k, extra_v, (cudaStream_t)stream);
 }
 
+bc_status bc_decode_attn_pair(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, void* out,
+                              const void* beacon_q, void* out_beacon, float sm_scale, const void* beacon_k,
+                              const void* beacon_v, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (n > BC_MAX_ATTN_BATCH) return BC_ERR_INVALID_ARG;
+  if (!q || !out || !beacon_q || !out_beacon || !beacon_k || !beacon_v) return BC_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out) || !aligned16(beacon_q) || !aligned16(out_beacon) || !aligned16(beacon_k) ||
+      !aligned16(beacon_v))
+    return BC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if ((c->cfg.flags & BC_FLAG_ATTN_REFERENCE) || c->cfg.q_heads / c->cfg.kv_heads > 8) {
+    // no shared pass for the debugging kernel and for groups of more than 8 query heads: two passes
+    st = attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s);
+    if (st) return st;
+    return attn_impl(c, layer, slots, n, beacon_q, out_beacon, sm_scale, beacon_k, beacon_v, s);
+  }
+  return attn_impl(c, layer, slots, n, q, out, sm_scale, beacon_k, beacon_v, s, nullptr, beacon_q, out_beacon);
+}
+
 bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, const void* k,
                          const void* v, void* out, float sm_scale, void* stream) {
   bc_status st = check_batch(c, layer, slots, n);
@@ -538,6 +568,35 @@ bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, 
   if (st) return st;
   BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
   BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
+  return BC_OK;
+}
+
+bc_status bc_fill_step_host(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q_host,
+                            const void* k_host, const void* v_host, const void* bq_host, const void* bk_host,
+                            const void* bv_host, void* out_host, void* out_beacon_host, float sm_scale, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (n > BC_MAX_ATTN_BATCH || !q_host || !k_host || !v_host || !bq_host || !bk_host || !bv_host || !out_host || !out_beacon_host)
+    return BC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
+  const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
+  void *dq, *dk, *dv, *dbq, *dbk, *dbv, *dout = c->work + c->wl.stage_out, *dout2 = c->work + c->wl.stage_out2;
+  int buf, buf2;
+  st = stage_inputs(c, n, q_host, k_host, v_host, s, &buf, &dq, &dk, &dv);
+  if (st) return st;
+  st = stage_inputs(c, n, bq_host, bk_host, bv_host, s, &buf2, &dbq, &dbk, &dbv);
+  if (st) return st;
+  st = bc_append(c, layer, slots, n, dk, dv, stream);
+  if (st) return st;
+  st = bc_decode_attn_pair(c, layer, slots, n, dq, dout, dbq, dout2, sm_scale, dbk, dbv, stream);
+  if (st) return st;
+  st = bc_compress(c, layer, slots, n, dbk, dbv, stream);
+  if (st) return st;
+  BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
+  BC_CUDA(c, cudaEventRecord(c->ev_used[buf2], s));
+  BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
+  BC_CUDA(c, cudaMemcpyAsync(out_beacon_host, dout2, ob, cudaMemcpyDeviceToHost, s));
   return BC_OK;
 }
 

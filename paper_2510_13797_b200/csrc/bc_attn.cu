@@ -273,8 +273,14 @@ __device__ __forceinline__ void combine_pieces(const float* part_o, const float*
 // out, the consumer warps write it into the shared-memory tile straight from the input, and the
 // service warp stores it to the pool for the steps to come.  So the step costs no second and third
 // launch and no fence.
-template <int D, bool G_LE_8, bool FUSED>
+// PAIR: every sequence has two sets of query heads, the token's (rows 0..G-1 of a warp's 16-row
+// fragment) and its beacon's (rows 8..8+G-1), which share one pass over the cache: the step whose token
+// fills the window and the encoding of the beacon that follows it (Algorithm 1) read the same entries.
+// The beacon's rows also see the extra entry (the beacon's own K/V).  Needs G <= 8 and is compiled
+// on the 16-row path (G_LE_8 = false); results go to out (token) and out2 (beacon).
+template <int D, bool G_LE_8, bool FUSED, bool PAIR = false>
 __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams p) {
+  static_assert(!PAIR || (!G_LE_8 && !FUSED), "the paired form runs on the 16-row path without the fused append");
   using L = PipeSmem<D>;
   constexpr int NSTAGE = L::kStages;
   constexpr int KSTEPS = D / 16;  // k-steps of QK^T
@@ -547,7 +553,11 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       qr[kk][0] = gq < G ? *reinterpret_cast<const uint32_t*>(qb + gq * D + d0) : 0u;
       qr[kk][2] = gq < G ? *reinterpret_cast<const uint32_t*>(qb + gq * D + d0 + 8) : 0u;
       if (G_LE_8) { qr[kk][1] = 0u; qr[kk][3] = 0u; }
-      else {
+      else if (PAIR) {   // rows 8 .. 8 + G - 1: the beacon's query heads of the same KV head
+        const __nv_bfloat16* qb2 = reinterpret_cast<const __nv_bfloat16*>(p.a.q2) + ((int64_t)i * Hq + kvh * G) * D;
+        qr[kk][1] = gq < G ? *reinterpret_cast<const uint32_t*>(qb2 + gq * D + d0) : 0u;
+        qr[kk][3] = gq < G ? *reinterpret_cast<const uint32_t*>(qb2 + gq * D + d0 + 8) : 0u;
+      } else {
         qr[kk][1] = gq + 8 < G ? *reinterpret_cast<const uint32_t*>(qb + (gq + 8) * D + d0) : 0u;
         qr[kk][3] = gq + 8 < G ? *reinterpret_cast<const uint32_t*>(qb + (gq + 8) * D + d0 + 8) : 0u;
       }
@@ -597,7 +607,8 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       }
       d0 += __shfl_xor_sync(0xffffffffu, d0, 1); d0 += __shfl_xor_sync(0xffffffffu, d0, 2);
       if (!G_LE_8) { d1 += __shfl_xor_sync(0xffffffffu, d1, 1); d1 += __shfl_xor_sync(0xffffffffu, d1, 2); }
-      const bool r0 = gq < G, r1 = !G_LE_8 && (gq + 8 < G);
+      // paired form: only the beacon's rows see the extra entry
+      const bool r0 = !PAIR && gq < G, r1 = PAIR ? gq < G : (!G_LE_8 && (gq + 8 < G));
       if (r0) { m0 = d0 * p.scale_log2; l0 = qd == 0 ? 1.f : 0.f; }
       if (r1) { m1 = d1 * p.scale_log2; l1 = qd == 0 ? 1.f : 0.f; }
 #pragma unroll
@@ -732,6 +743,87 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     // ---- end of piece: merge the groups of each KV head in shared memory, then write -------------
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     if (!G_LE_8) { l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2); }
+    if constexpr (PAIR) {
+      // How this piece leaves: 0 = the whole sequence is here, 1 = final piece and every other piece is
+      // published (merge now), 2 = publish.  The same for the token's and the beacon's heads, which go
+      // through the merge buffer one after the other.
+      int mode = whole ? 0 : 2;
+      int first = 0, last = 0;
+      if (!whole) {
+        first = cta_of(s_cum[i]); last = cta_of(s_cum[i + 1] - 1);
+        if (!has_next) {
+          if (tid == 0) s_pend[4] = ld_acquire(p.a.tickets + i);
+          consumer_bar();
+          if (s_pend[4] == last - first) { mode = 1; __threadfence(); }
+        }
+      }
+      const int64_t pslot = (int64_t)cta + i;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        for (int gi = 0; gi < p.n_groups; ++gi) {
+          if (grp == gi && gq < G) {
+            const int h = kvh * G + gq;
+            const float mm = half ? m1 : m0, ll = half ? l1 : l0;
+            float sa = 0.f, sb = 1.f, mnew = mm, lnew = ll;
+            if (gi > 0) {
+              const float mb = merge_ml[h * 2], lb = merge_ml[h * 2 + 1];
+              mnew = fmaxf(mb, mm);
+              const float msafe = mnew == -INFINITY ? 0.f : mnew;
+              sa = exp2f(mb - msafe); sb = exp2f(mm - msafe);
+              lnew = lb * sa + ll * sb;
+            }
+            float* orow = merge_o + h * D;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+              const int d = nt * 8 + qd * 2;
+              float2 cur = gi > 0 ? *reinterpret_cast<float2*>(orow + d) : make_float2(0.f, 0.f);
+              cur.x = cur.x * sa + (half ? o[nt][2] : o[nt][0]) * sb;
+              cur.y = cur.y * sa + (half ? o[nt][3] : o[nt][1]) * sb;
+              *reinterpret_cast<float2*>(orow + d) = cur;
+            }
+            __syncwarp(__activemask());
+            if (qd == 0) { merge_ml[h * 2] = mnew; merge_ml[h * 2 + 1] = lnew; }
+          }
+          consumer_bar();
+        }
+        void* outp = half ? p.a.out2 : p.a.out;
+        float* part_o = half ? p.a.part_o2 : p.a.part_o;
+        float* part_ml = half ? p.a.part_ml2 : p.a.part_ml;
+        if (mode == 0) {
+          const int64_t obase = (int64_t)i * Hq * D;
+          for (int idx = tid; idx < Hq * D; idx += kConsumerWarps * 32) {
+            const int h = idx / D;
+            const float l = merge_ml[h * 2 + 1];
+            const float val = l > 0.f ? merge_o[idx] / l : 0.f;
+            if (p.a.out_f32) reinterpret_cast<float*>(outp)[obase + idx] = val;
+            else reinterpret_cast<__nv_bfloat16*>(outp)[obase + idx] = __float2bfloat16_rn(val);
+          }
+        } else if (mode == 1) {
+          combine_pieces(part_o, part_ml, outp, p.a.out_f32, Hq, D, i, first, last, cta, merge_o, merge_ml, tid);
+        } else {
+          float* po = part_o + pslot * Hq * D;
+          for (int idx = tid; idx < Hq * D; idx += kConsumerWarps * 32) po[idx] = merge_o[idx];
+          if (tid < Hq * 2) part_ml[pslot * Hq * 2 + tid] = merge_ml[tid];
+        }
+        consumer_bar();  // the merge buffer is reused by the other half and by the next piece
+      }
+      if (mode == 1) {
+        if (tid == 0) p.a.tickets[i] = 0;  // ready for the next launch
+      } else if (mode == 2) {
+        if (has_next) {
+          // the block's first piece: hand it to the service warp and go on streaming
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_pub);
+        } else {
+          if (tid == 0) {
+            __threadfence();
+            pend_tk = atomicAdd(p.a.tickets + i, 1);
+            pend_seq = i;
+          }
+          published_last = true;
+        }
+      }
+    } else {
     for (int gi = 0; gi < p.n_groups; ++gi) {
       if (grp == gi) {
 #pragma unroll
@@ -814,6 +906,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
         }
       }
     }
+    }
     if (has_next) {
 #pragma unroll
       for (int kk = 0; kk < KSTEPS; ++kk) {
@@ -837,6 +930,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     if (tk == last - first) {
       __threadfence();
       combine_pieces(p.a.part_o, p.a.part_ml, p.a.out, p.a.out_f32, Hq, D, seq, first, last, -1, nullptr, nullptr, tid);
+      if (PAIR) combine_pieces(p.a.part_o2, p.a.part_ml2, p.a.out2, p.a.out_f32, Hq, D, seq, first, last, -1, nullptr, nullptr, tid);
       if (tid == 0) p.a.tickets[seq] = 0;  // ready for the next launch
     }
   }
@@ -907,18 +1001,18 @@ FastDiv make_fast_div(uint32_t d) {
   return f;
 }
 
-template <int D, bool G8, bool FUSED>
+template <int D, bool G8, bool FUSED, bool PAIR = false>
 cudaError_t launch_pipe(const PipeParams& p, cudaStream_t s) {
-  k_attn_pipe<D, G8, FUSED><<<p.a.ctas, kPipeThreads, PipeSmem<D>::kTotal, s>>>(p);
+  k_attn_pipe<D, G8, FUSED, PAIR><<<p.a.ctas, kPipeThreads, PipeSmem<D>::kTotal, s>>>(p);
   return cudaGetLastError();
 }
 
 }  // namespace
 
 namespace {
-template <int D, bool G8, bool FUSED>
+template <int D, bool G8, bool FUSED, bool PAIR = false>
 cudaError_t opt_in_smem() {
-  return cudaFuncSetAttribute(k_attn_pipe<D, G8, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<D>::kTotal);
+  return cudaFuncSetAttribute(k_attn_pipe<D, G8, FUSED, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<D>::kTotal);
 }
 }  // namespace
 
@@ -928,9 +1022,10 @@ cudaError_t bc_attn_setup(int* sm_count) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  const cudaError_t r[8] = {opt_in_smem<128, true, false>(), opt_in_smem<128, false, false>(), opt_in_smem<64, true, false>(),
-                            opt_in_smem<64, false, false>(), opt_in_smem<128, true, true>(), opt_in_smem<128, false, true>(),
-                            opt_in_smem<64, true, true>(), opt_in_smem<64, false, true>()};
+  const cudaError_t r[10] = {opt_in_smem<128, true, false>(), opt_in_smem<128, false, false>(), opt_in_smem<64, true, false>(),
+                             opt_in_smem<64, false, false>(), opt_in_smem<128, true, true>(), opt_in_smem<128, false, true>(),
+                             opt_in_smem<64, true, true>(), opt_in_smem<64, false, true>(),
+                             opt_in_smem<128, false, false, true>(), opt_in_smem<64, false, false, true>()};
   for (cudaError_t x : r)
     if (x != cudaSuccess) return x;
   return cudaSuccess;
@@ -956,7 +1051,9 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   cudaError_t e;
   if (ev_start) { e = cudaEventRecord(ev_start, s); if (e != cudaSuccess) return e; }
   const bool g8 = p.G <= 8;
-  if (fused) {
+  if (a.q2 != nullptr) {   // the paired form (token and beacon queries in one pass); the caller has checked G <= 8
+    e = g.head_dim == 128 ? launch_pipe<128, false, false, true>(p, s) : launch_pipe<64, false, false, true>(p, s);
+  } else if (fused) {
     if (g.head_dim == 128) e = g8 ? launch_pipe<128, true, true>(p, s) : launch_pipe<128, false, true>(p, s);
     else e = g8 ? launch_pipe<64, true, true>(p, s) : launch_pipe<64, false, true>(p, s);
   } else {

@@ -85,6 +85,11 @@ struct BcAttnArgs {
   float* part_ml;        // [(ctas + n)][q_heads][2]
   int32_t* tickets;      // [n] pieces of each sequence published so far; zero between launches
   int32_t ctas;
+  // the paired form (NULL otherwise): the beacons' queries, their outputs and their partial buffers
+  const void* q2 = nullptr;
+  void* out2 = nullptr;
+  float* part_o2 = nullptr;
+  float* part_ml2 = nullptr;
 };
 // Configures the kernels once per process/device (shared-memory opt-in).  Returns the SM count.
 cudaError_t bc_attn_setup(int* sm_count);

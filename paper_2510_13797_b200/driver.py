@@ -21,9 +21,11 @@ from .workloads import InputStream
 
 
 class DecodeDriver:
-    def __init__(self, w, device, seed_offset=0, fused=False):
+    def __init__(self, w, device, seed_offset=0, fused=False, paired=True):
         self.w, self.dev = w, torch.device(device)
         self.fused = fused                             # True: regular steps through bc_decode_step (one launch)
+        self.paired = paired                           # True: the step that fills a window attends for the token and
+                                                       # for its beacon in one pass over the cache (bc_decode_attn_pair)
         c, ps, Bn = w.cs[0], w.page_size, w.batch
         P, T = w.prompt_lens[0], w.steps
         assert all(x == c for x in w.cs) and all(x == P for x in w.prompt_lens), "uniform batches only"
@@ -72,6 +74,13 @@ class DecodeDriver:
         """One decode step of the whole batch through the device-pointer calls.  Returns True if the
         window filled and the beacon step (beacon-query attention into out_b, then compress) ran."""
         c, j = self.cache, self.t % self.ring
+        if self.paired and self.c > 1 and (self.t + 1) % self.c == 0:
+            b = ((self.t + 1) // self.c) % 4
+            c.bc_append(0, self.slots, self.k[j], self.v[j])
+            c.bc_decode_attn_pair(0, self.slots, self.q[j], self.out, self.bq[b], self.out_b, self.w.sm_scale, self.bk[b], self.bv[b])
+            self.t += 1
+            c.bc_compress(0, self.slots, self.bk[b], self.bv[b])
+            return True
         if self.fused:
             c.bc_decode_step(0, self.slots, self.q[j], self.k[j], self.v[j], self.out, self.w.sm_scale)
         else:
@@ -103,6 +112,12 @@ class DecodeDriver:
             hbk, hbv, hbq = packed(self.bk, self.bv, self.bq)
             self.h = dict(q=hq, k=hk, v=hv, bq=hbq, bk=hbk, bv=hbv, out=pin(self.out), out_b=pin(self.out_b))
         c, j, h = self.cache, self.t % self.ring, self.h
+        if self.paired and self.c > 1 and (self.t + 1) % self.c == 0:
+            b = ((self.t + 1) // self.c) % 4
+            c.bc_fill_step_host(0, self.slots, h["q"][j], h["k"][j], h["v"][j], h["bq"][b], h["bk"][b], h["bv"][b],
+                                h["out"], h["out_b"], self.w.sm_scale)
+            self.t += 1
+            return
         c.bc_decode_step_host(0, self.slots, h["q"][j], h["k"][j], h["v"][j], h["out"], self.w.sm_scale)
         self.t += 1
         if self.c > 1 and self.t % self.c == 0:

@@ -367,7 +367,7 @@ def report_cfg2(args):
     from paper_2510_13797_b200.workloads import make_workload
     torch.cuda.set_device(0)
     w = make_workload("cfg2")
-    r = make_runner(w, torch.device("cuda", 0))
+    r = make_runner(w, torch.device("cuda", 0), paired=not args.no_pair)
     K = max(16, (min(args.steps, 1024) // 16) * 16)
     t_mid = ((w.steps - K) // 2 // 16) * 16
     r.reset_to(t_mid - 32)
@@ -429,7 +429,9 @@ def report_ragged(args):
     all_slots = np.arange(Bn)
     cache.bc_seq_open(i32(all_slots), i32(P), i32(C))
     cache.bc_prefill(0, i32(all_slots), i32(cu), int(cu[-1]), pk, pv)
-    out, outb = cache.new_out(Bn), cache.new_out(Bn)
+    out, outb, out2 = cache.new_out(Bn), cache.new_out(Bn), cache.new_out(Bn)
+    paired = args.pair        # off by default here: with the small, shrinking batches of this run the paired
+                              # kernel's longer per-tile arithmetic costs more than the saved traffic gains (measured)
     order = np.argsort(T, kind="stable")
     T_max = int(T.max())
     PERIOD = 16                                        # the call pattern of a fixed batch repeats every 16 steps
@@ -441,11 +443,17 @@ def report_ragged(args):
               "groups": []}
         Cl = C[live]
         for ph in range(PERIOD):                       # sequences whose window fills at steps t = ph (mod 16)
-            pos = np.nonzero((ph % Cl) == 0)[0] if ph else np.arange(len(live))
+            fill = ((ph % Cl) == 0) if ph else np.ones(len(live), dtype=bool)
+            pos, rest = np.nonzero(fill)[0], np.nonzero(~fill)[0]
             if len(pos):
                 gi = torch.tensor(live[pos], dtype=torch.int64, device=dev)
-                ep["groups"].append((i32(live[pos]), bq[0].index_select(0, gi), bk[0].index_select(0, gi),
-                                     bv[0].index_select(0, gi)))
+                grp = [i32(live[pos]), bq[0].index_select(0, gi), bk[0].index_select(0, gi), bv[0].index_select(0, gi)]
+                if paired:      # the step's own queries of the two groups (step t uses ring row (t - 1) % 16)
+                    jq = (ph - 1) % ring
+                    pi, ri = torch.tensor(pos, dtype=torch.int64, device=dev), torch.tensor(rest, dtype=torch.int64, device=dev)
+                    grp += [ep["q"][jq].index_select(0, pi).contiguous(),
+                            (i32(live[rest]), ep["q"][jq].index_select(0, ri).contiguous()) if len(rest) else None]
+                ep["groups"].append(tuple(grp))
             else:
                 ep["groups"].append(None)
         return ep
@@ -454,10 +462,18 @@ def report_ragged(args):
         """Decode step t (1-based) of the epoch's batch: append, attend, and the beacon step where due."""
         j = (t - 1) % ring
         cache.bc_append(0, ep["sl"], ep["k"][j], ep["v"][j])
-        cache.bc_decode_attn(0, ep["sl"], ep["q"][j], out, w.sm_scale)
         grp = ep["groups"][t % PERIOD]
+        if grp is not None and paired:
+            # the sequences whose window this token fills: token and beacon queries in one pass; the rest: plain
+            gsl, gq, gk, gv, tq, rest = grp
+            cache.bc_decode_attn_pair(0, gsl, tq, out, gq, outb, w.sm_scale, gk, gv)
+            if rest is not None:
+                cache.bc_decode_attn(0, rest[0], rest[1], out2, w.sm_scale)
+            cache.bc_compress(0, gsl, gk, gv)
+            return
+        cache.bc_decode_attn(0, ep["sl"], ep["q"][j], out, w.sm_scale)
         if grp is not None:
-            gsl, gq, gk, gv = grp
+            gsl, gq, gk, gv = grp[:4]
             cache.bc_decode_attn(0, gsl, gq, outb, w.sm_scale, gk, gv)
             cache.bc_compress(0, gsl, gk, gv)
 
@@ -509,7 +525,8 @@ def report_ragged(args):
         Cl, Pl = C[alive], P[alive]
         kv_entries += int((Pl + (t - 1) // Cl + (t - 1) % Cl + 1).sum())
         full = (t % Cl) == 0
-        kv_entries += int((Pl[full] + (t // Cl[full] - 1) + Cl[full]).sum())
+        if not paired:           # the beacon's second pass over the cache
+            kv_entries += int((Pl[full] + (t // Cl[full] - 1) + Cl[full]).sum())
         if t % 16 == 0 or t == T_max:
             nbp, wl2 = t // Cl, t % Cl
             high_water = max(high_water, int((cd(Pl, ps) + cd(nbp, ps) + cd(wl2, ps)).sum()))
@@ -528,6 +545,7 @@ def report_ragged(args):
         "cache_bytes_high_water": high_water * ps * E, "uncompressed_bytes_high_water": high_water_unc * ps * E,
         "gpu_launches": int(cache.bc_kernel_launches() - n_launch0 + replayed_launches), "host_seconds": host_s,
         "all_pages_returned": True, "graphs": len(graphs),
+        "beacon_steps": "paired with the token's attention (one pass over the cache)" if paired else "second attention pass",
         "note": "between two sequence finishes the batch is fixed and its call pattern repeats every 16 steps: "
                 "those steps run as replays of one CUDA graph per epoch, the rest as plain launches"}))
 
@@ -570,21 +588,29 @@ def report_depth(args):
         cache.bc_prefill(l, slots, cu, Bn * P, pk, pv)
         ins.append((stream.step_chunk(l, 0, ring), stream.beacon_chunk(l, 0, 2)))
         del pk, pv
-    out = cache.new_out(Bn)
+    out, out_b = cache.new_out(Bn), cache.new_out(Bn)
+    paired = not args.no_pair
     state = {"t": 0}
 
     def step(attend=True):
         t = state["t"]; j = t % ring
         for l in range(L):
             (q, k, v), _ = ins[l]
-            if attend and args.fused:
+            if attend and paired and (t + 1) % c == 0:
+                # the token fills the window: per layer append, then token and beacon queries in one pass, then compress
+                _, (bq, bk, bv) = ins[l]
+                m = ((t + 1) // c) % 2
+                cache.bc_append(l, slots, k[j], v[j])
+                cache.bc_decode_attn_pair(l, slots, q[j], out, bq[m], out_b, w.sm_scale, bk[m], bv[m])
+                cache.bc_compress(l, slots, bk[m], bv[m])
+            elif attend and args.fused:
                 cache.bc_decode_step(l, slots, q[j], k[j], v[j], out, w.sm_scale)
             else:
                 cache.bc_append(l, slots, k[j], v[j])
                 if attend:
                     cache.bc_decode_attn(l, slots, q[j], out, w.sm_scale)
         state["t"] = t = t + 1
-        if t % c == 0:
+        if t % c == 0 and not (attend and paired):
             m = (t // c) % 2
             for l in range(L):
                 _, (bq, bk, bv) = ins[l]
@@ -621,11 +647,12 @@ def report_depth(args):
     code, slot, call = cache.bc_poll_error()
     assert code == 0, (code, slot, call)
     reg = sum(entries_attended(P, n, c) for n in range(t_begin + 1, t_begin + K + 1))
-    bea = sum(entries_beacon_query(P, n, c) for n in range(t_begin + 1, t_begin + K + 1) if n % c == 0)
+    bea = 0 if paired else sum(entries_beacon_query(P, n, c) for n in range(t_begin + 1, t_begin + K + 1) if n % c == 0)
     kv = (reg + bea) * E * Bn * L
     end_entries = P + T // c + T % c
     line = {
         "workload": "depth: 28 layers, B=256, 12/2 heads, D=128, P=512, T=8192, c=8, page 8",
+        "beacon_steps": "paired with the token's attention (one pass over the cache per layer)" if paired else "second attention pass",
         "steps": K, "t_window": [t_begin, t_begin + K], "ms_per_step": ms / K,
         "attention_tokens_per_s": Bn * K / (ms * 1e-3), "layer_tokens_per_s": Bn * K * L / (ms * 1e-3),
         "kv_bytes_per_step": kv / K, "kv_gbs": kv / (ms * 1e-3) / 1e9,
@@ -839,6 +866,7 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-pair", action="store_true", help="beacon steps as a second attention pass instead of bc_decode_attn_pair")
+    ap.add_argument("--pair", action="store_true", help="ragged workload: pair the beacon steps too (off by default there)")
     ap.add_argument("--fused", action="store_true", help="depth workload: regular steps through bc_decode_step (append + attention in one launch per layer)")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")

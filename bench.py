@@ -810,7 +810,7 @@ def report_model(args):
     Bn, N, reps = 64, 512 if args.steps >= 512 else 128, 3
     rows, base, weights = [], None, None
     for c in (1,) + RATIOS:
-        m = ToyDecoder(Bn, c, gen_len=reps * N + 128, device="cuda", weights=weights)
+        m = ToyDecoder(Bn, c, gen_len=reps * N + 128, device="cuda", weights=weights, paired=not args.no_pair)
         weights = m.weights                                 # one set of weights, at one address, for every ratio
         m.capture()
         torch.cuda.synchronize()
@@ -830,7 +830,8 @@ def report_model(args):
         del m
         torch.cuda.empty_cache()
     print(json.dumps({"workload": f"model: random-weight decoder of the 1.5B shape, batch {Bn}, prompt 512, {N} generated tokens "
-                                  "per sequence, one CUDA graph per token step and per beacon step",
+                                  "per sequence, one CUDA graph per token step and per beacon step"
+                                  + ("" if args.no_pair else "; the beacon is encoded in the same 2-token pass as the token that fills the window"),
                       "paper_latency_table_qwen_sr": {"2": 1.990, "4": 1.546, "8": 1.593, "16": 1.646, "32": 1.468},
                       "rows": rows}))
 

@@ -10,7 +10,11 @@ embedding, the LM head and greedy sampling -- are plain PyTorch operators standi
 (random weights: the token stream is meaningless, the shapes and the data flow are real).  Every
 sampled token is fed back, and when a window fills, the beacon token's forward pass runs through
 the same layers: its query attends with its own K/V as the extra entry, then the window is evicted
-(Algorithm 1).  One decode step (and one beacon step) is captured in a CUDA graph and replayed.
+(Algorithm 1).  By default the beacon does not get a pass of its own: it is fed together with the
+token that fills the window, as a 2-token forward pass (the beacon's input is a fixed special token,
+so nothing it needs depends on that token's output), and per layer the two query sets share one pass
+over the cache (bc_decode_attn_pair).  One decode step (and one fill or beacon step) is captured in a
+CUDA graph and replayed.
 """
 from __future__ import annotations
 
@@ -23,8 +27,10 @@ from . import binding as B
 
 class ToyDecoder:
     def __init__(self, batch, c, gen_len, prompt_len=512, layers=28, hidden=1536, q_heads=12, kv_heads=2, head_dim=128,
-                 mlp=8960, vocab=151936, device="cuda", seed=0, weights=None):
+                 mlp=8960, vocab=151936, device="cuda", seed=0, weights=None, paired=True):
         self.B, self.c, self.L, self.H = batch, c, layers, hidden
+        self.paired = paired    # True: the beacon is encoded together with the token that fills the window
+                                # (one 2-token forward pass, bc_decode_attn_pair), False: in a forward pass of its own
         self.Hq, self.Hkv, self.D, self.V = q_heads, kv_heads, head_dim, vocab
         self.dev = torch.device(device)
         g = torch.Generator(device=self.dev); g.manual_seed(seed)
@@ -55,6 +61,7 @@ class ToyDecoder:
         self.tok = torch.zeros(batch, dtype=torch.int64, device=self.dev)      # last sampled token
         self.pos = torch.full((1,), prompt_len, dtype=torch.int64, device=self.dev)
         self.attn_out = self.cache.new_out(batch)
+        self.attn_out2 = self.cache.new_out(2 * batch)         # the paired step: token rows, then beacon rows
         self.inv_freq = 1.0 / (10000.0 ** (torch.arange(0, head_dim, 2, device=self.dev, dtype=torch.float32) / head_dim))
         self.scale = 1.0 / math.sqrt(head_dim)
         self.graph_tok = self.graph_bea = None
@@ -64,8 +71,9 @@ class ToyDecoder:
     def _norm(x):
         return (x.float() * torch.rsqrt(x.float().pow(2).mean(-1, keepdim=True) + 1e-6)).to(torch.bfloat16)
 
-    def _rope(self, x):
-        ang = self.pos.float() * self.inv_freq
+    def _rope(self, x, offset=None):
+        pos = self.pos.float() if offset is None else (self.pos.float() + offset).view(-1, 1, 1)
+        ang = pos * self.inv_freq
         cos, sin = ang.cos(), ang.sin()
         x1, x2 = x.float()[..., 0::2], x.float()[..., 1::2]
         return torch.stack((x1 * cos - x2 * sin, x1 * sin + x2 * cos), dim=-1).flatten(-2).to(torch.bfloat16)
@@ -90,6 +98,34 @@ class ToyDecoder:
             h = h + (torch.nn.functional.silu(gate) * up) @ self.wdown[l]
         return h
 
+    def _forward_pair(self):
+        """The token that fills the window and the beacon as one 2-token pass: rows [0, B) are the
+        tokens (position pos), rows [B, 2B) the beacons (position pos + 1).  Per layer the token's entry
+        is appended, both query sets attend in one pass over the cache (the beacon also sees its own
+        entry), and the window is evicted."""
+        Bn, Hq, Hkv, D = self.B, self.Hq, self.Hkv, self.D
+        h = self.emb[torch.cat((self.tok, torch.full_like(self.tok, self.V)))]
+        offset = torch.cat((torch.zeros(Bn, device=self.dev), torch.ones(Bn, device=self.dev)))
+        for l in range(self.L):
+            qkv = self._norm(h) @ self.wqkv[l]
+            q = self._rope(qkv[:, :Hq * D].view(-1, Hq, D), offset).contiguous()
+            k = self._rope(qkv[:, Hq * D:(Hq + Hkv) * D].view(-1, Hkv, D), offset).contiguous()
+            v = qkv[:, (Hq + Hkv) * D:].view(-1, Hkv, D).contiguous()
+            self.cache.bc_append(l, self.slots, k[:Bn], v[:Bn])
+            self.cache.bc_decode_attn_pair(l, self.slots, q[:Bn], self.attn_out2[:Bn], q[Bn:], self.attn_out2[Bn:], self.scale,
+                                           k[Bn:], v[Bn:])
+            self.cache.bc_compress(l, self.slots, k[Bn:], v[Bn:])
+            h = h + self.attn_out2.view(-1, Hq * D) @ self.wo[l]
+            gu = self._norm(h) @ self.wgu[l]
+            gate, up = gu.chunk(2, dim=-1)
+            h = h + (torch.nn.functional.silu(gate) * up) @ self.wdown[l]
+        return h[:Bn]
+
+    def _fill_step(self):
+        h = self._forward_pair()
+        self.tok.copy_(torch.argmax(self._norm(h) @ self.head, dim=-1))
+        self.pos.add_(2)
+
     def _token_step(self):
         h = self._forward(self.tok, beacon=False)
         self.tok.copy_(torch.argmax(self._norm(h) @ self.head, dim=-1))
@@ -105,18 +141,19 @@ class ToyDecoder:
         advances the generation by a whole number of windows, so the state stays consistent."""
         warm = self.c if self.c > 1 else 1
         for i in range(1, warm + 1):
-            self._token_step()
-            if self.c > 1 and i % self.c == 0:
-                self._beacon_step()
+            self._step_eager(i)
         torch.cuda.synchronize()
         s = torch.cuda.Stream(); s.wait_stream(torch.cuda.current_stream())
         self.graph_tok = torch.cuda.CUDAGraph()
         with torch.cuda.graph(self.graph_tok, stream=s, capture_error_mode="thread_local"):
             self._token_step()
-        if self.c > 1:
+        if self.c > 1:      # the captures enqueue nothing: the cache state is untouched by them
             self.graph_bea = torch.cuda.CUDAGraph()
             with torch.cuda.graph(self.graph_bea, stream=s, capture_error_mode="thread_local"):
-                self._beacon_step()
+                if self.paired:
+                    self._fill_step()
+                else:
+                    self._beacon_step()
         torch.cuda.current_stream().wait_stream(s)
         self.generate(warm)          # first replays upload the graphs: keep that out of any timing
         torch.cuda.synchronize()
@@ -125,9 +162,22 @@ class ToyDecoder:
     def generate(self, n_tokens):
         """Replays n_tokens token steps (n_tokens a multiple of c), with a beacon step after every c."""
         for i in range(1, n_tokens + 1):
-            self.graph_tok.replay()
-            if self.c > 1 and i % self.c == 0:
-                self.graph_bea.replay()
+            fill = self.c > 1 and i % self.c == 0
+            if fill and self.paired:
+                self.graph_bea.replay()          # the token that fills the window and its beacon, one pass
+            else:
+                self.graph_tok.replay()
+                if fill:
+                    self.graph_bea.replay()
+
+    def _step_eager(self, i):
+        fill = self.c > 1 and i % self.c == 0
+        if fill and self.paired:
+            self._fill_step()
+        else:
+            self._token_step()
+            if fill:
+                self._beacon_step()
 
     def check(self):
         code, slot, call = self.cache.bc_poll_error()

@@ -247,6 +247,7 @@ class _Passes:
         e0.record()
         for _ in range(K):
             self.step_host()
+        self.cache.bc_host_outputs_ready()            # the last outputs' copies, before the closing event
         e1.record()
         torch.cuda.synchronize()
         return e0.elapsed_time(e1)

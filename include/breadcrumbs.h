@@ -87,7 +87,8 @@ enum {
 
 enum {
   BC_FLAG_OUT_F32 = 1u,        /* bc_decode_attn writes fp32 instead of bf16 */
-  BC_FLAG_ATTN_REFERENCE = 2u  /* use the slow one-warp-per-head device kernel (debugging aid) */
+  BC_FLAG_ATTN_REFERENCE = 2u, /* use the slow one-warp-per-head device kernel (debugging aid) */
+  BC_FLAG_HOST_PIPELINED = 4u  /* host-buffer steps: outputs are copied back on a stream of the cache's own, see bc_host_outputs_ready */
 };
 
 typedef struct bc_cache bc_cache; /* opaque host-side handle */
@@ -274,6 +275,14 @@ BC_API bc_status bc_seq_close(bc_cache* cache, const int32_t* slots, int32_t n, 
 BC_API bc_status bc_decode_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                               const void* q_host, const void* k_host, const void* v_host,
                               void* out_host, float sm_scale, void* stream);
+/* With BC_FLAG_HOST_PIPELINED the host-buffer steps copy their outputs back on a stream the cache owns
+ * (from two staging sets used in turn), so the next step's kernels do not wait behind the copy.  The
+ * price: `stream` alone no longer orders the outputs.  out_host of every step issued so far is
+ * complete once bc_host_outputs_ready(cache, stream) has been called and `stream` has passed it (or
+ * after a device-wide synchronisation); without the flag the call does nothing.  At most two steps'
+ * outputs are in flight: the staging set of a step is reused two host-buffer calls later. */
+BC_API bc_status bc_host_outputs_ready(bc_cache* cache, void* stream);
+
 /* The step that fills a window, with host buffers: bc_append of the token, bc_decode_attn_pair for
  * the token and its beacon (one pass over the cache), bc_compress.  Equivalent to
  * bc_decode_step_host followed by bc_compress_step_host; same conventions. */

@@ -20,7 +20,7 @@ BC_OK = 0
 BC_ERR_INVALID_ARG, BC_ERR_BAD_SLOT, BC_ERR_NO_PAGES, BC_ERR_CAPACITY = -1, -2, -3, -4
 BC_ERR_WINDOW_NOT_FULL, BC_ERR_WINDOW_FULL, BC_ERR_ORDER, BC_ERR_CUDA = -5, -6, -7, -8
 BC_ERR_UNSUPPORTED, BC_ERR_TIMEOUT, BC_ERR_TOO_LARGE = -9, -10, -11
-BC_FLAG_OUT_F32, BC_FLAG_ATTN_REFERENCE = 1, 2
+BC_FLAG_OUT_F32, BC_FLAG_ATTN_REFERENCE, BC_FLAG_HOST_PIPELINED = 1, 2, 4
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SLOT", -3: "NO_PAGES", -4: "CAPACITY",
                 -5: "WINDOW_NOT_FULL", -6: "WINDOW_FULL", -7: "ORDER", -8: "CUDA",
                 -9: "UNSUPPORTED", -10: "TIMEOUT", -11: "TOO_LARGE"}
@@ -59,6 +59,7 @@ SYMBOLS = {
     "bc_append": (_I32, [_P, _I32, _P, _I32, _P, _P, _P]),
     "bc_decode_attn": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
     "bc_decode_step": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P]),
+    "bc_host_outputs_ready": (_I32, [_P, _P]),
     "bc_fill_step_host": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _P, _P, _P, _P, _F, _P]),
     "bc_decode_attn_pair": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _F, _P, _P, _P]),
     "bc_decode_attn_static": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _P, _P]),
@@ -164,6 +165,9 @@ class Cache:
     def bc_decode_attn(self, layer, slots, q, out, sm_scale, extra_k=None, extra_v=None, stream=None):
         _check(lib().bc_decode_attn(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(out), sm_scale,
                                     _ptr(extra_k), _ptr(extra_v), _stream(stream)), "bc_decode_attn")
+
+    def bc_host_outputs_ready(self, stream=None):
+        _check(lib().bc_host_outputs_ready(self.handle, _stream(stream)), "bc_host_outputs_ready")
 
     def bc_fill_step_host(self, layer, slots, q, k, v, beacon_q, beacon_k, beacon_v, out, out_beacon, sm_scale, stream=None):
         _check(lib().bc_fill_step_host(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(k), _ptr(v), _ptr(beacon_q),

@@ -33,7 +33,7 @@ MetaLayout meta_layout(const bc_config& c) {
 
 struct WorkLayout {
   size_t append_row, append_pos, compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[2],
-      stage_out, stage_out2,
+      stage_out[2], stage_out2[2],
       total;
 };
 WorkLayout work_layout(const bc_config& c) {
@@ -52,8 +52,10 @@ WorkLayout work_layout(const bc_config& c) {
   l.part_o2 = take(pieces * c.q_heads * c.head_dim * 4);
   // host-buffer entry points: two input staging buffers, each k | v | q packed for the call's batch
   for (int b = 0; b < 2; ++b) l.stage_in[b] = take((size_t)BC_MAX_ATTN_BATCH * (c.q_heads + 2 * c.kv_heads) * c.head_dim * 2);
-  l.stage_out = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
-  l.stage_out2 = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
+  for (int b = 0; b < 2; ++b) {   // two sets of output staging (a set: token output, beacon output)
+    l.stage_out[b] = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
+    l.stage_out2[b] = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
+  }
   l.total = o;
   return l;
 }
@@ -106,6 +108,11 @@ struct bc_cache {
   cudaEvent_t ev_in[2] = {nullptr, nullptr};    // the copies into staging buffer b have been issued up to here
   cudaEvent_t ev_used[2] = {nullptr, nullptr};  // the kernels reading staging buffer b have been issued up to here
   int stage_next = 0;
+  // BC_FLAG_HOST_PIPELINED: outputs leave on a stream of their own from alternating staging sets
+  cudaStream_t out_stream = nullptr;
+  cudaEvent_t ev_kern[2] = {nullptr, nullptr};   // the kernels writing output set b have been issued up to here
+  cudaEvent_t ev_d2h[2] = {nullptr, nullptr};    // the copies out of set b have been issued up to here
+  int out_next = 0;
 };
 
 namespace {
@@ -303,8 +310,11 @@ bc_status bc_cache_destroy(bc_cache* c) {
   for (int b = 0; b < 2; ++b) {
     if (c->ev_in[b]) cudaEventDestroy(c->ev_in[b]);
     if (c->ev_used[b]) cudaEventDestroy(c->ev_used[b]);
+    if (c->ev_kern[b]) cudaEventDestroy(c->ev_kern[b]);
+    if (c->ev_d2h[b]) cudaEventDestroy(c->ev_d2h[b]);
   }
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->out_stream) cudaStreamDestroy(c->out_stream);
   delete c;
   return BC_OK;
 }
@@ -548,7 +558,50 @@ bc_status stage_inputs(bc_cache* c, int32_t n, const void* q_host, const void* k
   return BC_OK;
 }
 
+// Output staging of a host-buffer step.  Plain mode: one set, the copies follow the kernels on `s`.
+// Pipelined mode (BC_FLAG_HOST_PIPELINED): two sets in turn; the copies of a step run on the cache's
+// output stream after its kernels, so the next step's kernels do not wait for them; `s` waits for
+// them only in bc_host_outputs_ready.
+bc_status begin_outputs(bc_cache* c, cudaStream_t s, int* set, void** dout, void** dout2) {
+  *set = 0;
+  if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) {
+    if (!c->out_stream) {
+      BC_CUDA(c, cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking));
+      for (int b = 0; b < 2; ++b) {
+        BC_CUDA(c, cudaEventCreateWithFlags(&c->ev_kern[b], cudaEventDisableTiming));
+        BC_CUDA(c, cudaEventCreateWithFlags(&c->ev_d2h[b], cudaEventDisableTiming));
+      }
+    }
+    *set = c->out_next;
+    c->out_next ^= 1;
+    BC_CUDA(c, cudaStreamWaitEvent(s, c->ev_d2h[*set], 0));   // the set's copies of two steps ago (long done)
+  }
+  *dout = c->work + c->wl.stage_out[*set];
+  *dout2 = c->work + c->wl.stage_out2[*set];
+  return BC_OK;
+}
+bc_status send_outputs(bc_cache* c, cudaStream_t s, int set, void* out_host, const void* dout, void* out2_host,
+                       const void* dout2, size_t bytes) {
+  cudaStream_t cs = s;
+  if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) {
+    BC_CUDA(c, cudaEventRecord(c->ev_kern[set], s));
+    BC_CUDA(c, cudaStreamWaitEvent(c->out_stream, c->ev_kern[set], 0));
+    cs = c->out_stream;
+  }
+  BC_CUDA(c, cudaMemcpyAsync(out_host, dout, bytes, cudaMemcpyDeviceToHost, cs));
+  if (out2_host) BC_CUDA(c, cudaMemcpyAsync(out2_host, dout2, bytes, cudaMemcpyDeviceToHost, cs));
+  if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) BC_CUDA(c, cudaEventRecord(c->ev_d2h[set], cs));
+  return BC_OK;
+}
+
 }  // namespace
+
+bc_status bc_host_outputs_ready(bc_cache* c, void* stream) {
+  if (!c) return BC_ERR_INVALID_ARG;
+  if (c->out_stream)
+    for (int b = 0; b < 2; ++b) BC_CUDA(c, cudaStreamWaitEvent((cudaStream_t)stream, c->ev_d2h[b], 0));
+  return BC_OK;
+}
 
 bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q_host,
                               const void* k_host, const void* v_host, void* out_host, float sm_scale, void* stream) {
@@ -558,17 +611,18 @@ bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, 
   cudaStream_t s = (cudaStream_t)stream;
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
-  void *dq, *dk, *dv, *dout = c->work + c->wl.stage_out;
-  int buf;
+  void *dq, *dk, *dv, *dout, *dout2;
+  int buf, set;
   st = stage_inputs(c, n, q_host, k_host, v_host, s, &buf, &dq, &dk, &dv);
+  if (st) return st;
+  st = begin_outputs(c, s, &set, &dout, &dout2);
   if (st) return st;
   st = bc_append(c, layer, slots, n, dk, dv, stream);
   if (st) return st;
   st = attn_impl(c, layer, slots, n, dq, dout, sm_scale, nullptr, nullptr, s);
   if (st) return st;
   BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
-  BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
-  return BC_OK;
+  return send_outputs(c, s, set, out_host, dout, nullptr, nullptr, ob);
 }
 
 bc_status bc_fill_step_host(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q_host,
@@ -581,11 +635,13 @@ bc_status bc_fill_step_host(bc_cache* c, int32_t layer, const int32_t* slots, in
   cudaStream_t s = (cudaStream_t)stream;
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
-  void *dq, *dk, *dv, *dbq, *dbk, *dbv, *dout = c->work + c->wl.stage_out, *dout2 = c->work + c->wl.stage_out2;
-  int buf, buf2;
+  void *dq, *dk, *dv, *dbq, *dbk, *dbv, *dout, *dout2;
+  int buf, buf2, set;
   st = stage_inputs(c, n, q_host, k_host, v_host, s, &buf, &dq, &dk, &dv);
   if (st) return st;
   st = stage_inputs(c, n, bq_host, bk_host, bv_host, s, &buf2, &dbq, &dbk, &dbv);
+  if (st) return st;
+  st = begin_outputs(c, s, &set, &dout, &dout2);
   if (st) return st;
   st = bc_append(c, layer, slots, n, dk, dv, stream);
   if (st) return st;
@@ -595,9 +651,7 @@ bc_status bc_fill_step_host(bc_cache* c, int32_t layer, const int32_t* slots, in
   if (st) return st;
   BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
   BC_CUDA(c, cudaEventRecord(c->ev_used[buf2], s));
-  BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
-  BC_CUDA(c, cudaMemcpyAsync(out_beacon_host, dout2, ob, cudaMemcpyDeviceToHost, s));
-  return BC_OK;
+  return send_outputs(c, s, set, out_host, dout, out_beacon_host, dout2, ob);
 }
 
 bc_status bc_compress_step_host(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* bq_host,
@@ -608,17 +662,18 @@ bc_status bc_compress_step_host(bc_cache* c, int32_t layer, const int32_t* slots
   cudaStream_t s = (cudaStream_t)stream;
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
-  void *dq, *dk, *dv, *dout = c->work + c->wl.stage_out;
-  int buf;
+  void *dq, *dk, *dv, *dout, *dout2;
+  int buf, set;
   st = stage_inputs(c, n, bq_host, bk_host, bv_host, s, &buf, &dq, &dk, &dv);
+  if (st) return st;
+  st = begin_outputs(c, s, &set, &dout, &dout2);
   if (st) return st;
   st = attn_impl(c, layer, slots, n, dq, dout, sm_scale, dk, dv, s);
   if (st) return st;
   st = bc_compress(c, layer, slots, n, dk, dv, stream);
   if (st) return st;
   BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
-  BC_CUDA(c, cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
-  return BC_OK;
+  return send_outputs(c, s, set, out_host, dout, nullptr, nullptr, ob);
 }
 
 bc_status bc_get_state(bc_cache* c, int32_t slot, bc_seq_state* out, int32_t* pages, int32_t pages_cap, void* stream) {

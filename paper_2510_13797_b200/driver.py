@@ -21,7 +21,7 @@ from .workloads import InputStream
 
 
 class DecodeDriver:
-    def __init__(self, w, device, seed_offset=0, fused=False, paired=True):
+    def __init__(self, w, device, seed_offset=0, fused=False, paired=True, host_pipelined=True):
         self.w, self.dev = w, torch.device(device)
         self.fused = fused                             # True: regular steps through bc_decode_step (one launch)
         self.paired = paired                           # True: the step that fills a window attends for the token and
@@ -38,8 +38,10 @@ class DecodeDriver:
             pages_per_seq = cd(P + T, ps) + 1
         self.pages_per_seq = pages_per_seq
         self.num_pages = Bn * pages_per_seq
+        # host-buffer steps return their outputs on the cache's own stream (bc_host_outputs_ready orders them)
         self.cache = B.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, c, ps, max_seqs=Bn,
-                             num_pages=self.num_pages, max_pages_per_seq=pages_per_seq, device=self.dev)
+                             num_pages=self.num_pages, max_pages_per_seq=pages_per_seq,
+                             flags=B.BC_FLAG_HOST_PIPELINED if host_pipelined else 0, device=self.dev)
         self.slots = torch.arange(Bn, dtype=torch.int32, device=self.dev)
         self.plens = torch.tensor(w.prompt_lens, dtype=torch.int32, device=self.dev)
         self.cu = torch.tensor([0] + list(itertools.accumulate(w.prompt_lens)), dtype=torch.int32, device=self.dev)

@@ -159,3 +159,51 @@ def test_fill_step_host_matches_oracle():
     pair.check_state()
     for s in slots:
         pair.check_content(0, s)
+
+
+def test_host_steps_with_pipelined_outputs():
+    """BC_FLAG_HOST_PIPELINED: the outputs come back on the cache's own stream from two staging sets in
+    turn.  Many steps are issued with nothing in between; the caller's stream is made to wait with
+    bc_host_outputs_ready and is then the only thing synchronised before the outputs are compared."""
+    Hkv, G, D, ps, c = 2, 4, 128, 16, 4
+    n, plens = 3, [200, 9, 64]
+    pair = Pair(1, Hkv, Hkv * G, D, ps, max_seqs=n, num_pages=96, max_pages_per_seq=32, flags=B.BC_FLAG_HOST_PIPELINED)
+    g = _gen(17)
+    slots = list(range(n))
+    assert pair.open(slots, plens, [c] * n) == [OK] * n
+    pair.prefill(0, slots, plens, randn_bf16(g, (sum(plens), Hkv, D), DEV), randn_bf16(g, (sum(plens), Hkv, D), DEV))
+    sl = torch.tensor(slots, dtype=torch.int32, device=DEV)
+    pin = lambda t: t.cpu().pin_memory()
+    stream = torch.cuda.Stream()
+    steps = []
+    for step in range(1, 3 * c + 1):
+        k, v, q = randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv * G, D), DEV)
+        bea = (randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv * G, D), DEV)) if step % c == 0 else None
+        steps.append((pin(k), pin(v), pin(q), None if bea is None else tuple(pin(x) for x in bea)))
+    torch.cuda.synchronize()
+    outs = []
+    with torch.cuda.stream(stream):
+        for k, v, q, bea in steps:
+            out_h = torch.empty((n, Hkv * G, D), dtype=torch.bfloat16).pin_memory()
+            if bea is None:
+                pair.gpu.bc_decode_step_host(0, sl, q, k, v, out_h, 0.1)
+                outs.append((out_h, None))
+            else:
+                out_b = torch.empty((n, Hkv * G, D), dtype=torch.bfloat16).pin_memory()
+                pair.gpu.bc_fill_step_host(0, sl, q, k, v, bea[2], bea[0], bea[1], out_h, out_b, 0.1)
+                outs.append((out_h, out_b))
+        pair.gpu.bc_host_outputs_ready()
+    stream.synchronize()                      # only the caller's stream
+    for (k, v, q, bea), (out_h, out_b) in zip(steps, outs):
+        assert pair.model.append(slots) == [OK] * n
+        for i, s in enumerate(slots):
+            pair.seqs[s].append(0, f64(k)[i], f64(v)[i])
+        assert_close(out_h, np.stack([pair.seqs[s].attend(0, f64(q)[i], 0.1) for i, s in enumerate(slots)]), "pipelined token rows")
+        if bea is not None:
+            bk, bv, bq = bea
+            assert_close(out_b, np.stack([pair.seqs[s].beacon_attend(0, f64(bq)[i], f64(bk)[i], f64(bv)[i], 0.1)
+                                          for i, s in enumerate(slots)]), "pipelined beacon rows")
+            assert pair.model.compress(slots) == [OK] * n
+            for i, s in enumerate(slots):
+                pair.seqs[s].compress(0, f64(bk)[i], f64(bv)[i])
+    pair.check_state()

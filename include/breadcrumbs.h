@@ -135,7 +135,9 @@ BC_API bc_status bc_cache_query_bytes(const bc_config* cfg, size_t* pool_bytes, 
 BC_API bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* workspace,
                           void* stream, bc_cache** out);
 
-/* Frees the host handle only. */
+/* Frees the host handle (and the streams and events the host-buffer entry points created, after
+ * waiting for the copies still running on them).  pool, meta and workspace stay the caller's; work
+ * the caller enqueued on its own streams is not waited for. */
 BC_API bc_status bc_cache_destroy(bc_cache* cache);
 
 /* Algorithm 1, initialisation: opens n sequence slots with their prompt lengths and compression

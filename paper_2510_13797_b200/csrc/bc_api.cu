@@ -306,6 +306,9 @@ bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* wo
 
 bc_status bc_cache_destroy(bc_cache* c) {
   if (!c) return BC_ERR_INVALID_ARG;
+  // the cache's own streams touch the caller's workspace: let them drain before the caller may free it
+  if (c->copy_stream) cudaStreamSynchronize(c->copy_stream);
+  if (c->out_stream) cudaStreamSynchronize(c->out_stream);
   for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
   for (int b = 0; b < 2; ++b) {
     if (c->ev_in[b]) cudaEventDestroy(c->ev_in[b]);

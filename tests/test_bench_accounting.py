@@ -22,3 +22,27 @@ def test_entries_attended_equal_the_literal_cache_length():
 def test_traffic_table_covers_the_sweep():
     assert set(bench.TRAFFIC_OVER_ALGORITHMIC) == set(bench.RATIOS)
     assert all(0.9 < v <= 1.0 for v in bench.TRAFFIC_OVER_ALGORITHMIC.values())
+
+
+def test_percentiles_of_window_times():
+    assert bench._percentiles([]) is None
+    assert bench._percentiles([3.0]) == [3.0, 3.0, 1]
+    xs = [float(i) for i in range(1, 101)]
+    assert bench._percentiles(xs) == [50.0, 99.0, 100]
+
+
+def test_paired_steps_read_the_cache_once():
+    """With the beacon's queries riding on the token's pass, a window-fill step reads what the token
+    reads and nothing more; unpaired, the beacon's pass reads the same stored entries again."""
+    class R(bench._Passes):
+        pass
+    r = R()
+    r.P, r.c, r.n = 512, 4, 64
+    r.w = type("W", (), {"entry_bytes": 4096})()
+    r.paired = False
+    reg, bea = r.kv_bytes(8, 8)
+    assert reg == sum(bench.entries_attended(512, n, 4) for n in range(9, 17)) * 4096 * 64
+    assert bea == sum(bench.entries_beacon_query(512, n, 4) for n in (12, 16)) * 4096 * 64
+    assert all(bench.entries_beacon_query(512, n, 4) == bench.entries_attended(512, n, 4) for n in (12, 16))
+    r.paired = True
+    assert r.kv_bytes(8, 8) == (reg, 0)

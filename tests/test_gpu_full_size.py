@@ -101,6 +101,47 @@ def test_sweep_mid_generation_fused_step():
     drv.check_error()
 
 
+@pytest.mark.parametrize("c,paired", [(2, True), (16, True), (16, False), (32, True)])
+def test_sweep_window_replayed_as_cuda_graph(c, paired):
+    """The launch configuration the benchmark times: whole windows of steps captured once as a CUDA
+    graph and replayed.  A replay feeds the inputs of the captured steps again, so the captured span
+    is a whole number of input periods (the step inputs repeat every `ring` steps, the beacons every
+    4 windows): then the replayed generation is the one the oracle rebuilds from the seeds.  After
+    three replays the outputs left by the last step (it fills a window: token rows and beacon rows,
+    paired or as two passes) and the bookkeeping must be those of the oracle for that step."""
+    w = make_workload("sweep", c=c)
+    drv = DecodeDriver(w, DEV, paired=paired)
+    span = math.lcm(drv.ring, 4 * c)
+    t0 = (w.steps // 2 // span) * span
+    drv.reset_to(t0)
+    for _ in range(span):                                # one eager span: warms every kernel
+        drv.step()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    t_save = drv.t
+    with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+        for _ in range(span):
+            drv.step()
+    drv.t = t_save                                       # the capture enqueued nothing
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        graph.replay()
+        drv.t += span
+    torch.cuda.synchronize()
+    drv.check_error()
+    t = drv.t                                            # the last replayed step; it filled the window
+    assert t % c == 0
+    scale, b = w.sm_scale, (t // c) % 4
+    for s in (0, 29, 63):
+        K, V = live_kv(drv, s, t)
+        assert_close(drv.out[s], attention(f64(drv.q[(t - 1) % drv.ring, s]), K, V, scale), f"graph c={c}: step {t} seq {s}")
+        Kb = np.concatenate([K, f64(drv.bk[b, s])[None]]); Vb = np.concatenate([V, f64(drv.bv[b, s])[None]])
+        assert_close(drv.out_b[s], attention(f64(drv.bq[b, s]), Kb, Vb, scale), f"graph c={c}: beacon rows at step {t} seq {s}")
+    check_lengths_and_conservation(drv)
+
+
 def test_sweep_uncompressed_mid_generation():
     w = make_workload("sweep", c=1)
     drv = DecodeDriver(w, DEV)

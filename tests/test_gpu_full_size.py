@@ -142,6 +142,29 @@ def test_sweep_window_replayed_as_cuda_graph(c, paired):
     check_lengths_and_conservation(drv)
 
 
+def test_sweep_host_buffer_steps_full_size():
+    """The end-to-end leg of the benchmark: host-buffer steps (packed pinned inputs on the cache's copy
+    stream, pipelined outputs) at the sweep's size, c = 4, across a window-fill step."""
+    w = make_workload("sweep", c=4)
+    drv = DecodeDriver(w, DEV)
+    t0 = (w.steps // 2 // 16) * 16 + 1
+    drv.reset_to(t0)
+    for _ in range(3):                                   # steps t0+1 .. t0+3; the last one fills the window (paired)
+        drv.step_host()
+    drv.cache.bc_host_outputs_ready()
+    torch.cuda.synchronize()
+    drv.check_error()
+    t = drv.t
+    assert t % 4 == 0
+    scale, b = w.sm_scale, (t // 4) % 4
+    for s in (1, 33, 62):
+        K, V = live_kv(drv, s, t)
+        assert_close(drv.h["out"][s], attention(f64(drv.q[(t - 1) % drv.ring, s]), K, V, scale), f"host step {t} seq {s}")
+        Kb = np.concatenate([K, f64(drv.bk[b, s])[None]]); Vb = np.concatenate([V, f64(drv.bv[b, s])[None]])
+        assert_close(drv.h["out_b"][s], attention(f64(drv.bq[b, s]), Kb, Vb, scale), f"host step {t} seq {s}: beacon rows")
+    check_lengths_and_conservation(drv)
+
+
 def test_sweep_uncompressed_mid_generation():
     w = make_workload("sweep", c=1)
     drv = DecodeDriver(w, DEV)

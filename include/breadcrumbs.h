@@ -35,6 +35,13 @@
  *    per layer (a forward pass computes layer l + 1's inputs from layer l's output, so this form
  *    serves replays and measurements, not a model).
  *  - A batch must not name the same slot twice.
+ *  - Overlap: the bookkeeping kernels of bc_append and bc_compress touch only the cache's metadata
+ *    and are launched with programmatic stream serialisation: they may begin while the kernel
+ *    enqueued just before them on `stream` is still finishing, provided that kernel releases its
+ *    dependents early.  This library's attention kernels do (once they have read the lengths they
+ *    need), ordinary kernels do not, so for them nothing changes.  The one thing these bookkeeping
+ *    kernels read from the caller is `slots`: it must not be written by a kernel that releases its
+ *    dependents early.  Everything else (K/V rows, queries, outputs) keeps plain stream order.
  *
  * Store layout (owned by the library inside the caller's `pool` buffer)
  *    pool[layer][page][slot_in_page][K|V][kv_head][head_dim] bf16: one token's entry of one layer

@@ -435,9 +435,28 @@ cudaError_t bc_launch_open(const BcMeta& m, const int32_t* slots, const int32_t*
   k_open<<<1, kBookThreads, 0, s>>>(m, slots, plens, cs, n, call);
   return cudaGetLastError();
 }
+// Launch of a bookkeeping kernel that touches nothing but the metadata (no K/V rows in the same
+// launch): with programmatic stream serialisation, so that it may begin while the attention kernel
+// enqueued before it -- which has read all the lengths it needs by the time it lets dependents go --
+// is still finishing its last blocks.  It waits for nothing of that kernel: it reads no output of it.
+// After any other predecessor the attribute changes nothing (no early trigger, ordinary order).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_book_overlapped(void (*kernel)(KArgs...), cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(1); cfg.blockDim = dim3(kBookThreads); cfg.dynamicSmemBytes = 0; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                   int32_t* dst_pos, const BcGeom& g, uint8_t* pool_layer, const void* k, const void* v,
                                   cudaStream_t s) {
+  if (k == nullptr)   // the rows follow in a launch of their own (ordinary order: it waits for everything before it)
+    return launch_book_overlapped(k_append_book, s, m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)nullptr,
+                                  (const uint8_t*)nullptr);
   k_append_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)k,
                                            (const uint8_t*)v);
   return cudaGetLastError();
@@ -445,6 +464,9 @@ cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, 
 cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                     int32_t* dst_pos, int phase, const BcGeom& g, uint8_t* pool_layer, const void* k,
                                     const void* v, cudaStream_t s) {
+  if (k == nullptr)
+    return launch_book_overlapped(k_compress_book, s, m, slots, n, call, dst_row, dst_pos, phase, g, pool_layer,
+                                  (const uint8_t*)nullptr, (const uint8_t*)nullptr);
   k_compress_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, phase, g, pool_layer,
                                              (const uint8_t*)k, (const uint8_t*)v);
   return cudaGetLastError();

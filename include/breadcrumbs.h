@@ -41,7 +41,9 @@
  *    dependents early.  This library's attention kernels do (once they have read the lengths they
  *    need), ordinary kernels do not, so for them nothing changes.  The one thing these bookkeeping
  *    kernels read from the caller is `slots`: it must not be written by a kernel that releases its
- *    dependents early.  Everything else (K/V rows, queries, outputs) keeps plain stream order.
+ *    dependents early.  Such a bookkeeping kernel does not end before the kernel it overtook has
+ *    ended, so everything else (K/V rows, queries, outputs, the caller's own kernels) keeps plain
+ *    stream order.
  *
  * Store layout (owned by the library inside the caller's `pool` buffer)
  *    pool[layer][page][slot_in_page][K|V][kv_head][head_dim] bf16: one token's entry of one layer

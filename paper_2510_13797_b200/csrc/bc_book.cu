@@ -95,12 +95,20 @@ k_open(BcMeta m, const int32_t* __restrict__ slots, const int32_t* __restrict__ 
   if (threadIdx.x == 0) *m.free_top = top0 - sh_used;
 }
 
+// Last statement of a bookkeeping kernel that may have started before the kernel ahead of it in the
+// stream had finished (programmatic stream serialisation): it ends only when that kernel has ended,
+// so that whatever is enqueued next -- above all the kernels that write K/V rows, possibly into pages
+// a compression has just recycled -- comes after BOTH, as plain stream order would have it.  Returns
+// at once when nothing was overtaken.
+__device__ __forceinline__ void wait_for_overtaken_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __global__ void __launch_bounds__(kBookThreads, 1)
 k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
               int32_t* dst_row, int32_t* dst_pos, BcGeom g, uint8_t* pool_layer, const uint8_t* k, const uint8_t* v) {
   append_book_block(m, slots, n, call, dst_row, dst_pos);
   __syncthreads();
   if (k != nullptr) block_write_rows(g, pool_layer, dst_row, dst_pos, k, v, n);  // layer 0's rows, same launch
+  wait_for_overtaken_kernel();
 }
 
 // phase & 1: validate, allocate the beacon slot, fill dst_row/dst_pos (dst_row < 0: item failed).
@@ -183,6 +191,7 @@ k_compress_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call
   __syncthreads();
   if (threadIdx.x == 0) *m.free_top = top;
   if (k != nullptr) block_write_rows(g, pool_layer, dst_row, dst_pos, k, v, n);  // the beacon rows, same launch
+  wait_for_overtaken_kernel();
 }
 
 __global__ void __launch_bounds__(kBookThreads, 1)

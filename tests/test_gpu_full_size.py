@@ -165,6 +165,29 @@ def test_sweep_host_buffer_steps_full_size():
     check_lengths_and_conservation(drv)
 
 
+def test_sweep_c2_long_run_content_bit_exact():
+    """400 steps back to back at c = 2 with pages of 2 entries: a window page is recycled at every
+    second step while the next step's bookkeeping may already run under the attention kernel's last
+    blocks.  Nothing may be overwritten early: the last outputs and the stored content of sampled
+    sequences (every prompt entry, beacon and window token, bit for bit) must be the oracle's."""
+    w = make_workload("sweep", c=2)
+    drv = DecodeDriver(w, DEV)
+    t0 = (w.steps // 2 // 16) * 16
+    drv.reset_to(t0)
+    for _ in range(399):
+        drv.step()
+    seqs = [0, 31, 63]
+    check_step(drv, seqs, "c=2 long run")               # step t0 + 400: fills a window (paired attention, then compress)
+    drv.check_error()
+    t = drv.t
+    for s in seqs:
+        K, V = live_kv(drv, s, t + 1)                   # what step t + 1 would read, minus its own new token
+        k, v = drv.cache.bc_export_seq(0, s, K.shape[0])
+        n_live = closed_form_length(drv.P, t, 2)
+        assert np.array_equal(f64(k)[:n_live], K[:n_live]) and np.array_equal(f64(v)[:n_live], V[:n_live]), f"content of sequence {s}"
+    check_lengths_and_conservation(drv)
+
+
 def test_sweep_uncompressed_mid_generation():
     w = make_workload("sweep", c=1)
     drv = DecodeDriver(w, DEV)

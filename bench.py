@@ -114,11 +114,11 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------ one ratio on the GPU
-def make_runner(w, device, seed_offset=0, paired=True):
+def make_runner(w, device, seed_offset=0, paired=True, fused=False):
     """A DecodeDriver (one cache, batch B at ratio c, driven through the C ABI) plus the timed passes."""
     import torch
     from paper_2510_13797_b200.driver import DecodeDriver
-    r = type("RatioRunner", (_Passes, DecodeDriver), {})(w, device, seed_offset, paired=paired)
+    r = type("RatioRunner", (_Passes, DecodeDriver), {})(w, device, seed_offset, fused=fused, paired=paired)
     r.torch = torch
     return r
 
@@ -921,7 +921,7 @@ def main():
     for c in sweep:
         w = make_workload("sweep", c=c)
         T = w.steps
-        r = make_runner(w, dev, seed_offset=sharding.rank_seed_offset(0, rank), paired=not args.no_pair)
+        r = make_runner(w, dev, seed_offset=sharding.rank_seed_offset(0, rank), paired=not args.no_pair, fused=args.fused)
         cyc = c if c > 1 else 16
         t_mid = max(0, ((T - K) // 2 // cyc) * cyc)
         # pass A: device-resident inputs, CUDA-graph replays: the headline time

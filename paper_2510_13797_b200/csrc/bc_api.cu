@@ -32,7 +32,7 @@ MetaLayout meta_layout(const bc_config& c) {
 }
 
 struct WorkLayout {
-  size_t append_row, append_pos, compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[2],
+  size_t append_row[2], append_pos[2], compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[2],
       stage_out[2], stage_out2[2],
       total;
 };
@@ -42,7 +42,10 @@ WorkLayout work_layout(const bc_config& c) {
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
   const size_t seq = (size_t)c.max_seqs * 4;
   const size_t pieces = BC_MAX_ATTN_CTAS + BC_MAX_ATTN_BATCH;
-  l.append_row = take(seq); l.append_pos = take(seq); l.compress_row = take(seq); l.compress_pos = take(seq);
+  // two sets of row destinations of bc_append, used by alternate steps: a fused attention kernel may
+  // still read one while the next step's bookkeeping already fills the other
+  for (int b = 0; b < 2; ++b) { l.append_row[b] = take(seq); l.append_pos[b] = take(seq); }
+  l.compress_row = take(seq); l.compress_pos = take(seq);
   l.restore_ok = take(seq); l.restore_bea = take(seq + 4);
   l.tickets = take(BC_MAX_ATTN_BATCH * 4);
   l.book_flag = take(4);
@@ -99,6 +102,7 @@ struct bc_cache {
   int append_next_layer;    // per-layer ordering of bc_append
   int compress_next_layer;  // per-layer ordering of bc_compress
   int restore_next_layer = 0;   // per-layer ordering of bc_restore
+  int append_set = 0;           // which set of append row destinations the current step uses (flips on layer 0)
   int last_cuda_error;
   // profiling
   std::vector<cudaEvent_t> ev;
@@ -389,8 +393,9 @@ bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n,
   if (st) return st;
   if (!k || !v || !aligned16(k) || !aligned16(v)) return BC_ERR_INVALID_ARG;
   if (layer != c->append_next_layer) return BC_ERR_ORDER;
-  int32_t* row = work_ptr<int32_t>(c, c->wl.append_row);
-  int32_t* pos = work_ptr<int32_t>(c, c->wl.append_pos);
+  if (layer == 0) c->append_set ^= 1;
+  int32_t* row = work_ptr<int32_t>(c, c->wl.append_row[c->append_set]);
+  int32_t* pos = work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]);
   cudaStream_t s = (cudaStream_t)stream;
   // Small batches: the bookkeeping block also copies the rows and a launch is saved.
   const bool fused = layer == 0 && (size_t)n * c->geom.entry_bytes <= kFusedRowBytes;
@@ -462,14 +467,25 @@ bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32
     if (st) return st;
     return attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s);
   }
+  // The bookkeeping runs as its own one-block kernel, which may start under the previous attention
+  // kernel's last blocks; the rows are written by the attention kernel itself (its service warps),
+  // which takes the new entries from the inputs.  So a step costs one full-size launch and no
+  // row-writing launch.  (The kernel can also run the bookkeeping in its block 0, do_book = 1: that
+  // form starts every other block late and is not used here.)
+  if (layer == 0) {
+    c->append_set ^= 1;
+    BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, ++c->calls, work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
+                                     work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), c->geom, layer_base(c, 0), nullptr,
+                                     nullptr, s));
+    c->launches += 1;
+  }
   BcFusedAppend f;
   f.new_k = k; f.new_v = v;
-  f.dst_row = work_ptr<int32_t>(c, c->wl.append_row);
-  f.dst_pos = work_ptr<int32_t>(c, c->wl.append_pos);
+  f.dst_row = work_ptr<int32_t>(c, c->wl.append_row[c->append_set]);
+  f.dst_pos = work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]);
   f.pool_layer = layer_base(c, layer);
   f.flag = work_ptr<int32_t>(c, c->wl.book_flag);
-  f.do_book = layer == 0 ? 1 : 0;
-  if (layer == 0) ++c->calls;
+  f.do_book = 0;
   f.call = c->calls;
   f.epoch = (int32_t)(c->calls & 0x7fffffff) | 1 << 30;   // never 0, the word's initial value
   st = attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s, &f);

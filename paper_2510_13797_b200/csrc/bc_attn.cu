@@ -385,9 +385,10 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   // below those lengths and never rewritten while they are): a kernel enqueued behind this one with
   // programmatic stream serialisation -- the next step's bookkeeping -- may start on the first SM
   // that frees up instead of after this kernel's last block.  Kernels launched the ordinary way wait
-  // for the whole grid as before.  Not in the fused form: its blocks go on reading the rows' destinations
-  // (dst_row, dst_pos), which the next step's bookkeeping rewrites.
-  if (!FUSED) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // for the whole grid as before.  The fused form goes on reading the rows' destinations (dst_row,
+  // dst_pos); the next step's bookkeeping fills the other of two sets, so it may start early as well --
+  // unless this launch did its own bookkeeping in block 0, whose flag word the next one would reuse.
+  if (!FUSED || !p.f.do_book) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // The block that ran the bookkeeping starts late; it takes no tiles, or it would finish last.
   const int idle = (FUSED && p.f.do_book && gridDim.x > 1) ? 1 : 0;
   const int n_ctas = (int)gridDim.x - idle;

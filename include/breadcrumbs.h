@@ -38,7 +38,9 @@
  *  - Overlap: the bookkeeping kernels of bc_append and bc_compress touch only the cache's metadata
  *    and are launched with programmatic stream serialisation: they may begin while the kernel
  *    enqueued just before them on `stream` is still finishing, provided that kernel releases its
- *    dependents early.  This library's attention kernels do (once they have read the lengths they
+ *    dependents early.  The attention kernels are launched the same way and do their planning (which
+ *    reads the metadata and `slots`, nothing else) before they wait for the kernel ahead of them;
+ *    every other read and every write of theirs comes after that wait.  This library's attention kernels do (once they have read the lengths they
  *    need), ordinary kernels do not, so for them nothing changes.  The one thing these bookkeeping
  *    kernels read from the caller is `slots`: it must not be written by a kernel that releases its
  *    dependents early.  Such a bookkeeping kernel does not end before the kernel it overtook has

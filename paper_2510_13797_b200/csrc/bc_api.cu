@@ -241,7 +241,7 @@ cudaError_t static_scratch_reset_tickets(cudaStream_t s) {
 
 extern "C" {
 
-int32_t bc_version(void) { return 113; }
+int32_t bc_version(void) { return 114; }
 
 const char* bc_status_string(bc_status s) {
   switch (s) {

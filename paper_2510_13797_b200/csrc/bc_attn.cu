@@ -389,6 +389,13 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   // dst_pos); the next step's bookkeeping fills the other of two sets, so it may start early as well --
   // unless this launch did its own bookkeeping in block 0, whose flag word the next one would reuse.
   if (!FUSED || !p.f.do_book) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // This kernel itself may have been started early (it is launched with programmatic stream
+  // serialisation): behind the row-writing kernel of its step, which releases it at once, or behind
+  // another attention launch.  Up to here it has read only the cache's metadata and `slots`; everything
+  // else -- the pool rows of this step, q, the extra entry, the partial buffers and tickets it shares
+  // with the launch before it -- is touched only after the kernel ahead has ended.  So the plan above
+  // (three dependent trips to memory) runs under the predecessor instead of after it.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // The block that ran the bookkeeping starts late; it takes no tiles, or it would finish last.
   const int idle = (FUSED && p.f.do_book && gridDim.x > 1) ? 1 : 0;
   const int n_ctas = (int)gridDim.x - idle;
@@ -1011,8 +1018,13 @@ FastDiv make_fast_div(uint32_t d) {
 
 template <int D, bool G8, bool FUSED, bool PAIR = false>
 cudaError_t launch_pipe(const PipeParams& p, cudaStream_t s) {
-  k_attn_pipe<D, G8, FUSED, PAIR><<<p.a.ctas, kPipeThreads, PipeSmem<D>::kTotal, s>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.a.ctas); cfg.blockDim = dim3(kPipeThreads); cfg.dynamicSmemBytes = PipeSmem<D>::kTotal; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;   // see the kernel: it waits for its predecessor after its plan
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_attn_pipe<D, G8, FUSED, PAIR>, p);
 }
 
 }  // namespace

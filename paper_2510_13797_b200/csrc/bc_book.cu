@@ -238,6 +238,8 @@ k_close(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call) {
 __global__ void k_write_rows(BcGeom g, uint8_t* __restrict__ pool_layer, const int32_t* __restrict__ dst_row,
                              const int32_t* __restrict__ dst_pos, const uint8_t* __restrict__ k,
                              const uint8_t* __restrict__ v, int n) {
+  // the attention kernel of the step may start planning now; it waits for this kernel before it reads a row
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int i = blockIdx.x;
   const int row = dst_row[i];
   if (row < 0) return;

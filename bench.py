@@ -805,14 +805,14 @@ def report_model(args):
     (28 layers, hidden 1536, 12/2 heads, D 128, MLP 8960, vocabulary 151,936; batch 64, prompt 512):
     time to generate N tokens per sequence at ratio c relative to the uncompressed cache -- the
     protocol of the paper's latency table.  The non-attention layers are PyTorch operators."""
-    import torch
-    from paper_2510_13797_b200.model_harness import ToyDecoder
-    torch.cuda.set_device(0)
     Bn, N, reps = 64, 512 if args.steps >= 512 else 128, 3
-    rows, base, weights = [], None, None
-    for c in (1,) + RATIOS:
-        m = ToyDecoder(Bn, c, gen_len=reps * N + 128, device="cuda", weights=weights, paired=not args.no_pair)
-        weights = m.weights                                 # one set of weights, at one address, for every ratio
+    if args.model_ratio is not None:
+        # one ratio, in a process of its own (see below): prints its row and nothing else
+        import torch
+        from paper_2510_13797_b200.model_harness import ToyDecoder
+        torch.cuda.set_device(0)
+        c = args.model_ratio
+        m = ToyDecoder(Bn, c, gen_len=reps * N + 128, device="cuda", paired=not args.no_pair)
         m.capture()
         torch.cuda.synchronize()
         times = []
@@ -825,11 +825,26 @@ def report_model(args):
             times.append(e0.elapsed_time(e1))
         st = m.check()
         ms = min(times)
-        base = ms if c == 1 else base
-        rows.append({"c": c, "ms": ms, "ms_per_token": ms / N, "tokens_per_s": Bn * N / (ms * 1e-3),
-                     "latency_vs_uncompressed": ms / base, "ms_all": times, "cache_entries_end": st["prompt_len"] + st["n_beacons"] + st["window_len"]})
-        del m
-        torch.cuda.empty_cache()
+        print(json.dumps({"c": c, "ms": ms, "ms_per_token": ms / N, "tokens_per_s": Bn * N / (ms * 1e-3), "ms_all": times,
+                          "cache_entries_end": st["prompt_len"] + st["n_beacons"] + st["window_len"]}))
+        return
+    # Every ratio runs in a fresh process.  The PyTorch part of a step is some 1100 small kernels in
+    # one CUDA graph, and in a process that has already built and dropped a decoder the same graph can
+    # replay with about 0.5 us more between consecutive kernels (same kernel times, 12 % more per
+    # token): more than the differences between ratios that this protocol is after.
+    rows, base = [], None
+    for c in (1,) + RATIOS:
+        cmd = [sys.executable, os.path.abspath(__file__), "--workload", "model", "--model-ratio", str(c), "--steps", str(args.steps)]
+        if args.no_pair:
+            cmd.append("--no-pair")
+        child = subprocess.run(cmd, capture_output=True, text=True)
+        if child.returncode != 0:
+            sys.stderr.write(child.stderr[-2000:])
+            raise SystemExit(f"model workload: the run at c = {c} exited {child.returncode}")
+        row = json.loads(child.stdout.strip().splitlines()[-1])
+        base = row["ms"] if c == 1 else base
+        row["latency_vs_uncompressed"] = row["ms"] / base
+        rows.append(row)
     print(json.dumps({"workload": f"model: random-weight decoder of the 1.5B shape, batch {Bn}, prompt 512, {N} generated tokens "
                                   "per sequence, one CUDA graph per token step and per beacon step"
                                   + ("" if args.no_pair else "; the beacon is encoded in the same 2-token pass as the token that fills the window"),
@@ -872,6 +887,7 @@ def main():
     ap.add_argument("--fused", action="store_true", help="depth workload: regular steps through bc_decode_step (append + attention in one launch per layer)")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
+    ap.add_argument("--model-ratio", type=int, default=None, help=argparse.SUPPRESS)   # model workload: one ratio (child process)
     ap.add_argument("--workload", default="sweep", choices=["sweep", "cfg2", "ragged", "depth", "maskform", "distill", "model"],
                     help="sweep (default): the benchmark line; cfg2 / ragged / depth: a report line for that "
                          "benchmark configuration (1 GPU)")

@@ -1024,10 +1024,10 @@ def main():
         line["batch_scaling"] = batch_scaling(dev, peak)
     if not args.no_cpu_baseline:
         w = make_workload("sweep", c=16)
-        wall, tok, cpu = oracle_sample(w, w.steps // 2, 16, 8)
+        wall, tok, cpu = oracle_sample(w, w.steps // 2, 64, 24)     # about ten seconds of CPU work
         line["cpu_baseline"] = {"value": tok / wall, "unit": "tokens/s", "cores": max(1, round(cpu / wall)),
                                 "kind": "oracle",
-                                "sample": "16 of 64 sequences, 8 decode steps at c=16, cache at generation step 8192"}
+                                "sample": "64 of 64 sequences, 24 decode steps (one of them fills a window) at c=16, cache at generation step 8192"}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

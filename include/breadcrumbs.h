@@ -277,7 +277,8 @@ BC_API bc_status bc_seq_close(bc_cache* cache, const int32_t* slots, int32_t n, 
 
 /* ---- end-to-end helpers with HOST buffers (pinned memory recommended) ------------------------
  * One decode step of one layer: copies q, k, v to device staging inside `workspace`, runs
- * bc_append + bc_decode_attn, copies out back.  n <= 512.  Asynchronous: out_host is valid, and the
+ * bc_decode_step (the append and the attention of the step; same ordering rule over the layers),
+ * copies out back.  n <= 512.  Asynchronous: out_host is valid, and the
  * three input buffers may be reused, once `stream` has passed the call.  The inputs are copied on a
  * stream the cache owns (created by the first such call, which therefore must not sit inside a
  * stream capture) into one of two staging buffers, so a call's inputs travel while the previous

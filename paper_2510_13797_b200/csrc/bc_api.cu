@@ -636,9 +636,7 @@ bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, 
   if (st) return st;
   st = begin_outputs(c, s, &set, &dout, &dout2);
   if (st) return st;
-  st = bc_append(c, layer, slots, n, dk, dv, stream);
-  if (st) return st;
-  st = attn_impl(c, layer, slots, n, dq, dout, sm_scale, nullptr, nullptr, s);
+  st = bc_decode_step(c, layer, slots, n, dq, dk, dv, dout, sm_scale, stream);   // two launches instead of three
   if (st) return st;
   BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
   return send_outputs(c, s, set, out_host, dout, nullptr, nullptr, ob);

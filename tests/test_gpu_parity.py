@@ -274,6 +274,59 @@ def test_reference_kernel_and_f32_output_agree():
         run_decode(pair, [0, 1], [100, 37], [c, c], 24, seed=13, sm_scale=1.0 / math.sqrt(D), check_state_every=8)
 
 
+def test_host_buffer_steps_over_two_layers():
+    """Host-buffer steps of a two-layer cache, layer after layer without synchronising in between:
+    regular steps (bc_decode_step_host) and window-filling steps (bc_fill_step_host)."""
+    L, Hkv, G, D, ps, c = 2, 2, 4, 128, 4, 3
+    n, plens = 5, [33, 0, 18, 7, 64]
+    pair = Pair(L, Hkv, Hkv * G, D, ps, max_seqs=n, num_pages=160, max_pages_per_seq=32)
+    g = _gen(23)
+    slots = list(range(n))
+    pair.open(slots, plens, [c] * n)
+    for l in range(L):
+        pair.prefill(l, slots, plens, randn_bf16(g, (sum(plens), Hkv, D), DEV), randn_bf16(g, (sum(plens), Hkv, D), DEV))
+    sl = torch.tensor(slots, dtype=torch.int32, device=DEV)
+    pin = lambda t: t.cpu().pin_memory()
+    kv = lambda: (randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv * G, D), DEV))
+    for step in range(1, 11):
+        fill = step % c == 0
+        ins = [kv() for _ in range(L)]
+        bea = [kv() for _ in range(L)] if fill else None
+        outs = [torch.empty((n, Hkv * G, D), dtype=torch.bfloat16).pin_memory() for _ in range(L)]
+        outs_b = [torch.empty((n, Hkv * G, D), dtype=torch.bfloat16).pin_memory() for _ in range(L)]
+        host = [[pin(x) for x in ins[l]] for l in range(L)]
+        host_b = [[pin(x) for x in bea[l]] for l in range(L)] if fill else None
+        for l in range(L):
+            k, v, q = host[l]
+            if fill:
+                bk, bv, bq = host_b[l]
+                pair.gpu.bc_fill_step_host(l, sl, q, k, v, bq, bk, bv, outs[l], outs_b[l], 0.1)
+            else:
+                pair.gpu.bc_decode_step_host(l, sl, q, k, v, outs[l], 0.1)
+        torch.cuda.synchronize()
+        pair._append_ok = pair.model.append(slots)
+        for l in range(L):
+            k, v, q = ins[l]
+            for i, s in enumerate(slots):
+                pair.seqs[s].append(l, f64(k)[i], f64(v)[i])
+            ref = np.stack([pair.seqs[s].attend(l, f64(q)[i], 0.1) for i, s in enumerate(slots)])
+            assert_close(outs[l], ref, f"step {step} layer {l}")
+        if fill:
+            for l in range(L):
+                bk, bv, bq = bea[l]
+                ref = np.stack([pair.seqs[s].beacon_attend(l, f64(bq)[i], f64(bk)[i], f64(bv)[i], 0.1) for i, s in enumerate(slots)])
+                assert_close(outs_b[l], ref, f"beacon of step {step} layer {l}")
+            pair.model.compress(slots)
+            for l in range(L):
+                bk, bv, _ = bea[l]
+                for i, s in enumerate(slots):
+                    pair.seqs[s].compress(l, f64(bk)[i], f64(bv)[i])
+        pair.check_state()
+    for l in range(L):
+        for s in slots:
+            pair.check_content(l, s)
+
+
 def test_host_buffer_entry_points():
     """bc_decode_step_host / bc_compress_step_host: same results as the device-pointer calls."""
     Hkv, G, D, ps, c = 2, 6, 128, 16, 4

@@ -21,7 +21,10 @@
  *  - Hot-path calls only enqueue work on `stream` and return; they never synchronise, so a decode
  *    step can be captured in a CUDA graph.  Argument errors are returned at once.  State errors
  *    found on the device (no free page, window full, ...) make the operation a no-op for that
- *    sequence and are latched (first one wins) in a device status record read by bc_poll_error.
+ *    sequence and are latched in a device status record read by bc_poll_error: the first call
+ *    in which an item fails writes the record, and of that call's failing items the one with the
+ *    lowest batch index is recorded (whichever check it failed); later failures change nothing
+ *    until bc_clear_error.
  *  - Tensors are bf16.  K/V tensors are [n, kv_heads, head_dim]; q and out are
  *    [n, q_heads, head_dim]; query head h reads KV head h / (q_heads / kv_heads).
  *  - Layers: `layer` in [0, layers) addresses one layer.  A sequence's bookkeeping (lengths, page
@@ -35,17 +38,24 @@
  *    per layer (a forward pass computes layer l + 1's inputs from layer l's output, so this form
  *    serves replays and measurements, not a model).
  *  - A batch must not name the same slot twice.
- *  - Overlap: the bookkeeping kernels of bc_append and bc_compress touch only the cache's metadata
- *    and are launched with programmatic stream serialisation: they may begin while the kernel
- *    enqueued just before them on `stream` is still finishing, provided that kernel releases its
- *    dependents early.  The attention kernels are launched the same way and do their planning (which
- *    reads the metadata and `slots`, nothing else) before they wait for the kernel ahead of them;
- *    every other read and every write of theirs comes after that wait.  This library's attention kernels do (once they have read the lengths they
- *    need), ordinary kernels do not, so for them nothing changes.  The one thing these bookkeeping
- *    kernels read from the caller is `slots`: it must not be written by a kernel that releases its
- *    dependents early.  Such a bookkeeping kernel does not end before the kernel it overtook has
- *    ended, so everything else (K/V rows, queries, outputs, the caller's own kernels) keeps plain
- *    stream order.
+ *  - Overlap (programmatic stream serialisation).  Three kinds of kernel of this library may begin
+ *    before the kernel enqueued just ahead of them on `stream` has ended, provided that kernel
+ *    releases its dependents early; after any other kernel (the caller's own, a copy) they keep
+ *    plain stream order.
+ *      (1) The bookkeeping kernels of bc_append and bc_compress (when the call's K/V rows go out in
+ *          a launch of their own).  They touch only the cache's metadata and `slots`, read nothing
+ *          an attention kernel writes, and end only once the kernel they overtook has ended, so
+ *          everything enqueued behind them is ordered after both.
+ *      (2) The attention kernels.  Before they wait for the kernel ahead they read only `slots` and
+ *          metadata (lengths, page-table entries) that a bookkeeping kernel which has ENDED wrote;
+ *          the queries, the extra entry, the pool rows, the outputs and the split-K scratch are
+ *          touched after the wait.  An attention kernel that follows its step's bookkeeping kernel
+ *          directly (bc_decode_step) reads nothing before the wait.
+ *      (3) Kernels that release their dependents early: the attention kernels (once they have read
+ *          the lengths they need) and the row-writing kernel of bc_append / bc_compress (at once).
+ *    What this asks of the caller: `slots` must not be written by a kernel that releases its
+ *    dependents early.  K/V rows, queries, outputs and the caller's own kernels keep plain stream
+ *    order.
  *
  * Store layout (owned by the library inside the caller's `pool` buffer)
  *    pool[layer][page][slot_in_page][K|V][kv_head][head_dim] bf16: one token's entry of one layer
@@ -223,8 +233,7 @@ BC_API bc_status bc_decode_attn_pair(bc_cache* cache, int32_t layer, const int32
  * How: the append bookkeeping runs as its own one-block kernel (on the layer-0 call; it may begin
  * under the last blocks of the attention kernel enqueued before it, see "Overlap" above); the
  * attention kernel takes the new entries from the input tensors where it needs them, and one of
- * its warps stores them to the pool for later steps.  Measured on the ratio sweep: about 1 % more
- * tokens/s than the separate calls (4 % at c = 32).
+ * its warps stores them to the pool for later steps.
  * q [n, q_heads, head_dim], k, v [n, kv_heads, head_dim], out like q; n <= 512.  With
  * BC_FLAG_ATTN_REFERENCE the call simply issues the two separate calls. */
 BC_API bc_status bc_decode_step(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n, const void* q,
@@ -248,10 +257,14 @@ BC_API bc_status bc_decode_step(bc_cache* cache, int32_t layer, const int32_t* s
  * about 4.9 MB of device memory that every GPU which loads the library keeps until the process
  * exits.  The call itself performs no device or host allocation and calls no allocating routine.
  *
- * Arguments, layouts, results and error behaviour are those of bc_decode_attn, with these limits:
- * n <= BC_STATIC_MAX_BATCH, at most BC_STATIC_MAX_CTAS thread blocks (fewer SMs are used on a
- * larger part), q_heads * head_dim <= 4096.  A call beyond them returns BC_ERR_TOO_LARGE and
- * enqueues nothing.  The cache's own `workspace` is not touched.
+ * Arguments, layouts, results and error behaviour are those of bc_decode_attn (layer =
+ * BC_ALL_LAYERS and BC_FLAG_ATTN_REFERENCE included; the debugging kernel of that flag uses no
+ * scratch), with these limits: n <= BC_STATIC_MAX_BATCH, at most BC_STATIC_MAX_CTAS thread blocks
+ * (fewer SMs are used on a larger part), q_heads * head_dim <= 4096.  A call beyond them returns
+ * BC_ERR_TOO_LARGE and enqueues nothing.  The cache's own `workspace` is not touched.  Two
+ * differences: the launches are not bracketed by bc_profile_enable, and the device that is current
+ * at the call must be the one the cache was created on (else BC_ERR_INVALID_ARG), because the
+ * built-in array exists once per device.
  *
  * The first call on each device looks up the device address of the built-in array (once per
  * device, with that device current); make that first call outside any stream capture.  All calls,
@@ -259,7 +272,15 @@ BC_API bc_status bc_decode_step(bc_cache* cache, int32_t layer, const int32_t* s
  * call's partials when the next call starts (every partial a call reads it has written first,
  * and every call returns the ticket counters to zero, so nothing needs clearing), and two calls
  * whose kernels overlap on the GPU race on it.  Issue them
- * on one stream, or order them with events. */
+ * on one stream, or order them with events.
+ *
+ * Errors.  A launch that gives up with BC_ERR_TIMEOUT (latched in the record of the cache that
+ * issued it) may leave counters of the shared array non-zero; until they are cleared, static calls
+ * of EVERY cache on that device can merge wrongly, and only the issuing cache's record says so.
+ * bc_clear_error of a cache that has used this entry point since its last clear zeroes the shared
+ * counters on the given stream: that is a write to the one array, so it has to be ordered (same
+ * stream, or events) against every static call of the process like a static call itself.  After
+ * such a timeout issue no further static call, from any cache, before that bc_clear_error. */
 BC_API bc_status bc_decode_attn_static(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                                        const void* q, void* out, float sm_scale, const void* extra_k,
                                        const void* extra_v, void* stream);
@@ -386,7 +407,10 @@ BC_API bc_status bc_get_free_list(bc_cache* cache, int32_t* pages, int32_t* coun
 BC_API bc_status bc_poll_error(bc_cache* cache, int32_t* code, int32_t* slot, int64_t* call_index,
                         void* stream);
 
-/* Clears the latched error record. */
+/* Clears the latched error record and zeroes the split-K ticket counters in the cache's workspace
+ * (a launch that gave up with BC_ERR_TIMEOUT may have left them non-zero).  If this cache has
+ * called bc_decode_attn_static since its last clear, the counters of the array built into the
+ * library are zeroed as well: see the ordering rule stated there. */
 BC_API bc_status bc_clear_error(bc_cache* cache, void* stream);
 
 /* Gathers the live entries of one sequence in logical order (prompt, beacons, window), with the

@@ -103,6 +103,12 @@ struct bc_cache {
   int compress_next_layer;  // per-layer ordering of bc_compress
   int restore_next_layer = 0;   // per-layer ordering of bc_restore
   int append_set = 0;           // which set of append row destinations the current step uses (flips on layer 0)
+  // true while the last kernel this handle enqueued that writes metadata (lengths, page table, free stack)
+  // has not been followed by an ordinarily launched kernel or an attention launch of this handle: an
+  // attention kernel enqueued now could begin before that writer has ended and must not read early
+  bool meta_unsettled = true;
+  int device = -1;              // the CUDA device that was current at bc_cache_create
+  bool static_used = false;     // a bc_decode_attn_static launch was issued since the last bc_clear_error
   int last_cuda_error;
   // profiling
   std::vector<cudaEvent_t> ev;
@@ -167,6 +173,8 @@ bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const v
   a.part_ml = work_ptr<float>(c, c->wl.part_ml);
   a.tickets = work_ptr<int32_t>(c, c->wl.tickets);
   a.ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
+  a.meta_settled = c->meta_unsettled ? 0 : 1;
+  c->meta_unsettled = false;   // whatever follows this launch starts after its blocks have waited for the writer
   if (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) {
     BC_CUDA(c, bc_launch_attn_reference(c->meta, c->geom, a, s));
     c->launches += 1;
@@ -241,7 +249,7 @@ cudaError_t static_scratch_reset_tickets(cudaStream_t s) {
 
 extern "C" {
 
-int32_t bc_version(void) { return 114; }
+int32_t bc_version(void) { return 200; }
 
 const char* bc_status_string(bc_status s) {
   switch (s) {
@@ -298,7 +306,8 @@ bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* wo
   g.head_row_bytes = cfg->head_dim * 2;
   g.entry_bytes = 2 * cfg->kv_heads * g.head_row_bytes;
   g.layer_bytes = (int64_t)cfg->num_pages * cfg->page_size * g.entry_bytes;
-  cudaError_t e = bc_attn_setup(&c->sm_count);
+  cudaError_t e = cudaGetDevice(&c->device);
+  if (e == cudaSuccess) e = bc_attn_setup(&c->sm_count);
   if (e == cudaSuccess) e = bc_launch_init(c->meta, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->work + c->wl.tickets, 0, BC_MAX_ATTN_BATCH * 4, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->work + c->wl.book_flag, 0, 4, (cudaStream_t)stream);
@@ -331,6 +340,7 @@ bc_status bc_seq_open(bc_cache* c, const int32_t* slots, const int32_t* prompt_l
   if (!c || !slots || !prompt_lens || n <= 0 || n > c->cfg.max_seqs) return BC_ERR_INVALID_ARG;
   BC_CUDA(c, bc_launch_open(c->meta, slots, prompt_lens, c_per_seq, n, ++c->calls, (cudaStream_t)stream));
   c->launches += 1;
+  c->meta_unsettled = true;
   return BC_OK;
 }
 
@@ -352,6 +362,7 @@ bc_status bc_prefill(bc_cache* c, int32_t layer, const int32_t* slots, const int
   if (!k || !v || !aligned16(k) || !aligned16(v)) return BC_ERR_INVALID_ARG;
   BC_CUDA(c, bc_launch_prefill(c->meta, c->geom, layer_base(c, layer), slots, cu, n, total, k, v, (cudaStream_t)stream));
   c->launches += 1;
+  c->meta_unsettled = false;
   return BC_OK;
 }
 
@@ -370,10 +381,12 @@ bc_status bc_restore(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n
   if (layer == 0) {
     BC_CUDA(c, bc_launch_restore_book(c->meta, slots, cu_tokens, n, ++c->calls, ok, bea, s));
     c->launches += 1;
+    c->meta_unsettled = true;
   }
   BC_CUDA(c, bc_launch_restore_rows(c->meta, c->geom, layer_base(c, layer), slots, ok, bea, cu_tokens, n, total_tokens,
                                    total_beacons, tok_k, tok_v, beacon_k, beacon_v, s));
   c->launches += (total_beacons > 0) + (total_tokens > 0);
+  if (total_beacons > 0 || total_tokens > 0) c->meta_unsettled = false;
   c->restore_next_layer = (layer + 1) % c->cfg.layers;
   return BC_OK;
 }
@@ -403,10 +416,12 @@ bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n,
     BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, ++c->calls, row, pos, c->geom, layer_base(c, 0),
                                      fused ? k : nullptr, fused ? v : nullptr, s));
     c->launches += 1;
+    c->meta_unsettled = true;
   }
   if (!fused) {
     BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, k, v, n, s));
     c->launches += 1;
+    c->meta_unsettled = false;
   }
   c->append_next_layer = (layer + 1) % c->cfg.layers;
   return BC_OK;
@@ -478,6 +493,7 @@ bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32
                                      work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), c->geom, layer_base(c, 0), nullptr,
                                      nullptr, s));
     c->launches += 1;
+    c->meta_unsettled = true;
   }
   BcFusedAppend f;
   f.new_k = k; f.new_v = v;
@@ -521,14 +537,17 @@ bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t 
     BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, L > 1 ? 1 : 3, c->geom, layer_base(c, 0),
                                        fused ? bk : nullptr, fused ? bv : nullptr, s));
     c->launches += 1;
+    c->meta_unsettled = true;
   }
   if (!fused) {
     BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, bk, bv, n, s));
     c->launches += 1;
+    c->meta_unsettled = false;
   }
   if (L > 1 && layer == L - 1) {
     BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, 2, c->geom, nullptr, nullptr, nullptr, s));
     c->launches += 1;
+    c->meta_unsettled = true;
   }
   c->compress_next_layer = (layer + 1) % L;
   return BC_OK;
@@ -538,6 +557,7 @@ bc_status bc_seq_close(bc_cache* c, const int32_t* slots, int32_t n, void* strea
   if (!c || !slots || n <= 0 || n > c->cfg.max_seqs) return BC_ERR_INVALID_ARG;
   BC_CUDA(c, bc_launch_close(c->meta, slots, n, ++c->calls, (cudaStream_t)stream));
   c->launches += 1;
+  c->meta_unsettled = true;
   return BC_OK;
 }
 
@@ -748,7 +768,13 @@ bc_status bc_clear_error(bc_cache* c, void* stream) {
   BC_CUDA(c, cudaMemsetAsync(c->meta.status, 0, 16, (cudaStream_t)stream));
   // an attention launch that gave up (BC_ERR_TIMEOUT) may have left ticket counters non-zero
   BC_CUDA(c, cudaMemsetAsync(c->work + c->wl.tickets, 0, BC_MAX_ATTN_BATCH * 4, (cudaStream_t)stream));
-  BC_CUDA(c, static_scratch_reset_tickets((cudaStream_t)stream));
+  // The counters of the built-in array are shared by every cache of the process: they are touched
+  // only when THIS cache has used the static entry point since its last clear (a launch of its own
+  // may have left them non-zero), never on behalf of a cache that did not.
+  if (c->static_used) {
+    BC_CUDA(c, static_scratch_reset_tickets((cudaStream_t)stream));
+    c->static_used = false;
+  }
   return BC_OK;
 }
 
@@ -798,6 +824,17 @@ bc_status bc_profile_read(bc_cache* c, int32_t* launches, float* total_ms) {
 
 bc_status bc_decode_attn_static(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, void* out,
                                 float sm_scale, const void* extra_k, const void* extra_v, void* stream) {
+  if (c && layer == BC_ALL_LAYERS) {   // as bc_decode_attn: tensors with a leading [layers] dimension, layer by layer
+    if (n <= 0) return BC_ERR_INVALID_ARG;
+    const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+    const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
+    for (int l = 0; l < c->cfg.layers; ++l) {
+      const bc_status st = bc_decode_attn_static(c, l, slots, n, layer_slice(q, l, qb), layer_slice(out, l, ob), sm_scale,
+                                                 layer_slice(extra_k, l, kb), layer_slice(extra_v, l, kb), stream);
+      if (st) return st;
+    }
+    return BC_OK;
+  }
   bc_status st = check_batch(c, layer, slots, n);
   if (st) return st;
   if (!q || !out || !aligned16(q) || !aligned16(out)) return BC_ERR_INVALID_ARG;
@@ -805,19 +842,32 @@ bc_status bc_decode_attn_static(bc_cache* c, int32_t layer, const int32_t* slots
   if (extra_k && (!aligned16(extra_k) || !aligned16(extra_v))) return BC_ERR_INVALID_ARG;
   if (n > BC_STATIC_MAX_BATCH || c->cfg.q_heads * c->cfg.head_dim > BC_MERGE_ELEMS || c->cfg.q_heads > 64)
     return BC_ERR_TOO_LARGE;
-  unsigned char* base = nullptr;
-  BC_CUDA(c, static_scratch(&base));
+  // the built-in array is per device: the one that is looked up must be the one the cache lives on
+  int dev = -1;
+  BC_CUDA(c, cudaGetDevice(&dev));
+  if (dev != c->device) return BC_ERR_INVALID_ARG;
   BcAttnArgs a;
   a.pool_layer = layer_base(c, layer);
   a.slots = slots; a.n = n; a.q = q; a.out = out;
   a.out_f32 = (c->cfg.flags & BC_FLAG_OUT_F32) ? 1 : 0;
   a.extra_k = extra_k; a.extra_v = extra_v; a.sm_scale = sm_scale;
+  if (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) {   // the debugging kernel needs no scratch at all
+    a.part_o = nullptr; a.part_ml = nullptr; a.tickets = nullptr; a.ctas = 0;
+    BC_CUDA(c, bc_launch_attn_reference(c->meta, c->geom, a, (cudaStream_t)stream));
+    c->launches += 1;
+    return BC_OK;
+  }
+  unsigned char* base = nullptr;
+  BC_CUDA(c, static_scratch(&base));
   a.part_o = reinterpret_cast<float*>(base);
   a.part_ml = reinterpret_cast<float*>(base + kStaticPartO);
   a.tickets = reinterpret_cast<int32_t*>(base + kStaticPartO + kStaticPartMl);
   int ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
   a.ctas = ctas < BC_STATIC_MAX_CTAS ? ctas : BC_STATIC_MAX_CTAS;
   int launches = 0;
+  a.meta_settled = c->meta_unsettled ? 0 : 1;
+  c->meta_unsettled = false;
+  c->static_used = true;
   BC_CUDA(c, bc_launch_attn(c->meta, c->geom, a, nullptr, (cudaStream_t)stream, nullptr, nullptr, &launches));
   c->launches += launches;
   return BC_OK;

@@ -175,6 +175,8 @@ struct PipeParams {
   int n_groups;       // 8 / kv_heads
   int G;              // q_heads / kv_heads
   FastDiv div_ps;     // division by page_size
+  int early_meta;     // 1: the cache's metadata was last written by a kernel that has ENDED, so the plan and the
+                      // first page-table reads may run before the wait for the kernel ahead; 0: wait first
 };
 
 template <int D>
@@ -323,6 +325,16 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     fence_proxy_async();
   }
 
+  // Launched with programmatic stream serialisation, this kernel may have begun before the kernel ahead
+  // of it on the stream has ended.  What it may read before it waits for that kernel is only what a kernel
+  // that has ended wrote.  The host says whether that holds for the cache's metadata (early_meta): it does
+  // when an ordinarily launched kernel (the row writes of the step) or another attention launch lies
+  // between the last bookkeeping kernel and this one; it does not when this launch follows a bookkeeping
+  // kernel directly (the fused step, small batches whose rows the bookkeeping block writes itself, a
+  // call right after open / close / restore): then the wait comes first and nothing is read early.
+  const bool early = !FUSED && p.early_meta;
+  if (!early) asm volatile("griddepcontrol.wait;" ::: "memory");
+
   if (FUSED && p.f.do_book) {
     __shared__ int sh_book_ok;
     if (blockIdx.x == 0) {
@@ -389,13 +401,12 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   // dst_pos); the next step's bookkeeping fills the other of two sets, so it may start early as well --
   // unless this launch did its own bookkeeping in block 0, whose flag word the next one would reuse.
   if (!FUSED || !p.f.do_book) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  // This kernel itself may have been started early (it is launched with programmatic stream
-  // serialisation): behind the row-writing kernel of its step, which releases it at once, or behind
-  // another attention launch.  Up to here it has read only the cache's metadata and `slots`; everything
-  // else -- the pool rows of this step, q, the extra entry, the partial buffers and tickets it shares
-  // with the launch before it -- is touched only after the kernel ahead has ended.  So the plan above
-  // (three dependent trips to memory) runs under the predecessor instead of after it.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // With early_meta the wait for the kernel ahead is still to come: every role below executes it before it
+  // touches anything but `slots` and the metadata -- the pool rows of this step, q, the extra entry, the
+  // partial buffers and tickets this launch shares with the one before it, and every output.  So the plan
+  // above (three dependent trips to memory) and the producer's first page-table reads run under the
+  // predecessor instead of after it.
+  auto wait_for_kernel_ahead = [&]() { if (early) asm volatile("griddepcontrol.wait;" ::: "memory"); };
   // The block that ran the bookkeeping starts late; it takes no tiles, or it would finish last.
   const int idle = (FUSED && p.f.do_book && gridDim.x > 1) ? 1 : 0;
   const int n_ctas = (int)gridDim.x - idle;
@@ -426,6 +437,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   }
   if (warp == kConsumerWarps + 1) {
     // ================================ service warp =============================================
+    wait_for_kernel_ahead();
     if (FUSED) {
       // store the new entries of the sequences whose last tile this block owns (for the steps to come)
       const int chunks = p.g.head_row_bytes >> 4, per_side = Hkv * chunks;
@@ -501,6 +513,12 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     // lookahead then grows by up to two tiles per iteration until it is kPidAhead deep.
     int described = 1;
     describe(g0, 0);
+    if (early) {
+      // the page-table entries of the first tiles travel while the kernel ahead finishes; the rows they
+      // name are read only after the wait
+      for (; described < kPidAhead && g0 + described < g1; ++described) describe(g0 + described, described);
+      wait_for_kernel_ahead();
+    }
     int it = 0;
     bool aborted = false;
 #pragma unroll 1
@@ -549,6 +567,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   }
 
   // ================================== consumer warps ===========================================
+  wait_for_kernel_ahead();
   const int kvh = warp % Hkv, grp = warp / Hkv;
   const int gq = lane >> 2, qd = lane & 3;  // fragment row and column-pair index
   // ldmatrix lane offsets inside this warp's 16 rows of a stage
@@ -1055,6 +1074,7 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
                            cudaEvent_t ev_start, cudaEvent_t ev_stop, int* launches) {
   PipeParams p;
   p.m = m; p.g = g; p.a = a;
+  p.early_meta = (a.meta_settled && !fused) ? 1 : 0;
   p.f = FusedArgs{};
   if (fused) {
     p.f.new_k = static_cast<const uint8_t*>(fused->new_k); p.f.new_v = static_cast<const uint8_t*>(fused->new_v);

@@ -85,6 +85,7 @@ struct BcAttnArgs {
   float* part_ml;        // [(ctas + n)][q_heads][2]
   int32_t* tickets;      // [n] pieces of each sequence published so far; zero between launches
   int32_t ctas;
+  int32_t meta_settled = 0;  // 1: the kernel that last wrote this cache's metadata has ended by the time this launch may begin
   // the paired form (NULL otherwise): the beacons' queries, their outputs and their partial buffers
   const void* q2 = nullptr;
   void* out2 = nullptr;

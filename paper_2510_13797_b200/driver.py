@@ -2,10 +2,15 @@
 
 A DecodeDriver owns one cache for a batch of sequences that all use the same prompt length and
 ratio c, the seeded input tensors, and the position t in the generation.  Step inputs are drawn
-once (a ring of `ring` distinct steps and 4 distinct beacons) and reused cyclically:
+once (a ring of `ring` distinct steps and `beacon_ring` distinct beacons) and reused cyclically:
 
     generated token n (1-based)      -> q, k, v row (n - 1) % ring
-    beacon m (1-based, at t = m * c) -> beacon q, k, v row m % 4
+    beacon m (1-based, at t = m * c) -> beacon q, k, v row m % beacon_ring
+
+The window's tokens are always distinct (ring >= c).  The beacons a cache holds are distinct only
+up to beacon_ring: the benchmark keeps the default of 4 (the values do not change the traffic),
+the parity tests pass a ring as long as the run (every stored beacon unique) or a prime longer
+than a page, so that a kernel that read beacon m +- k for m, or beacon page j for page k, fails.
 
 so the cache content at any step is a pure function of the workload's seed, which is what lets a
 test rebuild it on the CPU without replaying the run.  Used by bench.py and by the full-size tests.
@@ -21,7 +26,7 @@ from .workloads import InputStream
 
 
 class DecodeDriver:
-    def __init__(self, w, device, seed_offset=0, fused=False, paired=True, host_pipelined=True):
+    def __init__(self, w, device, seed_offset=0, fused=False, paired=True, host_pipelined=True, beacon_ring=4):
         self.w, self.dev = w, torch.device(device)
         self.fused = fused                             # True: regular steps through bc_decode_step (one launch)
         self.paired = paired                           # True: the step that fills a window attends for the token and
@@ -49,7 +54,8 @@ class DecodeDriver:
         self.pk, self.pv = stream.prompt_kv(0)
         self.ring = max(c, 16)                         # distinct step inputs, reused cyclically
         self.q, self.k, self.v = stream.step_chunk(0, seed_offset, self.ring)
-        self.bq, self.bk, self.bv = stream.beacon_chunk(0, seed_offset, 4)
+        self.bring = int(beacon_ring)                  # distinct beacons, reused cyclically
+        self.bq, self.bk, self.bv = stream.beacon_chunk(0, seed_offset, self.bring)
         self.out = self.cache.new_out(Bn)
         self.out_b = self.cache.new_out(Bn)
         self.t = 0
@@ -69,7 +75,7 @@ class DecodeDriver:
             c.bc_append(0, self.slots, self.k[j], self.v[j])
             self.t += 1
             if self.c > 1 and self.t % self.c == 0:
-                b = (self.t // self.c) % 4
+                b = (self.t // self.c) % self.bring
                 c.bc_compress(0, self.slots, self.bk[b], self.bv[b])
 
     def step(self):
@@ -77,7 +83,7 @@ class DecodeDriver:
         window filled and the beacon step (beacon-query attention into out_b, then compress) ran."""
         c, j = self.cache, self.t % self.ring
         if self.paired and self.c > 1 and (self.t + 1) % self.c == 0:
-            b = ((self.t + 1) // self.c) % 4
+            b = ((self.t + 1) // self.c) % self.bring
             c.bc_append(0, self.slots, self.k[j], self.v[j])
             c.bc_decode_attn_pair(0, self.slots, self.q[j], self.out, self.bq[b], self.out_b, self.w.sm_scale, self.bk[b], self.bv[b])
             self.t += 1
@@ -90,7 +96,7 @@ class DecodeDriver:
             c.bc_decode_attn(0, self.slots, self.q[j], self.out, self.w.sm_scale)
         self.t += 1
         if self.c > 1 and self.t % self.c == 0:
-            b = (self.t // self.c) % 4
+            b = (self.t // self.c) % self.bring
             c.bc_decode_attn(0, self.slots, self.bq[b], self.out_b, self.w.sm_scale, self.bk[b], self.bv[b])
             c.bc_compress(0, self.slots, self.bk[b], self.bv[b])
             return True
@@ -115,7 +121,7 @@ class DecodeDriver:
             self.h = dict(q=hq, k=hk, v=hv, bq=hbq, bk=hbk, bv=hbv, out=pin(self.out), out_b=pin(self.out_b))
         c, j, h = self.cache, self.t % self.ring, self.h
         if self.paired and self.c > 1 and (self.t + 1) % self.c == 0:
-            b = ((self.t + 1) // self.c) % 4
+            b = ((self.t + 1) // self.c) % self.bring
             c.bc_fill_step_host(0, self.slots, h["q"][j], h["k"][j], h["v"][j], h["bq"][b], h["bk"][b], h["bv"][b],
                                 h["out"], h["out_b"], self.w.sm_scale)
             self.t += 1
@@ -123,7 +129,7 @@ class DecodeDriver:
         c.bc_decode_step_host(0, self.slots, h["q"][j], h["k"][j], h["v"][j], h["out"], self.w.sm_scale)
         self.t += 1
         if self.c > 1 and self.t % self.c == 0:
-            b = (self.t // self.c) % 4
+            b = (self.t // self.c) % self.bring
             c.bc_compress_step_host(0, self.slots, h["bq"][b], h["bk"][b], h["bv"][b], h["out_b"], self.w.sm_scale)
 
     def check_error(self):

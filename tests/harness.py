@@ -109,9 +109,11 @@ class Pair:
             ref[i] = seq.attend(layer, qq[i], sm_scale)
         return self._append_ok, out, ref
 
-    def attend(self, layer, slots, q, sm_scale, extra_k=None, extra_v=None):
+    def attend(self, layer, slots, q, sm_scale, extra_k=None, extra_v=None, static=False):
+        """static=True: through bc_decode_attn_static (split-K scratch inside the library image)."""
         out = self.gpu.new_out(len(slots))
-        self.gpu.bc_decode_attn(layer, self._i32(slots), q, out, sm_scale, extra_k, extra_v)
+        call = self.gpu.bc_decode_attn_static if static else self.gpu.bc_decode_attn
+        call(layer, self._i32(slots), q, out, sm_scale, extra_k, extra_v)
         qq = f64(q)
         ref = np.zeros((len(slots), self.Hq, self.D))
         for i, slot in enumerate(slots):

@@ -31,14 +31,16 @@ def live_kv(drv: DecodeDriver, s: int, t: int):
     P, c = drv.P, drv.c
     ids = closed_form_live_ids(P, t - 1, c) + [("token", t - 1)]
     pk, pv = f64(drv.pk[s * P:(s + 1) * P]), f64(drv.pv[s * P:(s + 1) * P])
+    bk, bv = f64(drv.bk[:, s]), f64(drv.bv[:, s])          # this sequence's beacon and token inputs, one copy each
+    tk, tv = f64(drv.k[:, s]), f64(drv.v[:, s])
     ks, vs = [], []
     for kind, ident in ids:
         if kind == "prompt":
             ks.append(pk[ident]); vs.append(pv[ident])
         elif kind == "beacon":
-            ks.append(f64(drv.bk[ident % 4, s])); vs.append(f64(drv.bv[ident % 4, s]))
+            ks.append(bk[ident % drv.bring]); vs.append(bv[ident % drv.bring])
         else:
-            ks.append(f64(drv.k[ident % drv.ring, s])); vs.append(f64(drv.v[ident % drv.ring, s]))
+            ks.append(tk[ident % drv.ring]); vs.append(tv[ident % drv.ring])
     return np.stack(ks), np.stack(vs)
 
 
@@ -53,7 +55,7 @@ def check_step(drv: DecodeDriver, seqs, what):
         ref = attention(f64(drv.q[(t - 1) % drv.ring, s]), K, V, scale)
         assert_close(drv.out[s], ref, f"{what}: step {t} seq {s}")
         if fired:
-            b = (t // drv.c) % 4
+            b = (t // drv.c) % drv.bring
             Kb = np.concatenate([K, f64(drv.bk[b, s])[None]]); Vb = np.concatenate([V, f64(drv.bv[b, s])[None]])
             refb = attention(f64(drv.bq[b, s]), Kb, Vb, scale)
             assert_close(drv.out_b[s], refb, f"{what}: beacon query at step {t} seq {s}")
@@ -78,7 +80,7 @@ def test_sweep_mid_generation(c):
     """The ratio sweep (batch 64, 32/8 heads, D 128, prompt 512, page_size = c) around the middle of
     the 16384-step generation: a whole window of steps including the beacon query and the eviction."""
     w = make_workload("sweep", c=c)
-    drv = DecodeDriver(w, DEV)
+    drv = DecodeDriver(w, DEV, beacon_ring=w.steps // 2 // c + 8)      # every beacon the cache holds is unique
     t0 = (w.steps // 2 // c) * c - 2
     drv.reset_to(t0)
     seqs = [0, 17, 63]
@@ -93,7 +95,7 @@ def test_sweep_mid_generation(c):
 def test_sweep_mid_generation_fused_step():
     """The same window at c = 16 with the regular steps issued as bc_decode_step (one launch)."""
     w = make_workload("sweep", c=16)
-    drv = DecodeDriver(w, DEV, fused=True)
+    drv = DecodeDriver(w, DEV, fused=True, beacon_ring=w.steps // 2 // 16 + 8)
     drv.reset_to((w.steps // 2 // 16) * 16 - 2)
     fired = sum(check_step(drv, [3, 31, 60], "sweep c=16 fused") for _ in range(6))
     assert fired >= 1
@@ -106,12 +108,13 @@ def test_sweep_window_replayed_as_cuda_graph(c, paired):
     """The launch configuration the benchmark times: whole windows of steps captured once as a CUDA
     graph and replayed.  A replay feeds the inputs of the captured steps again, so the captured span
     is a whole number of input periods (the step inputs repeat every `ring` steps, the beacons every
-    4 windows): then the replayed generation is the one the oracle rebuilds from the seeds.  After
+    37 windows -- a prime longer than a page of beacons, so neighbouring beacons and neighbouring
+    beacon pages differ): then the replayed generation is the one the oracle rebuilds from the seeds.  After
     three replays the outputs left by the last step (it fills a window: token rows and beacon rows,
     paired or as two passes) and the bookkeeping must be those of the oracle for that step."""
     w = make_workload("sweep", c=c)
-    drv = DecodeDriver(w, DEV, paired=paired)
-    span = math.lcm(drv.ring, 4 * c)
+    drv = DecodeDriver(w, DEV, paired=paired, beacon_ring=37)
+    span = math.lcm(drv.ring, drv.bring * c)
     t0 = (w.steps // 2 // span) * span
     drv.reset_to(t0)
     for _ in range(span):                                # one eager span: warms every kernel
@@ -133,7 +136,7 @@ def test_sweep_window_replayed_as_cuda_graph(c, paired):
     drv.check_error()
     t = drv.t                                            # the last replayed step; it filled the window
     assert t % c == 0
-    scale, b = w.sm_scale, (t // c) % 4
+    scale, b = w.sm_scale, (t // c) % drv.bring
     for s in (0, 29, 63):
         K, V = live_kv(drv, s, t)
         assert_close(drv.out[s], attention(f64(drv.q[(t - 1) % drv.ring, s]), K, V, scale), f"graph c={c}: step {t} seq {s}")
@@ -146,7 +149,7 @@ def test_sweep_host_buffer_steps_full_size():
     """The end-to-end leg of the benchmark: host-buffer steps (packed pinned inputs on the cache's copy
     stream, pipelined outputs) at the sweep's size, c = 4, across a window-fill step."""
     w = make_workload("sweep", c=4)
-    drv = DecodeDriver(w, DEV)
+    drv = DecodeDriver(w, DEV, beacon_ring=37)
     t0 = (w.steps // 2 // 16) * 16 + 1
     drv.reset_to(t0)
     for _ in range(3):                                   # steps t0+1 .. t0+3; the last one fills the window (paired)
@@ -156,7 +159,7 @@ def test_sweep_host_buffer_steps_full_size():
     drv.check_error()
     t = drv.t
     assert t % 4 == 0
-    scale, b = w.sm_scale, (t // 4) % 4
+    scale, b = w.sm_scale, (t // 4) % drv.bring
     for s in (1, 33, 62):
         K, V = live_kv(drv, s, t)
         assert_close(drv.h["out"][s], attention(f64(drv.q[(t - 1) % drv.ring, s]), K, V, scale), f"host step {t} seq {s}")
@@ -171,8 +174,8 @@ def test_sweep_c2_long_run_content_bit_exact():
     blocks.  Nothing may be overwritten early: the last outputs and the stored content of sampled
     sequences (every prompt entry, beacon and window token, bit for bit) must be the oracle's."""
     w = make_workload("sweep", c=2)
-    drv = DecodeDriver(w, DEV)
     t0 = (w.steps // 2 // 16) * 16
+    drv = DecodeDriver(w, DEV, beacon_ring=(t0 + 400) // 2 + 8)         # every stored beacon is unique
     drv.reset_to(t0)
     for _ in range(399):
         drv.step()
@@ -202,7 +205,7 @@ def test_sweep_c16_end_of_run_pages_bit_exact():
     """c = 16 to the last step of the generation: page lists and the free stack equal the paging
     model replayed over the same 16384 appends and 1024 compressions."""
     w = make_workload("sweep", c=16)
-    drv = DecodeDriver(w, DEV)
+    drv = DecodeDriver(w, DEV, beacon_ring=w.steps // 16 + 7)           # 1031 > 1024 beacons: all unique
     model = PagingModel(drv.num_pages, w.page_size, w.batch, drv.pages_per_seq, 0, 16)
     slots = list(range(w.batch))
     assert model.open(slots, w.prompt_lens) == [OK] * w.batch
@@ -228,7 +231,7 @@ def test_cfg2_sampled_steps():
     """Batch 32, 12/2 heads, prompt 256, 4096 steps, c = 16: keys pre-scaled by 1/sqrt(128), beacon
     keys left N(0,1), softmax scale 1 (diffuse logits plus sharp beacon peaks)."""
     w = make_workload("cfg2")
-    drv = DecodeDriver(w, DEV)
+    drv = DecodeDriver(w, DEV, beacon_ring=w.steps // 16 + 1)           # 257 > 256 beacons: all unique
     model = PagingModel(drv.num_pages, w.page_size, w.batch, drv.pages_per_seq, 0, 16)
     slots = list(range(w.batch))
     model.open(slots, w.prompt_lens)
@@ -266,7 +269,8 @@ def test_ragged_batch_full_size():
     pk, pv = stream.prompt_kv(0)
     ring = 16
     q, k, v = stream.step_chunk(0, 0, ring)
-    bq, bk, bv = stream.beacon_chunk(0, 0, 4)
+    BR = 37                                              # distinct beacons per sequence: a prime longer than a page
+    bq, bk, bv = stream.beacon_chunk(0, 0, BR)
     i32 = lambda xs: torch.tensor(list(xs), dtype=torch.int32, device=DEV)
     i64 = lambda xs: torch.tensor(list(xs), dtype=torch.int64, device=DEV)
     all_slots = list(range(Bn))
@@ -283,8 +287,8 @@ def test_ragged_batch_full_size():
         P, c = w.prompt_lens[s], w.cs[s]
         t_done = t - 1 if t % c == 0 else t
         nb = t_done // c
-        ks = [f64(pk[cu[s]:cu[s + 1]])] + [f64(bk[m % 4, s])[None] for m in range(1, nb + 1)]
-        vs = [f64(pv[cu[s]:cu[s + 1]])] + [f64(bv[m % 4, s])[None] for m in range(1, nb + 1)]
+        ks = [f64(pk[cu[s]:cu[s + 1]])] + [f64(bk[m % BR, s])[None] for m in range(1, nb + 1)]
+        vs = [f64(pv[cu[s]:cu[s + 1]])] + [f64(bv[m % BR, s])[None] for m in range(1, nb + 1)]
         for i in range(nb * c, t):
             ks.append(f64(k[i % ring, s])[None]); vs.append(f64(v[i % ring, s])[None])
         return np.concatenate(ks), np.concatenate(vs)
@@ -306,11 +310,9 @@ def test_ragged_batch_full_size():
         if full:
             fidx, fsl = i64(full), i32(full)
             b = None
-            # beacon number m = t / c differs per sequence: group by m % 4
-            for r in range(4):
-                grp = [s for s in full if (t // w.cs[s]) % 4 == r]
-                if not grp:
-                    continue
+            # beacon number m = t / c differs per sequence: group by m % BR
+            for r in sorted(set((t // w.cs[s]) % BR for s in full)):
+                grp = [s for s in full if (t // w.cs[s]) % BR == r]
                 gidx, gsl = i64(grp), i32(grp)
                 gbk, gbv = bk[r].index_select(0, gidx), bv[r].index_select(0, gidx)
                 outb = cache.new_out(len(grp))

@@ -248,6 +248,48 @@ def test_device_side_errors_match_the_model():
     pair2.check_state()
 
 
+def test_several_failures_in_one_call_latch_the_lowest_item():
+    """The status record after calls with two and three failing items of different kinds, against
+    records written out by hand from the rule in breadcrumbs.h (first failing call; within it the
+    failing item with the lowest batch index), not against the model."""
+    i32 = lambda xs: torch.tensor(xs, dtype=torch.int32, device=DEV)
+    z = lambda n: torch.zeros((n, 1, 64), dtype=torch.bfloat16, device=DEV)
+    name = lambda cache: (lambda c, s, k: (B.STATUS_NAMES[c], s, k))(*cache.bc_poll_error())
+    # open (call 1): item 0 fails at allocation (3 pages of 1, 2 free), item 1 at validation (slot 9), item 2 too (c = 0)
+    a = B.Cache(1, 1, 2, 64, 1, 1, max_seqs=4, num_pages=2, max_pages_per_seq=8)
+    a.bc_seq_open(i32([3, 9, 1]), i32([3, 1, 1]), i32([1, 1, 0]))
+    assert name(a) == ("NO_PAGES", 3, 1)
+    assert a.bc_get_free_list() == [1, 0] and all(a.bc_get_state(s) is None for s in range(4))
+    # append (call 4): [WINDOW_FULL, OK, BAD_SLOT]; a later call (5) with other failures changes nothing
+    b = B.Cache(1, 1, 2, 64, 2, 2, max_seqs=8, num_pages=16, max_pages_per_seq=8)
+    b.bc_seq_open(i32([5, 2]), i32([1, 1]))
+    b.bc_append(0, i32([5]), z(1), z(1)); b.bc_append(0, i32([5]), z(1), z(1))
+    assert name(b) == ("OK", 0, 0)
+    b.bc_append(0, i32([5, 2, 7]), z(3), z(3))
+    assert name(b) == ("WINDOW_FULL", 5, 4)
+    assert b.bc_get_state(2)["window_len"] == 1 and b.bc_get_state(5)["window_len"] == 2
+    b.bc_append(0, i32([7, 5]), z(2), z(2))
+    assert name(b) == ("WINDOW_FULL", 5, 4)
+    # compress (call 3): lowest index, not lowest slot id, not the last failure
+    c3 = B.Cache(1, 1, 2, 64, 2, 2, max_seqs=8, num_pages=16, max_pages_per_seq=8)
+    c3.bc_seq_open(i32([2]), i32([1])); c3.bc_append(0, i32([2]), z(1), z(1))
+    c3.bc_compress(0, i32([6, 2, 0]), z(3), z(3))
+    assert name(c3) == ("BAD_SLOT", 6, 3)
+    # compress (call 4): allocation failures at items 0 and 1 (no page left), validation failure at item 2
+    d = B.Cache(1, 1, 2, 64, 2, 1, max_seqs=4, num_pages=4, max_pages_per_seq=8)
+    d.bc_seq_open(i32([0, 1]), i32([0, 0]))
+    d.bc_append(0, i32([0, 1]), z(2), z(2)); d.bc_append(0, i32([0, 1]), z(2), z(2))
+    assert d.bc_get_free_list() == []
+    d.bc_compress(0, i32([1, 0, 3]), z(3), z(3))
+    assert name(d) == ("NO_PAGES", 1, 4)
+    assert d.bc_get_state(1)["window_len"] == 2 and d.bc_get_state(0)["n_beacons"] == 0
+    # close (call 2)
+    e = B.Cache(1, 1, 2, 64, 4, 4, max_seqs=4, num_pages=8, max_pages_per_seq=16)
+    e.bc_seq_open(i32([0]), i32([0]))
+    e.bc_seq_close(i32([3, 0, 2]))
+    assert name(e) == ("BAD_SLOT", 3, 2)
+
+
 def test_host_argument_errors():
     pair = Pair(1, 1, 2, 64, 4, max_seqs=2, num_pages=8, max_pages_per_seq=8)
     slots = torch.tensor([0], dtype=torch.int32, device=DEV)

@@ -322,6 +322,61 @@ def test_paging_exhaustion_and_capacity():
     assert m3.append([0]) == [OK] and m3.append([0]) == [CAPACITY]
 
 
+def test_latched_error_is_the_lowest_failing_item_of_the_first_failing_call():
+    """The rule breadcrumbs.h states for the status record: the first call with a failing item
+    latches, and of that call's failing items the one with the lowest batch index is recorded
+    (code, slot, 1-based call index); later failures change nothing.  Every expected record below
+    is worked out by hand from that sentence.  The cases are chosen so that other plausible rules
+    give a different record: "first failure met while processing" (validation failures are met
+    before allocation failures, whatever their batch position), "last failure", "lowest slot id",
+    "highest severity / lowest code"."""
+    # open: item 0 passes validation and fails at ALLOCATION (needs 3 pages, 2 free); item 1 fails
+    # VALIDATION (slot out of range); item 2 fails validation (c = 0).  Lowest index: item 0.
+    m = PagingModel(num_pages=2, page_size=1, max_seqs=4, max_pages_per_seq=8)
+    assert m.open([3, 9, 1], [3, 1, 1], [1, 1, 0]) == [NO_PAGES, BAD_SLOT, "INVALID_ARG"]
+    assert m.first_error == (NO_PAGES, 3, 1)
+    assert m.free_list() == [1, 0] and not m.seqs            # a failed item changes nothing
+    # append: [WINDOW_FULL, OK, BAD_SLOT] in one call, on a store that has no error yet
+    m = PagingModel(num_pages=16, page_size=2, max_seqs=8, max_pages_per_seq=8)
+    assert m.open([5, 2], [1, 1], [2, 2]) == [OK, OK]                        # call 1
+    assert m.append([5]) == [OK] and m.append([5]) == [OK]                   # calls 2, 3: slot 5's window is full
+    assert m.first_error is None
+    assert m.append([5, 2, 7]) == [WINDOW_FULL, OK, BAD_SLOT]                # call 4
+    assert m.first_error == (WINDOW_FULL, 5, 4)
+    assert m.state(2)["window_len"] == 1 and m.state(5)["window_len"] == 2   # the good item went through
+    # a later failing call does not replace the record, even one with a "worse" or lower-indexed failure
+    assert m.append([7, 5]) == [BAD_SLOT, WINDOW_FULL]                       # call 5
+    assert m.first_error == (WINDOW_FULL, 5, 4)
+    # the failing item with the lowest INDEX, not the lowest slot id and not the last one:
+    # items [slot 6 (not open), slot 2 (window of 1: not full), slot 0 (not open)]
+    m2 = PagingModel(num_pages=16, page_size=2, max_seqs=8, max_pages_per_seq=8)
+    assert m2.open([2], [1], [2]) == [OK] and m2.append([2]) == [OK]         # calls 1, 2
+    assert m2.compress([6, 2, 0]) == [BAD_SLOT, WINDOW_NOT_FULL, BAD_SLOT]   # call 3
+    assert m2.first_error == (BAD_SLOT, 6, 3)
+    # compress: allocation failure at a lower index than a validation failure.  Page size 1, pool of
+    # 4: slots 0 and 1 (P = 0, c = 2) take 2 window pages each, so no page is free when both
+    # windows are full; compress needs a beacon page for each -> NO_PAGES for item 0 and item 1;
+    # item 2 names a closed slot.  Lowest index: item 0, an allocation failure.
+    m3 = PagingModel(num_pages=4, page_size=1, max_seqs=4, max_pages_per_seq=8)
+    assert m3.open([0, 1], [0, 0], [2, 2]) == [OK, OK]                       # call 1
+    assert m3.append([0, 1]) == [OK, OK] and m3.append([0, 1]) == [OK, OK]   # calls 2, 3
+    assert m3.free_list() == []
+    assert m3.compress([1, 0, 3]) == [NO_PAGES, NO_PAGES, BAD_SLOT]          # call 4
+    assert m3.first_error == (NO_PAGES, 1, 4)
+    assert m3.state(1)["window_len"] == 2 and m3.state(0)["n_beacons"] == 0
+    # close and restore report the same way
+    # restore: T = 132 at c = 4 is 33 beacons = 9 pages of 4, the pool has 8 -> allocation failure
+    # at item 0; item 1 names a closed slot; item 2 has a negative length
+    m4 = PagingModel(num_pages=8, page_size=4, max_seqs=4, max_pages_per_seq=16)
+    assert m4.open([0, 1], [0, 0], [4, 4]) == [OK, OK]                       # call 1
+    assert m4.restore([1, 2, 0], [132, 1, -1]) == [NO_PAGES, BAD_SLOT, "INVALID_ARG"]   # call 2
+    assert m4.first_error == (NO_PAGES, 1, 2)
+    m5 = PagingModel(num_pages=8, page_size=4, max_seqs=4, max_pages_per_seq=16)
+    assert m5.open([0], [0], [4]) == [OK]                                    # call 1
+    assert m5.close([3, 0, 2]) == [BAD_SLOT, OK, BAD_SLOT]                   # call 2
+    assert m5.first_error == (BAD_SLOT, 3, 2)
+
+
 
 @pytest.mark.parametrize("ps,c", [(1, 2), (4, 4), (16, 8), (8, 32), (16, 1)])
 def test_paging_restore_equals_replay_counts_and_conserves_pages(ps, c):

@@ -349,8 +349,9 @@ BC_API bc_status bc_compress_step_host(bc_cache* cache, int32_t layer, const int
  * even from fp32 (accumulation in fp32, softmax weights rounded to bf16 before the second product).
  * head_dim must be 128 and q_heads / kv_heads <= 16 (else BC_ERR_UNSUPPORTED); sm_scale > 0.  `workspace`: device
  * memory of at least bc_mask_attn_query_bytes bytes, 256-byte aligned (it receives the list of
- * query tiles and the status word).  All inputs must be finite: rows of K and V next to a sequence's
- * own are read along with it and enter the products with weight zero.  Asynchronous on `stream`; the two host arrays are read before the
+ * query tiles and the status word).  A sequence's rows depend on that sequence's inputs only: rows of K
+ * and V that a tile reads beyond the sequence's own are masked (K) and cleared (V) before they can enter a
+ * product, so non-finite values in a neighbouring sequence do not spread.  Asynchronous on `stream`; the two host arrays are read before the
  * call returns (pageable host memory is staged by the copy, so do not call this inside a stream
  * capture).  One call at a time per workspace.  A bounded device-side wait that expires is reported
  * by bc_mask_attn_status as BC_ERR_TIMEOUT (the outputs are then incomplete). */
@@ -430,6 +431,24 @@ BC_API bc_status bc_set_attn_ctas(bc_cache* cache, int32_t ctas);
  * bracketed launches and the sum of their durations in milliseconds. */
 BC_API bc_status bc_profile_enable(bc_cache* cache, int32_t max_launches);
 BC_API bc_status bc_profile_read(bc_cache* cache, int32_t* launches, float* total_ms);
+
+/* Where a decode-attention launch spends its time.  While a buffer is set, thread 0 of every thread
+ * block of every attention kernel this handle launches (bc_decode_attn, _pair, bc_decode_step; not
+ * the static entry point) stores nanosecond stamps of the GPU's global timer, so that the figures a
+ * design discussion rests on can be regenerated: device_words is device memory of at least
+ * blocks * BC_TIMELINE_WORDS uint64 (blocks >= 304, the largest grid), block b writing words
+ * [b * BC_TIMELINE_WORDS ..): 0 block entered the kernel, 1 its plan is built, 2 it has waited for the
+ * kernel ahead on the stream, 3 its first tile has landed in shared memory, 4 the last tile of its
+ * final piece is consumed, 5 that piece is written / merged / published, 6 the ticket of its first
+ * piece is known, 7 it leaves (after the merges it owed); word 8 = tiles << 32 | first sequence;
+ * word 9 = how it ended: bit 0 its final piece was a whole sequence, bit 1 it merged that piece's
+ * sequence at once, bit 2 it published the piece, bits 3 / 4 it merged the sequence of its first /
+ * final piece after taking that sequence's last ticket.
+ * A block without tiles writes only 0 and 1.  Each launch overwrites the last one's stamps; zero
+ * the buffer before the launch of interest and read it after synchronising.  NULL switches it off
+ * (the default; the kernel then executes a few predicated-off stores per block and nothing else). */
+#define BC_TIMELINE_WORDS 16
+BC_API bc_status bc_attn_timeline(bc_cache* cache, void* device_words, int32_t blocks);
 
 /* Kernels launched by this handle since creation (for launch accounting). */
 BC_API int64_t bc_kernel_launches(const bc_cache* cache);

@@ -78,6 +78,7 @@ SYMBOLS = {
     "bc_clear_error": (_I32, [_P, _P]),
     "bc_export_seq": (_I32, [_P, _I32, _I32, _P, _P, _I32, _P]),
     "bc_set_attn_ctas": (_I32, [_P, _I32]),
+    "bc_attn_timeline": (_I32, [_P, _P, _I32]),
     "bc_profile_enable": (_I32, [_P, _I32]),
     "bc_profile_read": (_I32, [_P, C.POINTER(_I32), C.POINTER(_F)]),
     "bc_kernel_launches": (_I64, [_P]),
@@ -245,6 +246,10 @@ class Cache:
 
     def bc_set_attn_ctas(self, ctas):
         _check(lib().bc_set_attn_ctas(self.handle, ctas), "bc_set_attn_ctas")
+
+    def bc_attn_timeline(self, words, blocks=0):
+        """words: uint64/int64 CUDA tensor of at least blocks * 16 elements, or None to switch it off."""
+        _check(lib().bc_attn_timeline(self.handle, _ptr(words), blocks), "bc_attn_timeline")
 
     def bc_profile_enable(self, max_launches):
         _check(lib().bc_profile_enable(self.handle, max_launches), "bc_profile_enable")

@@ -107,6 +107,7 @@ struct bc_cache {
   // has not been followed by an ordinarily launched kernel or an attention launch of this handle: an
   // attention kernel enqueued now could begin before that writer has ended and must not read early
   bool meta_unsettled = true;
+  void* timeline = nullptr;     // bc_attn_timeline: device buffer the attention kernel stamps, or NULL
   int device = -1;              // the CUDA device that was current at bc_cache_create
   bool static_used = false;     // a bc_decode_attn_static launch was issued since the last bc_clear_error
   int last_cuda_error;
@@ -173,6 +174,7 @@ bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const v
   a.part_ml = work_ptr<float>(c, c->wl.part_ml);
   a.tickets = work_ptr<int32_t>(c, c->wl.tickets);
   a.ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
+  a.timeline = c->timeline;
   a.meta_settled = c->meta_unsettled ? 0 : 1;
   c->meta_unsettled = false;   // whatever follows this launch starts after its blocks have waited for the writer
   if (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) {
@@ -791,6 +793,14 @@ bc_status bc_export_seq(bc_cache* c, int32_t layer, int32_t slot, void* k_out, v
 bc_status bc_set_attn_ctas(bc_cache* c, int32_t ctas) {
   if (!c || ctas < 0 || ctas > BC_MAX_ATTN_CTAS) return BC_ERR_INVALID_ARG;
   c->attn_ctas = ctas;
+  return BC_OK;
+}
+
+bc_status bc_attn_timeline(bc_cache* c, void* device_words, int32_t blocks) {
+  if (!c) return BC_ERR_INVALID_ARG;
+  if (device_words == nullptr) { c->timeline = nullptr; return BC_OK; }
+  if ((reinterpret_cast<uintptr_t>(device_words) & 7) || blocks < BC_MAX_ATTN_CTAS) return BC_ERR_INVALID_ARG;
+  c->timeline = device_words;
   return BC_OK;
 }
 

@@ -38,6 +38,7 @@ constexpr int kPidAhead = 4;               // tiles of page-id lookahead of the 
 constexpr int kInFlight = 2;               // stages whose copies may be outstanding at once: HBM
                                            // delivers less when every SM keeps more in flight
 constexpr int kNewRowBit = 1 << 30;        // in the plan's slot word: the sequence got a new entry in this launch
+constexpr int kTimelineSlots = BC_TIMELINE_SLOTS;
 constexpr int kPidSlot = 136;              // ints per descriptor slot: 4 header + up to 132 page ids
 
 // ---------------------------------------------------------------- PTX helpers
@@ -126,6 +127,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 __device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
 // Bounded wait; returns false when it gave up or another warp already aborted.
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   uint32_t polls = 0;
@@ -175,6 +182,7 @@ struct PipeParams {
   int n_groups;       // 8 / kv_heads
   int G;              // q_heads / kv_heads
   FastDiv div_ps;     // division by page_size
+  unsigned long long* timeline;   // NULL, or [gridDim.x][kTimelineSlots] device words: %globaltimer stamps of one thread per block
   int early_meta;     // 1: the cache's metadata was last written by a kernel that has ENDED, so the plan and the
                       // first page-table reads may run before the wait for the kernel ahead; 0: wait first
 };
@@ -313,6 +321,15 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   const int n = p.a.n, T = p.rows_per_tile, TS = p.tile_shift, E = p.g.entry_bytes, ps = p.g.page_size;
   const int Hkv = p.g.kv_heads, Hq = p.g.q_heads, G = p.G;
 
+  // Timeline (bc_attn_timeline): thread 0 of every block stamps a few points of its life with the global
+  // nanosecond timer; a handful of predicated stores per block, none per tile.
+  auto stamp = [&](int k) {
+    if (p.timeline != nullptr && tid == 0) p.timeline[(size_t)blockIdx.x * kTimelineSlots + k] = global_timer_ns();
+  };
+  auto stamp_val = [&](int k, unsigned long long v) {
+    if (p.timeline != nullptr && tid == 0) p.timeline[(size_t)blockIdx.x * kTimelineSlots + k] = v;
+  };
+  stamp(0);
   if (tid == 0) {
     for (int s = 0; s < NSTAGE; ++s) {
       mbar_init(bar_full + s * 8, 1);
@@ -393,6 +410,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   }
   __syncthreads();
   const int total_tiles = s_cum[n];
+  stamp(1);
   // Every read of the sequences' lengths is done (the page-table columns the producer reads later are
   // below those lengths and never rewritten while they are): a kernel enqueued behind this one with
   // programmatic stream serialisation -- the next step's bookkeeping -- may start on the first SM
@@ -487,15 +505,15 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     };
     load_seq(fi);
     auto describe = [&](int gt, int it) {
-      int nrows = 0, p0 = 0, pg0 = 0;
+      int nrows = 0, p0 = 0, pg0 = 0, settled = 1;
       const int slot_idx = (it % RING) * kPidSlot;
       if (gt < g1) {
         while (gt >= s_cum[fi + 1]) { ++fi; load_seq(fi); }
         const int t = gt - s_cum[fi];
         int len, tt, col;
         if (t < f_tp) { len = f_P; tt = t; col = 0; }
-        else if (t < f_tpb) { len = f_nb; tt = t - f_tp; col = f_bcol; }
-        else { len = f_w; tt = t - f_tpb; col = f_wcol; }
+        else if (t < f_tpb) { len = f_nb; tt = t - f_tp; col = f_bcol; settled = t != f_tpb - 1; }
+        else { len = f_w; tt = t - f_tpb; col = f_wcol; settled = gt != s_cum[fi + 1] - 1; }
         p0 = tt << TS;
         nrows = max(min(T, len - p0), 0);
         if (FUSED && f_new && gt == s_cum[fi + 1] - 1) nrows -= 1;  // the new row comes from the input, not the pool
@@ -506,25 +524,30 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
             cp_async4(desc_ring + (uint32_t)(slot_idx + 4 + pg - pg0) * 4u, f_tab + col + pg);
         }
       }
-      if (lane == 0) { s_desc[slot_idx] = nrows; s_desc[slot_idx + 1] = p0; s_desc[slot_idx + 2] = pg0; }
+      // settled: every row of the tile was stored by a kernel that has ended by the time this one may
+      // begin -- all but the last tile of a beacon or window segment, where the newest entry lives
+      if (lane == 0) { s_desc[slot_idx] = nrows; s_desc[slot_idx + 1] = p0; s_desc[slot_idx + 2] = pg0; s_desc[slot_idx + 3] = settled; }
       cp_async_commit();  // one group per described tile
     };
     // The first tile is described alone so that its copies start as early as possible; the
     // lookahead then grows by up to two tiles per iteration until it is kPidAhead deep.
     int described = 1;
     describe(g0, 0);
-    if (early) {
-      // the page-table entries of the first tiles travel while the kernel ahead finishes; the rows they
-      // name are read only after the wait
-      for (; described < kPidAhead && g0 + described < g1; ++described) describe(g0 + described, described);
-      wait_for_kernel_ahead();
-    }
+    // With early_meta the producer does not wait for the kernel ahead before it starts to stream: page-table
+    // entries and "settled" tiles may be fetched while that kernel finishes.  The kernels of this library
+    // that can still be running then (they release their dependents early) are the row-writing kernel and
+    // another attention kernel, and in the pool those write nothing but the newest entry of a beacon or
+    // window segment, which lies in the segment's last tile.  Before the first tile that is not settled
+    // the producer waits like everybody else.  (The consumers wait before they touch q or a tile, so the
+    // ring fills up to its three stages and stalls there until the kernel ahead has ended.)
+    bool waited = !early;
     int it = 0;
     bool aborted = false;
 #pragma unroll 1
     for (int gt = g0; gt < g1; ++gt, ++it) {
       cp_async_wait_dyn(described - it - 1);  // the page ids of tile gt have landed
       __syncwarp();
+      if (!waited && !s_desc[(it % RING) * kPidSlot + 3]) { wait_for_kernel_ahead(); waited = true; }
       const int stage = it % NSTAGE;
       const uint32_t full = bar_full + stage * 8, empty = bar_empty + stage * 8;
       if (!aborted && !bounded_wait(empty, ((it / NSTAGE) & 1) ^ 1, s_abort)) aborted = true;
@@ -568,6 +591,8 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
 
   // ================================== consumer warps ===========================================
   wait_for_kernel_ahead();
+  stamp(2);
+  stamp_val(8, ((unsigned long long)(g1 - g0) << 32) | (unsigned)seq0);
   const int kvh = warp % Hkv, grp = warp / Hkv;
   const int gq = lane >> 2, qd = lane & 3;  // fragment row and column-pair index
   // ldmatrix lane offsets inside this warp's 16 rows of a stage
@@ -602,6 +627,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   int it = 0;
   int gt = g0;
   int pend_seq = -1, pend_tk = 0;  // thread 0: ticket of the block's final piece, if it had to be published
+  unsigned tl_path = 0;            // timeline word 9: how the block's final piece left and which merges it owed
   bool published_last = false;
   uint32_t qf[KSTEPS][4];
   load_q(qf, seq0);
@@ -672,6 +698,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
         }
       }
       const bool ok = __all_sync(0xffffffffu, bounded_wait(bar_full + stage * 8, (it / NSTAGE) & 1, s_abort));
+      if (it == 0) stamp(3);
       if (!ok && lane == 0 && p.m.status[0] == 0) { p.m.status[0] = BC_ERR_TIMEOUT; p.m.status[1] = -1; }
       // rows of this tile that hold entries; my warp looks at rows grp*16 .. grp*16+15 of it
       int seg_left;
@@ -775,6 +802,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     }
 
     // ---- end of piece: merge the groups of each KV head in shared memory, then write -------------
+    if (!has_next) stamp(4);
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     if (!G_LE_8) { l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2); }
     if constexpr (PAIR) {
@@ -900,6 +928,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
         else reinterpret_cast<__nv_bfloat16*>(p.a.out)[obase + idx] = __float2bfloat16_rn(val);
       }
       consumer_bar();  // the merge buffer is reused by the next piece
+      if (!has_next) tl_path |= 1u;
     } else {
       const int first = cta_of(s_cum[i]), last = cta_of(s_cum[i + 1] - 1);
       bool merged = false;
@@ -914,6 +943,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
           combine_pieces(p.a.part_o, p.a.part_ml, p.a.out, p.a.out_f32, Hq, D, i, first, last, cta, merge_o, merge_ml, tid);
           if (tid == 0) p.a.tickets[i] = 0;  // ready for the next launch
           merged = true;
+          tl_path |= 2u;
         }
       }
       if (!merged) {
@@ -937,6 +967,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
             pend_seq = i;
           }
           published_last = true;
+          tl_path |= 4u;
         }
       }
     }
@@ -951,7 +982,9 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   }
 
   // ---- all tiles streamed: merge the sequences whose last ticket this block took -----------------
+  stamp(5);
   if (svc_publishes) bounded_wait(bar_tk, 0, s_abort);
+  stamp(6);
   if (published_last) {
     if (tid == 0) { s_pend[2] = pend_seq; s_pend[3] = pend_tk; }
     consumer_bar();
@@ -962,12 +995,15 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     if (seq < 0) continue;
     const int first = cta_of(s_cum[seq]), last = cta_of(s_cum[seq + 1] - 1);
     if (tk == last - first) {
+      tl_path |= 8u << k;
       __threadfence();
       combine_pieces(p.a.part_o, p.a.part_ml, p.a.out, p.a.out_f32, Hq, D, seq, first, last, -1, nullptr, nullptr, tid);
       if (PAIR) combine_pieces(p.a.part_o2, p.a.part_ml2, p.a.out2, p.a.out_f32, Hq, D, seq, first, last, -1, nullptr, nullptr, tid);
       if (tid == 0) p.a.tickets[seq] = 0;  // ready for the next launch
     }
   }
+  stamp(7);
+  stamp_val(9, tl_path);
 }
 
 // ---------------------------------------------------------------- slow device reference
@@ -1075,6 +1111,7 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   PipeParams p;
   p.m = m; p.g = g; p.a = a;
   p.early_meta = (a.meta_settled && !fused) ? 1 : 0;
+  p.timeline = reinterpret_cast<unsigned long long*>(a.timeline);
   p.f = FusedArgs{};
   if (fused) {
     p.f.new_k = static_cast<const uint8_t*>(fused->new_k); p.f.new_v = static_cast<const uint8_t*>(fused->new_v);

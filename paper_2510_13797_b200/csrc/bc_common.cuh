@@ -12,6 +12,7 @@
 #define BC_MAX_ATTN_CTAS 304   // thread blocks of the decode-attention kernel
 #define BC_MAX_ATTN_BATCH 512  // sequences per bc_decode_attn call
 #define BC_MERGE_ELEMS 4096    // q_heads * head_dim that fits the in-block merge buffer
+#define BC_TIMELINE_SLOTS 16   // 64-bit words per thread block in a bc_attn_timeline buffer
 
 // Device view of the bookkeeping ("meta" buffer).  All arrays are int32.
 struct BcMeta {
@@ -85,6 +86,7 @@ struct BcAttnArgs {
   float* part_ml;        // [(ctas + n)][q_heads][2]
   int32_t* tickets;      // [n] pieces of each sequence published so far; zero between launches
   int32_t ctas;
+  void* timeline = nullptr;  // NULL, or the device buffer of bc_attn_timeline
   int32_t meta_settled = 0;  // 1: the kernel that last wrote this cache's metadata has ended by the time this launch may begin
   // the paired form (NULL otherwise): the beacons' queries, their outputs and their partial buffers
   const void* q2 = nullptr;

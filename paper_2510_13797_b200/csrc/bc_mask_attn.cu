@@ -24,8 +24,9 @@
 //     first, dealt out in alternating direction), keep their tensor memory and barriers, and request the next item's
 //     first tiles while the current item's output is still being written.
 // K and V rows past the end of a sequence belong to the next sequence (or read as zero past the end
-// of the array); their scores are masked and their weights are exactly zero, so inputs must be
-// finite everywhere.  Every wait is bounded; on expiry the block records BC_ERR_TIMEOUT, releases
+// of the array): their scores are overwritten with -inf, their weights are exactly zero, and their V
+// rows are cleared in shared memory before the second product, so whatever a neighbouring sequence
+// holds (infinities, NaNs) cannot reach this sequence's rows.  Every wait is bounded; on expiry the block records BC_ERR_TIMEOUT, releases
 // its tensor memory and returns.
 #include <cuda.h>
 
@@ -506,6 +507,23 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
 #pragma unroll
             for (int j = 0; j < 32; ++j) u[j] *= alpha;
             tmem_st32(tO + lane_base + cb * 32, u);
+          }
+        }
+        // A key tile that reaches past its segment has loaded rows that are not this sequence's (the next
+        // sequence's, or zeros past the end of the array).  Their scores were set to -inf above and their
+        // weights are exactly 0, but 0 * inf would still poison the second product: once the V tile has
+        // landed, the threads whose row index lies past the segment's end clear that key's V row.
+        {
+          const int seg_len = kind == 0 ? td.P : (kind == 1 ? td.nb : td.T);
+          const int nvalid = min(max(seg_len - k0, 0), kTile);
+          if (nvalid < kTile) {   // the same for the whole block
+            const bool okv = mbar_wait_or_fail(bar_v, t & 1u, s_fail);
+            if (!__all_sync(0xffffffffu, okv)) { failed = true; break; }
+            if (tid >= nvalid) {
+#pragma unroll
+              for (int ch = 0; ch < 16; ++ch) st_zero16(sV + swz(tid, ch));
+            }
+            proxy_fence();   // the product reads shared memory through the asynchronous proxy
           }
         }
         tmem_wait_st();

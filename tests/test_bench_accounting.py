@@ -46,3 +46,15 @@ def test_paired_steps_read_the_cache_once():
     assert all(bench.entries_beacon_query(512, n, 4) == bench.entries_attended(512, n, 4) for n in (12, 16))
     r.paired = True
     assert r.kv_bytes(8, 8) == (reg, 0)
+
+
+def test_step_kinds_when_fewer_steps_than_a_window_are_timed():
+    """The timed graph holds exactly the K timed steps, whatever K is; with K < c it holds part of a
+    window: no window-filling step, or exactly one."""
+    assert bench.step_kinds(8160, 20, 32) == (20, 0)        # steps 8161..8180: the window fills at 8192
+    assert bench.step_kinds(8180, 20, 32) == (19, 1)        # steps 8181..8200 contain 8192
+    assert bench.step_kinds(8176, 20, 16) == (19, 1)        # 8177..8196: 8192
+    assert bench.step_kinds(8184, 20, 8) == (18, 2)         # 8192, 8200
+    assert bench.step_kinds(8182, 20, 2) == (10, 10)
+    assert bench.step_kinds(8000, 20, 1) == (20, 0)         # uncompressed: never fills
+    assert sum(bench.step_kinds(7936, 512, 32)) == 512 and bench.step_kinds(7936, 512, 32)[1] == 16

@@ -60,3 +60,92 @@ def test_mask_form_sharp_logits():
     """Unscaled N(0,1) keys give logits with standard deviation ~ 1 after the softmax scale; keys
     scaled by 4 make the rows sharply peaked, which exercises the running maximum across tiles."""
     run_case([150], [200], 8, 8, 2, seed=9, k_scale=4.0)
+
+
+def _sampled_rows(T, c, per, rng):
+    """Token indices worth checking in a trajectory of T tokens: first and last, both sides of every
+    query-tile boundary (`per` tokens per tile) in a few regions, both sides of window boundaries,
+    and some random ones."""
+    rows = {0, 1, T - 2, T - 1}
+    for base in (0, T // 2, T - 4 * per):
+        for k in range(4):
+            b = (base // per + k) * per
+            rows |= {b - 1, b, b + 1}
+    for m in (1, 2, T // (2 * c), T // c - 1, T // c):
+        rows |= {m * c - 1, m * c, m * c + 1}
+    rows |= set(int(x) for x in rng.randint(0, T, size=24))
+    return sorted(r for r in rows if 0 <= r < T)
+
+
+@pytest.mark.parametrize("T,c", [(2048, 2), (2048, 32), (16384, 2)])
+def test_mask_form_at_benchmarked_sizes_sampled_rows(T, c):
+    """The sizes bench.py reports (sweep shape: 32/8 heads, D 128, prompt 512; T = 2048 and 16384):
+    a work item walks up to ~70 key tiles with a beacon segment of up to 64 tiles.  Sampled token
+    and beacon rows against the plain softmax definition over the oracle's closed-form live set
+    (what the eviction form's cache holds when that row is computed) -- no dense N x N mask.  Two
+    trajectories, so that tiles at the end of the first read into the second."""
+    from oracle.breadcrumbs_oracle import attention, closed_form_live_ids
+    Hq, Hkv, D, P, n = 32, 8, 128, 512, 2
+    G = Hq // Hkv
+    per = 128 // G
+    g = torch.Generator(device=DEV); g.manual_seed(100 + c)
+    nb = T // c
+    pk, pv = randn_bf16(g, (n * P, Hkv, D), DEV), randn_bf16(g, (n * P, Hkv, D), DEV)
+    tq, tk, tv = randn_bf16(g, (n * T, Hq, D), DEV), randn_bf16(g, (n * T, Hkv, D), DEV), randn_bf16(g, (n * T, Hkv, D), DEV)
+    bq, bk, bv = randn_bf16(g, (n * nb, Hq, D), DEV), randn_bf16(g, (n * nb, Hkv, D), DEV), randn_bf16(g, (n * nb, Hkv, D), DEV)
+    scale = 1.0 / math.sqrt(D)
+    out_t, out_b = B.bc_mask_attn_forward([P] * n, [T] * n, c, pk, pv, tq, tk, tv, bq, bk, bv, scale)
+    torch.cuda.synchronize()
+    rng = np.random.RandomState(c)
+    for s in range(n):
+        hpk, hpv = f64(pk[s * P:(s + 1) * P]), f64(pv[s * P:(s + 1) * P])
+        htk, htv, htq = f64(tk[s * T:(s + 1) * T]), f64(tv[s * T:(s + 1) * T]), f64(tq[s * T:(s + 1) * T])
+        hbk, hbv, hbq = f64(bk[s * nb:(s + 1) * nb]), f64(bv[s * nb:(s + 1) * nb]), f64(bq[s * nb:(s + 1) * nb])
+
+        def kv_of(ids):
+            K = np.stack([hpk[i] if kind == "prompt" else (hbk[i - 1] if kind == "beacon" else htk[i]) for kind, i in ids])
+            V = np.stack([hpv[i] if kind == "prompt" else (hbv[i - 1] if kind == "beacon" else htv[i]) for kind, i in ids])
+            return K, V
+
+        for i in _sampled_rows(T, c, per, rng):
+            # token i (0-based) is generated token i + 1: it reads the live set after i tokens plus itself
+            K, V = kv_of(closed_form_live_ids(P, i, c) + [("token", i)])
+            assert_close(out_t[s * T + i], attention(htq[i], K, V, scale), f"T={T} c={c} seq {s} token {i}")
+        beacons = sorted({1, 2, nb // 2, nb - 1, nb} | set(int(x) for x in rng.randint(1, nb + 1, size=8)) |
+                         {m for b in (per, 2 * per, (nb // per) * per) for m in (b - 1, b, b + 1, b + 2)})
+        for m in (m for m in beacons if 1 <= m <= nb):
+            # beacon m closes the window of tokens (m-1)c .. mc-1: prompt, beacons 1..m-1, that window, itself
+            ids = [("prompt", j) for j in range(P)] + [("beacon", b) for b in range(1, m)] + \
+                  [("token", i) for i in range((m - 1) * c, m * c)] + [("beacon", m)]
+            K, V = kv_of(ids)
+            assert_close(out_b[s * nb + m - 1], attention(hbq[m - 1], K, V, scale), f"T={T} c={c} seq {s} beacon {m}")
+
+
+def test_mask_form_rows_do_not_see_a_neighbouring_sequence():
+    """Key tiles at the end of a sequence's segments read rows of the next sequence along with its own.
+    The middle sequence holds infinities and NaNs in every input; the rows of the sequences before
+    and after it must still be the oracle's (finite, within tolerance)."""
+    Hq, Hkv, D, c = 8, 2, 128, 8
+    plens, tlens = [70, 33, 50], [150, 77, 90]
+    g = torch.Generator(device=DEV); g.manual_seed(21)
+    nbs = [t // c for t in tlens]
+    sp, st, sb = sum(plens), sum(tlens), sum(nbs)
+    pk, pv = randn_bf16(g, (sp, Hkv, D), DEV), randn_bf16(g, (sp, Hkv, D), DEV)
+    tq, tk, tv = randn_bf16(g, (st, Hq, D), DEV), randn_bf16(g, (st, Hkv, D), DEV), randn_bf16(g, (st, Hkv, D), DEV)
+    bq, bk, bv = randn_bf16(g, (sb, Hq, D), DEV), randn_bf16(g, (sb, Hkv, D), DEV), randn_bf16(g, (sb, Hkv, D), DEV)
+    bad = torch.tensor([float("inf"), float("-inf"), float("nan")], dtype=torch.bfloat16, device=DEV)
+    for arr, lens in ((pk, plens), (pv, plens), (tq, tlens), (tk, tlens), (tv, tlens), (bq, nbs), (bk, nbs), (bv, nbs)):
+        a, b = lens[0], lens[0] + lens[1]
+        arr[a:b] = bad[torch.arange((b - a) * arr.shape[1] * D, device=DEV) % 3].view(b - a, arr.shape[1], D)
+    scale = 1.0 / math.sqrt(D)
+    out_t, out_b = B.bc_mask_attn_forward(plens, tlens, c, pk, pv, tq, tk, tv, bq, bk, bv, scale)
+    torch.cuda.synchronize()
+    op = ot = ob = 0
+    for i, (P, T, nb) in enumerate(zip(plens, tlens, nbs)):
+        if i != 1:
+            ref_t, ref_b = mask_form_outputs(f64(pk[op:op + P]), f64(pv[op:op + P]), f64(tk[ot:ot + T]), f64(tv[ot:ot + T]),
+                                             f64(tq[ot:ot + T]), f64(bk[ob:ob + nb]), f64(bv[ob:ob + nb]), f64(bq[ob:ob + nb]),
+                                             c, scale)
+            assert_close(out_t[ot:ot + T], ref_t, f"tokens of sequence {i}")
+            assert_close(out_b[ob:ob + nb], ref_b, f"beacons of sequence {i}")
+        op, ot, ob = op + P, ot + T, ob + nb

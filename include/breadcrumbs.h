@@ -103,13 +103,22 @@ enum {
   BC_ERR_CUDA = -8,            /* a CUDA runtime call failed; see bc_last_cuda_error */
   BC_ERR_UNSUPPORTED = -9,     /* shape outside what the kernels are built for */
   BC_ERR_TIMEOUT = -10,        /* a bounded device-side wait gave up (kernel returned early) */
-  BC_ERR_TOO_LARGE = -11       /* bc_decode_attn_static: the call does not fit the built-in scratch */
+  BC_ERR_TOO_LARGE = -11,      /* bc_decode_attn_static: the call does not fit the built-in scratch */
+  BC_ERR_DEBUG_CHECK = -12     /* BC_FLAG_DEBUG_BOUNDS: a checked index was out of range, or a batch named a slot twice */
 };
 
 enum {
   BC_FLAG_OUT_F32 = 1u,        /* bc_decode_attn writes fp32 instead of bf16 */
   BC_FLAG_ATTN_REFERENCE = 2u, /* use the slow one-warp-per-head device kernel (debugging aid) */
-  BC_FLAG_HOST_PIPELINED = 4u  /* host-buffer steps: outputs are copied back on a stream of the cache's own, see bc_host_outputs_ready */
+  BC_FLAG_HOST_PIPELINED = 4u, /* host-buffer steps: outputs are copied back on a stream of the cache's own, see bc_host_outputs_ready */
+  BC_FLAG_DEBUG_BOUNDS = 8u    /* Checked mode (stands in for a memory checker).  Every kernel that turns a page id, a
+                                  page-table column or a pool row into an address checks it first: a column must lie
+                                  inside the page-table row, a page id inside the pool, a row inside the pool.  A failed
+                                  check latches BC_ERR_DEBUG_CHECK (the offending value in the record's slot field) and
+                                  the access is skipped, or, in the attention kernel, redirected to page 0, so that the
+                                  kernel still finishes; nothing traps.  The bookkeeping calls also refuse, with the
+                                  same code, every batch item whose slot an item with a lower index of the same call
+                                  names (that first item goes through).  Costs a few compares per page, no extra pass. */
 };
 
 typedef struct bc_cache bc_cache; /* opaque host-side handle */
@@ -364,6 +373,11 @@ BC_API bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t k
                                       const void* beacon_q, const void* beacon_k, const void* beacon_v,
                                       void* out_tok, void* out_beacon, float sm_scale, void* workspace,
                                       size_t workspace_bytes, void* stream);
+/* Poll limit of the bounded waits of bc_mask_attn_forward (process-wide; 0 = the default).  A block
+ * whose wait runs out waits, with the full default limit, for the tensor copies and products it has in
+ * flight, releases its tensor memory and returns; bc_mask_attn_status then reports BC_ERR_TIMEOUT. */
+BC_API bc_status bc_mask_attn_set_wait_limit(uint32_t polls);
+
 /* Synchronises `stream` and returns in *code the status the last bc_mask_attn_forward on this
  * workspace left on the device (BC_OK or BC_ERR_TIMEOUT).  The totals are those of that call. */
 BC_API bc_status bc_mask_attn_status(const void* workspace, int32_t n_seqs, int32_t q_heads, int32_t kv_heads,
@@ -431,6 +445,14 @@ BC_API bc_status bc_set_attn_ctas(bc_cache* cache, int32_t ctas);
  * bracketed launches and the sum of their durations in milliseconds. */
 BC_API bc_status bc_profile_enable(bc_cache* cache, int32_t max_launches);
 BC_API bc_status bc_profile_read(bc_cache* cache, int32_t* launches, float* total_ms);
+
+/* Poll limit of the bounded waits inside the decode-attention kernels this handle launches (0 = the
+ * default, about a quarter of a second).  A wait that runs out makes its thread block stop issuing
+ * copies, wait (with the full default limit) for the copies it has in flight, record BC_ERR_TIMEOUT
+ * in the status record and return; the call's outputs are then undefined and split-K ticket counters may
+ * be left non-zero until bc_clear_error.  A limit of 1 makes practically every launch give up at
+ * once: that is how the expiry path is exercised without hanging or faulting anything. */
+BC_API bc_status bc_set_wait_limit(bc_cache* cache, uint32_t polls);
 
 /* Where a decode-attention launch spends its time.  While a buffer is set, thread 0 of every thread
  * block of every attention kernel this handle launches (bc_decode_attn, _pair, bc_decode_step; not

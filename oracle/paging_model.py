@@ -23,6 +23,11 @@ include/breadcrumbs.h, written here independently with plain Python lists:
 * A failed item is a no-op for its sequence; the first failure of the store's
   lifetime is latched as (code, slot, call index); when several items of one
   call fail, the one with the lowest batch index is reported.
+* Checked mode (``debug_bounds=True``, the library's BC_FLAG_DEBUG_BOUNDS): a
+  batch must not name a slot twice; every item whose (valid) slot an item with
+  a lower index of the same call names is refused with DEBUG_CHECK, after the
+  slot check and before every other check, and the first occurrence goes
+  through alone.  Without the flag such a batch is outside the contract.
 
 Pinned by tests/test_oracle_pins.py: conservation (owned + free = all pages,
 no page twice), per-segment page counts = ceil(len / page_size), lengths equal
@@ -37,6 +42,7 @@ CAPACITY = "CAPACITY"
 WINDOW_NOT_FULL = "WINDOW_NOT_FULL"
 WINDOW_FULL = "WINDOW_FULL"
 INVALID_ARG = "INVALID_ARG"
+DEBUG_CHECK = "DEBUG_CHECK"
 
 
 def _ceil_div(a, b):
@@ -56,13 +62,14 @@ class _Seq:
 
 class PagingModel:
     def __init__(self, num_pages, page_size, max_seqs, max_pages_per_seq,
-                 max_entries_per_seq=0, c_default=1):
+                 max_entries_per_seq=0, c_default=1, debug_bounds=False):
         self.ps = page_size
         self.num_pages = num_pages
         self.max_seqs = max_seqs
         self.max_pages_per_seq = max_pages_per_seq
         self.max_entries = max_entries_per_seq
         self.c_default = c_default
+        self.debug_bounds = debug_bounds
         self.stack = list(range(num_pages - 1, -1, -1))   # stack[-1] == page 0
         self.seqs = {}
         self.first_error = None       # (code, slot, call_index)
@@ -70,6 +77,10 @@ class PagingModel:
         self.calls = 0
 
     # ------------------------------------------------------------------ utils
+    def _dup(self, slots, i):
+        """Checked mode: does an item with a lower batch index name the same slot?"""
+        return self.debug_bounds and slots[i] in slots[:i]
+
     def _fail(self, code, slot, item):
         self._pending.append((item, code, slot))
         return code
@@ -109,6 +120,8 @@ class PagingModel:
             P = prompt_lens[i]
             if not (0 <= slot < self.max_seqs) or slot in self.seqs:
                 res[i] = self._fail(BAD_SLOT, slot, i); continue
+            if self._dup(slots, i):
+                res[i] = self._fail(DEBUG_CHECK, slot, i); continue
             if c < 1 or P < 0:
                 res[i] = self._fail(INVALID_ARG, slot, i); continue
             npp = _ceil_div(P, self.ps)
@@ -132,6 +145,8 @@ class PagingModel:
             s = self.seqs.get(slot)
             if s is None:
                 res[i] = self._fail(BAD_SLOT, slot, i); continue
+            if self._dup(slots, i):
+                res[i] = self._fail(DEBUG_CHECK, slot, i); continue
             if s.c > 1 and s.window_len >= s.c:
                 res[i] = self._fail(WINDOW_FULL, slot, i); continue
             if self.max_entries and s.n_beacons + s.window_len + 1 > self.max_entries:
@@ -157,6 +172,8 @@ class PagingModel:
             s = self.seqs.get(slot)
             if s is None:
                 res[i] = self._fail(BAD_SLOT, slot, i); continue
+            if self._dup(slots, i):
+                res[i] = self._fail(DEBUG_CHECK, slot, i); continue
             if s.c <= 1 or s.window_len != s.c:
                 res[i] = self._fail(WINDOW_NOT_FULL, slot, i); continue
             need = 1 if s.n_beacons % self.ps == 0 else 0
@@ -190,6 +207,8 @@ class PagingModel:
             T = gen_lens[i]
             if s is None:
                 res[i] = self._fail(BAD_SLOT, slot, i); continue
+            if self._dup(slots, i):
+                res[i] = self._fail(DEBUG_CHECK, slot, i); continue
             if T < 0 or s.t != 0 or s.n_beacons != 0 or s.window_len != 0:
                 res[i] = self._fail(INVALID_ARG, slot, i); continue
             nb = T // s.c if s.c > 1 else 0
@@ -215,10 +234,13 @@ class PagingModel:
     def close(self, slots):
         self.calls += 1
         res = [None] * len(slots)
+        open_at_start = set(self.seqs)           # every item is validated against the state the call finds
         for i, slot in enumerate(slots):
-            s = self.seqs.get(slot)
-            if s is None:
+            if slot not in open_at_start or (not self.debug_bounds and slot not in self.seqs):
                 res[i] = self._fail(BAD_SLOT, slot, i); continue
+            if self._dup(slots, i):
+                res[i] = self._fail(DEBUG_CHECK, slot, i); continue
+            s = self.seqs[slot]
             self.stack.extend(s.prompt_pages + s.beacon_pages + s.window_pages)
             del self.seqs[slot]; res[i] = OK
         return self._latch(res)

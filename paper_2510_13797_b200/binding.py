@@ -19,11 +19,11 @@ from . import build as _build
 BC_OK = 0
 BC_ERR_INVALID_ARG, BC_ERR_BAD_SLOT, BC_ERR_NO_PAGES, BC_ERR_CAPACITY = -1, -2, -3, -4
 BC_ERR_WINDOW_NOT_FULL, BC_ERR_WINDOW_FULL, BC_ERR_ORDER, BC_ERR_CUDA = -5, -6, -7, -8
-BC_ERR_UNSUPPORTED, BC_ERR_TIMEOUT, BC_ERR_TOO_LARGE = -9, -10, -11
-BC_FLAG_OUT_F32, BC_FLAG_ATTN_REFERENCE, BC_FLAG_HOST_PIPELINED = 1, 2, 4
+BC_ERR_UNSUPPORTED, BC_ERR_TIMEOUT, BC_ERR_TOO_LARGE, BC_ERR_DEBUG_CHECK = -9, -10, -11, -12
+BC_FLAG_OUT_F32, BC_FLAG_ATTN_REFERENCE, BC_FLAG_HOST_PIPELINED, BC_FLAG_DEBUG_BOUNDS = 1, 2, 4, 8
 STATUS_NAMES = {0: "OK", -1: "INVALID_ARG", -2: "BAD_SLOT", -3: "NO_PAGES", -4: "CAPACITY",
                 -5: "WINDOW_NOT_FULL", -6: "WINDOW_FULL", -7: "ORDER", -8: "CUDA",
-                -9: "UNSUPPORTED", -10: "TIMEOUT", -11: "TOO_LARGE"}
+                -9: "UNSUPPORTED", -10: "TIMEOUT", -11: "TOO_LARGE", -12: "DEBUG_CHECK"}
 
 
 class BcConfig(C.Structure):
@@ -79,6 +79,8 @@ SYMBOLS = {
     "bc_export_seq": (_I32, [_P, _I32, _I32, _P, _P, _I32, _P]),
     "bc_set_attn_ctas": (_I32, [_P, _I32]),
     "bc_attn_timeline": (_I32, [_P, _P, _I32]),
+    "bc_set_wait_limit": (_I32, [_P, C.c_uint32]),
+    "bc_mask_attn_set_wait_limit": (_I32, [C.c_uint32]),
     "bc_profile_enable": (_I32, [_P, _I32]),
     "bc_profile_read": (_I32, [_P, C.POINTER(_I32), C.POINTER(_F)]),
     "bc_kernel_launches": (_I64, [_P]),
@@ -246,6 +248,9 @@ class Cache:
 
     def bc_set_attn_ctas(self, ctas):
         _check(lib().bc_set_attn_ctas(self.handle, ctas), "bc_set_attn_ctas")
+
+    def bc_set_wait_limit(self, polls):
+        _check(lib().bc_set_wait_limit(self.handle, polls), "bc_set_wait_limit")
 
     def bc_attn_timeline(self, words, blocks=0):
         """words: uint64/int64 CUDA tensor of at least blocks * 16 elements, or None to switch it off."""

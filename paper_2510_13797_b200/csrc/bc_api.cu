@@ -14,7 +14,7 @@ namespace {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct MetaLayout {
-  size_t status, free_top, open, prompt_len, n_beacons, window_len, c, t, window_off, beacon_off, free_stack,
+  size_t status, free_top, open, prompt_len, n_beacons, window_len, c, t, window_off, beacon_off, dup_mark, free_stack,
       page_table, total;
 };
 MetaLayout meta_layout(const bc_config& c) {
@@ -25,6 +25,7 @@ MetaLayout meta_layout(const bc_config& c) {
   l.status = take(16); l.free_top = take(4);
   l.open = take(seq); l.prompt_len = take(seq); l.n_beacons = take(seq); l.window_len = take(seq);
   l.c = take(seq); l.t = take(seq); l.window_off = take(seq); l.beacon_off = take(seq);
+  l.dup_mark = take(2 * seq);
   l.free_stack = take((size_t)c.num_pages * 4);
   l.page_table = take((size_t)c.max_seqs * c.max_pages_per_seq * 4);
   l.total = o;
@@ -107,6 +108,7 @@ struct bc_cache {
   // has not been followed by an ordinarily launched kernel or an attention launch of this handle: an
   // attention kernel enqueued now could begin before that writer has ended and must not read early
   bool meta_unsettled = true;
+  uint32_t wait_limit = 0;      // bc_set_wait_limit: polls of the attention kernel's bounded waits (0: default)
   void* timeline = nullptr;     // bc_attn_timeline: device buffer the attention kernel stamps, or NULL
   int device = -1;              // the CUDA device that was current at bc_cache_create
   bool static_used = false;     // a bc_decode_attn_static launch was issued since the last bc_clear_error
@@ -175,6 +177,8 @@ bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const v
   a.tickets = work_ptr<int32_t>(c, c->wl.tickets);
   a.ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
   a.timeline = c->timeline;
+  a.spin_limit = c->wait_limit;
+  a.debug = c->meta.debug;
   a.meta_settled = c->meta_unsettled ? 0 : 1;
   c->meta_unsettled = false;   // whatever follows this launch starts after its blocks have waited for the writer
   if (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) {
@@ -267,6 +271,7 @@ const char* bc_status_string(bc_status s) {
     case BC_ERR_UNSUPPORTED: return "BC_ERR_UNSUPPORTED";
     case BC_ERR_TIMEOUT: return "BC_ERR_TIMEOUT";
     case BC_ERR_TOO_LARGE: return "BC_ERR_TOO_LARGE";
+    case BC_ERR_DEBUG_CHECK: return "BC_ERR_DEBUG_CHECK";
     default: return "BC_ERR_UNKNOWN";
   }
 }
@@ -301,6 +306,8 @@ bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* wo
   m.open = at(c->ml.open); m.prompt_len = at(c->ml.prompt_len); m.n_beacons = at(c->ml.n_beacons);
   m.window_len = at(c->ml.window_len); m.c = at(c->ml.c); m.t = at(c->ml.t);
   m.window_off = at(c->ml.window_off); m.beacon_off = at(c->ml.beacon_off); m.page_table = at(c->ml.page_table);
+  m.dup_mark = reinterpret_cast<unsigned long long*>(c->meta_base + c->ml.dup_mark);
+  m.debug = (cfg->flags & BC_FLAG_DEBUG_BOUNDS) ? 1 : 0;
   m.max_seqs = cfg->max_seqs; m.num_pages = cfg->num_pages; m.max_pages_per_seq = cfg->max_pages_per_seq;
   m.max_entries = cfg->max_entries_per_seq; m.page_size = cfg->page_size; m.c_default = cfg->c_default;
   BcGeom& g = c->geom;
@@ -421,7 +428,7 @@ bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n,
     c->meta_unsettled = true;
   }
   if (!fused) {
-    BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, k, v, n, s));
+    BC_CUDA(c, bc_launch_write_rows(c->meta, c->geom, layer_base(c, layer), row, pos, k, v, n, s));
     c->launches += 1;
     c->meta_unsettled = false;
   }
@@ -542,7 +549,7 @@ bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t 
     c->meta_unsettled = true;
   }
   if (!fused) {
-    BC_CUDA(c, bc_launch_write_rows(c->geom, layer_base(c, layer), row, pos, bk, bv, n, s));
+    BC_CUDA(c, bc_launch_write_rows(c->meta, c->geom, layer_base(c, layer), row, pos, bk, bv, n, s));
     c->launches += 1;
     c->meta_unsettled = false;
   }
@@ -796,6 +803,12 @@ bc_status bc_set_attn_ctas(bc_cache* c, int32_t ctas) {
   return BC_OK;
 }
 
+bc_status bc_set_wait_limit(bc_cache* c, uint32_t polls) {
+  if (!c) return BC_ERR_INVALID_ARG;
+  c->wait_limit = polls;
+  return BC_OK;
+}
+
 bc_status bc_attn_timeline(bc_cache* c, void* device_words, int32_t blocks) {
   if (!c) return BC_ERR_INVALID_ARG;
   if (device_words == nullptr) { c->timeline = nullptr; return BC_OK; }
@@ -875,6 +888,8 @@ bc_status bc_decode_attn_static(bc_cache* c, int32_t layer, const int32_t* slots
   int ctas = c->attn_ctas > 0 ? c->attn_ctas : c->sm_count;
   a.ctas = ctas < BC_STATIC_MAX_CTAS ? ctas : BC_STATIC_MAX_CTAS;
   int launches = 0;
+  a.spin_limit = c->wait_limit;
+  a.debug = c->meta.debug;
   a.meta_settled = c->meta_unsettled ? 0 : 1;
   c->meta_unsettled = false;
   c->static_used = true;

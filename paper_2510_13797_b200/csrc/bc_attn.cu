@@ -134,11 +134,30 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 }
 
 // Bounded wait; returns false when it gave up or another warp already aborted.
-__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {   // never suspends the thread
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+constexpr uint32_t kShortLimit = 1024;   // limits below this poll without suspending (try_wait may sleep for a while inside)
+
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
+  if (limit < kShortLimit) {   // a deliberately short limit (bc_set_wait_limit): a few non-blocking looks, then give up
+    for (uint32_t polls = 0; polls <= limit; ++polls)
+      if (mbar_test_wait(bar, parity)) return true;
+    *abort_flag = 1;
+    return false;
+  }
   uint32_t polls = 0;
   while (!mbar_try_wait(bar, parity)) {
     if (++polls > 1024) __nanosleep(64);
-    if (polls > kSpinLimit || *abort_flag) {
+    if (polls > limit || *abort_flag) {
       *abort_flag = 1;
       return false;
     }
@@ -182,6 +201,10 @@ struct PipeParams {
   int n_groups;       // 8 / kv_heads
   int G;              // q_heads / kv_heads
   FastDiv div_ps;     // division by page_size
+  uint32_t spin_limit;            // polls after which a wait of a consumer, producer or service warp gives up
+                                  // (kSpinLimit unless bc_set_wait_limit lowered it); the final drain of copies
+                                  // in flight always uses kSpinLimit
+  int debug;                      // BC_FLAG_DEBUG_BOUNDS: every page-table column, page id and pool row is checked
   unsigned long long* timeline;   // NULL, or [gridDim.x][kTimelineSlots] device words: %globaltimer stamps of one thread per block
   int early_meta;     // 1: the cache's metadata was last written by a kernel that has ENDED, so the plan and the
                       // first page-table reads may run before the wait for the kernel ahead; 0: wait first
@@ -461,6 +484,10 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       const int chunks = p.g.head_row_bytes >> 4, per_side = Hkv * chunks;
       for (int i = seq0; i < n && s_cum[i + 1] - 1 < g1; ++i) {
         if (s_cum[i + 1] - 1 < g0 || !(s_slot[i] & kNewRowBit)) continue;
+        if (p.debug && (unsigned)p.f.dst_row[i] >= (unsigned)(p.m.num_pages * ps)) {   // row outside the pool: not written
+          if (lane == 0) debug_note(p.m, p.f.dst_row[i]);
+          continue;
+        }
         uint8_t* dst = p.f.pool_w + (int64_t)p.f.dst_row[i] * E;
         const int key = p.f.dst_pos[i] & 7;
         for (int idx = lane; idx < 2 * per_side; idx += 32) {
@@ -472,7 +499,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       }
     }
     if (svc_publishes) {
-      const bool ok = bounded_wait(bar_pub, 0, s_abort);  // every consumer warp has stored its share
+      const bool ok = bounded_wait(bar_pub, 0, s_abort, p.spin_limit);  // every consumer warp has stored its share
       if (lane == 0) {
         if (ok) {
           __threadfence();
@@ -520,8 +547,14 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
         if (nrows > 0) {
           pg0 = fast_div(p0, p.div_ps);
           const int pg_last = fast_div(p0 + nrows - 1, p.div_ps);
-          for (int pg = pg0 + lane; pg <= pg_last; pg += 32)
-            cp_async4(desc_ring + (uint32_t)(slot_idx + 4 + pg - pg0) * 4u, f_tab + col + pg);
+          for (int pg = pg0 + lane; pg <= pg_last; pg += 32) {
+            if (p.debug && (unsigned)(col + pg) >= (unsigned)p.m.max_pages_per_seq) {   // column outside the row
+              debug_note(p.m, col + pg);
+              s_desc[slot_idx + 4 + pg - pg0] = 0;
+            } else {
+              cp_async4(desc_ring + (uint32_t)(slot_idx + 4 + pg - pg0) * 4u, f_tab + col + pg);
+            }
+          }
         }
       }
       // settled: every row of the tile was stored by a kernel that has ended by the time this one may
@@ -550,12 +583,13 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       if (!waited && !s_desc[(it % RING) * kPidSlot + 3]) { wait_for_kernel_ahead(); waited = true; }
       const int stage = it % NSTAGE;
       const uint32_t full = bar_full + stage * 8, empty = bar_empty + stage * 8;
-      if (!aborted && !bounded_wait(empty, ((it / NSTAGE) & 1) ^ 1, s_abort)) aborted = true;
+      if (!bounded_wait(empty, ((it / NSTAGE) & 1) ^ 1, s_abort, p.spin_limit)) aborted = true;
       // at most kInFlight stages in flight: the copies of tile it - kInFlight must have landed
       if (!aborted && it >= kInFlight &&
-          !bounded_wait(bar_full + ((it - kInFlight) % NSTAGE) * 8, ((it - kInFlight) / NSTAGE) & 1, s_abort))
+          !bounded_wait(bar_full + ((it - kInFlight) % NSTAGE) * 8, ((it - kInFlight) / NSTAGE) & 1, s_abort, p.spin_limit))
         aborted = true;
-      if (!aborted) {
+      if (aborted) break;   // `it` stages have been armed; the consumers see the abort flag in their own waits
+      {
         const int* d = s_desc + (it % RING) * kPidSlot;
         const int nrows = d[0], p0 = d[1], pg0 = d[2];
         if (lane == 0) {
@@ -567,7 +601,9 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
           const int pg = pg0 + k;
           const int lo = max(p0, pg * ps), hi = min(p0 + nrows, pg * ps + ps);
           if (lo >= hi) break;
-          const uint8_t* src = p.a.pool_layer + ((int64_t)d[4 + k] * ps + (lo - pg * ps)) * E;
+          int page = d[4 + k];
+          if (p.debug && (unsigned)page >= (unsigned)p.m.num_pages) { debug_note(p.m, page); page = 0; }   // read a valid page instead
+          const uint8_t* src = p.a.pool_layer + ((int64_t)page * ps + (lo - pg * ps)) * E;
           bulk_g2s(stage_base + (uint32_t)(lo - p0) * (uint32_t)E, src, (uint32_t)(hi - lo) * (uint32_t)E, full, stream_policy);
         }
       }
@@ -697,7 +733,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
                                                         ((int64_t)i * Hkv + kvh) * p.g.head_row_bytes + ((lane & 15) << 4));
         }
       }
-      const bool ok = __all_sync(0xffffffffu, bounded_wait(bar_full + stage * 8, (it / NSTAGE) & 1, s_abort));
+      const bool ok = __all_sync(0xffffffffu, bounded_wait(bar_full + stage * 8, (it / NSTAGE) & 1, s_abort, p.spin_limit));
       if (it == 0) stamp(3);
       if (!ok && lane == 0 && p.m.status[0] == 0) { p.m.status[0] = BC_ERR_TIMEOUT; p.m.status[1] = -1; }
       // rows of this tile that hold entries; my warp looks at rows grp*16 .. grp*16+15 of it
@@ -983,7 +1019,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
 
   // ---- all tiles streamed: merge the sequences whose last ticket this block took -----------------
   stamp(5);
-  if (svc_publishes) bounded_wait(bar_tk, 0, s_abort);
+  if (svc_publishes) bounded_wait(bar_tk, 0, s_abort, p.spin_limit);
   stamp(6);
   if (published_last) {
     if (tid == 0) { s_pend[2] = pend_seq; s_pend[3] = pend_tk; }
@@ -1112,6 +1148,8 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   p.m = m; p.g = g; p.a = a;
   p.early_meta = (a.meta_settled && !fused) ? 1 : 0;
   p.timeline = reinterpret_cast<unsigned long long*>(a.timeline);
+  p.spin_limit = a.spin_limit ? a.spin_limit : kSpinLimit;
+  p.debug = a.debug;
   p.f = FusedArgs{};
   if (fused) {
     p.f.new_k = static_cast<const uint8_t*>(fused->new_k); p.f.new_v = static_cast<const uint8_t*>(fused->new_v);

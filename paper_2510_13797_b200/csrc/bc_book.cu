@@ -16,7 +16,7 @@ constexpr int kBookThreads = 1024;
 // per thread and step, applying the chunk permutation of the store layout.  Items with
 // dst_row < 0 (failed validation) are skipped.  Used by the single-block kernels that have just
 // computed dst_row/dst_pos (their global writes are visible to the block after __syncthreads).
-__device__ void block_write_rows(const BcGeom& g, uint8_t* __restrict__ pool_layer, const int32_t* dst_row,
+__device__ void block_write_rows(const BcMeta& m, const BcGeom& g, uint8_t* __restrict__ pool_layer, const int32_t* dst_row,
                                  const int32_t* dst_pos, const uint8_t* __restrict__ k,
                                  const uint8_t* __restrict__ v, int n) {
   const int chunks_per_head = g.head_row_bytes >> 4;
@@ -26,6 +26,7 @@ __device__ void block_write_rows(const BcGeom& g, uint8_t* __restrict__ pool_lay
     const int i = idx / per_item, r = idx - i * per_item;
     const int row = dst_row[i];
     if (row < 0) continue;
+    if (m.debug && row >= m.num_pages * g.page_size) { debug_note(m, row); continue; }
     const int which = r / per_side, rem = r - which * per_side;
     const int h = rem / chunks_per_head, j = rem - h * chunks_per_head;
     const uint8_t* src = (which ? v : k) + ((int64_t)i * g.kv_heads + h) * g.head_row_bytes + (j << 4);
@@ -40,6 +41,7 @@ __global__ void k_init(BcMeta m) {
   for (int i = tid; i < m.max_seqs; i += nth) {
     m.open[i] = 0; m.prompt_len[i] = 0; m.n_beacons[i] = 0; m.window_len[i] = 0;
     m.c[i] = 0; m.t[i] = 0; m.window_off[i] = 0; m.beacon_off[i] = 0;
+    m.dup_mark[i] = 0ull;
   }
   if (tid == 0) {
     *m.free_top = m.num_pages;
@@ -52,6 +54,7 @@ k_open(BcMeta m, const int32_t* __restrict__ slots, const int32_t* __restrict__ 
        const int32_t* __restrict__ cs, int n, int64_t call) {
   __shared__ int sh_first;
   ErrLatch latch; latch.init(&sh_first);
+  dup_prepass(m, slots, n, call);
   const int top0 = *m.free_top;
   __syncthreads();
   int base = 0, used = 0, my_code = 0, my_item = -1, my_slot = 0;
@@ -62,6 +65,7 @@ k_open(BcMeta m, const int32_t* __restrict__ slots, const int32_t* __restrict__ 
     if (i < n) {
       slot = slots[i]; P = plens[i]; c = cs ? cs[i] : m.c_default;
       if (slot < 0 || slot >= m.max_seqs || m.open[slot]) code = BC_ERR_BAD_SLOT;
+      else if (is_dup(m, slot, i, call)) code = BC_ERR_DEBUG_CHECK;
       else if (c < 1 || P < 0) code = BC_ERR_INVALID_ARG;
       else {
         need = ceil_div(P, m.page_size);
@@ -107,7 +111,7 @@ k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
               int32_t* dst_row, int32_t* dst_pos, BcGeom g, uint8_t* pool_layer, const uint8_t* k, const uint8_t* v) {
   append_book_block(m, slots, n, call, dst_row, dst_pos);
   __syncthreads();
-  if (k != nullptr) block_write_rows(g, pool_layer, dst_row, dst_pos, k, v, n);  // layer 0's rows, same launch
+  if (k != nullptr) block_write_rows(m, g, pool_layer, dst_row, dst_pos, k, v, n);  // layer 0's rows, same launch
   wait_for_overtaken_kernel();
 }
 
@@ -124,6 +128,7 @@ k_compress_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call
   __syncthreads();
   if (phase & 1) {
     ErrLatch latch; latch.init(&sh_first);
+    dup_prepass(m, slots, n, call);
     int base = 0, used = 0, my_code = 0, my_item = -1, my_slot = 0;
     for (int chunk = 0; chunk < n; chunk += blockDim.x) {
       const int i = chunk + threadIdx.x;
@@ -132,6 +137,7 @@ k_compress_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call
       if (i < n) {
         slot = slots[i];
         if (slot < 0 || slot >= m.max_seqs || !m.open[slot]) code = BC_ERR_BAD_SLOT;
+        else if (is_dup(m, slot, i, call)) code = BC_ERR_DEBUG_CHECK;
         else {
           const int c = m.c[slot];
           nb = m.n_beacons[slot];
@@ -152,7 +158,7 @@ k_compress_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call
         if (need == 0 || off + need <= top) {
           int32_t* col = m.page_table + (int64_t)slot * m.max_pages_per_seq + m.beacon_off[slot] + nb / ps;
           if (need) { *col = m.free_stack[top - 1 - off]; used = max(used, off + 1); }
-          row_out = *col * ps + nb % ps;
+          if (debug_page_ok(m, *col)) row_out = *col * ps + nb % ps;
         } else code = BC_ERR_NO_PAGES;
       }
       if (i < n) { dst_row[i] = row_out; dst_pos[i] = nb; }
@@ -190,7 +196,7 @@ k_compress_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call
   }
   __syncthreads();
   if (threadIdx.x == 0) *m.free_top = top;
-  if (k != nullptr) block_write_rows(g, pool_layer, dst_row, dst_pos, k, v, n);  // the beacon rows, same launch
+  if (k != nullptr) block_write_rows(m, g, pool_layer, dst_row, dst_pos, k, v, n);  // the beacon rows, same launch
   wait_for_overtaken_kernel();
 }
 
@@ -198,6 +204,7 @@ __global__ void __launch_bounds__(kBookThreads, 1)
 k_close(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call) {
   __shared__ int sh_first;
   ErrLatch latch; latch.init(&sh_first);
+  dup_prepass(m, slots, n, call);
   const int ps = m.page_size;
   const int top = *m.free_top;
   __syncthreads();
@@ -208,6 +215,7 @@ k_close(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call) {
     if (i < n) {
       slot = slots[i];
       if (slot < 0 || slot >= m.max_seqs || !m.open[slot]) { code = BC_ERR_BAD_SLOT; slot = -1; }
+      else if (is_dup(m, slot, i, call)) { code = BC_ERR_DEBUG_CHECK; slot = -1; }
       else {
         np = ceil_div(m.prompt_len[slot], ps);
         nbp = ceil_div(m.n_beacons[slot], ps);
@@ -235,7 +243,7 @@ k_close(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call) {
 
 // One block per batch item: copies the item's K and V rows (all heads) into its pool row,
 // 16 bytes per thread, applying the chunk permutation of the store layout.
-__global__ void k_write_rows(BcGeom g, uint8_t* __restrict__ pool_layer, const int32_t* __restrict__ dst_row,
+__global__ void k_write_rows(BcMeta m, BcGeom g, uint8_t* __restrict__ pool_layer, const int32_t* __restrict__ dst_row,
                              const int32_t* __restrict__ dst_pos, const uint8_t* __restrict__ k,
                              const uint8_t* __restrict__ v, int n) {
   // the attention kernel of the step may start planning now; it waits for this kernel before it reads a row
@@ -243,6 +251,7 @@ __global__ void k_write_rows(BcGeom g, uint8_t* __restrict__ pool_layer, const i
   const int i = blockIdx.x;
   const int row = dst_row[i];
   if (row < 0) return;
+  if (m.debug && row >= m.num_pages * g.page_size) { if (threadIdx.x == 0) debug_note(m, row); return; }
   const int pos = dst_pos[i];
   const int chunks_per_head = g.head_row_bytes >> 4;
   const int per_side = g.kv_heads * chunks_per_head;
@@ -267,8 +276,12 @@ __global__ void k_prefill(BcMeta m, BcGeom g, uint8_t* __restrict__ pool_layer, 
     const int slot = slots[lo], pos = tok - cu[lo];
     int row = -1;
     if (slot >= 0 && slot < m.max_seqs && m.open[slot] && pos < m.prompt_len[slot]) {
-      const int page = m.page_table[(int64_t)slot * m.max_pages_per_seq + pos / g.page_size];
-      row = page * g.page_size + pos % g.page_size;
+      const int col = pos / g.page_size;
+      if (m.debug && col >= m.max_pages_per_seq) debug_note(m, col);
+      else {
+        const int page = m.page_table[(int64_t)slot * m.max_pages_per_seq + col];
+        if (debug_page_ok(m, page)) row = page * g.page_size + pos % g.page_size;
+      }
     }
     sh_row = row; sh_pos = pos;
   }
@@ -298,6 +311,7 @@ k_restore_book(BcMeta m, const int32_t* __restrict__ slots, const int32_t* __res
                int32_t* __restrict__ ok, int32_t* __restrict__ bea) {
   __shared__ int sh_first;
   ErrLatch latch; latch.init(&sh_first);
+  dup_prepass(m, slots, n, call);
   const int top0 = *m.free_top;
   const int ps = m.page_size;
   __syncthreads();
@@ -312,8 +326,9 @@ k_restore_book(BcMeta m, const int32_t* __restrict__ slots, const int32_t* __res
       if (slot < 0 || slot >= m.max_seqs || !m.open[slot]) code = BC_ERR_BAD_SLOT;
       else {
         const int c = m.c[slot];
-        if (T >= 0) { nb = c > 1 ? T / c : 0; w = T - nb * c; rows = nb; }
-        if (T < 0 || m.t[slot] != 0 || m.n_beacons[slot] != 0 || m.window_len[slot] != 0) code = BC_ERR_INVALID_ARG;
+        if (T >= 0) { nb = c > 1 ? T / c : 0; w = T - nb * c; rows = nb; }   // an open slot's item has beacon rows in the packed input
+        if (is_dup(m, slot, i, call)) code = BC_ERR_DEBUG_CHECK;
+        else if (T < 0 || m.t[slot] != 0 || m.n_beacons[slot] != 0 || m.window_len[slot] != 0) code = BC_ERR_INVALID_ARG;
         else if (m.max_entries > 0 && nb + w > m.max_entries) code = BC_ERR_CAPACITY;
         else {
           nbp = ceil_div(nb, ps); nwp = ceil_div(w, ps);
@@ -380,8 +395,12 @@ __global__ void k_restore_beacons(BcMeta m, BcGeom g, uint8_t* __restrict__ pool
       if (ok[lo]) {
         const int slot = slots[lo];
         pos = b - bea[lo];
-        const int page = m.page_table[(int64_t)slot * m.max_pages_per_seq + m.beacon_off[slot] + pos / g.page_size];
-        row = page * g.page_size + pos % g.page_size;
+        const int col = m.beacon_off[slot] + pos / g.page_size;
+        if (m.debug && (unsigned)col >= (unsigned)m.max_pages_per_seq) debug_note(m, col);
+        else {
+          const int page = m.page_table[(int64_t)slot * m.max_pages_per_seq + col];
+          if (debug_page_ok(m, page)) row = page * g.page_size + pos % g.page_size;
+        }
       }
     }
     sh_row = row; sh_pos = pos;
@@ -403,7 +422,13 @@ __global__ void k_restore_window(BcMeta m, BcGeom g, uint8_t* __restrict__ pool_
   const int32_t* cols = m.page_table + (int64_t)slot * m.max_pages_per_seq + m.window_off[slot];
   for (int j = blockIdx.y; j < w; j += gridDim.y) {
     if (first + j < 0 || first + j >= total_tokens) continue;
-    copy_entry(g, pool_layer, cols[j / g.page_size] * g.page_size + j % g.page_size, j, k, v, first + j);
+    if (m.debug && (unsigned)(m.window_off[slot] + j / g.page_size) >= (unsigned)m.max_pages_per_seq) {
+      if (threadIdx.x == 0) debug_note(m, m.window_off[slot] + j / g.page_size);
+      continue;
+    }
+    const int page = cols[j / g.page_size];
+    if (m.debug && (unsigned)page >= (unsigned)m.num_pages) { if (threadIdx.x == 0) debug_note(m, page); continue; }
+    copy_entry(g, pool_layer, page * g.page_size + j % g.page_size, j, k, v, first + j);
   }
 }
 
@@ -418,7 +443,12 @@ __global__ void k_export(BcMeta m, BcGeom g, const uint8_t* __restrict__ pool_la
   if (e < P) { pos = e; col0 = 0; }
   else if (e < P + nb) { pos = e - P; col0 = m.beacon_off[slot]; }
   else { pos = e - P - nb; col0 = m.window_off[slot]; }
+  if (m.debug && (unsigned)(col0 + pos / g.page_size) >= (unsigned)m.max_pages_per_seq) {
+    if (threadIdx.x == 0) debug_note(m, col0 + pos / g.page_size);
+    return;
+  }
   const int page = m.page_table[(int64_t)slot * m.max_pages_per_seq + col0 + pos / g.page_size];
+  if (m.debug && (unsigned)page >= (unsigned)m.num_pages) { if (threadIdx.x == 0) debug_note(m, page); return; }
   const uint8_t* src = pool_layer + ((int64_t)page * g.page_size + pos % g.page_size) * g.entry_bytes;
   const int chunks_per_head = g.head_row_bytes >> 4;
   const int per_side = g.kv_heads * chunks_per_head;
@@ -486,9 +516,9 @@ cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_
   k_close<<<1, kBookThreads, 0, s>>>(m, slots, n, call);
   return cudaGetLastError();
 }
-cudaError_t bc_launch_write_rows(const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
+cudaError_t bc_launch_write_rows(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
                                  const void* k, const void* v, int n, cudaStream_t s) {
-  k_write_rows<<<n, copy_threads(g), 0, s>>>(g, pool_layer, dst_row, dst_pos, (const uint8_t*)k, (const uint8_t*)v, n);
+  k_write_rows<<<n, copy_threads(g), 0, s>>>(m, g, pool_layer, dst_row, dst_pos, (const uint8_t*)k, (const uint8_t*)v, n);
   return cudaGetLastError();
 }
 cudaError_t bc_launch_prefill(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* slots,

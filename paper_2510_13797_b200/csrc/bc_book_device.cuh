@@ -37,6 +37,34 @@ __device__ int block_exclusive_scan(int x, int* total) {
   return warp_sums[warp] + incl - x;
 }
 
+// ---- BC_FLAG_DEBUG_BOUNDS -------------------------------------------------------------------------
+// Records a failed check (the offending value in the record's slot field) unless an error is latched
+// already.  The caller skips or redirects the access; nothing traps.
+__device__ __forceinline__ void debug_note(const BcMeta& m, int value) {
+  if (atomicCAS(m.status, 0, BC_ERR_DEBUG_CHECK) == 0) m.status[1] = value;
+}
+// A page id read from the page table or the free stack: true if it lies in the pool.
+__device__ __forceinline__ bool debug_page_ok(const BcMeta& m, int page) {
+  if (!m.debug || (unsigned)page < (unsigned)m.num_pages) return true;
+  debug_note(m, page);
+  return false;
+}
+// A batch must not name a slot twice.  With the flag set every bookkeeping kernel (one thread block)
+// first marks, per slot, the lowest batch index that names it in this call; an item that is not that
+// one is refused with BC_ERR_DEBUG_CHECK, so the first occurrence goes through alone.
+__device__ void dup_prepass(const BcMeta& m, const int32_t* __restrict__ slots, int n, int64_t call) {
+  if (!m.debug) return;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int slot = slots[i];
+    if (slot >= 0 && slot < m.max_seqs)
+      atomicMax(m.dup_mark + slot, ((unsigned long long)call << 32) | (0xffffffffu - (unsigned)i));
+  }
+  __syncthreads();
+}
+__device__ __forceinline__ bool is_dup(const BcMeta& m, int slot, int i, int64_t call) {
+  return m.debug && m.dup_mark[slot] != (((unsigned long long)call << 32) | (0xffffffffu - (unsigned)i));
+}
+
 // Per-call error latch: the failing item with the lowest batch index reports, and only if no
 // earlier call has latched an error.
 struct ErrLatch {
@@ -67,6 +95,7 @@ __device__ void append_book_block(const BcMeta& m, const int32_t* __restrict__ s
                                   int32_t* dst_pos) {
   __shared__ int sh_first;
   ErrLatch latch; latch.init(&sh_first);
+  dup_prepass(m, slots, n, call);
   const int top0 = *m.free_top;
   const int ps = m.page_size;
   __syncthreads();
@@ -78,6 +107,7 @@ __device__ void append_book_block(const BcMeta& m, const int32_t* __restrict__ s
     if (i < n) {
       slot = slots[i];
       if (slot < 0 || slot >= m.max_seqs || !m.open[slot]) code = BC_ERR_BAD_SLOT;
+      else if (is_dup(m, slot, i, call)) code = BC_ERR_DEBUG_CHECK;
       else {
         const int c = m.c[slot], nb = m.n_beacons[slot];
         w = m.window_len[slot];
@@ -99,9 +129,11 @@ __device__ void append_book_block(const BcMeta& m, const int32_t* __restrict__ s
       if (need == 0 || off + need <= top0) {
         int32_t* col = m.page_table + (int64_t)slot * m.max_pages_per_seq + m.window_off[slot] + w / ps;
         if (need) { *col = m.free_stack[top0 - 1 - off]; used = max(used, off + 1); }
-        row_out = *col * ps + w % ps;
-        m.window_len[slot] = w + 1;
-        m.t[slot] += 1;
+        if (debug_page_ok(m, *col)) {
+          row_out = *col * ps + w % ps;
+          m.window_len[slot] = w + 1;
+          m.t[slot] += 1;
+        }
       } else code = BC_ERR_NO_PAGES;
     }
     if (i < n) { dst_row[i] = row_out; dst_pos[i] = w; }

@@ -28,7 +28,9 @@ struct BcMeta {
   int32_t* window_off;  // [max_seqs] column of the first window page in the page-table row
   int32_t* beacon_off;  // [max_seqs] column of the first beacon page
   int32_t* page_table;  // [max_seqs][max_pages_per_seq]: prompt pages from column 0
+  unsigned long long* dup_mark;  // [max_seqs] BC_FLAG_DEBUG_BOUNDS: (call index << 32 | ~first batch index) of the last call naming the slot
   int32_t max_seqs, num_pages, max_pages_per_seq, max_entries, page_size, c_default;
+  int32_t debug;        // BC_FLAG_DEBUG_BOUNDS set
 };
 
 // Geometry of the K/V pool for one cache.
@@ -59,7 +61,8 @@ cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n
                                     int32_t* dst_pos, int phase, const BcGeom& g, uint8_t* pool_layer, const void* k,
                                     const void* v, cudaStream_t s);
 cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_t call, cudaStream_t s);
-cudaError_t bc_launch_write_rows(const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
+// m is used for the checks of BC_FLAG_DEBUG_BOUNDS only
+cudaError_t bc_launch_write_rows(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
                                  const void* k, const void* v, int n, cudaStream_t s);
 cudaError_t bc_launch_restore_book(const BcMeta& m, const int32_t* slots, const int32_t* cu, int n, int64_t call, int32_t* ok,
                                    int32_t* bea, cudaStream_t s);
@@ -87,6 +90,8 @@ struct BcAttnArgs {
   int32_t* tickets;      // [n] pieces of each sequence published so far; zero between launches
   int32_t ctas;
   void* timeline = nullptr;  // NULL, or the device buffer of bc_attn_timeline
+  uint32_t spin_limit = 0;   // 0: the default poll limit of the bounded waits
+  int32_t debug = 0;         // BC_FLAG_DEBUG_BOUNDS
   int32_t meta_settled = 0;  // 1: the kernel that last wrote this cache's metadata has ended by the time this launch may begin
   // the paired form (NULL otherwise): the beacons' queries, their outputs and their partial buffers
   const void* q2 = nullptr;

@@ -90,6 +90,7 @@ struct MaskArgs {
   int32_t* status;     // device int: first error code
   int32_t Hq, Hkv, G, c, rows_per_tile;  // rows_per_tile = tokens per query tile = 128 / G
   float scale_log2;
+  uint32_t wait_limit;   // polls after which a wait gives up (kWaitLimit unless bc_mask_attn_set_wait_limit lowered it)
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -216,8 +217,20 @@ __device__ __forceinline__ void mbar_arrive_cta(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Bounded wait that also gives up as soon as another thread of the block has reported a failure.
-__device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity, volatile int* fail) {
-  for (uint32_t polls = 0; polls < kWaitLimit; ++polls) {
+__device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity, volatile int* fail, uint32_t limit) {
+  if (limit < 1024) {   // a deliberately short limit (bc_mask_attn_set_wait_limit): non-blocking looks, then give up
+    for (uint32_t polls = 0; polls < limit; ++polls) {
+      uint32_t ok;
+      asm volatile(
+          "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(ok)
+          : "r"(bar), "r"(parity)
+          : "memory");
+      if (ok) return true;
+    }
+    return false;
+  }
+  for (uint32_t polls = 0; polls < limit; ++polls) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -253,18 +266,18 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sQ = smem_addr(smem), sK = sQ + kOperandBytes, sV = sK + kOperandBytes;
-  __shared__ __align__(8) uint64_t s_bars[7];
+  __shared__ __align__(8) uint64_t s_bars[8];
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail_word;
   volatile int* s_fail = &s_fail_word;
   const uint32_t bar_k = smem_addr(&s_bars[0]), bar_v = bar_k + 8, bar_s = bar_k + 16, bar_p = bar_k + 24, bar_o = bar_k + 32,
-                 bar_f = bar_k + 40, bar_e = bar_k + 48;
+                 bar_f = bar_k + 40, bar_e = bar_k + 48, bar_d = bar_k + 56;   // bar_d: drain of the products on the give-up path
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = a.G, Hq = a.Hq, Hkv = a.Hkv, c = a.c;
 
   if (tid == 0) {
-    const uint32_t counts[7] = {1, 1, 1, (uint32_t)kRowThreads, 1, 1, (uint32_t)kRowThreads};
-    for (int i = 0; i < 7; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_k + i * 8), "r"(counts[i]) : "memory");
+    const uint32_t counts[8] = {1, 1, 1, (uint32_t)kRowThreads, 1, 1, (uint32_t)kRowThreads, 1};
+    for (int i = 0; i < 8; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_k + i * 8), "r"(counts[i]) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     *s_fail = 0;
   }
@@ -334,7 +347,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
       // one lane polls, the warp takes its answer
       auto wait_all = [&](uint32_t bar, uint32_t parity) {
         int ok1 = 1;
-        if (lane == 0) ok1 = mbar_wait_or_fail(bar, parity, s_fail) ? 1 : 0;
+        if (lane == 0) ok1 = mbar_wait_or_fail(bar, parity, s_fail, a.wait_limit) ? 1 : 0;
         return __shfl_sync(0xffffffffu, ok1, 0) != 0;
       };
       const uint32_t q_bytes = (uint32_t)(box_rows * kD * 2);
@@ -348,10 +361,14 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
         issue_v(td, pl, kvh, 0);
       }
       __syncwarp();
+      // copies requested / copies seen to land (for the give-up path: what is still in flight)
+      uint32_t k_req = 1, k_got = 0, v_req = 1, v_got = 0;
+      bool products_issued = false;
       uint32_t ph_k = 0, ph_v = 0, ph_o = 0, t = 0, e = 0;
       bool ok = wait_all(bar_k, ph_k);
-      ph_k ^= 1;
+      if (ok) { ph_k ^= 1; ++k_got; }
       if (ok) {
+        products_issued = true;
         tc_fence_after();
         if (elect_one()) { qk(); umma_commit(bar_s); }
         __syncwarp();
@@ -377,12 +394,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
               issue_k(ntd, npl, nkvh, 0);
             }
           }
+          if (more) ++k_req;
           __syncwarp();
           // everything the products below need besides P is waited for while the rows are busy
           ok = wait_all(bar_v, ph_v);
-          ph_v ^= 1;
+          if (ok) { ph_v ^= 1; ++v_got; }
           if (ok && n == 0 && e > 0) ok = wait_all(bar_e, (e - 1) & 1u);       // the rows have read the last O
-          if (ok && more) { ok = wait_all(bar_k, ph_k); ph_k ^= 1; }           // the next K (and Q) has landed
+          if (ok && more) { ok = wait_all(bar_k, ph_k); if (ok) { ph_k ^= 1; ++k_got; } }   // the next K (and Q) has landed
           ok = ok && wait_all(bar_p, t & 1u);
           if (!ok) break;
           tc_fence_after();
@@ -405,13 +423,29 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
             ph_o ^= 1;
             if (!ok) break;
             if (elect_one()) { if (!last) issue_v(td, pl, kvh, n + 1); else issue_v(ntd, npl, nkvh, 0); }
+            ++v_req;
             __syncwarp();
           }
         }
         if (nitem < 0) break;
         td = ntd; pl = npl; kvh = nkvh;
       }
-      if (!ok) *s_fail = 1;
+      if (!ok) {
+        // Giving up: nothing may still be on its way into this block's shared or tensor memory when the block
+        // leaves.  Wait, with the full limit, for the tensor copies that were requested and not yet seen to
+        // land, and for every product issued so far (one more commit arrives when all of them are done).
+        *s_fail = 1;
+        __syncwarp();
+        if (elect_one()) {   // the lane that issued the copies and the products
+          int never = 0;
+          if (k_req > k_got) mbar_wait_or_fail(bar_k, ph_k, &never, kWaitLimit);
+          if (v_req > v_got) mbar_wait_or_fail(bar_v, ph_v, &never, kWaitLimit);
+          if (products_issued) {
+            umma_commit(bar_d);
+            mbar_wait_or_fail(bar_d, 0, &never, kWaitLimit);
+          }
+        }
+      }
     }
     __syncwarp();
   } else {
@@ -443,7 +477,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
       float m_ref = -INFINITY, l_run = 0.f;
 
       for (int n = 0; n < pl.N; ++n, ++t) {
-        const bool ok = mbar_wait_or_fail(bar_s, t & 1u, s_fail);
+        const bool ok = mbar_wait_or_fail(bar_s, t & 1u, s_fail, a.wait_limit);
         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
         tc_fence_after();
         const int kind = plan_kind(pl, n), k0 = plan_k0(pl, n, kind);
@@ -517,7 +551,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
           const int seg_len = kind == 0 ? td.P : (kind == 1 ? td.nb : td.T);
           const int nvalid = min(max(seg_len - k0, 0), kTile);
           if (nvalid < kTile) {   // the same for the whole block
-            const bool okv = mbar_wait_or_fail(bar_v, t & 1u, s_fail);
+            const bool okv = mbar_wait_or_fail(bar_v, t & 1u, s_fail, a.wait_limit);
             if (!__all_sync(0xffffffffu, okv)) { failed = true; break; }
             if (tid >= nvalid) {
 #pragma unroll
@@ -536,7 +570,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
       const int nitem = item_of(r + 1);
       TileDesc ntd = {};
       if (nitem >= 0) ntd = a.tiles[nitem / Hkv];   // in flight during the wait below
-      const bool ok = mbar_wait_or_fail(bar_f, e & 1u, s_fail);
+      const bool ok = mbar_wait_or_fail(bar_f, e & 1u, s_fail, a.wait_limit);
       if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       tc_fence_after();
       float o[kD];
@@ -617,6 +651,8 @@ MaskLayout mask_layout(int n_seqs, int q_heads, int kv_heads, int64_t total_toke
   l.total = o;
   return l;
 }
+
+uint32_t g_mask_wait_limit = 0;   // bc_mask_attn_set_wait_limit (0: kWaitLimit)
 
 int sm_count() {
   static int n = 0;
@@ -703,6 +739,7 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
   a.status = reinterpret_cast<int32_t*>(ws + l.status);
   a.Hq = q_heads; a.Hkv = kv_heads; a.G = G; a.c = c; a.rows_per_tile = per;
   a.scale_log2 = sm_scale * 1.4426950408889634f;
+  a.wait_limit = g_mask_wait_limit ? g_mask_wait_limit : kWaitLimit;
   const int smem_bytes = 3 * kOperandBytes + 1024;
   if (cudaFuncSetAttribute(k_mask_attn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return BC_ERR_CUDA;
   if (!encode_tiled()) return BC_ERR_CUDA;
@@ -720,6 +757,11 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
   const int grid = a.n_items < 2 * sm_count() ? a.n_items : 2 * sm_count();   // two resident blocks per SM
   k_mask_attn<<<grid, kThreads, smem_bytes, s>>>(a, maps);
   return cudaGetLastError() == cudaSuccess ? BC_OK : BC_ERR_CUDA;
+}
+
+bc_status bc_mask_attn_set_wait_limit(uint32_t polls) {
+  g_mask_wait_limit = polls;
+  return BC_OK;
 }
 
 bc_status bc_mask_attn_status(const void* workspace, int32_t n_seqs, int32_t q_heads, int32_t kv_heads,

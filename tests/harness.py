@@ -41,7 +41,8 @@ class Pair:
         self.L, self.Hkv, self.Hq, self.D = layers, kv_heads, q_heads, head_dim
         self.gpu = B.Cache(layers, kv_heads, q_heads, head_dim, c_default, page_size, max_seqs, num_pages,
                            max_pages_per_seq, max_entries, flags, device=device)
-        self.model = PagingModel(num_pages, page_size, max_seqs, max_pages_per_seq, max_entries, c_default)
+        self.model = PagingModel(num_pages, page_size, max_seqs, max_pages_per_seq, max_entries, c_default,
+                                 debug_bounds=bool(flags & B.BC_FLAG_DEBUG_BOUNDS))
         self.seqs = {}
         self.max_seqs = max_seqs
         self._append_ok = None

@@ -15,20 +15,28 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-@pytest.mark.parametrize("seed,ps,num_pages,max_pps,max_entries", [
-    (0, 1, 40, 12, 0), (1, 2, 24, 8, 0), (2, 3, 30, 9, 7), (3, 4, 64, 16, 0), (4, 16, 12, 4, 0), (5, 5, 50, 6, 11),
+@pytest.mark.parametrize("seed,ps,num_pages,max_pps,max_entries,checked", [
+    (0, 1, 40, 12, 0, False), (1, 2, 24, 8, 0, False), (2, 3, 30, 9, 7, False), (3, 4, 64, 16, 0, False),
+    (4, 16, 12, 4, 0, False), (5, 5, 50, 6, 11, False),
+    # checked mode (BC_FLAG_DEBUG_BOUNDS): the same programs, every index checked on the device, and
+    # batches that name a slot more than once (the later items are refused)
+    (6, 2, 24, 8, 0, True), (7, 3, 30, 9, 7, True), (8, 16, 12, 4, 0, True), (9, 1, 40, 12, 0, True),
 ])
-def test_random_programs(seed, ps, num_pages, max_pps, max_entries):
+def test_random_programs(seed, ps, num_pages, max_pps, max_entries, checked):
     rng = np.random.RandomState(seed)
     S, Hkv, G, D = 8, 1, 2, 64
     pair = Pair(1, Hkv, Hkv * G, D, ps, max_seqs=S, num_pages=num_pages, max_pages_per_seq=max_pps,
-                max_entries=max_entries, c_default=int(rng.choice([1, 2, 3, 5])))
+                max_entries=max_entries, c_default=int(rng.choice([1, 2, 3, 5])),
+                flags=B.BC_FLAG_DEBUG_BOUNDS if checked else 0)
     g = torch.Generator(device=DEV); g.manual_seed(seed)
     kv = lambda n: (randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV))
     for step in range(160):
         op = rng.choice(["open", "restore", "append", "append", "append", "compress", "close"])
         n = int(rng.randint(1, S + 1))
         slots = [int(x) for x in rng.choice(S + 2, size=n, replace=False) - 1]      # -1 and S are invalid slots
+        if checked and rng.rand() < 0.3:                                             # name some slots again
+            slots = [int(x) for x in rng.choice(slots, size=min(S, n + int(rng.randint(1, 4))))]
+            n = len(slots)
         if op == "open":
             plens = [int(rng.randint(0, 3 * ps + 2)) for _ in slots]
             cs = None if rng.rand() < 0.3 else [int(rng.choice([1, 2, 3, 4, 7])) for _ in slots]
@@ -38,6 +46,7 @@ def test_random_programs(seed, ps, num_pages, max_pps, max_entries):
             fresh = [s for s in range(S) if (st := pair.model.state(s)) and st["t"] == 0]
             if fresh and rng.rand() < 0.7:
                 slots = fresh[:n]
+                n = len(slots)
             gen_lens = [int(rng.randint(0, 4 * ps + 6)) for _ in slots]
             nb = sum(T // st["c"] for s, T in zip(slots, gen_lens) if (st := pair.model.state(s)) and st["c"] > 1)
             tk, tv = kv(max(sum(gen_lens), 1))

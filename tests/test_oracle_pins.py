@@ -438,3 +438,25 @@ def test_replay_is_algorithm1_stepwise():
         w = T - nb * c
         assert np.array_equal(K[3:3 + nb], bk) and np.array_equal(K[3 + nb:], tk[T - w:])
 
+
+
+def test_checked_mode_refuses_the_later_items_of_a_repeated_slot():
+    """Checked mode (the library's BC_FLAG_DEBUG_BOUNDS), worked by hand: of the items of one call
+    that name the same slot the first goes through and the others get DEBUG_CHECK; an invalid
+    slot stays BAD_SLOT however often it is named; pages are allocated for the first item only."""
+    m = PagingModel(num_pages=16, page_size=2, max_seqs=4, max_pages_per_seq=8, debug_bounds=True)
+    assert m.open([1, 1, 2, 7, 7], [3, 5, 1, 1, 1], [2, 2, 2, 2, 2]) == [OK, "DEBUG_CHECK", OK, BAD_SLOT, BAD_SLOT]
+    assert m.state(1)["prompt_pages"] == [0, 1] and m.state(2)["prompt_pages"] == [2]     # P = 3, not 5
+    assert m.first_error == ("DEBUG_CHECK", 1, 1)
+    m.first_error = None
+    assert m.append([2, 1, 2, 2]) == [OK, OK, "DEBUG_CHECK", "DEBUG_CHECK"]
+    assert m.state(2)["window_len"] == 1 and m.state(2)["t"] == 1                        # appended once
+    assert m.first_error == ("DEBUG_CHECK", 2, 2)
+    assert m.append([1, 2]) == [OK, OK]
+    m.first_error = None
+    assert m.compress([1, 1]) == [OK, "DEBUG_CHECK"]
+    assert m.state(1)["n_beacons"] == 1 and m.state(1)["window_len"] == 0
+    assert m.close([2, 2, 3]) == [OK, "DEBUG_CHECK", BAD_SLOT]
+    assert m.first_error == ("DEBUG_CHECK", 1, 4)
+    # without the flag the model does not look for repeats (such a batch is outside the contract)
+    assert PagingModel(4, 2, 4, 4).open([0, 1], [1, 1]) == [OK, OK]

@@ -33,7 +33,7 @@ MetaLayout meta_layout(const bc_config& c) {
 }
 
 struct WorkLayout {
-  size_t append_row[2], append_pos[2], compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[2],
+  size_t append_row[2], append_pos[2], compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[4],
       stage_out[2], stage_out2[2],
       total;
 };
@@ -54,11 +54,13 @@ WorkLayout work_layout(const bc_config& c) {
   l.part_o = take(pieces * c.q_heads * c.head_dim * 4);
   l.part_ml2 = take(pieces * c.q_heads * 2 * 4);            // the beacons' partials of the paired form
   l.part_o2 = take(pieces * c.q_heads * c.head_dim * 4);
-  // host-buffer entry points: two input staging buffers, each k | v | q packed for the call's batch
-  for (int b = 0; b < 2; ++b) l.stage_in[b] = take((size_t)BC_MAX_ATTN_BATCH * (c.q_heads + 2 * c.kv_heads) * c.head_dim * 2);
+  // host-buffer entry points: a ring of four input staging buffers, each k | v | q packed for the largest
+  // batch a call can carry (a step that fills a window takes two of them, token and beacon inputs)
+  const size_t max_n = c.max_seqs < BC_MAX_ATTN_BATCH ? c.max_seqs : BC_MAX_ATTN_BATCH;
+  for (int b = 0; b < 4; ++b) l.stage_in[b] = take(max_n * (c.q_heads + 2 * c.kv_heads) * c.head_dim * 2);
   for (int b = 0; b < 2; ++b) {   // two sets of output staging (a set: token output, beacon output)
-    l.stage_out[b] = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
-    l.stage_out2[b] = take((size_t)BC_MAX_ATTN_BATCH * c.q_heads * c.head_dim * 4);
+    l.stage_out[b] = take(max_n * c.q_heads * c.head_dim * 4);
+    l.stage_out2[b] = take(max_n * c.q_heads * c.head_dim * 4);
   }
   l.total = o;
   return l;
@@ -116,16 +118,31 @@ struct bc_cache {
   // profiling
   std::vector<cudaEvent_t> ev;
   int prof_cap, prof_used;
-  // host-buffer entry points: inputs are copied on a stream of their own into alternating staging buffers
+  // host-buffer entry points: inputs are copied on a stream of their own into a ring of staging buffers
+  static constexpr int kStageRing = 4;
   cudaStream_t copy_stream = nullptr;
-  cudaEvent_t ev_in[2] = {nullptr, nullptr};    // the copies into staging buffer b have been issued up to here
-  cudaEvent_t ev_used[2] = {nullptr, nullptr};  // the kernels reading staging buffer b have been issued up to here
+  cudaEvent_t ev_in[kStageRing] = {};      // the copies into staging buffer b have been issued up to here
+  cudaEvent_t buf_done[kStageRing] = {};   // not owned: the event after which buffer b's last readers have finished
   int stage_next = 0;
+  // one event per host-buffer step, recorded on the caller's stream behind the step's kernels
+  static constexpr int kDoneRing = 8;
+  cudaEvent_t ev_done[kDoneRing] = {};
+  int done_next = 0;
   // BC_FLAG_HOST_PIPELINED: outputs leave on a stream of their own from alternating staging sets
   cudaStream_t out_stream = nullptr;
-  cudaEvent_t ev_kern[2] = {nullptr, nullptr};   // the kernels writing output set b have been issued up to here
   cudaEvent_t ev_d2h[2] = {nullptr, nullptr};    // the copies out of set b have been issued up to here
   int out_next = 0;
+  // BC_FLAG_HOST_PIPELINED: what the last host-buffer step still owes -- its completion event and the
+  // copies of its outputs.  They are issued by the next host-buffer call right behind that call's
+  // bookkeeping kernel (which may then start under this step's attention kernel), or by
+  // bc_host_outputs_ready / bc_cache_destroy.
+  struct Pending {
+    bool valid = false;
+    int set = 0, bufs[2] = {-1, -1};
+    void* out_host = nullptr; void* out2_host = nullptr;
+    size_t bytes = 0;
+    cudaStream_t stream = nullptr;
+  } pending;
 };
 
 namespace {
@@ -196,6 +213,37 @@ bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const v
 
 }  // namespace
 
+namespace {
+// Layer-0 bookkeeping of a step's append, launched on its own (no K/V rows in the same launch).
+bc_status append_book_only(bc_cache* c, const int32_t* slots, int n, cudaStream_t s) {
+  c->append_set ^= 1;
+  BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, ++c->calls, work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
+                                   work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), c->geom, layer_base(c, 0), nullptr,
+                                   nullptr, s));
+  c->launches += 1;
+  c->meta_unsettled = true;
+  return BC_OK;
+}
+
+// The attention half of bc_decode_step: the step's append bookkeeping (layer 0) has been launched.
+bc_status decode_step_attn(bc_cache* c, int layer, const int32_t* slots, int n, const void* q, const void* k, const void* v,
+                           void* out, float sm_scale, cudaStream_t s) {
+  BcFusedAppend f;
+  f.new_k = k; f.new_v = v;
+  f.dst_row = work_ptr<int32_t>(c, c->wl.append_row[c->append_set]);
+  f.dst_pos = work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]);
+  f.pool_layer = layer_base(c, layer);
+  f.flag = work_ptr<int32_t>(c, c->wl.book_flag);
+  f.do_book = 0;
+  f.call = c->calls;
+  f.epoch = (int32_t)(c->calls & 0x7fffffff) | 1 << 30;   // never 0, the word's initial value
+  const bc_status st = attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s, &f);
+  if (st) return st;
+  c->append_next_layer = (layer + 1) % c->cfg.layers;
+  return BC_OK;
+}
+}  // namespace
+
 // ---- bc_decode_attn_static: split-K scratch inside the library image -------------------------------
 //
 // Layout of the built-in array: partial outputs [pieces][4096] fp32, then (max, sum) pairs
@@ -254,6 +302,10 @@ cudaError_t static_scratch_reset_tickets(cudaStream_t s) {
 
 
 extern "C" {
+
+namespace {
+bc_status flush_pending(bc_cache* c);   // defined with the host-buffer entry points below
+}
 
 int32_t bc_version(void) { return 200; }
 
@@ -329,15 +381,13 @@ bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* wo
 bc_status bc_cache_destroy(bc_cache* c) {
   if (!c) return BC_ERR_INVALID_ARG;
   // the cache's own streams touch the caller's workspace: let them drain before the caller may free it
+  if (c->pending.valid) flush_pending(c);
   if (c->copy_stream) cudaStreamSynchronize(c->copy_stream);
   if (c->out_stream) cudaStreamSynchronize(c->out_stream);
   for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
-  for (int b = 0; b < 2; ++b) {
-    if (c->ev_in[b]) cudaEventDestroy(c->ev_in[b]);
-    if (c->ev_used[b]) cudaEventDestroy(c->ev_used[b]);
-    if (c->ev_kern[b]) cudaEventDestroy(c->ev_kern[b]);
-    if (c->ev_d2h[b]) cudaEventDestroy(c->ev_d2h[b]);
-  }
+  for (cudaEvent_t e : c->ev_in) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->ev_done) if (e) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->ev_d2h) if (e) cudaEventDestroy(e);
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   if (c->out_stream) cudaStreamDestroy(c->out_stream);
   delete c;
@@ -497,26 +547,10 @@ bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32
   // row-writing launch.  (The kernel can also run the bookkeeping in its block 0, do_book = 1: that
   // form starts every other block late and is not used here.)
   if (layer == 0) {
-    c->append_set ^= 1;
-    BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, ++c->calls, work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
-                                     work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), c->geom, layer_base(c, 0), nullptr,
-                                     nullptr, s));
-    c->launches += 1;
-    c->meta_unsettled = true;
+    st = append_book_only(c, slots, n, s);
+    if (st) return st;
   }
-  BcFusedAppend f;
-  f.new_k = k; f.new_v = v;
-  f.dst_row = work_ptr<int32_t>(c, c->wl.append_row[c->append_set]);
-  f.dst_pos = work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]);
-  f.pool_layer = layer_base(c, layer);
-  f.flag = work_ptr<int32_t>(c, c->wl.book_flag);
-  f.do_book = 0;
-  f.call = c->calls;
-  f.epoch = (int32_t)(c->calls & 0x7fffffff) | 1 << 30;   // never 0, the word's initial value
-  st = attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s, &f);
-  if (st) return st;
-  c->append_next_layer = (layer + 1) % c->cfg.layers;
-  return BC_OK;
+  return decode_step_attn(c, layer, slots, n, q, k, v, out, sm_scale, s);
 }
 
 bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* bk, const void* bv,
@@ -572,25 +606,30 @@ bc_status bc_seq_close(bc_cache* c, const int32_t* slots, int32_t n, void* strea
 
 namespace {
 
+bc_status host_setup(bc_cache* c) {   // first host-buffer call on this cache
+  if (c->copy_stream) return BC_OK;
+  BC_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+  for (cudaEvent_t& e : c->ev_in) BC_CUDA(c, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  for (cudaEvent_t& e : c->ev_done) BC_CUDA(c, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) {
+    BC_CUDA(c, cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking));
+    for (cudaEvent_t& e : c->ev_d2h) BC_CUDA(c, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  }
+  return BC_OK;
+}
+
 // Stages k, v, q of a host-buffer step: the copies run on the cache's own copy stream, so the next
-// step's inputs travel while this step's kernels run; `s` waits for them before the kernels.
-// Returns the staging buffer used; record ev_used[buf] on `s` after the kernels that read it.
+// steps' inputs travel while this step's kernels run; `s` waits for them before the kernels that read
+// them.  Returns the staging buffer used.
 bc_status stage_inputs(bc_cache* c, int32_t n, const void* q_host, const void* k_host, const void* v_host, cudaStream_t s,
                        int* buf_out, void** dq, void** dk, void** dv) {
-  if (!c->copy_stream) {   // first host-buffer call on this cache
-    BC_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
-    for (int b = 0; b < 2; ++b) {
-      BC_CUDA(c, cudaEventCreateWithFlags(&c->ev_in[b], cudaEventDisableTiming));
-      BC_CUDA(c, cudaEventCreateWithFlags(&c->ev_used[b], cudaEventDisableTiming));
-    }
-  }
   const int buf = c->stage_next;
-  c->stage_next ^= 1;
+  c->stage_next = (buf + 1) % bc_cache::kStageRing;
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
   uint8_t* base = c->work + c->wl.stage_in[buf];
   *dk = base; *dv = base + kb; *dq = base + 2 * kb;
-  // the buffer's previous readers (two steps ago) must be done; an event never recorded does not block
-  BC_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_used[buf], 0));
+  // the buffer's previous readers (a whole turn of the ring ago) must be done
+  if (c->buf_done[buf]) BC_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->buf_done[buf], 0));
   const uint8_t *kh = static_cast<const uint8_t*>(k_host), *vh = static_cast<const uint8_t*>(v_host),
                 *qh = static_cast<const uint8_t*>(q_host);
   if (vh == kh + kb && qh == vh + kb) {   // one packed host buffer k | v | q: one copy
@@ -613,13 +652,6 @@ bc_status stage_inputs(bc_cache* c, int32_t n, const void* q_host, const void* k
 bc_status begin_outputs(bc_cache* c, cudaStream_t s, int* set, void** dout, void** dout2) {
   *set = 0;
   if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) {
-    if (!c->out_stream) {
-      BC_CUDA(c, cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking));
-      for (int b = 0; b < 2; ++b) {
-        BC_CUDA(c, cudaEventCreateWithFlags(&c->ev_kern[b], cudaEventDisableTiming));
-        BC_CUDA(c, cudaEventCreateWithFlags(&c->ev_d2h[b], cudaEventDisableTiming));
-      }
-    }
     *set = c->out_next;
     c->out_next ^= 1;
     BC_CUDA(c, cudaStreamWaitEvent(s, c->ev_d2h[*set], 0));   // the set's copies of two steps ago (long done)
@@ -628,24 +660,48 @@ bc_status begin_outputs(bc_cache* c, cudaStream_t s, int* set, void** dout, void
   *dout2 = c->work + c->wl.stage_out2[*set];
   return BC_OK;
 }
-bc_status send_outputs(bc_cache* c, cudaStream_t s, int set, void* out_host, const void* dout, void* out2_host,
-                       const void* dout2, size_t bytes) {
-  cudaStream_t cs = s;
+
+// What follows a host-buffer step's kernels: ONE event on the caller's stream (the input staging
+// buffers the step read are free after it, and the output copies may start after it), then the copies
+// of the outputs -- on `s` itself in plain mode, on the cache's output stream in pipelined mode.
+bc_status finish_step(bc_cache* c, const bc_cache::Pending& p) {
+  cudaEvent_t done = c->ev_done[c->done_next];
+  c->done_next = (c->done_next + 1) % bc_cache::kDoneRing;
+  BC_CUDA(c, cudaEventRecord(done, p.stream));
+  for (int b : p.bufs) if (b >= 0) c->buf_done[b] = done;
+  cudaStream_t cs = p.stream;
   if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) {
-    BC_CUDA(c, cudaEventRecord(c->ev_kern[set], s));
-    BC_CUDA(c, cudaStreamWaitEvent(c->out_stream, c->ev_kern[set], 0));
+    BC_CUDA(c, cudaStreamWaitEvent(c->out_stream, done, 0));
     cs = c->out_stream;
   }
-  BC_CUDA(c, cudaMemcpyAsync(out_host, dout, bytes, cudaMemcpyDeviceToHost, cs));
-  if (out2_host) BC_CUDA(c, cudaMemcpyAsync(out2_host, dout2, bytes, cudaMemcpyDeviceToHost, cs));
-  if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) BC_CUDA(c, cudaEventRecord(c->ev_d2h[set], cs));
+  BC_CUDA(c, cudaMemcpyAsync(p.out_host, c->work + c->wl.stage_out[p.set], p.bytes, cudaMemcpyDeviceToHost, cs));
+  if (p.out2_host) BC_CUDA(c, cudaMemcpyAsync(p.out2_host, c->work + c->wl.stage_out2[p.set], p.bytes, cudaMemcpyDeviceToHost, cs));
+  if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) BC_CUDA(c, cudaEventRecord(c->ev_d2h[p.set], cs));
   return BC_OK;
+}
+
+bc_status flush_pending(bc_cache* c) {
+  if (!c->pending.valid) return BC_OK;
+  c->pending.valid = false;
+  return finish_step(c, c->pending);
+}
+
+// The end of a host-buffer call: in plain mode the step's event and output copies are issued at once;
+// in pipelined mode they are left to the next host-buffer call (see bc_cache::Pending).
+bc_status close_step(bc_cache* c, cudaStream_t s, int set, int buf, int buf2, void* out_host, void* out2_host, size_t bytes) {
+  bc_cache::Pending p;
+  p.valid = true; p.set = set; p.bufs[0] = buf; p.bufs[1] = buf2; p.out_host = out_host; p.out2_host = out2_host;
+  p.bytes = bytes; p.stream = s;
+  if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) { c->pending = p; return BC_OK; }
+  return finish_step(c, p);
 }
 
 }  // namespace
 
 bc_status bc_host_outputs_ready(bc_cache* c, void* stream) {
   if (!c) return BC_ERR_INVALID_ARG;
+  bc_status st = flush_pending(c);
+  if (st) return st;
   if (c->out_stream)
     for (int b = 0; b < 2; ++b) BC_CUDA(c, cudaStreamWaitEvent((cudaStream_t)stream, c->ev_d2h[b], 0));
   return BC_OK;
@@ -656,19 +712,35 @@ bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, 
   bc_status st = check_batch(c, layer, slots, n);
   if (st) return st;
   if (n > BC_MAX_ATTN_BATCH || !q_host || !k_host || !v_host || !out_host) return BC_ERR_INVALID_ARG;
+  if (layer != c->append_next_layer) return BC_ERR_ORDER;
   cudaStream_t s = (cudaStream_t)stream;
+  st = host_setup(c);
+  if (st) return st;
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
+  const bool reference = (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) != 0;
+  // The step's bookkeeping needs nothing from the host, so it goes out first, directly behind the last
+  // step's attention kernel (under whose last blocks it may start); only then the events and copies
+  // that the last step still owes, and this step's own copies.
+  if (layer == 0 && !reference) {
+    st = append_book_only(c, slots, n, s);
+    if (st) return st;
+  }
+  st = flush_pending(c);
+  if (st) return st;
   void *dq, *dk, *dv, *dout, *dout2;
   int buf, set;
   st = stage_inputs(c, n, q_host, k_host, v_host, s, &buf, &dq, &dk, &dv);
   if (st) return st;
   st = begin_outputs(c, s, &set, &dout, &dout2);
   if (st) return st;
-  st = bc_decode_step(c, layer, slots, n, dq, dk, dv, dout, sm_scale, stream);   // two launches instead of three
+  if (reference) {
+    st = bc_decode_step(c, layer, slots, n, dq, dk, dv, dout, sm_scale, stream);
+  } else {
+    st = decode_step_attn(c, layer, slots, n, dq, dk, dv, dout, sm_scale, s);
+  }
   if (st) return st;
-  BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
-  return send_outputs(c, s, set, out_host, dout, nullptr, nullptr, ob);
+  return close_step(c, s, set, buf, -1, out_host, nullptr, ob);
 }
 
 bc_status bc_fill_step_host(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q_host,
@@ -678,9 +750,22 @@ bc_status bc_fill_step_host(bc_cache* c, int32_t layer, const int32_t* slots, in
   if (st) return st;
   if (n > BC_MAX_ATTN_BATCH || !q_host || !k_host || !v_host || !bq_host || !bk_host || !bv_host || !out_host || !out_beacon_host)
     return BC_ERR_INVALID_ARG;
+  if (layer != c->append_next_layer || layer != c->compress_next_layer) return BC_ERR_ORDER;
   cudaStream_t s = (cudaStream_t)stream;
+  st = host_setup(c);
+  if (st) return st;
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
+  // as in bc_decode_step_host: the append's bookkeeping first (when its rows go out in a launch of their own)
+  const bool rows_apart = (size_t)n * c->geom.entry_bytes > kFusedRowBytes;
+  bool book_done = false;
+  if (layer == 0 && rows_apart) {
+    st = append_book_only(c, slots, n, s);
+    if (st) return st;
+    book_done = true;
+  }
+  st = flush_pending(c);
+  if (st) return st;
   void *dq, *dk, *dv, *dbq, *dbk, *dbv, *dout, *dout2;
   int buf, buf2, set;
   st = stage_inputs(c, n, q_host, k_host, v_host, s, &buf, &dq, &dk, &dv);
@@ -689,15 +774,21 @@ bc_status bc_fill_step_host(bc_cache* c, int32_t layer, const int32_t* slots, in
   if (st) return st;
   st = begin_outputs(c, s, &set, &dout, &dout2);
   if (st) return st;
-  st = bc_append(c, layer, slots, n, dk, dv, stream);
-  if (st) return st;
+  if (book_done || (layer > 0 && rows_apart)) {   // the rows of this layer (the bookkeeping is done, or was done on layer 0)
+    BC_CUDA(c, bc_launch_write_rows(c->meta, c->geom, layer_base(c, layer), work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
+                                    work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), dk, dv, n, s));
+    c->launches += 1;
+    c->meta_unsettled = false;
+    c->append_next_layer = (layer + 1) % c->cfg.layers;
+  } else {
+    st = bc_append(c, layer, slots, n, dk, dv, stream);
+    if (st) return st;
+  }
   st = bc_decode_attn_pair(c, layer, slots, n, dq, dout, dbq, dout2, sm_scale, dbk, dbv, stream);
   if (st) return st;
   st = bc_compress(c, layer, slots, n, dbk, dbv, stream);
   if (st) return st;
-  BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
-  BC_CUDA(c, cudaEventRecord(c->ev_used[buf2], s));
-  return send_outputs(c, s, set, out_host, dout, out_beacon_host, dout2, ob);
+  return close_step(c, s, set, buf, buf2, out_host, out_beacon_host, ob);
 }
 
 bc_status bc_compress_step_host(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* bq_host,
@@ -706,6 +797,10 @@ bc_status bc_compress_step_host(bc_cache* c, int32_t layer, const int32_t* slots
   if (st) return st;
   if (n > BC_MAX_ATTN_BATCH || !bq_host || !bk_host || !bv_host || !out_host) return BC_ERR_INVALID_ARG;
   cudaStream_t s = (cudaStream_t)stream;
+  st = host_setup(c);
+  if (st) return st;
+  st = flush_pending(c);
+  if (st) return st;
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
   void *dq, *dk, *dv, *dout, *dout2;
@@ -718,8 +813,7 @@ bc_status bc_compress_step_host(bc_cache* c, int32_t layer, const int32_t* slots
   if (st) return st;
   st = bc_compress(c, layer, slots, n, dk, dv, stream);
   if (st) return st;
-  BC_CUDA(c, cudaEventRecord(c->ev_used[buf], s));
-  return send_outputs(c, s, set, out_host, dout, nullptr, nullptr, ob);
+  return close_step(c, s, set, buf, -1, out_host, nullptr, ob);
 }
 
 bc_status bc_get_state(bc_cache* c, int32_t slot, bc_seq_state* out, int32_t* pages, int32_t pages_cap, void* stream) {

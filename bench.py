@@ -414,6 +414,9 @@ def run_timeline(args):
                                   ("published_only", ((path & 4) > 0) & ((path & 24) == 0)),
                                   ("published_then_merged", ((path & 4) > 0) & ((path & 16) > 0)),
                                   ("merged_first_piece_too", (path & 8) > 0))}
+            if args.timeline_raw:     # per block: [tiles, first sequence, ending bits, then the eight stamps in us]
+                row["blocks_raw"] = [[int(a[b, 8] >> 32), int(a[b, 8] & 0xffffffff), int(a[b, 9])] +
+                                     [round(float((a[b, k] - t0) / 1e3), 2) for k in range(8)] for b in range(BLOCKS) if live[b]]
             if prev_end is not None:
                 row["enter_after_previous_launch_left_us"] = round(float((t0 - prev_end) / 1e3), 2)
             prev_end = a[live, 7].max()
@@ -990,7 +993,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-pair", action="store_true", help="beacon steps as a second attention pass instead of bc_decode_attn_pair")
     ap.add_argument("--pair", action="store_true", help="ragged workload: pair the beacon steps too (off by default there)")
-    ap.add_argument("--fused", action="store_true", help="depth workload: regular steps through bc_decode_step (append + attention in one launch per layer)")
+    ap.add_argument("--fused", action="store_true", help="depth workload and --timeline: regular steps through bc_decode_step (append + attention in one launch per layer)")
+    ap.add_argument("--no-fused", action="store_true", help="sweep: regular steps as bc_append + bc_decode_attn instead of bc_decode_step")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
     ap.add_argument("--model-ratio", type=int, default=None, help=argparse.SUPPRESS)   # model workload: one ratio (child process)
@@ -1001,6 +1005,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the short mask-form and distillation runs of the default line")
     ap.add_argument("--timeline", type=int, default=0, metavar="C",
                     help="per-block time stamps of the attention kernel (bc_attn_timeline) on the small case of ratio C")
+    ap.add_argument("--timeline-raw", action="store_true", help="with --timeline: also print every block's stamps")
     ap.add_argument("--profile-case", type=int, default=0, metavar="C",
                     help="small case for profilers: ratio C with a prompt as long as the mid-generation cache, "
                          "--steps plain decode steps, no fast-forward, no graphs")
@@ -1049,7 +1054,7 @@ def main():
     for c in sweep:
         w = make_workload("sweep", c=c)
         T = w.steps
-        r = make_runner(w, dev, seed_offset=sharding.rank_seed_offset(0, rank), paired=not args.no_pair, fused=args.fused)
+        r = make_runner(w, dev, seed_offset=sharding.rank_seed_offset(0, rank), paired=not args.no_pair, fused=not args.no_fused)
         cyc = c if c > 1 else 16
         t_mid = max(0, ((T - K) // 2 // cyc) * cyc)
         # pass A: device-resident inputs, CUDA-graph replays: the headline time
@@ -1124,6 +1129,8 @@ def main():
                    "launch": "per ratio, the K timed steps are one CUDA graph replayed once under the event pair "
                              "(captured at the timed position, warmed by one replay, caches rewound); sweep[].graph "
                              "gives the steps it holds", "per_gpu_batch": B * n_c,
+                   "regular_steps": "bc_append + bc_decode_attn" if args.no_fused else
+                                    "bc_decode_step (the append's bookkeeping kernel, then one attention kernel that takes the new entries from the inputs)",
                    "beacon_steps": "second attention pass" if args.no_pair else
                                    "paired with the token's attention (bc_decode_attn_pair: one pass over the cache)"},
         "e2e": {"value": world * B * n_c * K / (e2e_ms * 1e-3), "unit": "tokens/s",

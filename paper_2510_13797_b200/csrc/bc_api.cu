@@ -33,7 +33,7 @@ MetaLayout meta_layout(const bc_config& c) {
 }
 
 struct WorkLayout {
-  size_t append_row[2], append_pos[2], compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[4],
+  size_t append_row[2], append_pos[2], plan[2], compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[4],
       stage_out[2], stage_out2[2],
       total;
 };
@@ -45,7 +45,7 @@ WorkLayout work_layout(const bc_config& c) {
   const size_t pieces = BC_MAX_ATTN_CTAS + BC_MAX_ATTN_BATCH;
   // two sets of row destinations of bc_append, used by alternate steps: a fused attention kernel may
   // still read one while the next step's bookkeeping already fills the other
-  for (int b = 0; b < 2; ++b) { l.append_row[b] = take(seq); l.append_pos[b] = take(seq); }
+  for (int b = 0; b < 2; ++b) { l.append_row[b] = take(seq); l.append_pos[b] = take(seq); l.plan[b] = take(BC_PLAN_INTS * 4); }
   l.compress_row = take(seq); l.compress_pos = take(seq);
   l.restore_ok = take(seq); l.restore_bea = take(seq + 4);
   l.tickets = take(BC_MAX_ATTN_BATCH * 4);
@@ -214,12 +214,18 @@ bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const v
 }  // namespace
 
 namespace {
+// The word a fused step's bookkeeping kernel publishes when its results are written: derived from the
+// index of the bookkeeping call, never 0 (the word's initial value).
+inline int32_t step_epoch(int64_t calls) { return (int32_t)(calls & 0x3fffffff) | 1 << 30; }
+
 // Layer-0 bookkeeping of a step's append, launched on its own (no K/V rows in the same launch).
-bc_status append_book_only(bc_cache* c, const int32_t* slots, int n, cudaStream_t s) {
+bc_status append_book_only(bc_cache* c, const int32_t* slots, int n, cudaStream_t s, bool with_plan = false) {
   c->append_set ^= 1;
-  BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, ++c->calls, work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
+  ++c->calls;
+  BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, c->calls, work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
                                    work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), c->geom, layer_base(c, 0), nullptr,
-                                   nullptr, s));
+                                   nullptr, s, with_plan ? work_ptr<int32_t>(c, c->wl.plan[c->append_set]) : nullptr,
+                                   work_ptr<int32_t>(c, c->wl.book_flag), step_epoch(c->calls)));
   c->launches += 1;
   c->meta_unsettled = true;
   return BC_OK;
@@ -234,9 +240,10 @@ bc_status decode_step_attn(bc_cache* c, int layer, const int32_t* slots, int n, 
   f.dst_pos = work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]);
   f.pool_layer = layer_base(c, layer);
   f.flag = work_ptr<int32_t>(c, c->wl.book_flag);
+  f.plan = work_ptr<int32_t>(c, c->wl.plan[c->append_set]);   // left by append_book_only(with_plan) of this step
   f.do_book = 0;
   f.call = c->calls;
-  f.epoch = (int32_t)(c->calls & 0x7fffffff) | 1 << 30;   // never 0, the word's initial value
+  f.epoch = step_epoch(c->calls);
   const bc_status st = attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s, &f);
   if (st) return st;
   c->append_next_layer = (layer + 1) % c->cfg.layers;
@@ -547,7 +554,7 @@ bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32
   // row-writing launch.  (The kernel can also run the bookkeeping in its block 0, do_book = 1: that
   // form starts every other block late and is not used here.)
   if (layer == 0) {
-    st = append_book_only(c, slots, n, s);
+    st = append_book_only(c, slots, n, s, true);
     if (st) return st;
   }
   return decode_step_attn(c, layer, slots, n, q, k, v, out, sm_scale, s);
@@ -630,6 +637,10 @@ bc_status stage_inputs(bc_cache* c, int32_t n, const void* q_host, const void* k
   *dk = base; *dv = base + kb; *dq = base + 2 * kb;
   // the buffer's previous readers (a whole turn of the ring ago) must be done
   if (c->buf_done[buf]) BC_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->buf_done[buf], 0));
+  // Pipelined outputs: the step that receives these inputs writes the output staging set whose last
+  // copies to the host (two steps ago) must be over.  The copy stream waits for them here, so that the
+  // one event the caller's stream waits for below covers both and no second wait sits between kernels.
+  if (c->out_stream) BC_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_d2h[c->out_next], 0));
   const uint8_t *kh = static_cast<const uint8_t*>(k_host), *vh = static_cast<const uint8_t*>(v_host),
                 *qh = static_cast<const uint8_t*>(q_host);
   if (vh == kh + kb && qh == vh + kb) {   // one packed host buffer k | v | q: one copy
@@ -652,9 +663,8 @@ bc_status stage_inputs(bc_cache* c, int32_t n, const void* q_host, const void* k
 bc_status begin_outputs(bc_cache* c, cudaStream_t s, int* set, void** dout, void** dout2) {
   *set = 0;
   if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) {
-    *set = c->out_next;
+    *set = c->out_next;   // its copies of two steps ago are over: stage_inputs made the copy stream wait for them
     c->out_next ^= 1;
-    BC_CUDA(c, cudaStreamWaitEvent(s, c->ev_d2h[*set], 0));   // the set's copies of two steps ago (long done)
   }
   *dout = c->work + c->wl.stage_out[*set];
   *dout2 = c->work + c->wl.stage_out2[*set];
@@ -723,7 +733,7 @@ bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, 
   // step's attention kernel (under whose last blocks it may start); only then the events and copies
   // that the last step still owes, and this step's own copies.
   if (layer == 0 && !reference) {
-    st = append_book_only(c, slots, n, s);
+    st = append_book_only(c, slots, n, s, true);
     if (st) return st;
   }
   st = flush_pending(c);

@@ -39,6 +39,7 @@ constexpr int kInFlight = 2;               // stages whose copies may be outstan
                                            // delivers less when every SM keeps more in flight
 constexpr int kNewRowBit = 1 << 30;        // in the plan's slot word: the sequence got a new entry in this launch
 constexpr int kTimelineSlots = BC_TIMELINE_SLOTS;
+static_assert(kNewRowBit == BC_PLAN_NEW_ROW, "the bookkeeping kernel's plan uses the same bit");
 constexpr int kPidSlot = 136;              // ints per descriptor slot: 4 header + up to 132 page ids
 
 // ---------------------------------------------------------------- PTX helpers
@@ -120,6 +121,14 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+// Takes a ticket: release for the piece this block has just stored (the stores of the other threads are
+// ordered before it by the block barrier ahead of the call), acquire for the pieces the earlier ticket
+// holders stored (the threads that read them come after a block barrier behind the call).
+__device__ __forceinline__ int ticket_acq_rel(int* counter) {
+  int old;
+  asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
+  return old;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -184,6 +193,7 @@ struct FusedArgs {
   int32_t* dst_row;       // [n] pool row of every item's new entry (-1: the item was refused)
   int32_t* dst_pos;       // [n] its position in the window
   uint8_t* pool_w;        // the layer's pool, writable
+  const int32_t* plan;    // the plan the bookkeeping kernel of the step left (bc_decode_step), or NULL
   int32_t* flag;          // set to `epoch` by block 0 once the bookkeeping of this launch is done
   int32_t epoch;
   int32_t do_book;        // 1 on the layer-0 call of a step
@@ -372,7 +382,27 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   // between the last bookkeeping kernel and this one; it does not when this launch follows a bookkeeping
   // kernel directly (the fused step, small batches whose rows the bookkeeping block writes itself, a
   // call right after open / close / restore): then the wait comes first and nothing is read early.
-  const bool early = !FUSED && p.early_meta;
+  bool early = !FUSED && p.early_meta;
+  if (FUSED && p.f.plan != nullptr && !p.f.do_book) {
+    // bc_decode_step: the kernel ahead is this step's bookkeeping kernel.  It is running (it is what let this
+    // kernel begin) and stores the step's epoch to a flag word, with release semantics, as soon as its
+    // results -- lengths, page-table column, row destinations, the plan -- are written; then it only waits
+    // for the kernel ahead of IT, the previous step's attention kernel, to end.  Reading the flag with
+    // acquire semantics makes those results visible here, so this kernel, too, can plan and stream settled
+    // tiles while the previous step's last blocks finish.  If the flag does not show up in a while the
+    // block simply waits for the kernel ahead to end, which makes everything visible the ordinary way.
+    __shared__ int sh_flag_seen;
+    if (tid == 0) {
+      int seen = 0;
+      for (uint32_t polls = 0; polls < 2048; ++polls) {
+        if (ld_acquire(p.f.flag) == p.f.epoch) { seen = 1; break; }
+        __nanosleep(40);
+      }
+      sh_flag_seen = seen;
+    }
+    __syncthreads();
+    early = sh_flag_seen != 0;
+  }
   if (!early) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (FUSED && p.f.do_book) {
@@ -403,35 +433,48 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   // ---- plan: tiles per sequence, prefix sums, this block's span --------------------------------
   // Each segment (prompt, beacons, window) starts a new tile, so a tile never straddles segments;
   // a partly filled tile costs masked arithmetic but no memory traffic.
-  for (int i = tid; i < n; i += kPipeThreads) {
-    const int slot = p.a.slots[i];
-    int P = 0, nb = 0, w = 0, bcol = 0, wcol = 0, sl = 0;
-    if (slot >= 0 && slot < p.m.max_seqs && p.m.open[slot]) {
-      P = p.m.prompt_len[slot]; nb = p.m.n_beacons[slot]; w = p.m.window_len[slot];
-      bcol = p.m.beacon_off[slot]; wcol = p.m.window_off[slot]; sl = slot;
+  if (FUSED && p.f.plan != nullptr) {
+    // bc_decode_step: the step's bookkeeping kernel, whose results are visible (the flag, or the wait,
+    // above), left the plan of this very batch: seven coalesced reads instead of slots -> lengths -> prefix sum
+    const int32_t* a = p.f.plan + BC_PLAN_HEADER;
+    for (int i = tid; i < n; i += kPipeThreads) {
+      s_P[i] = a[i]; s_nb[i] = a[BC_MAX_ATTN_BATCH + i]; s_w[i] = a[2 * BC_MAX_ATTN_BATCH + i];
+      s_slot[i] = a[3 * BC_MAX_ATTN_BATCH + i]; s_bcol[i] = a[4 * BC_MAX_ATTN_BATCH + i]; s_wcol[i] = a[5 * BC_MAX_ATTN_BATCH + i];
+      s_cum[i] = a[6 * BC_MAX_ATTN_BATCH + i];
     }
-    if (FUSED && w > 0 && p.f.dst_row[i] >= 0) sl |= kNewRowBit;  // the window's last entry is this launch's
-    s_P[i] = P; s_nb[i] = nb; s_w[i] = w; s_slot[i] = sl; s_bcol[i] = bcol; s_wcol[i] = wcol;
-    const int tiles = ((P + T - 1) >> TS) + ((nb + T - 1) >> TS) + ((w + T - 1) >> TS);
-    s_cum[i + 1] = tiles > 0 ? tiles : 1;  // an empty sequence still owns one (empty) tile
-  }
-  __syncthreads();
-  if (warp == 0) {  // inclusive scan of s_cum[1..n]
-    int carry = 0;
-    for (int base = 0; base < n; base += 32) {
-      const int i = base + lane;
-      int x = i < n ? s_cum[i + 1] : 0;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        int y = __shfl_up_sync(0xffffffffu, x, d);
-        if (lane >= d) x += y;
+    if (tid == 0) s_cum[n] = a[6 * BC_MAX_ATTN_BATCH + n];
+    __syncthreads();
+  } else {
+    for (int i = tid; i < n; i += kPipeThreads) {
+      const int slot = p.a.slots[i];
+      int P = 0, nb = 0, w = 0, bcol = 0, wcol = 0, sl = 0;
+      if (slot >= 0 && slot < p.m.max_seqs && p.m.open[slot]) {
+        P = p.m.prompt_len[slot]; nb = p.m.n_beacons[slot]; w = p.m.window_len[slot];
+        bcol = p.m.beacon_off[slot]; wcol = p.m.window_off[slot]; sl = slot;
       }
-      if (i < n) s_cum[i + 1] = carry + x;
-      carry += __shfl_sync(0xffffffffu, x, 31);
+      if (FUSED && w > 0 && p.f.dst_row[i] >= 0) sl |= kNewRowBit;  // the window's last entry is this launch's
+      s_P[i] = P; s_nb[i] = nb; s_w[i] = w; s_slot[i] = sl; s_bcol[i] = bcol; s_wcol[i] = wcol;
+      const int tiles = ((P + T - 1) >> TS) + ((nb + T - 1) >> TS) + ((w + T - 1) >> TS);
+      s_cum[i + 1] = tiles > 0 ? tiles : 1;  // an empty sequence still owns one (empty) tile
     }
-    if (lane == 0) s_cum[0] = 0;
+    __syncthreads();
+    if (warp == 0) {  // inclusive scan of s_cum[1..n]
+      int carry = 0;
+      for (int base = 0; base < n; base += 32) {
+        const int i = base + lane;
+        int x = i < n ? s_cum[i + 1] : 0;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          int y = __shfl_up_sync(0xffffffffu, x, d);
+          if (lane >= d) x += y;
+        }
+        if (i < n) s_cum[i + 1] = carry + x;
+        carry += __shfl_sync(0xffffffffu, x, 31);
+      }
+      if (lane == 0) s_cum[0] = 0;
+    }
+    __syncthreads();
   }
-  __syncthreads();
   const int total_tiles = s_cum[n];
   stamp(1);
   // Every read of the sequences' lengths is done (the page-table columns the producer reads later are
@@ -684,6 +727,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    int early_cnt = -1;   // thread 0: the ticket counter as seen at the start of the final piece's last tile
 
     // ---- the extra (unstored) entry seeds the state of the piece that owns tile 0 ---------------
     if (p.a.extra_k != nullptr && ta == 0 && grp == 0) {
@@ -721,6 +765,10 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       // FUSED: the sequence's last tile lacks this launch's new entry (the bulk copy left it out);
       // the warps whose 16-row group holds it fetch their head's K and V chunks of it from the input
       // (lanes 0-15: K, lanes 16-31: V) while the tile is still in flight.
+      // The final piece's last tile: look at the sequence's ticket counter now, while the tile is still
+      // in flight.  If every other piece is there already, the merge after the tile starts at once (the
+      // count cannot go back); if not, the counter is read again after the tile.
+      if (!PAIR && !has_next && !whole && t == tb - 1 && tid == 0) early_cnt = ld_acquire(p.a.tickets + i);
       bool patch = false;
       int patch_row = 0;
       uint4 patch_val = make_uint4(0u, 0u, 0u, 0u);
@@ -969,10 +1017,12 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       const int first = cta_of(s_cum[i]), last = cta_of(s_cum[i + 1] - 1);
       bool merged = false;
       if (!has_next) {
-        // The block's final piece.  Usually every other piece of this sequence was published long
-        // ago (the rest of the sequence is some other block's first piece): then this block merges
-        // right away, taking its own piece from shared memory, and publishes nothing.
-        if (tid == 0) s_pend[4] = ld_acquire(p.a.tickets + i);
+        // The block's final piece.  If every other piece of this sequence was there already when the last
+        // tile began (the counter was read then, under the tile), this block merges right away, taking
+        // its own piece from shared memory, and publishes nothing.  Otherwise it publishes and takes a
+        // ticket like everybody else -- no second look at the counter: the blocks of a sequence finish
+        // within a microsecond or two of each other, so a look now mostly fails and costs a trip to L2.
+        if (tid == 0) s_pend[4] = early_cnt;
         consumer_bar();
         if (s_pend[4] == last - first) {
           __threadfence();
@@ -998,8 +1048,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
         } else {
           consumer_bar();  // orders every thread's stores before thread 0's fence
           if (tid == 0) {
-            __threadfence();
-            pend_tk = atomicAdd(p.a.tickets + i, 1);
+            pend_tk = ticket_acq_rel(p.a.tickets + i);
             pend_seq = i;
           }
           published_last = true;
@@ -1032,8 +1081,11 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     const int first = cta_of(s_cum[seq]), last = cta_of(s_cum[seq + 1] - 1);
     if (tk == last - first) {
       tl_path |= 8u << k;
-      __threadfence();
-      combine_pieces(p.a.part_o, p.a.part_ml, p.a.out, p.a.out_f32, Hq, D, seq, first, last, -1, nullptr, nullptr, tid);
+      if (k == 0 || PAIR) __threadfence();   // the service warp's and the paired form's tickets are plain atomics
+      // the final piece is still in the merge buffer (nothing followed it); the first piece is not
+      const bool own_here = k == 1 && !PAIR;
+      combine_pieces(p.a.part_o, p.a.part_ml, p.a.out, p.a.out_f32, Hq, D, seq, first, last, own_here ? cta : -1,
+                     own_here ? merge_o : nullptr, own_here ? merge_ml : nullptr, tid);
       if (PAIR) combine_pieces(p.a.part_o2, p.a.part_ml2, p.a.out2, p.a.out_f32, Hq, D, seq, first, last, -1, nullptr, nullptr, tid);
       if (tid == 0) p.a.tickets[seq] = 0;  // ready for the next launch
     }
@@ -1155,6 +1207,7 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
     p.f.new_k = static_cast<const uint8_t*>(fused->new_k); p.f.new_v = static_cast<const uint8_t*>(fused->new_v);
     p.f.dst_row = fused->dst_row; p.f.dst_pos = fused->dst_pos; p.f.pool_w = fused->pool_layer;
     p.f.flag = fused->flag; p.f.epoch = fused->epoch; p.f.do_book = fused->do_book; p.f.call = fused->call;
+    p.f.plan = fused->do_book ? nullptr : fused->plan;
   }
   p.scale_log2 = a.sm_scale * 1.4426950408889634f;
   p.n_groups = kConsumerWarps / g.kv_heads;

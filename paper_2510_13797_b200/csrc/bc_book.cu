@@ -108,9 +108,28 @@ __device__ __forceinline__ void wait_for_overtaken_kernel() { asm volatile("grid
 
 __global__ void __launch_bounds__(kBookThreads, 1)
 k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
-              int32_t* dst_row, int32_t* dst_pos, BcGeom g, uint8_t* pool_layer, const uint8_t* k, const uint8_t* v) {
-  append_book_block(m, slots, n, call, dst_row, dst_pos);
+              int32_t* dst_row, int32_t* dst_pos, BcGeom g, uint8_t* pool_layer, const uint8_t* k, const uint8_t* v,
+              int32_t* plan, int32_t* flag, int32_t epoch) {
+  // With a plan to leave, this is the bookkeeping of a fused decode step, and the kernel enqueued behind it
+  // is that step's attention kernel.  Its blocks may take their places on the SMs now; what they read of
+  // this kernel's results they read after the flag below (release here, acquire there), and everything the
+  // kernel ahead of this one may still be writing only after this kernel has ended.
+  if (plan != nullptr) {
+    // The flag word still holds an older epoch -- possibly this very one, when a captured step is replayed.
+    // It is cleared, and the clearing made visible device-wide, before any block of the dependent kernel
+    // can exist.
+    if (threadIdx.x == 0) { *reinterpret_cast<volatile int32_t*>(flag) = 0; __threadfence(); }
+    __syncthreads();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
+  int tile_shift = 4;   // rows per tile of the attention kernel: 16 * (8 / kv_heads)
+  while ((16 << (tile_shift - 4)) * g.kv_heads < 128) ++tile_shift;
+  append_book_block(m, slots, n, call, dst_row, dst_pos, plan, tile_shift);
   __syncthreads();
+  if (plan != nullptr && threadIdx.x == 0) {   // lengths, page-table column, row destinations and plan are written
+    __threadfence();
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(epoch) : "memory");
+  }
   if (k != nullptr) block_write_rows(m, g, pool_layer, dst_row, dst_pos, k, v, n);  // layer 0's rows, same launch
   wait_for_overtaken_kernel();
 }
@@ -494,12 +513,12 @@ cudaError_t launch_book_overlapped(void (*kernel)(KArgs...), cudaStream_t s, Arg
 
 cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                   int32_t* dst_pos, const BcGeom& g, uint8_t* pool_layer, const void* k, const void* v,
-                                  cudaStream_t s) {
+                                  cudaStream_t s, int32_t* plan, int32_t* flag, int32_t epoch) {
   if (k == nullptr)   // the rows follow in a launch of their own (ordinary order: it waits for everything before it)
     return launch_book_overlapped(k_append_book, s, m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)nullptr,
-                                  (const uint8_t*)nullptr);
+                                  (const uint8_t*)nullptr, plan, flag, epoch);
   k_append_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)k,
-                                           (const uint8_t*)v);
+                                           (const uint8_t*)v, (int32_t*)nullptr, (int32_t*)nullptr, 0);
   return cudaGetLastError();
 }
 cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,

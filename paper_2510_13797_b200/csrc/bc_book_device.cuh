@@ -91,8 +91,11 @@ struct ErrLatch {
 // size (block-wide prefix sum: deterministic page ids), bumps window_len and t, and writes for
 // every item its pool row (dst_row; -1 if the item failed) and its position in the window
 // (dst_pos).  The first failing item is latched.  Every thread of the block must call it.
+// With `plan` non-NULL the block also leaves the decode-attention kernel's plan for this batch, as the
+// lengths stand after the append (see BcPlan in bc_common.cuh): one coalesced read there instead of
+// slots -> lengths -> prefix sum.
 __device__ void append_book_block(const BcMeta& m, const int32_t* __restrict__ slots, int n, int64_t call, int32_t* dst_row,
-                                  int32_t* dst_pos) {
+                                  int32_t* dst_pos, int32_t* plan = nullptr, int tile_shift = 0) {
   __shared__ int sh_first;
   ErrLatch latch; latch.init(&sh_first);
   dup_prepass(m, slots, n, call);
@@ -147,4 +150,32 @@ __device__ void append_book_block(const BcMeta& m, const int32_t* __restrict__ s
   latch.commit(m, my_item, my_code, my_slot, call);
   __syncthreads();
   if (threadIdx.x == 0) *m.free_top = top0 - sh_used;
+  if (plan != nullptr && n <= BC_MAX_ATTN_BATCH) {
+    // every thread sees the block's own writes to the lengths after the barrier above
+    const int T = 1 << tile_shift;
+    int32_t* a = plan + BC_PLAN_HEADER;
+    int carry = 0;
+    for (int chunk = 0; chunk < n; chunk += blockDim.x) {
+      const int i = chunk + threadIdx.x;
+      int tiles = 0;
+      if (i < n) {
+        const int slot = slots[i];
+        int P = 0, nb = 0, w = 0, bcol = 0, wcol = 0, sl = 0;
+        if (slot >= 0 && slot < m.max_seqs && m.open[slot]) {
+          P = m.prompt_len[slot]; nb = m.n_beacons[slot]; w = m.window_len[slot];
+          bcol = m.beacon_off[slot]; wcol = m.window_off[slot]; sl = slot;
+        }
+        if (w > 0 && dst_row[i] >= 0) sl |= BC_PLAN_NEW_ROW;
+        a[0 * BC_MAX_ATTN_BATCH + i] = P; a[1 * BC_MAX_ATTN_BATCH + i] = nb; a[2 * BC_MAX_ATTN_BATCH + i] = w;
+        a[3 * BC_MAX_ATTN_BATCH + i] = sl; a[4 * BC_MAX_ATTN_BATCH + i] = bcol; a[5 * BC_MAX_ATTN_BATCH + i] = wcol;
+        tiles = ((P + T - 1) >> tile_shift) + ((nb + T - 1) >> tile_shift) + ((w + T - 1) >> tile_shift);
+        if (tiles == 0) tiles = 1;   // an empty sequence still owns one (empty) tile
+      }
+      int total;
+      const int off = carry + block_exclusive_scan(tiles, &total);
+      if (i < n) a[6 * BC_MAX_ATTN_BATCH + i] = off;
+      carry += total;
+    }
+    if (threadIdx.x == 0) { a[6 * BC_MAX_ATTN_BATCH + n] = carry; plan[0] = n; plan[1] = carry; plan[2] = tile_shift; }
+  }
 }

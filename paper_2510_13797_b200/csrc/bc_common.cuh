@@ -12,6 +12,13 @@
 #define BC_MAX_ATTN_CTAS 304   // thread blocks of the decode-attention kernel
 #define BC_MAX_ATTN_BATCH 512  // sequences per bc_decode_attn call
 #define BC_MERGE_ELEMS 4096    // q_heads * head_dim that fits the in-block merge buffer
+// The attention plan the append bookkeeping can leave for the fused decode step: BC_PLAN_HEADER ints
+// {n, total tiles, log2(rows per tile), -}, then seven arrays of BC_MAX_ATTN_BATCH (+1 for the last) ints:
+// prompt length, beacons, window length, slot (| BC_PLAN_NEW_ROW if the step appended an entry), first
+// beacon column, first window column, and the exclusive prefix sums of the sequences' tile counts.
+#define BC_PLAN_HEADER 4
+#define BC_PLAN_INTS (BC_PLAN_HEADER + 7 * BC_MAX_ATTN_BATCH + 4)
+#define BC_PLAN_NEW_ROW (1 << 30)
 #define BC_TIMELINE_SLOTS 16   // 64-bit words per thread block in a bc_attn_timeline buffer
 
 // Device view of the bookkeeping ("meta" buffer).  All arrays are int32.
@@ -53,9 +60,11 @@ cudaError_t bc_launch_open(const BcMeta& m, const int32_t* slots, const int32_t*
                            int n, int64_t call, cudaStream_t s);
 // k, v non-null: the same launch also writes the rows into pool_layer (what bc_launch_write_rows
 // does), which saves a launch when the batch is small enough for one thread block to copy.
+// plan non-null (k, v null): the launch also leaves the attention plan of the batch (BC_PLAN_INTS ints) and
+// then stores `epoch` to *flag with release semantics
 cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                   int32_t* dst_pos, const BcGeom& g, uint8_t* pool_layer, const void* k, const void* v,
-                                  cudaStream_t s);
+                                  cudaStream_t s, int32_t* plan = nullptr, int32_t* flag = nullptr, int32_t epoch = 0);
 // phase bit 1: allocate the beacon slot; phase bit 2: evict the window and bump the counters
 cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                     int32_t* dst_pos, int phase, const BcGeom& g, uint8_t* pool_layer, const void* k,
@@ -108,6 +117,7 @@ struct BcFusedAppend {
   int32_t* dst_row;      // [n] workspace: pool row of each item's new entry, -1 if refused (written on layer 0)
   int32_t* dst_pos;      // [n] workspace: its position in the window
   uint8_t* pool_layer;   // the layer's pool (writable)
+  const int32_t* plan;   // NULL, or the plan the step's bookkeeping kernel left (BC_PLAN_INTS ints)
   int32_t* flag;         // workspace word: "the bookkeeping of launch `epoch` is done"
   int32_t epoch;
   int32_t do_book;       // 1: this launch runs the bookkeeping (the layer-0 call of the step)

@@ -103,8 +103,9 @@ def test_sweep_mid_generation_fused_step():
     drv.check_error()
 
 
-@pytest.mark.parametrize("c,paired", [(2, True), (16, True), (16, False), (32, True)])
-def test_sweep_window_replayed_as_cuda_graph(c, paired):
+@pytest.mark.parametrize("c,paired,fused", [(2, True, True), (16, True, True), (16, False, False), (32, True, True), (32, True, False),
+                                            (4, False, True)])
+def test_sweep_window_replayed_as_cuda_graph(c, paired, fused):
     """The launch configuration the benchmark times: whole windows of steps captured once as a CUDA
     graph and replayed.  A replay feeds the inputs of the captured steps again, so the captured span
     is a whole number of input periods (the step inputs repeat every `ring` steps, the beacons every
@@ -113,7 +114,7 @@ def test_sweep_window_replayed_as_cuda_graph(c, paired):
     three replays the outputs left by the last step (it fills a window: token rows and beacon rows,
     paired or as two passes) and the bookkeeping must be those of the oracle for that step."""
     w = make_workload("sweep", c=c)
-    drv = DecodeDriver(w, DEV, paired=paired, beacon_ring=37)
+    drv = DecodeDriver(w, DEV, paired=paired, fused=fused, beacon_ring=37)   # fused: regular steps through bc_decode_step, as bench.py times them
     span = math.lcm(drv.ring, drv.bring * c)
     t0 = (w.steps // 2 // span) * span
     drv.reset_to(t0)

@@ -57,8 +57,8 @@ def entries_beacon_query(P, t, c):
 # case of each ratio (--profile-case C: same bytes per launch and page size as mid-generation), for
 # the library version named here; see profiles/.  Slightly below 1: part of the stream stays in L2
 # from the previous step.  A different library version invalidates the figures (traffic: null).
-TRAFFIC_FOR_VERSION = 114
-TRAFFIC_OVER_ALGORITHMIC = {2: 0.996, 4: 0.981, 8: 0.960, 16: 0.943, 32: 0.982}
+TRAFFIC_FOR_VERSION = 200
+TRAFFIC_OVER_ALGORITHMIC = {2: 0.996, 4: 0.980, 8: 0.960, 16: 0.943, 32: 0.979}
 
 
 def traffic_per_launch(c, algorithmic_bytes):
@@ -362,7 +362,7 @@ def run_profile_case(args):
     mid = entries_attended(w.prompt_lens[0], w.steps // 2, c)
     w = make_workload("sweep", c=c, prompt_lens=[mid] * w.batch, gen_lens=[4 * max(c, 16) + args.steps + 64] * w.batch)
     torch.cuda.set_device(0)
-    r = make_runner(w, torch.device("cuda", 0))
+    r = make_runner(w, torch.device("cuda", 0), fused=not args.no_fused)
     r.reset_to(0)
     ms, n, nbytes, region = r.timed_kernels(args.steps, max(args.warmup, 3))
     r.check_error()
@@ -1002,6 +1002,7 @@ def main():
                     help="sweep (default): the benchmark line; cfg2 / ragged / depth: a report line for that "
                          "benchmark configuration (1 GPU)")
     ap.add_argument("--no-batch-scaling", action="store_true")
+    ap.add_argument("--replays", type=int, default=3, help="rewind-and-replay rounds of the timed graph (the first one is the reported time)")
     ap.add_argument("--no-extras", action="store_true", help="skip the short mask-form and distillation runs of the default line")
     ap.add_argument("--timeline", type=int, default=0, metavar="C",
                     help="per-block time stamps of the attention kernel (bc_attn_timeline) on the small case of ratio C")
@@ -1060,7 +1061,7 @@ def main():
         # pass A: device-resident inputs, CUDA-graph replays: the headline time
         r.reset_to(max(0, t_mid - W - cyc))
         barrier()
-        ms, t_begin, launches = r.timed_graph(K, max(W, t_mid - r.t - cyc))
+        ms, t_begin, launches = r.timed_graph(K, max(W, t_mid - r.t - cyc), replays=args.replays)
         # pass B: plain launches, every attention kernel bracketed by events: the roofline figures
         Kp = min(K, 256)
         r.reset_to(max(0, t_mid - W))

@@ -961,6 +961,25 @@ def report_model(args):
                       "rows": rows}))
 
 
+def read_stream_peak(dev):
+    """GB/s of a read-only pass over 4 GiB with the attention kernel's copy pattern and no arithmetic
+    (bc_probe_read_stream): best of five after two warm-up passes."""
+    import torch
+    from paper_2510_13797_b200 import binding as B
+    buf = torch.empty(4 << 30, dtype=torch.uint8, device=dev)
+    buf.fill_(1)
+    best = 0.0
+    for i in range(7):
+        e0, e1 = _event_pair(torch)
+        e0.record(); B.bc_probe_read_stream(buf); e1.record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            best = max(best, buf.numel() / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del buf
+    torch.cuda.empty_cache()
+    return best
+
+
 def batch_scaling(dev, peak):
     """The attention kernel alone at larger batches (same shape, mid-generation cache): the time per
     launch that does not stream (start-up, merging) is spread over more bytes."""
@@ -1162,6 +1181,12 @@ def main():
                                    "whole step"},
         "sweep": rows,
     }
+    if world == 1:
+        rs = read_stream_peak(dev)
+        line["roofline"]["read_stream_gbs"] = rs
+        line["roofline"]["frac_of_read_stream"] = achieved / rs
+        line["roofline"]["read_stream_note"] = ("read-only pass with the kernel's own copy pattern and no arithmetic "
+                                                "(bc_probe_read_stream): unlike the copy benchmark behind `peak`, a ceiling")
     if not args.no_batch_scaling and world == 1:
         line["batch_scaling"] = batch_scaling(dev, peak)
     if not args.no_extras and world == 1:

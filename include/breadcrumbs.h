@@ -472,6 +472,15 @@ BC_API bc_status bc_set_wait_limit(bc_cache* cache, uint32_t polls);
 #define BC_TIMELINE_WORDS 16
 BC_API bc_status bc_attn_timeline(bc_cache* cache, void* device_words, int32_t blocks);
 
+/* A measurement aid, no part of the method: reads `bytes` (rounded down to a multiple of 64 KB) of
+ * device memory once, with the decode-attention kernel's own access pattern (one thread block per SM,
+ * 64 KB bulk copies into a three-stage shared-memory ring, two in flight, evict-first) and no
+ * arithmetic.  Timed by the caller with events, bytes / time is the read bandwidth that pattern can
+ * reach on the device at hand: the ceiling for the attention kernel's streaming phase, and a
+ * denominator that, unlike a copy benchmark's, keeps roofline fractions below 1.  Asynchronous on
+ * `stream`; device_buf 16-byte aligned, bytes >= 64 KB. */
+BC_API bc_status bc_probe_read_stream(const void* device_buf, size_t bytes, void* stream);
+
 /* Kernels launched by this handle since creation (for launch accounting). */
 BC_API int64_t bc_kernel_launches(const bc_cache* cache);
 

@@ -83,6 +83,7 @@ SYMBOLS = {
     "bc_mask_attn_set_wait_limit": (_I32, [C.c_uint32]),
     "bc_profile_enable": (_I32, [_P, _I32]),
     "bc_profile_read": (_I32, [_P, C.POINTER(_I32), C.POINTER(_F)]),
+    "bc_probe_read_stream": (_I32, [_P, C.c_size_t, _P]),
     "bc_kernel_launches": (_I64, [_P]),
     "bc_last_cuda_error": (_I32, [_P]),
     "bc_status_string": (C.c_char_p, [_I32]),
@@ -299,6 +300,11 @@ def bc_mask_attn_forward(prompt_lens, token_lens, c, prompt_k, prompt_v, tok_q, 
                                          C.byref(code)), "bc_mask_attn_status")
         _check(code.value, "bc_mask_attn_forward (device)")
     return out_tok, out_bea
+
+
+def bc_probe_read_stream(buf, stream=None):
+    """Reads the CUDA tensor `buf` once with the attention kernel's copy pattern (breadcrumbs.h)."""
+    _check(lib().bc_probe_read_stream(_ptr(buf), buf.numel() * buf.element_size(), _stream(stream)), "bc_probe_read_stream")
 
 
 def bc_distill_loss(cu_rows, student_logits, teacher_idx, teacher_logprob, with_grad=False, stream=None):

@@ -1002,6 +1002,11 @@ bc_status bc_decode_attn_static(bc_cache* c, int32_t layer, const int32_t* slots
   return BC_OK;
 }
 
+bc_status bc_probe_read_stream(const void* device_buf, size_t bytes, void* stream) {
+  if (!device_buf || bytes < (64u << 10) || (reinterpret_cast<uintptr_t>(device_buf) & 15)) return BC_ERR_INVALID_ARG;
+  return bc_launch_read_stream(device_buf, bytes, nullptr, (cudaStream_t)stream) == cudaSuccess ? BC_OK : BC_ERR_CUDA;
+}
+
 int64_t bc_kernel_launches(const bc_cache* c) { return c ? c->launches : 0; }
 int32_t bc_last_cuda_error(const bc_cache* c) { return c ? c->last_cuda_error : 0; }
 

@@ -1094,6 +1094,61 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   stamp_val(9, tl_path);
 }
 
+// ---------------------------------------------------------------- read-only streaming probe
+// What the decode kernel's own access pattern can draw from HBM when nothing is computed: every block
+// copies its share of a buffer in 64 KB pieces into a three-stage ring with the same 1-D bulk copies,
+// the same evict-first policy and the same limit of two stages in flight; one warp consumes (waits
+// for a stage and hands it back).  A measurement aid for the roofline's denominator: the copy
+// benchmark that defines the reported peak reads AND writes, a decode step only reads.
+__global__ void __launch_bounds__(64, 1) k_read_stream(const uint8_t* __restrict__ buf, long long pieces, int* sink) {
+  constexpr int kPiece = 64 << 10, kRing = 3;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  __shared__ __align__(8) uint64_t bars[2 * kRing];
+  __shared__ int s_abort_word;
+  volatile int* s_abort = &s_abort_word;
+  const uint32_t ring = smem_u32(smem), bar_full = smem_u32(bars), bar_empty = bar_full + kRing * 8;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kRing; ++s) { mbar_init(bar_full + s * 8, 1); mbar_init(bar_empty + s * 8, 1); }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_proxy_async();
+  }
+  __syncthreads();
+  const long long per = pieces / gridDim.x, rem = pieces % gridDim.x;
+  const long long p0 = blockIdx.x * per + (blockIdx.x < rem ? blockIdx.x : rem), p1 = p0 + per + (blockIdx.x < rem ? 1 : 0);
+  if (warp == 0) {
+    const uint64_t policy = l2_policy_evict_first();
+    int it = 0;
+    bool ok = true;
+    for (long long pc = p0; pc < p1 && ok; ++pc, ++it) {
+      const int stage = it % kRing;
+      ok = bounded_wait(bar_empty + stage * 8, ((it / kRing) & 1) ^ 1, s_abort, kSpinLimit);
+      if (ok && it >= kInFlight) ok = bounded_wait(bar_full + ((it - kInFlight) % kRing) * 8, ((it - kInFlight) / kRing) & 1, s_abort, kSpinLimit);
+      if (!ok) break;
+      if (lane == 0) {
+        mbar_arrive_expect_tx(bar_full + stage * 8, kPiece);
+        bulk_g2s(ring + stage * kPiece, buf + pc * kPiece, kPiece, bar_full + stage * 8, policy);
+      }
+      __syncwarp();
+    }
+    for (int k = max(0, it - kRing); k < it; ++k) {   // nothing may be in flight when the block leaves
+      uint32_t polls = 0;
+      while (!mbar_try_wait(bar_full + (k % kRing) * 8, (k / kRing) & 1) && ++polls < kSpinLimit) __nanosleep(64);
+    }
+  } else {
+    int it = 0, acc = 0;
+    for (long long pc = p0; pc < p1; ++pc, ++it) {
+      const int stage = it % kRing;
+      if (!bounded_wait(bar_full + stage * 8, (it / kRing) & 1, s_abort, kSpinLimit)) break;
+      acc ^= reinterpret_cast<const int*>(smem + stage * kPiece)[lane];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_empty + stage * 8);
+    }
+    if (acc == 0x7fffffff && sink) *sink = acc;   // keeps the read alive
+  }
+}
+
 // ---------------------------------------------------------------- slow device reference
 // grid (n, q_heads), one warp per block; lanes split head_dim.
 __global__ void k_attn_reference(BcMeta m, BcGeom g, BcAttnArgs a) {
@@ -1232,6 +1287,16 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   if (ev_stop) { e = cudaEventRecord(ev_stop, s); if (e != cudaSuccess) return e; }
   *launches = 1;
   return cudaSuccess;
+}
+
+cudaError_t bc_launch_read_stream(const void* buf, size_t bytes, int* sink, cudaStream_t s) {
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_read_stream, cudaFuncAttributeMaxDynamicSharedMemorySize, 3 * (64 << 10));
+  if (e != cudaSuccess) return e;
+  k_read_stream<<<sms, 64, 3 * (64 << 10), s>>>(static_cast<const uint8_t*>(buf), (long long)(bytes >> 16), sink);
+  return cudaGetLastError();
 }
 
 cudaError_t bc_launch_attn_reference(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, cudaStream_t s) {

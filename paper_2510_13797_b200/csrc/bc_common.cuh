@@ -127,5 +127,7 @@ struct BcFusedAppend {
 // the same launch appends the step's new entries first.  *launches gets the number of kernels.
 cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, const BcFusedAppend* fused,
                            cudaStream_t s, cudaEvent_t ev_start, cudaEvent_t ev_stop, int* launches);
+// Read-only streaming probe: reads bytes (rounded down to 64 KB) of buf once with the attention kernel's copy pattern.
+cudaError_t bc_launch_read_stream(const void* buf, size_t bytes, int* sink, cudaStream_t s);
 // Slow device reference (one warp per query head).
 cudaError_t bc_launch_attn_reference(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, cudaStream_t s);

@@ -384,6 +384,11 @@ def run_timeline(args):
     w = make_workload("sweep", c=c)
     mid = entries_attended(w.prompt_lens[0], w.steps // 2, c)
     w = make_workload("sweep", c=c, prompt_lens=[mid] * w.batch, gen_lens=[8 * max(c, 16) + 64] * w.batch)
+    if args.timeline_shape == "depth":     # one layer of the full-depth configuration: batch 256, 12/2 heads, page = c
+        d = make_workload("depth", c=c)
+        mid = entries_attended(d.prompt_lens[0], d.steps // 2, c)
+        w = make_workload("sweep", c=c, batch=d.batch, q_heads=d.q_heads, kv_heads=d.kv_heads, page_size=d.page_size,
+                          prompt_lens=[mid] * d.batch, gen_lens=[8 * max(c, 16) + 64] * d.batch, cs=[c] * d.batch)
     torch.cuda.set_device(0)
     r = make_runner(w, torch.device("cuda", 0), fused=args.fused)
     r.reset_to(1)
@@ -700,7 +705,7 @@ def report_depth(args):
                 cache.bc_append(l, slots, k[j], v[j])
                 cache.bc_decode_attn_pair(l, slots, q[j], out, bq[m], out_b, w.sm_scale, bk[m], bv[m])
                 cache.bc_compress(l, slots, bk[m], bv[m])
-            elif attend and args.fused:
+            elif attend and not args.no_fused:
                 cache.bc_decode_step(l, slots, q[j], k[j], v[j], out, w.sm_scale)
             else:
                 cache.bc_append(l, slots, k[j], v[j])
@@ -750,6 +755,7 @@ def report_depth(args):
     line = {
         "workload": "depth: 28 layers, B=256, 12/2 heads, D=128, P=512, T=8192, c=8, page 8",
         "beacon_steps": "paired with the token's attention (one pass over the cache per layer)" if paired else "second attention pass",
+        "regular_steps": "bc_append + bc_decode_attn per layer" if args.no_fused else "bc_decode_step per layer",
         "steps": K, "t_window": [t_begin, t_begin + K], "ms_per_step": ms / K,
         "attention_tokens_per_s": Bn * K / (ms * 1e-3), "layer_tokens_per_s": Bn * K * L / (ms * 1e-3),
         "kv_bytes_per_step": kv / K, "kv_gbs": kv / (ms * 1e-3) / 1e9,
@@ -1012,8 +1018,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-pair", action="store_true", help="beacon steps as a second attention pass instead of bc_decode_attn_pair")
     ap.add_argument("--pair", action="store_true", help="ragged workload: pair the beacon steps too (off by default there)")
-    ap.add_argument("--fused", action="store_true", help="depth workload and --timeline: regular steps through bc_decode_step (append + attention in one launch per layer)")
-    ap.add_argument("--no-fused", action="store_true", help="sweep: regular steps as bc_append + bc_decode_attn instead of bc_decode_step")
+    ap.add_argument("--fused", action="store_true", help="--timeline: regular steps through bc_decode_step")
+    ap.add_argument("--no-fused", action="store_true", help="sweep, depth, --profile-case: regular steps as bc_append + bc_decode_attn instead of bc_decode_step")
     ap.add_argument("--ratios", default="")
     ap.add_argument("--skip-uncompressed", action="store_true")
     ap.add_argument("--model-ratio", type=int, default=None, help=argparse.SUPPRESS)   # model workload: one ratio (child process)
@@ -1025,6 +1031,7 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the short mask-form and distillation runs of the default line")
     ap.add_argument("--timeline", type=int, default=0, metavar="C",
                     help="per-block time stamps of the attention kernel (bc_attn_timeline) on the small case of ratio C")
+    ap.add_argument("--timeline-shape", default="sweep", choices=["sweep", "depth"], help="with --timeline: the sweep's head shape and batch, or one layer of the full-depth configuration")
     ap.add_argument("--timeline-raw", action="store_true", help="with --timeline: also print every block's stamps")
     ap.add_argument("--profile-case", type=int, default=0, metavar="C",
                     help="small case for profilers: ratio C with a prompt as long as the mid-generation cache, "

@@ -446,8 +446,10 @@ BC_API bc_status bc_set_attn_ctas(bc_cache* cache, int32_t ctas);
 BC_API bc_status bc_profile_enable(bc_cache* cache, int32_t max_launches);
 BC_API bc_status bc_profile_read(bc_cache* cache, int32_t* launches, float* total_ms);
 
-/* Poll limit of the bounded waits inside the decode-attention kernels this handle launches (0 = the
- * default, about a quarter of a second).  A wait that runs out makes its thread block stop issuing
+/* Poll limit of the bounded waits inside the kernels of bc_decode_attn and bc_decode_step this handle
+ * launches (0 = the default, about a quarter of a second; the paired form keeps the default).  The
+ * settable limit lives in kernel variants of its own, built for head_dim 128 with at most 8 query
+ * heads per KV head: other shapes return BC_ERR_UNSUPPORTED.  A wait that runs out makes its thread block stop issuing
  * copies, wait (with the full default limit) for the copies it has in flight, record BC_ERR_TIMEOUT
  * in the status record and return; the call's outputs are then undefined and split-K ticket counters may
  * be left non-zero until bc_clear_error.  A limit of 1 makes practically every launch give up at

@@ -909,6 +909,7 @@ bc_status bc_set_attn_ctas(bc_cache* c, int32_t ctas) {
 
 bc_status bc_set_wait_limit(bc_cache* c, uint32_t polls) {
   if (!c) return BC_ERR_INVALID_ARG;
+  if (polls != 0 && (c->cfg.head_dim != 128 || c->cfg.q_heads / c->cfg.kv_heads > 8)) return BC_ERR_UNSUPPORTED;
   c->wait_limit = polls;
   return BC_OK;
 }

@@ -156,17 +156,24 @@ __device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity
 }
 constexpr uint32_t kShortLimit = 1024;   // limits below this poll without suspending (try_wait may sleep for a while inside)
 
+// Bounded wait; returns false when it gave up or another warp already aborted.  The ordinary
+// instantiation has a compile-time limit: with the limit as a run-time value the polling loop compiles
+// into something measurably slower (3 us per launch on 64-row tiles), so the settable limit of
+// bc_set_wait_limit lives in instantiations of its own (SHORTW), which the host picks only when a
+// limit has been set.  Limits below kShortLimit poll with test_wait, which never suspends the thread.
+template <bool SHORTW>
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
-  if (limit < kShortLimit) {   // a deliberately short limit (bc_set_wait_limit): a few non-blocking looks, then give up
+  if (SHORTW && limit < kShortLimit) {
     for (uint32_t polls = 0; polls <= limit; ++polls)
       if (mbar_test_wait(bar, parity)) return true;
     *abort_flag = 1;
     return false;
   }
+  const uint32_t lim = SHORTW ? limit : kSpinLimit;
   uint32_t polls = 0;
   while (!mbar_try_wait(bar, parity)) {
     if (++polls > 1024) __nanosleep(64);
-    if (polls > limit || *abort_flag) {
+    if (polls > lim || *abort_flag) {
       *abort_flag = 1;
       return false;
     }
@@ -321,7 +328,7 @@ __device__ __forceinline__ void combine_pieces(const float* part_o, const float*
 // fills the window and the encoding of the beacon that follows it (Algorithm 1) read the same entries.
 // The beacon's rows also see the extra entry (the beacon's own K/V).  Needs G <= 8 and is compiled
 // on the 16-row path (G_LE_8 = false); results go to out (token) and out2 (beacon).
-template <int D, bool G_LE_8, bool FUSED, bool PAIR = false>
+template <int D, bool G_LE_8, bool FUSED, bool PAIR = false, bool SHORTW = false>
 __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams p) {
   static_assert(!PAIR || (!G_LE_8 && !FUSED), "the paired form runs on the 16-row path without the fused append");
   using L = PipeSmem<D>;
@@ -542,7 +549,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       }
     }
     if (svc_publishes) {
-      const bool ok = bounded_wait(bar_pub, 0, s_abort, p.spin_limit);  // every consumer warp has stored its share
+      const bool ok = bounded_wait<SHORTW>(bar_pub, 0, s_abort, p.spin_limit);  // every consumer warp has stored its share
       if (lane == 0) {
         if (ok) {
           __threadfence();
@@ -626,10 +633,10 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       if (!waited && !s_desc[(it % RING) * kPidSlot + 3]) { wait_for_kernel_ahead(); waited = true; }
       const int stage = it % NSTAGE;
       const uint32_t full = bar_full + stage * 8, empty = bar_empty + stage * 8;
-      if (!bounded_wait(empty, ((it / NSTAGE) & 1) ^ 1, s_abort, p.spin_limit)) aborted = true;
+      if (!bounded_wait<SHORTW>(empty, ((it / NSTAGE) & 1) ^ 1, s_abort, p.spin_limit)) aborted = true;
       // at most kInFlight stages in flight: the copies of tile it - kInFlight must have landed
       if (!aborted && it >= kInFlight &&
-          !bounded_wait(bar_full + ((it - kInFlight) % NSTAGE) * 8, ((it - kInFlight) / NSTAGE) & 1, s_abort, p.spin_limit))
+          !bounded_wait<SHORTW>(bar_full + ((it - kInFlight) % NSTAGE) * 8, ((it - kInFlight) / NSTAGE) & 1, s_abort, p.spin_limit))
         aborted = true;
       if (aborted) break;   // `it` stages have been armed; the consumers see the abort flag in their own waits
       {
@@ -781,7 +788,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
                                                         ((int64_t)i * Hkv + kvh) * p.g.head_row_bytes + ((lane & 15) << 4));
         }
       }
-      const bool ok = __all_sync(0xffffffffu, bounded_wait(bar_full + stage * 8, (it / NSTAGE) & 1, s_abort, p.spin_limit));
+      const bool ok = __all_sync(0xffffffffu, bounded_wait<SHORTW>(bar_full + stage * 8, (it / NSTAGE) & 1, s_abort, p.spin_limit));
       if (it == 0) stamp(3);
       if (!ok && lane == 0 && p.m.status[0] == 0) { p.m.status[0] = BC_ERR_TIMEOUT; p.m.status[1] = -1; }
       // rows of this tile that hold entries; my warp looks at rows grp*16 .. grp*16+15 of it
@@ -1068,7 +1075,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
 
   // ---- all tiles streamed: merge the sequences whose last ticket this block took -----------------
   stamp(5);
-  if (svc_publishes) bounded_wait(bar_tk, 0, s_abort, p.spin_limit);
+  if (svc_publishes) bounded_wait<SHORTW>(bar_tk, 0, s_abort, p.spin_limit);
   stamp(6);
   if (published_last) {
     if (tid == 0) { s_pend[2] = pend_seq; s_pend[3] = pend_tk; }
@@ -1123,8 +1130,8 @@ __global__ void __launch_bounds__(64, 1) k_read_stream(const uint8_t* __restrict
     bool ok = true;
     for (long long pc = p0; pc < p1 && ok; ++pc, ++it) {
       const int stage = it % kRing;
-      ok = bounded_wait(bar_empty + stage * 8, ((it / kRing) & 1) ^ 1, s_abort, kSpinLimit);
-      if (ok && it >= kInFlight) ok = bounded_wait(bar_full + ((it - kInFlight) % kRing) * 8, ((it - kInFlight) / kRing) & 1, s_abort, kSpinLimit);
+      ok = bounded_wait<false>(bar_empty + stage * 8, ((it / kRing) & 1) ^ 1, s_abort, kSpinLimit);
+      if (ok && it >= kInFlight) ok = bounded_wait<false>(bar_full + ((it - kInFlight) % kRing) * 8, ((it - kInFlight) / kRing) & 1, s_abort, kSpinLimit);
       if (!ok) break;
       if (lane == 0) {
         mbar_arrive_expect_tx(bar_full + stage * 8, kPiece);
@@ -1140,7 +1147,7 @@ __global__ void __launch_bounds__(64, 1) k_read_stream(const uint8_t* __restrict
     int it = 0, acc = 0;
     for (long long pc = p0; pc < p1; ++pc, ++it) {
       const int stage = it % kRing;
-      if (!bounded_wait(bar_full + stage * 8, (it / kRing) & 1, s_abort, kSpinLimit)) break;
+      if (!bounded_wait<false>(bar_full + stage * 8, (it / kRing) & 1, s_abort, kSpinLimit)) break;
       acc ^= reinterpret_cast<const int*>(smem + stage * kPiece)[lane];
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_empty + stage * 8);
@@ -1214,7 +1221,7 @@ FastDiv make_fast_div(uint32_t d) {
   return f;
 }
 
-template <int D, bool G8, bool FUSED, bool PAIR = false>
+template <int D, bool G8, bool FUSED, bool PAIR = false, bool SHORTW = false>
 cudaError_t launch_pipe(const PipeParams& p, cudaStream_t s) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p.a.ctas); cfg.blockDim = dim3(kPipeThreads); cfg.dynamicSmemBytes = PipeSmem<D>::kTotal; cfg.stream = s;
@@ -1222,15 +1229,15 @@ cudaError_t launch_pipe(const PipeParams& p, cudaStream_t s) {
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;   // see the kernel: it waits for its predecessor after its plan
   cfg.attrs = at; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, k_attn_pipe<D, G8, FUSED, PAIR>, p);
+  return cudaLaunchKernelEx(&cfg, k_attn_pipe<D, G8, FUSED, PAIR, SHORTW>, p);
 }
 
 }  // namespace
 
 namespace {
-template <int D, bool G8, bool FUSED, bool PAIR = false>
+template <int D, bool G8, bool FUSED, bool PAIR = false, bool SHORTW = false>
 cudaError_t opt_in_smem() {
-  return cudaFuncSetAttribute(k_attn_pipe<D, G8, FUSED, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<D>::kTotal);
+  return cudaFuncSetAttribute(k_attn_pipe<D, G8, FUSED, PAIR, SHORTW>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<D>::kTotal);
 }
 }  // namespace
 
@@ -1240,7 +1247,8 @@ cudaError_t bc_attn_setup(int* sm_count) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  const cudaError_t r[10] = {opt_in_smem<128, true, false>(), opt_in_smem<128, false, false>(), opt_in_smem<64, true, false>(),
+  const cudaError_t r[12] = {opt_in_smem<128, true, false, false, true>(), opt_in_smem<128, true, true, false, true>(),
+                             opt_in_smem<128, true, false>(), opt_in_smem<128, false, false>(), opt_in_smem<64, true, false>(),
                              opt_in_smem<64, false, false>(), opt_in_smem<128, true, true>(), opt_in_smem<128, false, true>(),
                              opt_in_smem<64, true, true>(), opt_in_smem<64, false, true>(),
                              opt_in_smem<128, false, false, true>(), opt_in_smem<64, false, false, true>()};
@@ -1256,6 +1264,8 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   p.early_meta = (a.meta_settled && !fused) ? 1 : 0;
   p.timeline = reinterpret_cast<unsigned long long*>(a.timeline);
   p.spin_limit = a.spin_limit ? a.spin_limit : kSpinLimit;
+  // a settable limit exists for head_dim 128 with groups of at most 8 query heads, plain and fused step
+  const bool shortw = a.spin_limit != 0 && g.head_dim == 128 && g.q_heads / g.kv_heads <= 8 && a.q2 == nullptr;
   p.debug = a.debug;
   p.f = FusedArgs{};
   if (fused) {
@@ -1276,6 +1286,8 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   const bool g8 = p.G <= 8;
   if (a.q2 != nullptr) {   // the paired form (token and beacon queries in one pass); the caller has checked G <= 8
     e = g.head_dim == 128 ? launch_pipe<128, false, false, true>(p, s) : launch_pipe<64, false, false, true>(p, s);
+  } else if (shortw) {
+    e = fused ? launch_pipe<128, true, true, false, true>(p, s) : launch_pipe<128, true, false, false, true>(p, s);
   } else if (fused) {
     if (g.head_dim == 128) e = g8 ? launch_pipe<128, true, true>(p, s) : launch_pipe<128, false, true>(p, s);
     else e = g8 ? launch_pipe<64, true, true>(p, s) : launch_pipe<64, false, true>(p, s);

@@ -216,10 +216,14 @@ __device__ __forceinline__ bool elect_one() {   // true in exactly one lane of a
 __device__ __forceinline__ void mbar_arrive_cta(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// Bounded wait that also gives up as soon as another thread of the block has reported a failure.
-__device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity, volatile int* fail, uint32_t limit) {
-  if (limit < 1024) {   // a deliberately short limit (bc_mask_attn_set_wait_limit): non-blocking looks, then give up
-    for (uint32_t polls = 0; polls < limit; ++polls) {
+// Bounded wait that also gives up as soon as another thread of the block has reported a failure.  The
+// ordinary instantiation has a compile-time limit (with a run-time limit the polling loops cost a
+// third of the kernel's throughput); the settable limit of bc_mask_attn_set_wait_limit lives in an
+// instantiation of its own (SHORTW), where limits below 1024 poll with the non-suspending test_wait.
+template <bool SHORTW>
+__device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity, volatile int* fail, uint32_t limit_arg) {
+  if (SHORTW && limit_arg < 1024) {
+    for (uint32_t polls = 0; polls < limit_arg; ++polls) {
       uint32_t ok;
       asm volatile(
           "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -230,6 +234,7 @@ __device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity,
     }
     return false;
   }
+  const uint32_t limit = SHORTW ? limit_arg : kWaitLimit;
   for (uint32_t polls = 0; polls < limit; ++polls) {
     uint32_t ok;
     asm volatile(
@@ -262,6 +267,7 @@ __device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity,
 //   bar_s: completion t = S of tile t is ready (and every earlier product has finished)
 //   bar_p: the 128 row threads have stored P of tile t                bar_o: P V of a tile has completed
 //   bar_f: completion e = O of item e is final                       bar_e: the rows have read O of item e
+template <bool SHORTW>
 __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, const __grid_constant__ MaskMaps maps) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -347,7 +353,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
       // one lane polls, the warp takes its answer
       auto wait_all = [&](uint32_t bar, uint32_t parity) {
         int ok1 = 1;
-        if (lane == 0) ok1 = mbar_wait_or_fail(bar, parity, s_fail, a.wait_limit) ? 1 : 0;
+        if (lane == 0) ok1 = mbar_wait_or_fail<SHORTW>(bar, parity, s_fail, a.wait_limit) ? 1 : 0;
         return __shfl_sync(0xffffffffu, ok1, 0) != 0;
       };
       const uint32_t q_bytes = (uint32_t)(box_rows * kD * 2);
@@ -399,6 +405,21 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
           // everything the products below need besides P is waited for while the rows are busy
           ok = wait_all(bar_v, ph_v);
           if (ok) { ph_v ^= 1; ++v_got; }
+          if (ok) {
+            // A key tile that reaches past its segment has loaded rows that are not this sequence's (the
+            // next sequence's, or zeros past the end of the array).  Their scores are overwritten with -inf
+            // and their weights are exactly 0, but 0 * inf would still poison the second product: the V
+            // rows past the segment's end are cleared here, by this warp, before the product is issued
+            // (partial tiles only; the row threads' code is untouched).
+            const int kind = plan_kind(pl, n), k0 = plan_k0(pl, n, kind);
+            const int seg_len = kind == 0 ? td.P : (kind == 1 ? td.nb : td.T);
+            const int nvalid = min(max(seg_len - k0, 0), kTile);
+            if (nvalid < kTile) {
+              for (int idx = nvalid * 16 + lane; idx < kTile * 16; idx += 32) st_zero16(sV + swz(idx >> 4, idx & 15));
+              proxy_fence();   // the product reads shared memory through the asynchronous proxy
+              __syncwarp();
+            }
+          }
           if (ok && n == 0 && e > 0) ok = wait_all(bar_e, (e - 1) & 1u);       // the rows have read the last O
           if (ok && more) { ok = wait_all(bar_k, ph_k); if (ok) { ph_k ^= 1; ++k_got; } }   // the next K (and Q) has landed
           ok = ok && wait_all(bar_p, t & 1u);
@@ -438,11 +459,11 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
         __syncwarp();
         if (elect_one()) {   // the lane that issued the copies and the products
           int never = 0;
-          if (k_req > k_got) mbar_wait_or_fail(bar_k, ph_k, &never, kWaitLimit);
-          if (v_req > v_got) mbar_wait_or_fail(bar_v, ph_v, &never, kWaitLimit);
+          if (k_req > k_got) mbar_wait_or_fail<false>(bar_k, ph_k, &never, kWaitLimit);
+          if (v_req > v_got) mbar_wait_or_fail<false>(bar_v, ph_v, &never, kWaitLimit);
           if (products_issued) {
             umma_commit(bar_d);
-            mbar_wait_or_fail(bar_d, 0, &never, kWaitLimit);
+            mbar_wait_or_fail<false>(bar_d, 0, &never, kWaitLimit);
           }
         }
       }
@@ -477,7 +498,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
       float m_ref = -INFINITY, l_run = 0.f;
 
       for (int n = 0; n < pl.N; ++n, ++t) {
-        const bool ok = mbar_wait_or_fail(bar_s, t & 1u, s_fail, a.wait_limit);
+        const bool ok = mbar_wait_or_fail<SHORTW>(bar_s, t & 1u, s_fail, a.wait_limit);
         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
         tc_fence_after();
         const int kind = plan_kind(pl, n), k0 = plan_k0(pl, n, kind);
@@ -543,23 +564,6 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
             tmem_st32(tO + lane_base + cb * 32, u);
           }
         }
-        // A key tile that reaches past its segment has loaded rows that are not this sequence's (the next
-        // sequence's, or zeros past the end of the array).  Their scores were set to -inf above and their
-        // weights are exactly 0, but 0 * inf would still poison the second product: once the V tile has
-        // landed, the threads whose row index lies past the segment's end clear that key's V row.
-        {
-          const int seg_len = kind == 0 ? td.P : (kind == 1 ? td.nb : td.T);
-          const int nvalid = min(max(seg_len - k0, 0), kTile);
-          if (nvalid < kTile) {   // the same for the whole block
-            const bool okv = mbar_wait_or_fail(bar_v, t & 1u, s_fail, a.wait_limit);
-            if (!__all_sync(0xffffffffu, okv)) { failed = true; break; }
-            if (tid >= nvalid) {
-#pragma unroll
-              for (int ch = 0; ch < 16; ++ch) st_zero16(sV + swz(tid, ch));
-            }
-            proxy_fence();   // the product reads shared memory through the asynchronous proxy
-          }
-        }
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive_cta(bar_p);
@@ -570,7 +574,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
       const int nitem = item_of(r + 1);
       TileDesc ntd = {};
       if (nitem >= 0) ntd = a.tiles[nitem / Hkv];   // in flight during the wait below
-      const bool ok = mbar_wait_or_fail(bar_f, e & 1u, s_fail, a.wait_limit);
+      const bool ok = mbar_wait_or_fail<SHORTW>(bar_f, e & 1u, s_fail, a.wait_limit);
       if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       tc_fence_after();
       float o[kD];
@@ -741,7 +745,9 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
   a.scale_log2 = sm_scale * 1.4426950408889634f;
   a.wait_limit = g_mask_wait_limit ? g_mask_wait_limit : kWaitLimit;
   const int smem_bytes = 3 * kOperandBytes + 1024;
-  if (cudaFuncSetAttribute(k_mask_attn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return BC_ERR_CUDA;
+  const bool shortw = g_mask_wait_limit != 0;
+  if (cudaFuncSetAttribute(shortw ? k_mask_attn<true> : k_mask_attn<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
+    return BC_ERR_CUDA;
   if (!encode_tiled()) return BC_ERR_CUDA;
   MaskMaps maps;
   const void* dummy = ws;   // arrays that do not exist (no prompt, no beacons) get a map that is never used
@@ -755,7 +761,8 @@ bc_status bc_mask_attn_forward(int32_t n_seqs, int32_t q_heads, int32_t kv_heads
             map_3d(&maps.v_bea, beacon_v ? beacon_v : dummy, kv_heads, total_beacons, 1, kTile);
   if (!ok) return BC_ERR_CUDA;
   const int grid = a.n_items < 2 * sm_count() ? a.n_items : 2 * sm_count();   // two resident blocks per SM
-  k_mask_attn<<<grid, kThreads, smem_bytes, s>>>(a, maps);
+  if (shortw) k_mask_attn<true><<<grid, kThreads, smem_bytes, s>>>(a, maps);
+  else k_mask_attn<false><<<grid, kThreads, smem_bytes, s>>>(a, maps);
   return cudaGetLastError() == cudaSuccess ? BC_OK : BC_ERR_CUDA;
 }
 

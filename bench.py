@@ -924,7 +924,7 @@ def report_model(args):
     if args.model_ratio is not None:
         # one ratio, in a process of its own (see below): prints its row and nothing else
         import torch
-        from paper_2510_13797_b200.model_harness import ToyDecoder
+        from bench_model import ToyDecoder
         torch.cuda.set_device(0)
         c = args.model_ratio
         m = ToyDecoder(Bn, c, gen_len=reps * N + 128, device="cuda", paired=not args.no_pair)

@@ -22,7 +22,7 @@ import math
 
 import torch
 
-from . import binding as B
+from paper_2510_13797_b200 import binding as B
 
 
 class ToyDecoder:

@@ -46,16 +46,20 @@
  *          a launch of their own).  They touch only the cache's metadata and `slots`, read nothing
  *          an attention kernel writes, and end only once the kernel they overtook has ended, so
  *          everything enqueued behind them is ordered after both.
- *      (2) The attention kernels.  Before they wait for the kernel ahead they read only `slots` and
- *          metadata (lengths, page-table entries) that a bookkeeping kernel which has ENDED wrote;
- *          the queries, the extra entry, the pool rows, the outputs and the split-K scratch are
- *          touched after the wait.  An attention kernel that follows its step's bookkeeping kernel
- *          directly (bc_decode_step) reads nothing before the wait.
+ *      (2) The attention kernels.  Before they wait for the kernel ahead they read `slots`, their
+ *          inputs (q, the extra entry, beacon_q) and, of the cache, only what a kernel that has ENDED
+ *          wrote: metadata and pool rows other than the newest entries of a beacon or window segment.
+ *          The split-K scratch, the ticket counters and every output are touched after the wait.  An
+ *          attention kernel that follows its step's bookkeeping kernel directly (bc_decode_step)
+ *          reads that kernel's results only after a release/acquire handshake with it.
  *      (3) Kernels that release their dependents early: the attention kernels (once they have read
  *          the lengths they need) and the row-writing kernel of bc_append / bc_compress (at once).
- *    What this asks of the caller: `slots` must not be written by a kernel that releases its
- *    dependents early.  K/V rows, queries, outputs and the caller's own kernels keep plain stream
- *    order.
+ *    What this asks of the caller: `slots` and the input tensors of an attention call (q, extra_k,
+ *    extra_v, beacon_q) must not be written by a kernel that releases its dependents early.  Kernels
+ *    launched the ordinary way (any GEMM or element-wise kernel that produces q) never do; of this
+ *    library's kernels only an attention kernel's OUTPUT could be in that position, so do not pass
+ *    the output buffer of one attention call as the query buffer of the next call on the stream.
+ *    K/V rows, outputs and the caller's own kernels keep plain stream order.
  *
  * Store layout (owned by the library inside the caller's `pool` buffer)
  *    pool[layer][page][slot_in_page][K|V][kv_head][head_dim] bf16: one token's entry of one layer

@@ -491,13 +491,21 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   // for the whole grid as before.  The fused form goes on reading the rows' destinations (dst_row,
   // dst_pos); the next step's bookkeeping fills the other of two sets, so it may start early as well --
   // unless this launch did its own bookkeeping in block 0, whose flag word the next one would reuse.
-  if (!FUSED || !p.f.do_book) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // A fused step that started early lets its dependents go only once it has waited for the kernel ahead
+  // (see wait_for_kernel_ahead): its service warps write pool rows, and at most two row-writing launches
+  // may be alive at a time for the "settled" rule below to hold.
+  if (FUSED ? (!p.f.do_book && !early) : true) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // With early_meta the wait for the kernel ahead is still to come: every role below executes it before it
   // touches anything but `slots` and the metadata -- the pool rows of this step, q, the extra entry, the
   // partial buffers and tickets this launch shares with the one before it, and every output.  So the plan
   // above (three dependent trips to memory) and the producer's first page-table reads run under the
   // predecessor instead of after it.
-  auto wait_for_kernel_ahead = [&]() { if (early) asm volatile("griddepcontrol.wait;" ::: "memory"); };
+  auto wait_for_kernel_ahead = [&]() {
+    if (early) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      if (FUSED) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    }
+  };
   // The block that ran the bookkeeping starts late; it takes no tiles, or it would finish last.
   const int idle = (FUSED && p.f.do_book && gridDim.x > 1) ? 1 : 0;
   const int n_ctas = (int)gridDim.x - idle;
@@ -590,7 +598,11 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
         int len, tt, col;
         if (t < f_tp) { len = f_P; tt = t; col = 0; }
         else if (t < f_tpb) { len = f_nb; tt = t - f_tp; col = f_bcol; settled = t != f_tpb - 1; }
-        else { len = f_w; tt = t - f_tpb; col = f_wcol; settled = gt != s_cum[fi + 1] - 1; }
+        else {
+          // a fused step may run while the fused step before it still stores ITS new window entry, which
+          // can lie in the tile before the last one: there the last two window tiles are left alone
+          len = f_w; tt = t - f_tpb; col = f_wcol; settled = gt < s_cum[fi + 1] - (FUSED ? 2 : 1);
+        }
         p0 = tt << TS;
         nrows = max(min(T, len - p0), 0);
         if (FUSED && f_new && gt == s_cum[fi + 1] - 1) nrows -= 1;  // the new row comes from the input, not the pool
@@ -676,8 +688,16 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   }
 
   // ================================== consumer warps ===========================================
-  wait_for_kernel_ahead();
-  stamp(2);
+  // The consumers do not wait for the kernel ahead before they start either: they read the queries and
+  // the extra entry (inputs, which no kernel that releases its dependents early may write) and whatever
+  // settled tiles the producer has brought in, and they write nothing outside the block until a piece
+  // ends.  They wait before the first thing they share with the launch before them: the ticket
+  // counters, the partial buffers, the outputs.
+  bool cons_waited = !early;
+  auto consumers_wait = [&]() {
+    if (!cons_waited) { wait_for_kernel_ahead(); cons_waited = true; stamp(2); }
+  };
+  if (!early) stamp(2);
   stamp_val(8, ((unsigned long long)(g1 - g0) << 32) | (unsigned)seq0);
   const int kvh = warp % Hkv, grp = warp / Hkv;
   const int gq = lane >> 2, qd = lane & 3;  // fragment row and column-pair index
@@ -775,7 +795,10 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       // The final piece's last tile: look at the sequence's ticket counter now, while the tile is still
       // in flight.  If every other piece is there already, the merge after the tile starts at once (the
       // count cannot go back); if not, the counter is read again after the tile.
-      if (!PAIR && !has_next && !whole && t == tb - 1 && tid == 0) early_cnt = ld_acquire(p.a.tickets + i);
+      if (!PAIR && !has_next && !whole && t == tb - 1) {
+        consumers_wait();   // the counter is shared with the launch before this one
+        if (tid == 0) early_cnt = ld_acquire(p.a.tickets + i);
+      }
       bool patch = false;
       int patch_row = 0;
       uint4 patch_val = make_uint4(0u, 0u, 0u, 0u);
@@ -893,6 +916,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     }
 
     // ---- end of piece: merge the groups of each KV head in shared memory, then write -------------
+    consumers_wait();
     if (!has_next) stamp(4);
     l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
     if (!G_LE_8) { l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2); }

@@ -5,7 +5,7 @@ import pytest
 import torch
 
 from oracle.breadcrumbs_oracle import closed_form_length
-from paper_2510_13797_b200.model_harness import ToyDecoder
+from bench_model import ToyDecoder
 
 pytestmark = pytest.mark.gpu
 

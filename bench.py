@@ -57,8 +57,8 @@ def entries_beacon_query(P, t, c):
 # case of each ratio (--profile-case C: same bytes per launch and page size as mid-generation), for
 # the library version named here; see profiles/.  Slightly below 1: part of the stream stays in L2
 # from the previous step.  A different library version invalidates the figures (traffic: null).
-TRAFFIC_FOR_VERSION = 200
-TRAFFIC_OVER_ALGORITHMIC = {2: 0.996, 4: 0.980, 8: 0.960, 16: 0.943, 32: 0.979}
+TRAFFIC_FOR_VERSION = 210
+TRAFFIC_OVER_ALGORITHMIC = {2: 0.997, 4: 0.982, 8: 0.962, 16: 0.949, 32: 0.981}
 
 
 def traffic_per_launch(c, algorithmic_bytes):
@@ -248,8 +248,10 @@ class _Passes:
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
+        t0 = time.perf_counter()
         for _ in range(K):
             self.step_host()
+        self.host_enqueue_ms = (time.perf_counter() - t0) * 1e3   # what the calls cost the host thread (no synchronisation inside)
         self.cache.bc_host_outputs_ready()            # the last outputs' copies, before the closing event
         e1.record()
         torch.cuda.synchronize()
@@ -768,8 +770,59 @@ def report_depth(args):
         "largest_batch_rule": "floor(0.90 * free HBM / (pages per sequence at the end of the run * page bytes * 28 "
                               "layers)), page_size = c (16 for c = 1)",
     }
+    # Secondary timing: the same steps with layer = -1, one launch per call for all 28 layers (the layers of a
+    # real forward pass depend on one another, so this is the cache traffic alone, without the kernel boundaries).
+    Qs, Ks, Vs = (torch.stack([ins[l][0][x] for l in range(L)], dim=1).contiguous() for x in range(3))      # [ring, L, B, H, D]
+    BQs, BKs, BVs = (torch.stack([ins[l][1][x] for l in range(L)], dim=1).contiguous() for x in range(3))   # [2, L, B, H, D]
+    out_all = torch.empty((L,) + tuple(out.shape), dtype=out.dtype, device=dev)
+
+    def step_all():
+        t = state["t"]; j = t % ring
+        if (t + 1) % c == 0:
+            m = ((t + 1) // c) % 2
+            cache.bc_append(-1, slots, Ks[j], Vs[j])
+            if paired:
+                for l in range(L):
+                    cache.bc_decode_attn_pair(l, slots, Qs[j, l], out, BQs[m, l], out_b, w.sm_scale, BKs[m, l], BVs[m, l])
+            else:
+                cache.bc_decode_attn(-1, slots, Qs[j], out_all, w.sm_scale)
+                cache.bc_decode_attn(-1, slots, BQs[m], out_all, w.sm_scale, BKs[m], BVs[m])
+            cache.bc_compress(-1, slots, BKs[m], BVs[m])
+        else:
+            cache.bc_decode_step(-1, slots, Qs[j], Ks[j], Vs[j], out_all, w.sm_scale)
+        state["t"] = t + 1
+
+    graph2 = torch.cuda.CUDAGraph()
+    l0, t_save = cache.bc_kernel_launches(), state["t"]
+    with torch.cuda.graph(graph2, stream=s, capture_error_mode="thread_local"):
+        for _ in range(c):
+            step_all()
+    per_graph2 = cache.bc_kernel_launches() - l0
+    state["t"] = t_save
+    torch.cuda.current_stream().wait_stream(s)
+    graph2.replay(); state["t"] += c
+    torch.cuda.synchronize()
+    t_begin2 = state["t"]
+    e0, e1 = _event_pair(torch)
+    e0.record()
+    for _ in range(K // c):
+        graph2.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    state["t"] += K
+    ms2 = e0.elapsed_time(e1)
+    code, slot, call = cache.bc_poll_error()
+    assert code == 0, (code, slot, call)
+    reg2 = sum(entries_attended(P, n, c) for n in range(t_begin2 + 1, t_begin2 + K + 1))
+    bea2 = 0 if paired else sum(entries_beacon_query(P, n, c) for n in range(t_begin2 + 1, t_begin2 + K + 1) if n % c == 0)
+    kv2 = (reg2 + bea2) * E * Bn * L
+    line["all_layers_per_launch"] = {
+        "what": "the same steps through layer = -1: a regular step is bc_decode_step(-1) = one bookkeeping kernel and ONE attention "
+                "launch whose grid walks the 28 layers; a window fill is bc_append(-1), the per-layer paired attention and bc_compress(-1)",
+        "t_window": [t_begin2, t_begin2 + K], "ms_per_step": ms2 / K, "kv_gbs": kv2 / (ms2 * 1e-3) / 1e9,
+        "pct_of_8tbs": 100 * kv2 / (ms2 * 1e-3) / 8e12, "gpu_launches": int(per_graph2 * (K // c))}
     # demonstration at c = 8: allocate the pool for that many sequences and decode a window with all of them
-    del cache, ins, graph
+    del cache, ins, graph, graph2, Qs, Ks, Vs, BQs, BKs, BVs, out_all
     torch.cuda.empty_cache()
     n_big = capacity["8"]
     big = B.Cache(L, w.kv_heads, w.q_heads, w.head_dim, c, ps, max_seqs=n_big, num_pages=n_big * pps,
@@ -927,7 +980,7 @@ def report_model(args):
         from bench_model import ToyDecoder
         torch.cuda.set_device(0)
         c = args.model_ratio
-        m = ToyDecoder(Bn, c, gen_len=reps * N + 128, device="cuda", paired=not args.no_pair)
+        m = ToyDecoder(Bn, c, gen_len=reps * N + 128, device="cuda", paired=not args.no_pair, lib_rope=not args.torch_rope)
         m.capture()
         torch.cuda.synchronize()
         times = []
@@ -952,6 +1005,8 @@ def report_model(args):
         cmd = [sys.executable, os.path.abspath(__file__), "--workload", "model", "--model-ratio", str(c), "--steps", str(args.steps)]
         if args.no_pair:
             cmd.append("--no-pair")
+        if args.torch_rope:
+            cmd.append("--torch-rope")
         child = subprocess.run(cmd, capture_output=True, text=True)
         if child.returncode != 0:
             sys.stderr.write(child.stderr[-2000:])
@@ -963,6 +1018,8 @@ def report_model(args):
     print(json.dumps({"workload": f"model: random-weight decoder of the 1.5B shape, batch {Bn}, prompt 512, {N} generated tokens "
                                   "per sequence, one CUDA graph per token step and per beacon step"
                                   + ("" if args.no_pair else "; the beacon is encoded in the same 2-token pass as the token that fills the window"),
+                      "rope_and_qkv_split": "PyTorch operators" if args.torch_rope else
+                      "bc_rope_split / bc_rope_decode_step (a token step: the rotation kernel, then one kernel that appends and attends)",
                       "paper_latency_table_qwen_sr": {"2": 1.990, "4": 1.546, "8": 1.593, "16": 1.646, "32": 1.468},
                       "rows": rows}))
 
@@ -1016,6 +1073,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=32)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--torch-rope", action="store_true",
+                    help="--workload model: rotary embedding and QKV split with PyTorch operators instead of the library's kernel")
     ap.add_argument("--no-pair", action="store_true", help="beacon steps as a second attention pass instead of bc_decode_attn_pair")
     ap.add_argument("--pair", action="store_true", help="ragged workload: pair the beacon steps too (off by default there)")
     ap.add_argument("--fused", action="store_true", help="--timeline: regular steps through bc_decode_step")
@@ -1108,6 +1167,7 @@ def main():
             "graph": f"one CUDA graph of the {K} timed steps ({regular} regular, {fills} window-filling), replayed once under the events",
             "ms_per_step_p50_p99_over_windows": _percentiles(r.window_step_ms),
             "e2e_tokens_per_s": world * w.batch * K / (h_ms * 1e-3),
+            "e2e_us_per_step": 1e3 * h_ms / K, "e2e_host_enqueue_us_per_step": 1e3 * r.host_enqueue_ms / K,
             "plain_launch_ms_per_step": plain_ms / Kp,
             "kv_gbs_step": (reg + bea) / (ms * 1e-3) / 1e9,
             "step_frac_of_peak": (reg + bea) / (ms * 1e-3) / 1e9 / peak,

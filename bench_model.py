@@ -5,8 +5,10 @@ What is measured with it: the time to generate N tokens per sequence with the un
 timing figure (its latency table: generation latency relative to the uncompressed teacher).
 
 Only the cache side (bc_append, bc_decode_attn, bc_compress) is this repository's product.  The
-rest of the forward pass -- embeddings, RMSNorm, the QKV / output / MLP projections, rotary
-embedding, the LM head and greedy sampling -- are plain PyTorch operators standing in for a model
+rest of the forward pass -- embeddings, RMSNorm, the QKV / output / MLP projections, the LM head
+and greedy sampling -- are plain PyTorch operators standing in for a model; the rotary embedding and the
+split of the packed QKV rows are the library's kernel (bc_rope_split, bc_rope_decode_step) unless
+lib_rope=False, which puts the PyTorch operators back for comparison
 (random weights: the token stream is meaningless, the shapes and the data flow are real).  Every
 sampled token is fed back, and when a window fills, the beacon token's forward pass runs through
 the same layers: its query attends with its own K/V as the extra entry, then the window is evicted
@@ -27,8 +29,9 @@ from paper_2510_13797_b200 import binding as B
 
 class ToyDecoder:
     def __init__(self, batch, c, gen_len, prompt_len=512, layers=28, hidden=1536, q_heads=12, kv_heads=2, head_dim=128,
-                 mlp=8960, vocab=151936, device="cuda", seed=0, weights=None, paired=True):
+                 mlp=8960, vocab=151936, device="cuda", seed=0, weights=None, paired=True, lib_rope=True, theta=1e6):
         self.B, self.c, self.L, self.H = batch, c, layers, hidden
+        self.lib_rope, self.theta = lib_rope, theta
         self.paired = paired    # True: the beacon is encoded together with the token that fills the window
                                 # (one 2-token forward pass, bc_decode_attn_pair), False: in a forward pass of its own
         self.Hq, self.Hkv, self.D, self.V = q_heads, kv_heads, head_dim, vocab
@@ -62,7 +65,13 @@ class ToyDecoder:
         self.pos = torch.full((1,), prompt_len, dtype=torch.int64, device=self.dev)
         self.attn_out = self.cache.new_out(batch)
         self.attn_out2 = self.cache.new_out(2 * batch)         # the paired step: token rows, then beacon rows
-        self.inv_freq = 1.0 / (10000.0 ** (torch.arange(0, head_dim, 2, device=self.dev, dtype=torch.float32) / head_dim))
+        self.inv_freq = 1.0 / (theta ** (torch.arange(0, head_dim, 2, device=self.dev, dtype=torch.float32) / head_dim))
+        # the library's rotation takes one position per row: rows [0, B) at pos, rows [B, 2B) (the beacons of a paired step) at pos + 1
+        self.posv = torch.cat((torch.full((batch,), prompt_len, dtype=torch.int32, device=self.dev),
+                               torch.full((batch,), prompt_len + 1, dtype=torch.int32, device=self.dev)))
+        self.q2 = self.cache.new_out(2 * batch)
+        self.k2 = torch.empty((2 * batch, kv_heads, head_dim), dtype=torch.bfloat16, device=self.dev)
+        self.v2 = torch.empty_like(self.k2)
         self.scale = 1.0 / math.sqrt(head_dim)
         self.graph_tok = self.graph_bea = None
 
@@ -78,14 +87,32 @@ class ToyDecoder:
         x1, x2 = x.float()[..., 0::2], x.float()[..., 1::2]
         return torch.stack((x1 * cos - x2 * sin, x1 * sin + x2 * cos), dim=-1).flatten(-2).to(torch.bfloat16)
 
+    def _split(self, qkv, offset=None):
+        """Rotated q and k and v of the packed rows: the library's kernel, or the PyTorch operators."""
+        Hq, Hkv, D = self.Hq, self.Hkv, self.D
+        n = qkv.shape[0]
+        if self.lib_rope:
+            q, k, v = self.q2[:n], self.k2[:n], self.v2[:n]
+            self.cache.bc_rope_split(qkv, self.posv[:n], self.theta, q, k, v)
+            return q, k, v
+        q = self._rope(qkv[:, :Hq * D].view(-1, Hq, D), offset).contiguous()
+        k = self._rope(qkv[:, Hq * D:(Hq + Hkv) * D].view(-1, Hkv, D), offset).contiguous()
+        v = qkv[:, (Hq + Hkv) * D:].view(-1, Hkv, D).contiguous()
+        return q, k, v
+
     def _forward(self, ids, beacon):
         h = self.emb[ids]
         Hq, Hkv, D = self.Hq, self.Hkv, self.D
         for l in range(self.L):
             qkv = self._norm(h) @ self.wqkv[l]
-            q = self._rope(qkv[:, :Hq * D].view(-1, Hq, D)).contiguous()
-            k = self._rope(qkv[:, Hq * D:(Hq + Hkv) * D].view(-1, Hkv, D)).contiguous()
-            v = qkv[:, (Hq + Hkv) * D:].view(-1, Hkv, D).contiguous()
+            if self.lib_rope and not beacon:    # rotation, then the append and the attention in one kernel
+                self.cache.bc_rope_decode_step(l, self.slots, qkv, self.posv[:self.B], self.theta, self.attn_out, self.scale)
+                h = h + self.attn_out.view(-1, Hq * D) @ self.wo[l]
+                gu = self._norm(h) @ self.wgu[l]
+                gate, up = gu.chunk(2, dim=-1)
+                h = h + (torch.nn.functional.silu(gate) * up) @ self.wdown[l]
+                continue
+            q, k, v = self._split(qkv)
             if beacon:      # the beacon's query sees the cache plus its own entry; then the window goes
                 self.cache.bc_decode_attn(l, self.slots, q, self.attn_out, self.scale, k, v)
                 self.cache.bc_compress(l, self.slots, k, v)
@@ -108,9 +135,7 @@ class ToyDecoder:
         offset = torch.cat((torch.zeros(Bn, device=self.dev), torch.ones(Bn, device=self.dev)))
         for l in range(self.L):
             qkv = self._norm(h) @ self.wqkv[l]
-            q = self._rope(qkv[:, :Hq * D].view(-1, Hq, D), offset).contiguous()
-            k = self._rope(qkv[:, Hq * D:(Hq + Hkv) * D].view(-1, Hkv, D), offset).contiguous()
-            v = qkv[:, (Hq + Hkv) * D:].view(-1, Hkv, D).contiguous()
+            q, k, v = self._split(qkv, offset)
             self.cache.bc_append(l, self.slots, k[:Bn], v[:Bn])
             self.cache.bc_decode_attn_pair(l, self.slots, q[:Bn], self.attn_out2[:Bn], q[Bn:], self.attn_out2[Bn:], self.scale,
                                            k[Bn:], v[Bn:])
@@ -124,16 +149,16 @@ class ToyDecoder:
     def _fill_step(self):
         h = self._forward_pair()
         self.tok.copy_(torch.argmax(self._norm(h) @ self.head, dim=-1))
-        self.pos.add_(2)
+        self.pos.add_(2); self.posv.add_(2)
 
     def _token_step(self):
         h = self._forward(self.tok, beacon=False)
         self.tok.copy_(torch.argmax(self._norm(h) @ self.head, dim=-1))
-        self.pos.add_(1)
+        self.pos.add_(1); self.posv.add_(1)
 
     def _beacon_step(self):
         self._forward(torch.full_like(self.tok, self.V), beacon=True)   # its logits are not needed
-        self.pos.add_(1)
+        self.pos.add_(1); self.posv.add_(1)
 
     # -- generation ---------------------------------------------------------------------------------
     def capture(self):

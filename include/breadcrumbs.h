@@ -32,11 +32,19 @@
  *    its layer-0 call, bc_compress allocates the beacon slot on its layer-0 call and evicts the
  *    window on its call for the last layer.  For one step, call the layers in ascending order
  *    with the same `slots`; anything else returns BC_ERR_ORDER.  bc_prefill, bc_append,
- *    bc_decode_attn and bc_compress also take layer = BC_ALL_LAYERS (-1): every per-layer tensor
- *    of the call (k, v, q, out, extra_k, extra_v, beacon_k, beacon_v) then carries a leading
- *    [layers] dimension and the call runs layer 0 .. layers - 1 in that order, one launch sequence
- *    per layer (a forward pass computes layer l + 1's inputs from layer l's output, so this form
- *    serves replays and measurements, not a model).
+ *    bc_decode_attn, bc_decode_step and bc_compress also take layer = BC_ALL_LAYERS (-1): every
+ *    per-layer tensor of the call (k, v, q, out, extra_k, extra_v, beacon_k, beacon_v) then carries
+ *    a leading [layers] dimension and the call covers layer 0 .. layers - 1; results are those of
+ *    the per-layer calls in ascending order (a forward pass computes layer l + 1's inputs from
+ *    layer l's output, so this form serves replays and measurements, not a model).  The call is
+ *    legal where the layer-0 call would be (else BC_ERR_ORDER) and leaves the order at layer 0.
+ *    Launches: bc_decode_attn and bc_decode_step run ONE attention kernel whose grid's second
+ *    dimension is the layer (the blocks of a layer are dispatched as those of the layer before
+ *    retire; every layer has its own split-K counters and partial buffers in the workspace), after
+ *    the one bookkeeping kernel in the case of bc_decode_step; bc_append and bc_compress run their
+ *    bookkeeping kernel and ONE kernel that writes the rows of every layer (bc_compress allocates
+ *    the beacon slot and evicts the window in the same bookkeeping launch).  bc_prefill, the
+ *    static entry point and a cache with BC_FLAG_ATTN_REFERENCE run one launch sequence per layer.
  *  - A batch must not name the same slot twice.
  *  - Overlap (programmatic stream serialisation).  Three kinds of kernel of this library may begin
  *    before the kernel enqueued just ahead of them on `stream` has ended, provided that kernel
@@ -248,9 +256,38 @@ BC_API bc_status bc_decode_attn_pair(bc_cache* cache, int32_t layer, const int32
  * attention kernel takes the new entries from the input tensors where it needs them, and one of
  * its warps stores them to the pool for later steps.
  * q [n, q_heads, head_dim], k, v [n, kv_heads, head_dim], out like q; n <= 512.  With
- * BC_FLAG_ATTN_REFERENCE the call simply issues the two separate calls. */
+ * BC_FLAG_ATTN_REFERENCE the call simply issues the two separate calls.  layer = BC_ALL_LAYERS:
+ * see the layer convention at the top of this file. */
 BC_API bc_status bc_decode_step(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n, const void* q,
                                 const void* k, const void* v, void* out, float sm_scale, void* stream);
+
+/* Rotary position embedding and split of a packed QKV projection: what sits between a decoder
+ * layer's QKV GEMM and the cache calls.  (The paper leaves the position encoding to the model,
+ * Section 2: attention is unchanged; its models use rotary embeddings.)  Row i of qkv is
+ * [q heads | k heads | v heads], (q_heads + 2 kv_heads) * head_dim bf16 values, of a token (or beacon)
+ * at position positions[i].  Every q and k head is rotated: coordinate j < head_dim/2 is paired
+ * with coordinate j + head_dim/2 (the half-split pairing of the paper's models) and the pair is
+ * turned by positions[i] * theta^(-2j/head_dim) radians; v is copied.  Angles are evaluated in double
+ * precision, the rotation in fp32, results rounded to nearest-even bf16.
+ * qkv: device, [n, (q_heads + 2 kv_heads) * head_dim] bf16, 16-byte aligned; positions: device int32[n],
+ * >= 0; theta > 1 (10000 in RoFormer, 1e6 in Qwen2.5); q_out [n, q_heads, head_dim], k_out, v_out
+ * [n, kv_heads, head_dim]: device bf16, 16-byte aligned, caller-owned, must not overlap qkv.  They are
+ * laid out as bc_append / bc_decode_attn / bc_decode_step / bc_compress take them.  The head counts and
+ * head_dim are the cache's; the call touches no cache state, records no error and may be issued at any
+ * point of the layer order.  One kernel launch; asynchronous on `stream`; it completes before any
+ * later kernel of the stream starts (it takes no part in the overlap described above).
+ * BC_ERR_INVALID_ARG: a null or misaligned pointer, n <= 0, theta <= 1. */
+BC_API bc_status bc_rope_split(bc_cache* cache, const void* qkv, const int32_t* positions, int32_t n, float theta,
+                               void* q_out, void* k_out, void* v_out, void* stream);
+
+/* bc_rope_split followed by bc_decode_step on its results: one decode step of one layer straight from
+ * the packed QKV projection (two launches: the rotation, then the attention kernel that also appends
+ * the new entries; plus the one-block bookkeeping kernel on layer 0).  The rotated q, k and v pass
+ * through a staging buffer the cache owns (one per cache: the next call of this entry point on the same
+ * stream reuses it, which stream order makes safe).  Arguments as for the two calls; n <= 512 and
+ * n <= max_seqs.  Errors: those of bc_decode_step and bc_rope_split. */
+BC_API bc_status bc_rope_decode_step(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n, const void* qkv,
+                                     const int32_t* positions, float theta, void* out, float sm_scale, void* stream);
 
 /* Limits of bc_decode_attn_static. */
 #define BC_STATIC_MAX_BATCH 128   /* sequences per call */

@@ -84,6 +84,8 @@ SYMBOLS = {
     "bc_profile_enable": (_I32, [_P, _I32]),
     "bc_profile_read": (_I32, [_P, C.POINTER(_I32), C.POINTER(_F)]),
     "bc_probe_read_stream": (_I32, [_P, C.c_size_t, _P]),
+    "bc_rope_split": (_I32, [_P, _P, _P, _I32, _F, _P, _P, _P, _P]),
+    "bc_rope_decode_step": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _F, _P]),
     "bc_kernel_launches": (_I64, [_P]),
     "bc_last_cuda_error": (_I32, [_P]),
     "bc_status_string": (C.c_char_p, [_I32]),
@@ -187,6 +189,16 @@ class Cache:
         """bc_append(k, v) + bc_decode_attn(q) in one launch."""
         _check(lib().bc_decode_step(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(k), _ptr(v), _ptr(out),
                                     sm_scale, _stream(stream)), "bc_decode_step")
+
+    def bc_rope_split(self, qkv, positions, theta, q_out, k_out, v_out, stream=None):
+        """Rotary embedding of the q and k heads of a packed QKV projection, split into the three arrays the cache calls take."""
+        _check(lib().bc_rope_split(self.handle, _ptr(qkv), _ptr(positions), positions.numel(), theta, _ptr(q_out), _ptr(k_out),
+                                   _ptr(v_out), _stream(stream)), "bc_rope_split")
+
+    def bc_rope_decode_step(self, layer, slots, qkv, positions, theta, out, sm_scale, stream=None):
+        """bc_rope_split + bc_decode_step: a layer's decode step straight from the packed QKV projection."""
+        _check(lib().bc_rope_decode_step(self.handle, layer, _ptr(slots), slots.numel(), _ptr(qkv), _ptr(positions), theta,
+                                         _ptr(out), sm_scale, _stream(stream)), "bc_rope_decode_step")
 
     def bc_decode_attn_static(self, layer, slots, q, out, sm_scale, extra_k=None, extra_v=None, stream=None):
         """bc_decode_attn with the split-K scratch taken from the array built into the library, for callers

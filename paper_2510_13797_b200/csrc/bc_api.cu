@@ -34,7 +34,7 @@ MetaLayout meta_layout(const bc_config& c) {
 
 struct WorkLayout {
   size_t append_row[2], append_pos[2], plan[2], compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[4],
-      stage_out[2], stage_out2[2],
+      stage_out[2], stage_out2[2], rope_stage,
       total;
 };
 WorkLayout work_layout(const bc_config& c) {
@@ -48,20 +48,25 @@ WorkLayout work_layout(const bc_config& c) {
   for (int b = 0; b < 2; ++b) { l.append_row[b] = take(seq); l.append_pos[b] = take(seq); l.plan[b] = take(BC_PLAN_INTS * 4); }
   l.compress_row = take(seq); l.compress_pos = take(seq);
   l.restore_ok = take(seq); l.restore_bea = take(seq + 4);
-  l.tickets = take(BC_MAX_ATTN_BATCH * 4);
+  // A call with layer = BC_ALL_LAYERS is one launch whose blocks work on several layers at a time: every layer
+  // has its own ticket counters and its own partial buffers of BC_MAX_ATTN_CTAS + max_n pieces.
+  const size_t max_n = c.max_seqs < BC_MAX_ATTN_BATCH ? c.max_seqs : BC_MAX_ATTN_BATCH;
+  const size_t layered = (size_t)c.layers * (BC_MAX_ATTN_CTAS + max_n);
+  const size_t pieces1 = layered > pieces ? layered : pieces;
+  l.tickets = take((size_t)BC_MAX_ATTN_BATCH * 4 * c.layers);
   l.book_flag = take(4);
-  l.part_ml = take(pieces * c.q_heads * 2 * 4);
-  l.part_o = take(pieces * c.q_heads * c.head_dim * 4);
+  l.part_ml = take(pieces1 * c.q_heads * 2 * 4);
+  l.part_o = take(pieces1 * c.q_heads * c.head_dim * 4);
   l.part_ml2 = take(pieces * c.q_heads * 2 * 4);            // the beacons' partials of the paired form
   l.part_o2 = take(pieces * c.q_heads * c.head_dim * 4);
   // host-buffer entry points: a ring of four input staging buffers, each k | v | q packed for the largest
   // batch a call can carry (a step that fills a window takes two of them, token and beacon inputs)
-  const size_t max_n = c.max_seqs < BC_MAX_ATTN_BATCH ? c.max_seqs : BC_MAX_ATTN_BATCH;
   for (int b = 0; b < 4; ++b) l.stage_in[b] = take(max_n * (c.q_heads + 2 * c.kv_heads) * c.head_dim * 2);
   for (int b = 0; b < 2; ++b) {   // two sets of output staging (a set: token output, beacon output)
     l.stage_out[b] = take(max_n * c.q_heads * c.head_dim * 4);
     l.stage_out2[b] = take(max_n * c.q_heads * c.head_dim * 4);
   }
+  l.rope_stage = take(max_n * (c.q_heads + 2 * c.kv_heads) * c.head_dim * 2);   // bc_rope_decode_step: q | k | v
   l.total = o;
   return l;
 }
@@ -178,8 +183,20 @@ bc_status check_batch(bc_cache* c, int layer, const int32_t* slots, int n) {
 
 bc_status attn_impl(bc_cache* c, int layer, const int32_t* slots, int n, const void* q, void* out, float sm_scale,
                     const void* extra_k, const void* extra_v, cudaStream_t s, const BcFusedAppend* fused = nullptr,
-                    const void* q2 = nullptr, void* out2 = nullptr) {
+                    const void* q2 = nullptr, void* out2 = nullptr, int layers = 1) {
   BcAttnArgs a;
+  if (layers > 1) {   // all layers in one launch: q, out, extra (or new) rows are [layers][n][...] arrays
+    const size_t max_n = c->cfg.max_seqs < BC_MAX_ATTN_BATCH ? c->cfg.max_seqs : BC_MAX_ATTN_BATCH;
+    const size_t pieces = BC_MAX_ATTN_CTAS + max_n;
+    a.layers = layers;
+    a.ls_pool = c->geom.layer_bytes;
+    a.ls_q = (int64_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
+    a.ls_out = (c->cfg.flags & BC_FLAG_OUT_F32) ? a.ls_q * 2 : a.ls_q;
+    a.ls_kv = (int64_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+    a.ls_part_o = (int64_t)pieces * c->cfg.q_heads * c->cfg.head_dim * 4;
+    a.ls_part_ml = (int64_t)pieces * c->cfg.q_heads * 2 * 4;
+    a.ls_tickets = BC_MAX_ATTN_BATCH;
+  }
   if (q2) {   // the paired form
     a.q2 = q2; a.out2 = out2;
     a.part_o2 = work_ptr<float>(c, c->wl.part_o2);
@@ -233,7 +250,7 @@ bc_status append_book_only(bc_cache* c, const int32_t* slots, int n, cudaStream_
 
 // The attention half of bc_decode_step: the step's append bookkeeping (layer 0) has been launched.
 bc_status decode_step_attn(bc_cache* c, int layer, const int32_t* slots, int n, const void* q, const void* k, const void* v,
-                           void* out, float sm_scale, cudaStream_t s) {
+                           void* out, float sm_scale, cudaStream_t s, int layers = 1) {
   BcFusedAppend f;
   f.new_k = k; f.new_v = v;
   f.dst_row = work_ptr<int32_t>(c, c->wl.append_row[c->append_set]);
@@ -244,9 +261,9 @@ bc_status decode_step_attn(bc_cache* c, int layer, const int32_t* slots, int n, 
   f.do_book = 0;
   f.call = c->calls;
   f.epoch = step_epoch(c->calls);
-  const bc_status st = attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s, &f);
+  const bc_status st = attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s, &f, nullptr, nullptr, layers);
   if (st) return st;
-  c->append_next_layer = (layer + 1) % c->cfg.layers;
+  c->append_next_layer = (layer + layers) % c->cfg.layers;
   return BC_OK;
 }
 }  // namespace
@@ -314,7 +331,7 @@ namespace {
 bc_status flush_pending(bc_cache* c);   // defined with the host-buffer entry points below
 }
 
-int32_t bc_version(void) { return 200; }
+int32_t bc_version(void) { return 210; }
 
 const char* bc_status_string(bc_status s) {
   switch (s) {
@@ -377,7 +394,7 @@ bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* wo
   cudaError_t e = cudaGetDevice(&c->device);
   if (e == cudaSuccess) e = bc_attn_setup(&c->sm_count);
   if (e == cudaSuccess) e = bc_launch_init(c->meta, (cudaStream_t)stream);
-  if (e == cudaSuccess) e = cudaMemsetAsync(c->work + c->wl.tickets, 0, BC_MAX_ATTN_BATCH * 4, (cudaStream_t)stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->work + c->wl.tickets, 0, (size_t)BC_MAX_ATTN_BATCH * 4 * c->cfg.layers, (cudaStream_t)stream);
   if (e == cudaSuccess) e = cudaMemsetAsync(c->work + c->wl.book_flag, 0, 4, (cudaStream_t)stream);
   if (e != cudaSuccess) { delete c; return BC_ERR_CUDA; }
   c->launches += 1;
@@ -460,12 +477,19 @@ bc_status bc_restore(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n
 bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* k, const void* v,
                     void* stream) {
   if (c && layer == BC_ALL_LAYERS) {
-    if (n <= 0) return BC_ERR_INVALID_ARG;
-    const size_t b = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
-    for (int l = 0; l < c->cfg.layers; ++l) {
-      const bc_status st = bc_append(c, l, slots, n, layer_slice(k, l, b), layer_slice(v, l, b), stream);
-      if (st) return st;
-    }
+    // the bookkeeping kernel, then ONE launch that writes the rows of every layer (same row and position in each)
+    bc_status st = check_batch(c, 0, slots, n);
+    if (st) return st;
+    if (!k || !v || !aligned16(k) || !aligned16(v)) return BC_ERR_INVALID_ARG;
+    if (c->append_next_layer != 0) return BC_ERR_ORDER;
+    cudaStream_t s = (cudaStream_t)stream;
+    st = append_book_only(c, slots, n, s);
+    if (st) return st;
+    BC_CUDA(c, bc_launch_write_rows(c->meta, c->geom, layer_base(c, 0), work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
+                                    work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), k, v, n, s, c->cfg.layers,
+                                    (long long)c->geom.layer_bytes, (long long)n * c->cfg.kv_heads * c->cfg.head_dim * 2));
+    c->launches += 1;
+    c->meta_unsettled = false;
     return BC_OK;
   }
   bc_status st = check_batch(c, layer, slots, n);
@@ -495,6 +519,17 @@ bc_status bc_append(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n,
 
 bc_status bc_decode_attn(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, void* out,
                          float sm_scale, const void* extra_k, const void* extra_v, void* stream) {
+  if (c && layer == BC_ALL_LAYERS && c->cfg.layers > 1 && !(c->cfg.flags & BC_FLAG_ATTN_REFERENCE)) {
+    // one launch: the grid's second dimension walks the layers
+    bc_status st = check_batch(c, 0, slots, n);
+    if (st) return st;
+    if (n > BC_MAX_ATTN_BATCH) return BC_ERR_INVALID_ARG;
+    if (!q || !out || !aligned16(q) || !aligned16(out)) return BC_ERR_INVALID_ARG;
+    if ((extra_k == nullptr) != (extra_v == nullptr)) return BC_ERR_INVALID_ARG;
+    if (extra_k && (!aligned16(extra_k) || !aligned16(extra_v))) return BC_ERR_INVALID_ARG;
+    return attn_impl(c, 0, slots, n, q, out, sm_scale, extra_k, extra_v, (cudaStream_t)stream, nullptr, nullptr, nullptr,
+                     c->cfg.layers);
+  }
   if (c && layer == BC_ALL_LAYERS) {
     if (n <= 0) return BC_ERR_INVALID_ARG;
     const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
@@ -537,12 +572,31 @@ bc_status bc_decode_attn_pair(bc_cache* c, int32_t layer, const int32_t* slots, 
 
 bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, const void* k,
                          const void* v, void* out, float sm_scale, void* stream) {
+  const bool all = c && layer == BC_ALL_LAYERS;
+  if (all) layer = 0;
   bc_status st = check_batch(c, layer, slots, n);
   if (st) return st;
   if (n > BC_MAX_ATTN_BATCH) return BC_ERR_INVALID_ARG;
   if (!q || !k || !v || !out || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BC_ERR_INVALID_ARG;
   if (layer != c->append_next_layer) return BC_ERR_ORDER;
   cudaStream_t s = (cudaStream_t)stream;
+  if (all && c->cfg.layers > 1) {
+    const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+    const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
+    if (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) {   // layer by layer
+      for (int l = 0; l < c->cfg.layers; ++l) {
+        st = bc_decode_step(c, l, slots, n, layer_slice(q, l, qb), layer_slice(k, l, kb), layer_slice(v, l, kb),
+                            layer_slice(out, l, ob), sm_scale, stream);
+        if (st) return st;
+      }
+      return BC_OK;
+    }
+    // the bookkeeping kernel, then ONE attention launch whose grid walks the layers: each layer's blocks take
+    // that layer's new entries from the [layers][n] inputs and store them to that layer's pool
+    st = append_book_only(c, slots, n, s, true);
+    if (st) return st;
+    return decode_step_attn(c, 0, slots, n, q, k, v, out, sm_scale, s, c->cfg.layers);
+  }
   if (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) {   // the debugging kernel has no fused form
     st = bc_append(c, layer, slots, n, k, v, stream);
     if (st) return st;
@@ -560,15 +614,49 @@ bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32
   return decode_step_attn(c, layer, slots, n, q, k, v, out, sm_scale, s);
 }
 
+bc_status bc_rope_split(bc_cache* c, const void* qkv, const int32_t* positions, int32_t n, float theta, void* q_out,
+                        void* k_out, void* v_out, void* stream) {
+  if (!c || !qkv || !positions || !q_out || !k_out || !v_out || n <= 0 || !(theta > 1.f)) return BC_ERR_INVALID_ARG;
+  if (!aligned16(qkv) || !aligned16(q_out) || !aligned16(k_out) || !aligned16(v_out)) return BC_ERR_INVALID_ARG;
+  BC_CUDA(c, bc_launch_rope_split(qkv, positions, n, c->cfg.q_heads, c->cfg.kv_heads, c->cfg.head_dim, (double)theta, q_out,
+                                  k_out, v_out, (cudaStream_t)stream));
+  c->launches += 1;
+  c->meta_unsettled = false;   // an ordinarily launched kernel: it starts after everything before it has ended
+  return BC_OK;
+}
+
+bc_status bc_rope_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* qkv,
+                              const int32_t* positions, float theta, void* out, float sm_scale, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (n > BC_MAX_ATTN_BATCH) return BC_ERR_INVALID_ARG;
+  if (layer != c->append_next_layer) return BC_ERR_ORDER;
+  uint8_t* q = work_ptr<uint8_t>(c, c->wl.rope_stage);
+  uint8_t* k = q + (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
+  uint8_t* v = k + (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
+  st = bc_rope_split(c, qkv, positions, n, theta, q, k, v, stream);
+  if (st) return st;
+  return bc_decode_step(c, layer, slots, n, q, k, v, out, sm_scale, stream);
+}
+
 bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* bk, const void* bv,
                       void* stream) {
   if (c && layer == BC_ALL_LAYERS) {
-    if (n <= 0) return BC_ERR_INVALID_ARG;
-    const size_t b = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
-    for (int l = 0; l < c->cfg.layers; ++l) {
-      const bc_status st = bc_compress(c, l, slots, n, layer_slice(bk, l, b), layer_slice(bv, l, b), stream);
-      if (st) return st;
-    }
+    // one bookkeeping launch (allocate the beacon slot and evict the window at once: the beacon rows do not
+    // depend on the eviction), then ONE launch that writes the beacon rows of every layer
+    bc_status st = check_batch(c, 0, slots, n);
+    if (st) return st;
+    if (!bk || !bv || !aligned16(bk) || !aligned16(bv)) return BC_ERR_INVALID_ARG;
+    if (c->compress_next_layer != 0) return BC_ERR_ORDER;
+    cudaStream_t s = (cudaStream_t)stream;
+    int32_t* row = work_ptr<int32_t>(c, c->wl.compress_row);
+    int32_t* pos = work_ptr<int32_t>(c, c->wl.compress_pos);
+    ++c->calls;
+    BC_CUDA(c, bc_launch_compress_book(c->meta, slots, n, c->calls, row, pos, 3, c->geom, layer_base(c, 0), nullptr, nullptr, s));
+    BC_CUDA(c, bc_launch_write_rows(c->meta, c->geom, layer_base(c, 0), row, pos, bk, bv, n, s, c->cfg.layers,
+                                    (long long)c->geom.layer_bytes, (long long)n * c->cfg.kv_heads * c->cfg.head_dim * 2));
+    c->launches += 2;
+    c->meta_unsettled = false;
     return BC_OK;
   }
   bc_status st = check_batch(c, layer, slots, n);
@@ -880,7 +968,7 @@ bc_status bc_clear_error(bc_cache* c, void* stream) {
   if (!c) return BC_ERR_INVALID_ARG;
   BC_CUDA(c, cudaMemsetAsync(c->meta.status, 0, 16, (cudaStream_t)stream));
   // an attention launch that gave up (BC_ERR_TIMEOUT) may have left ticket counters non-zero
-  BC_CUDA(c, cudaMemsetAsync(c->work + c->wl.tickets, 0, BC_MAX_ATTN_BATCH * 4, (cudaStream_t)stream));
+  BC_CUDA(c, cudaMemsetAsync(c->work + c->wl.tickets, 0, (size_t)BC_MAX_ATTN_BATCH * 4 * c->cfg.layers, (cudaStream_t)stream));
   // The counters of the built-in array are shared by every cache of the process: they are touched
   // only when THIS cache has used the static entry point since its last clear (a launch of its own
   // may have left them non-zero), never on behalf of a cache that did not.

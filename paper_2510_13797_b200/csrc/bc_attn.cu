@@ -223,6 +223,10 @@ struct PipeParams {
                                   // in flight always uses kSpinLimit
   int debug;                      // BC_FLAG_DEBUG_BOUNDS: every page-table column, page id and pool row is checked
   unsigned long long* timeline;   // NULL, or [gridDim.x][kTimelineSlots] device words: %globaltimer stamps of one thread per block
+  // layer == BC_ALL_LAYERS in one launch: blockIdx.y is the layer, and the block moves every per-layer pointer
+  // by these strides (bytes; tickets: counters).  The metadata, slots, plan and row destinations are shared.
+  long long ls_pool, ls_q, ls_out, ls_kv, ls_part_o, ls_part_ml;
+  int ls_tickets;
   int early_meta;     // 1: the cache's metadata was last written by a kernel that has ENDED, so the plan and the
                       // first page-table reads may run before the wait for the kernel ahead; 0: wait first
 };
@@ -328,9 +332,35 @@ __device__ __forceinline__ void combine_pieces(const float* part_o, const float*
 // fills the window and the encoding of the beacon that follows it (Algorithm 1) read the same entries.
 // The beacon's rows also see the extra entry (the beacon's own K/V).  Needs G <= 8 and is compiled
 // on the 16-row path (G_LE_8 = false); results go to out (token) and out2 (beacon).
-template <int D, bool G_LE_8, bool FUSED, bool PAIR = false, bool SHORTW = false>
-__global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams p) {
+// LAYERED: one launch for all layers of a call with layer = BC_ALL_LAYERS.  The grid is (blocks, layers):
+// the blocks of layer l + 1 are dispatched as those of layer l retire, so the layers follow one another
+// without a kernel boundary; each layer has its own ticket counters and partial buffers, because the last
+// blocks of one layer and the first of the next run side by side.
+template <int D, bool G_LE_8, bool FUSED, bool PAIR = false, bool SHORTW = false, bool LAYERED = false>
+__global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams p_in) {
   static_assert(!PAIR || (!G_LE_8 && !FUSED), "the paired form runs on the 16-row path without the fused append");
+  static_assert(!LAYERED || (!PAIR && !SHORTW), "the all-layers launch exists for the plain and the fused step");
+  PipeParams p_layer;
+  if constexpr (LAYERED) {
+    p_layer = p_in;
+    const long long l = blockIdx.y;
+    p_layer.a.pool_layer = p_in.a.pool_layer + l * p_in.ls_pool;
+    p_layer.a.q = static_cast<const uint8_t*>(p_in.a.q) + l * p_in.ls_q;
+    p_layer.a.out = static_cast<uint8_t*>(p_in.a.out) + l * p_in.ls_out;
+    if (p_in.a.extra_k != nullptr) {
+      p_layer.a.extra_k = static_cast<const uint8_t*>(p_in.a.extra_k) + l * p_in.ls_kv;
+      p_layer.a.extra_v = static_cast<const uint8_t*>(p_in.a.extra_v) + l * p_in.ls_kv;
+    }
+    p_layer.a.part_o = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(p_in.a.part_o) + l * p_in.ls_part_o);
+    p_layer.a.part_ml = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(p_in.a.part_ml) + l * p_in.ls_part_ml);
+    p_layer.a.tickets = p_in.a.tickets + l * p_in.ls_tickets;
+    if (FUSED) {
+      p_layer.f.new_k = p_in.f.new_k + l * p_in.ls_kv;
+      p_layer.f.new_v = p_in.f.new_v + l * p_in.ls_kv;
+      p_layer.f.pool_w = p_in.f.pool_w + l * p_in.ls_pool;
+    }
+  }
+  const PipeParams& p = LAYERED ? p_layer : p_in;
   using L = PipeSmem<D>;
   constexpr int NSTAGE = L::kStages;
   constexpr int KSTEPS = D / 16;  // k-steps of QK^T
@@ -1245,23 +1275,23 @@ FastDiv make_fast_div(uint32_t d) {
   return f;
 }
 
-template <int D, bool G8, bool FUSED, bool PAIR = false, bool SHORTW = false>
+template <int D, bool G8, bool FUSED, bool PAIR = false, bool SHORTW = false, bool LAYERED = false>
 cudaError_t launch_pipe(const PipeParams& p, cudaStream_t s) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(p.a.ctas); cfg.blockDim = dim3(kPipeThreads); cfg.dynamicSmemBytes = PipeSmem<D>::kTotal; cfg.stream = s;
+  cfg.gridDim = dim3(p.a.ctas, LAYERED ? p.a.layers : 1); cfg.blockDim = dim3(kPipeThreads); cfg.dynamicSmemBytes = PipeSmem<D>::kTotal; cfg.stream = s;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;   // see the kernel: it waits for its predecessor after its plan
   cfg.attrs = at; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, k_attn_pipe<D, G8, FUSED, PAIR, SHORTW>, p);
+  return cudaLaunchKernelEx(&cfg, k_attn_pipe<D, G8, FUSED, PAIR, SHORTW, LAYERED>, p);
 }
 
 }  // namespace
 
 namespace {
-template <int D, bool G8, bool FUSED, bool PAIR = false, bool SHORTW = false>
+template <int D, bool G8, bool FUSED, bool PAIR = false, bool SHORTW = false, bool LAYERED = false>
 cudaError_t opt_in_smem() {
-  return cudaFuncSetAttribute(k_attn_pipe<D, G8, FUSED, PAIR, SHORTW>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<D>::kTotal);
+  return cudaFuncSetAttribute(k_attn_pipe<D, G8, FUSED, PAIR, SHORTW, LAYERED>, cudaFuncAttributeMaxDynamicSharedMemorySize, PipeSmem<D>::kTotal);
 }
 }  // namespace
 
@@ -1271,7 +1301,11 @@ cudaError_t bc_attn_setup(int* sm_count) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  const cudaError_t r[12] = {opt_in_smem<128, true, false, false, true>(), opt_in_smem<128, true, true, false, true>(),
+  const cudaError_t r[20] = {opt_in_smem<128, true, false, false, false, true>(), opt_in_smem<128, false, false, false, false, true>(),
+                             opt_in_smem<64, true, false, false, false, true>(), opt_in_smem<64, false, false, false, false, true>(),
+                             opt_in_smem<128, true, true, false, false, true>(), opt_in_smem<128, false, true, false, false, true>(),
+                             opt_in_smem<64, true, true, false, false, true>(), opt_in_smem<64, false, true, false, false, true>(),
+                             opt_in_smem<128, true, false, false, true>(), opt_in_smem<128, true, true, false, true>(),
                              opt_in_smem<128, true, false>(), opt_in_smem<128, false, false>(), opt_in_smem<64, true, false>(),
                              opt_in_smem<64, false, false>(), opt_in_smem<128, true, true>(), opt_in_smem<128, false, true>(),
                              opt_in_smem<64, true, true>(), opt_in_smem<64, false, true>(),
@@ -1308,7 +1342,19 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   cudaError_t e;
   if (ev_start) { e = cudaEventRecord(ev_start, s); if (e != cudaSuccess) return e; }
   const bool g8 = p.G <= 8;
-  if (a.q2 != nullptr) {   // the paired form (token and beacon queries in one pass); the caller has checked G <= 8
+  p.ls_pool = a.ls_pool; p.ls_q = a.ls_q; p.ls_out = a.ls_out; p.ls_kv = a.ls_kv; p.ls_part_o = a.ls_part_o;
+  p.ls_part_ml = a.ls_part_ml; p.ls_tickets = a.ls_tickets;
+  if (a.layers > 1) {      // every layer in this launch (no paired form, no settable wait limit, no timeline)
+    if (a.q2 != nullptr) return cudaErrorInvalidValue;
+    p.timeline = nullptr;
+    if (fused) {
+      if (g.head_dim == 128) e = g8 ? launch_pipe<128, true, true, false, false, true>(p, s) : launch_pipe<128, false, true, false, false, true>(p, s);
+      else e = g8 ? launch_pipe<64, true, true, false, false, true>(p, s) : launch_pipe<64, false, true, false, false, true>(p, s);
+    } else {
+      if (g.head_dim == 128) e = g8 ? launch_pipe<128, true, false, false, false, true>(p, s) : launch_pipe<128, false, false, false, false, true>(p, s);
+      else e = g8 ? launch_pipe<64, true, false, false, false, true>(p, s) : launch_pipe<64, false, false, false, false, true>(p, s);
+    }
+  } else if (a.q2 != nullptr) {   // the paired form (token and beacon queries in one pass); the caller has checked G <= 8
     e = g.head_dim == 128 ? launch_pipe<128, false, false, true>(p, s) : launch_pipe<64, false, false, true>(p, s);
   } else if (shortw) {
     e = fused ? launch_pipe<128, true, true, false, true>(p, s) : launch_pipe<128, true, false, false, true>(p, s);

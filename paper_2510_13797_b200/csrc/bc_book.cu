@@ -264,9 +264,11 @@ k_close(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call) {
 // 16 bytes per thread, applying the chunk permutation of the store layout.
 __global__ void k_write_rows(BcMeta m, BcGeom g, uint8_t* __restrict__ pool_layer, const int32_t* __restrict__ dst_row,
                              const int32_t* __restrict__ dst_pos, const uint8_t* __restrict__ k,
-                             const uint8_t* __restrict__ v, int n) {
+                             const uint8_t* __restrict__ v, int n, long long ls_pool, long long ls_kv) {
   // the attention kernel of the step may start planning now; it waits for this kernel before it reads a row
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // blockIdx.y: the layer, when one launch writes the rows of all layers (same row and position in every layer)
+  pool_layer += blockIdx.y * ls_pool; k += blockIdx.y * ls_kv; v += blockIdx.y * ls_kv;
   const int i = blockIdx.x;
   const int row = dst_row[i];
   if (row < 0) return;
@@ -536,8 +538,10 @@ cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_
   return cudaGetLastError();
 }
 cudaError_t bc_launch_write_rows(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
-                                 const void* k, const void* v, int n, cudaStream_t s) {
-  k_write_rows<<<n, copy_threads(g), 0, s>>>(m, g, pool_layer, dst_row, dst_pos, (const uint8_t*)k, (const uint8_t*)v, n);
+                                 const void* k, const void* v, int n, cudaStream_t s, int layers, long long ls_pool,
+                                 long long ls_kv) {
+  k_write_rows<<<dim3(n, layers), copy_threads(g), 0, s>>>(m, g, pool_layer, dst_row, dst_pos, (const uint8_t*)k, (const uint8_t*)v, n,
+                                                           ls_pool, ls_kv);
   return cudaGetLastError();
 }
 cudaError_t bc_launch_prefill(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* slots,

@@ -72,7 +72,8 @@ cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n
 cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_t call, cudaStream_t s);
 // m is used for the checks of BC_FLAG_DEBUG_BOUNDS only
 cudaError_t bc_launch_write_rows(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* dst_row, const int32_t* dst_pos,
-                                 const void* k, const void* v, int n, cudaStream_t s);
+                                 const void* k, const void* v, int n, cudaStream_t s, int layers = 1, long long ls_pool = 0,
+                                 long long ls_kv = 0);   // layers > 1: the rows of every layer ([layers][n] inputs) in one launch
 cudaError_t bc_launch_restore_book(const BcMeta& m, const int32_t* slots, const int32_t* cu, int n, int64_t call, int32_t* ok,
                                    int32_t* bea, cudaStream_t s);
 cudaError_t bc_launch_restore_rows(const BcMeta& m, const BcGeom& g, uint8_t* pool_layer, const int32_t* slots, const int32_t* ok,
@@ -102,6 +103,11 @@ struct BcAttnArgs {
   uint32_t spin_limit = 0;   // 0: the default poll limit of the bounded waits
   int32_t debug = 0;         // BC_FLAG_DEBUG_BOUNDS
   int32_t meta_settled = 0;  // 1: the kernel that last wrote this cache's metadata has ended by the time this launch may begin
+  // layer == BC_ALL_LAYERS as one launch: the number of layers and the byte strides from one layer to the next of
+  // the pool, q, out, the extra (or new) K/V rows and the partial buffers; tickets: counters per layer
+  int32_t layers = 1;
+  int64_t ls_pool = 0, ls_q = 0, ls_out = 0, ls_kv = 0, ls_part_o = 0, ls_part_ml = 0;
+  int32_t ls_tickets = 0;
   // the paired form (NULL otherwise): the beacons' queries, their outputs and their partial buffers
   const void* q2 = nullptr;
   void* out2 = nullptr;
@@ -127,6 +133,9 @@ struct BcFusedAppend {
 // the same launch appends the step's new entries first.  *launches gets the number of kernels.
 cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, const BcFusedAppend* fused,
                            cudaStream_t s, cudaEvent_t ev_start, cudaEvent_t ev_stop, int* launches);
+// Rotary embedding of the q and k heads of n packed QKV rows, split into three contiguous arrays.
+cudaError_t bc_launch_rope_split(const void* qkv, const int32_t* positions, int n, int q_heads, int kv_heads, int head_dim,
+                                 double theta, void* q_out, void* k_out, void* v_out, cudaStream_t s);
 // Read-only streaming probe: reads bytes (rounded down to 64 KB) of buf once with the attention kernel's copy pattern.
 cudaError_t bc_launch_read_stream(const void* buf, size_t bytes, int* sink, cudaStream_t s);
 // Slow device reference (one warp per query head).

@@ -11,6 +11,7 @@ import torch
 
 from oracle.breadcrumbs_oracle import SeqCache
 from oracle.paging_model import OK, PagingModel
+from oracle.rope_oracle import split_and_rope
 from paper_2510_13797_b200 import binding as B
 
 ABS_TOL = 2e-2   # max-abs error of a head vector (bf16 in, fp32 accumulate)
@@ -102,6 +103,24 @@ class Pair:
         if layer == 0:
             self._append_ok = self.model.append(list(slots))
         kk, vv, qq = f64(k), f64(v), f64(q)
+        ref = np.zeros((len(slots), self.Hq, self.D))
+        for i, slot in enumerate(slots):
+            if self._append_ok[i] == OK:
+                self.seqs[slot].append(layer, kk[i], vv[i])
+            seq = self.seqs.get(slot) or SeqCache(self.L, 1)
+            ref[i] = seq.attend(layer, qq[i], sm_scale)
+        return self._append_ok, out, ref
+
+    def rope_step(self, layer, slots, qkv, positions, theta, sm_scale):
+        """bc_rope_decode_step: the step straight from the packed QKV projection.  The oracle rotates in fp64
+        and rounds q, k to bf16 (the precision the entries are stored in) before its own append and attend."""
+        out = self.gpu.new_out(len(slots))
+        self.gpu.bc_rope_decode_step(layer, self._i32(slots), qkv, self._i32(positions), theta, out, sm_scale)
+        if layer == 0:
+            self._append_ok = self.model.append(list(slots))
+        bf = lambda a: torch.from_numpy(a).to(torch.bfloat16).to(torch.float64).numpy()
+        qq, kk, vv = split_and_rope(f64(qkv), list(positions), self.Hq, self.Hkv, self.D, theta)
+        qq, kk = bf(qq), bf(kk)
         ref = np.zeros((len(slots), self.Hq, self.D))
         for i, slot in enumerate(slots):
             if self._append_ok[i] == OK:

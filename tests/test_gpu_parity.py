@@ -580,3 +580,63 @@ def test_all_layers_in_one_call():
     for l in range(L):
         for s in slots:
             pair.check_content(l, s)
+
+
+@pytest.mark.parametrize("L,Hkv,G,D,ps,c,ctas", [(4, 2, 6, 128, 16, 8, 0), (3, 8, 4, 128, 4, 4, 7), (5, 1, 12, 64, 16, 16, 0),
+                                                  (2, 4, 2, 64, 8, 2, 3)])
+def test_all_layers_one_launch_per_call(L, Hkv, G, D, ps, c, ctas):
+    """layer = -1 is ONE attention launch whose grid walks the layers (and one row-writing launch for an
+    append or a compression): long ragged sequences cut into pieces across blocks, every layer with its own
+    counters and partial buffers; the fused step (bc_decode_step) and the separate calls alternate.  Outputs
+    per layer against the oracle, bookkeeping against the model, launch counts as documented."""
+    Hq = Hkv * G
+    n, plens = 4, [900, 0, 77, 2100]
+    pair = Pair(L, Hkv, Hq, D, ps, max_seqs=n, num_pages=4 * (3200 // ps + 8), max_pages_per_seq=3200 // ps + 8)
+    if ctas:
+        pair.gpu.bc_set_attn_ctas(ctas)
+    g = _gen(31)
+    slots = list(range(n))
+    sl = torch.tensor(slots, dtype=torch.int32, device=DEV)
+    pair.open(slots, plens, [c] * n)
+    P = sum(plens)
+    pk, pv = randn_bf16(g, (L, P, Hkv, D), DEV), randn_bf16(g, (L, P, Hkv, D), DEV)
+    cu = torch.tensor([0] + list(np.cumsum(plens)), dtype=torch.int32, device=DEV)
+    pair.gpu.bc_prefill(-1, sl, cu, P, pk, pv)
+    for l in range(L):
+        for i, s in enumerate(slots):
+            a, b = int(cu[i]), int(cu[i + 1])
+            pair.seqs[s].prefill(l, f64(pk[l, a:b]), f64(pv[l, a:b]))
+    for step in range(1, 2 * c + 2):
+        k, v, q = randn_bf16(g, (L, n, Hkv, D), DEV), randn_bf16(g, (L, n, Hkv, D), DEV), randn_bf16(g, (L, n, Hq, D), DEV)
+        out = torch.full((L, n, Hq, D), float("nan"), dtype=torch.bfloat16, device=DEV)
+        before = pair.gpu.bc_kernel_launches()
+        if step % 2:
+            pair.gpu.bc_decode_step(-1, sl, q, k, v, out, 0.09)
+            assert pair.gpu.bc_kernel_launches() - before == 2          # bookkeeping, attention
+        else:
+            pair.gpu.bc_append(-1, sl, k, v)
+            pair.gpu.bc_decode_attn(-1, sl, q, out, 0.09)
+            assert pair.gpu.bc_kernel_launches() - before == 3          # bookkeeping, rows, attention
+        assert pair.model.append(slots) == [OK] * n
+        for l in range(L):
+            for i, s in enumerate(slots):
+                pair.seqs[s].append(l, f64(k[l, i]), f64(v[l, i]))
+            ref = np.stack([pair.seqs[s].attend(l, f64(q[l, i]), 0.09) for i, s in enumerate(slots)])
+            assert_close(out[l], ref, f"step {step} layer {l}")
+        if step % c == 0:
+            bk, bv, bq = randn_bf16(g, (L, n, Hkv, D), DEV), randn_bf16(g, (L, n, Hkv, D), DEV), randn_bf16(g, (L, n, Hq, D), DEV)
+            before = pair.gpu.bc_kernel_launches()
+            pair.gpu.bc_decode_attn(-1, sl, bq, out, 0.09, bk, bv)
+            pair.gpu.bc_compress(-1, sl, bk, bv)
+            assert pair.gpu.bc_kernel_launches() - before == 3          # attention; bookkeeping, rows
+            assert pair.model.compress(slots) == [OK] * n
+            for l in range(L):
+                ref = np.stack([pair.seqs[s].beacon_attend(l, f64(bq[l, i]), f64(bk[l, i]), f64(bv[l, i]), 0.09)
+                                for i, s in enumerate(slots)])
+                assert_close(out[l], ref, f"beacon step {step} layer {l}")
+                for i, s in enumerate(slots):
+                    pair.seqs[s].compress(l, f64(bk[l, i]), f64(bv[l, i]))
+        pair.check_state()
+    for l in range(L):
+        for s in slots:
+            pair.check_content(l, s)

@@ -24,3 +24,25 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(params=["pinned", "pageable", "mixed"])
+def host_route(request, monkeypatch):
+    """The host-buffer entry points accept page-locked and pageable host memory.  Tests that build their host
+    buffers with Tensor.pin_memory() run three times: as written ("pinned"), with every buffer left pageable
+    ("pageable"), and with the buffers pinned in runs of twelve ("mixed": calls with buffers of both kinds follow
+    one another without a synchronisation)."""
+    import torch
+    if request.param == "pinned":
+        return request.param
+    real = torch.Tensor.pin_memory
+    count = {"n": 0}
+
+    def maybe_pin(self, *a, **kw):
+        count["n"] += 1
+        if request.param == "mixed" and (count["n"] // 12) % 2 == 0:
+            return real(self, *a, **kw)
+        return self.clone() if self.device.type == "cpu" else self.cpu()
+
+    monkeypatch.setattr(torch.Tensor, "pin_memory", maybe_pin)
+    return request.param

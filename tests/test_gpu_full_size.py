@@ -146,14 +146,15 @@ def test_sweep_window_replayed_as_cuda_graph(c, paired, fused):
     check_lengths_and_conservation(drv)
 
 
-def test_sweep_host_buffer_steps_full_size():
-    """The end-to-end leg of the benchmark: host-buffer steps (packed pinned inputs on the cache's copy
-    stream, pipelined outputs) at the sweep's size, c = 4, across a window-fill step."""
+def test_sweep_host_buffer_steps_full_size(host_route):
+    """The end-to-end leg of the benchmark: host-buffer steps (packed inputs on the cache's copy stream,
+    pipelined outputs; page-locked and pageable buffers) at the sweep's size, c = 4, seven steps back to
+    back across two window-fill steps."""
     w = make_workload("sweep", c=4)
     drv = DecodeDriver(w, DEV, beacon_ring=37)
     t0 = (w.steps // 2 // 16) * 16 + 1
     drv.reset_to(t0)
-    for _ in range(3):                                   # steps t0+1 .. t0+3; the last one fills the window (paired)
+    for _ in range(7):                                   # steps t0+1 .. t0+7; the third and the last fill the window (paired)
         drv.step_host()
     drv.cache.bc_host_outputs_ready()
     torch.cuda.synchronize()

@@ -120,7 +120,7 @@ def test_pair_equals_two_separate_calls_bitwise_on_whole_sequences():
     assert torch.equal(o1, p1) and torch.equal(o2, p2)
 
 
-def test_fill_step_host_matches_oracle():
+def test_fill_step_host_matches_oracle(host_route):
     """bc_fill_step_host: append + paired attention + compress with host buffers, issued back to back
     with ordinary host steps; outputs and bookkeeping against the oracle."""
     Hkv, G, D, ps, c = 2, 4, 128, 16, 4
@@ -161,7 +161,7 @@ def test_fill_step_host_matches_oracle():
         pair.check_content(0, s)
 
 
-def test_host_steps_with_pipelined_outputs():
+def test_host_steps_with_pipelined_outputs(host_route):
     """BC_FLAG_HOST_PIPELINED: the outputs come back on the cache's own stream from two staging sets in
     turn.  Many steps are issued with nothing in between; the caller's stream is made to wait with
     bc_host_outputs_ready and is then the only thing synchronised before the outputs are compared."""

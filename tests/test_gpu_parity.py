@@ -316,7 +316,7 @@ def test_reference_kernel_and_f32_output_agree():
         run_decode(pair, [0, 1], [100, 37], [c, c], 24, seed=13, sm_scale=1.0 / math.sqrt(D), check_state_every=8)
 
 
-def test_host_buffer_steps_over_two_layers():
+def test_host_buffer_steps_over_two_layers(host_route):
     """Host-buffer steps of a two-layer cache, layer after layer without synchronising in between:
     regular steps (bc_decode_step_host) and window-filling steps (bc_fill_step_host)."""
     L, Hkv, G, D, ps, c = 2, 2, 4, 128, 4, 3
@@ -369,7 +369,7 @@ def test_host_buffer_steps_over_two_layers():
             pair.check_content(l, s)
 
 
-def test_host_buffer_entry_points():
+def test_host_buffer_entry_points(host_route):
     """bc_decode_step_host / bc_compress_step_host: same results as the device-pointer calls."""
     Hkv, G, D, ps, c = 2, 6, 128, 16, 4
     n, plens = 3, [40, 7, 90]
@@ -475,7 +475,7 @@ def test_fused_decode_step_refusals_and_block_counts():
         pair.check_content(0, s)
 
 
-def test_host_buffer_steps_back_to_back_packed():
+def test_host_buffer_steps_back_to_back_packed(host_route):
     """Host-buffer steps issued without a synchronisation in between, each with its inputs in one
     packed pinned block k | v | q (moved by a single copy): the copies of a step run on the cache's
     copy stream while the previous step's kernels run, in alternating staging buffers.  Every step's

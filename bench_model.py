@@ -74,6 +74,7 @@ class ToyDecoder:
         self.v2 = torch.empty_like(self.k2)
         self.scale = 1.0 / math.sqrt(head_dim)
         self.graph_tok = self.graph_bea = None
+        self.trace = None       # a list: every cache call of an eager step appends (kind, layer, packed QKV rows, positions, outputs)
 
     # -- stand-ins for the rest of the model -------------------------------------------------------
     @staticmethod
@@ -100,6 +101,10 @@ class ToyDecoder:
         v = qkv[:, (Hq + Hkv) * D:].view(-1, Hkv, D).contiguous()
         return q, k, v
 
+    def _record(self, kind, layer, qkv, n, out):
+        if self.trace is not None:
+            self.trace.append((kind, layer, qkv.clone(), self.posv[:n].clone(), out.clone()))
+
     def _forward(self, ids, beacon):
         h = self.emb[ids]
         Hq, Hkv, D = self.Hq, self.Hkv, self.D
@@ -107,6 +112,7 @@ class ToyDecoder:
             qkv = self._norm(h) @ self.wqkv[l]
             if self.lib_rope and not beacon:    # rotation, then the append and the attention in one kernel
                 self.cache.bc_rope_decode_step(l, self.slots, qkv, self.posv[:self.B], self.theta, self.attn_out, self.scale)
+                self._record("token", l, qkv, self.B, self.attn_out)
                 h = h + self.attn_out.view(-1, Hq * D) @ self.wo[l]
                 gu = self._norm(h) @ self.wgu[l]
                 gate, up = gu.chunk(2, dim=-1)
@@ -116,6 +122,7 @@ class ToyDecoder:
             if beacon:      # the beacon's query sees the cache plus its own entry; then the window goes
                 self.cache.bc_decode_attn(l, self.slots, q, self.attn_out, self.scale, k, v)
                 self.cache.bc_compress(l, self.slots, k, v)
+                self._record("beacon", l, qkv, self.B, self.attn_out)
             else:
                 self.cache.bc_append(l, self.slots, k, v)
                 self.cache.bc_decode_attn(l, self.slots, q, self.attn_out, self.scale)
@@ -140,6 +147,7 @@ class ToyDecoder:
             self.cache.bc_decode_attn_pair(l, self.slots, q[:Bn], self.attn_out2[:Bn], q[Bn:], self.attn_out2[Bn:], self.scale,
                                            k[Bn:], v[Bn:])
             self.cache.bc_compress(l, self.slots, k[Bn:], v[Bn:])
+            self._record("pair", l, qkv, 2 * Bn, self.attn_out2)
             h = h + self.attn_out2.view(-1, Hq * D) @ self.wo[l]
             gu = self._norm(h) @ self.wgu[l]
             gate, up = gu.chunk(2, dim=-1)

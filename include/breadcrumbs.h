@@ -360,11 +360,14 @@ BC_API bc_status bc_decode_step_host(bc_cache* cache, int32_t layer, const int32
                               const void* q_host, const void* k_host, const void* v_host,
                               void* out_host, float sm_scale, void* stream);
 /* With BC_FLAG_HOST_PIPELINED the host-buffer steps copy their outputs back on a stream the cache owns
- * (from two staging sets used in turn), so the next step's kernels do not wait behind the copy.  The
- * price: `stream` alone no longer orders the outputs.  out_host of every step issued so far is
- * complete once bc_host_outputs_ready(cache, stream) has been called and `stream` has passed it (or
- * after a device-wide synchronisation); without the flag the call does nothing.  At most two steps'
- * outputs are in flight: the staging set of a step is reused two host-buffer calls later. */
+ * (from eight staging sets used in turn), so the next step's kernels do not wait behind the copy.  The
+ * price: `stream` alone no longer orders the outputs, and the copies of a step's outputs are enqueued
+ * by the NEXT host-buffer call (directly behind that call's bookkeeping kernel), by
+ * bc_host_outputs_ready or by bc_cache_destroy.  out_host of every step issued so far is complete
+ * once bc_host_outputs_ready(cache, stream) has been called and `stream` has passed it; without the
+ * flag the call does nothing.  No wait the library enqueues depends on a call still to be made, so
+ * the caller may synchronise the device at any point.  At most eight steps' outputs are in flight:
+ * the staging set of a step is reused eight host-buffer calls later. */
 BC_API bc_status bc_host_outputs_ready(bc_cache* cache, void* stream);
 
 /* The step that fills a window, with host buffers: bc_append of the token, bc_decode_attn_pair for

@@ -7,6 +7,8 @@
 #include <new>
 #include <vector>
 
+#include <cuda.h>
+
 #include "bc_common.cuh"
 
 namespace {
@@ -32,9 +34,14 @@ MetaLayout meta_layout(const bc_config& c) {
   return l;
 }
 
+// Host-buffer steps: input staging buffers and output staging sets, each used in turn.  Eight deep: a buffer is
+// refilled (and a set rewritten) eight steps after its use, so the stream operations that wait for its last
+// reader are satisfied long before the copy is needed, whatever the latency with which a blocked stream notices.
+constexpr int kHostRing = 8;
+
 struct WorkLayout {
-  size_t append_row[2], append_pos[2], plan[2], compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[4],
-      stage_out[2], stage_out2[2], rope_stage,
+  size_t append_row[2], append_pos[2], plan[2], compress_row, compress_pos, restore_ok, restore_bea, tickets, book_flag, part_ml, part_o, part_ml2, part_o2, stage_in[kHostRing],
+      stage_out[kHostRing], stage_out2[kHostRing], rope_stage, host_words,
       total;
 };
 WorkLayout work_layout(const bc_config& c) {
@@ -59,10 +66,11 @@ WorkLayout work_layout(const bc_config& c) {
   l.part_o = take(pieces1 * c.q_heads * c.head_dim * 4);
   l.part_ml2 = take(pieces * c.q_heads * 2 * 4);            // the beacons' partials of the paired form
   l.part_o2 = take(pieces * c.q_heads * c.head_dim * 4);
-  // host-buffer entry points: a ring of four input staging buffers, each k | v | q packed for the largest
+  // host-buffer entry points: a ring of input staging buffers, each k | v | q packed for the largest
   // batch a call can carry (a step that fills a window takes two of them, token and beacon inputs)
-  for (int b = 0; b < 4; ++b) l.stage_in[b] = take(max_n * (c.q_heads + 2 * c.kv_heads) * c.head_dim * 2);
-  for (int b = 0; b < 2; ++b) {   // two sets of output staging (a set: token output, beacon output)
+  for (int b = 0; b < kHostRing; ++b) l.stage_in[b] = take(max_n * (c.q_heads + 2 * c.kv_heads) * c.head_dim * 2);
+  l.host_words = take((kHostRing + 1) * 4);   // one input word per staging buffer, then the "done" word
+  for (int b = 0; b < kHostRing; ++b) {   // sets of output staging (a set: token output, beacon output)
     l.stage_out[b] = take(max_n * c.q_heads * c.head_dim * 4);
     l.stage_out2[b] = take(max_n * c.q_heads * c.head_dim * 4);
   }
@@ -124,18 +132,28 @@ struct bc_cache {
   std::vector<cudaEvent_t> ev;
   int prof_cap, prof_used;
   // host-buffer entry points: inputs are copied on a stream of their own into a ring of staging buffers
-  static constexpr int kStageRing = 4;
+  static constexpr int kStageRing = kHostRing;
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_in[kStageRing] = {};      // the copies into staging buffer b have been issued up to here
   cudaEvent_t buf_done[kStageRing] = {};   // not owned: the event after which buffer b's last readers have finished
   int stage_next = 0;
+  // Host-buffer decode steps of single-layer caches with BC_FLAG_HOST_PIPELINED are tied to their copies by two
+  // kinds of words in device memory instead of events on the caller's stream (which then carries nothing but
+  // kernels): the copy stream writes a step's number behind its inputs and the step's bookkeeping kernel polls
+  // it; every bookkeeping kernel stores the number of the step before it to the "done" word when it ends, and
+  // the output stream and the copy stream wait for that word (stream memory operations).
+  int32_t host_seq = 0;                       // number of the last such step (0: none yet; 0 is skipped on wrap-around)
+  int32_t done_issued = 0;                    // highest step number that an enqueued kernel will store to the done word
+  int32_t buf_reader_seq[kStageRing] = {};    // number of the last such step that read staging buffer b (0: none)
+  cudaStream_t host_stream = nullptr;         // the caller's stream those steps were enqueued on
   // one event per host-buffer step, recorded on the caller's stream behind the step's kernels
-  static constexpr int kDoneRing = 8;
+  static constexpr int kDoneRing = 2 * kHostRing;
   cudaEvent_t ev_done[kDoneRing] = {};
   int done_next = 0;
   // BC_FLAG_HOST_PIPELINED: outputs leave on a stream of their own from alternating staging sets
   cudaStream_t out_stream = nullptr;
-  cudaEvent_t ev_d2h[2] = {nullptr, nullptr};    // the copies out of set b have been issued up to here
+  static constexpr int kOutSets = kHostRing;
+  cudaEvent_t ev_d2h[kOutSets] = {};             // the copies out of set b have been issued up to here
   int out_next = 0;
   // BC_FLAG_HOST_PIPELINED: what the last host-buffer step still owes -- its completion event and the
   // copies of its outputs.  They are issued by the next host-buffer call right behind that call's
@@ -147,6 +165,7 @@ struct bc_cache {
     void* out_host = nullptr; void* out2_host = nullptr;
     size_t bytes = 0;
     cudaStream_t stream = nullptr;
+    int32_t word_seq = 0;   // a step ordered by words (its number), else 0: ordered by an event
   } pending;
 };
 
@@ -236,13 +255,14 @@ namespace {
 inline int32_t step_epoch(int64_t calls) { return (int32_t)(calls & 0x3fffffff) | 1 << 30; }
 
 // Layer-0 bookkeeping of a step's append, launched on its own (no K/V rows in the same launch).
-bc_status append_book_only(bc_cache* c, const int32_t* slots, int n, cudaStream_t s, bool with_plan = false) {
+bc_status append_book_only(bc_cache* c, const int32_t* slots, int n, cudaStream_t s, bool with_plan = false,
+                           const BcHostSync* hs = nullptr) {
   c->append_set ^= 1;
   ++c->calls;
   BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, c->calls, work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
                                    work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), c->geom, layer_base(c, 0), nullptr,
                                    nullptr, s, with_plan ? work_ptr<int32_t>(c, c->wl.plan[c->append_set]) : nullptr,
-                                   work_ptr<int32_t>(c, c->wl.book_flag), step_epoch(c->calls)));
+                                   work_ptr<int32_t>(c, c->wl.book_flag), step_epoch(c->calls), hs));
   c->launches += 1;
   c->meta_unsettled = true;
   return BC_OK;
@@ -405,7 +425,7 @@ bc_status bc_cache_create(const bc_config* cfg, void* pool, void* meta, void* wo
 bc_status bc_cache_destroy(bc_cache* c) {
   if (!c) return BC_ERR_INVALID_ARG;
   // the cache's own streams touch the caller's workspace: let them drain before the caller may free it
-  if (c->pending.valid) flush_pending(c);
+  flush_pending(c);   // what the last host-buffer steps are owed: their event and copies, or the kernel that vouches for them
   if (c->copy_stream) cudaStreamSynchronize(c->copy_stream);
   if (c->out_stream) cudaStreamSynchronize(c->out_stream);
   for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
@@ -713,18 +733,60 @@ bc_status host_setup(bc_cache* c) {   // first host-buffer call on this cache
   return BC_OK;
 }
 
+// Stream memory operations (driver entry points, looked up once): a 32-bit word in device memory written, or
+// waited for, in the order of a stream, without a kernel.
+typedef CUresult (*StreamValueFn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+StreamValueFn stream_value_fn(const char* name) {
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint(name, &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) return nullptr;
+  return reinterpret_cast<StreamValueFn>(p);
+}
+StreamValueFn stream_wait_value() { static StreamValueFn fn = stream_value_fn("cuStreamWaitValue32"); return fn; }
+StreamValueFn stream_write_value() { static StreamValueFn fn = stream_value_fn("cuStreamWriteValue32"); return fn; }
+#define BC_DRV(c, expr)                                               \
+  do {                                                                \
+    if ((expr) != CUDA_SUCCESS) return cuda_fail((c), cudaErrorUnknown); \
+  } while (0)
+
+inline int32_t* in_word(bc_cache* c, int buf) { return work_ptr<int32_t>(c, c->wl.host_words) + buf; }
+inline int32_t* done_word(bc_cache* c) { return work_ptr<int32_t>(c, c->wl.host_words) + bc_cache::kStageRing; }
+
+// The host-buffer steps whose completion no enqueued kernel vouches for yet get a one-thread kernel that does,
+// behind everything enqueued on their stream so far.
+bc_status vouch_for_host_steps(bc_cache* c) {
+  if (c->done_issued == c->host_seq) return BC_OK;
+  BC_CUDA(c, bc_launch_host_steps_done(done_word(c), c->host_seq, c->host_stream));
+  c->launches += 1;
+  c->done_issued = c->host_seq;
+  return BC_OK;
+}
+
+// The copy stream waits until staging buffer `buf` has no reader left: the event of its last reader among the
+// steps ordered by events, the done word for its last reader among the steps ordered by words.
+bc_status wait_buffer_free(bc_cache* c, int buf) {
+  if (c->buf_done[buf]) BC_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->buf_done[buf], 0));
+  if (c->buf_reader_seq[buf])
+    BC_DRV(c, stream_wait_value()((CUstream)c->copy_stream, (CUdeviceptr)done_word(c), (cuuint32_t)c->buf_reader_seq[buf],
+                                  CU_STREAM_WAIT_VALUE_GEQ));
+  return BC_OK;
+}
+
 // Stages k, v, q of a host-buffer step: the copies run on the cache's own copy stream, so the next
 // steps' inputs travel while this step's kernels run; `s` waits for them before the kernels that read
 // them.  Returns the staging buffer used.
 bc_status stage_inputs(bc_cache* c, int32_t n, const void* q_host, const void* k_host, const void* v_host, cudaStream_t s,
-                       int* buf_out, void** dq, void** dk, void** dv) {
+                       int* buf_out, void** dq, void** dk, void** dv, int32_t word_seq = 0) {
   const int buf = c->stage_next;
   c->stage_next = (buf + 1) % bc_cache::kStageRing;
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2, kb = (size_t)n * c->cfg.kv_heads * c->cfg.head_dim * 2;
   uint8_t* base = c->work + c->wl.stage_in[buf];
   *dk = base; *dv = base + kb; *dq = base + 2 * kb;
   // the buffer's previous readers (a whole turn of the ring ago) must be done
-  if (c->buf_done[buf]) BC_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->buf_done[buf], 0));
+  {
+    const bc_status st = wait_buffer_free(c, buf);
+    if (st) return st;
+  }
   // Pipelined outputs: the step that receives these inputs writes the output staging set whose last
   // copies to the host (two steps ago) must be over.  The copy stream waits for them here, so that the
   // one event the caller's stream waits for below covers both and no second wait sits between kernels.
@@ -738,21 +800,29 @@ bc_status stage_inputs(bc_cache* c, int32_t n, const void* q_host, const void* k
     BC_CUDA(c, cudaMemcpyAsync(*dv, vh, kb, cudaMemcpyHostToDevice, c->copy_stream));
     BC_CUDA(c, cudaMemcpyAsync(*dq, qh, qb, cudaMemcpyHostToDevice, c->copy_stream));
   }
-  BC_CUDA(c, cudaEventRecord(c->ev_in[buf], c->copy_stream));
-  BC_CUDA(c, cudaStreamWaitEvent(s, c->ev_in[buf], 0));
+  if (word_seq != 0) {   // the step's bookkeeping kernel polls the word: no wait on the caller's stream
+    BC_DRV(c, stream_write_value()((CUstream)c->copy_stream, (CUdeviceptr)in_word(c, buf), (cuuint32_t)word_seq,
+                                   CU_STREAM_WRITE_VALUE_DEFAULT));
+    c->buf_reader_seq[buf] = word_seq;
+    c->buf_done[buf] = nullptr;
+  } else {
+    BC_CUDA(c, cudaEventRecord(c->ev_in[buf], c->copy_stream));
+    BC_CUDA(c, cudaStreamWaitEvent(s, c->ev_in[buf], 0));
+    c->buf_reader_seq[buf] = 0;   // finish_step names the event of this step's readers
+  }
   *buf_out = buf;
   return BC_OK;
 }
 
 // Output staging of a host-buffer step.  Plain mode: one set, the copies follow the kernels on `s`.
-// Pipelined mode (BC_FLAG_HOST_PIPELINED): two sets in turn; the copies of a step run on the cache's
+// Pipelined mode (BC_FLAG_HOST_PIPELINED): four sets in turn; the copies of a step run on the cache's
 // output stream after its kernels, so the next step's kernels do not wait for them; `s` waits for
 // them only in bc_host_outputs_ready.
 bc_status begin_outputs(bc_cache* c, cudaStream_t s, int* set, void** dout, void** dout2) {
   *set = 0;
   if (c->cfg.flags & BC_FLAG_HOST_PIPELINED) {
-    *set = c->out_next;   // its copies of two steps ago are over: stage_inputs made the copy stream wait for them
-    c->out_next ^= 1;
+    *set = c->out_next;   // its copies of four steps ago are over: the copy stream waited for them before this step's inputs
+    c->out_next = (c->out_next + 1) % bc_cache::kOutSets;
   }
   *dout = c->work + c->wl.stage_out[*set];
   *dout2 = c->work + c->wl.stage_out2[*set];
@@ -779,8 +849,22 @@ bc_status finish_step(bc_cache* c, const bc_cache::Pending& p) {
 }
 
 bc_status flush_pending(bc_cache* c) {
+  {   // steps ordered by words that nothing vouches for yet: what follows is ordered by events
+    const bc_status st = vouch_for_host_steps(c);
+    if (st) return st;
+  }
   if (!c->pending.valid) return BC_OK;
   c->pending.valid = false;
+  if (c->pending.word_seq) {
+    // A kernel that stores this step's number to the done word is enqueued by now (the next step's bookkeeping
+    // kernel, or the one-thread kernel above): the wait below never depends on a call still to be made, so a
+    // device-wide synchronisation by the caller cannot block on it.
+    const bc_cache::Pending& p = c->pending;
+    BC_DRV(c, stream_wait_value()((CUstream)c->out_stream, (CUdeviceptr)done_word(c), (cuuint32_t)p.word_seq, CU_STREAM_WAIT_VALUE_GEQ));
+    BC_CUDA(c, cudaMemcpyAsync(p.out_host, c->work + c->wl.stage_out[p.set], p.bytes, cudaMemcpyDeviceToHost, c->out_stream));
+    BC_CUDA(c, cudaEventRecord(c->ev_d2h[p.set], c->out_stream));
+    return BC_OK;
+  }
   return finish_step(c, c->pending);
 }
 
@@ -798,10 +882,10 @@ bc_status close_step(bc_cache* c, cudaStream_t s, int set, int buf, int buf2, vo
 
 bc_status bc_host_outputs_ready(bc_cache* c, void* stream) {
   if (!c) return BC_ERR_INVALID_ARG;
-  bc_status st = flush_pending(c);
+  bc_status st = flush_pending(c);   // also vouches for the steps ordered by words
   if (st) return st;
   if (c->out_stream)
-    for (int b = 0; b < 2; ++b) BC_CUDA(c, cudaStreamWaitEvent((cudaStream_t)stream, c->ev_d2h[b], 0));
+    for (int b = 0; b < bc_cache::kOutSets; ++b) BC_CUDA(c, cudaStreamWaitEvent((cudaStream_t)stream, c->ev_d2h[b], 0));
   return BC_OK;
 }
 
@@ -817,6 +901,40 @@ bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, 
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
   const bool reference = (c->cfg.flags & BC_FLAG_ATTN_REFERENCE) != 0;
+  if (c->cfg.layers == 1 && (c->cfg.flags & BC_FLAG_HOST_PIPELINED) && !reference && stream_wait_value() && stream_write_value()) {
+    // Ordered by words (see bc_cache::host_seq): the caller's stream gets the bookkeeping kernel and the attention
+    // kernel, nothing else, so the step overlaps with its neighbours exactly as a device-resident bc_decode_step.
+    if ((c->pending.valid && !c->pending.word_seq) || c->host_stream != s) {
+      // a step ordered by events is still owed its event and output copies; or the caller changed streams: the
+      // steps so far are vouched for on the stream they were enqueued on
+      st = flush_pending(c);
+      if (st) return st;
+      c->host_stream = s;
+    }
+    const int32_t prev = c->host_seq;
+    int32_t id = prev + 1;
+    if (id == 0) id = 1;
+    void *dq, *dk, *dv, *dout, *dout2;
+    int buf, set;
+    st = stage_inputs(c, n, q_host, k_host, v_host, s, &buf, &dq, &dk, &dv, id);   // also waits for the output set's last copies
+    if (st) return st;
+    st = begin_outputs(c, s, &set, &dout, &dout2);
+    if (st) return st;
+    BcHostSync hs = {in_word(c, buf), id, prev ? done_word(c) : nullptr, prev};
+    st = append_book_only(c, slots, n, s, true, &hs);
+    if (st) return st;
+    c->done_issued = prev;       // that kernel vouches for every step before this one ...
+    st = flush_pending(c);       // ... so the last step's output rows may be sent on their way now
+    if (st) return st;
+    c->host_seq = id;
+    st = decode_step_attn(c, layer, slots, n, dq, dk, dv, dout, sm_scale, s);
+    if (st) return st;
+    // this step's output rows leave with the next host-buffer call, bc_host_outputs_ready or bc_cache_destroy
+    bc_cache::Pending p;
+    p.valid = true; p.set = set; p.out_host = out_host; p.bytes = ob; p.stream = s; p.word_seq = id;
+    c->pending = p;
+    return BC_OK;
+  }
   // The step's bookkeeping needs nothing from the host, so it goes out first, directly behind the last
   // step's attention kernel (under whose last blocks it may start); only then the events and copies
   // that the last step still owes, and this step's own copies.

@@ -109,7 +109,7 @@ __device__ __forceinline__ void wait_for_overtaken_kernel() { asm volatile("grid
 __global__ void __launch_bounds__(kBookThreads, 1)
 k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
               int32_t* dst_row, int32_t* dst_pos, BcGeom g, uint8_t* pool_layer, const uint8_t* k, const uint8_t* v,
-              int32_t* plan, int32_t* flag, int32_t epoch) {
+              int32_t* plan, int32_t* flag, int32_t epoch, BcHostSync hs) {
   // With a plan to leave, this is the bookkeeping of a fused decode step, and the kernel enqueued behind it
   // is that step's attention kernel.  Its blocks may take their places on the SMs now; what they read of
   // this kernel's results they read after the flag below (release here, acquire there), and everything the
@@ -127,11 +127,46 @@ k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
   append_book_block(m, slots, n, call, dst_row, dst_pos, plan, tile_shift);
   __syncthreads();
   if (plan != nullptr && threadIdx.x == 0) {   // lengths, page-table column, row destinations and plan are written
-    __threadfence();
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(epoch) : "memory");
+    // A host-buffer step: q, k, v travel on the cache's copy stream, which writes the step's number to a word
+    // behind the copy (a stream memory operation, not a kernel).  The flag below lets the attention kernel read
+    // those inputs, so it is published only once the word shows this step; the caller's stream then needs no
+    // wait for the copy between this kernel and the attention kernel.  If the word does not show up within the
+    // limit the step is reported (BC_ERR_TIMEOUT) and no flag is published.
+    bool inputs_in = true;
+    if (hs.in_word != nullptr) {
+      inputs_in = false;
+      for (uint32_t polls = 0; polls < (1u << 21); ++polls) {
+        int seen;
+        asm volatile("ld.acquire.sys.global.s32 %0, [%1];" : "=r"(seen) : "l"(hs.in_word) : "memory");
+        if (seen == hs.in_seq) { inputs_in = true; break; }
+        __nanosleep(100);
+      }
+      if (!inputs_in && m.status[0] == 0) {
+        m.status[0] = BC_ERR_TIMEOUT; m.status[1] = -1;
+        *reinterpret_cast<int64_t*>(m.status + 2) = call;
+      }
+    }
+    if (inputs_in) {
+      __threadfence();
+      asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(flag), "r"(epoch) : "memory");
+    }
   }
   if (k != nullptr) block_write_rows(m, g, pool_layer, dst_row, dst_pos, k, v, n);  // layer 0's rows, same launch
   wait_for_overtaken_kernel();
+  // Everything enqueued ahead of this kernel has ended, the previous host-buffer step's attention kernel
+  // included: its output rows may be copied to the host and its input staging buffer refilled.  The word is
+  // read by stream memory operations of the cache's other streams.
+  if (hs.done_word != nullptr && threadIdx.x == 0) {
+    __threadfence_system();
+    *reinterpret_cast<volatile int32_t*>(hs.done_word) = hs.done_seq;
+  }
+}
+
+// Writes the number of the last host-buffer step to the "done" word once everything ahead of it on the stream
+// has ended (an ordinary launch): for the step that no later bookkeeping kernel vouches for.
+__global__ void k_host_steps_done(int32_t* done_word, int32_t seq) {
+  __threadfence_system();
+  *reinterpret_cast<volatile int32_t*>(done_word) = seq;
 }
 
 // phase & 1: validate, allocate the beacon slot, fill dst_row/dst_pos (dst_row < 0: item failed).
@@ -515,12 +550,17 @@ cudaError_t launch_book_overlapped(void (*kernel)(KArgs...), cudaStream_t s, Arg
 
 cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                   int32_t* dst_pos, const BcGeom& g, uint8_t* pool_layer, const void* k, const void* v,
-                                  cudaStream_t s, int32_t* plan, int32_t* flag, int32_t epoch) {
+                                  cudaStream_t s, int32_t* plan, int32_t* flag, int32_t epoch, const BcHostSync* hs) {
+  const BcHostSync none = {nullptr, 0, nullptr, 0};
   if (k == nullptr)   // the rows follow in a launch of their own (ordinary order: it waits for everything before it)
     return launch_book_overlapped(k_append_book, s, m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)nullptr,
-                                  (const uint8_t*)nullptr, plan, flag, epoch);
+                                  (const uint8_t*)nullptr, plan, flag, epoch, hs ? *hs : none);
   k_append_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)k,
-                                           (const uint8_t*)v, (int32_t*)nullptr, (int32_t*)nullptr, 0);
+                                           (const uint8_t*)v, (int32_t*)nullptr, (int32_t*)nullptr, 0, none);
+  return cudaGetLastError();
+}
+cudaError_t bc_launch_host_steps_done(int32_t* done_word, int32_t seq, cudaStream_t s) {
+  k_host_steps_done<<<1, 1, 0, s>>>(done_word, seq);
   return cudaGetLastError();
 }
 cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,

@@ -62,9 +62,20 @@ cudaError_t bc_launch_open(const BcMeta& m, const int32_t* slots, const int32_t*
 // does), which saves a launch when the batch is small enough for one thread block to copy.
 // plan non-null (k, v null): the launch also leaves the attention plan of the batch (BC_PLAN_INTS ints) and
 // then stores `epoch` to *flag with release semantics
+// Host-buffer steps whose copies are tied to the kernels by words in device memory instead of events on the
+// caller's stream: the bookkeeping kernel waits (bounded) until *in_word == in_seq before it lets the attention
+// kernel read the step's inputs, and stores done_seq to *done_word when everything ahead of it has ended.
+struct BcHostSync {
+  const int32_t* in_word;   // NULL: no wait
+  int32_t in_seq;
+  int32_t* done_word;       // NULL: no store
+  int32_t done_seq;
+};
+cudaError_t bc_launch_host_steps_done(int32_t* done_word, int32_t seq, cudaStream_t s);
 cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                   int32_t* dst_pos, const BcGeom& g, uint8_t* pool_layer, const void* k, const void* v,
-                                  cudaStream_t s, int32_t* plan = nullptr, int32_t* flag = nullptr, int32_t epoch = 0);
+                                  cudaStream_t s, int32_t* plan = nullptr, int32_t* flag = nullptr, int32_t epoch = 0,
+                                  const BcHostSync* hs = nullptr);
 // phase bit 1: allocate the beacon slot; phase bit 2: evict the window and bump the counters
 cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                     int32_t* dst_pos, int phase, const BcGeom& g, uint8_t* pool_layer, const void* k,

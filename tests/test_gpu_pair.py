@@ -207,3 +207,53 @@ def test_host_steps_with_pipelined_outputs(host_route):
             for i, s in enumerate(slots):
                 pair.seqs[s].compress(0, f64(bk)[i], f64(bv)[i])
     pair.check_state()
+
+
+def test_pipelined_host_steps_with_device_synchronisations_in_between():
+    """Single-layer cache, pipelined outputs: a regular host-buffer step leaves nothing on the caller's stream but
+    its kernels, and the copies are released through words in device memory.  None of the library's waits may
+    depend on a call still to be made: the device is synchronised after every call (and pinned memory is
+    allocated, which synchronises implicitly), a stream switch sits in the middle, and only
+    bc_host_outputs_ready is called before the outputs are read."""
+    Hkv, G, D, ps, c = 2, 4, 128, 16, 5
+    n, plens = 3, [90, 0, 300]
+    pair = Pair(1, Hkv, Hkv * G, D, ps, max_seqs=n, num_pages=96, max_pages_per_seq=32, flags=B.BC_FLAG_HOST_PIPELINED)
+    g = _gen(41)
+    slots = list(range(n))
+    assert pair.open(slots, plens, [c] * n) == [OK] * n
+    pair.prefill(0, slots, plens, randn_bf16(g, (sum(plens), Hkv, D), DEV), randn_bf16(g, (sum(plens), Hkv, D), DEV))
+    sl = torch.tensor(slots, dtype=torch.int32, device=DEV)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    pending = []
+    for step in range(1, 2 * c + 3):
+        k, v, q = randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv * G, D), DEV)
+        assert pair.model.append(slots) == [OK] * n
+        for i, s in enumerate(slots):
+            pair.seqs[s].append(0, f64(k)[i], f64(v)[i])
+        ref = np.stack([pair.seqs[s].attend(0, f64(q)[i], 0.1) for i, s in enumerate(slots)])
+        hk, hv, hq = k.cpu().pin_memory(), v.cpu().pin_memory(), q.cpu().pin_memory()
+        out_h = torch.full((n, Hkv * G, D), float("nan"), dtype=torch.bfloat16).pin_memory()
+        stream = s1 if step <= c + 1 else s2
+        torch.cuda.synchronize()                       # everything enqueued so far, the library's own streams included
+        with torch.cuda.stream(stream):
+            if step % c:
+                pair.gpu.bc_decode_step_host(0, sl, hq, hk, hv, out_h, 0.1)
+                pending.append((out_h, ref, f"host step {step}", (hk, hv, hq)))
+            else:
+                bk, bv, bq = randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv * G, D), DEV)
+                out_b = torch.full((n, Hkv * G, D), float("nan"), dtype=torch.bfloat16).pin_memory()
+                hb = (bq.cpu().pin_memory(), bk.cpu().pin_memory(), bv.cpu().pin_memory())
+                pair.gpu.bc_fill_step_host(0, sl, hq, hk, hv, hb[0], hb[1], hb[2], out_h, out_b, 0.1)
+                ref_b = np.stack([pair.seqs[s].beacon_attend(0, f64(bq)[i], f64(bk)[i], f64(bv)[i], 0.1) for i, s in enumerate(slots)])
+                pending.append((out_h, ref, f"fill step {step}: token", (hk, hv, hq, hb)))
+                pending.append((out_b, ref_b, f"fill step {step}: beacon", None))
+                assert pair.model.compress(slots) == [OK] * n
+                for i, s in enumerate(slots):
+                    pair.seqs[s].compress(0, f64(bk)[i], f64(bv)[i])
+    with torch.cuda.stream(s2):
+        pair.gpu.bc_host_outputs_ready()
+    s2.synchronize()
+    for o, r, what, _ in pending:
+        assert_close(o, r, what)
+    pair.check_state()

@@ -704,9 +704,12 @@ def report_depth(args):
                 # the token fills the window: per layer append, then token and beacon queries in one pass, then compress
                 _, (bq, bk, bv) = ins[l]
                 m = ((t + 1) // c) % 2
-                cache.bc_append(l, slots, k[j], v[j])
-                cache.bc_decode_attn_pair(l, slots, q[j], out, bq[m], out_b, w.sm_scale, bk[m], bv[m])
-                cache.bc_compress(l, slots, bk[m], bv[m])
+                if not args.no_fused:
+                    cache.bc_fill_step(l, slots, q[j], k[j], v[j], bq[m], bk[m], bv[m], out, out_b, w.sm_scale)
+                else:
+                    cache.bc_append(l, slots, k[j], v[j])
+                    cache.bc_decode_attn_pair(l, slots, q[j], out, bq[m], out_b, w.sm_scale, bk[m], bv[m])
+                    cache.bc_compress(l, slots, bk[m], bv[m])
             elif attend and not args.no_fused:
                 cache.bc_decode_step(l, slots, q[j], k[j], v[j], out, w.sm_scale)
             else:
@@ -1219,7 +1222,10 @@ def main():
                    "regular_steps": "bc_append + bc_decode_attn" if args.no_fused else
                                     "bc_decode_step (the append's bookkeeping kernel, then one attention kernel that takes the new entries from the inputs)",
                    "beacon_steps": "second attention pass" if args.no_pair else
-                                   "paired with the token's attention (bc_decode_attn_pair: one pass over the cache)"},
+                                   ("paired with the token's attention (bc_append, bc_decode_attn_pair: one pass over the cache, bc_compress)"
+                                    if args.no_fused else
+                                    "bc_fill_step (the append's bookkeeping kernel, one paired attention kernel that takes the token's entry "
+                                    "from the inputs and serves the token's and the beacon's rows in one pass over the cache, bc_compress)")},
         "e2e": {"value": world * B * n_c * K / (e2e_ms * 1e-3), "unit": "tokens/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(total_launches),

@@ -289,6 +289,22 @@ BC_API bc_status bc_rope_split(bc_cache* cache, const void* qkv, const int32_t* 
 BC_API bc_status bc_rope_decode_step(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n, const void* qkv,
                                      const int32_t* positions, float theta, void* out, float sm_scale, void* stream);
 
+/* The step whose token fills the window, in one call: bc_append(k, v), bc_decode_attn_pair(q, beacon_q;
+ * extra = beacon_k, beacon_v) and bc_compress(beacon_k, beacon_v) (Algorithm 1: the token's forward
+ * pass, the beacon's forward pass, the eviction).  Results, bookkeeping, layer-order rule (the layer
+ * must be the next one of both the append and the compress order) and error behaviour are exactly
+ * those of the three calls made one after the other.  How: as in bc_decode_step the append's
+ * bookkeeping runs as its own one-block kernel and ONE attention launch takes the token's entry from
+ * the inputs, serves the token's and the beacon's query heads in one pass over the cache and stores
+ * the entry; then the compression (bookkeeping kernel, beacon rows).  Two launches fewer than the
+ * three calls, and the attention kernel overlaps with the step before it like a regular step's.
+ * q, beacon_q [n, q_heads, head_dim], k, v, beacon_k, beacon_v [n, kv_heads, head_dim], out,
+ * out_beacon like q; all device, 16-byte aligned; n <= 512.  For groups of more than 8 query heads
+ * per KV head, and with BC_FLAG_ATTN_REFERENCE, the call issues the three calls. */
+BC_API bc_status bc_fill_step(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n, const void* q,
+                              const void* k, const void* v, const void* beacon_q, const void* beacon_k,
+                              const void* beacon_v, void* out, void* out_beacon, float sm_scale, void* stream);
+
 /* Limits of bc_decode_attn_static. */
 #define BC_STATIC_MAX_BATCH 128   /* sequences per call */
 #define BC_STATIC_MAX_CTAS 160    /* thread blocks it will use at most */
@@ -370,9 +386,10 @@ BC_API bc_status bc_decode_step_host(bc_cache* cache, int32_t layer, const int32
  * the staging set of a step is reused eight host-buffer calls later. */
 BC_API bc_status bc_host_outputs_ready(bc_cache* cache, void* stream);
 
-/* The step that fills a window, with host buffers: bc_append of the token, bc_decode_attn_pair for
- * the token and its beacon (one pass over the cache), bc_compress.  Equivalent to
- * bc_decode_step_host followed by bc_compress_step_host; same conventions. */
+/* The step that fills a window, with host buffers: bc_fill_step (bc_append of the token,
+ * bc_decode_attn_pair for the token and its beacon in one pass over the cache, bc_compress).
+ * Equivalent to bc_decode_step_host followed by bc_compress_step_host; same conventions, the
+ * ordering by words on single-layer caches with BC_FLAG_HOST_PIPELINED included. */
 BC_API bc_status bc_fill_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                                    const void* q_host, const void* k_host, const void* v_host,
                                    const void* beacon_q_host, const void* beacon_k_host,

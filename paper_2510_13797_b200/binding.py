@@ -84,6 +84,7 @@ SYMBOLS = {
     "bc_profile_enable": (_I32, [_P, _I32]),
     "bc_profile_read": (_I32, [_P, C.POINTER(_I32), C.POINTER(_F)]),
     "bc_probe_read_stream": (_I32, [_P, C.c_size_t, _P]),
+    "bc_fill_step": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _P, _P, _P, _P, _F, _P]),
     "bc_rope_split": (_I32, [_P, _P, _P, _I32, _F, _P, _P, _P, _P]),
     "bc_rope_decode_step": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _F, _P]),
     "bc_kernel_launches": (_I64, [_P]),
@@ -189,6 +190,12 @@ class Cache:
         """bc_append(k, v) + bc_decode_attn(q) in one launch."""
         _check(lib().bc_decode_step(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(k), _ptr(v), _ptr(out),
                                     sm_scale, _stream(stream)), "bc_decode_step")
+
+    def bc_fill_step(self, layer, slots, q, k, v, beacon_q, beacon_k, beacon_v, out, out_beacon, sm_scale, stream=None):
+        """The step that fills a window: bc_append + bc_decode_attn_pair + bc_compress, the append inside the attention launch."""
+        _check(lib().bc_fill_step(self.handle, layer, _ptr(slots), slots.numel(), _ptr(q), _ptr(k), _ptr(v), _ptr(beacon_q),
+                                  _ptr(beacon_k), _ptr(beacon_v), _ptr(out), _ptr(out_beacon), sm_scale, _stream(stream)),
+               "bc_fill_step")
 
     def bc_rope_split(self, qkv, positions, theta, q_out, k_out, v_out, stream=None):
         """Rotary embedding of the q and k heads of a packed QKV projection, split into the three arrays the cache calls take."""

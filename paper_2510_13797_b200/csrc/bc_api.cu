@@ -119,6 +119,7 @@ struct bc_cache {
   int compress_next_layer;  // per-layer ordering of bc_compress
   int restore_next_layer = 0;   // per-layer ordering of bc_restore
   int append_set = 0;           // which set of append row destinations the current step uses (flips on layer 0)
+  int64_t append_call = 0;      // index of the step's append bookkeeping call (its flag's epoch; other calls may lie between the layers)
   // true while the last kernel this handle enqueued that writes metadata (lengths, page table, free stack)
   // has not been followed by an ordinarily launched kernel or an attention launch of this handle: an
   // attention kernel enqueued now could begin before that writer has ended and must not read early
@@ -259,6 +260,7 @@ bc_status append_book_only(bc_cache* c, const int32_t* slots, int n, cudaStream_
                            const BcHostSync* hs = nullptr) {
   c->append_set ^= 1;
   ++c->calls;
+  c->append_call = c->calls;
   BC_CUDA(c, bc_launch_append_book(c->meta, slots, n, c->calls, work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
                                    work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), c->geom, layer_base(c, 0), nullptr,
                                    nullptr, s, with_plan ? work_ptr<int32_t>(c, c->wl.plan[c->append_set]) : nullptr,
@@ -269,8 +271,10 @@ bc_status append_book_only(bc_cache* c, const int32_t* slots, int n, cudaStream_
 }
 
 // The attention half of bc_decode_step: the step's append bookkeeping (layer 0) has been launched.
+// With beacon_q .. out_beacon: the step that fills a window (the paired form of the same kernel).
 bc_status decode_step_attn(bc_cache* c, int layer, const int32_t* slots, int n, const void* q, const void* k, const void* v,
-                           void* out, float sm_scale, cudaStream_t s, int layers = 1) {
+                           void* out, float sm_scale, cudaStream_t s, int layers = 1, const void* beacon_q = nullptr,
+                           const void* beacon_k = nullptr, const void* beacon_v = nullptr, void* out_beacon = nullptr) {
   BcFusedAppend f;
   f.new_k = k; f.new_v = v;
   f.dst_row = work_ptr<int32_t>(c, c->wl.append_row[c->append_set]);
@@ -279,9 +283,9 @@ bc_status decode_step_attn(bc_cache* c, int layer, const int32_t* slots, int n, 
   f.flag = work_ptr<int32_t>(c, c->wl.book_flag);
   f.plan = work_ptr<int32_t>(c, c->wl.plan[c->append_set]);   // left by append_book_only(with_plan) of this step
   f.do_book = 0;
-  f.call = c->calls;
-  f.epoch = step_epoch(c->calls);
-  const bc_status st = attn_impl(c, layer, slots, n, q, out, sm_scale, nullptr, nullptr, s, &f, nullptr, nullptr, layers);
+  f.call = c->append_call;
+  f.epoch = step_epoch(c->append_call);
+  const bc_status st = attn_impl(c, layer, slots, n, q, out, sm_scale, beacon_k, beacon_v, s, &f, beacon_q, out_beacon, layers);
   if (st) return st;
   c->append_next_layer = (layer + layers) % c->cfg.layers;
   return BC_OK;
@@ -659,6 +663,36 @@ bc_status bc_rope_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, 
   return bc_decode_step(c, layer, slots, n, q, k, v, out, sm_scale, stream);
 }
 
+bc_status bc_fill_step(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* q, const void* k,
+                       const void* v, const void* beacon_q, const void* beacon_k, const void* beacon_v, void* out,
+                       void* out_beacon, float sm_scale, void* stream) {
+  bc_status st = check_batch(c, layer, slots, n);
+  if (st) return st;
+  if (n > BC_MAX_ATTN_BATCH) return BC_ERR_INVALID_ARG;
+  if (!q || !k || !v || !beacon_q || !beacon_k || !beacon_v || !out || !out_beacon) return BC_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(beacon_q) || !aligned16(beacon_k) || !aligned16(beacon_v) ||
+      !aligned16(out) || !aligned16(out_beacon))
+    return BC_ERR_INVALID_ARG;
+  if (layer != c->append_next_layer || layer != c->compress_next_layer) return BC_ERR_ORDER;
+  cudaStream_t s = (cudaStream_t)stream;
+  if ((c->cfg.flags & BC_FLAG_ATTN_REFERENCE) || c->cfg.q_heads / c->cfg.kv_heads > 8) {   // no paired kernel: the three calls
+    st = bc_append(c, layer, slots, n, k, v, stream);
+    if (st) return st;
+    st = bc_decode_attn_pair(c, layer, slots, n, q, out, beacon_q, out_beacon, sm_scale, beacon_k, beacon_v, stream);
+    if (st) return st;
+    return bc_compress(c, layer, slots, n, beacon_k, beacon_v, stream);
+  }
+  // the append's bookkeeping kernel (it leaves the plan and its flag), ONE attention launch that takes the token's
+  // entry from the inputs and serves both sets of query heads, then the compression
+  if (layer == 0) {
+    st = append_book_only(c, slots, n, s, true);
+    if (st) return st;
+  }
+  st = decode_step_attn(c, layer, slots, n, q, k, v, out, sm_scale, s, 1, beacon_q, beacon_k, beacon_v, out_beacon);
+  if (st) return st;
+  return bc_compress(c, layer, slots, n, beacon_k, beacon_v, stream);
+}
+
 bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* bk, const void* bv,
                       void* stream) {
   if (c && layer == BC_ALL_LAYERS) {
@@ -862,6 +896,8 @@ bc_status flush_pending(bc_cache* c) {
     const bc_cache::Pending& p = c->pending;
     BC_DRV(c, stream_wait_value()((CUstream)c->out_stream, (CUdeviceptr)done_word(c), (cuuint32_t)p.word_seq, CU_STREAM_WAIT_VALUE_GEQ));
     BC_CUDA(c, cudaMemcpyAsync(p.out_host, c->work + c->wl.stage_out[p.set], p.bytes, cudaMemcpyDeviceToHost, c->out_stream));
+    if (p.out2_host)
+      BC_CUDA(c, cudaMemcpyAsync(p.out2_host, c->work + c->wl.stage_out2[p.set], p.bytes, cudaMemcpyDeviceToHost, c->out_stream));
     BC_CUDA(c, cudaEventRecord(c->ev_d2h[p.set], c->out_stream));
     return BC_OK;
   }
@@ -920,7 +956,7 @@ bc_status bc_decode_step_host(bc_cache* c, int32_t layer, const int32_t* slots, 
     if (st) return st;
     st = begin_outputs(c, s, &set, &dout, &dout2);
     if (st) return st;
-    BcHostSync hs = {in_word(c, buf), id, prev ? done_word(c) : nullptr, prev};
+    BcHostSync hs = {in_word(c, buf), id, prev ? done_word(c) : nullptr, prev, nullptr};
     st = append_book_only(c, slots, n, s, true, &hs);
     if (st) return st;
     c->done_issued = prev;       // that kernel vouches for every step before this one ...
@@ -972,24 +1008,66 @@ bc_status bc_fill_step_host(bc_cache* c, int32_t layer, const int32_t* slots, in
   if (st) return st;
   const size_t qb = (size_t)n * c->cfg.q_heads * c->cfg.head_dim * 2;
   const size_t ob = (c->cfg.flags & BC_FLAG_OUT_F32) ? qb * 2 : qb;
-  // as in bc_decode_step_host: the append's bookkeeping first (when its rows go out in a launch of their own)
+  void *dq, *dk, *dv, *dbq, *dbk, *dbv, *dout, *dout2;
+  int buf, buf2, set;
+  const bool paired_kernel = !(c->cfg.flags & BC_FLAG_ATTN_REFERENCE) && c->cfg.q_heads / c->cfg.kv_heads <= 8;
+  if (paired_kernel && c->cfg.layers == 1 && (c->cfg.flags & BC_FLAG_HOST_PIPELINED) && stream_wait_value() && stream_write_value()) {
+    // Ordered by words, like the regular step (see bc_decode_step_host): the bookkeeping kernel polls the words of
+    // both sets of inputs; the caller's stream carries the kernels of bc_fill_step and nothing else.
+    if ((c->pending.valid && !c->pending.word_seq) || c->host_stream != s) {
+      st = flush_pending(c);
+      if (st) return st;
+      c->host_stream = s;
+    }
+    const int32_t prev = c->host_seq;
+    int32_t id = prev + 1;
+    if (id == 0) id = 1;
+    st = stage_inputs(c, n, q_host, k_host, v_host, s, &buf, &dq, &dk, &dv, id);
+    if (st) return st;
+    st = stage_inputs(c, n, bq_host, bk_host, bv_host, s, &buf2, &dbq, &dbk, &dbv, id);
+    if (st) return st;
+    st = begin_outputs(c, s, &set, &dout, &dout2);
+    if (st) return st;
+    BcHostSync hs = {in_word(c, buf), id, prev ? done_word(c) : nullptr, prev, in_word(c, buf2)};
+    st = append_book_only(c, slots, n, s, true, &hs);
+    if (st) return st;
+    c->done_issued = prev;
+    st = flush_pending(c);
+    if (st) return st;
+    c->host_seq = id;
+    st = decode_step_attn(c, layer, slots, n, dq, dk, dv, dout, sm_scale, s, 1, dbq, dbk, dbv, dout2);
+    if (st) return st;
+    st = bc_compress(c, layer, slots, n, dbk, dbv, stream);
+    if (st) return st;
+    bc_cache::Pending p;
+    p.valid = true; p.set = set; p.out_host = out_host; p.out2_host = out_beacon_host; p.bytes = ob; p.stream = s; p.word_seq = id;
+    c->pending = p;
+    return BC_OK;
+  }
+  // as in bc_decode_step_host: the append's bookkeeping first (when its rows go out in a launch of their own, or
+  // when the attention kernel takes them from the inputs)
   const bool rows_apart = (size_t)n * c->geom.entry_bytes > kFusedRowBytes;
   bool book_done = false;
-  if (layer == 0 && rows_apart) {
-    st = append_book_only(c, slots, n, s);
+  if (layer == 0 && (rows_apart || paired_kernel)) {
+    st = append_book_only(c, slots, n, s, paired_kernel);
     if (st) return st;
     book_done = true;
   }
   st = flush_pending(c);
   if (st) return st;
-  void *dq, *dk, *dv, *dbq, *dbk, *dbv, *dout, *dout2;
-  int buf, buf2, set;
   st = stage_inputs(c, n, q_host, k_host, v_host, s, &buf, &dq, &dk, &dv);
   if (st) return st;
   st = stage_inputs(c, n, bq_host, bk_host, bv_host, s, &buf2, &dbq, &dbk, &dbv);
   if (st) return st;
   st = begin_outputs(c, s, &set, &dout, &dout2);
   if (st) return st;
+  if (paired_kernel) {   // one attention launch appends the token's entry and serves both sets of rows
+    st = decode_step_attn(c, layer, slots, n, dq, dk, dv, dout, sm_scale, s, 1, dbq, dbk, dbv, dout2);
+    if (st) return st;
+    st = bc_compress(c, layer, slots, n, dbk, dbv, stream);
+    if (st) return st;
+    return close_step(c, s, set, buf, buf2, out_host, out_beacon_host, ob);
+  }
   if (book_done || (layer > 0 && rows_apart)) {   // the rows of this layer (the bookkeeping is done, or was done on layer 0)
     BC_CUDA(c, bc_launch_write_rows(c->meta, c->geom, layer_base(c, layer), work_ptr<int32_t>(c, c->wl.append_row[c->append_set]),
                                     work_ptr<int32_t>(c, c->wl.append_pos[c->append_set]), dk, dv, n, s));

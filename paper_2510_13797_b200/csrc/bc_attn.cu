@@ -331,14 +331,16 @@ __device__ __forceinline__ void combine_pieces(const float* part_o, const float*
 // fragment) and its beacon's (rows 8..8+G-1), which share one pass over the cache: the step whose token
 // fills the window and the encoding of the beacon that follows it (Algorithm 1) read the same entries.
 // The beacon's rows also see the extra entry (the beacon's own K/V).  Needs G <= 8 and is compiled
-// on the 16-row path (G_LE_8 = false); results go to out (token) and out2 (beacon).
+// on the 16-row path (G_LE_8 = false); results go to out (token) and out2 (beacon).  FUSED and PAIR
+// together are the step that fills a window as one launch: the token's entry comes from the inputs as in
+// a regular fused step, and both sets of rows see it.
 // LAYERED: one launch for all layers of a call with layer = BC_ALL_LAYERS.  The grid is (blocks, layers):
 // the blocks of layer l + 1 are dispatched as those of layer l retire, so the layers follow one another
 // without a kernel boundary; each layer has its own ticket counters and partial buffers, because the last
 // blocks of one layer and the first of the next run side by side.
 template <int D, bool G_LE_8, bool FUSED, bool PAIR = false, bool SHORTW = false, bool LAYERED = false>
 __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams p_in) {
-  static_assert(!PAIR || (!G_LE_8 && !FUSED), "the paired form runs on the 16-row path without the fused append");
+  static_assert(!PAIR || !G_LE_8, "the paired form runs on the 16-row path");
   static_assert(!LAYERED || (!PAIR && !SHORTW), "the all-layers launch exists for the plain and the fused step");
   PipeParams p_layer;
   if constexpr (LAYERED) {
@@ -1301,7 +1303,8 @@ cudaError_t bc_attn_setup(int* sm_count) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  const cudaError_t r[20] = {opt_in_smem<128, true, false, false, false, true>(), opt_in_smem<128, false, false, false, false, true>(),
+  const cudaError_t r[22] = {opt_in_smem<128, false, true, true>(), opt_in_smem<64, false, true, true>(),
+                             opt_in_smem<128, true, false, false, false, true>(), opt_in_smem<128, false, false, false, false, true>(),
                              opt_in_smem<64, true, false, false, false, true>(), opt_in_smem<64, false, false, false, false, true>(),
                              opt_in_smem<128, true, true, false, false, true>(), opt_in_smem<128, false, true, false, false, true>(),
                              opt_in_smem<64, true, true, false, false, true>(), opt_in_smem<64, false, true, false, false, true>(),
@@ -1355,7 +1358,8 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
       else e = g8 ? launch_pipe<64, true, false, false, false, true>(p, s) : launch_pipe<64, false, false, false, false, true>(p, s);
     }
   } else if (a.q2 != nullptr) {   // the paired form (token and beacon queries in one pass); the caller has checked G <= 8
-    e = g.head_dim == 128 ? launch_pipe<128, false, false, true>(p, s) : launch_pipe<64, false, false, true>(p, s);
+    if (fused) e = g.head_dim == 128 ? launch_pipe<128, false, true, true>(p, s) : launch_pipe<64, false, true, true>(p, s);
+    else e = g.head_dim == 128 ? launch_pipe<128, false, false, true>(p, s) : launch_pipe<64, false, false, true>(p, s);
   } else if (shortw) {
     e = fused ? launch_pipe<128, true, true, false, true>(p, s) : launch_pipe<128, true, false, false, true>(p, s);
   } else if (fused) {

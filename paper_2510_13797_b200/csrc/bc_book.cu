@@ -136,9 +136,10 @@ k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
     if (hs.in_word != nullptr) {
       inputs_in = false;
       for (uint32_t polls = 0; polls < (1u << 21); ++polls) {
-        int seen;
+        int seen, seen2 = hs.in_seq;
         asm volatile("ld.acquire.sys.global.s32 %0, [%1];" : "=r"(seen) : "l"(hs.in_word) : "memory");
-        if (seen == hs.in_seq) { inputs_in = true; break; }
+        if (hs.in_word2 != nullptr) asm volatile("ld.acquire.sys.global.s32 %0, [%1];" : "=r"(seen2) : "l"(hs.in_word2) : "memory");
+        if (seen == hs.in_seq && seen2 == hs.in_seq) { inputs_in = true; break; }
         __nanosleep(100);
       }
       if (!inputs_in && m.status[0] == 0) {
@@ -551,7 +552,7 @@ cudaError_t launch_book_overlapped(void (*kernel)(KArgs...), cudaStream_t s, Arg
 cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                   int32_t* dst_pos, const BcGeom& g, uint8_t* pool_layer, const void* k, const void* v,
                                   cudaStream_t s, int32_t* plan, int32_t* flag, int32_t epoch, const BcHostSync* hs) {
-  const BcHostSync none = {nullptr, 0, nullptr, 0};
+  const BcHostSync none = {nullptr, 0, nullptr, 0, nullptr};
   if (k == nullptr)   // the rows follow in a launch of their own (ordinary order: it waits for everything before it)
     return launch_book_overlapped(k_append_book, s, m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)nullptr,
                                   (const uint8_t*)nullptr, plan, flag, epoch, hs ? *hs : none);

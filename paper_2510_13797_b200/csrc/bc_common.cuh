@@ -70,6 +70,7 @@ struct BcHostSync {
   int32_t in_seq;
   int32_t* done_word;       // NULL: no store
   int32_t done_seq;
+  const int32_t* in_word2;  // the step that fills a window has two sets of inputs (token, beacon); NULL: one
 };
 cudaError_t bc_launch_host_steps_done(int32_t* done_word, int32_t seq, cudaStream_t s);
 cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,

@@ -84,6 +84,11 @@ class DecodeDriver:
         c, j = self.cache, self.t % self.ring
         if self.paired and self.c > 1 and (self.t + 1) % self.c == 0:
             b = ((self.t + 1) // self.c) % self.bring
+            if self.fused:      # append inside the paired attention launch
+                c.bc_fill_step(0, self.slots, self.q[j], self.k[j], self.v[j], self.bq[b], self.bk[b], self.bv[b], self.out, self.out_b,
+                               self.w.sm_scale)
+                self.t += 1
+                return True
             c.bc_append(0, self.slots, self.k[j], self.v[j])
             c.bc_decode_attn_pair(0, self.slots, self.q[j], self.out, self.bq[b], self.out_b, self.w.sm_scale, self.bk[b], self.bv[b])
             self.t += 1

@@ -257,3 +257,69 @@ def test_pipelined_host_steps_with_device_synchronisations_in_between():
     for o, r, what, _ in pending:
         assert_close(o, r, what)
     pair.check_state()
+
+
+def _run_fill_steps(pair, g, slots, c, steps, sm_scale, what):
+    """Regular steps through bc_decode_step, window-filling steps through bc_fill_step; every output against the
+    oracle, the bookkeeping against the model."""
+    n = len(slots)
+    sl = torch.tensor(slots, dtype=torch.int32, device=DEV)
+    L = pair.L
+    for step in range(1, steps + 1):
+        fill = step % c == 0
+        for l in range(L):
+            q, k, v = randn_bf16(g, (n, pair.Hq, pair.D), DEV), randn_bf16(g, (n, pair.Hkv, pair.D), DEV), randn_bf16(g, (n, pair.Hkv, pair.D), DEV)
+            out = torch.full((n, pair.Hq, pair.D), float("nan"), dtype=torch.bfloat16, device=DEV)
+            if fill:
+                bq, bk, bv = randn_bf16(g, (n, pair.Hq, pair.D), DEV), randn_bf16(g, (n, pair.Hkv, pair.D), DEV), randn_bf16(g, (n, pair.Hkv, pair.D), DEV)
+                out_b = torch.full_like(out, float("nan"))
+                pair.gpu.bc_fill_step(l, sl, q, k, v, bq, bk, bv, out, out_b, sm_scale)
+            else:
+                pair.gpu.bc_decode_step(l, sl, q, k, v, out, sm_scale)
+            torch.cuda.synchronize()
+            if l == 0:
+                assert pair.model.append(slots) == [OK] * n
+            for i, s in enumerate(slots):
+                pair.seqs[s].append(l, f64(k)[i], f64(v)[i])
+            ref = np.stack([pair.seqs[s].attend(l, f64(q)[i], sm_scale) for i, s in enumerate(slots)])
+            assert_close(out, ref, f"{what}: step {step} layer {l} token rows")
+            if fill:
+                ref_b = np.stack([pair.seqs[s].beacon_attend(l, f64(bq)[i], f64(bk)[i], f64(bv)[i], sm_scale) for i, s in enumerate(slots)])
+                assert_close(out_b, ref_b, f"{what}: step {step} layer {l} beacon rows")
+                if l == L - 1:
+                    assert pair.model.compress(slots) == [OK] * n
+                for i, s in enumerate(slots):
+                    pair.seqs[s].compress(l, f64(bk)[i], f64(bv)[i])
+        pair.check_state()
+    for l in range(L):
+        for s in slots:
+            pair.check_content(l, s)
+
+
+@pytest.mark.parametrize("L,Hkv,G,D,ps,c", [(1, 2, 4, 128, 16, 8), (2, 8, 4, 128, 4, 4), (1, 1, 1, 64, 16, 16), (1, 2, 6, 128, 8, 2),
+                                            (1, 4, 8, 64, 16, 3), (1, 1, 12, 128, 16, 4)])
+def test_fill_step_matches_oracle_small(L, Hkv, G, D, ps, c):
+    """bc_fill_step on short ragged sequences (an empty prompt among them), two layers, G = 12 (the three-call
+    route) and the reference-free paired kernel with the append inside."""
+    pair = Pair(L, Hkv, Hkv * G, D, ps, max_seqs=4, num_pages=4 * (200 // ps + 12), max_pages_per_seq=200 // ps + 12)
+    g = _gen(51)
+    slots, plens = [0, 1, 2, 3], [33, 0, 100, 7]
+    assert pair.open(slots, plens, [c] * 4) == [OK] * 4
+    for l in range(L):
+        pair.prefill(l, slots, plens, randn_bf16(g, (sum(plens), Hkv, D), DEV), randn_bf16(g, (sum(plens), Hkv, D), DEV))
+    _run_fill_steps(pair, g, slots, c, 3 * c + 1, 1.0 / math.sqrt(D), f"G={G}")
+
+
+@pytest.mark.parametrize("ctas", [0, 1, 2, 5, 37])
+def test_fill_step_split_over_blocks(ctas):
+    """Long sequences cut into pieces by several blocks, the window's last tile (with the entry that comes from
+    the inputs) owned by one block and the pieces merged by another; repeated launches."""
+    Hkv, G, D, ps, c = 8, 4, 128, 16, 16
+    pair = Pair(1, Hkv, Hkv * G, D, ps, max_seqs=5, num_pages=700, max_pages_per_seq=160)
+    if ctas:
+        pair.gpu.bc_set_attn_ctas(ctas)
+    g = _gen(53)
+    slots, plens = [0, 1, 2, 3, 4], [1500, 40, 900, 2047, 3]
+    assert pair.open(slots, plens, [c] * 5) == [OK] * 5
+    pair.prefill(0, slots, plens, randn_bf16(g, (sum(plens), Hkv, D), DEV), randn_bf16(g, (sum(plens), Hkv, D), DEV))
+    _run_fill_steps(pair, g, slots, c, 2 * c + 2, 0.09, f"ctas={ctas}")

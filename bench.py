@@ -1021,8 +1021,9 @@ def report_model(args):
     print(json.dumps({"workload": f"model: random-weight decoder of the 1.5B shape, batch {Bn}, prompt 512, {N} generated tokens "
                                   "per sequence, one CUDA graph per token step and per beacon step"
                                   + ("" if args.no_pair else "; the beacon is encoded in the same 2-token pass as the token that fills the window"),
-                      "rope_and_qkv_split": "PyTorch operators" if args.torch_rope else
-                      "bc_rope_split / bc_rope_decode_step (a token step: the rotation kernel, then one kernel that appends and attends)",
+                      "operators_between_the_gemms": "PyTorch operators" if args.torch_rope else
+                      "the library's kernels: bc_rope_decode_step / bc_rope_split + bc_fill_step (rotation, append, attention), "
+                      "bc_add_rmsnorm (residual add and norm), bc_swiglu, bc_argmax; the GEMMs and the embedding lookup are PyTorch's",
                       "paper_latency_table_qwen_sr": {"2": 1.990, "4": 1.546, "8": 1.593, "16": 1.646, "32": 1.468},
                       "rows": rows}))
 
@@ -1077,7 +1078,7 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--torch-rope", action="store_true",
-                    help="--workload model: rotary embedding and QKV split with PyTorch operators instead of the library's kernel")
+                    help="--workload model: rotary embedding, QKV split, norms, gated activation and argmax with PyTorch operators instead of the library's kernels")
     ap.add_argument("--no-pair", action="store_true", help="beacon steps as a second attention pass instead of bc_decode_attn_pair")
     ap.add_argument("--pair", action="store_true", help="ragged workload: pair the beacon steps too (off by default there)")
     ap.add_argument("--fused", action="store_true", help="--timeline: regular steps through bc_decode_step")

@@ -5,10 +5,11 @@ What is measured with it: the time to generate N tokens per sequence with the un
 timing figure (its latency table: generation latency relative to the uncompressed teacher).
 
 Only the cache side (bc_append, bc_decode_attn, bc_compress) is this repository's product.  The
-rest of the forward pass -- embeddings, RMSNorm, the QKV / output / MLP projections, the LM head
-and greedy sampling -- are plain PyTorch operators standing in for a model; the rotary embedding and the
-split of the packed QKV rows are the library's kernel (bc_rope_split, bc_rope_decode_step) unless
-lib_rope=False, which puts the PyTorch operators back for comparison
+rest of the forward pass -- the embedding lookup and the QKV / output / MLP / LM-head projections (GEMMs) --
+are plain PyTorch operators standing in for a model; the rotary embedding and the split of the packed QKV
+rows (bc_rope_split, bc_rope_decode_step), the residual add with RMSNorm (bc_add_rmsnorm), the gated MLP
+activation (bc_swiglu) and the greedy choice (bc_argmax) are the library's kernels unless lib_rope=False,
+which puts the PyTorch operators back for comparison
 (random weights: the token stream is meaningless, the shapes and the data flow are real).  Every
 sampled token is fed back, and when a window fills, the beacon token's forward pass runs through
 the same layers: its query attends with its own K/V as the extra entry, then the window is evicted
@@ -69,6 +70,8 @@ class ToyDecoder:
         # the library's rotation takes one position per row: rows [0, B) at pos, rows [B, 2B) (the beacons of a paired step) at pos + 1
         self.posv = torch.cat((torch.full((batch,), prompt_len, dtype=torch.int32, device=self.dev),
                                torch.full((batch,), prompt_len + 1, dtype=torch.int32, device=self.dev)))
+        self.xbuf = torch.empty((2 * batch, hidden), dtype=torch.bfloat16, device=self.dev)    # norm output
+        self.actbuf = torch.empty((2 * batch, mlp), dtype=torch.bfloat16, device=self.dev)     # gated MLP activation
         self.q2 = self.cache.new_out(2 * batch)
         self.k2 = torch.empty((2 * batch, kv_heads, head_dim), dtype=torch.bfloat16, device=self.dev)
         self.v2 = torch.empty_like(self.k2)
@@ -105,63 +108,86 @@ class ToyDecoder:
         if self.trace is not None:
             self.trace.append((kind, layer, qkv.clone(), self.posv[:n].clone(), out.clone()))
 
+    def _pre(self, h, delta):
+        """Residual add and the norm in front of a block: returns (h + delta, norm(h + delta))."""
+        if self.lib_rope:
+            x = self.xbuf[:h.shape[0]]
+            B.bc_add_rmsnorm(h, delta, None, 1e-6, h, x)          # in place on the residual stream
+            return h, x
+        if delta is not None:
+            h = h + delta
+        return h, self._norm(h)
+
+    def _mlp_act(self, gu):
+        if self.lib_rope:
+            act = self.actbuf[:gu.shape[0]]
+            B.bc_swiglu(gu, act)
+            return act
+        gate, up = gu.chunk(2, dim=-1)
+        return torch.nn.functional.silu(gate) * up
+
+    def _sample(self, h, delta):
+        """Final norm, LM head, greedy choice into self.tok."""
+        _, x = self._pre(h, delta)
+        logits = x @ self.head
+        if self.lib_rope:
+            B.bc_argmax(logits, self.tok)
+        else:
+            self.tok.copy_(torch.argmax(logits, dim=-1))
+
     def _forward(self, ids, beacon):
-        h = self.emb[ids]
+        h, delta = self.emb[ids], None
         Hq, Hkv, D = self.Hq, self.Hkv, self.D
         for l in range(self.L):
-            qkv = self._norm(h) @ self.wqkv[l]
+            h, x = self._pre(h, delta)
+            qkv = x @ self.wqkv[l]
             if self.lib_rope and not beacon:    # rotation, then the append and the attention in one kernel
                 self.cache.bc_rope_decode_step(l, self.slots, qkv, self.posv[:self.B], self.theta, self.attn_out, self.scale)
                 self._record("token", l, qkv, self.B, self.attn_out)
-                h = h + self.attn_out.view(-1, Hq * D) @ self.wo[l]
-                gu = self._norm(h) @ self.wgu[l]
-                gate, up = gu.chunk(2, dim=-1)
-                h = h + (torch.nn.functional.silu(gate) * up) @ self.wdown[l]
-                continue
-            q, k, v = self._split(qkv)
-            if beacon:      # the beacon's query sees the cache plus its own entry; then the window goes
-                self.cache.bc_decode_attn(l, self.slots, q, self.attn_out, self.scale, k, v)
-                self.cache.bc_compress(l, self.slots, k, v)
-                self._record("beacon", l, qkv, self.B, self.attn_out)
             else:
-                self.cache.bc_append(l, self.slots, k, v)
-                self.cache.bc_decode_attn(l, self.slots, q, self.attn_out, self.scale)
-            h = h + self.attn_out.view(-1, Hq * D) @ self.wo[l]
-            gu = self._norm(h) @ self.wgu[l]
-            gate, up = gu.chunk(2, dim=-1)
-            h = h + (torch.nn.functional.silu(gate) * up) @ self.wdown[l]
-        return h
+                q, k, v = self._split(qkv)
+                if beacon:      # the beacon's query sees the cache plus its own entry; then the window goes
+                    self.cache.bc_decode_attn(l, self.slots, q, self.attn_out, self.scale, k, v)
+                    self.cache.bc_compress(l, self.slots, k, v)
+                    self._record("beacon", l, qkv, self.B, self.attn_out)
+                else:
+                    self.cache.bc_append(l, self.slots, k, v)
+                    self.cache.bc_decode_attn(l, self.slots, q, self.attn_out, self.scale)
+            h, x = self._pre(h, self.attn_out.view(-1, Hq * D) @ self.wo[l])
+            delta = self._mlp_act(x @ self.wgu[l]) @ self.wdown[l]
+        return h, delta
 
     def _forward_pair(self):
         """The token that fills the window and the beacon as one 2-token pass: rows [0, B) are the
         tokens (position pos), rows [B, 2B) the beacons (position pos + 1).  Per layer the token's entry
         is appended, both query sets attend in one pass over the cache (the beacon also sees its own
-        entry), and the window is evicted."""
+        entry), and the window is evicted (bc_fill_step; with lib_rope=False the three separate calls)."""
         Bn, Hq, Hkv, D = self.B, self.Hq, self.Hkv, self.D
-        h = self.emb[torch.cat((self.tok, torch.full_like(self.tok, self.V)))]
+        h, delta = self.emb[torch.cat((self.tok, torch.full_like(self.tok, self.V)))], None
         offset = torch.cat((torch.zeros(Bn, device=self.dev), torch.ones(Bn, device=self.dev)))
         for l in range(self.L):
-            qkv = self._norm(h) @ self.wqkv[l]
+            h, x = self._pre(h, delta)
+            qkv = x @ self.wqkv[l]
             q, k, v = self._split(qkv, offset)
-            self.cache.bc_append(l, self.slots, k[:Bn], v[:Bn])
-            self.cache.bc_decode_attn_pair(l, self.slots, q[:Bn], self.attn_out2[:Bn], q[Bn:], self.attn_out2[Bn:], self.scale,
-                                           k[Bn:], v[Bn:])
-            self.cache.bc_compress(l, self.slots, k[Bn:], v[Bn:])
+            if self.lib_rope:
+                self.cache.bc_fill_step(l, self.slots, q[:Bn], k[:Bn], v[:Bn], q[Bn:], k[Bn:], v[Bn:], self.attn_out2[:Bn],
+                                        self.attn_out2[Bn:], self.scale)
+            else:
+                self.cache.bc_append(l, self.slots, k[:Bn], v[:Bn])
+                self.cache.bc_decode_attn_pair(l, self.slots, q[:Bn], self.attn_out2[:Bn], q[Bn:], self.attn_out2[Bn:], self.scale,
+                                               k[Bn:], v[Bn:])
+                self.cache.bc_compress(l, self.slots, k[Bn:], v[Bn:])
             self._record("pair", l, qkv, 2 * Bn, self.attn_out2)
-            h = h + self.attn_out2.view(-1, Hq * D) @ self.wo[l]
-            gu = self._norm(h) @ self.wgu[l]
-            gate, up = gu.chunk(2, dim=-1)
-            h = h + (torch.nn.functional.silu(gate) * up) @ self.wdown[l]
-        return h[:Bn]
+            h, x = self._pre(h, self.attn_out2.view(-1, Hq * D) @ self.wo[l])
+            delta = self._mlp_act(x @ self.wgu[l]) @ self.wdown[l]
+        return h[:Bn], delta[:Bn]
 
     def _fill_step(self):
-        h = self._forward_pair()
-        self.tok.copy_(torch.argmax(self._norm(h) @ self.head, dim=-1))
+        self._sample(*self._forward_pair())
         self.pos.add_(2); self.posv.add_(2)
 
     def _token_step(self):
-        h = self._forward(self.tok, beacon=False)
-        self.tok.copy_(torch.argmax(self._norm(h) @ self.head, dim=-1))
+        self._sample(*self._forward(self.tok, beacon=False))
         self.pos.add_(1); self.posv.add_(1)
 
     def _beacon_step(self):

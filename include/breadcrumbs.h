@@ -305,6 +305,26 @@ BC_API bc_status bc_fill_step(bc_cache* cache, int32_t layer, const int32_t* slo
                               const void* k, const void* v, const void* beacon_q, const void* beacon_k,
                               const void* beacon_v, void* out, void* out_beacon, float sm_scale, void* stream);
 
+/* ---- the operators of a decoder layer between its GEMMs and the cache calls --------------------
+ * (Experimental Setup: the paper's models are pre-norm decoders with RMSNorm, a SiLU-gated MLP and a
+ * residual stream in bf16; Algorithm 1 samples the next token, the latency protocol greedily.)
+ * Stateless: no cache handle, nothing is latched; errors are the return value.  All pointers device,
+ * 16-byte aligned; one kernel launch each, asynchronous on `stream`, ordinary stream order.
+ *
+ * bc_add_rmsnorm: h' = h + delta rounded to bf16 (delta NULL: h' = h), stored to h_out (NULL: not
+ *   stored; h_out may be h itself), and normed_out = h' / sqrt(mean(h'^2) + eps) * weight (weight
+ *   NULL: ones), the mean over the hidden dimension of the stored bf16 values, arithmetic in fp32.
+ *   h, delta, h_out, normed_out [n, hidden] bf16, weight [hidden] bf16; hidden a multiple of 8 and
+ *   <= 8192 (else BC_ERR_UNSUPPORTED); eps >= 0.
+ * bc_swiglu: out[r, j] = silu(gate_up[r, j]) * gate_up[r, m + j], silu(x) = x / (1 + exp(-x));
+ *   gate_up [n, 2 m] bf16 (gate in the first half of a row), out [n, m] bf16; m a multiple of 8.
+ * bc_argmax: out[r] = the lowest index at which row r of logits [n, vocab] bf16 attains its maximum
+ *   (int64, the type token ids usually have); vocab a multiple of 8. */
+BC_API bc_status bc_add_rmsnorm(const void* h, const void* delta, const void* weight, int32_t n, int32_t hidden,
+                                float eps, void* h_out, void* normed_out, void* stream);
+BC_API bc_status bc_swiglu(const void* gate_up, int32_t n, int32_t m, void* out, void* stream);
+BC_API bc_status bc_argmax(const void* logits, int32_t n, int32_t vocab, int64_t* out, void* stream);
+
 /* Limits of bc_decode_attn_static. */
 #define BC_STATIC_MAX_BATCH 128   /* sequences per call */
 #define BC_STATIC_MAX_CTAS 160    /* thread blocks it will use at most */

@@ -85,6 +85,9 @@ SYMBOLS = {
     "bc_profile_read": (_I32, [_P, C.POINTER(_I32), C.POINTER(_F)]),
     "bc_probe_read_stream": (_I32, [_P, C.c_size_t, _P]),
     "bc_fill_step": (_I32, [_P, _I32, _P, _I32, _P, _P, _P, _P, _P, _P, _P, _P, _F, _P]),
+    "bc_add_rmsnorm": (_I32, [_P, _P, _P, _I32, _I32, _F, _P, _P, _P]),
+    "bc_swiglu": (_I32, [_P, _I32, _I32, _P, _P]),
+    "bc_argmax": (_I32, [_P, _I32, _I32, _P, _P]),
     "bc_rope_split": (_I32, [_P, _P, _P, _I32, _F, _P, _P, _P, _P]),
     "bc_rope_decode_step": (_I32, [_P, _I32, _P, _I32, _P, _P, _F, _P, _F, _P]),
     "bc_kernel_launches": (_I64, [_P]),
@@ -324,6 +327,23 @@ def bc_mask_attn_forward(prompt_lens, token_lens, c, prompt_k, prompt_v, tok_q, 
 def bc_probe_read_stream(buf, stream=None):
     """Reads the CUDA tensor `buf` once with the attention kernel's copy pattern (breadcrumbs.h)."""
     _check(lib().bc_probe_read_stream(_ptr(buf), buf.numel() * buf.element_size(), _stream(stream)), "bc_probe_read_stream")
+
+
+def bc_add_rmsnorm(h, delta, weight, eps, h_out, normed_out, stream=None):
+    """h' = h + delta (bf16), normed_out = rmsnorm(h') * weight (breadcrumbs.h); delta, weight, h_out may be None."""
+    n, hidden = h.shape[0], h.shape[-1]
+    _check(lib().bc_add_rmsnorm(_ptr(h), _ptr(delta), _ptr(weight), n, hidden, eps, _ptr(h_out), _ptr(normed_out), _stream(stream)),
+           "bc_add_rmsnorm")
+
+
+def bc_swiglu(gate_up, out, stream=None):
+    """out = silu(gate) * up for packed rows [gate | up] (breadcrumbs.h)."""
+    _check(lib().bc_swiglu(_ptr(gate_up), gate_up.shape[0], gate_up.shape[-1] // 2, _ptr(out), _stream(stream)), "bc_swiglu")
+
+
+def bc_argmax(logits, out, stream=None):
+    """out[r] (int64) = lowest index of the maximum of row r of bf16 logits (breadcrumbs.h)."""
+    _check(lib().bc_argmax(_ptr(logits), logits.shape[0], logits.shape[-1], _ptr(out), _stream(stream)), "bc_argmax")
 
 
 def bc_distill_loss(cu_rows, student_logits, teacher_idx, teacher_logprob, with_grad=False, stream=None):

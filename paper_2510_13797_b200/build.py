@@ -16,7 +16,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(PKG_DIR, "libbreadcrumbs.so")
-SOURCES = ["bc_api.cu", "bc_book.cu", "bc_attn.cu", "bc_mask_attn.cu", "bc_distill.cu", "bc_rope.cu"]
+SOURCES = ["bc_api.cu", "bc_book.cu", "bc_attn.cu", "bc_mask_attn.cu", "bc_distill.cu", "bc_rope.cu", "bc_model_ops.cu"]
 
 
 def _nvcc():

@@ -649,6 +649,31 @@ bc_status bc_rope_split(bc_cache* c, const void* qkv, const int32_t* positions, 
   return BC_OK;
 }
 
+bc_status bc_add_rmsnorm(const void* h, const void* delta, const void* weight, int32_t n, int32_t hidden, float eps, void* h_out,
+                         void* normed_out, void* stream) {
+  if (!h || !normed_out || n <= 0 || hidden <= 0 || !(eps >= 0.f)) return BC_ERR_INVALID_ARG;
+  if (!aligned16(h) || !aligned16(normed_out) || (delta && !aligned16(delta)) || (weight && !aligned16(weight)) ||
+      (h_out && !aligned16(h_out)))
+    return BC_ERR_INVALID_ARG;
+  if (hidden % 8 || hidden > bc_rmsnorm_max_hidden()) return BC_ERR_UNSUPPORTED;
+  if (bc_launch_add_rmsnorm(h, delta, weight, n, hidden, eps, h_out, normed_out, (cudaStream_t)stream) != cudaSuccess) return BC_ERR_CUDA;
+  return BC_OK;
+}
+
+bc_status bc_swiglu(const void* gate_up, int32_t n, int32_t m, void* out, void* stream) {
+  if (!gate_up || !out || n <= 0 || m <= 0 || !aligned16(gate_up) || !aligned16(out)) return BC_ERR_INVALID_ARG;
+  if (m % 8) return BC_ERR_UNSUPPORTED;
+  if (bc_launch_swiglu(gate_up, n, m, out, (cudaStream_t)stream) != cudaSuccess) return BC_ERR_CUDA;
+  return BC_OK;
+}
+
+bc_status bc_argmax(const void* logits, int32_t n, int32_t vocab, int64_t* out, void* stream) {
+  if (!logits || !out || n <= 0 || vocab <= 0 || !aligned16(logits)) return BC_ERR_INVALID_ARG;
+  if (vocab % 8) return BC_ERR_UNSUPPORTED;
+  if (bc_launch_argmax(logits, n, vocab, reinterpret_cast<long long*>(out), (cudaStream_t)stream) != cudaSuccess) return BC_ERR_CUDA;
+  return BC_OK;
+}
+
 bc_status bc_rope_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32_t n, const void* qkv,
                               const int32_t* positions, float theta, void* out, float sm_scale, void* stream) {
   bc_status st = check_batch(c, layer, slots, n);

@@ -145,6 +145,12 @@ struct BcFusedAppend {
 // the same launch appends the step's new entries first.  *launches gets the number of kernels.
 cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a, const BcFusedAppend* fused,
                            cudaStream_t s, cudaEvent_t ev_start, cudaEvent_t ev_stop, int* launches);
+// Decoder-layer operators around the cache calls (bc_model_ops.cu).
+cudaError_t bc_launch_add_rmsnorm(const void* h, const void* delta, const void* weight, int n, int hidden, float eps, void* h_out,
+                                  void* normed, cudaStream_t s);
+cudaError_t bc_launch_swiglu(const void* gate_up, int n, int m, void* out, cudaStream_t s);
+cudaError_t bc_launch_argmax(const void* logits, int n, int vocab, long long* out, cudaStream_t s);
+int bc_rmsnorm_max_hidden();
 // Rotary embedding of the q and k heads of n packed QKV rows, split into three contiguous arrays.
 cudaError_t bc_launch_rope_split(const void* qkv, const int32_t* positions, int n, int q_heads, int kv_heads, int head_dim,
                                  double theta, void* q_out, void* k_out, void* v_out, cudaStream_t s);

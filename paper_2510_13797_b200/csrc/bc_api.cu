@@ -282,7 +282,6 @@ bc_status decode_step_attn(bc_cache* c, int layer, const int32_t* slots, int n, 
   f.pool_layer = layer_base(c, layer);
   f.flag = work_ptr<int32_t>(c, c->wl.book_flag);
   f.plan = work_ptr<int32_t>(c, c->wl.plan[c->append_set]);   // left by append_book_only(with_plan) of this step
-  f.do_book = 0;
   f.call = c->append_call;
   f.epoch = step_epoch(c->append_call);
   const bc_status st = attn_impl(c, layer, slots, n, q, out, sm_scale, beacon_k, beacon_v, s, &f, beacon_q, out_beacon, layers);
@@ -629,8 +628,7 @@ bc_status bc_decode_step(bc_cache* c, int32_t layer, const int32_t* slots, int32
   // The bookkeeping runs as its own one-block kernel, which may start under the previous attention
   // kernel's last blocks; the rows are written by the attention kernel itself (its service warps),
   // which takes the new entries from the inputs.  So a step costs one full-size launch and no
-  // row-writing launch.  (The kernel can also run the bookkeeping in its block 0, do_book = 1: that
-  // form starts every other block late and is not used here.)
+  // row-writing launch.
   if (layer == 0) {
     st = append_book_only(c, slots, n, s, true);
     if (st) return st;

@@ -203,7 +203,6 @@ struct FusedArgs {
   const int32_t* plan;    // the plan the bookkeeping kernel of the step left (bc_decode_step), or NULL
   int32_t* flag;          // set to `epoch` by block 0 once the bookkeeping of this launch is done
   int32_t epoch;
-  int32_t do_book;        // 1 on the layer-0 call of a step
   int64_t call;           // index of the bookkeeping call (for the error latch)
 };
 
@@ -321,8 +320,8 @@ __device__ __forceinline__ void combine_pieces(const float* part_o, const float*
   }
 }
 
-// FUSED: the launch also appends the step's new entries (bc_decode_step).  Block 0 runs the append
-// bookkeeping first and publishes a flag; the others wait for it (block 0 waits for nobody).  The new
+// FUSED: the launch also appends the step's new entries (bc_decode_step).  The step's bookkeeping kernel,
+// enqueued just ahead, leaves the plan and publishes a flag; the blocks of this kernel poll it.  The new
 // rows are not read back from the pool: the bulk copy of a sequence's last tile leaves the new row
 // out, the consumer warps write it into the shared-memory tile straight from the input, and the
 // service warp stores it to the pool for the steps to come.  So the step costs no second and third
@@ -422,7 +421,7 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   // kernel directly (the fused step, small batches whose rows the bookkeeping block writes itself, a
   // call right after open / close / restore): then the wait comes first and nothing is read early.
   bool early = !FUSED && p.early_meta;
-  if (FUSED && p.f.plan != nullptr && !p.f.do_book) {
+  if (FUSED && p.f.plan != nullptr) {
     // bc_decode_step: the kernel ahead is this step's bookkeeping kernel.  It is running (it is what let this
     // kernel begin) and stores the step's epoch to a flag word, with release semantics, as soon as its
     // results -- lengths, page-table column, row destinations, the plan -- are written; then it only waits
@@ -430,44 +429,19 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
     // acquire semantics makes those results visible here, so this kernel, too, can plan and stream settled
     // tiles while the previous step's last blocks finish.  If the flag does not show up in a while the
     // block simply waits for the kernel ahead to end, which makes everything visible the ordinary way.
-    __shared__ int sh_flag_seen;
+    volatile int* sh_flag_seen = s_abort + 6;   // a word of the block's own scratch: no static shared memory in this kernel
     if (tid == 0) {
       int seen = 0;
       for (uint32_t polls = 0; polls < 2048; ++polls) {
         if (ld_acquire(p.f.flag) == p.f.epoch) { seen = 1; break; }
         __nanosleep(40);
       }
-      sh_flag_seen = seen;
+      *sh_flag_seen = seen;
     }
     __syncthreads();
-    early = sh_flag_seen != 0;
+    early = *sh_flag_seen != 0;
   }
   if (!early) asm volatile("griddepcontrol.wait;" ::: "memory");
-
-  if (FUSED && p.f.do_book) {
-    __shared__ int sh_book_ok;
-    if (blockIdx.x == 0) {
-      append_book_block(p.m, p.a.slots, n, p.f.call, p.f.dst_row, p.f.dst_pos);
-      __syncthreads();
-      if (tid == 0) {
-        __threadfence();
-        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p.f.flag), "r"(p.f.epoch) : "memory");
-        sh_book_ok = 1;
-      }
-    } else if (tid == 0) {
-      int ok = 0;
-      for (uint32_t polls = 0; polls < kSpinLimit; ++polls) {
-        if (ld_acquire(p.f.flag) == p.f.epoch) { ok = 1; break; }
-        __nanosleep(32);
-      }
-      sh_book_ok = ok;
-    }
-    __syncthreads();
-    if (!sh_book_ok) {  // block 0 never reported: give up before anything is in flight
-      if (tid == 0 && p.m.status[0] == 0) { p.m.status[0] = BC_ERR_TIMEOUT; p.m.status[1] = -1; }
-      return;
-    }
-  }
 
   // ---- plan: tiles per sequence, prefix sums, this block's span --------------------------------
   // Each segment (prompt, beacons, window) starts a new tile, so a tile never straddles segments;
@@ -521,12 +495,11 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
   // programmatic stream serialisation -- the next step's bookkeeping -- may start on the first SM
   // that frees up instead of after this kernel's last block.  Kernels launched the ordinary way wait
   // for the whole grid as before.  The fused form goes on reading the rows' destinations (dst_row,
-  // dst_pos); the next step's bookkeeping fills the other of two sets, so it may start early as well --
-  // unless this launch did its own bookkeeping in block 0, whose flag word the next one would reuse.
+  // dst_pos); the next step's bookkeeping fills the other of two sets, so it may start early as well.
   // A fused step that started early lets its dependents go only once it has waited for the kernel ahead
   // (see wait_for_kernel_ahead): its service warps write pool rows, and at most two row-writing launches
   // may be alive at a time for the "settled" rule below to hold.
-  if (FUSED ? (!p.f.do_book && !early) : true) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (FUSED ? !early : true) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // With early_meta the wait for the kernel ahead is still to come: every role below executes it before it
   // touches anything but `slots` and the metadata -- the pool rows of this step, q, the extra entry, the
   // partial buffers and tickets this launch shares with the one before it, and every output.  So the plan
@@ -538,12 +511,9 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       if (FUSED) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     }
   };
-  // The block that ran the bookkeeping starts late; it takes no tiles, or it would finish last.
-  const int idle = (FUSED && p.f.do_book && gridDim.x > 1) ? 1 : 0;
-  const int n_ctas = (int)gridDim.x - idle;
-  if ((int)blockIdx.x < idle) return;
+  const int n_ctas = (int)gridDim.x;
   const int per = total_tiles / n_ctas, rem = total_tiles % n_ctas;
-  const int cta = (int)blockIdx.x - idle;
+  const int cta = (int)blockIdx.x;
   const int g0 = cta * per + min(cta, rem);
   const int g1 = g0 + per + (cta < rem ? 1 : 0);
   if (g0 >= g1) return;
@@ -1332,8 +1302,8 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
   if (fused) {
     p.f.new_k = static_cast<const uint8_t*>(fused->new_k); p.f.new_v = static_cast<const uint8_t*>(fused->new_v);
     p.f.dst_row = fused->dst_row; p.f.dst_pos = fused->dst_pos; p.f.pool_w = fused->pool_layer;
-    p.f.flag = fused->flag; p.f.epoch = fused->epoch; p.f.do_book = fused->do_book; p.f.call = fused->call;
-    p.f.plan = fused->do_book ? nullptr : fused->plan;
+    p.f.flag = fused->flag; p.f.epoch = fused->epoch; p.f.call = fused->call;
+    p.f.plan = fused->plan;
   }
   p.scale_log2 = a.sm_scale * 1.4426950408889634f;
   p.n_groups = kConsumerWarps / g.kv_heads;

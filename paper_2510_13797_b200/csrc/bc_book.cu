@@ -106,7 +106,14 @@ k_open(BcMeta m, const int32_t* __restrict__ slots, const int32_t* __restrict__ 
 // at once when nothing was overtaken.
 __device__ __forceinline__ void wait_for_overtaken_kernel() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-__global__ void __launch_bounds__(kBookThreads, 1)
+// WARP: launched as ONE warp, and then without a byte of shared memory.  The attention kernel's blocks hold an
+// SM's shared memory but for the kilobyte every block is charged, and nearly all registers of two of its four
+// sub-partitions; a one-warp block without shared memory still finds room beside such a block (measured), a
+// block of several warps or with shared memory of its own does not and has to wait for the first SM the
+// attention kernel leaves.  So the bookkeeping of a small batch begins as soon as the attention kernel ahead
+// has let its dependents go, and the next attention launch finds its plan and its flag waiting.
+template <bool WARP>
+__global__ void __launch_bounds__(WARP ? 32 : kBookThreads, 1)
 k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
               int32_t* dst_row, int32_t* dst_pos, BcGeom g, uint8_t* pool_layer, const uint8_t* k, const uint8_t* v,
               int32_t* plan, int32_t* flag, int32_t epoch, BcHostSync hs) {
@@ -119,13 +126,13 @@ k_append_book(BcMeta m, const int32_t* __restrict__ slots, int n, int64_t call,
     // It is cleared, and the clearing made visible device-wide, before any block of the dependent kernel
     // can exist.
     if (threadIdx.x == 0) { *reinterpret_cast<volatile int32_t*>(flag) = 0; __threadfence(); }
-    __syncthreads();
+    group_sync<WARP>();
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   }
   int tile_shift = 4;   // rows per tile of the attention kernel: 16 * (8 / kv_heads)
   while ((16 << (tile_shift - 4)) * g.kv_heads < 128) ++tile_shift;
-  append_book_block(m, slots, n, call, dst_row, dst_pos, plan, tile_shift);
-  __syncthreads();
+  append_book_block<WARP>(m, slots, n, call, dst_row, dst_pos, plan, tile_shift);
+  group_sync<WARP>();
   if (plan != nullptr && threadIdx.x == 0) {   // lengths, page-table column, row destinations and plan are written
     // A host-buffer step: q, k, v travel on the cache's copy stream, which writes the step's number to a word
     // behind the copy (a stream memory operation, not a kernel).  The flag below lets the attention kernel read
@@ -538,10 +545,11 @@ cudaError_t bc_launch_open(const BcMeta& m, const int32_t* slots, const int32_t*
 // enqueued before it -- which has read all the lengths it needs by the time it lets dependents go --
 // is still finishing its last blocks.  It waits for nothing of that kernel: it reads no output of it.
 // After any other predecessor the attribute changes nothing (no early trigger, ordinary order).
+constexpr int kWarpBookItems = 128;
 template <typename... KArgs, typename... Args>
-cudaError_t launch_book_overlapped(void (*kernel)(KArgs...), cudaStream_t s, Args... args) {
+cudaError_t launch_book_overlapped(void (*kernel)(KArgs...), cudaStream_t s, int threads, Args... args) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(1); cfg.blockDim = dim3(kBookThreads); cfg.dynamicSmemBytes = 0; cfg.stream = s;
+  cfg.gridDim = dim3(1); cfg.blockDim = dim3(threads); cfg.dynamicSmemBytes = 0; cfg.stream = s;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
@@ -553,10 +561,14 @@ cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, 
                                   int32_t* dst_pos, const BcGeom& g, uint8_t* pool_layer, const void* k, const void* v,
                                   cudaStream_t s, int32_t* plan, int32_t* flag, int32_t epoch, const BcHostSync* hs) {
   const BcHostSync none = {nullptr, 0, nullptr, 0, nullptr};
-  if (k == nullptr)   // the rows follow in a launch of their own (ordinary order: it waits for everything before it)
-    return launch_book_overlapped(k_append_book, s, m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)nullptr,
-                                  (const uint8_t*)nullptr, plan, flag, epoch, hs ? *hs : none);
-  k_append_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)k,
+  if (k == nullptr) {  // the rows follow in a launch of their own (ordinary order: it waits for everything before it)
+    if (n <= kWarpBookItems)   // one warp walks them in at most four rounds of dependent reads
+      return launch_book_overlapped(k_append_book<true>, s, 32, m, slots, n, call, dst_row, dst_pos, g, pool_layer,
+                                    (const uint8_t*)nullptr, (const uint8_t*)nullptr, plan, flag, epoch, hs ? *hs : none);
+    return launch_book_overlapped(k_append_book<false>, s, kBookThreads, m, slots, n, call, dst_row, dst_pos, g, pool_layer,
+                                  (const uint8_t*)nullptr, (const uint8_t*)nullptr, plan, flag, epoch, hs ? *hs : none);
+  }
+  k_append_book<false><<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, g, pool_layer, (const uint8_t*)k,
                                            (const uint8_t*)v, (int32_t*)nullptr, (int32_t*)nullptr, 0, none);
   return cudaGetLastError();
 }
@@ -568,7 +580,7 @@ cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n
                                     int32_t* dst_pos, int phase, const BcGeom& g, uint8_t* pool_layer, const void* k,
                                     const void* v, cudaStream_t s) {
   if (k == nullptr)
-    return launch_book_overlapped(k_compress_book, s, m, slots, n, call, dst_row, dst_pos, phase, g, pool_layer,
+    return launch_book_overlapped(k_compress_book, s, kBookThreads, m, slots, n, call, dst_row, dst_pos, phase, g, pool_layer,
                                   (const uint8_t*)nullptr, (const uint8_t*)nullptr);
   k_compress_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, phase, g, pool_layer,
                                              (const uint8_t*)k, (const uint8_t*)v);

@@ -37,6 +37,29 @@ __device__ int block_exclusive_scan(int x, int* total) {
   return warp_sums[warp] + incl - x;
 }
 
+// The same over ONE warp, without shared memory (the one-warp form of the append bookkeeping).
+__device__ __forceinline__ int warp_exclusive_scan(int x, int* total) {
+  const int lane = threadIdx.x & 31;
+  int incl = x;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    int y = __shfl_up_sync(0xffffffffu, incl, d);
+    if (lane >= d) incl += y;
+  }
+  *total = __shfl_sync(0xffffffffu, incl, 31);
+  return incl - x;
+}
+template <bool WARP>
+__device__ __forceinline__ int group_exclusive_scan(int x, int* total) {
+  if constexpr (WARP) return warp_exclusive_scan(x, total);
+  else return block_exclusive_scan(x, total);
+}
+template <bool WARP>
+__device__ __forceinline__ void group_sync() {
+  if constexpr (WARP) __syncwarp();
+  else __syncthreads();
+}
+
 // ---- BC_FLAG_DEBUG_BOUNDS -------------------------------------------------------------------------
 // Records a failed check (the offending value in the record's slot field) unless an error is latched
 // already.  The caller skips or redirects the access; nothing traps.
@@ -52,6 +75,7 @@ __device__ __forceinline__ bool debug_page_ok(const BcMeta& m, int page) {
 // A batch must not name a slot twice.  With the flag set every bookkeeping kernel (one thread block)
 // first marks, per slot, the lowest batch index that names it in this call; an item that is not that
 // one is refused with BC_ERR_DEBUG_CHECK, so the first occurrence goes through alone.
+template <bool WARP = false>
 __device__ void dup_prepass(const BcMeta& m, const int32_t* __restrict__ slots, int n, int64_t call) {
   if (!m.debug) return;
   for (int i = threadIdx.x; i < n; i += blockDim.x) {
@@ -59,7 +83,7 @@ __device__ void dup_prepass(const BcMeta& m, const int32_t* __restrict__ slots, 
     if (slot >= 0 && slot < m.max_seqs)
       atomicMax(m.dup_mark + slot, ((unsigned long long)call << 32) | (0xffffffffu - (unsigned)i));
   }
-  __syncthreads();
+  group_sync<WARP>();
 }
 __device__ __forceinline__ bool is_dup(const BcMeta& m, int slot, int i, int64_t call) {
   return m.debug && m.dup_mark[slot] != (((unsigned long long)call << 32) | (0xffffffffu - (unsigned)i));
@@ -94,14 +118,19 @@ struct ErrLatch {
 // With `plan` non-NULL the block also leaves the decode-attention kernel's plan for this batch, as the
 // lengths stand after the append (see BcPlan in bc_common.cuh): one coalesced read there instead of
 // slots -> lengths -> prefix sum.
+// WARP: the block is one warp; the same steps with shuffles and warp barriers and no shared memory.
+template <bool WARP = false>
 __device__ void append_book_block(const BcMeta& m, const int32_t* __restrict__ slots, int n, int64_t call, int32_t* dst_row,
                                   int32_t* dst_pos, int32_t* plan = nullptr, int tile_shift = 0) {
-  __shared__ int sh_first;
-  ErrLatch latch; latch.init(&sh_first);
-  dup_prepass(m, slots, n, call);
+  ErrLatch latch;
+  if constexpr (!WARP) {
+    __shared__ int sh_first;
+    latch.init(&sh_first);
+  }
+  dup_prepass<WARP>(m, slots, n, call);
   const int top0 = *m.free_top;
   const int ps = m.page_size;
-  __syncthreads();
+  group_sync<WARP>();
   int base = 0, used = 0, my_code = 0, my_item = -1, my_slot = 0;
   for (int chunk = 0; chunk < n; chunk += blockDim.x) {
     const int i = chunk + threadIdx.x;
@@ -125,7 +154,7 @@ __device__ void append_book_block(const BcMeta& m, const int32_t* __restrict__ s
       }
     }
     int total;
-    const int off = base + block_exclusive_scan(need, &total);
+    const int off = base + group_exclusive_scan<WARP>(need, &total);
     base += total;
     int row_out = -1;
     if (valid) {
@@ -140,16 +169,31 @@ __device__ void append_book_block(const BcMeta& m, const int32_t* __restrict__ s
       } else code = BC_ERR_NO_PAGES;
     }
     if (i < n) { dst_row[i] = row_out; dst_pos[i] = w; }
-    if (code && my_code == 0) { my_code = code; my_item = i; my_slot = slot; latch.note(i); }
+    if (code && my_code == 0) {
+      my_code = code; my_item = i; my_slot = slot;
+      if constexpr (!WARP) latch.note(i);
+    }
   }
   used = __reduce_max_sync(0xffffffffu, used);
-  __shared__ int sh_used;
-  if (threadIdx.x == 0) sh_used = 0;
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) atomicMax(&sh_used, used);
-  latch.commit(m, my_item, my_code, my_slot, call);
-  __syncthreads();
-  if (threadIdx.x == 0) *m.free_top = top0 - sh_used;
+  if constexpr (WARP) {
+    // the failing item with the lowest batch index reports, if no earlier call has latched an error
+    const int first = __reduce_min_sync(0xffffffffu, my_code ? my_item : 0x7fffffff);
+    if (my_code != 0 && my_item == first && m.status[0] == 0) {
+      m.status[0] = my_code;
+      m.status[1] = my_slot;
+      *reinterpret_cast<int64_t*>(m.status + 2) = call;
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) *m.free_top = top0 - used;
+  } else {
+    __shared__ int sh_used;
+    if (threadIdx.x == 0) sh_used = 0;
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) atomicMax(&sh_used, used);
+    latch.commit(m, my_item, my_code, my_slot, call);
+    __syncthreads();
+    if (threadIdx.x == 0) *m.free_top = top0 - sh_used;
+  }
   if (plan != nullptr && n <= BC_MAX_ATTN_BATCH) {
     // every thread sees the block's own writes to the lengths after the barrier above
     const int T = 1 << tile_shift;
@@ -172,7 +216,7 @@ __device__ void append_book_block(const BcMeta& m, const int32_t* __restrict__ s
         if (tiles == 0) tiles = 1;   // an empty sequence still owns one (empty) tile
       }
       int total;
-      const int off = carry + block_exclusive_scan(tiles, &total);
+      const int off = carry + group_exclusive_scan<WARP>(tiles, &total);
       if (i < n) a[6 * BC_MAX_ATTN_BATCH + i] = off;
       carry += total;
     }

@@ -138,7 +138,6 @@ struct BcFusedAppend {
   const int32_t* plan;   // NULL, or the plan the step's bookkeeping kernel left (BC_PLAN_INTS ints)
   int32_t* flag;         // workspace word: "the bookkeeping of launch `epoch` is done"
   int32_t epoch;
-  int32_t do_book;       // 1: this launch runs the bookkeeping (the layer-0 call of the step)
   int64_t call;          // bookkeeping call index (error latch)
 };
 // Launches the pipelined decode-attention kernel (the split combine is part of it); with `fused`

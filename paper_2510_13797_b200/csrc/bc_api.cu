@@ -95,6 +95,7 @@ bool config_ok(const bc_config* c, bc_status* why) {
   return true;
 }
 
+constexpr size_t kFusedBeaconRowBytes = 512u << 10;  // the same for the beacon rows of bc_compress (see there)
 constexpr size_t kFusedRowBytes = 32u << 10;  // rows of a batch that the bookkeeping block copies itself (a
                                                 // single block moves more than this slower than a second launch)
 
@@ -744,7 +745,11 @@ bc_status bc_compress(bc_cache* c, int32_t layer, const int32_t* slots, int32_t 
   int32_t* pos = work_ptr<int32_t>(c, c->wl.compress_pos);
   cudaStream_t s = (cudaStream_t)stream;
   const int L = c->cfg.layers;
-  const bool fused = layer == 0 && (size_t)n * c->geom.entry_bytes <= kFusedRowBytes;
+  // The beacon rows of layer 0 are written by the bookkeeping block itself when they are few (64 entries of 4 KB take
+  // it 3 us): that kernel may run under the last blocks of the attention kernel ahead, which reads neither the
+  // beacon slot being filled nor a page taken from the free stack, whereas a row-writing launch of its own waits
+  // for that kernel to end.
+  const bool fused = layer == 0 && (size_t)n * c->geom.entry_bytes <= kFusedBeaconRowBytes;
   if (layer == 0) {
     ++c->calls;
     // several layers: allocate now, evict on the last layer's call; a single layer: allocate and

@@ -579,12 +579,10 @@ cudaError_t bc_launch_host_steps_done(int32_t* done_word, int32_t seq, cudaStrea
 cudaError_t bc_launch_compress_book(const BcMeta& m, const int32_t* slots, int n, int64_t call, int32_t* dst_row,
                                     int32_t* dst_pos, int phase, const BcGeom& g, uint8_t* pool_layer, const void* k,
                                     const void* v, cudaStream_t s) {
-  if (k == nullptr)
-    return launch_book_overlapped(k_compress_book, s, kBookThreads, m, slots, n, call, dst_row, dst_pos, phase, g, pool_layer,
-                                  (const uint8_t*)nullptr, (const uint8_t*)nullptr);
-  k_compress_book<<<1, kBookThreads, 0, s>>>(m, slots, n, call, dst_row, dst_pos, phase, g, pool_layer,
-                                             (const uint8_t*)k, (const uint8_t*)v);
-  return cudaGetLastError();
+  // With rows as without: the beacon rows come from the caller's inputs, which no kernel of this library writes,
+  // and go to slots and pages that the kernel which may still be running ahead does not read.
+  return launch_book_overlapped(k_compress_book, s, kBookThreads, m, slots, n, call, dst_row, dst_pos, phase, g, pool_layer,
+                                (const uint8_t*)k, (const uint8_t*)v);
 }
 cudaError_t bc_launch_close(const BcMeta& m, const int32_t* slots, int n, int64_t call, cudaStream_t s) {
   k_close<<<1, kBookThreads, 0, s>>>(m, slots, n, call);

@@ -129,6 +129,31 @@ class Pair:
             ref[i] = seq.attend(layer, qq[i], sm_scale)
         return self._append_ok, out, ref
 
+    def fill(self, layer, slots, q, k, v, bq, bk, bv, sm_scale):
+        """bc_fill_step: the token's append, the token's and the beacon's attention, the compression; items the
+        bookkeeping refuses behave as in the three separate calls.  Returns (append results, compress results,
+        out, out_beacon, reference out, reference out_beacon)."""
+        n = len(slots)
+        out, out_b = self.gpu.new_out(n), self.gpu.new_out(n)
+        self.gpu.bc_fill_step(layer, self._i32(slots), q, k, v, bq, bk, bv, out, out_b, sm_scale)
+        if layer == 0:
+            self._append_ok = self.model.append(list(slots))
+        qq, kk, vv, bqq, bkk, bvv = (f64(x) for x in (q, k, v, bq, bk, bv))
+        ref, ref_b = np.zeros((n, self.Hq, self.D)), np.zeros((n, self.Hq, self.D))
+        for i, slot in enumerate(slots):
+            if self._append_ok[i] == OK:
+                self.seqs[slot].append(layer, kk[i], vv[i])
+        for i, slot in enumerate(slots):
+            seq = self.seqs.get(slot) or SeqCache(self.L, 1)
+            ref[i] = seq.attend(layer, qq[i], sm_scale)
+            ref_b[i] = seq.beacon_attend(layer, bqq[i], bkk[i], bvv[i], sm_scale)
+        if layer == 0:
+            self._compress_ok = self.model.compress(list(slots))
+        for i, slot in enumerate(slots):
+            if self._compress_ok[i] == OK:
+                self.seqs[slot].compress(layer, bkk[i], bvv[i])
+        return self._append_ok, self._compress_ok, out, out_b, ref, ref_b
+
     def attend(self, layer, slots, q, sm_scale, extra_k=None, extra_v=None, static=False):
         """static=True: through bc_decode_attn_static (split-K scratch inside the library image)."""
         out = self.gpu.new_out(len(slots))

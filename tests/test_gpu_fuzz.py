@@ -1,4 +1,4 @@
-"""Random programs of open / restore / append / compress / close against the oracle's paging model.
+"""Random programs of open / restore / append / decode step / fill step / compress / close against the oracle.
 
 Small pools and odd page sizes make the programs hit every refusal (no pages, window full, window
 not full, bad slot, capacity); after every call the lengths, page lists, free stack and the latched
@@ -9,7 +9,7 @@ import pytest
 import torch
 
 from paper_2510_13797_b200 import binding as B
-from tests.harness import Pair, randn_bf16
+from tests.harness import Pair, assert_close, randn_bf16
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -31,16 +31,19 @@ def test_random_programs(seed, ps, num_pages, max_pps, max_entries, checked):
     g = torch.Generator(device=DEV); g.manual_seed(seed)
     kv = lambda n: (randn_bf16(g, (n, Hkv, D), DEV), randn_bf16(g, (n, Hkv, D), DEV))
     for step in range(160):
-        op = rng.choice(["open", "restore", "append", "append", "append", "compress", "close"])
+        op = rng.choice(["open", "restore", "append", "append", "step", "step", "fill", "compress", "close"])
         n = int(rng.randint(1, S + 1))
         slots = [int(x) for x in rng.choice(S + 2, size=n, replace=False) - 1]      # -1 and S are invalid slots
-        if checked and rng.rand() < 0.3:                                             # name some slots again
+        if checked and op not in ("step", "fill") and rng.rand() < 0.3:              # name some slots again
             slots = [int(x) for x in rng.choice(slots, size=min(S, n + int(rng.randint(1, 4))))]
             n = len(slots)
         if op == "open":
             plens = [int(rng.randint(0, 3 * ps + 2)) for _ in slots]
             cs = None if rng.rand() < 0.3 else [int(rng.choice([1, 2, 3, 4, 7])) for _ in slots]
-            pair.open(slots, plens, cs)
+            res = pair.open(slots, plens, cs)
+            opened = [(s_, p_) for s_, p_, r_ in zip(slots, plens, res) if r_ == "OK"]
+            if opened and sum(p_ for _, p_ in opened):     # the prompts' K/V, so that the attention outputs below mean something
+                pair.prefill(0, [s_ for s_, _ in opened], [p_ for _, p_ in opened], *kv(sum(p_ for _, p_ in opened)))
         elif op == "restore":
             # mostly onto sequences that are still fresh, so that restores succeed too
             fresh = [s for s in range(S) if (st := pair.model.state(s)) and st["t"] == 0]
@@ -54,6 +57,23 @@ def test_random_programs(seed, ps, num_pages, max_pps, max_entries, checked):
             pair.restore(0, slots, gen_lens, tk[:sum(gen_lens)], tv[:sum(gen_lens)], bk[:nb], bv[:nb])
         elif op == "append":
             pair.append(0, slots, *kv(n))
+        elif op == "step":      # bc_decode_step: refused items (bad slot, full window, no page) still get their attention
+            q = randn_bf16(g, (n, Hkv * G, D), DEV)
+            _, out, ref = pair.step(0, slots, q, *kv(n), 0.2)
+            torch.cuda.synchronize()
+            assert_close(out, ref, f"program step {step}: bc_decode_step")
+        elif op == "fill":      # bc_fill_step, mostly on sequences one entry short of a full window
+            ready = [s for s in range(S) if (st := pair.model.state(s)) and st["c"] > 1 and st["window_len"] == st["c"] - 1]
+            if ready and rng.rand() < 0.7:
+                slots = ready[:n]
+                n = len(slots)
+            q, bq = randn_bf16(g, (n, Hkv * G, D), DEV), randn_bf16(g, (n, Hkv * G, D), DEV)
+            k, v = kv(n)
+            bk, bv = kv(n)
+            _, _, out, out_b, ref, ref_b = pair.fill(0, slots, q, k, v, bq, bk, bv, 0.2)
+            torch.cuda.synchronize()
+            assert_close(out, ref, f"program step {step}: bc_fill_step token rows")
+            assert_close(out_b, ref_b, f"program step {step}: bc_fill_step beacon rows")
         elif op == "compress":
             # favour the sequences whose window is full, so that compressions succeed too
             full = [s for s in range(S) if (st := pair.model.state(s)) and st["c"] > 1 and st["window_len"] == st["c"]]

@@ -50,10 +50,13 @@
  *    before the kernel enqueued just ahead of them on `stream` has ended, provided that kernel
  *    releases its dependents early; after any other kernel (the caller's own, a copy) they keep
  *    plain stream order.
- *      (1) The bookkeeping kernels of bc_append and bc_compress (when the call's K/V rows go out in
- *          a launch of their own).  They touch only the cache's metadata and `slots`, read nothing
- *          an attention kernel writes, and end only once the kernel they overtook has ended, so
- *          everything enqueued behind them is ordered after both.
+ *      (1) The bookkeeping kernels of bc_append (when the call's K/V rows go out in a launch of
+ *          their own or are taken by the attention kernel: bc_decode_step, bc_fill_step) and of
+ *          bc_compress.  They touch only the cache's metadata and `slots`, read nothing an attention
+ *          kernel writes, and end only once the kernel they overtook has ended, so everything enqueued
+ *          behind them is ordered after both.  The bookkeeping kernel of bc_compress also stores the
+ *          beacon rows of layer 0 when they are few (up to 512 KB): it reads beacon_k / beacon_v, and
+ *          writes slots and pages that no kernel still running ahead of it reads.
  *      (2) The attention kernels.  Before they wait for the kernel ahead they read `slots`, their
  *          inputs (q, the extra entry, beacon_q) and, of the cache, only what a kernel that has ENDED
  *          wrote: metadata and pool rows other than the newest entries of a beacon or window segment.
@@ -62,8 +65,9 @@
  *          reads that kernel's results only after a release/acquire handshake with it.
  *      (3) Kernels that release their dependents early: the attention kernels (once they have read
  *          the lengths they need) and the row-writing kernel of bc_append / bc_compress (at once).
- *    What this asks of the caller: `slots` and the input tensors of an attention call (q, extra_k,
- *    extra_v, beacon_q) must not be written by a kernel that releases its dependents early.  Kernels
+ *    What this asks of the caller: `slots`, the input tensors of an attention call (q, extra_k,
+ *    extra_v, beacon_q) and the beacon_k / beacon_v of bc_compress must not be written by a kernel
+ *    that releases its dependents early.  Kernels
  *    launched the ordinary way (any GEMM or element-wise kernel that produces q) never do; of this
  *    library's kernels only an attention kernel's OUTPUT could be in that position, so do not pass
  *    the output buffer of one attention call as the query buffer of the next call on the stream.

@@ -548,7 +548,7 @@ cudaError_t bc_launch_open(const BcMeta& m, const int32_t* slots, const int32_t*
 // enqueued before it -- which has read all the lengths it needs by the time it lets dependents go --
 // is still finishing its last blocks.  It waits for nothing of that kernel: it reads no output of it.
 // After any other predecessor the attribute changes nothing (no early trigger, ordinary order).
-constexpr int kWarpBookItems = 128;
+constexpr int kWarpBookItems = 256;
 template <typename... KArgs, typename... Args>
 cudaError_t launch_book_overlapped(void (*kernel)(KArgs...), cudaStream_t s, int threads, Args... args) {
   cudaLaunchConfig_t cfg = {};
@@ -565,7 +565,7 @@ cudaError_t bc_launch_append_book(const BcMeta& m, const int32_t* slots, int n, 
                                   cudaStream_t s, int32_t* plan, int32_t* flag, int32_t epoch, const BcHostSync* hs) {
   const BcHostSync none = {nullptr, 0, nullptr, 0, nullptr};
   if (k == nullptr) {  // the rows follow in a launch of their own (ordinary order: it waits for everything before it)
-    if (n <= kWarpBookItems)   // one warp walks them in at most four rounds of dependent reads
+    if (n <= kWarpBookItems)   // one warp walks them in at most eight rounds of dependent reads
       return launch_book_overlapped(k_append_book<true>, s, 32, m, slots, n, call, dst_row, dst_pos, g, pool_layer,
                                     (const uint8_t*)nullptr, (const uint8_t*)nullptr, plan, flag, epoch, hs ? *hs : none);
     return launch_book_overlapped(k_append_book<false>, s, kBookThreads, m, slots, n, call, dst_row, dst_pos, g, pool_layer,

@@ -170,14 +170,17 @@ def test_sweep_host_buffer_steps_full_size(host_route):
     check_lengths_and_conservation(drv)
 
 
-def test_sweep_c2_long_run_content_bit_exact():
+@pytest.mark.parametrize("fused", [False, True])
+def test_sweep_c2_long_run_content_bit_exact(fused):
     """400 steps back to back at c = 2 with pages of 2 entries: a window page is recycled at every
-    second step while the next step's bookkeeping may already run under the attention kernel's last
-    blocks.  Nothing may be overwritten early: the last outputs and the stored content of sampled
+    second step while the next step's bookkeeping already runs beside (one warp) or under the last
+    blocks of the attention kernel, and with fused=True (bc_decode_step, bc_fill_step: the calls the
+    benchmark times) the compression's kernel stores its beacon rows under that kernel as well.
+    Nothing may be overwritten early: the last outputs and the stored content of sampled
     sequences (every prompt entry, beacon and window token, bit for bit) must be the oracle's."""
     w = make_workload("sweep", c=2)
     t0 = (w.steps // 2 // 16) * 16
-    drv = DecodeDriver(w, DEV, beacon_ring=(t0 + 400) // 2 + 8)         # every stored beacon is unique
+    drv = DecodeDriver(w, DEV, fused=fused, beacon_ring=(t0 + 400) // 2 + 8)         # every stored beacon is unique
     drv.reset_to(t0)
     for _ in range(399):
         drv.step()

@@ -565,8 +565,16 @@ def report_ragged(args):
     def step(t, ep):
         """Decode step t (1-based) of the epoch's batch: append, attend, and the beacon step where due."""
         j = (t - 1) % ring
-        cache.bc_append(0, ep["sl"], ep["k"][j], ep["v"][j])
         grp = ep["groups"][t % PERIOD]
+        if not args.no_fused and not (grp is not None and paired):
+            # append and attention of the whole batch in one launch behind the bookkeeping kernel
+            cache.bc_decode_step(0, ep["sl"], ep["q"][j], ep["k"][j], ep["v"][j], out, w.sm_scale)
+            if grp is not None:
+                gsl, gq, gk, gv = grp[:4]
+                cache.bc_decode_attn(0, gsl, gq, outb, w.sm_scale, gk, gv)
+                cache.bc_compress(0, gsl, gk, gv)
+            return
+        cache.bc_append(0, ep["sl"], ep["k"][j], ep["v"][j])
         if grp is not None and paired:
             # the sequences whose window this token fills: token and beacon queries in one pass; the rest: plain
             gsl, gq, gk, gv, tq, rest = grp
@@ -650,6 +658,7 @@ def report_ragged(args):
         "gpu_launches": int(cache.bc_kernel_launches() - n_launch0 + replayed_launches), "host_seconds": host_s,
         "all_pages_returned": True, "graphs": len(graphs),
         "beacon_steps": "paired with the token's attention (one pass over the cache)" if paired else "second attention pass",
+        "regular_steps": "bc_append + bc_decode_attn" if (args.no_fused or paired) else "bc_decode_step",
         "note": "between two sequence finishes the batch is fixed and its call pattern repeats every 16 steps: "
                 "those steps run as replays of one CUDA graph per epoch, the rest as plain launches"}))
 

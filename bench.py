@@ -471,7 +471,7 @@ def report_cfg2(args):
     from paper_2510_13797_b200.workloads import make_workload
     torch.cuda.set_device(0)
     w = make_workload("cfg2")
-    r = make_runner(w, torch.device("cuda", 0), paired=not args.no_pair)
+    r = make_runner(w, torch.device("cuda", 0), paired=not args.no_pair, fused=not args.no_fused)
     K = max(16, (min(args.steps, 1024) // 16) * 16)
     t_mid = ((w.steps - K) // 2 // 16) * 16
     r.reset_to(t_mid - 32)
@@ -503,6 +503,7 @@ def report_cfg2(args):
         "us_per_bc_decode_attn": 1e3 * a_ms / a_n, "attn_kernel_gbs": a_bytes / (a_ms * 1e-3) / 1e9,
         "us_per_bc_append_bracketed": med(app), "us_per_bc_compress_bracketed": med(comp),
         "cache_bytes_mid": live, "uncompressed_bytes_mid": unc, "gpu_launches": int(launches),
+        "steps_through": "bc_append + bc_decode_attn (+ bc_decode_attn_pair, bc_compress)" if args.no_fused else "bc_decode_step, bc_fill_step",
         "note": "13 MB of KV per step stays in L2: the HBM roofline does not bound this configuration"}))
 
 

@@ -348,9 +348,11 @@ def test_ragged_batch_full_size():
     assert code == 0 and model.first_error is None
 
 
-def test_depth_config_first_windows():
+@pytest.mark.parametrize("fused", [False, True])
+def test_depth_config_first_windows(fused):
     """28 layers, batch 256, 12/2 heads, prompt 512, c = 8, page 8: three windows of per-layer calls
-    in dependency order; sampled (layer, sequence) outputs, and the shared bookkeeping."""
+    in dependency order; sampled (layer, sequence) outputs, and the shared bookkeeping.  fused: the calls
+    the benchmark issues (bc_decode_step per layer, bc_fill_step per layer at the step that fills the window)."""
     w = make_workload("depth")
     L, Bn, ps, Hkv, Hq, D, c, P = w.layers, w.batch, w.page_size, w.kv_heads, w.q_heads, w.head_dim, w.cs[0], w.prompt_lens[0]
     steps = 3 * c + 1
@@ -370,7 +372,7 @@ def test_depth_config_first_windows():
         cache.bc_prefill(l, slots, cu, Bn * P, pk, pv)
         if l in sample_layers:
             kept[l] = dict(pk=pk, pv=pv, step=stream.step_chunk(l, 0, steps), beacon=stream.beacon_chunk(l, 0, 4))
-    out = cache.new_out(Bn)
+    out, out_b = cache.new_out(Bn), cache.new_out(Bn)
 
     def content(l, s, t):
         d = kept[l]
@@ -383,16 +385,32 @@ def test_depth_config_first_windows():
         return np.concatenate(ks), np.concatenate(vs)
 
     for t in range(1, steps + 1):
+        fill_now = fused and t % c == 0
         for l in range(L):
             q, k, v = kept[l]["step"] if l in kept else stream.step_chunk(l, 0, steps)
-            cache.bc_append(l, slots, k[t - 1], v[t - 1])
-            cache.bc_decode_attn(l, slots, q[t - 1], out, w.sm_scale)
+            if fill_now:      # append, token and beacon rows in one pass, eviction: one call per layer
+                m = t // c
+                bq, bk, bv = kept[l]["beacon"] if l in kept else stream.beacon_chunk(l, 0, 4)
+                cache.bc_fill_step(l, slots, q[t - 1], k[t - 1], v[t - 1], bq[m], bk[m], bv[m], out, out_b, w.sm_scale)
+                if l in kept:
+                    s = sample_seqs[1]
+                    K, V = content(l, s, t)
+                    ref = attention(f64(bq[m, s]), np.concatenate([K, f64(bk[m, s])[None]]),
+                                    np.concatenate([V, f64(bv[m, s])[None]]), w.sm_scale)
+                    assert_close(out_b[s], ref, f"depth beacon rows, step {t} layer {l}")
+            elif fused:
+                cache.bc_decode_step(l, slots, q[t - 1], k[t - 1], v[t - 1], out, w.sm_scale)
+            else:
+                cache.bc_append(l, slots, k[t - 1], v[t - 1])
+                cache.bc_decode_attn(l, slots, q[t - 1], out, w.sm_scale)
             if l in kept:
                 for s in sample_seqs:
                     K, V = content(l, s, t)
                     assert_close(out[s], attention(f64(q[t - 1, s]), K, V, w.sm_scale), f"depth step {t} layer {l} seq {s}")
         model.append(slots_l)
-        if t % c == 0:
+        if fill_now:
+            model.compress(slots_l)
+        elif t % c == 0:
             m = t // c
             for l in range(L):
                 bq, bk, bv = kept[l]["beacon"] if l in kept else stream.beacon_chunk(l, 0, 4)

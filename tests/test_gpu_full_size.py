@@ -232,11 +232,14 @@ def test_sweep_c16_end_of_run_pages_bit_exact():
     drv.check_error()
 
 
-def test_cfg2_sampled_steps():
+@pytest.mark.parametrize("fused", [False, True])
+def test_cfg2_sampled_steps(fused):
     """Batch 32, 12/2 heads, prompt 256, 4096 steps, c = 16: keys pre-scaled by 1/sqrt(128), beacon
-    keys left N(0,1), softmax scale 1 (diffuse logits plus sharp beacon peaks)."""
+    keys left N(0,1), softmax scale 1 (diffuse logits plus sharp beacon peaks).  fused: through
+    bc_decode_step / bc_fill_step, all 4096 steps back to back (the small batch's bookkeeping is one warp
+    that runs beside the attention kernel of the step before)."""
     w = make_workload("cfg2")
-    drv = DecodeDriver(w, DEV, beacon_ring=w.steps // 16 + 1)           # 257 > 256 beacons: all unique
+    drv = DecodeDriver(w, DEV, fused=fused, beacon_ring=w.steps // 16 + 1)           # 257 > 256 beacons: all unique
     model = PagingModel(drv.num_pages, w.page_size, w.batch, drv.pages_per_seq, 0, 16)
     slots = list(range(w.batch))
     model.open(slots, w.prompt_lens)

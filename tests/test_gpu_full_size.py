@@ -261,7 +261,8 @@ def test_cfg2_sampled_steps(fused):
     drv.check_error()
 
 
-def test_ragged_batch_full_size():
+@pytest.mark.parametrize("fused", [False, True])
+def test_ragged_batch_full_size(fused):
     """Batch 128, 12/2 heads, page 16; per-sequence prompt U[64,1024], generation U[1024,32768], c from
     {4,8,16}.  Sequences finish at their own step and free their pages on the device; bookkeeping is
     compared with the paging model at every close and at sampled steps, outputs at sampled
@@ -304,11 +305,14 @@ def test_ragged_batch_full_size():
     for t in range(1, T_max + 1):
         j = (t - 1) % ring
         idx, sl = i64(live), i32(live)
-        cache.bc_append(0, sl, k[j].index_select(0, idx), v[j].index_select(0, idx))
-        model.append(live)
         out = cache.new_out(len(live))
         qs = q[j].index_select(0, idx)
-        cache.bc_decode_attn(0, sl, qs, out, w.sm_scale)
+        if fused:       # as bench.py --workload ragged issues the regular steps
+            cache.bc_decode_step(0, sl, qs, k[j].index_select(0, idx), v[j].index_select(0, idx), out, w.sm_scale)
+        else:
+            cache.bc_append(0, sl, k[j].index_select(0, idx), v[j].index_select(0, idx))
+            cache.bc_decode_attn(0, sl, qs, out, w.sm_scale)
+        model.append(live)
         if t in check_steps:
             for pos in sorted(set(int(x) for x in rng.randint(0, len(live), size=3))):
                 s = live[pos]

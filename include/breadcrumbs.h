@@ -391,11 +391,21 @@ BC_API bc_status bc_seq_close(bc_cache* cache, const int32_t* slots, int32_t n, 
  * bc_decode_step (the append and the attention of the step; same ordering rule over the layers),
  * copies out back.  n <= 512.  Asynchronous: out_host is valid, and the
  * three input buffers may be reused, once `stream` has passed the call.  The inputs are copied on a
- * stream the cache owns (created by the first such call, which therefore must not sit inside a
- * stream capture) into one of two staging buffers, so a call's inputs travel while the previous
- * call's kernels run: they are read from the moment of the call, not in the order of `stream` --
- * they must be complete in host memory when the call is made.  If the three buffers are one packed
- * block k | v | q (v_host == k_host + bytes(k), q_host == v_host + bytes(v)) a single copy moves them. */
+ * stream the cache owns (created by the first such call) into one of eight staging buffers used in
+ * turn, so a call's inputs travel while the previous calls' kernels run: they are read from the
+ * moment of the call, not in the order of `stream` -- they must be complete in host memory when the
+ * call is made.  If the three buffers are one packed block k | v | q (v_host == k_host + bytes(k),
+ * q_host == v_host + bytes(v)) a single copy moves them.  The host-buffer calls use streams of the
+ * library's own beside `stream` and must not be made inside a stream capture.
+ * On a single-layer cache created with BC_FLAG_HOST_PIPELINED the call puts nothing but its two
+ * kernels on `stream` (no event, no wait): the copy stream writes the step's number to a word in
+ * `workspace` behind the inputs (a stream memory operation) and the step's bookkeeping kernel polls
+ * that word (bounded: if the inputs do not arrive within about a second the step is reported as
+ * BC_ERR_TIMEOUT by bc_poll_error and its output is undefined) before it lets the attention kernel
+ * read them; the output copies of a step are released by a word the next step's bookkeeping kernel
+ * (or bc_host_outputs_ready, or bc_cache_destroy) stores once the step's kernels have ended.
+ * Consecutive steps then overlap as device-resident bc_decode_step calls do.  Issue such steps on
+ * one stream; a change of stream is handled, at the price of one small kernel on the old stream. */
 BC_API bc_status bc_decode_step_host(bc_cache* cache, int32_t layer, const int32_t* slots, int32_t n,
                               const void* q_host, const void* k_host, const void* v_host,
                               void* out_host, float sm_scale, void* stream);

@@ -10,7 +10,11 @@
 // All three are bound by memory latency at decode sizes (a few hundred KB per call; the logits of a step are
 // 19 MB); each replaces a chain of framework kernels (seven for the norm, three for the gate, and the residual
 // add) by one launch.  Arithmetic in fp32, 16-byte accesses, one block per row for the two row-wise ones.
+#include <cooperative_groups.h>
+
 #include "bc_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace {
 
@@ -106,23 +110,34 @@ __global__ void __launch_bounds__(256) k_swiglu(const uint4* __restrict__ gate_u
 }
 
 constexpr int kArgThreads = 512;
+constexpr int kArgCluster = 8;   // thread blocks per row: a cluster, reduced through distributed shared memory
 __device__ __forceinline__ void take(float& best, int& at, float v, int i) {
   if (v > best || (v == best && i < at)) { best = v; at = i; }
 }
+// One CLUSTER of kArgCluster blocks per row (19 MB of logits per decode step of the 1.5B model: 64 rows are too few
+// blocks to draw the memory bandwidth with one block each).  Every block scans its slice of the row with 16-byte
+// loads, reduces it to (maximum, lowest index), and leaves the pair in its shared memory; after a cluster barrier
+// the first block of the cluster folds the pairs of all blocks, read through distributed shared memory.
 __global__ void __launch_bounds__(kArgThreads) k_argmax_rows(const __nv_bfloat16* __restrict__ z, int vocab, long long* __restrict__ out) {
-  const __nv_bfloat16* row = z + (int64_t)blockIdx.x * vocab;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int part = (int)cluster.block_rank(), parts = (int)cluster.num_blocks();
+  const int64_t r = blockIdx.x / parts;
+  const __nv_bfloat16* row = z + r * vocab;
   float best = -INFINITY;
   int at = 0x7fffffff;
   const int chunks = vocab >> 3;   // the row starts on a 16-byte boundary when vocab is a multiple of 8 (checked by the host)
+  const int per = (chunks + parts - 1) / parts, c0 = part * per, c1 = min(chunks, c0 + per);
   const uint4* r4 = reinterpret_cast<const uint4*>(row);
-  for (int ch = threadIdx.x; ch < chunks; ch += kArgThreads) {
-    const uint4 a = r4[ch];
+  for (int ch = c0 + threadIdx.x; ch < c1; ch += kArgThreads) {
+    const uint4 a = __ldcs(r4 + ch);
     const int i = ch << 3;
     take(best, at, bf_lo(a.x), i); take(best, at, bf_hi(a.x), i + 1); take(best, at, bf_lo(a.y), i + 2); take(best, at, bf_hi(a.y), i + 3);
     take(best, at, bf_lo(a.z), i + 4); take(best, at, bf_hi(a.z), i + 5); take(best, at, bf_lo(a.w), i + 6); take(best, at, bf_hi(a.w), i + 7);
   }
   __shared__ float sh_v[kArgThreads / 32];
   __shared__ int sh_i[kArgThreads / 32];
+  __shared__ float blk_v;
+  __shared__ int blk_i;
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) {
     const float v = __shfl_xor_sync(0xffffffffu, best, d);
@@ -140,8 +155,14 @@ __global__ void __launch_bounds__(kArgThreads) k_argmax_rows(const __nv_bfloat16
       const int i = __shfl_xor_sync(0xffffffffu, at, d);
       take(best, at, v, i);
     }
-    if (threadIdx.x == 0) out[blockIdx.x] = at == 0x7fffffff ? 0 : at;   // a row of -inf / NaN: index 0
+    if (threadIdx.x == 0) { blk_v = best; blk_i = at; }
   }
+  cluster.sync();   // every block's pair is in its shared memory
+  if (part == 0 && threadIdx.x == 0) {
+    for (int b = 1; b < parts; ++b) take(best, at, *cluster.map_shared_rank(&blk_v, b), *cluster.map_shared_rank(&blk_i, b));
+    out[r] = at == 0x7fffffff ? 0 : at;   // a row of -inf / NaN: index 0
+  }
+  cluster.sync();   // no block leaves while its shared memory may still be read
 }
 
 }  // namespace
@@ -159,7 +180,12 @@ cudaError_t bc_launch_swiglu(const void* gate_up, int n, int m, void* out, cudaS
   return cudaGetLastError();
 }
 cudaError_t bc_launch_argmax(const void* logits, int n, int vocab, long long* out, cudaStream_t s) {
-  k_argmax_rows<<<n, kArgThreads, 0, s>>>((const __nv_bfloat16*)logits, vocab, out);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)n * kArgCluster); cfg.blockDim = dim3(kArgThreads); cfg.dynamicSmemBytes = 0; cfg.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = kArgCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, k_argmax_rows, (const __nv_bfloat16*)logits, vocab, out);
 }
 int bc_rmsnorm_max_hidden() { return kRowThreads * kMaxChunksPerThread * 8; }

@@ -89,9 +89,14 @@ def test_argmax_matches_oracle(n, V):
     z[1, 0] = 1000.0
     if V >= 1000:
         z[2, 17] = 999.0; z[2, 600] = 999.0; z[2, 999] = 999.0          # the lowest index of equal maxima
+    if V > 100000:
+        z[3, 150000] = 998.0; z[3, 100] = 998.0; z[3, 100000] = 998.0   # equal maxima in slices of different blocks of the row's cluster
+        z[4, :] = float("-inf")                                          # nothing exceeds the start value: index 0
     out = torch.full((n,), -1, dtype=torch.int64, device=DEV)
     B.bc_argmax(z, out)
     torch.cuda.synchronize()
     ref = argmax_rows(f64(z))
     assert np.array_equal(out.cpu().numpy(), ref)
     assert int(out[0]) == V - 1 and int(out[1]) == 0
+    if V > 100000:
+        assert int(out[3]) == 100 and int(out[4]) == 0

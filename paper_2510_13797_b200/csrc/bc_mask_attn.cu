@@ -350,11 +350,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
           umma(tS, dQ + off, dK + off, kk > 0);
         }
       };
-      // one lane polls, the warp takes its answer
+      // Every lane polls (one warp-wide instruction on one address) and a vote joins the answers.  Barrier
+      // polls and shuffles go through the same queue as the special-function instructions the rows keep it
+      // full of, so each costs this warp a couple of hundred cycles: a poll by one lane followed by a
+      // shuffle of its answer would be two of them per wait.
       auto wait_all = [&](uint32_t bar, uint32_t parity) {
-        int ok1 = 1;
-        if (lane == 0) ok1 = mbar_wait_or_fail<SHORTW>(bar, parity, s_fail, a.wait_limit) ? 1 : 0;
-        return __shfl_sync(0xffffffffu, ok1, 0) != 0;
+        const bool ok1 = mbar_wait_or_fail<SHORTW>(bar, parity, s_fail, a.wait_limit);
+        return __all_sync(0xffffffffu, ok1);
       };
       const uint32_t q_bytes = (uint32_t)(box_rows * kD * 2);
       TileDesc td = a.tiles[item / Hkv];

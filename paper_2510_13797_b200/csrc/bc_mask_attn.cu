@@ -263,7 +263,9 @@ __device__ __forceinline__ bool mbar_wait_or_fail(uint32_t bar, uint32_t parity,
 // first product into O waits until the rows have read the finished O.
 //
 // Barriers (single-phase mbarriers; t counts key tiles, e work items, parity = count & 1):
-//   bar_k: a K tile (with Q, at the start of an item) has landed      bar_v: a V tile has landed
+//   bar_k: the block's first Q and K have landed
+//   bar_in: V of tile t and K of tile t + 1 (with Q, at the start of an item) have landed: two arrivals per
+//           tile, the two requests, or a plain arrival in place of the K request after the block's last tile
 //   bar_s: completion t = S of tile t is ready (and every earlier product has finished)
 //   bar_p: the 128 row threads have stored P of tile t                bar_o: P V of a tile has completed
 //   bar_f: completion e = O of item e is final                       bar_e: the rows have read O of item e
@@ -276,13 +278,13 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail_word;
   volatile int* s_fail = &s_fail_word;
-  const uint32_t bar_k = smem_addr(&s_bars[0]), bar_v = bar_k + 8, bar_s = bar_k + 16, bar_p = bar_k + 24, bar_o = bar_k + 32,
+  const uint32_t bar_k = smem_addr(&s_bars[0]), bar_in = bar_k + 8, bar_s = bar_k + 16, bar_p = bar_k + 24, bar_o = bar_k + 32,
                  bar_f = bar_k + 40, bar_e = bar_k + 48, bar_d = bar_k + 56;   // bar_d: drain of the products on the give-up path
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = a.G, Hq = a.Hq, Hkv = a.Hkv, c = a.c;
 
   if (tid == 0) {
-    const uint32_t counts[8] = {1, 1, 1, (uint32_t)kRowThreads, 1, 1, (uint32_t)kRowThreads, 1};
+    const uint32_t counts[8] = {1, 2, 1, (uint32_t)kRowThreads, 1, 1, (uint32_t)kRowThreads, 1};   // bar_in: two arrivals per tile
     for (int i = 0; i < 8; ++i) asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar_k + i * 8), "r"(counts[i]) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     *s_fail = 0;
@@ -319,28 +321,28 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
     // are warp-uniform; one elected lane issues the copies and the products.
     int item = item_of(0);
     if (item >= 0) {
-      auto issue_q = [&](const TileDesc& td, int kvh) {
+      auto issue_q = [&](const TileDesc& td, int kvh, uint32_t bar) {
         // rows of Q beyond the tile's tokens belong to the next sequence or are zero-filled: they are never
         // visible (their outputs are not written and they contribute to no other row)
         const CUtensorMap* qm = td.kind == 0 ? &maps.q_tok : &maps.q_bea;
         const int qrow = (td.kind == 0 ? td.tok_row : td.bea_row) + td.first;
-        tma_3d(sQ, qm, 0, kvh * G, qrow, bar_k);
-        tma_3d(sQ + kTile * 128, qm, 64, kvh * G, qrow, bar_k);
+        tma_3d(sQ, qm, 0, kvh * G, qrow, bar);
+        tma_3d(sQ + kTile * 128, qm, 64, kvh * G, qrow, bar);
       };
-      auto issue_k = [&](const TileDesc& td, const TilePlan& pl, int kvh, int n) {
+      auto issue_k = [&](const TileDesc& td, const TilePlan& pl, int kvh, int n, uint32_t bar) {
         const int kind = plan_kind(pl, n), k0 = plan_k0(pl, n, kind);
         const CUtensorMap* km = kind == 0 ? &maps.k_prompt : (kind == 1 ? &maps.k_bea : &maps.k_tok);
         const int row = (kind == 0 ? td.prompt_row : (kind == 1 ? td.bea_row : td.tok_row)) + k0;
-        tma_3d(sK, km, 0, kvh, row, bar_k);
-        tma_3d(sK + kTile * 128, km, 64, kvh, row, bar_k);
+        tma_3d(sK, km, 0, kvh, row, bar);
+        tma_3d(sK + kTile * 128, km, 64, kvh, row, bar);
       };
       auto issue_v = [&](const TileDesc& td, const TilePlan& pl, int kvh, int n) {
         const int kind = plan_kind(pl, n), k0 = plan_k0(pl, n, kind);
         const CUtensorMap* vm = kind == 0 ? &maps.v_prompt : (kind == 1 ? &maps.v_bea : &maps.v_tok);
         const int row = (kind == 0 ? td.prompt_row : (kind == 1 ? td.bea_row : td.tok_row)) + k0;
-        mbar_expect_tx(bar_v, (uint32_t)kOperandBytes);
-        tma_3d(sV, vm, 0, kvh, row, bar_v);
-        tma_3d(sV + kTile * 128, vm, 64, kvh, row, bar_v);
+        mbar_expect_tx(bar_in, (uint32_t)kOperandBytes);
+        tma_3d(sV, vm, 0, kvh, row, bar_in);
+        tma_3d(sV + kTile * 128, vm, 64, kvh, row, bar_in);
       };
       const uint64_t dQ = umma_desc(sQ), dK = umma_desc(sK), dV = umma_desc_nmajor(sV);
       auto qk = [&]() {   // descriptor start addresses advance in 16-byte units
@@ -363,18 +365,20 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
       int kvh = item % Hkv;
       TilePlan pl = make_plan(td, c);
       if (elect_one()) {
-        mbar_expect_tx(bar_k, q_bytes + (uint32_t)kOperandBytes);
-        issue_q(td, kvh);
-        issue_k(td, pl, kvh, 0);
+        mbar_expect_tx(bar_k, q_bytes + (uint32_t)kOperandBytes);   // the first Q and K: a barrier of their own
+        issue_q(td, kvh, bar_k);
+        issue_k(td, pl, kvh, 0, bar_k);
         issue_v(td, pl, kvh, 0);
       }
       __syncwarp();
-      // copies requested / copies seen to land (for the give-up path: what is still in flight)
-      uint32_t k_req = 1, k_got = 0, v_req = 1, v_got = 0;
-      bool products_issued = false;
-      uint32_t ph_k = 0, ph_v = 0, ph_o = 0, t = 0, e = 0;
-      bool ok = wait_all(bar_k, ph_k);
-      if (ok) { ph_k ^= 1; ++k_got; }
+      // for the give-up path (what is still in flight): the first copies not seen to land; the number of
+      // bar_in completions begun (tile t is completion t: V_t, then K_{t+1} or a plain arrival); whether the
+      // last one begun still lacks its second arrival
+      bool first_out = true, in_open = true, products_issued = false;
+      uint32_t n_in = 1;
+      uint32_t ph_o = 0, t = 0, e = 0;
+      bool ok = wait_all(bar_k, 0);
+      if (ok) first_out = false;
       if (ok) {
         products_issued = true;
         tc_fence_after();
@@ -392,21 +396,24 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
           if (!ok) break;
           const bool last = n + 1 == pl.N;
           const bool more = !last || nitem >= 0;                               // another tile follows, here or in the next item
-          if (more && elect_one()) {
-            if (!last) {
-              mbar_expect_tx(bar_k, (uint32_t)kOperandBytes);
-              issue_k(td, pl, kvh, n + 1);
+          // the second arrival of this tile's bar_in completion (the first was the request of V_t): the
+          // request of the next K, or a plain arrival where no tile follows
+          if (elect_one()) {
+            if (!more) mbar_arrive_cta(bar_in);
+            else if (!last) {
+              mbar_expect_tx(bar_in, (uint32_t)kOperandBytes);
+              issue_k(td, pl, kvh, n + 1, bar_in);
             } else {                                                           // ... and so is the Q buffer
-              mbar_expect_tx(bar_k, q_bytes + (uint32_t)kOperandBytes);
-              issue_q(ntd, nkvh);
-              issue_k(ntd, npl, nkvh, 0);
+              mbar_expect_tx(bar_in, q_bytes + (uint32_t)kOperandBytes);
+              issue_q(ntd, nkvh, bar_in);
+              issue_k(ntd, npl, nkvh, 0, bar_in);
             }
           }
-          if (more) ++k_req;
           __syncwarp();
-          // everything the products below need besides P is waited for while the rows are busy
-          ok = wait_all(bar_v, ph_v);
-          if (ok) { ph_v ^= 1; ++v_got; }
+          in_open = false;
+          // everything the products below need besides P is waited for while the rows are busy: V_t and
+          // K_{t+1} (with its Q) have landed -- one barrier, one wait
+          ok = wait_all(bar_in, t & 1u);
           if (ok) {
             // A key tile that reaches past its segment has loaded rows that are not this sequence's (the
             // next sequence's, or zeros past the end of the array).  Their scores are overwritten with -inf
@@ -423,7 +430,6 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
             }
           }
           if (ok && n == 0 && e > 0) ok = wait_all(bar_e, (e - 1) & 1u);       // the rows have read the last O
-          if (ok && more) { ok = wait_all(bar_k, ph_k); if (ok) { ph_k ^= 1; ++k_got; } }   // the next K (and Q) has landed
           ok = ok && wait_all(bar_p, t & 1u);
           if (!ok) break;
           tc_fence_after();
@@ -446,7 +452,7 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
             ph_o ^= 1;
             if (!ok) break;
             if (elect_one()) { if (!last) issue_v(td, pl, kvh, n + 1); else issue_v(ntd, npl, nkvh, 0); }
-            ++v_req;
+            in_open = true; ++n_in;
             __syncwarp();
           }
         }
@@ -461,8 +467,9 @@ __global__ void __launch_bounds__(kThreads, 2) k_mask_attn(const MaskArgs a, con
         __syncwarp();
         if (elect_one()) {   // the lane that issued the copies and the products
           int never = 0;
-          if (k_req > k_got) mbar_wait_or_fail<false>(bar_k, ph_k, &never, kWaitLimit);
-          if (v_req > v_got) mbar_wait_or_fail<false>(bar_v, ph_v, &never, kWaitLimit);
+          if (in_open) mbar_arrive_cta(bar_in);   // a completion with only its first arrival gets its second one
+          if (first_out) mbar_wait_or_fail<false>(bar_k, 0, &never, kWaitLimit);
+          mbar_wait_or_fail<false>(bar_in, (n_in - 1) & 1u, &never, kWaitLimit);
           if (products_issued) {
             umma_commit(bar_d);
             mbar_wait_or_fail<false>(bar_d, 0, &never, kWaitLimit);

@@ -57,8 +57,8 @@ def entries_beacon_query(P, t, c):
 # case of each ratio (--profile-case C: same bytes per launch and page size as mid-generation), for
 # the library version named here; see profiles/.  Slightly below 1: part of the stream stays in L2
 # from the previous step.  A different library version invalidates the figures (traffic: null).
-TRAFFIC_FOR_VERSION = 230
-TRAFFIC_OVER_ALGORITHMIC = {2: 0.997, 4: 0.981, 8: 0.962, 16: 0.945, 32: 0.985}
+TRAFFIC_FOR_VERSION = 231
+TRAFFIC_OVER_ALGORITHMIC = {2: 0.997, 4: 0.983, 8: 0.962, 16: 0.947, 32: 0.982}
 
 
 def traffic_per_launch(c, algorithmic_bytes):

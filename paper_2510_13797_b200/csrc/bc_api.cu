@@ -355,7 +355,7 @@ namespace {
 bc_status flush_pending(bc_cache* c);   // defined with the host-buffer entry points below
 }
 
-int32_t bc_version(void) { return 230; }
+int32_t bc_version(void) { return 231; }
 
 const char* bc_status_string(bc_status s) {
   switch (s) {

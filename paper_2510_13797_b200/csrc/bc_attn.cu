@@ -329,8 +329,9 @@ __device__ __forceinline__ void combine_pieces(const float* part_o, const float*
 // PAIR: every sequence has two sets of query heads, the token's (rows 0..G-1 of a warp's 16-row
 // fragment) and its beacon's (rows 8..8+G-1), which share one pass over the cache: the step whose token
 // fills the window and the encoding of the beacon that follows it (Algorithm 1) read the same entries.
-// The beacon's rows also see the extra entry (the beacon's own K/V).  Needs G <= 8 and is compiled
-// on the 16-row path (G_LE_8 = false); results go to out (token) and out2 (beacon).  FUSED and PAIR
+// The beacon's rows also see the extra entry (the beacon's own K/V).  Needs G <= 8; with 2 G <= 8 both
+// sets of heads share the first 8 rows (token rows 0..G-1, beacon rows G..2G-1: the instantiation with
+// G_LE_8 = true), else it runs on the 16-row path; results go to out (token) and out2 (beacon).  FUSED and PAIR
 // together are the step that fills a window as one launch: the token's entry comes from the inputs as in
 // a regular fused step, and both sets of rows see it.
 // LAYERED: one launch for all layers of a call with layer = BC_ALL_LAYERS.  The grid is (blocks, layers):
@@ -339,7 +340,10 @@ __device__ __forceinline__ void combine_pieces(const float* part_o, const float*
 // blocks of one layer and the first of the next run side by side.
 template <int D, bool G_LE_8, bool FUSED, bool PAIR = false, bool SHORTW = false, bool LAYERED = false>
 __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams p_in) {
-  static_assert(!PAIR || !G_LE_8, "the paired form runs on the 16-row path");
+  // PAIR with G_LE_8: the packed paired form, for 2 G <= 8: the token's heads in rows 0..G-1 and the
+  // beacon's in rows G..2G-1 of the same 8-row half, so that a tile costs what it costs the plain kernel
+  // (one softmax per 16 keys instead of two).  PAIR without G_LE_8: token rows 0..G-1, beacon rows 8..8+G-1.
+  constexpr bool PACK = PAIR && G_LE_8;
   static_assert(!LAYERED || (!PAIR && !SHORTW), "the all-layers launch exists for the plain and the fused step");
   PipeParams p_layer;
   if constexpr (LAYERED) {
@@ -717,6 +721,14 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
 #pragma unroll
     for (int kk = 0; kk < KSTEPS; ++kk) {
       const int d0 = kk * 16 + qd * 2;
+      if (PACK) {
+        const __nv_bfloat16* qb2 = reinterpret_cast<const __nv_bfloat16*>(p.a.q2) + ((int64_t)i * Hq + kvh * G) * D;
+        const __nv_bfloat16* src = gq < G ? qb + gq * D : qb2 + (gq - G) * D;
+        qr[kk][0] = gq < 2 * G ? *reinterpret_cast<const uint32_t*>(src + d0) : 0u;
+        qr[kk][2] = gq < 2 * G ? *reinterpret_cast<const uint32_t*>(src + d0 + 8) : 0u;
+        qr[kk][1] = 0u; qr[kk][3] = 0u;
+        continue;
+      }
       qr[kk][0] = gq < G ? *reinterpret_cast<const uint32_t*>(qb + gq * D + d0) : 0u;
       qr[kk][2] = gq < G ? *reinterpret_cast<const uint32_t*>(qb + gq * D + d0 + 8) : 0u;
       if (G_LE_8) { qr[kk][1] = 0u; qr[kk][3] = 0u; }
@@ -777,7 +789,8 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
       d0 += __shfl_xor_sync(0xffffffffu, d0, 1); d0 += __shfl_xor_sync(0xffffffffu, d0, 2);
       if (!G_LE_8) { d1 += __shfl_xor_sync(0xffffffffu, d1, 1); d1 += __shfl_xor_sync(0xffffffffu, d1, 2); }
       // paired form: only the beacon's rows see the extra entry
-      const bool r0 = !PAIR && gq < G, r1 = PAIR ? gq < G : (!G_LE_8 && (gq + 8 < G));
+      const bool r0 = PACK ? (gq >= G && gq < 2 * G) : (!PAIR && gq < G);
+      const bool r1 = PACK ? false : (PAIR ? gq < G : (!G_LE_8 && (gq + 8 < G)));
       if (r0) { m0 = d0 * p.scale_log2; l0 = qd == 0 ? 1.f : 0.f; }
       if (r1) { m1 = d1 * p.scale_log2; l1 = qd == 0 ? 1.f : 0.f; }
 #pragma unroll
@@ -940,9 +953,11 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         for (int gi = 0; gi < p.n_groups; ++gi) {
-          if (grp == gi && gq < G) {
-            const int h = kvh * G + gq;
-            const float mm = half ? m1 : m0, ll = half ? l1 : l0;
+          const bool takes_part = PACK ? (gq >= half * G && gq < (half + 1) * G) : gq < G;
+          if (grp == gi && takes_part) {
+            const int h = kvh * G + (PACK ? gq - half * G : gq);
+            const bool second = half && !PACK;   // the row's state: rows 8..15 of the fragment, or (packed) rows 0..7
+            const float mm = second ? m1 : m0, ll = second ? l1 : l0;
             float sa = 0.f, sb = 1.f, mnew = mm, lnew = ll;
             if (gi > 0) {
               const float mb = merge_ml[h * 2], lb = merge_ml[h * 2 + 1];
@@ -956,8 +971,8 @@ __global__ void __launch_bounds__(kPipeThreads, 1) k_attn_pipe(const PipeParams 
             for (int nt = 0; nt < NT; ++nt) {
               const int d = nt * 8 + qd * 2;
               float2 cur = gi > 0 ? *reinterpret_cast<float2*>(orow + d) : make_float2(0.f, 0.f);
-              cur.x = cur.x * sa + (half ? o[nt][2] : o[nt][0]) * sb;
-              cur.y = cur.y * sa + (half ? o[nt][3] : o[nt][1]) * sb;
+              cur.x = cur.x * sa + (second ? o[nt][2] : o[nt][0]) * sb;
+              cur.y = cur.y * sa + (second ? o[nt][3] : o[nt][1]) * sb;
               *reinterpret_cast<float2*>(orow + d) = cur;
             }
             __syncwarp(__activemask());
@@ -1273,7 +1288,9 @@ cudaError_t bc_attn_setup(int* sm_count) {
   if (e != cudaSuccess) return e;
   e = cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  const cudaError_t r[22] = {opt_in_smem<128, false, true, true>(), opt_in_smem<64, false, true, true>(),
+  const cudaError_t r[26] = {opt_in_smem<128, true, true, true>(), opt_in_smem<64, true, true, true>(),
+                             opt_in_smem<128, true, false, true>(), opt_in_smem<64, true, false, true>(),
+                             opt_in_smem<128, false, true, true>(), opt_in_smem<64, false, true, true>(),
                              opt_in_smem<128, true, false, false, false, true>(), opt_in_smem<128, false, false, false, false, true>(),
                              opt_in_smem<64, true, false, false, false, true>(), opt_in_smem<64, false, false, false, false, true>(),
                              opt_in_smem<128, true, true, false, false, true>(), opt_in_smem<128, false, true, false, false, true>(),
@@ -1328,7 +1345,11 @@ cudaError_t bc_launch_attn(const BcMeta& m, const BcGeom& g, const BcAttnArgs& a
       else e = g8 ? launch_pipe<64, true, false, false, false, true>(p, s) : launch_pipe<64, false, false, false, false, true>(p, s);
     }
   } else if (a.q2 != nullptr) {   // the paired form (token and beacon queries in one pass); the caller has checked G <= 8
-    if (fused) e = g.head_dim == 128 ? launch_pipe<128, false, true, true>(p, s) : launch_pipe<64, false, true, true>(p, s);
+    const bool pack = 2 * p.G <= 8;   // both sets of heads fit the first 8 rows of a fragment
+    if (pack) {
+      if (fused) e = g.head_dim == 128 ? launch_pipe<128, true, true, true>(p, s) : launch_pipe<64, true, true, true>(p, s);
+      else e = g.head_dim == 128 ? launch_pipe<128, true, false, true>(p, s) : launch_pipe<64, true, false, true>(p, s);
+    } else if (fused) e = g.head_dim == 128 ? launch_pipe<128, false, true, true>(p, s) : launch_pipe<64, false, true, true>(p, s);
     else e = g.head_dim == 128 ? launch_pipe<128, false, false, true>(p, s) : launch_pipe<64, false, false, true>(p, s);
   } else if (shortw) {
     e = fused ? launch_pipe<128, true, true, false, true>(p, s) : launch_pipe<128, true, false, false, true>(p, s);
